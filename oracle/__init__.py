@@ -1,0 +1,175 @@
+"""ctypes front end of the CPU oracle (``hs2_oracle.c``).
+
+TEST INFRASTRUCTURE ONLY: imported by ``tests/``, by the smoke check and by the
+benchmark's CPU-baseline leg.  The CUDA library and its Python binding never import it.
+
+Tensors are numpy arrays: fp32 as ``float32``, bf16 as ``uint16`` bit patterns, packed
+``[B, L, H, D]``.  Results are fp64.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import math
+import os
+import subprocess
+from typing import Optional, Sequence, Tuple
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "hs2_oracle.c")
+_LIB = os.path.join(_HERE, "libhs2_oracle.so")
+
+AGG_MAX_PROB, AGG_MAX_LOGIT, AGG_SUM_PROB = 0, 1, 2
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle with gcc (OpenMP only spreads whole rows over threads)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + ".tmp%d" % os.getpid()
+        subprocess.check_call(["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c11",
+                               "-o", tmp, _SRC, "-lm"])
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+class _Problem(C.Structure):
+    _fields_ = [("batch", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32),
+                ("head_dim", C.c_int32), ("q_len", C.c_int32), ("kv_len", C.c_int32),
+                ("k_sel", C.c_int32), ("window", C.c_int32), ("scale", C.c_double),
+                ("dtype", C.c_int32), ("agg", C.c_int32),
+                ("q_start", C.c_void_p), ("kv_lens", C.c_void_p)]
+
+
+_lib = None
+
+
+def _get():
+    global _lib
+    if _lib is None:
+        _lib = C.CDLL(build())
+        _lib.hs2o_num_threads.restype = C.c_int
+    return _lib
+
+
+def num_threads() -> int:
+    return int(_get().hs2o_num_threads())
+
+
+def _ptr(a: Optional[np.ndarray]):
+    return None if a is None else a.ctypes.data_as(C.c_void_p)
+
+
+def _as_input(x) -> Tuple[np.ndarray, int]:
+    """numpy view of an input tensor: float32 -> dtype 0, uint16 (bf16 bits) -> dtype 1.
+
+    torch tensors (CPU) are accepted for convenience and viewed without a copy.
+    """
+    if not isinstance(x, np.ndarray):
+        import torch
+        x = x.detach().contiguous()
+        if x.dtype == torch.bfloat16:
+            x = x.view(torch.int16).numpy().view(np.uint16)
+        else:
+            x = x.numpy()
+    x = np.ascontiguousarray(x)
+    if x.dtype == np.float32:
+        return x, 0
+    if x.dtype == np.uint16:
+        return x, 1
+    raise TypeError("oracle inputs are float32 or bf16 bit patterns (uint16), got %s" % x.dtype)
+
+
+class Problem:
+    """Shapes and budgets of one call (mirrors the library's problem statement)."""
+
+    def __init__(self, q, k, k_sel: int, window: int, scale: Optional[float] = None,
+                 q_start: Optional[Sequence[int]] = None, kv_lens: Optional[Sequence[int]] = None,
+                 agg: int = AGG_MAX_PROB):
+        self.q, dq = _as_input(q)
+        self.k, dk = _as_input(k)
+        assert dq == dk and self.q.ndim == 4 and self.k.ndim == 4
+        B, Lq, Hq, D = self.q.shape
+        Bk, Lk, Hkv, Dk = self.k.shape
+        assert B == Bk and D == Dk and Hq % Hkv == 0
+        self.shape = (B, Lq, Lk, Hq, Hkv, D)
+        self.k_sel, self.window = int(k_sel), int(window)
+        self.q_start = None if q_start is None else np.ascontiguousarray(q_start, dtype=np.int32)
+        self.kv_lens = None if kv_lens is None else np.ascontiguousarray(kv_lens, dtype=np.int32)
+        self.c = _Problem(B, Hq, Hkv, D, Lq, Lk, self.k_sel, self.window,
+                          float(scale) if scale else 1.0 / math.sqrt(D), dq, agg,
+                          _ptr(self.q_start), _ptr(self.kv_lens))
+
+    def pos(self, b: int, i: int) -> int:
+        kvl = self.shape[2] if self.kv_lens is None else int(self.kv_lens[b])
+        q0 = kvl - self.shape[1] if self.q_start is None else int(self.q_start[b])
+        return q0 + i
+
+    def kvlen(self, b: int) -> int:
+        return self.shape[2] if self.kv_lens is None else int(self.kv_lens[b])
+
+
+def _rows(prob: Problem, rows):
+    if rows is None:
+        B, Lq = prob.shape[0], prob.shape[1]
+        rows = [(b, i) for b in range(B) for i in range(Lq)]
+    rb = np.ascontiguousarray([r[0] for r in rows], dtype=np.int32)
+    ri = np.ascontiguousarray([r[1] for r in rows], dtype=np.int32)
+    return rb, ri
+
+
+def full_attn_select(q, k, v, k_sel, window, rows=None, scale=None, q_start=None, kv_lens=None,
+                     agg=AGG_MAX_PROB, want_idx=True, want_scores=False):
+    """Full causal attention + selection for the listed (b, i) rows (all rows when None).
+
+    Returns ``(O [n,Hq,D], LSE [n,Hq], idx [n,Hkv,k] | None, scores [n,Hkv,Lk] | None)``;
+    scores are the aggregated selection scores (probabilities unless ``agg`` says logits),
+    ``-inf`` for keys the query cannot see.
+    """
+    prob = Problem(q, k, k_sel, window, scale, q_start, kv_lens, agg)
+    vv, _ = _as_input(v)
+    B, Lq, Lk, Hq, Hkv, D = prob.shape
+    rb, ri = _rows(prob, rows)
+    n = len(rb)
+    O = np.zeros((n, Hq, D), dtype=np.float64)
+    LSE = np.zeros((n, Hq), dtype=np.float64)
+    idx = np.full((n, Hkv, k_sel), -1, dtype=np.int32) if want_idx else None
+    sc = np.zeros((n, Hkv, Lk), dtype=np.float64) if want_scores else None
+    _get().hs2o_full_attn_select_rows(C.byref(prob.c), _ptr(prob.q), _ptr(prob.k), _ptr(vv), C.c_int(n),
+                                      _ptr(rb), _ptr(ri), _ptr(O), _ptr(LSE), _ptr(idx), _ptr(sc))
+    return O, LSE, idx, sc
+
+
+def select(scores, pos, kvlen, window: int, k_sel: int) -> np.ndarray:
+    """Top-k outside the window on given scores ``[n, Lk]`` (any float dtype) -> idx ``[n, k]``."""
+    sc = np.ascontiguousarray(scores, dtype=np.float64)
+    n, Lk = sc.shape
+    pos = np.ascontiguousarray(np.broadcast_to(np.asarray(pos, dtype=np.int32), (n,)))
+    kvlen = np.ascontiguousarray(np.broadcast_to(np.asarray(kvlen, dtype=np.int32), (n,)))
+    idx = np.full((n, k_sel), -1, dtype=np.int32)
+    _get().hs2o_select_rows(_ptr(sc), C.c_int(Lk), C.c_int(n), _ptr(pos), _ptr(kvlen),
+                            C.c_int(window), C.c_int(k_sel), _ptr(idx))
+    return idx
+
+
+def sparse_attn(q, k, v, idx, window, rows=None, sink=None, scale=None, q_start=None, kv_lens=None,
+                want_member=False):
+    """Sparse attention over (valid idx) U window for the listed rows.
+
+    ``idx`` is ``[n, Hkv, k]`` aligned with ``rows``.  Returns ``(O [n,Hq,D], LSE [n,Hq], member)``.
+    """
+    idx = np.ascontiguousarray(idx, dtype=np.int32)
+    k_sel = idx.shape[-1]
+    prob = Problem(q, k, k_sel, window, scale, q_start, kv_lens)
+    vv, _ = _as_input(v)
+    B, Lq, Lk, Hq, Hkv, D = prob.shape
+    rb, ri = _rows(prob, rows)
+    n = len(rb)
+    assert idx.shape == (n, Hkv, k_sel), (idx.shape, (n, Hkv, k_sel))
+    O = np.zeros((n, Hq, D), dtype=np.float64)
+    LSE = np.zeros((n, Hq), dtype=np.float64)
+    member = np.zeros((n, Hkv, Lk), dtype=np.uint8) if want_member else None
+    sk = None if sink is None else np.ascontiguousarray(sink, dtype=np.float64)
+    _get().hs2o_sparse_attn_rows(C.byref(prob.c), _ptr(prob.q), _ptr(prob.k), _ptr(vv), _ptr(idx), _ptr(sk),
+                                 C.c_int(n), _ptr(rb), _ptr(ri), _ptr(O), _ptr(LSE), _ptr(member))
+    return O, LSE, member
