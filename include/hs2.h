@@ -1,0 +1,149 @@
+/*
+ * hs2 — hybrid sparse attention hot path of HySparse2 on B200 (sm_100a).  C ABI.
+ *
+ * One hybrid block of the paper is a full-attention (FA) layer followed by sparse-attention
+ * (SA) layers that reuse the FA layer's KV cache and its token-level selection indices
+ * (Section 3.3, "Cross-Layer KV Reuse"; Figure 2, right).  The library covers the attention
+ * operators of that block:
+ *
+ *   hs2_full_attn_select     FA layer: causal softmax attention, which also emits, per query token
+ *                            and per KV head, the indices of the k highest-scoring tokens outside
+ *                            the forced local window (Sections 3.3 and 3.4).
+ *   hs2_topk_select          the same token-level top-k on a score tensor the caller provides.
+ *   hs2_sparse_attn_prefill  SA layer: attention over (reused indices) U (forced window of the most
+ *                            recent w tokens), K/V read from the FA layer's cache (Section 3.3).
+ *   hs2_sparse_attn_decode   the SA layer for one new token per sequence (split over the KV set).
+ *
+ * Conventions
+ *   - Every tensor pointer is a DEVICE pointer owned by the caller; `hs2_problem` itself is a
+ *     host struct read during the call.  `q_start` / `kv_lens` inside it are device arrays.
+ *   - Layouts: Q, O  [batch, q_len, n_q_heads, head_dim]; K, V [batch, kv_len, n_kv_heads, head_dim]
+ *     (token major; last dimension contiguous; strides in elements, 0 = packed);
+ *     idx [batch, n_kv_heads, q_len, k_sel] int32, packed; LSE [batch, n_q_heads, q_len] float, packed.
+ *   - Query head h reads KV head h / (n_q_heads / n_kv_heads).  No positional encoding is applied
+ *     (Section 4.1: full and sparse attention use NoPE).
+ *   - Query i of sequence b sits at absolute position pos = q_start[b] + i and sees keys
+ *     0 .. min(pos, kv_lens[b]-1).  The forced window is [pos-w+1, pos] (the token itself counts);
+ *     selection candidates are keys 0 .. pos-w.
+ *   - The library allocates no memory, keeps no state between calls, enqueues its work on the
+ *     given CUDA stream and returns without synchronising.  Scratch comes from the caller
+ *     (`ws`, at least hs2_workspace_bytes() bytes, 256-byte aligned).
+ *   - Argument errors are found on the host before anything is launched and reported through the
+ *     status; nothing throws, aborts or traps.  There is no CPU fallback: without a CUDA device
+ *     every compute entry point returns HS2_ERR_CUDA.
+ */
+#ifndef HS2_H_
+#define HS2_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    HS2_OK = 0,
+    HS2_ERR_INVALID_ARG = 1,         /* NULL where a pointer is required, non-positive size, bad head ratio ... */
+    HS2_ERR_UNSUPPORTED = 2,         /* valid problem outside what the kernels cover (e.g. head_dim > 256) */
+    HS2_ERR_WORKSPACE_TOO_SMALL = 3, /* ws_bytes < hs2_workspace_bytes() or ws not 256-byte aligned */
+    HS2_ERR_CUDA = 4                 /* a CUDA runtime call failed; see hs2_last_cuda_error() */
+} hs2_status;
+
+typedef enum { HS2_F32 = 0, HS2_BF16 = 1 } hs2_dtype;
+
+typedef enum {
+    HS2_OP_FULL_ATTN_SELECT = 0,
+    HS2_OP_TOPK_SELECT = 1,
+    HS2_OP_SPARSE_ATTN_PREFILL = 2,
+    HS2_OP_SPARSE_ATTN_DECODE = 3
+} hs2_op;
+
+typedef struct {
+    int32_t batch;
+    int32_t n_q_heads, n_kv_heads;   /* n_q_heads % n_kv_heads == 0 (GQA; MQA when n_kv_heads == 1) */
+    int32_t head_dim;                /* 1..256; K and V share it */
+    int32_t q_len, kv_len;           /* tensor extents in tokens */
+    int32_t k_sel;                   /* k: tokens selected outside the window (Section 4.1 uses 1024) */
+    int32_t window;                  /* w: forced most-recent tokens, the query's own included (paper: 128) */
+    float softmax_scale;             /* 0 => 1/sqrt(head_dim) */
+    hs2_dtype dtype;                 /* element type of Q, K, V, O */
+    const int32_t *q_start;          /* device [batch] or NULL => kv_lens[b] - q_len */
+    const int32_t *kv_lens;          /* device [batch] or NULL => kv_len */
+    int64_t q_stride[3];             /* elements: (batch, token, head); all 0 => packed */
+    int64_t kv_stride[3];            /* shared by K and V */
+    int64_t o_stride[3];
+} hs2_problem;
+
+/* Bytes of scratch `op` needs for this problem (a host-side computation; 0 is a valid answer).
+ * Returns 0 for an invalid problem. */
+size_t hs2_workspace_bytes(const hs2_problem *p, hs2_op op);
+
+/*
+ * FA layer of a hybrid block (Section 3.4: the full-attention layers "serve as indexers, using
+ * exact attention scores"; Section 3.3: top-k over individual tokens, outside the forced window).
+ *
+ *   O    out  attention output, same layout/dtype as Q
+ *   LSE  out  log-sum-exp of the scaled logits per (batch, head, query), natural log; required
+ *   idx  out  [batch, n_kv_heads, q_len, k_sel] or NULL to skip the selection.  Row (b,g,i) holds the
+ *             min(k_sel, pos-w+1) candidates with the highest group score
+ *                 a[j] = max over the query heads h of group g of (scale*<q_h,k_j> - LSE_h)
+ *             (the log of the largest softmax probability any head of the group gives key j),
+ *             ties to the lower key index, written in ascending key order and padded with -1.
+ *   scores_dbg out, NULL or float [batch, n_kv_heads, q_len, kv_len]: the a[j] the selection used
+ *             (-inf for keys the query cannot see).  Meant for small problems and tests.
+ *   ws   scratch for the score strips (unused when idx is NULL or scores_dbg is given).
+ *             hs2_workspace_bytes(p, HS2_OP_FULL_ATTN_SELECT) is the recommended size (all rows, at most
+ *             1 GiB); any 256-byte aligned buffer of at least 16*ceil(kv_len/4) bytes is accepted, a
+ *             smaller one only means that fewer query rows are scored per launch.
+ */
+hs2_status hs2_full_attn_select(const hs2_problem *p, const void *Q, const void *K, const void *V,
+                                void *O, float *LSE, int32_t *idx, float *scores_dbg,
+                                void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
+ * Token-level top-k outside the window (Section 3.3) on caller-provided scores.
+ *   scores in  float [batch, n_kv_heads, q_len, kv_len], packed.  Any finite floats or infinities;
+ *              +0 and -0 compare equal; NaN is a caller error.
+ *   idx    out as above.  The result is a pure function of the score bits: equal inputs give equal
+ *              indices (order: score descending, then key index ascending).
+ * head_dim, n_q_heads, dtype and the strides of `p` are ignored.
+ */
+hs2_status hs2_topk_select(const hs2_problem *p, const float *scores, int32_t *idx,
+                           void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
+ * SA layer, prefill (Section 3.3: the window "is always selected, followed by the highest-scoring
+ * tokens outside the window. Both selected sets are read from the full-attention KV cache").
+ *   Q     in  this SA layer's own queries; K, V: the FA layer's cache; idx: the FA layer's indices.
+ *   An idx entry is ignored when it is negative, greater than pos-w (inside the window or in the
+ *   future) or >= kv_lens[b]; the attended set is the union with the window and no entry can cause
+ *   an out-of-bounds read.  Repeating an index inside one row is a caller error (it is counted twice).
+ *   sink  in  NULL or float [n_q_heads]: per-head sink bias added to the softmax denominator only
+ *             (Section 4.1: sparse layers use learnable per-head sink biases).
+ *   O     out; LSE out, nullable.  A query whose attended set is empty gets O = 0, LSE = -inf.
+ */
+hs2_status hs2_sparse_attn_prefill(const hs2_problem *p, const void *Q, const void *K, const void *V,
+                                   const int32_t *idx, const float *sink, void *O, float *LSE,
+                                   void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
+ * SA layer, decode: q_len must be 1 (one new token per sequence, its K/V already in the cache).
+ * The attended set of each (sequence, KV head) is split over several warps; the partial results
+ * are merged on the device by the last split to finish (no kernel waits on another).
+ * Arguments as for the prefill call.
+ */
+hs2_status hs2_sparse_attn_decode(const hs2_problem *p, const void *Q, const void *K, const void *V,
+                                  const int32_t *idx, const float *sink, void *O, float *LSE,
+                                  void *ws, size_t ws_bytes, void *cuda_stream);
+
+/* Static, never-NULL description of a status. */
+const char *hs2_status_string(hs2_status s);
+
+/* The cudaError_t (as int) behind the calling thread's most recent HS2_ERR_CUDA, 0 if none. */
+int hs2_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* HS2_H_ */

@@ -1,0 +1,218 @@
+"""Thin ctypes binding of ``libhs2.so``: argument marshalling only.
+
+Every step of the path runs inside the CUDA library; this module turns torch tensors into
+device pointers, fills the ``hs2_problem`` struct, allocates outputs / scratch with torch when the
+caller did not pass them, and raises on a non-zero status.  There is no fallback: a missing
+library or a missing GPU is an error.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Optional
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libhs2.so")
+
+HS2_OK, HS2_ERR_INVALID_ARG, HS2_ERR_UNSUPPORTED, HS2_ERR_WORKSPACE_TOO_SMALL, HS2_ERR_CUDA = range(5)
+HS2_F32, HS2_BF16 = 0, 1
+HS2_OP_FULL_ATTN_SELECT, HS2_OP_TOPK_SELECT, HS2_OP_SPARSE_ATTN_PREFILL, HS2_OP_SPARSE_ATTN_DECODE = range(4)
+
+EXPORTS = ["hs2_workspace_bytes", "hs2_full_attn_select", "hs2_topk_select", "hs2_sparse_attn_prefill",
+           "hs2_sparse_attn_decode", "hs2_status_string", "hs2_last_cuda_error"]
+
+
+class HS2Error(RuntimeError):
+    def __init__(self, status: int, where: str, detail: str = ""):
+        self.status = status
+        super().__init__("%s: %s%s" % (where, hs2_status_string(status), detail))
+
+
+class _CProblem(C.Structure):
+    _fields_ = [("batch", C.c_int32), ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32),
+                ("head_dim", C.c_int32), ("q_len", C.c_int32), ("kv_len", C.c_int32),
+                ("k_sel", C.c_int32), ("window", C.c_int32), ("softmax_scale", C.c_float),
+                ("dtype", C.c_int), ("q_start", C.c_void_p), ("kv_lens", C.c_void_p),
+                ("q_stride", C.c_int64 * 3), ("kv_stride", C.c_int64 * 3), ("o_stride", C.c_int64 * 3)]
+
+
+_lib = None
+
+
+def library_path() -> str:
+    return _LIB_PATH
+
+
+def load_library():
+    """dlopen the in-tree library; raises if it has not been built."""
+    global _lib
+    if _lib is None:
+        if not os.path.exists(_LIB_PATH):
+            raise ImportError("%s is missing: build it with `python -m paper_2609_26368_b200.build`" % _LIB_PATH)
+        lib = C.CDLL(_LIB_PATH)
+        lib.hs2_workspace_bytes.restype = C.c_size_t
+        lib.hs2_workspace_bytes.argtypes = [C.POINTER(_CProblem), C.c_int]
+        lib.hs2_status_string.restype = C.c_char_p
+        lib.hs2_status_string.argtypes = [C.c_int]
+        lib.hs2_last_cuda_error.restype = C.c_int
+        vp, sz = C.c_void_p, C.c_size_t
+        pp = C.POINTER(_CProblem)
+        lib.hs2_full_attn_select.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        lib.hs2_topk_select.argtypes = [pp, vp, vp, vp, sz, vp]
+        lib.hs2_sparse_attn_prefill.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        lib.hs2_sparse_attn_decode.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        for f in ("hs2_full_attn_select", "hs2_topk_select", "hs2_sparse_attn_prefill", "hs2_sparse_attn_decode"):
+            getattr(lib, f).restype = C.c_int
+        _lib = lib
+    return _lib
+
+
+def hs2_status_string(status: int) -> str:
+    return load_library().hs2_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str):
+    if status != HS2_OK:
+        detail = ""
+        if status == HS2_ERR_CUDA:
+            detail = " (cudaError %d)" % load_library().hs2_last_cuda_error()
+        raise HS2Error(status, where, detail)
+
+
+def _dp(t: Optional[torch.Tensor]):
+    return None if t is None else C.c_void_p(t.data_ptr())
+
+
+def _stream(stream) -> C.c_void_p:
+    s = torch.cuda.current_stream() if stream is None else stream
+    return C.c_void_p(s.cuda_stream)
+
+
+def _strides(t: torch.Tensor):
+    assert t.stride(3) == 1, "last dimension must be contiguous"
+    return (C.c_int64 * 3)(t.stride(0), t.stride(1), t.stride(2))
+
+
+class Problem:
+    """Host-side description of one call; mirrors ``hs2_problem``."""
+
+    def __init__(self, batch, q_len, kv_len, n_q_heads, n_kv_heads, head_dim, k_sel, window, dtype=torch.bfloat16,
+                 softmax_scale: float = 0.0, q_start: Optional[torch.Tensor] = None,
+                 kv_lens: Optional[torch.Tensor] = None):
+        self.batch, self.q_len, self.kv_len = int(batch), int(q_len), int(kv_len)
+        self.n_q_heads, self.n_kv_heads, self.head_dim = int(n_q_heads), int(n_kv_heads), int(head_dim)
+        self.k_sel, self.window = int(k_sel), int(window)
+        self.dtype = dtype
+        self.softmax_scale = float(softmax_scale)
+        self.q_start, self.kv_lens = q_start, kv_lens
+        for t in (q_start, kv_lens):
+            assert t is None or (t.dtype == torch.int32 and t.is_cuda and t.is_contiguous())
+
+    @classmethod
+    def from_tensors(cls, q, k, k_sel, window, **kw):
+        B, Lq, Hq, D = q.shape
+        _, Lk, Hkv, _ = k.shape
+        return cls(B, Lq, Lk, Hq, Hkv, D, k_sel, window, dtype=q.dtype, **kw)
+
+    def c_struct(self, q=None, kv=None, o=None) -> _CProblem:
+        if self.dtype not in (torch.float32, torch.bfloat16):
+            raise TypeError("hs2 tensors are float32 or bfloat16")
+        c = _CProblem(self.batch, self.n_q_heads, self.n_kv_heads, self.head_dim, self.q_len, self.kv_len,
+                      self.k_sel, self.window, self.softmax_scale,
+                      HS2_F32 if self.dtype == torch.float32 else HS2_BF16,
+                      None if self.q_start is None else self.q_start.data_ptr(),
+                      None if self.kv_lens is None else self.kv_lens.data_ptr())
+        if q is not None:
+            c.q_stride = _strides(q)
+        if kv is not None:
+            c.kv_stride = _strides(kv)
+        if o is not None:
+            c.o_stride = _strides(o)
+        return c
+
+
+def hs2_workspace_bytes(prob: Problem, op: int) -> int:
+    c = prob.c_struct()
+    return int(load_library().hs2_workspace_bytes(C.byref(c), int(op)))
+
+
+def _workspace(prob: Problem, op: int, device, ws: Optional[torch.Tensor]):
+    if ws is not None:
+        return ws
+    n = hs2_workspace_bytes(prob, op)
+    return torch.empty(max(n, 256), dtype=torch.uint8, device=device)
+
+
+def _check_inputs(prob: Problem, q, k, v):
+    assert q.is_cuda and k.is_cuda and v.is_cuda, "hs2 runs on CUDA tensors only"
+    assert q.dtype == k.dtype == v.dtype == prob.dtype
+    assert tuple(q.shape) == (prob.batch, prob.q_len, prob.n_q_heads, prob.head_dim)
+    assert tuple(k.shape) == tuple(v.shape) == (prob.batch, prob.kv_len, prob.n_kv_heads, prob.head_dim)
+    assert k.stride() == v.stride(), "K and V share one stride triple"
+
+
+def hs2_full_attn_select(prob: Problem, q, k, v, *, out=None, lse=None, idx=None, want_idx=True,
+                         scores_dbg=None, want_scores=False, ws=None, stream=None):
+    """FA layer: returns ``(O, LSE, idx | None, scores_dbg | None)``."""
+    _check_inputs(prob, q, k, v)
+    dev = q.device
+    out = torch.empty_like(q) if out is None else out
+    lse = torch.empty(prob.batch, prob.n_q_heads, prob.q_len, dtype=torch.float32, device=dev) if lse is None else lse
+    if idx is None and want_idx:
+        idx = torch.empty(prob.batch, prob.n_kv_heads, prob.q_len, prob.k_sel, dtype=torch.int32, device=dev)
+    if scores_dbg is None and want_scores:
+        scores_dbg = torch.empty(prob.batch, prob.n_kv_heads, prob.q_len, prob.kv_len, dtype=torch.float32, device=dev)
+    if idx is not None and scores_dbg is None:
+        ws = _workspace(prob, HS2_OP_FULL_ATTN_SELECT, dev, ws)
+    c = prob.c_struct(q, k, out)
+    st = load_library().hs2_full_attn_select(C.byref(c), _dp(q), _dp(k), _dp(v), _dp(out), _dp(lse), _dp(idx),
+                                             _dp(scores_dbg), _dp(ws), 0 if ws is None else ws.numel(), _stream(stream))
+    _check(st, "hs2_full_attn_select")
+    return out, lse, idx, scores_dbg
+
+
+def hs2_topk_select(prob: Problem, scores, *, idx=None, stream=None):
+    """Token-level top-k outside the window on a float32 score tensor ``[B, Hkv, Lq, Lk]``."""
+    assert scores.is_cuda and scores.dtype == torch.float32 and scores.is_contiguous()
+    assert tuple(scores.shape) == (prob.batch, prob.n_kv_heads, prob.q_len, prob.kv_len)
+    if idx is None:
+        idx = torch.empty(prob.batch, prob.n_kv_heads, prob.q_len, prob.k_sel, dtype=torch.int32, device=scores.device)
+    c = prob.c_struct()
+    st = load_library().hs2_topk_select(C.byref(c), _dp(scores), _dp(idx), None, 0, _stream(stream))
+    _check(st, "hs2_topk_select")
+    return idx
+
+
+def _sparse(fn_name, op, prob, q, k, v, idx, sink, out, lse, want_lse, ws, stream):
+    _check_inputs(prob, q, k, v)
+    dev = q.device
+    if idx is not None:
+        assert idx.dtype == torch.int32 and idx.is_contiguous() and idx.is_cuda
+        assert tuple(idx.shape) == (prob.batch, prob.n_kv_heads, prob.q_len, prob.k_sel)
+    if sink is not None:
+        assert sink.dtype == torch.float32 and sink.is_cuda and sink.numel() == prob.n_q_heads
+    out = torch.empty_like(q) if out is None else out
+    if lse is None and want_lse:
+        lse = torch.empty(prob.batch, prob.n_q_heads, prob.q_len, dtype=torch.float32, device=dev)
+    ws = _workspace(prob, op, dev, ws)
+    c = prob.c_struct(q, k, out)
+    st = getattr(load_library(), fn_name)(C.byref(c), _dp(q), _dp(k), _dp(v), _dp(idx), _dp(sink), _dp(out), _dp(lse),
+                                          _dp(ws), ws.numel(), _stream(stream))
+    _check(st, fn_name)
+    return out, lse
+
+
+def hs2_sparse_attn_prefill(prob: Problem, q, k, v, idx, *, sink=None, out=None, lse=None, want_lse=False,
+                            ws=None, stream=None):
+    """SA layer, prefill: attention over (idx) U (forced window); returns ``(O, LSE | None)``."""
+    return _sparse("hs2_sparse_attn_prefill", HS2_OP_SPARSE_ATTN_PREFILL, prob, q, k, v, idx, sink, out, lse,
+                   want_lse, ws, stream)
+
+
+def hs2_sparse_attn_decode(prob: Problem, q, k, v, idx, *, sink=None, out=None, lse=None, want_lse=False,
+                           ws=None, stream=None):
+    """SA layer, decode (q_len == 1, split over the attended set); returns ``(O, LSE | None)``."""
+    return _sparse("hs2_sparse_attn_decode", HS2_OP_SPARSE_ATTN_DECODE, prob, q, k, v, idx, sink, out, lse,
+                   want_lse, ws, stream)

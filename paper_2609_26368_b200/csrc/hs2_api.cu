@@ -1,0 +1,222 @@
+// C ABI of the hs2 library: argument validation, default resolution, workspace carving, dispatch.
+#include <math.h>
+
+#include "hs2_common.cuh"
+
+namespace hs2 {
+namespace {
+
+thread_local int g_last_cuda_error = 0;
+
+hs2_status cuda_fail(cudaError_t e)
+{
+    g_last_cuda_error = (int)e;
+    return HS2_ERR_CUDA;
+}
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+constexpr size_t kStripCapBytes = (size_t)1 << 30;   // default bound on the score strips of one launch
+
+// Validate the host-visible part of a problem and resolve defaults.
+hs2_status resolve(const hs2_problem *hp, bool need_tensors, Params *out)
+{
+    if (!hp) return HS2_ERR_INVALID_ARG;
+    if (hp->batch <= 0 || hp->n_kv_heads <= 0 || hp->q_len <= 0 || hp->kv_len <= 0) return HS2_ERR_INVALID_ARG;
+    if (hp->k_sel < 0 || hp->window < 0) return HS2_ERR_INVALID_ARG;
+    if (hp->k_sel == 0 && hp->window == 0) return HS2_ERR_INVALID_ARG;   // every attended set would be empty
+    Params p{};
+    p.B = hp->batch; p.Hkv = hp->n_kv_heads; p.Lq = hp->q_len; p.Lk = hp->kv_len;
+    p.k = hp->k_sel; p.w = hp->window;
+    p.q_start = hp->q_start; p.kv_lens = hp->kv_lens;
+    p.Hq = hp->n_q_heads; p.D = hp->head_dim;
+    if (need_tensors) {
+        if (hp->n_q_heads <= 0 || hp->n_q_heads % hp->n_kv_heads != 0 || hp->head_dim <= 0) return HS2_ERR_INVALID_ARG;
+        if (hp->dtype != HS2_F32 && hp->dtype != HS2_BF16) return HS2_ERR_INVALID_ARG;
+        if (!(hp->softmax_scale >= 0.f) || isinf(hp->softmax_scale)) return HS2_ERR_INVALID_ARG;
+        if (hp->head_dim > 256) return HS2_ERR_UNSUPPORTED;
+        p.G = p.Hq / p.Hkv;
+        p.scale = hp->softmax_scale > 0.f ? hp->softmax_scale : 1.0f / sqrtf((float)p.D);
+        p.scale_log2 = p.scale * kLog2e;
+        auto strides = [](const int64_t s[3], int64_t L, int64_t H, int64_t D, int64_t &sb, int64_t &st, int64_t &sh) {
+            if (s[0] == 0 && s[1] == 0 && s[2] == 0) { sh = D; st = H * D; sb = L * H * D; return true; }
+            sb = s[0]; st = s[1]; sh = s[2];
+            return s[2] >= D && s[1] >= 0 && s[0] >= 0;
+        };
+        if (!strides(hp->q_stride, p.Lq, p.Hq, p.D, p.qs_b, p.qs_t, p.qs_h)) return HS2_ERR_INVALID_ARG;
+        if (!strides(hp->kv_stride, p.Lk, p.Hkv, p.D, p.ks_b, p.ks_t, p.ks_h)) return HS2_ERR_INVALID_ARG;
+        if (!strides(hp->o_stride, p.Lq, p.Hq, p.D, p.os_b, p.os_t, p.os_h)) return HS2_ERR_INVALID_ARG;
+    } else {
+        p.G = 1;
+    }
+    *out = p;
+    return HS2_OK;
+}
+
+int64_t select_rows(const Params &p) { return (int64_t)p.B * p.Hkv * p.Lq; }
+
+size_t strip_row_bytes(const Params &p) { return align_up((size_t)p.Lk * sizeof(float), 16); }
+
+size_t full_select_ws_bytes(const Params &p)
+{
+    const size_t row = strip_row_bytes(p);
+    size_t rows = (size_t)select_rows(p);
+    const size_t cap_rows = kStripCapBytes / row > 0 ? kStripCapBytes / row : 1;
+    if (rows > cap_rows) rows = cap_rows;
+    return align_up(rows * row, 256);
+}
+
+bool ws_ok(const void *ws, size_t ws_bytes, size_t need)
+{
+    if (need == 0) return true;
+    return ws != nullptr && ws_bytes >= need && reinterpret_cast<uintptr_t>(ws) % 256 == 0;
+}
+
+hs2_status check_device()
+{
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return cuda_fail(e);
+    return HS2_OK;
+}
+
+hs2_status sparse_common(const hs2_problem *hp, const void *Q, const void *K, const void *V, const int32_t *idx,
+                         void *O, Params *p)
+{
+    hs2_status s = resolve(hp, true, p);
+    if (s != HS2_OK) return s;
+    if (!Q || !K || !V || !O) return HS2_ERR_INVALID_ARG;
+    if (p->k > 0 && !idx) return HS2_ERR_INVALID_ARG;
+    return HS2_OK;
+}
+
+}  // namespace
+}  // namespace hs2
+
+using namespace hs2;
+
+extern "C" {
+
+size_t hs2_workspace_bytes(const hs2_problem *hp, hs2_op op)
+{
+    Params p;
+    switch (op) {
+        case HS2_OP_FULL_ATTN_SELECT:
+            if (resolve(hp, true, &p) != HS2_OK) return 0;
+            return p.k > 0 ? full_select_ws_bytes(p) : 0;
+        case HS2_OP_TOPK_SELECT:
+        case HS2_OP_SPARSE_ATTN_PREFILL:
+            return 0;
+        case HS2_OP_SPARSE_ATTN_DECODE:
+            if (resolve(hp, true, &p) != HS2_OK) return 0;
+            if (p.Lq != 1) return 0;
+            return sparse_mma_supported(p, hp->dtype) ? sparse_mma_decode_ws_bytes(p) : 0;
+    }
+    return 0;
+}
+
+hs2_status hs2_full_attn_select(const hs2_problem *hp, const void *Q, const void *K, const void *V, void *O,
+                                float *LSE, int32_t *idx, float *scores_dbg, void *ws, size_t ws_bytes,
+                                void *cuda_stream)
+{
+    Params p;
+    hs2_status s = resolve(hp, true, &p);
+    if (s != HS2_OK) return s;
+    if (!Q || !K || !V || !O || !LSE) return HS2_ERR_INVALID_ARG;
+    const bool want_sel = idx != nullptr && p.k > 0;
+    const size_t row_bytes = strip_row_bytes(p);
+    // any aligned buffer holding at least one strip row works; a smaller buffer only means more launches
+    if (want_sel && !scores_dbg && !ws_ok(ws, ws_bytes, row_bytes)) return HS2_ERR_WORKSPACE_TOO_SMALL;
+    if ((s = check_device()) != HS2_OK) return s;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    const hs2_dtype dt = hp->dtype;
+    const bool mma = full_mma_supported(p, dt);
+    cudaError_t e = mma ? launch_full_attn_mma(p, Q, K, V, O, LSE, st) : launch_full_attn_generic(p, dt, Q, K, V, O, LSE, st);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (!want_sel && !scores_dbg) return HS2_OK;
+
+    const int64_t rows = select_rows(p);
+    if (scores_dbg) {
+        // scores for every visible key go straight to the caller's tensor; the selection reads them from there
+        e = mma ? launch_scores_mma(p, Q, K, LSE, scores_dbg, p.Lk, 0, rows, true, st)
+                : launch_scores_generic(p, dt, Q, K, LSE, scores_dbg, p.Lk, 0, rows, true, st);
+        if (e != cudaSuccess) return cuda_fail(e);
+        if (want_sel && (e = launch_topk(p, scores_dbg, p.Lk, idx, 0, rows, st)) != cudaSuccess) return cuda_fail(e);
+        return HS2_OK;
+    }
+    // bounded strips: score a block of query rows into the workspace, select from it, move on
+    const int64_t stride = (int64_t)(row_bytes / sizeof(float));
+    int64_t block = (int64_t)(ws_bytes / row_bytes);
+    if (block > rows) block = rows;
+    float *strip = (float *)ws;
+    for (int64_t r0 = 0; r0 < rows; r0 += block) {
+        const int64_t n = rows - r0 < block ? rows - r0 : block;
+        e = mma ? launch_scores_mma(p, Q, K, LSE, strip, stride, r0, n, false, st)
+                : launch_scores_generic(p, dt, Q, K, LSE, strip, stride, r0, n, false, st);
+        if (e != cudaSuccess) return cuda_fail(e);
+        if ((e = launch_topk(p, strip, stride, idx, r0, n, st)) != cudaSuccess) return cuda_fail(e);
+    }
+    return HS2_OK;
+}
+
+hs2_status hs2_topk_select(const hs2_problem *hp, const float *scores, int32_t *idx, void *ws, size_t ws_bytes,
+                           void *cuda_stream)
+{
+    (void)ws; (void)ws_bytes;
+    Params p;
+    hs2_status s = resolve(hp, false, &p);
+    if (s != HS2_OK) return s;
+    if (p.k > 0 && (!scores || !idx)) return HS2_ERR_INVALID_ARG;
+    if ((s = check_device()) != HS2_OK) return s;
+    cudaError_t e = launch_topk(p, scores, p.Lk, idx, 0, select_rows(p), (cudaStream_t)cuda_stream);
+    return e == cudaSuccess ? HS2_OK : cuda_fail(e);
+}
+
+hs2_status hs2_sparse_attn_prefill(const hs2_problem *hp, const void *Q, const void *K, const void *V,
+                                   const int32_t *idx, const float *sink, void *O, float *LSE, void *ws,
+                                   size_t ws_bytes, void *cuda_stream)
+{
+    (void)ws; (void)ws_bytes;
+    Params p;
+    hs2_status s = sparse_common(hp, Q, K, V, idx, O, &p);
+    if (s != HS2_OK) return s;
+    if ((s = check_device()) != HS2_OK) return s;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    cudaError_t e = sparse_mma_supported(p, hp->dtype)
+                        ? launch_sparse_mma_prefill(p, Q, K, V, idx, sink, O, LSE, st)
+                        : launch_sparse_generic(p, hp->dtype, Q, K, V, idx, sink, O, LSE, st);
+    return e == cudaSuccess ? HS2_OK : cuda_fail(e);
+}
+
+hs2_status hs2_sparse_attn_decode(const hs2_problem *hp, const void *Q, const void *K, const void *V,
+                                  const int32_t *idx, const float *sink, void *O, float *LSE, void *ws,
+                                  size_t ws_bytes, void *cuda_stream)
+{
+    Params p;
+    hs2_status s = sparse_common(hp, Q, K, V, idx, O, &p);
+    if (s != HS2_OK) return s;
+    if (p.Lq != 1) return HS2_ERR_INVALID_ARG;
+    const bool mma = sparse_mma_supported(p, hp->dtype);
+    if (mma && !ws_ok(ws, ws_bytes, sparse_mma_decode_ws_bytes(p))) return HS2_ERR_WORKSPACE_TOO_SMALL;
+    if ((s = check_device()) != HS2_OK) return s;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    cudaError_t e = mma ? launch_sparse_mma_decode(p, Q, K, V, idx, sink, O, LSE, ws, ws_bytes, st)
+                        : launch_sparse_generic(p, hp->dtype, Q, K, V, idx, sink, O, LSE, st);
+    return e == cudaSuccess ? HS2_OK : cuda_fail(e);
+}
+
+const char *hs2_status_string(hs2_status s)
+{
+    switch (s) {
+        case HS2_OK: return "ok";
+        case HS2_ERR_INVALID_ARG: return "invalid argument";
+        case HS2_ERR_UNSUPPORTED: return "unsupported problem";
+        case HS2_ERR_WORKSPACE_TOO_SMALL: return "workspace too small or misaligned";
+        case HS2_ERR_CUDA: return "CUDA runtime error";
+    }
+    return "unknown status";
+}
+
+int hs2_last_cuda_error(void) { return g_last_cuda_error; }
+
+}  // extern "C"

@@ -1,0 +1,92 @@
+// Internal declarations shared by the hs2 translation units (not part of the C ABI).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "hs2.h"
+
+namespace hs2 {
+
+// A validated problem with every default resolved; passed to kernels by value.
+struct Params {
+    int B, Hq, Hkv, G, D;
+    int Lq, Lk;
+    int k, w;
+    float scale;        // softmax scale
+    float scale_log2;   // scale * log2(e): logits are kept in the base-2 domain inside the kernels
+    const int32_t *q_start;
+    const int32_t *kv_lens;
+    int64_t qs_b, qs_t, qs_h;   // element strides
+    int64_t ks_b, ks_t, ks_h;
+    int64_t os_b, os_t, os_h;
+};
+
+// per-sequence geometry, clamped so that no later index arithmetic can leave the tensors
+__device__ __forceinline__ int kvlen_of(const Params &p, int b)
+{
+    int n = p.kv_lens ? p.kv_lens[b] : p.Lk;
+    return n < 0 ? 0 : (n > p.Lk ? p.Lk : n);
+}
+__device__ __forceinline__ int pos_of(const Params &p, int b, int i)
+{
+    const int kvl = p.kv_lens ? p.kv_lens[b] : p.Lk;
+    const int q0 = p.q_start ? p.q_start[b] : kvl - p.Lq;
+    return q0 + i;
+}
+
+constexpr float kLog2e = 1.4426950408889634f;
+constexpr float kLn2 = 0.6931471805599453f;
+
+__device__ __forceinline__ float to_f32(float x) { return x; }
+__device__ __forceinline__ float to_f32(__nv_bfloat16 x) { return __bfloat162float(x); }
+__device__ __forceinline__ void from_f32(float &dst, float x) { dst = x; }
+__device__ __forceinline__ void from_f32(__nv_bfloat16 &dst, float x) { dst = __float2bfloat16_rn(x); }
+
+__device__ __forceinline__ float warp_max(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+__device__ __forceinline__ float warp_sum(float v)
+{
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
+    return v;
+}
+
+// ---- launchers (one per translation unit); each returns the cudaError_t of its launches ----
+
+// Generic SIMT kernels: fp32 arithmetic on fp32 or bf16 tensors, any head_dim <= 256, any group size.
+cudaError_t launch_full_attn_generic(const Params &p, hs2_dtype dt, const void *Q, const void *K, const void *V,
+                                     void *O, float *LSE, cudaStream_t st);
+// Group scores a[j] for rows [row0, row0+n_rows) of the flattened (b, g, i) index into `out`
+// (row stride out_stride).  all_visible: also write window keys and -inf beyond the causal limit.
+cudaError_t launch_scores_generic(const Params &p, hs2_dtype dt, const void *Q, const void *K, const float *LSE,
+                                  float *out, int64_t out_stride, int64_t row0, int64_t n_rows, bool all_visible,
+                                  cudaStream_t st);
+cudaError_t launch_sparse_generic(const Params &p, hs2_dtype dt, const void *Q, const void *K, const void *V,
+                                  const int32_t *idx, const float *sink, void *O, float *LSE, cudaStream_t st);
+
+// Radix select over score rows [row0, row0+n_rows); `scores` points at row row0.
+cudaError_t launch_topk(const Params &p, const float *scores, int64_t score_stride, int32_t *idx,
+                        int64_t row0, int64_t n_rows, cudaStream_t st);
+
+// Tensor-core bf16 kernels (head_dim 128, group <= 8).
+bool sparse_mma_supported(const Params &p, hs2_dtype dt);
+cudaError_t launch_sparse_mma_prefill(const Params &p, const void *Q, const void *K, const void *V, const int32_t *idx,
+                                      const float *sink, void *O, float *LSE, cudaStream_t st);
+size_t sparse_mma_decode_ws_bytes(const Params &p);
+cudaError_t launch_sparse_mma_decode(const Params &p, const void *Q, const void *K, const void *V, const int32_t *idx,
+                                     const float *sink, void *O, float *LSE, void *ws, size_t ws_bytes,
+                                     cudaStream_t st);
+
+bool full_mma_supported(const Params &p, hs2_dtype dt);
+cudaError_t launch_full_attn_mma(const Params &p, const void *Q, const void *K, const void *V, void *O, float *LSE,
+                                 cudaStream_t st);
+cudaError_t launch_scores_mma(const Params &p, const void *Q, const void *K, const float *LSE, float *out,
+                              int64_t out_stride, int64_t row0, int64_t n_rows, bool all_visible, cudaStream_t st);
+
+}  // namespace hs2

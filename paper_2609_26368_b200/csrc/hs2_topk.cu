@@ -1,0 +1,187 @@
+// Token-level top-k outside the forced window on a materialised score row (Section 3.3).
+//
+// One CTA per (batch, KV head, query) row.  The row's candidates are keys 0 .. pos-w.  An exact
+// radix select on order-preserving 32-bit keys (four 8-bit digits, most significant first) finds
+// the value of the take-th largest score and how many candidates equal to it are still needed;
+// one ordered compaction pass then writes the kept indices in ascending key order, taking equal
+// scores from the lowest index upwards.  The result depends only on the score bits.
+#include "hs2_common.cuh"
+
+namespace hs2 {
+namespace {
+
+constexpr int kThreads = 1024;
+constexpr int kWarps = kThreads / 32;
+constexpr int kItems = 4;                    // consecutive scores per thread per step
+constexpr int kChunk = kThreads * kItems;
+
+// float -> uint32 whose unsigned order is the float order; -0 is folded onto +0 first.
+__device__ __forceinline__ uint32_t order_key(float f)
+{
+    uint32_t u = __float_as_uint(f);
+    if (u == 0x80000000u) u = 0u;
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+template <bool VEC>
+__device__ __forceinline__ void load_keys(const float *row, int j0, int nc, uint32_t (&key)[kItems], bool (&ok)[kItems])
+{
+    if (VEC && j0 + kItems <= nc) {
+        const float4 v = *reinterpret_cast<const float4 *>(row + j0);
+        key[0] = order_key(v.x); key[1] = order_key(v.y); key[2] = order_key(v.z); key[3] = order_key(v.w);
+        ok[0] = ok[1] = ok[2] = ok[3] = true;
+    } else {
+#pragma unroll
+        for (int e = 0; e < kItems; ++e) {
+            ok[e] = j0 + e < nc;
+            key[e] = ok[e] ? order_key(row[j0 + e]) : 0u;
+        }
+    }
+}
+
+template <bool VEC>
+__global__ void __launch_bounds__(kThreads)
+k_topk(const Params p, const float *__restrict__ scores, int64_t score_stride, int32_t *__restrict__ idx,
+       int64_t row0)
+{
+    __shared__ unsigned hist[256];
+    __shared__ unsigned s_warp[kWarps];
+    __shared__ unsigned s_prefix, s_need;
+    __shared__ unsigned s_run_gt, s_run_eq;
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int64_t row = row0 + blockIdx.x;   // (b, g, i), i fastest
+    const int i = (int)(row % p.Lq);
+    const int b = (int)(row / ((int64_t)p.Lq * p.Hkv));
+    const int kvl = kvlen_of(p, b);
+    const int pos = pos_of(p, b, i);
+    const int nc = max(0, min(pos - p.w + 1, kvl));   // candidates are keys 0..nc-1
+    const int take = min(p.k, nc);
+    int32_t *out = idx + row * p.k;
+    const float *srow = scores + (int64_t)blockIdx.x * score_stride;
+
+    if (take == nc) {   // every candidate is kept: no need to look at the scores
+        for (int t = tid; t < p.k; t += kThreads) out[t] = t < nc ? t : -1;
+        return;
+    }
+
+    // ---- radix select: value of the take-th largest key
+    unsigned prefix = 0, need = (unsigned)take;
+    for (int round = 0; round < 4; ++round) {
+        const int shift = 24 - 8 * round;
+        if (tid < 256) hist[tid] = 0;
+        __syncthreads();
+        for (int base = 0; base < nc; base += kChunk) {
+            uint32_t key[kItems];
+            bool ok[kItems];
+            load_keys<VEC>(srow, base + tid * kItems, nc, key, ok);
+#pragma unroll
+            for (int e = 0; e < kItems; ++e) {
+                const bool live = ok[e] && (round == 0 || (key[e] >> (shift + 8)) == prefix);
+                const unsigned digit = live ? ((key[e] >> shift) & 255u) : 256u;
+                const unsigned peers = __match_any_sync(0xffffffffu, digit);   // one atomic per distinct digit per warp
+                if (live && lane == __ffs(peers) - 1) atomicAdd(&hist[digit], __popc(peers));
+            }
+        }
+        __syncthreads();
+        if (warp == 0) {
+            // lane l owns digits 255-8l .. 248-8l (descending); find the digit where the count from the top reaches need
+            unsigned mine = 0;
+#pragma unroll
+            for (int e = 0; e < 8; ++e) mine += hist[255 - 8 * lane - e];
+            unsigned incl = mine;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const unsigned t = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += t;
+            }
+            const unsigned before = incl - mine;
+            if (before < need && need <= incl) {
+                unsigned cum = before;
+                for (int e = 0; e < 8; ++e) {
+                    const unsigned c = hist[255 - 8 * lane - e];
+                    if (cum + c >= need) {
+                        s_prefix = (prefix << 8) | (unsigned)(255 - 8 * lane - e);
+                        s_need = need - cum;
+                        break;
+                    }
+                    cum += c;
+                }
+            }
+        }
+        __syncthreads();
+        prefix = s_prefix;
+        need = s_need;
+    }
+    const uint32_t tau = prefix;      // key of the take-th largest candidate
+    const unsigned need_eq = need;    // how many candidates equal to tau are kept (lowest indices first)
+
+    // ---- ordered compaction: kept = key > tau, or key == tau and fewer than need_eq equal keys before it
+    if (tid == 0) { s_run_gt = 0; s_run_eq = 0; }
+    __syncthreads();
+    for (int base = 0; base < nc; base += kChunk) {
+        uint32_t key[kItems];
+        bool ok[kItems];
+        const int j0 = base + tid * kItems;
+        load_keys<VEC>(srow, j0, nc, key, ok);
+        unsigned n_gt = 0, n_eq = 0;
+#pragma unroll
+        for (int e = 0; e < kItems; ++e) {
+            n_gt += ok[e] && key[e] > tau;
+            n_eq += ok[e] && key[e] == tau;
+        }
+        // exclusive scan of (gt, eq) over the block in thread order; both counts fit 16 bits per chunk
+        const unsigned packed = (n_gt << 16) | n_eq;
+        unsigned incl = packed;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const unsigned t = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += t;
+        }
+        if (lane == 31) s_warp[warp] = incl;
+        __syncthreads();
+        const unsigned run_gt = s_run_gt, run_eq = s_run_eq;
+        unsigned wsum = lane < kWarps ? s_warp[lane] : 0u;   // every warp scans the 32 warp totals itself
+        unsigned wincl = wsum;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const unsigned t = __shfl_up_sync(0xffffffffu, wincl, o);
+            if (lane >= o) wincl += t;
+        }
+        const unsigned warp_excl = __shfl_sync(0xffffffffu, wincl - wsum, warp);
+        const unsigned total = __shfl_sync(0xffffffffu, wincl, 31);
+        const unsigned excl = warp_excl + incl - packed;
+        unsigned gt_before = run_gt + (excl >> 16), eq_before = run_eq + (excl & 0xffffu);
+#pragma unroll
+        for (int e = 0; e < kItems; ++e) {
+            if (!ok[e]) continue;
+            if (key[e] > tau) {
+                out[gt_before + min(eq_before, need_eq)] = j0 + e;
+                ++gt_before;
+            } else if (key[e] == tau) {
+                if (eq_before < need_eq) out[gt_before + eq_before] = j0 + e;
+                ++eq_before;
+            }
+        }
+        __syncthreads();   // everyone has read s_warp and the running totals
+        if (tid == 0) { s_run_gt = run_gt + (total >> 16); s_run_eq = run_eq + (total & 0xffffu); }
+    }
+    for (int t = take + tid; t < p.k; t += kThreads) out[t] = -1;
+}
+
+}  // namespace
+
+cudaError_t launch_topk(const Params &p, const float *scores, int64_t score_stride, int32_t *idx, int64_t row0,
+                        int64_t n_rows, cudaStream_t st)
+{
+    if (n_rows == 0 || p.k == 0) return cudaSuccess;
+    const bool vec = (score_stride % 4 == 0) && (reinterpret_cast<uintptr_t>(scores) % 16 == 0);
+    // grid.x is limited to 2^31-1 rows per launch, far above any row block used here
+    if (vec)
+        k_topk<true><<<(unsigned)n_rows, kThreads, 0, st>>>(p, scores, score_stride, idx, row0);
+    else
+        k_topk<false><<<(unsigned)n_rows, kThreads, 0, st>>>(p, scores, score_stride, idx, row0);
+    return cudaGetLastError();
+}
+
+}  // namespace hs2

@@ -1,0 +1,220 @@
+"""GPU parity: the CUDA library, called through the C ABI, against the CPU oracle on the same seeded bytes."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+import paper_2609_26368_b200 as hs2
+from gen import CONFIGS, make_inputs, scaled
+from parity import BlockRun, TOL, assert_output_close, to_host
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _need_gpu():
+    assert torch.cuda.is_available(), "GPU tests need a CUDA device"
+    hs2.load_library()
+
+
+# ---------------------------------------------------------------- configuration 1 (fp32), everything, every row
+
+def test_cfg1_block_every_row():
+    run = BlockRun(make_inputs(CONFIGS["cfg1"])).run_full(want_scores=True)
+    run.check_full(check_scores=True)
+    run.check_idx_bitexact_on_gpu_scores()
+    out, lse = run.run_sparse(0)
+    run.check_sparse(out, lse, 0)
+
+
+def test_cfg1_strip_path_equals_debug_path():
+    """Without scores_dbg the scores go through bounded workspace strips, a few rows at a time."""
+    inp = make_inputs(CONFIGS["cfg1"])
+    a = BlockRun(inp).run_full(want_scores=True)
+    ws = torch.empty(7 * 512 * 4 + 256, dtype=torch.uint8, device="cuda")      # 7 rows per launch
+    b = BlockRun(inp).run_full(want_scores=False, ws=ws)
+    assert torch.equal(a.idx, b.idx)
+    c = BlockRun(inp).run_full(want_scores=False)                               # recommended workspace
+    assert torch.equal(a.idx, c.idx)
+    assert torch.equal(a.O, c.O)
+
+
+# ---------------------------------------------------------------- top-k on given scores: bit exact
+
+def _topk_case(scores: torch.Tensor, k, w, q_start=None, kv_lens=None):
+    B, Hkv, Lq, Lk = scores.shape
+    qs = None if q_start is None else torch.tensor(q_start, dtype=torch.int32, device="cuda")
+    kl = None if kv_lens is None else torch.tensor(kv_lens, dtype=torch.int32, device="cuda")
+    prob = hs2.Problem(B, Lq, Lk, Hkv, Hkv, 1, k, w, dtype=torch.float32, q_start=qs, kv_lens=kl)
+    got = hs2.hs2_topk_select(prob, scores.cuda().contiguous()).cpu().numpy()
+    pos, kvl = [], []
+    for b in range(B):
+        n = Lk if kv_lens is None else kv_lens[b]
+        q0 = n - Lq if q_start is None else q_start[b]
+        for g in range(Hkv):
+            for i in range(Lq):
+                pos.append(q0 + i)
+                kvl.append(n)
+    want = oracle.select(scores.numpy().reshape(-1, Lk), np.array(pos), np.array(kvl), w, k)
+    assert np.array_equal(got.reshape(-1, k), want)
+
+
+@pytest.mark.parametrize("Lk,k,w", [(512, 64, 16), (1000, 100, 0), (4099, 257, 33), (9001, 1024, 128)])
+def test_topk_random_scores(Lk, k, w):
+    g = torch.Generator().manual_seed(Lk)
+    _topk_case(torch.randn(2, 2, 37, Lk, generator=g), k, w, q_start=[Lk - 37, Lk // 2], kv_lens=[Lk, Lk - 5])
+
+
+def test_topk_adversarial_rows():
+    Lk = 2500
+    g = torch.Generator().manual_seed(5)
+    rows = [
+        torch.zeros(Lk),                                                   # all equal: lowest indices win
+        torch.full((Lk,), -3.25),
+        torch.randint(0, 4, (Lk,), generator=g).float(),                   # four distinct values
+        torch.where(torch.arange(Lk) % 2 == 0, torch.tensor(0.0), torch.tensor(-0.0)),     # +0 / -0 tie
+        torch.randn(Lk, generator=g) * 1e-41,                              # denormals
+        torch.cat([torch.full((Lk // 2,), float("-inf")), torch.randn(Lk - Lk // 2, generator=g)]),
+        torch.cat([torch.full((5,), float("inf")), torch.randn(Lk - 5, generator=g)]),
+        -torch.rand(Lk, generator=g) * 30.0,                               # log-probability like
+        torch.arange(Lk).float(),                                          # ascending: the last k candidates
+        -torch.arange(Lk).float(),                                         # descending: the first k
+        torch.randn(Lk, generator=g).abs().log(),
+        (torch.randn(Lk, generator=g) * 4).round() / 4 - 12.0,             # dense near-ties
+    ]
+    scores = torch.stack(rows).view(1, 1, len(rows), Lk)
+    for k, w in [(1, 0), (300, 7), (1024, 128), (2400, 50), (4000, 0)]:     # k >= candidates included
+        _topk_case(scores, k, w, q_start=[Lk - 1 - len(rows) + 1])
+
+
+def test_topk_edges_window_and_lengths():
+    g = torch.Generator().manual_seed(9)
+    s = torch.randn(1, 3, 1, 777, generator=g)
+    _topk_case(s, 50, 10)                                                  # Lq = 1 (decode)
+    _topk_case(s, 50, 777)                                                 # window covers everything: all -1
+    _topk_case(s, 50, 5000)
+    _topk_case(s, 900, 3)                                                  # k above the context
+    s2 = torch.randn(2, 1, 40, 129, generator=g)
+    _topk_case(s2, 16, 4, q_start=[0, 60], kv_lens=[129, 77])              # early rows; query past a short cache
+    _topk_case(s2, 16, 4, q_start=[-3, 200], kv_lens=[129, 0])             # negative positions; empty cache
+
+
+# ---------------------------------------------------------------- small shapes, both dtypes, ragged tails, strides
+
+SMALL = [
+    # name, overrides
+    ("cfg1", dict(q_len=131, kv_len=131, k_sel=17, window=5)),
+    ("cfg1", dict(q_len=40, kv_len=300, k_sel=33, window=9, n_q_heads=6, n_kv_heads=2, head_dim=32)),
+    ("cfg2", dict(q_len=333, kv_len=333, k_sel=48, window=13, n_needles=8)),
+    ("cfg2", dict(q_len=257, kv_len=257, k_sel=64, window=16, n_q_heads=8, n_kv_heads=2, head_dim=64, n_needles=8)),
+    ("cfg2", dict(q_len=96, kv_len=1029, k_sel=128, window=32, n_needles=8, batch=2)),
+    ("cfg4", dict(q_len=600, kv_len=600, k_sel=100, window=20, n_clusters=8)),
+    ("cfg2", dict(q_len=200, kv_len=200, k_sel=300, window=8, n_needles=4)),            # k above the context
+    ("cfg2", dict(q_len=200, kv_len=200, k_sel=0, window=24, n_needles=4)),              # pure sliding window
+    ("cfg2", dict(q_len=200, kv_len=200, k_sel=40, window=0, n_needles=4)),              # no window
+    ("cfg2", dict(q_len=150, kv_len=150, k_sel=16, window=4, n_q_heads=4, n_kv_heads=4, n_needles=4)),   # group of 1
+    ("cfg2", dict(q_len=150, kv_len=150, k_sel=16, window=4, n_q_heads=16, n_kv_heads=1, n_needles=4)),  # MQA 16
+]
+
+
+@pytest.mark.parametrize("name,over", SMALL)
+def test_small_block_every_row(name, over):
+    wl = scaled(name, **over)
+    run = BlockRun(make_inputs(wl)).run_full(want_scores=True)
+    run.check_full(check_scores=True)
+    if wl.k_sel > 0:
+        run.check_idx_bitexact_on_gpu_scores()
+    for layer in range(len(run.qs)):
+        out, lse = run.run_sparse(layer)
+        run.check_sparse(out, lse, layer)
+
+
+def test_ragged_lengths_offsets_strides_and_sink():
+    wl = scaled("cfg2", batch=3, q_len=70, kv_len=400, k_sel=40, window=12, n_needles=4)
+    inp = make_inputs(wl)
+    dev = "cuda"
+    q_start, kv_lens = [330, 100, 0], [400, 250, 64]
+    qs_t = torch.tensor(q_start, dtype=torch.int32, device=dev)
+    kl_t = torch.tensor(kv_lens, dtype=torch.int32, device=dev)
+    # non-packed views: Q inside a wider buffer, K/V as slices of a fused [.., 2, Hkv, D] cache
+    B, Lq, Hq, D = inp.q_full.shape
+    qbuf = torch.zeros(B, Lq, Hq + 3, D + 8, dtype=inp.q_full.dtype, device=dev)
+    q = qbuf[:, :, 1:1 + Hq, :D]
+    q.copy_(inp.q_full)
+    kvbuf = torch.zeros(B, wl.kv_len, 2, wl.n_kv_heads, D, dtype=inp.k.dtype, device=dev)
+    kvbuf[:, :, 0].copy_(inp.k)
+    kvbuf[:, :, 1].copy_(inp.v)
+    k, v = kvbuf[:, :, 0], kvbuf[:, :, 1]
+    prob = hs2.Problem.from_tensors(q, k, wl.k_sel, wl.window, softmax_scale=0.11, q_start=qs_t, kv_lens=kl_t)
+    O, LSE, idx, sc = hs2.hs2_full_attn_select(prob, q, k, v, want_scores=True)
+    torch.cuda.synchronize()
+    Oo, LSEo, idxo, sco = oracle.full_attn_select(inp.q_full, inp.k, inp.v, wl.k_sel, wl.window, scale=0.11,
+                                                  q_start=q_start, kv_lens=kv_lens, want_scores=True)
+    dt = wl.torch_dtype
+    assert_output_close(O.reshape(-1, Hq, D), Oo, dt, "full O")
+    from parity import check_idx_against_oracle
+    idx_rows = idx.permute(0, 2, 1, 3).reshape(B * Lq, wl.n_kv_heads, wl.k_sel).cpu().numpy()
+    check_idx_against_oracle(idx_rows, idxo, sco)
+    sink = torch.linspace(-1.0, 2.0, Hq, device=dev)
+    qsp = inp.q_sparse[0].to(dev)
+    for fn_sink in (None, sink):
+        out, lse = hs2.hs2_sparse_attn_prefill(prob, qsp, k, v, idx, sink=fn_sink, want_lse=True)
+        torch.cuda.synchronize()
+        Os, LSEs, _ = oracle.sparse_attn(inp.q_sparse[0], inp.k, inp.v, idx_rows, wl.window, scale=0.11,
+                                         q_start=q_start, kv_lens=kv_lens,
+                                         sink=None if fn_sink is None else fn_sink.cpu().numpy())
+        assert_output_close(out.reshape(-1, Hq, D), Os, dt, "sparse O")
+        l = lse.permute(0, 2, 1).reshape(B * Lq, Hq).cpu().numpy()
+        fin = np.isfinite(LSEs)
+        assert np.array_equal(np.isfinite(l), fin)
+        assert np.abs(l[fin] - LSEs[fin]).max() <= TOL[dt]["lse"]
+
+
+def test_malformed_indices_cannot_read_out_of_bounds():
+    wl = scaled("cfg2", q_len=64, kv_len=64, k_sel=32, window=8, n_needles=4)
+    inp = make_inputs(wl)
+    run = BlockRun(inp)
+    g = torch.Generator().manual_seed(3)
+    idx = torch.randint(-50, 1 << 30, (1, wl.n_kv_heads, 64, 32), generator=g, dtype=torch.int32)
+    idx[..., ::3] = torch.randint(0, 64, idx[..., ::3].shape, generator=g, dtype=torch.int32)
+    # keep the rows free of repeated valid entries (repeats are a documented caller error)
+    for gh in range(wl.n_kv_heads):
+        for i in range(64):
+            row = idx[0, gh, i]
+            seen = set()
+            for t in range(32):
+                j = int(row[t])
+                if 0 <= j <= i - 8:
+                    if j in seen:
+                        row[t] = -1
+                    seen.add(j)
+    run.idx = idx.cuda()
+    out, lse = run.run_sparse(0)
+    run.check_sparse(out, lse, 0)
+
+
+# ---------------------------------------------------------------- decode
+
+def test_decode_small_matches_oracle_and_prefill_last_row():
+    wl = scaled("cfg5", batch=5, kv_len=3000, k_sel=256, window=32, n_needles=8)
+    run = BlockRun(make_inputs(wl)).run_full(want_scores=True)
+    run.check_full(check_scores=True)
+    run.check_idx_bitexact_on_gpu_scores()
+    out_d, lse_d = run.run_sparse(0, decode=True)
+    run.check_sparse(out_d, lse_d, 0)
+    out_p, lse_p = run.run_sparse(0, decode=False)
+    assert (out_d.float() - out_p.float()).abs().max() <= 2e-2
+    kv_lens = torch.tensor([3000, 1, 17, 2999, 300], dtype=torch.int32, device="cuda")
+    prob = hs2.Problem.from_tensors(run.q, run.k, wl.k_sel, wl.window, kv_lens=kv_lens)
+    O, LSE, idx, _ = hs2.hs2_full_attn_select(prob, run.q, run.k, run.v)
+    out, _ = hs2.hs2_sparse_attn_decode(prob, run.qs[0], run.k, run.v, idx)
+    torch.cuda.synchronize()
+    Oo, _, idxo, sco = oracle.full_attn_select(to_host(run.q), to_host(run.k), to_host(run.v), wl.k_sel, wl.window,
+                                               kv_lens=kv_lens.cpu().numpy(), want_scores=True)
+    assert_output_close(O[:, 0], Oo, wl.torch_dtype, "ragged decode full O")
+    idx_rows = idx[:, :, 0].cpu().numpy()
+    from parity import check_idx_against_oracle
+    check_idx_against_oracle(idx_rows, idxo, sco)
+    Os, _, _ = oracle.sparse_attn(to_host(run.qs[0]), to_host(run.k), to_host(run.v), idx_rows, wl.window,
+                                  kv_lens=kv_lens.cpu().numpy())
+    assert_output_close(out[:, 0], Os, wl.torch_dtype, "ragged decode sparse O")
