@@ -111,7 +111,7 @@ class BlockRun:
         swaps = check_idx_against_oracle(idx_gpu, idxo, sco)
         if check_scores and self.scores is not None:
             sg = gather_rows(self.scores, rows, "bgik").cpu().numpy().astype(np.float64)
-            vis = np.isfinite(np.log(sco))
+            vis = ~np.isneginf(sco)
             assert np.array_equal(np.isneginf(sg), ~vis), "visibility pattern of scores_dbg"
             err = np.abs(sg[vis] - np.log(sco[vis]))
             assert err.max() <= TOL[dt]["score"], "log-score max-abs %.3e" % err.max()
