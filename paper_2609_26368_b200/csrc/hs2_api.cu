@@ -72,6 +72,12 @@ bool ws_ok(const void *ws, size_t ws_bytes, size_t need)
     return ws != nullptr && ws_bytes >= need && reinterpret_cast<uintptr_t>(ws) % 256 == 0;
 }
 
+bool aligned16(const void *a, const void *b, const void *c, const void *d)
+{
+    return ((reinterpret_cast<uintptr_t>(a) | reinterpret_cast<uintptr_t>(b) | reinterpret_cast<uintptr_t>(c) |
+             reinterpret_cast<uintptr_t>(d)) & 15) == 0;
+}
+
 hs2_status check_device()
 {
     int dev = -1;
@@ -130,7 +136,7 @@ hs2_status hs2_full_attn_select(const hs2_problem *hp, const void *Q, const void
     if ((s = check_device()) != HS2_OK) return s;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     const hs2_dtype dt = hp->dtype;
-    const bool mma = full_mma_supported(p, dt);
+    const bool mma = full_mma_supported(p, dt) && aligned16(Q, K, V, O);
     cudaError_t e = mma ? launch_full_attn_mma(p, Q, K, V, O, LSE, st) : launch_full_attn_generic(p, dt, Q, K, V, O, LSE, st);
     if (e != cudaSuccess) return cuda_fail(e);
     if (!want_sel && !scores_dbg) return HS2_OK;
@@ -182,7 +188,7 @@ hs2_status hs2_sparse_attn_prefill(const hs2_problem *hp, const void *Q, const v
     if (s != HS2_OK) return s;
     if ((s = check_device()) != HS2_OK) return s;
     cudaStream_t st = (cudaStream_t)cuda_stream;
-    cudaError_t e = sparse_mma_supported(p, hp->dtype)
+    cudaError_t e = (sparse_mma_supported(p, hp->dtype) && aligned16(Q, K, V, O))
                         ? launch_sparse_mma_prefill(p, Q, K, V, idx, sink, O, LSE, st)
                         : launch_sparse_generic(p, hp->dtype, Q, K, V, idx, sink, O, LSE, st);
     return e == cudaSuccess ? HS2_OK : cuda_fail(e);
@@ -196,7 +202,7 @@ hs2_status hs2_sparse_attn_decode(const hs2_problem *hp, const void *Q, const vo
     hs2_status s = sparse_common(hp, Q, K, V, idx, O, &p);
     if (s != HS2_OK) return s;
     if (p.Lq != 1) return HS2_ERR_INVALID_ARG;
-    const bool mma = sparse_mma_supported(p, hp->dtype);
+    const bool mma = sparse_mma_supported(p, hp->dtype) && aligned16(Q, K, V, O);
     if (mma && !ws_ok(ws, ws_bytes, sparse_mma_decode_ws_bytes(p))) return HS2_ERR_WORKSPACE_TOO_SMALL;
     if ((s = check_device()) != HS2_OK) return s;
     cudaStream_t st = (cudaStream_t)cuda_stream;

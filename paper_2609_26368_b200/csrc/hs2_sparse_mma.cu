@@ -1,10 +1,530 @@
-// placeholder until the tensor-core sparse kernels land
+// Sparse attention over (reused top-k indices) U (forced window) for bf16, head_dim 128, group <= 8
+// (Section 3.3: both selected sets are read from the full-attention layer's KV cache).
+//
+// The work is a gather: per (query, KV head) up to k+w rows of K and of V, 256 bytes each, are
+// fetched once and shared by the G query heads of the group.  It is bound by memory, so the design
+// goal is bytes in flight, not flops:
+//   * one warp owns one (query, KV head) item (prefill) or one split of it (decode) and runs its own
+//     cp.async pipeline: NSTAGE stages of KT key rows (K and V), 16-byte copies, rows placed in
+//     shared memory with an XOR swizzle so that ldmatrix is conflict free; no CTA-wide barriers;
+//   * the G x keys products go through tensor cores only because plain FMAs could not keep up with
+//     the memory system at 8 flop/byte: S^T = K Q^T with the keys on the MMA M dimension and the
+//     (padded to 8) heads on N, so nothing of the m16n8k16 tile is wasted; P^T is re-laid out for the
+//     second product with movmatrix; O^T = V^T P^T reads V through ldmatrix.trans;
+//   * online softmax in the base-2 domain with warp shuffles across the 8 key rows of a fragment.
+// Decode splits the attended set of one (sequence, KV head) over several warps; each writes an
+// un-normalised partial (m, l, O) and the last one to arrive (an atomic ticket, nobody waits) merges.
 #include "hs2_common.cuh"
+
+#ifndef HS2_SP_KT
+#define HS2_SP_KT 16
+#endif
+#ifndef HS2_SP_NSTAGE
+#define HS2_SP_NSTAGE 4
+#endif
+#ifndef HS2_SP_WARPS
+#define HS2_SP_WARPS 6
+#endif
+
 namespace hs2 {
-bool sparse_mma_supported(const Params &, hs2_dtype) { return false; }
-cudaError_t launch_sparse_mma_prefill(const Params &, const void *, const void *, const void *, const int32_t *,
-                                      const float *, void *, float *, cudaStream_t) { return cudaErrorNotSupported; }
-size_t sparse_mma_decode_ws_bytes(const Params &) { return 0; }
-cudaError_t launch_sparse_mma_decode(const Params &, const void *, const void *, const void *, const int32_t *,
-                                     const float *, void *, float *, void *, size_t, cudaStream_t) { return cudaErrorNotSupported; }
+namespace {
+
+constexpr int HD = 128;                      // head_dim
+constexpr int kRowBytes = HD * 2;            // one K or V row
+constexpr int KT = HS2_SP_KT;                // key rows per pipeline stage (16 or 32)
+constexpr int NSTAGE = HS2_SP_NSTAGE;
+constexpr int WARPS = HS2_SP_WARPS;
+constexpr int kStageBytes = 2 * KT * kRowBytes;           // K tile then V tile
+constexpr int kWarpSmem = NSTAGE * kStageBytes + NSTAGE * 32 * 4;   // + per-stage key index of each row
+constexpr int kMaxSplits = 32;
+static_assert(KT == 16 || KT == 32, "a stage holds 16 or 32 key rows");
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, int src_bytes)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(src_bytes));
 }
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N)); }
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a)
+{
+    uint32_t d;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;\n" : "=r"(d) : "r"(a));
+    return d;
+}
+__device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
+{
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t *>(&v);
+}
+
+// Accumulators of one warp.  Thread (g = lane/4, t = lane%4) owns heads 2t and 2t+1 of the group:
+// o[dt][0..3] = O^T at (d = 16 dt + g, head 2t), (same d, head 2t+1), (d + 8, head 2t), (d + 8, head 2t+1);
+// m is replicated over g, l is this thread's partial sum (reduced over g at the end).
+struct Acc {
+    float o[8][4];
+    float m[2], l[2];
+};
+
+struct Item {
+    const char *Kb, *Vb;      // first row of this (sequence, KV head), bytes
+    int64_t row_stride;       // bytes between consecutive tokens
+    const int32_t *irow;      // idx row of this (query, KV head), or nullptr when k == 0
+    int pos, kvl;
+};
+
+// key index held by slot s of the virtual slot array [idx row | window], -1 when the slot is void
+__device__ __forceinline__ int slot_key(const Params &p, const Item &it, int tile, int lane)
+{
+    const int s = tile * KT + lane;
+    int j = -1;
+    if (lane < KT) {
+        if (s < p.k) {
+            j = __ldg(it.irow + s);
+            if (j > it.pos - p.w || j >= it.kvl) j = -1;
+        } else if (s < p.k + p.w) {
+            j = it.pos - p.w + 1 + (s - p.k);
+            if (j > it.pos || j >= it.kvl) j = -1;
+        }
+    }
+    return j;   // negative entries stay negative
+}
+
+__device__ __forceinline__ void issue_stage(const Item &it, uint32_t stage_base, int j, int lane)
+{
+    const int c = lane & 15;
+#pragma unroll
+    for (int r0 = 0; r0 < KT; r0 += 2) {
+        const int r = r0 + (lane >> 4);
+        const int jr = __shfl_sync(0xffffffffu, j, r);
+        const uint32_t dst = stage_base + r * kRowBytes + ((c ^ (r & 7)) << 4);
+        const int64_t off = (int64_t)(jr < 0 ? 0 : jr) * it.row_stride + c * 16;
+        const int nbytes = jr < 0 ? 0 : 16;   // void rows are zero filled, nothing is read
+        cp_async16(dst, it.Kb + off, nbytes);
+        cp_async16(dst + KT * kRowBytes, it.Vb + off, nbytes);
+    }
+}
+
+__device__ __forceinline__ void consume_stage(Acc &acc, const uint32_t (&qf)[16], uint32_t stage_base, unsigned mask,
+                                              float scale_log2, int lane)
+{
+    const int g = lane >> 2;
+    const int mi = lane >> 3, rr = lane & 7;
+    constexpr int MT = KT / 16;
+    float s[MT][4];
+    // S^T = K Q^T : rows = keys, columns = heads
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt) {
+        s[mt][0] = s[mt][1] = s[mt][2] = s[mt][3] = 0.f;
+        const uint32_t rowaddr = stage_base + (mt * 16 + (mi & 1) * 8 + rr) * kRowBytes;
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+            uint32_t a[4];
+            ldmatrix_x4(a, rowaddr + (((2 * ks + (mi >> 1)) ^ rr) << 4));
+            mma_bf16(s[mt], a, qf[2 * ks], qf[2 * ks + 1]);
+        }
+    }
+    // online softmax, base-2 domain; this thread: heads 2t+hh, keys 16 mt + g + 8 r
+    float mx[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+        for (int r = 0; r < 2; ++r) {
+            const bool ok = (mask >> (mt * 16 + g + 8 * r)) & 1u;
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {
+                const float t2 = ok ? s[mt][2 * r + hh] * scale_log2 : -INFINITY;
+                s[mt][2 * r + hh] = t2;
+                mx[hh] = fmaxf(mx[hh], t2);
+            }
+        }
+    float corr[2], muse[2];
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh) {
+        mx[hh] = fmaxf(mx[hh], __shfl_xor_sync(0xffffffffu, mx[hh], 4));
+        mx[hh] = fmaxf(mx[hh], __shfl_xor_sync(0xffffffffu, mx[hh], 8));
+        mx[hh] = fmaxf(mx[hh], __shfl_xor_sync(0xffffffffu, mx[hh], 16));
+        const float m_new = fmaxf(acc.m[hh], mx[hh]);
+        muse[hh] = m_new == -INFINITY ? 0.f : m_new;
+        corr[hh] = exp2f(acc.m[hh] - muse[hh]);
+        acc.m[hh] = m_new;
+        acc.l[hh] *= corr[hh];
+    }
+    uint32_t pb[MT][2];
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt) {
+        float pv[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            pv[e] = exp2f(s[mt][e] - muse[e & 1]);
+            acc.l[e & 1] += pv[e];
+        }
+        pb[mt][0] = movmatrix_trans(pack_bf16(pv[0], pv[1]));   // keys 16 mt + 0..7
+        pb[mt][1] = movmatrix_trans(pack_bf16(pv[2], pv[3]));   // keys 16 mt + 8..15
+    }
+#pragma unroll
+    for (int dt = 0; dt < 8; ++dt) {
+        acc.o[dt][0] *= corr[0]; acc.o[dt][1] *= corr[1];
+        acc.o[dt][2] *= corr[0]; acc.o[dt][3] *= corr[1];
+    }
+    // O^T += V^T P^T : rows = output dimensions, contraction over the keys of the stage
+    const uint32_t vbase = stage_base + KT * kRowBytes;
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt) {
+        const uint32_t rowaddr = vbase + (mt * 16 + (mi >> 1) * 8 + rr) * kRowBytes;
+#pragma unroll
+        for (int dt = 0; dt < 8; ++dt) {
+            uint32_t a[4];
+            ldmatrix_x4_trans(a, rowaddr + (((2 * dt + (mi & 1)) ^ rr) << 4));
+            mma_bf16(acc.o[dt], a, pb[mt][0], pb[mt][1]);
+        }
+    }
+}
+
+// Fold slot tiles [t_begin, t_end) of one item into acc with an NSTAGE-deep cp.async pipeline.
+__device__ __forceinline__ void run_tiles(const Params &p, const Item &it, const uint32_t (&qf)[16], Acc &acc,
+                                          int t_begin, int t_end, char *wsm, int lane)
+{
+    const uint32_t sbase = smem_u32(wsm);
+    int *sj = reinterpret_cast<int *>(wsm + NSTAGE * kStageBytes);
+    int next = t_begin;
+    int jn = next < t_end ? slot_key(p, it, next, lane) : -1;
+    auto try_issue = [&](int stage) -> bool {
+        while (next < t_end) {
+            const int j = jn;
+            ++next;
+            if (next < t_end) jn = slot_key(p, it, next, lane);
+            if (__ballot_sync(0xffffffffu, j >= 0)) {
+                sj[stage * 32 + lane] = j;
+                issue_stage(it, sbase + stage * kStageBytes, j, lane);
+                return true;
+            }
+        }
+        return false;
+    };
+    int n_issued = 0, n_done = 0;
+#pragma unroll
+    for (int s = 0; s < NSTAGE - 1; ++s) {
+        if (try_issue(n_issued % NSTAGE)) ++n_issued;
+        cp_async_commit();
+    }
+    while (n_done < n_issued) {
+        cp_async_wait<NSTAGE - 2>();
+        __syncwarp();
+        if (try_issue(n_issued % NSTAGE)) ++n_issued;
+        cp_async_commit();
+        const int stage = n_done % NSTAGE;
+        const unsigned mask = __ballot_sync(0xffffffffu, sj[stage * 32 + lane] >= 0);
+        consume_stage(acc, qf, sbase + stage * kStageBytes, mask, p.scale_log2, lane);
+        ++n_done;
+    }
+    cp_async_wait<0>();
+    __syncwarp();
+}
+
+__device__ __forceinline__ void load_q_frags(const Params &p, const __nv_bfloat16 *Q, int b, int i, int gkv, int lane,
+                                             uint32_t (&qf)[16])
+{
+    const int g = lane >> 2, t = lane & 3;
+    if (g < p.G) {
+        const uint32_t *q = reinterpret_cast<const uint32_t *>(Q + b * p.qs_b + i * p.qs_t + (gkv * p.G + g) * p.qs_h);
+#pragma unroll
+        for (int ks = 0; ks < 8; ++ks) {
+            qf[2 * ks] = __ldg(q + ks * 8 + t);
+            qf[2 * ks + 1] = __ldg(q + ks * 8 + 4 + t);
+        }
+    } else {
+#pragma unroll
+        for (int e = 0; e < 16; ++e) qf[e] = 0u;
+    }
+}
+
+__device__ __forceinline__ void init_acc(Acc &acc, const Params &p, const float *sink, int gkv, int lane, bool with_sink)
+{
+    const int g = lane >> 2, t = lane & 3;
+#pragma unroll
+    for (int dt = 0; dt < 8; ++dt) acc.o[dt][0] = acc.o[dt][1] = acc.o[dt][2] = acc.o[dt][3] = 0.f;
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh) {
+        const int head = 2 * t + hh;
+        float m = -INFINITY;
+        if (with_sink && sink && head < p.G) m = sink[gkv * p.G + head] * kLog2e;
+        acc.m[hh] = m;
+        acc.l[hh] = (m != -INFINITY && g == 0) ? 1.f : 0.f;   // e^{sink - m} = 1, counted once
+    }
+}
+
+__device__ __forceinline__ void reduce_l(Acc &acc)
+{
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh) {
+        acc.l[hh] += __shfl_xor_sync(0xffffffffu, acc.l[hh], 4);
+        acc.l[hh] += __shfl_xor_sync(0xffffffffu, acc.l[hh], 8);
+        acc.l[hh] += __shfl_xor_sync(0xffffffffu, acc.l[hh], 16);
+    }
+}
+
+// Normalise and store one (query, KV head) result: O rows of the G heads (16-byte stores, staged
+// through the warp's shared memory) and LSE.
+__device__ __forceinline__ void store_output(const Params &p, const Acc &acc, __nv_bfloat16 *O, float *LSE, int b, int i,
+                                             int gkv, char *wsm, int lane)
+{
+    const int g = lane >> 2, t = lane & 3;
+    constexpr int kPitch = HD + 8;   // bf16 elements per staged head row (bank spread)
+    __nv_bfloat16 *so = reinterpret_cast<__nv_bfloat16 *>(wsm);
+    float inv[2];
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh) inv[hh] = acc.l[hh] > 0.f ? 1.f / acc.l[hh] : 0.f;
+#pragma unroll
+    for (int dt = 0; dt < 8; ++dt)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int head = 2 * t + (e & 1), d = 16 * dt + g + 8 * (e >> 1);
+            so[head * kPitch + d] = __float2bfloat16_rn(acc.o[dt][e] * inv[e & 1]);
+        }
+    __syncwarp();
+#pragma unroll
+    for (int v = lane; v < 8 * 16; v += 32) {
+        const int head = v >> 4, c = v & 15;
+        if (head < p.G) {
+            const uint4 val = *reinterpret_cast<const uint4 *>(so + head * kPitch + c * 8);
+            *reinterpret_cast<uint4 *>(O + b * p.os_b + i * p.os_t + (gkv * p.G + head) * p.os_h + c * 8) = val;
+        }
+    }
+    if (LSE && g == 0) {
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {
+            const int head = 2 * t + hh;
+            if (head < p.G)
+                LSE[((int64_t)b * p.Hq + gkv * p.G + head) * p.Lq + i] =
+                    acc.l[hh] > 0.f ? (acc.m[hh] + log2f(acc.l[hh])) * kLn2 : -INFINITY;
+        }
+    }
+    __syncwarp();
+}
+
+__device__ __forceinline__ Item make_item(const Params &p, const __nv_bfloat16 *K, const __nv_bfloat16 *V,
+                                          const int32_t *idx, int b, int gkv, int i)
+{
+    Item it;
+    const int64_t base = b * p.ks_b + gkv * p.ks_h;
+    it.Kb = reinterpret_cast<const char *>(K + base);
+    it.Vb = reinterpret_cast<const char *>(V + base);
+    it.row_stride = p.ks_t * 2;
+    it.irow = idx ? idx + (((int64_t)b * p.Hkv + gkv) * p.Lq + i) * p.k : nullptr;
+    it.pos = pos_of(p, b, i);
+    it.kvl = kvlen_of(p, b);
+    return it;
+}
+
+// ---------------------------------------------------------------- prefill: one warp per (b, g, i)
+__global__ void __launch_bounds__(WARPS * 32)
+k_sparse_prefill(const Params p, const __nv_bfloat16 *__restrict__ Q, const __nv_bfloat16 *__restrict__ K,
+                 const __nv_bfloat16 *__restrict__ V, const int32_t *__restrict__ idx, const float *__restrict__ sink,
+                 __nv_bfloat16 *__restrict__ O, float *__restrict__ LSE)
+{
+    extern __shared__ __align__(128) char smem[];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t item = (int64_t)blockIdx.x * WARPS + warp;   // (b, g, i), i fastest
+    if (item >= (int64_t)p.B * p.Hkv * p.Lq) return;
+    const int i = (int)(item % p.Lq);
+    const int gkv = (int)((item / p.Lq) % p.Hkv);
+    const int b = (int)(item / ((int64_t)p.Lq * p.Hkv));
+    char *wsm = smem + warp * kWarpSmem;
+    const Item it = make_item(p, K, V, idx, b, gkv, i);
+    uint32_t qf[16];
+    load_q_frags(p, Q, b, i, gkv, lane, qf);
+    Acc acc;
+    init_acc(acc, p, sink, gkv, lane, true);
+    const int n_tiles = (p.k + p.w + KT - 1) / KT;
+    run_tiles(p, it, qf, acc, 0, n_tiles, wsm, lane);
+    reduce_l(acc);
+    store_output(p, acc, O, LSE, b, i, gkv, wsm, lane);
+}
+
+// ---------------------------------------------------------------- decode: one warp per (b, g, split)
+struct DecodeWs {
+    int *tickets;     // [B * Hkv]
+    float *ml;        // [items][2][8]   m then l per head
+    float4 *opart;    // [items][8][32]  o[dt] of every lane
+};
+
+__global__ void __launch_bounds__(WARPS * 32)
+k_sparse_decode(const Params p, const __nv_bfloat16 *__restrict__ Q, const __nv_bfloat16 *__restrict__ K,
+                const __nv_bfloat16 *__restrict__ V, const int32_t *__restrict__ idx, const float *__restrict__ sink,
+                __nv_bfloat16 *__restrict__ O, float *__restrict__ LSE, DecodeWs ws, int n_splits, int tiles_per_split)
+{
+    extern __shared__ __align__(128) char smem[];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t item = (int64_t)blockIdx.x * WARPS + warp;   // (b, g, split), split fastest
+    if (item >= (int64_t)p.B * p.Hkv * n_splits) return;
+    const int split = (int)(item % n_splits);
+    const int bg = (int)(item / n_splits);
+    const int gkv = bg % p.Hkv, b = bg / p.Hkv;
+    const int g = lane >> 2, t = lane & 3;
+    char *wsm = smem + warp * kWarpSmem;
+    const Item it = make_item(p, K, V, idx, b, gkv, 0);
+    uint32_t qf[16];
+    load_q_frags(p, Q, b, 0, gkv, lane, qf);
+    Acc acc;
+    init_acc(acc, p, sink, gkv, lane, split == 0);   // the sink joins the denominator once
+    const int n_tiles = (p.k + p.w + KT - 1) / KT;
+    const int t0 = split * tiles_per_split;
+    run_tiles(p, it, qf, acc, t0, min(n_tiles, t0 + tiles_per_split), wsm, lane);
+    reduce_l(acc);
+    // publish the un-normalised partial
+    float4 *op = ws.opart + item * 8 * 32;
+#pragma unroll
+    for (int dt = 0; dt < 8; ++dt) op[dt * 32 + lane] = make_float4(acc.o[dt][0], acc.o[dt][1], acc.o[dt][2], acc.o[dt][3]);
+    if (g == 0) {
+        float *ml = ws.ml + item * 16;
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) { ml[2 * t + hh] = acc.m[hh]; ml[8 + 2 * t + hh] = acc.l[hh]; }
+    }
+    __threadfence();
+    __syncwarp();
+    int ticket = 0;
+    if (lane == 0) ticket = atomicAdd(ws.tickets + bg, 1);
+    ticket = __shfl_sync(0xffffffffu, ticket, 0);
+    if (ticket != n_splits - 1) return;   // someone else finishes later and merges
+    __threadfence();
+    // merge the partials of all splits of this (sequence, KV head)
+    const int64_t first = (int64_t)bg * n_splits;
+    float M[2] = {-INFINITY, -INFINITY};
+    for (int s = 0; s < n_splits; ++s) {
+        const float *ml = ws.ml + (first + s) * 16;
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) M[hh] = fmaxf(M[hh], __ldcg(ml + 2 * t + hh));
+    }
+    Acc tot;
+#pragma unroll
+    for (int dt = 0; dt < 8; ++dt) tot.o[dt][0] = tot.o[dt][1] = tot.o[dt][2] = tot.o[dt][3] = 0.f;
+    tot.l[0] = tot.l[1] = 0.f;
+    tot.m[0] = M[0]; tot.m[1] = M[1];
+    for (int s = 0; s < n_splits; ++s) {
+        const float *ml = ws.ml + (first + s) * 16;
+        float wgt[2];
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {
+            const float ms = __ldcg(ml + 2 * t + hh);
+            wgt[hh] = ms == -INFINITY ? 0.f : exp2f(ms - M[hh]);
+            tot.l[hh] += wgt[hh] * __ldcg(ml + 8 + 2 * t + hh);
+        }
+        const float4 *ops = ws.opart + (first + s) * 8 * 32;
+#pragma unroll
+        for (int dt = 0; dt < 8; ++dt) {
+            const float4 v = __ldcg(ops + dt * 32 + lane);
+            tot.o[dt][0] += wgt[0] * v.x; tot.o[dt][1] += wgt[1] * v.y;
+            tot.o[dt][2] += wgt[0] * v.z; tot.o[dt][3] += wgt[1] * v.w;
+        }
+    }
+    store_output(p, tot, O, LSE, b, 0, gkv, wsm, lane);
+}
+
+size_t ws_tickets_bytes(const Params &p) { return ((size_t)p.B * p.Hkv * sizeof(int) + 255) / 256 * 256; }
+
+int g_sm_count = 0;
+cudaError_t sm_count(int *n)
+{
+    if (g_sm_count == 0) {
+        int dev = 0, v = 0;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e != cudaSuccess) return e;
+        e = cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev);
+        if (e != cudaSuccess) return e;
+        g_sm_count = v;
+    }
+    *n = g_sm_count;
+    return cudaSuccess;
+}
+
+bool g_attr_set = false;
+cudaError_t set_attrs()
+{
+    if (g_attr_set) return cudaSuccess;
+    cudaError_t e = cudaFuncSetAttribute(k_sparse_prefill, cudaFuncAttributeMaxDynamicSharedMemorySize, WARPS * kWarpSmem);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(k_sparse_decode, cudaFuncAttributeMaxDynamicSharedMemorySize, WARPS * kWarpSmem);
+    if (e != cudaSuccess) return e;
+    g_attr_set = true;
+    return cudaSuccess;
+}
+
+}  // namespace
+
+bool sparse_mma_supported(const Params &p, hs2_dtype dt)
+{
+    auto m8 = [](int64_t x) { return x % 8 == 0; };
+    return dt == HS2_BF16 && p.D == HD && p.G >= 1 && p.G <= 8 && m8(p.qs_b) && m8(p.qs_t) && m8(p.qs_h) &&
+           m8(p.ks_b) && m8(p.ks_t) && m8(p.ks_h) && m8(p.os_b) && m8(p.os_t) && m8(p.os_h);
+}
+
+cudaError_t launch_sparse_mma_prefill(const Params &p, const void *Q, const void *K, const void *V, const int32_t *idx,
+                                      const float *sink, void *O, float *LSE, cudaStream_t st)
+{
+    cudaError_t e = set_attrs();
+    if (e != cudaSuccess) return e;
+    const int64_t items = (int64_t)p.B * p.Hkv * p.Lq;
+    const unsigned blocks = (unsigned)((items + WARPS - 1) / WARPS);
+    k_sparse_prefill<<<blocks, WARPS * 32, WARPS * kWarpSmem, st>>>(
+        p, (const __nv_bfloat16 *)Q, (const __nv_bfloat16 *)K, (const __nv_bfloat16 *)V, idx, sink, (__nv_bfloat16 *)O, LSE);
+    return cudaGetLastError();
+}
+
+size_t sparse_mma_decode_ws_bytes(const Params &p)
+{
+    const size_t items = (size_t)p.B * p.Hkv * kMaxSplits;
+    return ws_tickets_bytes(p) + items * 16 * sizeof(float) + items * 8 * 32 * sizeof(float4);
+}
+
+cudaError_t launch_sparse_mma_decode(const Params &p, const void *Q, const void *K, const void *V, const int32_t *idx,
+                                     const float *sink, void *O, float *LSE, void *ws, size_t ws_bytes, cudaStream_t st)
+{
+    cudaError_t e = set_attrs();
+    if (e != cudaSuccess) return e;
+    int sms = 0;
+    if ((e = sm_count(&sms)) != cudaSuccess) return e;
+    const int bg = p.B * p.Hkv;
+    const int n_tiles = (p.k + p.w + KT - 1) / KT;
+    // as many splits as fill every warp slot of the GPU once, each split at least two tiles long
+    int n_splits = (sms * WARPS) / bg;
+    n_splits = n_splits < 1 ? 1 : (n_splits > kMaxSplits ? kMaxSplits : n_splits);
+    if (n_splits > (n_tiles + 1) / 2) n_splits = (n_tiles + 1) / 2 > 0 ? (n_tiles + 1) / 2 : 1;
+    const int tiles_per_split = (n_tiles + n_splits - 1) / n_splits;
+    n_splits = (n_tiles + tiles_per_split - 1) / tiles_per_split;
+    if (n_splits <= 1)
+        return launch_sparse_mma_prefill(p, Q, K, V, idx, sink, O, LSE, st);
+    DecodeWs w;
+    char *base = (char *)ws;
+    const size_t items = (size_t)bg * kMaxSplits;
+    w.tickets = (int *)base;
+    w.ml = (float *)(base + ws_tickets_bytes(p));
+    w.opart = (float4 *)(base + ws_tickets_bytes(p) + items * 16 * sizeof(float));
+    (void)ws_bytes;
+    if ((e = cudaMemsetAsync(w.tickets, 0, (size_t)bg * sizeof(int), st)) != cudaSuccess) return e;
+    const int64_t n_items = (int64_t)bg * n_splits;
+    const unsigned blocks = (unsigned)((n_items + WARPS - 1) / WARPS);
+    k_sparse_decode<<<blocks, WARPS * 32, WARPS * kWarpSmem, st>>>(
+        p, (const __nv_bfloat16 *)Q, (const __nv_bfloat16 *)K, (const __nv_bfloat16 *)V, idx, sink, (__nv_bfloat16 *)O, LSE,
+        w, n_splits, tiles_per_split);
+    return cudaGetLastError();
+}
+
+}  // namespace hs2
