@@ -143,6 +143,9 @@ const char *hs2_status_string(hs2_status s);
 /* The cudaError_t (as int) behind the calling thread's most recent HS2_ERR_CUDA, 0 if none. */
 int hs2_last_cuda_error(void);
 
+/* Number of kernels this library has launched in the process so far (all threads, all streams). */
+unsigned long long hs2_launch_count(void);
+
 #ifdef __cplusplus
 }
 #endif

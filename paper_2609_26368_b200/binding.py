@@ -21,7 +21,7 @@ HS2_F32, HS2_BF16 = 0, 1
 HS2_OP_FULL_ATTN_SELECT, HS2_OP_TOPK_SELECT, HS2_OP_SPARSE_ATTN_PREFILL, HS2_OP_SPARSE_ATTN_DECODE = range(4)
 
 EXPORTS = ["hs2_workspace_bytes", "hs2_full_attn_select", "hs2_topk_select", "hs2_sparse_attn_prefill",
-           "hs2_sparse_attn_decode", "hs2_status_string", "hs2_last_cuda_error"]
+           "hs2_sparse_attn_decode", "hs2_status_string", "hs2_last_cuda_error", "hs2_launch_count"]
 
 
 class HS2Error(RuntimeError):
@@ -57,6 +57,7 @@ def load_library():
         lib.hs2_status_string.restype = C.c_char_p
         lib.hs2_status_string.argtypes = [C.c_int]
         lib.hs2_last_cuda_error.restype = C.c_int
+        lib.hs2_launch_count.restype = C.c_ulonglong
         vp, sz = C.c_void_p, C.c_size_t
         pp = C.POINTER(_CProblem)
         lib.hs2_full_attn_select.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
@@ -67,6 +68,11 @@ def load_library():
             getattr(lib, f).restype = C.c_int
         _lib = lib
     return _lib
+
+
+def hs2_launch_count() -> int:
+    """Kernels launched by the library in this process so far."""
+    return int(load_library().hs2_launch_count())
 
 
 def hs2_status_string(status: int) -> str:

@@ -46,7 +46,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
             raise RuntimeError("nvcc failed on %s" % src)
         objs.append(obj)
     tmp = LIB + ".tmp%d" % os.getpid()
-    subprocess.check_call([nvcc, "-shared", "-o", tmp] + objs + ["-lcudart"])
+    subprocess.check_call([nvcc, "-shared", "-Wno-deprecated-gpu-targets", "-o", tmp] + objs + ["-lcudart"])
     os.replace(tmp, LIB)
     return LIB
 

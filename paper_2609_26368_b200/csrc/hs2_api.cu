@@ -1,9 +1,15 @@
 // C ABI of the hs2 library: argument validation, default resolution, workspace carving, dispatch.
 #include <math.h>
 
+#include <atomic>
+
 #include "hs2_common.cuh"
 
 namespace hs2 {
+
+static std::atomic<unsigned long long> g_launches{0};
+void count_launch(int n) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
+
 namespace {
 
 thread_local int g_last_cuda_error = 0;
@@ -224,5 +230,7 @@ const char *hs2_status_string(hs2_status s)
 }
 
 int hs2_last_cuda_error(void) { return g_last_cuda_error; }
+
+unsigned long long hs2_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 
 }  // extern "C"

@@ -57,6 +57,9 @@ __device__ __forceinline__ float warp_sum(float v)
     return v;
 }
 
+// every kernel launch of the library is counted here (read through hs2_launch_count)
+void count_launch(int n = 1);
+
 // ---- launchers (one per translation unit); each returns the cudaError_t of its launches ----
 
 // Generic SIMT kernels: fp32 arithmetic on fp32 or bf16 tensors, any head_dim <= 256, any group size.

@@ -262,6 +262,7 @@ cudaError_t launch_full_attn_generic(const Params &p, hs2_dtype dt, const void *
     else
         k_full_generic<__nv_bfloat16><<<blocks, kWarpsPerBlock * 32, smem, st>>>(
             p, (const __nv_bfloat16 *)Q, (const __nv_bfloat16 *)K, (const __nv_bfloat16 *)V, (__nv_bfloat16 *)O, LSE);
+    count_launch();
     return cudaGetLastError();
 }
 
@@ -282,6 +283,7 @@ cudaError_t launch_scores_generic(const Params &p, hs2_dtype dt, const void *Q, 
         k_scores_generic<__nv_bfloat16><<<blocks, kWarpsPerBlock * 32, smem, st>>>(
             p, (const __nv_bfloat16 *)Q, (const __nv_bfloat16 *)K, LSE, out, out_stride, row0, n_rows, all_visible);
     }
+    count_launch();
     return cudaGetLastError();
 }
 
@@ -299,6 +301,7 @@ cudaError_t launch_sparse_generic(const Params &p, hs2_dtype dt, const void *Q, 
         k_sparse_generic<__nv_bfloat16><<<blocks, kWarpsPerBlock * 32, smem, st>>>(
             p, (const __nv_bfloat16 *)Q, (const __nv_bfloat16 *)K, (const __nv_bfloat16 *)V, idx, sink,
             (__nv_bfloat16 *)O, LSE);
+    count_launch();
     return cudaGetLastError();
 }
 

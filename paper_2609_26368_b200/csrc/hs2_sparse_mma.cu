@@ -16,14 +16,24 @@
 // un-normalised partial (m, l, O) and the last one to arrive (an atomic ticket, nobody waits) merges.
 #include "hs2_common.cuh"
 
+// Tuning knobs (compile time): key rows per stage, pipeline depth, warps per CTA; prefill and decode.
 #ifndef HS2_SP_KT
 #define HS2_SP_KT 16
 #endif
 #ifndef HS2_SP_NSTAGE
-#define HS2_SP_NSTAGE 4
+#define HS2_SP_NSTAGE 2
 #endif
 #ifndef HS2_SP_WARPS
-#define HS2_SP_WARPS 6
+#define HS2_SP_WARPS 12
+#endif
+#ifndef HS2_SPD_KT
+#define HS2_SPD_KT 16
+#endif
+#ifndef HS2_SPD_NSTAGE
+#define HS2_SPD_NSTAGE 2
+#endif
+#ifndef HS2_SPD_WARPS
+#define HS2_SPD_WARPS 6
 #endif
 
 namespace hs2 {
@@ -31,13 +41,19 @@ namespace {
 
 constexpr int HD = 128;                      // head_dim
 constexpr int kRowBytes = HD * 2;            // one K or V row
-constexpr int KT = HS2_SP_KT;                // key rows per pipeline stage (16 or 32)
-constexpr int NSTAGE = HS2_SP_NSTAGE;
-constexpr int WARPS = HS2_SP_WARPS;
-constexpr int kStageBytes = 2 * KT * kRowBytes;           // K tile then V tile
-constexpr int kWarpSmem = NSTAGE * kStageBytes + NSTAGE * 32 * 4;   // + per-stage key index of each row
-constexpr int kMaxSplits = 32;
-static_assert(KT == 16 || KT == 32, "a stage holds 16 or 32 key rows");
+constexpr int kMaxSplits = 32;               // warp-level splits of one (sequence, KV head) in decode
+
+// KT key rows per pipeline stage (16 or 32), NSTAGE stages per warp, WARPS warps per CTA
+template <int KT_, int NSTAGE_, int WARPS_>
+struct Cfg {
+    static constexpr int KT = KT_, NSTAGE = NSTAGE_, WARPS = WARPS_;
+    static constexpr int kStageBytes = 2 * KT * kRowBytes;                       // K tile then V tile
+    static constexpr int kWarpSmem = NSTAGE * kStageBytes + NSTAGE * 32 * 4;     // + key index of each staged row
+    static_assert(KT == 16 || KT == 32, "a stage holds 16 or 32 key rows");
+    static_assert(NSTAGE >= 2, "double buffering at least");
+};
+using PrefillCfg = Cfg<HS2_SP_KT, HS2_SP_NSTAGE, HS2_SP_WARPS>;
+using DecodeCfg = Cfg<HS2_SPD_KT, HS2_SPD_NSTAGE, HS2_SPD_WARPS>;
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, int src_bytes)
@@ -91,6 +107,7 @@ struct Item {
 };
 
 // key index held by slot s of the virtual slot array [idx row | window], -1 when the slot is void
+template <int KT>
 __device__ __forceinline__ int slot_key(const Params &p, const Item &it, int tile, int lane)
 {
     const int s = tile * KT + lane;
@@ -107,6 +124,7 @@ __device__ __forceinline__ int slot_key(const Params &p, const Item &it, int til
     return j;   // negative entries stay negative
 }
 
+template <int KT>
 __device__ __forceinline__ void issue_stage(const Item &it, uint32_t stage_base, int j, int lane)
 {
     const int c = lane & 15;
@@ -122,6 +140,7 @@ __device__ __forceinline__ void issue_stage(const Item &it, uint32_t stage_base,
     }
 }
 
+template <int KT>
 __device__ __forceinline__ void consume_stage(Acc &acc, const uint32_t (&qf)[16], uint32_t stage_base, unsigned mask,
                                               float scale_log2, int lane)
 {
@@ -129,17 +148,22 @@ __device__ __forceinline__ void consume_stage(Acc &acc, const uint32_t (&qf)[16]
     const int mi = lane >> 3, rr = lane & 7;
     constexpr int MT = KT / 16;
     float s[MT][4];
-    // S^T = K Q^T : rows = keys, columns = heads
+    // S^T = K Q^T : rows = keys, columns = heads.  Two accumulator chains per tile keep the tensor pipe busy.
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt) {
+        float s2[4] = {0.f, 0.f, 0.f, 0.f};
         s[mt][0] = s[mt][1] = s[mt][2] = s[mt][3] = 0.f;
         const uint32_t rowaddr = stage_base + (mt * 16 + (mi & 1) * 8 + rr) * kRowBytes;
 #pragma unroll
-        for (int ks = 0; ks < 8; ++ks) {
-            uint32_t a[4];
+        for (int ks = 0; ks < 8; ks += 2) {
+            uint32_t a[4], a2[4];
             ldmatrix_x4(a, rowaddr + (((2 * ks + (mi >> 1)) ^ rr) << 4));
+            ldmatrix_x4(a2, rowaddr + (((2 * ks + 2 + (mi >> 1)) ^ rr) << 4));
             mma_bf16(s[mt], a, qf[2 * ks], qf[2 * ks + 1]);
+            mma_bf16(s2, a2, qf[2 * ks + 2], qf[2 * ks + 3]);
         }
+#pragma unroll
+        for (int e = 0; e < 4; ++e) s[mt][e] += s2[e];
     }
     // online softmax, base-2 domain; this thread: heads 2t+hh, keys 16 mt + g + 8 r
     float mx[2] = {-INFINITY, -INFINITY};
@@ -179,10 +203,12 @@ __device__ __forceinline__ void consume_stage(Acc &acc, const uint32_t (&qf)[16]
         pb[mt][0] = movmatrix_trans(pack_bf16(pv[0], pv[1]));   // keys 16 mt + 0..7
         pb[mt][1] = movmatrix_trans(pack_bf16(pv[2], pv[3]));   // keys 16 mt + 8..15
     }
+    if (__any_sync(0xffffffffu, corr[0] != 1.f || corr[1] != 1.f)) {   // the running max moved for some head
 #pragma unroll
-    for (int dt = 0; dt < 8; ++dt) {
-        acc.o[dt][0] *= corr[0]; acc.o[dt][1] *= corr[1];
-        acc.o[dt][2] *= corr[0]; acc.o[dt][3] *= corr[1];
+        for (int dt = 0; dt < 8; ++dt) {
+            acc.o[dt][0] *= corr[0]; acc.o[dt][1] *= corr[1];
+            acc.o[dt][2] *= corr[0]; acc.o[dt][3] *= corr[1];
+        }
     }
     // O^T += V^T P^T : rows = output dimensions, contraction over the keys of the stage
     const uint32_t vbase = stage_base + KT * kRowBytes;
@@ -199,21 +225,23 @@ __device__ __forceinline__ void consume_stage(Acc &acc, const uint32_t (&qf)[16]
 }
 
 // Fold slot tiles [t_begin, t_end) of one item into acc with an NSTAGE-deep cp.async pipeline.
+template <class C>
 __device__ __forceinline__ void run_tiles(const Params &p, const Item &it, const uint32_t (&qf)[16], Acc &acc,
                                           int t_begin, int t_end, char *wsm, int lane)
 {
+    constexpr int KT = C::KT, NSTAGE = C::NSTAGE, kStageBytes = C::kStageBytes;
     const uint32_t sbase = smem_u32(wsm);
     int *sj = reinterpret_cast<int *>(wsm + NSTAGE * kStageBytes);
     int next = t_begin;
-    int jn = next < t_end ? slot_key(p, it, next, lane) : -1;
+    int jn = next < t_end ? slot_key<KT>(p, it, next, lane) : -1;
     auto try_issue = [&](int stage) -> bool {
         while (next < t_end) {
             const int j = jn;
             ++next;
-            if (next < t_end) jn = slot_key(p, it, next, lane);
+            if (next < t_end) jn = slot_key<KT>(p, it, next, lane);
             if (__ballot_sync(0xffffffffu, j >= 0)) {
                 sj[stage * 32 + lane] = j;
-                issue_stage(it, sbase + stage * kStageBytes, j, lane);
+                issue_stage<KT>(it, sbase + stage * kStageBytes, j, lane);
                 return true;
             }
         }
@@ -232,7 +260,7 @@ __device__ __forceinline__ void run_tiles(const Params &p, const Item &it, const
         cp_async_commit();
         const int stage = n_done % NSTAGE;
         const unsigned mask = __ballot_sync(0xffffffffu, sj[stage * 32 + lane] >= 0);
-        consume_stage(acc, qf, sbase + stage * kStageBytes, mask, p.scale_log2, lane);
+        consume_stage<KT>(acc, qf, sbase + stage * kStageBytes, mask, p.scale_log2, lane);
         ++n_done;
     }
     cp_async_wait<0>();
@@ -335,61 +363,130 @@ __device__ __forceinline__ Item make_item(const Params &p, const __nv_bfloat16 *
 }
 
 // ---------------------------------------------------------------- prefill: one warp per (b, g, i)
-__global__ void __launch_bounds__(WARPS * 32)
+template <class C>
+__global__ void __launch_bounds__(C::WARPS * 32)
 k_sparse_prefill(const Params p, const __nv_bfloat16 *__restrict__ Q, const __nv_bfloat16 *__restrict__ K,
                  const __nv_bfloat16 *__restrict__ V, const int32_t *__restrict__ idx, const float *__restrict__ sink,
                  __nv_bfloat16 *__restrict__ O, float *__restrict__ LSE)
 {
     extern __shared__ __align__(128) char smem[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int64_t item = (int64_t)blockIdx.x * WARPS + warp;   // (b, g, i), i fastest
+    const int64_t item = (int64_t)blockIdx.x * C::WARPS + warp;   // (b, g, i), i fastest
     if (item >= (int64_t)p.B * p.Hkv * p.Lq) return;
     const int i = (int)(item % p.Lq);
     const int gkv = (int)((item / p.Lq) % p.Hkv);
     const int b = (int)(item / ((int64_t)p.Lq * p.Hkv));
-    char *wsm = smem + warp * kWarpSmem;
+    char *wsm = smem + warp * C::kWarpSmem;
     const Item it = make_item(p, K, V, idx, b, gkv, i);
     uint32_t qf[16];
     load_q_frags(p, Q, b, i, gkv, lane, qf);
     Acc acc;
     init_acc(acc, p, sink, gkv, lane, true);
-    const int n_tiles = (p.k + p.w + KT - 1) / KT;
-    run_tiles(p, it, qf, acc, 0, n_tiles, wsm, lane);
+    const int n_tiles = (p.k + p.w + C::KT - 1) / C::KT;
+    run_tiles<C>(p, it, qf, acc, 0, n_tiles, wsm, lane);
     reduce_l(acc);
     store_output(p, acc, O, LSE, b, i, gkv, wsm, lane);
 }
 
-// ---------------------------------------------------------------- decode: one warp per (b, g, split)
+// ---------------------------------------------------------------- decode
+// (a) enough (sequence, KV head) pairs to fill the GPU: one CTA per pair, its warps are the splits,
+//     merged through shared memory.  No scratch, no atomics.
+template <class C>
+__global__ void __launch_bounds__(C::WARPS * 32)
+k_sparse_decode_cta(const Params p, const __nv_bfloat16 *__restrict__ Q, const __nv_bfloat16 *__restrict__ K,
+                    const __nv_bfloat16 *__restrict__ V, const int32_t *__restrict__ idx,
+                    const float *__restrict__ sink, __nv_bfloat16 *__restrict__ O, float *__restrict__ LSE)
+{
+    extern __shared__ __align__(128) char smem[];
+    constexpr int W = C::WARPS;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int bg = blockIdx.x;
+    const int gkv = bg % p.Hkv, b = bg / p.Hkv;
+    const int g = lane >> 2, t = lane & 3;
+    char *wsm = smem + warp * C::kWarpSmem;
+    float *sml = reinterpret_cast<float *>(smem + W * C::kWarpSmem);   // [W][16]: m then l per head
+    const Item it = make_item(p, K, V, idx, b, gkv, 0);
+    uint32_t qf[16];
+    load_q_frags(p, Q, b, 0, gkv, lane, qf);
+    Acc acc;
+    init_acc(acc, p, sink, gkv, lane, warp == 0);   // the sink joins the denominator once
+    const int n_tiles = (p.k + p.w + C::KT - 1) / C::KT;
+    const int per = (n_tiles + W - 1) / W;
+    run_tiles<C>(p, it, qf, acc, warp * per, min(n_tiles, (warp + 1) * per), wsm, lane);
+    reduce_l(acc);
+    float4 *op = reinterpret_cast<float4 *>(wsm);   // the warp's own staging area: [8][32] float4
+#pragma unroll
+    for (int dt = 0; dt < 8; ++dt) op[dt * 32 + lane] = make_float4(acc.o[dt][0], acc.o[dt][1], acc.o[dt][2], acc.o[dt][3]);
+    if (g == 0) {
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) { sml[warp * 16 + 2 * t + hh] = acc.m[hh]; sml[warp * 16 + 8 + 2 * t + hh] = acc.l[hh]; }
+    }
+    __syncthreads();
+    if (warp != 0) return;
+    Acc tot;
+    float wgt[W][2];
+    tot.m[0] = tot.m[1] = -INFINITY;
+#pragma unroll
+    for (int s = 0; s < W; ++s)
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) tot.m[hh] = fmaxf(tot.m[hh], sml[s * 16 + 2 * t + hh]);
+    tot.l[0] = tot.l[1] = 0.f;
+#pragma unroll
+    for (int s = 0; s < W; ++s)
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {
+            const float ms = sml[s * 16 + 2 * t + hh];
+            wgt[s][hh] = ms == -INFINITY ? 0.f : exp2f(ms - tot.m[hh]);
+            tot.l[hh] += wgt[s][hh] * sml[s * 16 + 8 + 2 * t + hh];
+        }
+#pragma unroll
+    for (int dt = 0; dt < 8; ++dt) {
+        float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int s = 0; s < W; ++s) {
+            const float4 v = reinterpret_cast<const float4 *>(smem + s * C::kWarpSmem)[dt * 32 + lane];
+            a.x += wgt[s][0] * v.x; a.y += wgt[s][1] * v.y; a.z += wgt[s][0] * v.z; a.w += wgt[s][1] * v.w;
+        }
+        tot.o[dt][0] = a.x; tot.o[dt][1] = a.y; tot.o[dt][2] = a.z; tot.o[dt][3] = a.w;
+    }
+    __syncwarp();
+    // the output staging must not overlap partials: it goes behind the per-warp areas
+    store_output(p, tot, O, LSE, b, 0, gkv, smem + W * C::kWarpSmem + W * 16 * 4, lane);
+}
+
+// (b) few pairs: one warp per (pair, split); every warp publishes an un-normalised partial to global
+//     scratch and the last one to arrive at the pair's ticket merges.  Nobody waits for anybody.
 struct DecodeWs {
     int *tickets;     // [B * Hkv]
     float *ml;        // [items][2][8]   m then l per head
     float4 *opart;    // [items][8][32]  o[dt] of every lane
 };
 
-__global__ void __launch_bounds__(WARPS * 32)
-k_sparse_decode(const Params p, const __nv_bfloat16 *__restrict__ Q, const __nv_bfloat16 *__restrict__ K,
-                const __nv_bfloat16 *__restrict__ V, const int32_t *__restrict__ idx, const float *__restrict__ sink,
-                __nv_bfloat16 *__restrict__ O, float *__restrict__ LSE, DecodeWs ws, int n_splits, int tiles_per_split)
+template <class C>
+__global__ void __launch_bounds__(C::WARPS * 32)
+k_sparse_decode_split(const Params p, const __nv_bfloat16 *__restrict__ Q, const __nv_bfloat16 *__restrict__ K,
+                      const __nv_bfloat16 *__restrict__ V, const int32_t *__restrict__ idx,
+                      const float *__restrict__ sink, __nv_bfloat16 *__restrict__ O, float *__restrict__ LSE,
+                      DecodeWs ws, int n_splits, int tiles_per_split)
 {
     extern __shared__ __align__(128) char smem[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int64_t item = (int64_t)blockIdx.x * WARPS + warp;   // (b, g, split), split fastest
+    const int64_t item = (int64_t)blockIdx.x * C::WARPS + warp;   // (b, g, split), split fastest
     if (item >= (int64_t)p.B * p.Hkv * n_splits) return;
     const int split = (int)(item % n_splits);
     const int bg = (int)(item / n_splits);
     const int gkv = bg % p.Hkv, b = bg / p.Hkv;
     const int g = lane >> 2, t = lane & 3;
-    char *wsm = smem + warp * kWarpSmem;
+    char *wsm = smem + warp * C::kWarpSmem;
     const Item it = make_item(p, K, V, idx, b, gkv, 0);
     uint32_t qf[16];
     load_q_frags(p, Q, b, 0, gkv, lane, qf);
     Acc acc;
-    init_acc(acc, p, sink, gkv, lane, split == 0);   // the sink joins the denominator once
-    const int n_tiles = (p.k + p.w + KT - 1) / KT;
+    init_acc(acc, p, sink, gkv, lane, split == 0);
+    const int n_tiles = (p.k + p.w + C::KT - 1) / C::KT;
     const int t0 = split * tiles_per_split;
-    run_tiles(p, it, qf, acc, t0, min(n_tiles, t0 + tiles_per_split), wsm, lane);
+    run_tiles<C>(p, it, qf, acc, t0, min(n_tiles, t0 + tiles_per_split), wsm, lane);
     reduce_l(acc);
-    // publish the un-normalised partial
     float4 *op = ws.opart + item * 8 * 32;
 #pragma unroll
     for (int dt = 0; dt < 8; ++dt) op[dt * 32 + lane] = make_float4(acc.o[dt][0], acc.o[dt][1], acc.o[dt][2], acc.o[dt][3]);
@@ -403,28 +500,26 @@ k_sparse_decode(const Params p, const __nv_bfloat16 *__restrict__ Q, const __nv_
     int ticket = 0;
     if (lane == 0) ticket = atomicAdd(ws.tickets + bg, 1);
     ticket = __shfl_sync(0xffffffffu, ticket, 0);
-    if (ticket != n_splits - 1) return;   // someone else finishes later and merges
+    if (ticket != n_splits - 1) return;   // a later arrival merges
     __threadfence();
-    // merge the partials of all splits of this (sequence, KV head)
     const int64_t first = (int64_t)bg * n_splits;
-    float M[2] = {-INFINITY, -INFINITY};
+    Acc tot;
+    tot.m[0] = tot.m[1] = -INFINITY;
     for (int s = 0; s < n_splits; ++s) {
         const float *ml = ws.ml + (first + s) * 16;
 #pragma unroll
-        for (int hh = 0; hh < 2; ++hh) M[hh] = fmaxf(M[hh], __ldcg(ml + 2 * t + hh));
+        for (int hh = 0; hh < 2; ++hh) tot.m[hh] = fmaxf(tot.m[hh], __ldcg(ml + 2 * t + hh));
     }
-    Acc tot;
 #pragma unroll
     for (int dt = 0; dt < 8; ++dt) tot.o[dt][0] = tot.o[dt][1] = tot.o[dt][2] = tot.o[dt][3] = 0.f;
     tot.l[0] = tot.l[1] = 0.f;
-    tot.m[0] = M[0]; tot.m[1] = M[1];
     for (int s = 0; s < n_splits; ++s) {
         const float *ml = ws.ml + (first + s) * 16;
         float wgt[2];
 #pragma unroll
         for (int hh = 0; hh < 2; ++hh) {
             const float ms = __ldcg(ml + 2 * t + hh);
-            wgt[hh] = ms == -INFINITY ? 0.f : exp2f(ms - M[hh]);
+            wgt[hh] = ms == -INFINITY ? 0.f : exp2f(ms - tot.m[hh]);
             tot.l[hh] += wgt[hh] * __ldcg(ml + 8 + 2 * t + hh);
         }
         const float4 *ops = ws.opart + (first + s) * 8 * 32;
@@ -439,6 +534,8 @@ k_sparse_decode(const Params p, const __nv_bfloat16 *__restrict__ Q, const __nv_
 }
 
 size_t ws_tickets_bytes(const Params &p) { return ((size_t)p.B * p.Hkv * sizeof(int) + 255) / 256 * 256; }
+
+constexpr int kDecodeCtaSmem = DecodeCfg::WARPS * DecodeCfg::kWarpSmem + DecodeCfg::WARPS * 16 * 4 + 8 * (HD + 8) * 2;
 
 int g_sm_count = 0;
 cudaError_t sm_count(int *n)
@@ -459,9 +556,13 @@ bool g_attr_set = false;
 cudaError_t set_attrs()
 {
     if (g_attr_set) return cudaSuccess;
-    cudaError_t e = cudaFuncSetAttribute(k_sparse_prefill, cudaFuncAttributeMaxDynamicSharedMemorySize, WARPS * kWarpSmem);
+    cudaError_t e = cudaFuncSetAttribute(k_sparse_prefill<PrefillCfg>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                         PrefillCfg::WARPS * PrefillCfg::kWarpSmem);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(k_sparse_decode, cudaFuncAttributeMaxDynamicSharedMemorySize, WARPS * kWarpSmem);
+    e = cudaFuncSetAttribute(k_sparse_decode_split<DecodeCfg>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             DecodeCfg::WARPS * DecodeCfg::kWarpSmem);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(k_sparse_decode_cta<DecodeCfg>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecodeCtaSmem);
     if (e != cudaSuccess) return e;
     g_attr_set = true;
     return cudaSuccess;
@@ -479,12 +580,14 @@ bool sparse_mma_supported(const Params &p, hs2_dtype dt)
 cudaError_t launch_sparse_mma_prefill(const Params &p, const void *Q, const void *K, const void *V, const int32_t *idx,
                                       const float *sink, void *O, float *LSE, cudaStream_t st)
 {
+    using C = PrefillCfg;
     cudaError_t e = set_attrs();
     if (e != cudaSuccess) return e;
     const int64_t items = (int64_t)p.B * p.Hkv * p.Lq;
-    const unsigned blocks = (unsigned)((items + WARPS - 1) / WARPS);
-    k_sparse_prefill<<<blocks, WARPS * 32, WARPS * kWarpSmem, st>>>(
+    const unsigned blocks = (unsigned)((items + C::WARPS - 1) / C::WARPS);
+    k_sparse_prefill<C><<<blocks, C::WARPS * 32, C::WARPS * C::kWarpSmem, st>>>(
         p, (const __nv_bfloat16 *)Q, (const __nv_bfloat16 *)K, (const __nv_bfloat16 *)V, idx, sink, (__nv_bfloat16 *)O, LSE);
+    count_launch();
     return cudaGetLastError();
 }
 
@@ -497,20 +600,34 @@ size_t sparse_mma_decode_ws_bytes(const Params &p)
 cudaError_t launch_sparse_mma_decode(const Params &p, const void *Q, const void *K, const void *V, const int32_t *idx,
                                      const float *sink, void *O, float *LSE, void *ws, size_t ws_bytes, cudaStream_t st)
 {
+    using C = DecodeCfg;
     cudaError_t e = set_attrs();
     if (e != cudaSuccess) return e;
     int sms = 0;
     if ((e = sm_count(&sms)) != cudaSuccess) return e;
     const int bg = p.B * p.Hkv;
-    const int n_tiles = (p.k + p.w + KT - 1) / KT;
+    const int n_tiles = (p.k + p.w + C::KT - 1) / C::KT;
+    const __nv_bfloat16 *q = (const __nv_bfloat16 *)Q, *k = (const __nv_bfloat16 *)K, *v = (const __nv_bfloat16 *)V;
+    bool cta_path = bg >= sms && n_tiles >= 2 * C::WARPS;
+#ifdef HS2_SP_SPLITS
+    cta_path = false;   // tuning builds only
+#endif
+    if (cta_path) {
+        k_sparse_decode_cta<C><<<bg, C::WARPS * 32, kDecodeCtaSmem, st>>>(p, q, k, v, idx, sink, (__nv_bfloat16 *)O, LSE);
+        count_launch();
+    return cudaGetLastError();
+    }
     // as many splits as fill every warp slot of the GPU once, each split at least two tiles long
-    int n_splits = (sms * WARPS) / bg;
+    const int ctas_per_sm = (227 * 1024) / (C::WARPS * C::kWarpSmem) > 0 ? (227 * 1024) / (C::WARPS * C::kWarpSmem) : 1;
+    int n_splits = (sms * ctas_per_sm * C::WARPS) / bg;
+#ifdef HS2_SP_SPLITS
+    n_splits = HS2_SP_SPLITS;
+#endif
     n_splits = n_splits < 1 ? 1 : (n_splits > kMaxSplits ? kMaxSplits : n_splits);
     if (n_splits > (n_tiles + 1) / 2) n_splits = (n_tiles + 1) / 2 > 0 ? (n_tiles + 1) / 2 : 1;
     const int tiles_per_split = (n_tiles + n_splits - 1) / n_splits;
     n_splits = (n_tiles + tiles_per_split - 1) / tiles_per_split;
-    if (n_splits <= 1)
-        return launch_sparse_mma_prefill(p, Q, K, V, idx, sink, O, LSE, st);
+    if (n_splits <= 1) return launch_sparse_mma_prefill(p, Q, K, V, idx, sink, O, LSE, st);
     DecodeWs w;
     char *base = (char *)ws;
     const size_t items = (size_t)bg * kMaxSplits;
@@ -520,10 +637,10 @@ cudaError_t launch_sparse_mma_decode(const Params &p, const void *Q, const void 
     (void)ws_bytes;
     if ((e = cudaMemsetAsync(w.tickets, 0, (size_t)bg * sizeof(int), st)) != cudaSuccess) return e;
     const int64_t n_items = (int64_t)bg * n_splits;
-    const unsigned blocks = (unsigned)((n_items + WARPS - 1) / WARPS);
-    k_sparse_decode<<<blocks, WARPS * 32, WARPS * kWarpSmem, st>>>(
-        p, (const __nv_bfloat16 *)Q, (const __nv_bfloat16 *)K, (const __nv_bfloat16 *)V, idx, sink, (__nv_bfloat16 *)O, LSE,
-        w, n_splits, tiles_per_split);
+    const unsigned blocks = (unsigned)((n_items + C::WARPS - 1) / C::WARPS);
+    k_sparse_decode_split<C><<<blocks, C::WARPS * 32, C::WARPS * C::kWarpSmem, st>>>(
+        p, q, k, v, idx, sink, (__nv_bfloat16 *)O, LSE, w, n_splits, tiles_per_split);
+    count_launch();
     return cudaGetLastError();
 }
 

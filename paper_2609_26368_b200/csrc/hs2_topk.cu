@@ -181,6 +181,7 @@ cudaError_t launch_topk(const Params &p, const float *scores, int64_t score_stri
         k_topk<true><<<(unsigned)n_rows, kThreads, 0, st>>>(p, scores, score_stride, idx, row0);
     else
         k_topk<false><<<(unsigned)n_rows, kThreads, 0, st>>>(p, scores, score_stride, idx, row0);
+    count_launch();
     return cudaGetLastError();
 }
 
