@@ -47,7 +47,8 @@ typedef enum {
     HS2_ERR_INVALID_ARG = 1,         /* NULL where a pointer is required, non-positive size, bad head ratio ... */
     HS2_ERR_UNSUPPORTED = 2,         /* valid problem outside what the kernels cover (e.g. head_dim > 256) */
     HS2_ERR_WORKSPACE_TOO_SMALL = 3, /* ws_bytes < hs2_workspace_bytes() or ws not 256-byte aligned */
-    HS2_ERR_CUDA = 4                 /* a CUDA runtime call failed; see hs2_last_cuda_error() */
+    HS2_ERR_CUDA = 4,                /* a CUDA runtime call failed; see hs2_last_cuda_error() */
+    HS2_ERR_STATIC_SCRATCH = 5       /* the problem needs more scratch than the library's built-in array holds */
 } hs2_status;
 
 typedef enum { HS2_F32 = 0, HS2_BF16 = 1 } hs2_dtype;
@@ -136,6 +137,34 @@ hs2_status hs2_sparse_attn_prefill(const hs2_problem *p, const void *Q, const vo
 hs2_status hs2_sparse_attn_decode(const hs2_problem *p, const void *Q, const void *K, const void *V,
                                   const int32_t *idx, const float *sink, void *O, float *LSE,
                                   void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
+ * hs2_sparse_attn_decode for callers that cannot hand over a scratch buffer.  (The paper has no
+ * counterpart to this call; it is a packaging variant of the decode operator above.)
+ *
+ * Who needs it: code that is not allowed to obtain device memory at the point where it decodes -
+ * a plugin that is given nothing but the tensors' pointers, a server that handed the whole device
+ * to its own pool at start-up and has none left to carve a workspace from, a latency-critical loop
+ * that cannot afford the device-wide synchronisation an allocation implies.  For them the partial
+ * results of the split kernel live in an array that is part of the library image:
+ * 8,519,936 bytes on every GPU that loads the library, held until the process exits.
+ *
+ *   - Same arguments and results as hs2_sparse_attn_decode, minus `ws`.  The call allocates nothing
+ *     and frees nothing, on the host or on the device.
+ *   - Limit: batch * n_kv_heads <= HS2_STATIC_DECODE_MAX_PAIRS (64); a larger problem returns
+ *     HS2_ERR_STATIC_SCRATCH and launches nothing.  It covers what the tensor-core decode kernel
+ *     covers (bf16, head_dim 128, group <= 8, 16-byte aligned tensors); anything else returns
+ *     HS2_ERR_UNSUPPORTED.
+ *   - The first call on each device looks up the array's device address; make that first call
+ *     outside any stream capture.
+ *   - All calls on a device share the one array, which still holds the previous call's data: the
+ *     call clears the part that must start at zero itself, and two calls whose kernels can overlap
+ *     on the GPU (different streams, no ordering between them) race on it.  Order them.
+ */
+#define HS2_STATIC_DECODE_MAX_PAIRS 64
+hs2_status hs2_sparse_attn_decode_static(const hs2_problem *p, const void *Q, const void *K, const void *V,
+                                         const int32_t *idx, const float *sink, void *O, float *LSE,
+                                         void *cuda_stream);
 
 /* Static, never-NULL description of a status. */
 const char *hs2_status_string(hs2_status s);

@@ -16,12 +16,15 @@ import torch
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _LIB_PATH = os.path.join(_HERE, "libhs2.so")
 
-HS2_OK, HS2_ERR_INVALID_ARG, HS2_ERR_UNSUPPORTED, HS2_ERR_WORKSPACE_TOO_SMALL, HS2_ERR_CUDA = range(5)
+HS2_OK, HS2_ERR_INVALID_ARG, HS2_ERR_UNSUPPORTED, HS2_ERR_WORKSPACE_TOO_SMALL, HS2_ERR_CUDA, \
+    HS2_ERR_STATIC_SCRATCH = range(6)
+HS2_STATIC_DECODE_MAX_PAIRS = 64
 HS2_F32, HS2_BF16 = 0, 1
 HS2_OP_FULL_ATTN_SELECT, HS2_OP_TOPK_SELECT, HS2_OP_SPARSE_ATTN_PREFILL, HS2_OP_SPARSE_ATTN_DECODE = range(4)
 
 EXPORTS = ["hs2_workspace_bytes", "hs2_full_attn_select", "hs2_topk_select", "hs2_sparse_attn_prefill",
-           "hs2_sparse_attn_decode", "hs2_status_string", "hs2_last_cuda_error", "hs2_launch_count"]
+           "hs2_sparse_attn_decode", "hs2_sparse_attn_decode_static", "hs2_status_string", "hs2_last_cuda_error",
+           "hs2_launch_count"]
 
 
 class HS2Error(RuntimeError):
@@ -64,7 +67,9 @@ def load_library():
         lib.hs2_topk_select.argtypes = [pp, vp, vp, vp, sz, vp]
         lib.hs2_sparse_attn_prefill.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         lib.hs2_sparse_attn_decode.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
-        for f in ("hs2_full_attn_select", "hs2_topk_select", "hs2_sparse_attn_prefill", "hs2_sparse_attn_decode"):
+        lib.hs2_sparse_attn_decode_static.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp]
+        for f in ("hs2_full_attn_select", "hs2_topk_select", "hs2_sparse_attn_prefill", "hs2_sparse_attn_decode",
+                  "hs2_sparse_attn_decode_static"):
             getattr(lib, f).restype = C.c_int
         _lib = lib
     return _lib
@@ -222,3 +227,20 @@ def hs2_sparse_attn_decode(prob: Problem, q, k, v, idx, *, sink=None, out=None, 
     """SA layer, decode (q_len == 1, split over the attended set); returns ``(O, LSE | None)``."""
     return _sparse("hs2_sparse_attn_decode", HS2_OP_SPARSE_ATTN_DECODE, prob, q, k, v, idx, sink, out, lse,
                    want_lse, ws, stream)
+
+
+def hs2_sparse_attn_decode_static(prob: Problem, q, k, v, idx, *, sink=None, out, lse=None, stream=None):
+    """Decode for callers that may not allocate: the split kernel's partials live in a fixed
+    8.5 MB array inside the library, so no workspace is passed and nothing is allocated - here
+    included, which is why ``out`` (and ``lse``, if wanted) must be given.  Limit:
+    ``batch * n_kv_heads <= 64``.  Calls on one device share that array: keep them ordered on the GPU.
+    """
+    _check_inputs(prob, q, k, v)
+    assert out is not None and out.is_cuda and out.shape == q.shape and out.dtype == q.dtype
+    if idx is not None:
+        assert idx.dtype == torch.int32 and idx.is_contiguous() and idx.is_cuda
+    c = prob.c_struct(q, k, out)
+    st = load_library().hs2_sparse_attn_decode_static(C.byref(c), _dp(q), _dp(k), _dp(v), _dp(idx), _dp(sink),
+                                                      _dp(out), _dp(lse), _stream(stream))
+    _check(st, "hs2_sparse_attn_decode_static")
+    return out, lse

@@ -217,6 +217,21 @@ hs2_status hs2_sparse_attn_decode(const hs2_problem *hp, const void *Q, const vo
     return e == cudaSuccess ? HS2_OK : cuda_fail(e);
 }
 
+hs2_status hs2_sparse_attn_decode_static(const hs2_problem *hp, const void *Q, const void *K, const void *V,
+                                         const int32_t *idx, const float *sink, void *O, float *LSE,
+                                         void *cuda_stream)
+{
+    Params p;
+    hs2_status s = sparse_common(hp, Q, K, V, idx, O, &p);
+    if (s != HS2_OK) return s;
+    if (p.Lq != 1) return HS2_ERR_INVALID_ARG;
+    if (!(sparse_mma_supported(p, hp->dtype) && aligned16(Q, K, V, O))) return HS2_ERR_UNSUPPORTED;
+    if (!sparse_mma_decode_static_fits(p)) return HS2_ERR_STATIC_SCRATCH;
+    if ((s = check_device()) != HS2_OK) return s;
+    cudaError_t e = launch_sparse_mma_decode_static(p, Q, K, V, idx, sink, O, LSE, (cudaStream_t)cuda_stream);
+    return e == cudaSuccess ? HS2_OK : cuda_fail(e);
+}
+
 const char *hs2_status_string(hs2_status s)
 {
     switch (s) {
@@ -225,6 +240,7 @@ const char *hs2_status_string(hs2_status s)
         case HS2_ERR_UNSUPPORTED: return "unsupported problem";
         case HS2_ERR_WORKSPACE_TOO_SMALL: return "workspace too small or misaligned";
         case HS2_ERR_CUDA: return "CUDA runtime error";
+        case HS2_ERR_STATIC_SCRATCH: return "problem needs more scratch than the library's built-in array holds";
     }
     return "unknown status";
 }

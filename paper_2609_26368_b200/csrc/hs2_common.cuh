@@ -86,6 +86,12 @@ cudaError_t launch_sparse_mma_decode(const Params &p, const void *Q, const void 
                                      const float *sink, void *O, float *LSE, void *ws, size_t ws_bytes,
                                      cudaStream_t st);
 
+// Decode with the partials in a static device array of the library (no caller scratch).
+constexpr int kStaticDecodeMaxPairs = HS2_STATIC_DECODE_MAX_PAIRS;
+bool sparse_mma_decode_static_fits(const Params &p);
+cudaError_t launch_sparse_mma_decode_static(const Params &p, const void *Q, const void *K, const void *V,
+                                            const int32_t *idx, const float *sink, void *O, float *LSE, cudaStream_t st);
+
 bool full_mma_supported(const Params &p, hs2_dtype dt);
 cudaError_t launch_full_attn_mma(const Params &p, const void *Q, const void *K, const void *V, void *O, float *LSE,
                                  cudaStream_t st);

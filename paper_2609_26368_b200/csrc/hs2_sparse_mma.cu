@@ -14,6 +14,8 @@
 //   * online softmax in the base-2 domain with warp shuffles across the 8 key rows of a fragment.
 // Decode splits the attended set of one (sequence, KV head) over several warps; each writes an
 // un-normalised partial (m, l, O) and the last one to arrive (an atomic ticket, nobody waits) merges.
+#include <mutex>
+
 #include "hs2_common.cuh"
 
 // Tuning knobs (compile time): key rows per stage, pipeline depth, warps per CTA; prefill and decode.
@@ -640,6 +642,83 @@ cudaError_t launch_sparse_mma_decode(const Params &p, const void *Q, const void 
     const unsigned blocks = (unsigned)((n_items + C::WARPS - 1) / C::WARPS);
     k_sparse_decode_split<C><<<blocks, C::WARPS * 32, C::WARPS * C::kWarpSmem, st>>>(
         p, q, k, v, idx, sink, (__nv_bfloat16 *)O, LSE, w, n_splits, tiles_per_split);
+    count_launch();
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------- decode without caller scratch
+// The split kernel above, with its partials and tickets in a fixed array that lives in the library
+// image instead of a caller buffer.  Every device that loads the library carries the array until the
+// process exits; all calls on a device share it.
+namespace {
+
+constexpr size_t kStaticTicketBytes = 256;
+constexpr size_t kStaticItems = (size_t)kStaticDecodeMaxPairs * kMaxSplits;
+constexpr size_t kStaticMlBytes = kStaticItems * 16 * sizeof(float);
+constexpr size_t kStaticOpartBytes = kStaticItems * 8 * 32 * sizeof(float4);
+constexpr size_t kStaticScratchBytes = kStaticTicketBytes + kStaticMlBytes + kStaticOpartBytes;   // 8,519,936 bytes
+static_assert(kStaticDecodeMaxPairs * sizeof(int) <= kStaticTicketBytes, "tickets fit their slot");
+
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+void *g_static_scratch_addr[kMaxDevices] = {};   // device address of the array, per device ordinal
+std::mutex g_static_mu;
+
+// In host code `g_static_scratch` is only a handle; the address a kernel may use has to be asked
+// for, once per device and with that device current.
+cudaError_t static_scratch_address(void **out)
+{
+    int dev = -1;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    std::lock_guard<std::mutex> lock(g_static_mu);
+    if (!g_static_scratch_addr[dev]) {
+        void *ptr = nullptr;
+        e = cudaGetSymbolAddress((void **)&ptr, g_static_scratch);
+        if (e != cudaSuccess) return e;
+        if (!ptr) return cudaErrorInvalidSymbol;
+        g_static_scratch_addr[dev] = ptr;
+    }
+    *out = g_static_scratch_addr[dev];
+    return cudaSuccess;
+}
+
+}  // namespace
+
+bool sparse_mma_decode_static_fits(const Params &p) { return (int64_t)p.B * p.Hkv <= kStaticDecodeMaxPairs; }
+
+cudaError_t launch_sparse_mma_decode_static(const Params &p, const void *Q, const void *K, const void *V,
+                                            const int32_t *idx, const float *sink, void *O, float *LSE, cudaStream_t st)
+{
+    using C = DecodeCfg;
+    cudaError_t e = set_attrs();
+    if (e != cudaSuccess) return e;
+    int sms = 0;
+    if ((e = sm_count(&sms)) != cudaSuccess) return e;
+    void *scratch = nullptr;
+    if ((e = static_scratch_address(&scratch)) != cudaSuccess) return e;
+    const int bg = p.B * p.Hkv;
+    const int n_tiles = (p.k + p.w + C::KT - 1) / C::KT;
+    const int ctas_per_sm = (227 * 1024) / (C::WARPS * C::kWarpSmem) > 0 ? (227 * 1024) / (C::WARPS * C::kWarpSmem) : 1;
+    int n_splits = (sms * ctas_per_sm * C::WARPS) / bg;
+    n_splits = n_splits < 1 ? 1 : (n_splits > kMaxSplits ? kMaxSplits : n_splits);
+    if (n_splits > (n_tiles + 1) / 2) n_splits = (n_tiles + 1) / 2 > 0 ? (n_tiles + 1) / 2 : 1;
+    const int tiles_per_split = (n_tiles + n_splits - 1) / n_splits;
+    n_splits = (n_tiles + tiles_per_split - 1) / tiles_per_split;
+    DecodeWs w;
+    char *base = (char *)scratch;
+    w.tickets = (int *)base;
+    w.ml = (float *)(base + kStaticTicketBytes);
+    w.opart = (float4 *)(base + kStaticTicketBytes + kStaticMlBytes);
+    // the array keeps whatever the previous call left: the tickets must start at zero
+    if ((e = cudaMemsetAsync(w.tickets, 0, (size_t)bg * sizeof(int), st)) != cudaSuccess) return e;
+    const int64_t n_items = (int64_t)bg * n_splits;
+    const unsigned blocks = (unsigned)((n_items + C::WARPS - 1) / C::WARPS);
+    k_sparse_decode_split<C><<<blocks, C::WARPS * 32, C::WARPS * C::kWarpSmem, st>>>(
+        p, (const __nv_bfloat16 *)Q, (const __nv_bfloat16 *)K, (const __nv_bfloat16 *)V, idx, sink, (__nv_bfloat16 *)O, LSE,
+        w, n_splits, tiles_per_split);
     count_launch();
     return cudaGetLastError();
 }

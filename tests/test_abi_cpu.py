@@ -30,8 +30,8 @@ def test_every_declared_symbol_is_exported(lib):
 
 
 def test_status_strings(lib):
-    texts = [hs2.hs2_status_string(s) for s in range(5)]
-    assert texts[0] == "ok" and len(set(texts)) == 5
+    texts = [hs2.hs2_status_string(s) for s in range(6)]
+    assert texts[0] == "ok" and len(set(texts)) == 6
     assert hs2.hs2_status_string(99) == "unknown status"
 
 
