@@ -251,7 +251,7 @@ def time_steps(block, steps, warmup, world, timing=True, before=None, after=None
 
 # ------------------------------------------------------------------ decode at 64K context (cfg5)
 
-def bench_decode_64k(device, peaks, reps=5, burst=40):
+def bench_decode_64k(device, peaks, reps=5, burst=40, ctx=65536):
     """Split-KV sparse decode on the 64K-context configuration; indices from the full layer's scores.
 
     The cache (8.6 GB) is far above L2; consecutive launches rotate over four query/index sets so
@@ -259,7 +259,8 @@ def bench_decode_64k(device, peaks, reps=5, burst=40):
     """
     import paper_2609_26368_b200 as hs2
     from paper_2609_26368_b200 import binding
-    wl = CONFIGS["cfg5"]
+    from dataclasses import replace
+    wl = replace(CONFIGS["cfg5"], kv_len=ctx)
     inp = make_inputs(wl, device)
     k, v = inp.k, inp.v
     B, _, Hq, D = inp.q_full.shape
@@ -296,11 +297,11 @@ def bench_decode_64k(device, peaks, reps=5, burst=40):
     us = statistics.median(per) * 1e3
     gb = gathered_kv_bytes(wl)
     ach = gb / (us * 1e-6) / 1e9
-    return {"workload": "cfg5: B=64, ctx 65536, 32q/4kv, D=128, bf16, k=2048, w=128",
+    return {"workload": "cfg5: B=64, ctx %d, 32q/4kv, D=128, bf16, k=2048, w=128" % ctx,
             "sparse_decode_us_per_step": round(us, 2), "gathered_kv_bytes": gb,
             "achieved_gbs": round(ach, 1), "peak_gbs": peaks["hbm_gbs"], "frac": round(ach / peaks["hbm_gbs"], 4),
             "full_attn_select_decode_ms": round(min(t_full[1:]), 3), "launches_back_to_back": burst,
-            "l2": "8.6 GB cache, 4 rotating query/index sets (1.1 GB of gathered rows) > L2"}
+            "l2": "%.1f GB cache, 4 rotating query/index sets (1.1 GB of gathered rows) > L2" % (2 * k.numel() * 2 / 1e9)}
 
 
 # ------------------------------------------------------------------ CPU oracle legs
@@ -372,7 +373,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2", choices=sorted(CONFIGS))
     ap.add_argument("--cpu-rows", type=int, default=64, help="query rows of the CPU-oracle sample")
-    ap.add_argument("--skip", default="", help="comma list of: decode64k, e2e, cpu")
+    ap.add_argument("--skip", default="", help="comma list of: block, decode64k, e2e, cpu")
+    ap.add_argument("--decode-ctx", type=int, default=65536, help="context length of the decode section (profiling: 8192)")
     args = ap.parse_args()
     wl = CONFIGS[args.workload]
     skip = set(s for s in args.skip.split(",") if s)
@@ -388,6 +390,9 @@ def main():
     peaks = measured_peaks()
     warmup = max(args.warmup, 3)
 
+    if "block" in skip:      # decode-section only (used for profiling captures)
+        print(json.dumps({"decode_64k": bench_decode_64k(device, peaks, ctx=args.decode_ctx)}))
+        return
     block = Block(wl, device, rank)
     tokens_per_step = wl.batch * wl.q_len
 
@@ -460,7 +465,7 @@ def main():
     if "decode64k" not in skip and world == 1:
         del block
         torch.cuda.empty_cache()
-        line["decode_64k"] = bench_decode_64k(device, peaks)
+        line["decode_64k"] = bench_decode_64k(device, peaks, ctx=args.decode_ctx)
     if "cpu" not in skip and world == 1:
         cb, _, _ = cpu_baseline(wl, args.cpu_rows)
         line["cpu_baseline"] = cb

@@ -115,7 +115,16 @@ size_t hs2_workspace_bytes(const hs2_problem *hp, hs2_op op)
     switch (op) {
         case HS2_OP_FULL_ATTN_SELECT:
             if (resolve(hp, true, &p) != HS2_OK) return 0;
-            return p.k > 0 ? full_select_ws_bytes(p) : 0;
+            {
+                size_t need = p.k > 0 ? full_select_ws_bytes(p) : 0;
+                if (p.Lq == 1 && sparse_mma_supported(p, hp->dtype)) {   // the decode-shaped layer may split over the keys
+                    Params pd = p;
+                    pd.k = 0; pd.w = p.Lk;
+                    const size_t dec = sparse_mma_decode_ws_bytes(pd);
+                    if (dec > need) need = dec;
+                }
+                return need;
+            }
         case HS2_OP_TOPK_SELECT:
         case HS2_OP_SPARSE_ATTN_PREFILL:
             return 0;
@@ -143,7 +152,17 @@ hs2_status hs2_full_attn_select(const hs2_problem *hp, const void *Q, const void
     cudaStream_t st = (cudaStream_t)cuda_stream;
     const hs2_dtype dt = hp->dtype;
     const bool mma = full_mma_supported(p, dt) && aligned16(Q, K, V, O);
-    cudaError_t e = mma ? launch_full_attn_mma(p, Q, K, V, O, LSE, st) : launch_full_attn_generic(p, dt, Q, K, V, O, LSE, st);
+    cudaError_t e;
+    // One query per sequence: the layer is a memory-bound sweep over the whole cache.  That is the
+    // sparse decode kernel with an empty index list and a window that covers the context.
+    bool as_decode = p.Lq == 1 && sparse_mma_supported(p, dt) && aligned16(Q, K, V, O);
+    Params pd = p;
+    pd.k = 0; pd.w = p.Lk;
+    if (as_decode && !ws_ok(ws, ws_bytes, sparse_mma_decode_ws_bytes(pd))) as_decode = false;
+    if (as_decode)
+        e = launch_sparse_mma_decode(pd, Q, K, V, nullptr, nullptr, O, LSE, ws, ws_bytes, st);
+    else
+        e = mma ? launch_full_attn_mma(p, Q, K, V, O, LSE, st) : launch_full_attn_generic(p, dt, Q, K, V, O, LSE, st);
     if (e != cudaSuccess) return cuda_fail(e);
     if (!want_sel && !scores_dbg) return HS2_OK;
 

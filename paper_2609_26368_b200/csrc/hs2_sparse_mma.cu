@@ -554,19 +554,23 @@ cudaError_t sm_count(int *n)
     return cudaSuccess;
 }
 
-bool g_attr_set = false;
+// the opt-in to large dynamic shared memory is a per-device attribute of each kernel
+bool g_attr_set[64] = {};
 cudaError_t set_attrs()
 {
-    if (g_attr_set) return cudaSuccess;
-    cudaError_t e = cudaFuncSetAttribute(k_sparse_prefill<PrefillCfg>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                         PrefillCfg::WARPS * PrefillCfg::kWarpSmem);
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64 && g_attr_set[dev]) return cudaSuccess;
+    e = cudaFuncSetAttribute(k_sparse_prefill<PrefillCfg>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             PrefillCfg::WARPS * PrefillCfg::kWarpSmem);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(k_sparse_decode_split<DecodeCfg>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              DecodeCfg::WARPS * DecodeCfg::kWarpSmem);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(k_sparse_decode_cta<DecodeCfg>, cudaFuncAttributeMaxDynamicSharedMemorySize, kDecodeCtaSmem);
     if (e != cudaSuccess) return e;
-    g_attr_set = true;
+    if (dev >= 0 && dev < 64) g_attr_set[dev] = true;
     return cudaSuccess;
 }
 
