@@ -215,12 +215,9 @@ def barrier(world):
 
 
 def max_over_ranks(x: float, world, device):
-    if world == 1:
-        return x
-    import torch.distributed as dist
-    t = torch.tensor([x], dtype=torch.float64, device=device)
-    dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    return float(t.item())
+    """Slowest rank's device time (the data path itself has no collective)."""
+    from paper_2609_26368_b200.replicas import aggregate_throughput
+    return aggregate_throughput(0.0, x, device)[2]
 
 
 def time_steps(block, steps, warmup, world, timing=True, before=None, after=None):
