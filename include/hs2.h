@@ -172,6 +172,11 @@ const char *hs2_status_string(hs2_status s);
 /* The cudaError_t (as int) behind the calling thread's most recent HS2_ERR_CUDA, 0 if none. */
 int hs2_last_cuda_error(void);
 
+/* Reads the library's device error word into *flags (0 = fine; bit 0: a bounded wait inside a kernel
+ * ran out and that kernel abandoned its work; bit 1: a kernel refused a misaligned shared-memory
+ * window).  Sticky until the process exits.  Synchronises the current device.  Returns an hs2_status. */
+int hs2_device_error_flags(unsigned *flags);
+
 /* Number of kernels this library has launched in the process so far (all threads, all streams). */
 unsigned long long hs2_launch_count(void);
 

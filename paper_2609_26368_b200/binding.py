@@ -24,7 +24,7 @@ HS2_OP_FULL_ATTN_SELECT, HS2_OP_TOPK_SELECT, HS2_OP_SPARSE_ATTN_PREFILL, HS2_OP_
 
 EXPORTS = ["hs2_workspace_bytes", "hs2_full_attn_select", "hs2_topk_select", "hs2_sparse_attn_prefill",
            "hs2_sparse_attn_decode", "hs2_sparse_attn_decode_static", "hs2_status_string", "hs2_last_cuda_error",
-           "hs2_launch_count"]
+           "hs2_launch_count", "hs2_device_error_flags"]
 
 
 class HS2Error(RuntimeError):
@@ -73,6 +73,13 @@ def load_library():
             getattr(lib, f).restype = C.c_int
         _lib = lib
     return _lib
+
+
+def hs2_device_error_flags() -> int:
+    """Device error word of the library (0 = fine); synchronises the device."""
+    v = C.c_uint(0)
+    _check(load_library().hs2_device_error_flags(C.byref(v)), "hs2_device_error_flags")
+    return int(v.value)
 
 
 def hs2_launch_count() -> int:

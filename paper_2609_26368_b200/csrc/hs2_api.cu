@@ -161,8 +161,14 @@ hs2_status hs2_full_attn_select(const hs2_problem *hp, const void *Q, const void
     if (as_decode && !ws_ok(ws, ws_bytes, sparse_mma_decode_ws_bytes(pd))) as_decode = false;
     if (as_decode)
         e = launch_sparse_mma_decode(pd, Q, K, V, nullptr, nullptr, O, LSE, ws, ws_bytes, st);
-    else
-        e = mma ? launch_full_attn_mma(p, Q, K, V, O, LSE, st) : launch_full_attn_generic(p, dt, Q, K, V, O, LSE, st);
+    else {
+        e = cudaErrorNotSupported;
+#ifndef HS2_NO_TC5
+        if (full_tc5_supported(p, dt) && aligned16(Q, K, V, O)) e = launch_full_attn_tc5(p, Q, K, V, O, LSE, st);
+#endif
+        if (e == cudaErrorNotSupported)
+            e = mma ? launch_full_attn_mma(p, Q, K, V, O, LSE, st) : launch_full_attn_generic(p, dt, Q, K, V, O, LSE, st);
+    }
     if (e != cudaSuccess) return cuda_fail(e);
     if (!want_sel && !scores_dbg) return HS2_OK;
 
@@ -265,6 +271,13 @@ const char *hs2_status_string(hs2_status s)
 }
 
 int hs2_last_cuda_error(void) { return g_last_cuda_error; }
+
+int hs2_device_error_flags(unsigned *flags)
+{
+    if (!flags) return HS2_ERR_INVALID_ARG;
+    cudaError_t e = read_tc5_error(flags);
+    return e == cudaSuccess ? HS2_OK : cuda_fail(e);
+}
 
 unsigned long long hs2_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }
 

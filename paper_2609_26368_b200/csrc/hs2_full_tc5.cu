@@ -1,0 +1,444 @@
+// Full causal attention on the 5th-generation tensor cores (tcgen05 + TMEM), bf16, head_dim 128
+// (Section 3.4: the full-attention layer; NoPE, Section 4.1).
+//
+// One CTA = 128 queries of one head (MMA M = 128), 192 threads, two CTAs per SM so that one CTA's
+// softmax overlaps the other's tensor work:
+//   warp 4   TMA producer: Q once, then K/V tiles of 64 keys into a 2-stage ring.  Every tile is a
+//            pair of 128-byte-swizzled halves ([rows][64 dims]), the canonical UMMA operand layout.
+//   warp 5   MMA issuer: S = Q K^T (M128 N64 K128, eight tcgen05.mma of K=16) into one of two S
+//            buffers in TMEM, and O += P V (M128 N128 K64, V as an MN-major B operand) into TMEM.
+//   warps 0-3 one thread per query row: tcgen05.ld of the S row, causal mask, online softmax in the
+//            base-2 domain with a lazily updated row maximum (O in TMEM is rescaled only when the
+//            maximum grows by more than 2^8), P written as bf16 into swizzled shared memory.
+// TMEM: columns 0-63 / 64-127 the two S buffers, 128-255 the O accumulator (fp32, lane = query row).
+// Every mbarrier wait is bounded; a wait that runs out sets a bit in a device error word, makes the
+// CTA abandon its loops, and the CTA still frees its TMEM before it returns.
+#include <cuda.h>
+
+#include "hs2_common.cuh"
+
+namespace hs2 {
+
+__device__ unsigned g_tc5_error;   // bit 0: an mbarrier wait ran out; bit 1: shared-memory base not alignable
+
+namespace {
+
+constexpr int BM = 128, BN = 64, HD = 128;
+constexpr int kThreads = 192;
+constexpr uint32_t kQBytes = 2 * BM * 128;        // two 64-dim halves
+constexpr uint32_t kKVStage = 2 * BN * 128;       // one K (or V) tile: two halves
+constexpr uint32_t kOffQ = 0;
+constexpr uint32_t kOffK = kOffQ + kQBytes;       // 2 stages
+constexpr uint32_t kOffV = kOffK + 2 * kKVStage;  // 2 stages
+constexpr uint32_t kOffP = kOffV + 2 * kKVStage;  // 128 rows x 64 keys bf16, K-major
+constexpr uint32_t kOffBar = kOffP + BM * 128;
+constexpr uint32_t kBarBytes = 128;
+constexpr uint32_t kAlignSlack = 896;             // the dynamic window is at least 128-byte aligned
+constexpr uint32_t kSmemBytes = kOffBar + kBarBytes + kAlignSlack;   // 115712 = (228 KB - 2 KB) / 2
+constexpr uint32_t kTmemCols = 256;
+constexpr uint32_t kSpinLimit = 1u << 22;
+constexpr float kRescaleThreshold = 8.f;          // log2 units
+
+enum Bar { Q_FULL = 0, KV_FULL0, KV_FULL1, KV_EMPTY0, KV_EMPTY1, S_FULL0, S_FULL1, S_FREE0, S_FREE1, P_FULL, PV_DONE, N_BARS };
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ bool elect_one()
+{
+    uint32_t pred;
+    asm volatile("{\n .reg .b32 rx;\n .reg .pred px;\n elect.sync rx|px, 0xffffffff;\n selp.b32 %0, 1, 0, px;\n}\n" : "=r"(pred));
+    return pred != 0;
+}
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];\n" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.b32 %0, 1, 0, p;\n}\n"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait: gives up after kSpinLimit polls (or when another thread of the CTA already gave up).
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag)
+{
+    for (uint32_t it = 0; it < kSpinLimit; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 255u) == 255u && *abort_flag) return false;
+    }
+    atomicOr(&g_tc5_error, 1u);
+    *abort_flag = 1;
+    return false;
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;\n" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;\n" ::: "memory"); }
+
+__device__ __forceinline__ void tma_load_4d(uint32_t dst, const CUtensorMap *tm, uint32_t bar, int c0, int c1, int c2, int c3)
+{
+    asm volatile("cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];\n"
+                 ::"r"(dst), "l"(tm), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3) : "memory");
+}
+
+// shared-memory matrix descriptor, 128-byte swizzle, version 1 (Blackwell)
+__device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes, uint32_t sbo_bytes)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((addr >> 4) & 0x3fffu);
+    d |= (uint64_t)((lbo_bytes >> 4) & 0x3fffu) << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3fffu) << 32;
+    d |= (uint64_t)1 << 46;    // descriptor version
+    d |= (uint64_t)2 << 61;    // SWIZZLE_128B
+    return d;
+}
+// instruction descriptor, kind::f16: bf16 x bf16 -> fp32, A K-major, B K-major (0) or MN-major (1)
+__host__ __device__ constexpr uint32_t idesc(int M, int N, int b_mn_major)
+{
+    return (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)b_mn_major << 16) | ((uint32_t)(N >> 3) << 17) | ((uint32_t)(M >> 4) << 24);
+}
+__device__ __forceinline__ void umma(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t id, uint32_t accumulate)
+{
+    asm volatile("{\n .reg .pred p;\n setp.ne.b32 p, %4, 0;\n tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}\n"
+                 ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(id), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];\n" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, float (&v)[32])
+{
+    uint32_t *r = reinterpret_cast<uint32_t *>(v);
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+                 "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];\n"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+                   "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+                   "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+                   "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+                 : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_st32(uint32_t taddr, const float (&v)[32])
+{
+    const uint32_t *r = reinterpret_cast<const uint32_t *>(v);
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,"
+                 "%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};\n"
+                 ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+                   "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+                   "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+                   "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+                 : "memory");
+}
+__device__ __forceinline__ void tmem_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;\n" ::: "memory"); }
+__device__ __forceinline__ void tmem_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;\n" ::: "memory"); }
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
+{
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t *>(&v);
+}
+
+__global__ void __launch_bounds__(kThreads, 2)
+k_full_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
+           const __grid_constant__ CUtensorMap tmV, const Params p, __nv_bfloat16 *__restrict__ O,
+           float *__restrict__ LSE)
+{
+    extern __shared__ char smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t pad = (1024u - (raw & 1023u)) & 1023u;
+    if (pad > kAlignSlack) {   // never seen; refuse rather than run on a misaligned tile
+        if (threadIdx.x == 0) atomicOr(&g_tc5_error, 2u);
+        return;
+    }
+    char *smem = smem_raw + pad;
+    const uint32_t sbase = raw + pad;
+    const uint32_t bars = sbase + kOffBar;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + kOffBar + N_BARS * 8);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + kOffBar + N_BARS * 8 + 4);
+    auto bar = [&](int i) { return bars + 8u * i; };
+
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int mblk = gridDim.x - 1 - blockIdx.x;   // long rows first
+    const int h = blockIdx.y % p.Hq, b = blockIdx.y / p.Hq;
+    const int gkv = h / p.G;
+    const int i0 = mblk * BM;
+    const int kvl = kvlen_of(p, b);
+    const int pos0 = pos_of(p, b, i0);
+    const int rows_here = min(BM, p.Lq - i0);
+    const int n_vis = max(0, min(pos0 + rows_here, kvl));
+    const int nblk = (n_vis + BN - 1) / BN;
+
+    if (tid == 0) {
+        *abort_flag = 0;
+        mbar_init(bar(Q_FULL), 1);
+        mbar_init(bar(KV_FULL0), 1); mbar_init(bar(KV_FULL1), 1);
+        mbar_init(bar(KV_EMPTY0), 1); mbar_init(bar(KV_EMPTY1), 1);
+        mbar_init(bar(S_FULL0), 1); mbar_init(bar(S_FULL1), 1);
+        mbar_init(bar(S_FREE0), 128); mbar_init(bar(S_FREE1), 128);
+        mbar_init(bar(P_FULL), 128);
+        mbar_init(bar(PV_DONE), 1);
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+    }
+    if (warp == 5) {   // TMEM allocation is a warp-wide operation
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp == 4) {
+        // ------------------------------------------------ TMA producer
+        if (elect_one() && nblk > 0) {
+            mbar_expect_tx(bar(Q_FULL), kQBytes);
+            tma_load_4d(sbase + kOffQ, &tmQ, bar(Q_FULL), 0, h, i0, b);
+            tma_load_4d(sbase + kOffQ + BM * 128, &tmQ, bar(Q_FULL), 64, h, i0, b);
+            int issued = 0;
+            for (int j = 0; j < nblk; ++j) {
+                const int st = j & 1;
+                if (!mbar_wait(bar(KV_EMPTY0 + st), ((j >> 1) & 1) ^ 1, abort_flag)) break;
+                issued = j + 1;
+                mbar_expect_tx(bar(KV_FULL0 + st), 2 * kKVStage);
+                const uint32_t kdst = sbase + kOffK + st * kKVStage, vdst = sbase + kOffV + st * kKVStage;
+                tma_load_4d(kdst, &tmK, bar(KV_FULL0 + st), 0, gkv, j * BN, b);
+                tma_load_4d(kdst + BN * 128, &tmK, bar(KV_FULL0 + st), 64, gkv, j * BN, b);
+                tma_load_4d(vdst, &tmV, bar(KV_FULL0 + st), 0, gkv, j * BN, b);
+                tma_load_4d(vdst + BN * 128, &tmV, bar(KV_FULL0 + st), 64, gkv, j * BN, b);
+            }
+            if (*abort_flag) {   // leaving early: let the copies already in flight land before the CTA goes away
+                for (int j = max(0, issued - 2); j < issued; ++j)
+                    for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait(bar(KV_FULL0 + (j & 1)), (j >> 1) & 1); ++it) {}
+                for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait(bar(Q_FULL), 0); ++it) {}
+            }
+        }
+    } else if (warp == 5) {
+        // ------------------------------------------------ MMA issuer
+        if (elect_one() && nblk > 0) {
+            constexpr uint32_t idS = idesc(BM, BN, 0), idPV = idesc(BM, HD, 1);
+            bool ok = mbar_wait(bar(Q_FULL), 0, abort_flag);
+            auto issue_s = [&](int j) -> bool {
+                const int st = j & 1, ph = (j >> 1) & 1;
+                if (!mbar_wait(bar(KV_FULL0 + st), ph, abort_flag)) return false;
+                if (!mbar_wait(bar(S_FREE0 + st), ph ^ 1, abort_flag)) return false;
+                tc_fence_after();
+                const uint32_t qa = sbase + kOffQ, ka = sbase + kOffK + st * kKVStage;
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    const uint32_t off = (ks & 3) * 32;   // 16 dims = 32 bytes inside the swizzled 128-byte row
+                    const uint64_t da = smem_desc(qa + (ks >> 2) * (BM * 128) + off, 16, 1024);
+                    const uint64_t db = smem_desc(ka + (ks >> 2) * (BN * 128) + off, 16, 1024);
+                    umma(tmem + st * BN, da, db, idS, ks > 0);
+                }
+                umma_commit(bar(S_FULL0 + st));
+                return true;
+            };
+            ok = ok && issue_s(0);
+            for (int j = 0; ok && j < nblk; ++j) {
+                if (j + 1 < nblk && !issue_s(j + 1)) break;
+                if (!mbar_wait(bar(P_FULL), j & 1, abort_flag)) break;
+                tc_fence_after();
+                const int st = j & 1;
+                const uint32_t pa = sbase + kOffP, va = sbase + kOffV + st * kKVStage;
+#pragma unroll
+                for (int kk = 0; kk < 4; ++kk) {   // 16 keys per instruction
+                    const uint64_t da = smem_desc(pa + kk * 32, 16, 1024);
+                    // V: MN-major, 64-dim halves BN*128 bytes apart (leading offset), 8-key groups 1024 bytes apart
+                    const uint64_t db = smem_desc(va + kk * 2048, BN * 128, 1024);
+                    umma(tmem + 2 * BN, da, db, idPV, (j > 0 || kk > 0) ? 1u : 0u);
+                }
+                umma_commit(bar(KV_EMPTY0 + st));
+                umma_commit(bar(PV_DONE));
+            }
+        }
+    } else {
+        // ------------------------------------------------ softmax: one thread per query row
+        const int row = tid;                       // 0..127, TMEM lane
+        const int i = i0 + row;
+        const int prow = pos0 + row;
+        const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
+        float m_used = -INFINITY, l = 0.f;
+        bool alive = true;
+        for (int j = 0; j < nblk && alive; ++j) {
+            const int sb = j & 1;
+            if (!__all_sync(0xffffffffu, mbar_wait(bar(S_FULL0 + sb), (j >> 1) & 1, abort_flag))) { alive = false; break; }
+            tc_fence_after();
+            float s[64];
+            {
+                float lo[32], hi[32];
+                tmem_ld32(lane_base + sb * BN, lo);
+                tmem_ld32(lane_base + sb * BN + 32, hi);
+                tmem_wait_ld();
+#pragma unroll
+                for (int e = 0; e < 32; ++e) { s[e] = lo[e]; s[32 + e] = hi[e]; }
+            }
+            tc_fence_before();
+            mbar_arrive(bar(S_FREE0 + sb));
+            const int j0 = j * BN;
+            const bool need_mask = (j0 + BN - 1 > pos0) || (j0 + BN > kvl);
+            float m_blk = -INFINITY;
+#pragma unroll
+            for (int e = 0; e < 64; ++e) {
+                float v = s[e] * p.scale_log2;
+                if (need_mask && (j0 + e > prow || j0 + e >= kvl)) v = -INFINITY;
+                s[e] = v;
+                m_blk = fmaxf(m_blk, v);
+            }
+            const bool need = m_blk > m_used + kRescaleThreshold;   // also true for the first finite block
+            const float m_new = need ? m_blk : m_used;
+            const float corr = need ? exp2f(m_used - m_new) : 1.f;  // 0 when nothing was accumulated yet
+            if (j > 0) {
+                if (!__all_sync(0xffffffffu, mbar_wait(bar(PV_DONE), (j - 1) & 1, abort_flag))) { alive = false; break; }
+                tc_fence_after();
+                if (__any_sync(0xffffffffu, need)) {   // rescale the O rows of this warp (a warp-wide TMEM access)
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        float o[32];
+                        tmem_ld32(lane_base + 2 * BN + c * 32, o);
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) o[e] *= corr;
+                        tmem_st32(lane_base + 2 * BN + c * 32, o);
+                    }
+                    tmem_wait_st();
+                }
+            }
+            l *= corr;
+            m_used = m_new;
+            const float muse = m_used == -INFINITY ? 0.f : m_used;
+            uint32_t pk[32];
+#pragma unroll
+            for (int e = 0; e < 64; e += 2) {
+                const float p0 = exp2f(s[e] - muse), p1 = exp2f(s[e + 1] - muse);
+                l += p0 + p1;
+                pk[e >> 1] = pack_bf16(p0, p1);
+            }
+            char *prow_ptr = smem + kOffP + row * 128;
+#pragma unroll
+            for (int c = 0; c < 8; ++c)   // 8 keys = one 16-byte chunk, chunk position XOR (row & 7)
+                *reinterpret_cast<uint4 *>(prow_ptr + ((c ^ (row & 7)) << 4)) = make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
+            fence_proxy_async();
+            tc_fence_before();
+            mbar_arrive(bar(P_FULL));
+        }
+        // ------------------------------------------------ epilogue
+        bool have_o = alive && nblk > 0;
+        if (have_o) have_o = mbar_wait(bar(PV_DONE), (nblk - 1) & 1, abort_flag);
+        have_o = __all_sync(0xffffffffu, have_o);   // TMEM loads below are warp-wide
+        tc_fence_after();
+        const float inv = l > 0.f ? 1.f / l : 0.f;
+        __nv_bfloat16 *orow = O + b * p.os_b + (int64_t)i * p.os_t + h * p.os_h;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            float o[32];
+            if (have_o) {   // uniform across the warp except after an abort
+                tmem_ld32(lane_base + 2 * BN + c * 32, o);
+                tmem_wait_ld();
+            } else {
+#pragma unroll
+                for (int e = 0; e < 32; ++e) o[e] = 0.f;
+            }
+            if (i < p.Lq) {
+#pragma unroll
+                for (int q4 = 0; q4 < 4; ++q4) {
+                    uint4 v;
+                    v.x = pack_bf16(o[8 * q4 + 0] * inv, o[8 * q4 + 1] * inv);
+                    v.y = pack_bf16(o[8 * q4 + 2] * inv, o[8 * q4 + 3] * inv);
+                    v.z = pack_bf16(o[8 * q4 + 4] * inv, o[8 * q4 + 5] * inv);
+                    v.w = pack_bf16(o[8 * q4 + 6] * inv, o[8 * q4 + 7] * inv);
+                    *reinterpret_cast<uint4 *>(orow + c * 32 + q4 * 8) = v;
+                }
+            }
+        }
+        if (i < p.Lq)
+            LSE[((int64_t)b * p.Hq + h) * p.Lq + i] = (have_o && l > 0.f) ? (m_used + log2f(l)) * kLn2 : -INFINITY;
+    }
+    // ------------------------------------------------ teardown: everybody arrives, then TMEM is returned
+    __syncwarp();
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 5) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(kTmemCols) : "memory");
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
+                                  const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode = nullptr;
+bool g_encode_tried = false;
+
+EncodeTiledFn encode_fn()
+{
+    if (!g_encode_tried) {
+        g_encode_tried = true;
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &fn, cudaEnableDefault, &qres) == cudaSuccess &&
+            qres == cudaDriverEntryPointSuccess)
+            g_encode = (EncodeTiledFn)fn;
+        (void)cudaGetLastError();
+    }
+    return g_encode;
+}
+
+// [B, L, H, 128] bf16 with element strides (sb, st, sh): box = 64 dims x `rows` tokens of one head, 128-byte swizzle
+bool make_map(CUtensorMap *tm, const void *base, int B, int L, int H, int64_t sb, int64_t st, int64_t sh, int rows)
+{
+    EncodeTiledFn enc = encode_fn();
+    if (!enc) return false;
+    const cuuint64_t dims[4] = {(cuuint64_t)HD, (cuuint64_t)H, (cuuint64_t)L, (cuuint64_t)B};
+    const cuuint64_t strides[3] = {(cuuint64_t)sh * 2, (cuuint64_t)st * 2, (cuuint64_t)sb * 2};
+    const cuuint32_t box[4] = {64, 1, (cuuint32_t)rows, 1};
+    const cuuint32_t estr[4] = {1, 1, 1, 1};
+    return enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), dims, strides, box, estr,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool g_attr_set[64] = {};
+
+}  // namespace
+
+bool full_tc5_supported(const Params &p, hs2_dtype dt)
+{
+    auto m8 = [](int64_t x) { return x % 8 == 0 && x > 0; };
+    return dt == HS2_BF16 && p.D == HD && m8(p.qs_b) && m8(p.qs_t) && m8(p.qs_h) && m8(p.ks_b) && m8(p.ks_t) &&
+           m8(p.ks_h) && m8(p.os_b) && m8(p.os_t) && m8(p.os_h) && (int64_t)p.B * p.Hq <= 65535 && encode_fn() != nullptr;
+}
+
+// Returns cudaErrorNotSupported when the tensor maps cannot be built (the caller then takes the mma.sync kernel).
+cudaError_t launch_full_attn_tc5(const Params &p, const void *Q, const void *K, const void *V, void *O, float *LSE,
+                                 cudaStream_t st)
+{
+    CUtensorMap tmQ, tmK, tmV;
+    if (!make_map(&tmQ, Q, p.B, p.Lq, p.Hq, p.qs_b, p.qs_t, p.qs_h, BM) ||
+        !make_map(&tmK, K, p.B, p.Lk, p.Hkv, p.ks_b, p.ks_t, p.ks_h, BN) ||
+        !make_map(&tmV, V, p.B, p.Lk, p.Hkv, p.ks_b, p.ks_t, p.ks_h, BN))
+        return cudaErrorNotSupported;
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (!(dev >= 0 && dev < 64 && g_attr_set[dev])) {
+        if ((e = cudaFuncSetAttribute(k_full_tc5, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes)) != cudaSuccess) return e;
+        if (dev >= 0 && dev < 64) g_attr_set[dev] = true;
+    }
+    dim3 grid((p.Lq + BM - 1) / BM, p.B * p.Hq);
+    k_full_tc5<<<grid, kThreads, kSmemBytes, st>>>(tmQ, tmK, tmV, p, (__nv_bfloat16 *)O, LSE);
+    count_launch();
+    return cudaGetLastError();
+}
+
+// Device error word of the tcgen05 kernels (0 = no bounded wait ever ran out).  Synchronises the device.
+cudaError_t read_tc5_error(unsigned *out)
+{
+    return cudaMemcpyFromSymbol(out, g_tc5_error, sizeof(unsigned));
+}
+
+}  // namespace hs2
