@@ -92,6 +92,20 @@ hs2_status check_device()
     return HS2_OK;
 }
 
+// the score sweep: tcgen05 where it applies, else mma.sync, else the generic kernel
+cudaError_t launch_scores(const Params &p, hs2_dtype dt, bool mma, bool aligned, const void *Q, const void *K, const float *LSE,
+                          float *out, int64_t out_stride, int64_t row0, int64_t n_rows, bool all_visible, cudaStream_t st)
+{
+    cudaError_t e = cudaErrorNotSupported;
+#ifndef HS2_NO_TC5
+    if (aligned && scores_tc5_supported(p, dt)) e = launch_scores_tc5(p, Q, K, LSE, out, out_stride, row0, n_rows, all_visible, st);
+#endif
+    if (e == cudaErrorNotSupported)
+        e = mma ? launch_scores_mma(p, Q, K, LSE, out, out_stride, row0, n_rows, all_visible, st)
+                : launch_scores_generic(p, dt, Q, K, LSE, out, out_stride, row0, n_rows, all_visible, st);
+    return e;
+}
+
 hs2_status sparse_common(const hs2_problem *hp, const void *Q, const void *K, const void *V, const int32_t *idx,
                          void *O, Params *p)
 {
@@ -175,8 +189,7 @@ hs2_status hs2_full_attn_select(const hs2_problem *hp, const void *Q, const void
     const int64_t rows = select_rows(p);
     if (scores_dbg) {
         // scores for every visible key go straight to the caller's tensor; the selection reads them from there
-        e = mma ? launch_scores_mma(p, Q, K, LSE, scores_dbg, p.Lk, 0, rows, true, st)
-                : launch_scores_generic(p, dt, Q, K, LSE, scores_dbg, p.Lk, 0, rows, true, st);
+        e = launch_scores(p, dt, mma, aligned16(Q, K, V, O), Q, K, LSE, scores_dbg, p.Lk, 0, rows, true, st);
         if (e != cudaSuccess) return cuda_fail(e);
         if (want_sel && (e = launch_topk(p, scores_dbg, p.Lk, idx, 0, rows, st)) != cudaSuccess) return cuda_fail(e);
         return HS2_OK;
@@ -188,8 +201,7 @@ hs2_status hs2_full_attn_select(const hs2_problem *hp, const void *Q, const void
     float *strip = (float *)ws;
     for (int64_t r0 = 0; r0 < rows; r0 += block) {
         const int64_t n = rows - r0 < block ? rows - r0 : block;
-        e = mma ? launch_scores_mma(p, Q, K, LSE, strip, stride, r0, n, false, st)
-                : launch_scores_generic(p, dt, Q, K, LSE, strip, stride, r0, n, false, st);
+        e = launch_scores(p, dt, mma, aligned16(Q, K, V, O), Q, K, LSE, strip, stride, r0, n, false, st);
         if (e != cudaSuccess) return cuda_fail(e);
         if ((e = launch_topk(p, strip, stride, idx, r0, n, st)) != cudaSuccess) return cuda_fail(e);
     }

@@ -102,6 +102,9 @@ cudaError_t launch_scores_mma(const Params &p, const void *Q, const void *K, con
 bool full_tc5_supported(const Params &p, hs2_dtype dt);
 cudaError_t launch_full_attn_tc5(const Params &p, const void *Q, const void *K, const void *V, void *O, float *LSE,
                                  cudaStream_t st);
+bool scores_tc5_supported(const Params &p, hs2_dtype dt);
+cudaError_t launch_scores_tc5(const Params &p, const void *Q, const void *K, const float *LSE, float *out,
+                              int64_t out_stride, int64_t row0, int64_t n_rows, bool all_visible, cudaStream_t st);
 cudaError_t read_tc5_error(unsigned *out);
 
 }  // namespace hs2

@@ -368,6 +368,184 @@ k_full_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
     }
 }
 
+
+// ---------------------------------------------------------------- selection scores on tcgen05
+// a[i][j] = max over the heads h of the group of (scale <q_h(i), k_j> - LSE_h(i))   (Section 3.4)
+// One CTA = TQ = 128/G consecutive queries of one (sequence, KV head) x one chunk of keys.  The MMA
+// computes S^T = K Q^T: 128 keys on M (TMEM lane = key), the TQ x G (query, head) pairs on N = 128,
+// so the G heads of a query are adjacent TMEM columns of one lane and their maximum is thread local.
+// Warp 4 feeds K tiles by TMA (2-stage ring), warp 5 issues the MMAs into two accumulator buffers,
+// warps 0-3 (thread = key) subtract LSE, take the group maximum and write 32 consecutive keys of a
+// strip row per warp instruction.
+constexpr int SC_KCHUNK = 4096;                   // keys per CTA
+constexpr uint32_t kScOffQ = 0;                   // [2 halves][128 (query, head) rows][128 B]
+constexpr uint32_t kScOffK = 32768;               // 2 stages x [2 halves][128 keys][128 B]
+constexpr uint32_t kScOffNl = kScOffK + 2 * 32768;   // float[128]: -LSE/scale per column
+constexpr uint32_t kScOffNq = kScOffNl + 512;     // int[128]: keys needed per query
+constexpr uint32_t kScOffRow = kScOffNq + 512;    // int64[128]: strip row of each query
+constexpr uint32_t kScOffBar = kScOffRow + 1024;
+constexpr uint32_t kScSmemBytes = kScOffBar + kBarBytes + kAlignSlack;
+enum ScBar { SQ_FULL = 0, SK_FULL0, SK_FULL1, SK_EMPTY0, SK_EMPTY1, ACC_FULL0, ACC_FULL1, ACC_FREE0, ACC_FREE1, SC_N_BARS };
+
+template <int G>
+__global__ void __launch_bounds__(kThreads, 2)
+k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, const Params p,
+             const float *__restrict__ LSE, float *__restrict__ out, int64_t out_stride, int64_t row0, int64_t n_rows,
+             int all_visible, int bg_first, int tiles_per_bg)
+{
+    constexpr int TQ = 128 / G;          // queries per CTA
+    constexpr int QPC = 32 / G > 0 ? 32 / G : 1;   // queries per 32-column chunk (G <= 32)
+    extern __shared__ char smem_raw[];
+    const uint32_t raw = smem_u32(smem_raw);
+    const uint32_t pad = (1024u - (raw & 1023u)) & 1023u;
+    if (pad > kAlignSlack) {
+        if (threadIdx.x == 0) atomicOr(&g_tc5_error, 2u);
+        return;
+    }
+    char *smem = smem_raw + pad;
+    const uint32_t sbase = raw + pad;
+    const uint32_t bars = sbase + kScOffBar;
+    uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + kScOffBar + SC_N_BARS * 8);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + kScOffBar + SC_N_BARS * 8 + 4);
+    auto bar = [&](int i) { return bars + 8u * i; };
+    float *s_nl = reinterpret_cast<float *>(smem + kScOffNl);
+    int *s_nq = reinterpret_cast<int *>(smem + kScOffNq);
+    int64_t *s_row = reinterpret_cast<int64_t *>(smem + kScOffRow);
+
+    const int tid = threadIdx.x, warp = tid >> 5;
+    const int bg = bg_first + blockIdx.y / tiles_per_bg;
+    const int qt = blockIdx.y % tiles_per_bg;
+    const int gkv = bg % p.Hkv, b = bg / p.Hkv;
+    const int kvl = kvlen_of(p, b);
+    const int iq0 = qt * TQ;
+    const int64_t bg_row0 = (int64_t)bg * p.Lq;
+    const int i_lo = (int)max((int64_t)0, row0 - bg_row0), i_hi = (int)min((int64_t)p.Lq, row0 + n_rows - bg_row0);
+    const int c_lo = max(iq0, i_lo), c_hi = min(iq0 + TQ, i_hi);
+    if (c_lo >= c_hi) return;
+    auto n_of = [&](int i) {
+        const int pos = pos_of(p, b, i);
+        return max(0, min(all_visible ? pos + 1 : pos - p.w + 1, kvl));
+    };
+    const int limit = n_of(c_hi - 1);
+    const int key0 = blockIdx.x * SC_KCHUNK;
+    const int key_end = min(limit, key0 + SC_KCHUNK);
+    if (key0 >= key_end) return;
+    const int ntile = (key_end - key0 + 127) / 128;
+
+    if (tid < 128) {   // per-column constants
+        const int t = tid / G, hh = tid % G;
+        const int i = iq0 + t;
+        const bool ok = i >= c_lo && i < c_hi;
+        s_nl[tid] = ok ? -LSE[((int64_t)b * p.Hq + gkv * G + hh) * p.Lq + i] / p.scale : 0.f;
+        if (hh == 0) {
+            s_nq[t] = ok ? n_of(i) : 0;
+            s_row[t] = ok ? (bg_row0 + i - row0) : 0;
+        }
+    }
+    if (tid == 0) {
+        *abort_flag = 0;
+        mbar_init(bar(SQ_FULL), 1);
+        mbar_init(bar(SK_FULL0), 1); mbar_init(bar(SK_FULL1), 1);
+        mbar_init(bar(SK_EMPTY0), 1); mbar_init(bar(SK_EMPTY1), 1);
+        mbar_init(bar(ACC_FULL0), 1); mbar_init(bar(ACC_FULL1), 1);
+        mbar_init(bar(ACC_FREE0), 128); mbar_init(bar(ACC_FREE1), 128);
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+    }
+    if (warp == 5) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = *tmem_slot;
+
+    if (warp == 4) {
+        if (elect_one()) {
+            mbar_expect_tx(bar(SQ_FULL), 32768);
+            tma_load_4d(sbase + kScOffQ, &tmQ, bar(SQ_FULL), 0, gkv * G, iq0, b);
+            tma_load_4d(sbase + kScOffQ + 16384, &tmQ, bar(SQ_FULL), 64, gkv * G, iq0, b);
+            int issued = 0;
+            for (int t = 0; t < ntile; ++t) {
+                const int st = t & 1;
+                if (!mbar_wait(bar(SK_EMPTY0 + st), ((t >> 1) & 1) ^ 1, abort_flag)) break;
+                issued = t + 1;
+                mbar_expect_tx(bar(SK_FULL0 + st), 32768);
+                const uint32_t kdst = sbase + kScOffK + st * 32768;
+                tma_load_4d(kdst, &tmK, bar(SK_FULL0 + st), 0, gkv, key0 + t * 128, b);
+                tma_load_4d(kdst + 16384, &tmK, bar(SK_FULL0 + st), 64, gkv, key0 + t * 128, b);
+            }
+            if (*abort_flag) {
+                for (int t = max(0, issued - 2); t < issued; ++t)
+                    for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait(bar(SK_FULL0 + (t & 1)), (t >> 1) & 1); ++it) {}
+                for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait(bar(SQ_FULL), 0); ++it) {}
+            }
+        }
+    } else if (warp == 5) {
+        if (elect_one()) {
+            constexpr uint32_t id = idesc(128, 128, 0);
+            bool ok = mbar_wait(bar(SQ_FULL), 0, abort_flag);
+            for (int t = 0; ok && t < ntile; ++t) {
+                const int st = t & 1, ph = (t >> 1) & 1;
+                if (!mbar_wait(bar(SK_FULL0 + st), ph, abort_flag)) break;
+                if (!mbar_wait(bar(ACC_FREE0 + st), ph ^ 1, abort_flag)) break;
+                tc_fence_after();
+                const uint32_t ka = sbase + kScOffK + st * 32768, qa = sbase + kScOffQ;
+#pragma unroll
+                for (int ks = 0; ks < 8; ++ks) {
+                    const uint32_t off = (ks >> 2) * 16384 + (ks & 3) * 32;
+                    umma(tmem + st * 128, smem_desc(ka + off, 16, 1024), smem_desc(qa + off, 16, 1024), id, ks > 0);
+                }
+                umma_commit(bar(SK_EMPTY0 + st));
+                umma_commit(bar(ACC_FULL0 + st));
+            }
+        }
+    } else {
+        const int row = tid;   // key inside the tile = TMEM lane
+        const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
+        for (int t = 0; t < ntile; ++t) {
+            const int ab = t & 1;
+            if (!__all_sync(0xffffffffu, mbar_wait(bar(ACC_FULL0 + ab), (t >> 1) & 1, abort_flag))) break;
+            tc_fence_after();
+            const int key = key0 + t * 128 + row;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                float v[32];
+                tmem_ld32(lane_base + ab * 128 + c * 32, v);
+                tmem_wait_ld();
+                const float4 *nl4 = reinterpret_cast<const float4 *>(s_nl + c * 32);
+#pragma unroll
+                for (int e4 = 0; e4 < 8; ++e4) {
+                    const float4 n4 = nl4[e4];
+                    v[4 * e4] += n4.x; v[4 * e4 + 1] += n4.y; v[4 * e4 + 2] += n4.z; v[4 * e4 + 3] += n4.w;
+                }
+#pragma unroll
+                for (int q = 0; q < QPC; ++q) {
+                    float a = v[q * G];
+#pragma unroll
+                    for (int hh = 1; hh < G; ++hh) a = fmaxf(a, v[q * G + hh]);
+                    const int tq = c * QPC + q;
+                    if (key < s_nq[tq]) out[s_row[tq] * out_stride + key] = a * p.scale;
+                }
+            }
+            tc_fence_before();
+            mbar_arrive(bar(ACC_FREE0 + ab));
+        }
+    }
+    __syncwarp();
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 5) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(kTmemCols) : "memory");
+    }
+}
+
+__global__ void k_fill_tc5(float *__restrict__ out, int64_t n, float v)
+{
+    for (int64_t e = (int64_t)blockIdx.x * blockDim.x + threadIdx.x; e < n; e += (int64_t)gridDim.x * blockDim.x) out[e] = v;
+}
+
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *, const cuuint64_t *,
                                   const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave, CUtensorMapSwizzle,
                                   CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
@@ -389,13 +567,14 @@ EncodeTiledFn encode_fn()
 }
 
 // [B, L, H, 128] bf16 with element strides (sb, st, sh): box = 64 dims x `rows` tokens of one head, 128-byte swizzle
-bool make_map(CUtensorMap *tm, const void *base, int B, int L, int H, int64_t sb, int64_t st, int64_t sh, int rows)
+bool make_map(CUtensorMap *tm, const void *base, int B, int L, int H, int64_t sb, int64_t st, int64_t sh, int rows,
+              int box_heads = 1)
 {
     EncodeTiledFn enc = encode_fn();
     if (!enc) return false;
     const cuuint64_t dims[4] = {(cuuint64_t)HD, (cuuint64_t)H, (cuuint64_t)L, (cuuint64_t)B};
     const cuuint64_t strides[3] = {(cuuint64_t)sh * 2, (cuuint64_t)st * 2, (cuuint64_t)sb * 2};
-    const cuuint32_t box[4] = {64, 1, (cuuint32_t)rows, 1};
+    const cuuint32_t box[4] = {64, (cuuint32_t)box_heads, (cuuint32_t)rows, 1};
     const cuuint32_t estr[4] = {1, 1, 1, 1};
     return enc(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(base), dims, strides, box, estr,
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
@@ -433,6 +612,63 @@ cudaError_t launch_full_attn_tc5(const Params &p, const void *Q, const void *K, 
     k_full_tc5<<<grid, kThreads, kSmemBytes, st>>>(tmQ, tmK, tmV, p, (__nv_bfloat16 *)O, LSE);
     count_launch();
     return cudaGetLastError();
+}
+
+template <int G>
+cudaError_t launch_scores_tc5_g(const CUtensorMap &tmQ, const CUtensorMap &tmK, const Params &p, const float *LSE, float *out,
+                                int64_t out_stride, int64_t row0, int64_t n_rows, bool all_visible, cudaStream_t st)
+{
+    static bool attr_set[64] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (!(dev >= 0 && dev < 64 && attr_set[dev])) {
+        if ((e = cudaFuncSetAttribute(k_scores_tc5<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kScSmemBytes)) != cudaSuccess) return e;
+        if (dev >= 0 && dev < 64) attr_set[dev] = true;
+    }
+    constexpr int TQ = 128 / G;
+    const int bg_first = (int)(row0 / p.Lq), bg_last = (int)((row0 + n_rows - 1) / p.Lq);
+    const int tiles_per_bg = (p.Lq + TQ - 1) / TQ;
+    const int64_t gy = (int64_t)(bg_last - bg_first + 1) * tiles_per_bg;
+    if (gy > 65535) return cudaErrorNotSupported;
+    dim3 grid((p.Lk + SC_KCHUNK - 1) / SC_KCHUNK, (unsigned)gy);
+    k_scores_tc5<G><<<grid, kThreads, kScSmemBytes, st>>>(tmQ, tmK, p, LSE, out, out_stride, row0, n_rows, all_visible ? 1 : 0,
+                                                         bg_first, tiles_per_bg);
+    count_launch();
+    return cudaGetLastError();
+}
+
+bool scores_tc5_supported(const Params &p, hs2_dtype dt)
+{
+    const bool g_ok = p.G == 1 || p.G == 2 || p.G == 4 || p.G == 8 || p.G == 16;
+    return g_ok && full_tc5_supported(p, dt);
+}
+
+// Returns cudaErrorNotSupported when the launch cannot be set up (the caller then takes the mma.sync sweep).
+cudaError_t launch_scores_tc5(const Params &p, const void *Q, const void *K, const float *LSE, float *out,
+                              int64_t out_stride, int64_t row0, int64_t n_rows, bool all_visible, cudaStream_t st)
+{
+    if (n_rows == 0) return cudaSuccess;
+    CUtensorMap tmQ, tmK;
+    if (!make_map(&tmQ, Q, p.B, p.Lq, p.Hq, p.qs_b, p.qs_t, p.qs_h, 128 / p.G, p.G) ||
+        !make_map(&tmK, K, p.B, p.Lk, p.Hkv, p.ks_b, p.ks_t, p.ks_h, 128))
+        return cudaErrorNotSupported;
+    if ((int64_t)((row0 + n_rows - 1) / p.Lq - row0 / p.Lq + 1) * ((p.Lq + 128 / p.G - 1) / (128 / p.G)) > 65535)
+        return cudaErrorNotSupported;
+    if (all_visible) {   // keys a query cannot see read -inf
+        const int64_t n = n_rows * out_stride;
+        const int64_t fb = (n + 255) / 256;
+        k_fill_tc5<<<(unsigned)(fb < 148 * 16 ? fb : 148 * 16), 256, 0, st>>>(out, n, -INFINITY);
+        count_launch();
+    }
+    switch (p.G) {
+        case 1: return launch_scores_tc5_g<1>(tmQ, tmK, p, LSE, out, out_stride, row0, n_rows, all_visible, st);
+        case 2: return launch_scores_tc5_g<2>(tmQ, tmK, p, LSE, out, out_stride, row0, n_rows, all_visible, st);
+        case 4: return launch_scores_tc5_g<4>(tmQ, tmK, p, LSE, out, out_stride, row0, n_rows, all_visible, st);
+        case 8: return launch_scores_tc5_g<8>(tmQ, tmK, p, LSE, out, out_stride, row0, n_rows, all_visible, st);
+        case 16: return launch_scores_tc5_g<16>(tmQ, tmK, p, LSE, out, out_stride, row0, n_rows, all_visible, st);
+    }
+    return cudaErrorNotSupported;
 }
 
 // Device error word of the tcgen05 kernels (0 = no bounded wait ever ran out).  Synchronises the device.
