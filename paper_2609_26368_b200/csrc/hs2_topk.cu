@@ -10,10 +10,7 @@
 namespace hs2 {
 namespace {
 
-constexpr int kThreads = 1024;
-constexpr int kWarps = kThreads / 32;
 constexpr int kItems = 4;                    // consecutive scores per thread per step
-constexpr int kChunk = kThreads * kItems;
 
 // float -> uint32 whose unsigned order is the float order; -0 is folded onto +0 first.
 __device__ __forceinline__ uint32_t order_key(float f)
@@ -39,13 +36,49 @@ __device__ __forceinline__ void load_keys(const float *row, int j0, int nc, uint
     }
 }
 
-template <bool VEC>
-__global__ void __launch_bounds__(kThreads)
+// Shared by both variants: find, from the top, the digit at which the running count reaches `need`.
+// hist[256] is complete; warp 0 scans it.  Writes the new prefix and the remaining need.
+__device__ __forceinline__ void pick_digit(const unsigned *hist, unsigned prefix, unsigned need, int lane, unsigned *s_prefix,
+                                           unsigned *s_need)
+{
+    // lane l owns digits 255-8l .. 248-8l (descending)
+    unsigned mine = 0;
+#pragma unroll
+    for (int e = 0; e < 8; ++e) mine += hist[255 - 8 * lane - e];
+    unsigned incl = mine;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const unsigned t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+    }
+    const unsigned before = incl - mine;
+    if (before < need && need <= incl) {
+        unsigned cum = before;
+        for (int e = 0; e < 8; ++e) {
+            const unsigned c = hist[255 - 8 * lane - e];
+            if (cum + c >= need) {
+                *s_prefix = (prefix << 8) | (unsigned)(255 - 8 * lane - e);
+                *s_need = need - cum;
+                break;
+            }
+            cum += c;
+        }
+    }
+}
+
+// THREADS threads per row.  CACHED: the row (at most THREADS * ITEMS candidates) is read once into
+// registers and every later pass runs on them; otherwise the row is re-read for every pass.
+// Element order (and so the tie-break and the output order) is the key index in both cases.
+template <int THREADS, int ITEMS, bool CACHED, bool VEC>
+__global__ void __launch_bounds__(THREADS)
 k_topk(const Params p, const float *__restrict__ scores, int64_t score_stride, int32_t *__restrict__ idx,
        int64_t row0)
 {
+    constexpr int WARPS = THREADS / 32;
+    constexpr int CHUNK = THREADS * kItems;           // candidates per step
+    constexpr int STEPS = ITEMS / kItems;             // steps held in registers (CACHED)
     __shared__ unsigned hist[256];
-    __shared__ unsigned s_warp[kWarps];
+    __shared__ unsigned s_warp[WARPS];
     __shared__ unsigned s_prefix, s_need;
     __shared__ unsigned s_run_gt, s_run_eq;
 
@@ -61,54 +94,64 @@ k_topk(const Params p, const float *__restrict__ scores, int64_t score_stride, i
     const float *srow = scores + (int64_t)blockIdx.x * score_stride;
 
     if (take == nc) {   // every candidate is kept: no need to look at the scores
-        for (int t = tid; t < p.k; t += kThreads) out[t] = t < nc ? t : -1;
+        for (int t = tid; t < p.k; t += THREADS) out[t] = t < nc ? t : -1;
         return;
     }
+    const int nsteps = (nc + CHUNK - 1) / CHUNK;
+
+    uint32_t ck[CACHED ? ITEMS : kItems];   // cached keys (CACHED) / scratch
+    if (CACHED) {
+#pragma unroll
+        for (int st = 0; st < STEPS; ++st) {
+            if (st < nsteps) {
+                uint32_t key[kItems];
+                bool ok[kItems];
+                load_keys<VEC>(srow, st * CHUNK + tid * kItems, nc, key, ok);
+#pragma unroll
+                for (int e = 0; e < kItems; ++e) ck[st * kItems + e] = key[e];
+            }
+        }
+    }
+    auto get = [&](int st, uint32_t (&key)[kItems], bool (&ok)[kItems]) {
+        if (CACHED) {
+#pragma unroll
+            for (int s2 = 0; s2 < STEPS; ++s2)
+                if (s2 == st) {
+#pragma unroll
+                    for (int e = 0; e < kItems; ++e) {
+                        key[e] = ck[s2 * kItems + e];
+                        ok[e] = st * CHUNK + tid * kItems + e < nc;
+                    }
+                }
+        } else {
+            load_keys<VEC>(srow, st * CHUNK + tid * kItems, nc, key, ok);
+        }
+    };
 
     // ---- radix select: value of the take-th largest key
     unsigned prefix = 0, need = (unsigned)take;
     for (int round = 0; round < 4; ++round) {
         const int shift = 24 - 8 * round;
         if (tid < 256) hist[tid] = 0;
+        if (THREADS < 256) for (int t = tid + THREADS; t < 256; t += THREADS) hist[t] = 0;
         __syncthreads();
-        for (int base = 0; base < nc; base += kChunk) {
-            uint32_t key[kItems];
-            bool ok[kItems];
-            load_keys<VEC>(srow, base + tid * kItems, nc, key, ok);
 #pragma unroll
-            for (int e = 0; e < kItems; ++e) {
-                const bool live = ok[e] && (round == 0 || (key[e] >> (shift + 8)) == prefix);
-                const unsigned digit = live ? ((key[e] >> shift) & 255u) : 256u;
-                const unsigned peers = __match_any_sync(0xffffffffu, digit);   // one atomic per distinct digit per warp
-                if (live && lane == __ffs(peers) - 1) atomicAdd(&hist[digit], __popc(peers));
-            }
-        }
-        __syncthreads();
-        if (warp == 0) {
-            // lane l owns digits 255-8l .. 248-8l (descending); find the digit where the count from the top reaches need
-            unsigned mine = 0;
+        for (int st = 0; st < (CACHED ? STEPS : 1); ++st) {
+            for (int sr = CACHED ? st : 0; sr < (CACHED ? min(st + 1, nsteps) : nsteps); ++sr) {
+                uint32_t key[kItems];
+                bool ok[kItems];
+                get(sr, key, ok);
 #pragma unroll
-            for (int e = 0; e < 8; ++e) mine += hist[255 - 8 * lane - e];
-            unsigned incl = mine;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const unsigned t = __shfl_up_sync(0xffffffffu, incl, o);
-                if (lane >= o) incl += t;
-            }
-            const unsigned before = incl - mine;
-            if (before < need && need <= incl) {
-                unsigned cum = before;
-                for (int e = 0; e < 8; ++e) {
-                    const unsigned c = hist[255 - 8 * lane - e];
-                    if (cum + c >= need) {
-                        s_prefix = (prefix << 8) | (unsigned)(255 - 8 * lane - e);
-                        s_need = need - cum;
-                        break;
-                    }
-                    cum += c;
+                for (int e = 0; e < kItems; ++e) {
+                    const bool live = ok[e] && (round == 0 || (key[e] >> (shift + 8)) == prefix);
+                    const unsigned digit = live ? ((key[e] >> shift) & 255u) : 256u;
+                    const unsigned peers = __match_any_sync(0xffffffffu, digit);   // one atomic per distinct digit per warp
+                    if (live && lane == __ffs(peers) - 1) atomicAdd(&hist[digit], __popc(peers));
                 }
             }
         }
+        __syncthreads();
+        if (warp == 0) pick_digit(hist, prefix, need, lane, &s_prefix, &s_need);
         __syncthreads();
         prefix = s_prefix;
         need = s_need;
@@ -119,68 +162,83 @@ k_topk(const Params p, const float *__restrict__ scores, int64_t score_stride, i
     // ---- ordered compaction: kept = key > tau, or key == tau and fewer than need_eq equal keys before it
     if (tid == 0) { s_run_gt = 0; s_run_eq = 0; }
     __syncthreads();
-    for (int base = 0; base < nc; base += kChunk) {
-        uint32_t key[kItems];
-        bool ok[kItems];
-        const int j0 = base + tid * kItems;
-        load_keys<VEC>(srow, j0, nc, key, ok);
-        unsigned n_gt = 0, n_eq = 0;
 #pragma unroll
-        for (int e = 0; e < kItems; ++e) {
-            n_gt += ok[e] && key[e] > tau;
-            n_eq += ok[e] && key[e] == tau;
-        }
-        // exclusive scan of (gt, eq) over the block in thread order; both counts fit 16 bits per chunk
-        const unsigned packed = (n_gt << 16) | n_eq;
-        unsigned incl = packed;
+    for (int st = 0; st < (CACHED ? STEPS : 1); ++st) {
+        for (int sr = CACHED ? st : 0; sr < (CACHED ? min(st + 1, nsteps) : nsteps); ++sr) {
+            uint32_t key[kItems];
+            bool ok[kItems];
+            const int j0 = sr * CHUNK + tid * kItems;
+            get(sr, key, ok);
+            unsigned n_gt = 0, n_eq = 0;
 #pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const unsigned t = __shfl_up_sync(0xffffffffu, incl, o);
-            if (lane >= o) incl += t;
-        }
-        if (lane == 31) s_warp[warp] = incl;
-        __syncthreads();
-        const unsigned run_gt = s_run_gt, run_eq = s_run_eq;
-        unsigned wsum = lane < kWarps ? s_warp[lane] : 0u;   // every warp scans the 32 warp totals itself
-        unsigned wincl = wsum;
-#pragma unroll
-        for (int o = 1; o < 32; o <<= 1) {
-            const unsigned t = __shfl_up_sync(0xffffffffu, wincl, o);
-            if (lane >= o) wincl += t;
-        }
-        const unsigned warp_excl = __shfl_sync(0xffffffffu, wincl - wsum, warp);
-        const unsigned total = __shfl_sync(0xffffffffu, wincl, 31);
-        const unsigned excl = warp_excl + incl - packed;
-        unsigned gt_before = run_gt + (excl >> 16), eq_before = run_eq + (excl & 0xffffu);
-#pragma unroll
-        for (int e = 0; e < kItems; ++e) {
-            if (!ok[e]) continue;
-            if (key[e] > tau) {
-                out[gt_before + min(eq_before, need_eq)] = j0 + e;
-                ++gt_before;
-            } else if (key[e] == tau) {
-                if (eq_before < need_eq) out[gt_before + eq_before] = j0 + e;
-                ++eq_before;
+            for (int e = 0; e < kItems; ++e) {
+                n_gt += ok[e] && key[e] > tau;
+                n_eq += ok[e] && key[e] == tau;
             }
+            // exclusive scan of (gt, eq) over the block in thread order; both counts fit 16 bits per step
+            const unsigned packed = (n_gt << 16) | n_eq;
+            unsigned incl = packed;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const unsigned t = __shfl_up_sync(0xffffffffu, incl, o);
+                if (lane >= o) incl += t;
+            }
+            if (lane == 31) s_warp[warp] = incl;
+            __syncthreads();
+            const unsigned run_gt = s_run_gt, run_eq = s_run_eq;
+            unsigned wsum = lane < WARPS ? s_warp[lane] : 0u;   // every warp scans the warp totals itself
+            unsigned wincl = wsum;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const unsigned t = __shfl_up_sync(0xffffffffu, wincl, o);
+                if (lane >= o) wincl += t;
+            }
+            const unsigned warp_excl = __shfl_sync(0xffffffffu, wincl - wsum, warp);
+            const unsigned total = __shfl_sync(0xffffffffu, wincl, WARPS - 1);
+            const unsigned excl = warp_excl + incl - packed;
+            unsigned gt_before = run_gt + (excl >> 16), eq_before = run_eq + (excl & 0xffffu);
+#pragma unroll
+            for (int e = 0; e < kItems; ++e) {
+                if (!ok[e]) continue;
+                if (key[e] > tau) {
+                    out[gt_before + min(eq_before, need_eq)] = j0 + e;
+                    ++gt_before;
+                } else if (key[e] == tau) {
+                    if (eq_before < need_eq) out[gt_before + eq_before] = j0 + e;
+                    ++eq_before;
+                }
+            }
+            __syncthreads();   // everyone has read s_warp and the running totals
+            if (tid == 0) { s_run_gt = run_gt + (total >> 16); s_run_eq = run_eq + (total & 0xffffu); }
         }
-        __syncthreads();   // everyone has read s_warp and the running totals
-        if (tid == 0) { s_run_gt = run_gt + (total >> 16); s_run_eq = run_eq + (total & 0xffffu); }
     }
-    for (int t = take + tid; t < p.k; t += kThreads) out[t] = -1;
+    for (int t = take + tid; t < p.k; t += THREADS) out[t] = -1;
 }
 
 }  // namespace
+
+template <int THREADS, int ITEMS, bool CACHED>
+void launch_variant(const Params &p, const float *scores, int64_t score_stride, int32_t *idx, int64_t row0, int64_t n_rows,
+                    bool vec, cudaStream_t st)
+{
+    if (vec)
+        k_topk<THREADS, ITEMS, CACHED, true><<<(unsigned)n_rows, THREADS, 0, st>>>(p, scores, score_stride, idx, row0);
+    else
+        k_topk<THREADS, ITEMS, CACHED, false><<<(unsigned)n_rows, THREADS, 0, st>>>(p, scores, score_stride, idx, row0);
+}
 
 cudaError_t launch_topk(const Params &p, const float *scores, int64_t score_stride, int32_t *idx, int64_t row0,
                         int64_t n_rows, cudaStream_t st)
 {
     if (n_rows == 0 || p.k == 0) return cudaSuccess;
     const bool vec = (score_stride % 4 == 0) && (reinterpret_cast<uintptr_t>(scores) % 16 == 0);
-    // grid.x is limited to 2^31-1 rows per launch, far above any row block used here
-    if (vec)
-        k_topk<true><<<(unsigned)n_rows, kThreads, 0, st>>>(p, scores, score_stride, idx, row0);
+    // no row is longer than Lk: short rows live in registers (read once), long rows are re-read per pass
+    if (p.Lk <= 256 * 32)
+        launch_variant<256, 32, true>(p, scores, score_stride, idx, row0, n_rows, vec, st);
+    else if (p.Lk <= 1024 * 32)
+        launch_variant<1024, 32, true>(p, scores, score_stride, idx, row0, n_rows, vec, st);
     else
-        k_topk<false><<<(unsigned)n_rows, kThreads, 0, st>>>(p, scores, score_stride, idx, row0);
+        launch_variant<1024, kItems, false>(p, scores, score_stride, idx, row0, n_rows, vec, st);
     count_launch();
     return cudaGetLastError();
 }
