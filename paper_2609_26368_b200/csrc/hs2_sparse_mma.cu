@@ -129,16 +129,21 @@ __device__ __forceinline__ int slot_key(const Params &p, const Item &it, int til
 template <int KT>
 __device__ __forceinline__ void issue_stage(const Item &it, uint32_t stage_base, int j, int lane)
 {
-    const int c = lane & 15;
+    // lane -> 16-byte chunk c of rows r0 + (lane >> 4), r0 = 0, 2, 4, ...  Because r0 is even,
+    // (c ^ (r & 7)) = (c ^ (lane >> 4)) ^ (r0 & 6): the lane part is hoisted, the rest is a constant.
+    const int c = lane & 15, hi = lane >> 4;
+    const uint32_t cx = (uint32_t)(c ^ hi);
+    const uint32_t dst_lane = stage_base + hi * kRowBytes;
+    const char *kc = it.Kb + c * 16, *vc = it.Vb + c * 16;
+    const int rs = (int)it.row_stride;
 #pragma unroll
     for (int r0 = 0; r0 < KT; r0 += 2) {
-        const int r = r0 + (lane >> 4);
-        const int jr = __shfl_sync(0xffffffffu, j, r);
-        const uint32_t dst = stage_base + r * kRowBytes + ((c ^ (r & 7)) << 4);
-        const int64_t off = (int64_t)(jr < 0 ? 0 : jr) * it.row_stride + c * 16;
-        const int nbytes = jr < 0 ? 0 : 16;   // void rows are zero filled, nothing is read
-        cp_async16(dst, it.Kb + off, nbytes);
-        cp_async16(dst + KT * kRowBytes, it.Vb + off, nbytes);
+        const int jr = __shfl_sync(0xffffffffu, j, r0 + hi);
+        const uint32_t dst = dst_lane + r0 * kRowBytes + ((cx ^ (uint32_t)(r0 & 6)) << 4);
+        const int64_t off = (int64_t)max(jr, 0) * rs;   // one wide multiply-add per tensor
+        const int nbytes = jr < 0 ? 0 : 16;             // void rows are zero filled, nothing is read
+        cp_async16(dst, kc + off, nbytes);
+        cp_async16(dst + KT * kRowBytes, vc + off, nbytes);
     }
 }
 
@@ -155,12 +160,14 @@ __device__ __forceinline__ void consume_stage(Acc &acc, const uint32_t (&qf)[16]
     for (int mt = 0; mt < MT; ++mt) {
         float s2[4] = {0.f, 0.f, 0.f, 0.f};
         s[mt][0] = s[mt][1] = s[mt][2] = s[mt][3] = 0.f;
+        // chunk = 2 ks + (mi >> 1); (chunk ^ rr) << 4 = (32 ks) ^ lx with lx = ((mi >> 1) ^ rr) << 4
         const uint32_t rowaddr = stage_base + (mt * 16 + (mi & 1) * 8 + rr) * kRowBytes;
+        const uint32_t lx = (uint32_t)((mi >> 1) ^ rr) << 4;
 #pragma unroll
         for (int ks = 0; ks < 8; ks += 2) {
             uint32_t a[4], a2[4];
-            ldmatrix_x4(a, rowaddr + (((2 * ks + (mi >> 1)) ^ rr) << 4));
-            ldmatrix_x4(a2, rowaddr + (((2 * ks + 2 + (mi >> 1)) ^ rr) << 4));
+            ldmatrix_x4(a, rowaddr + (lx ^ (uint32_t)(32 * ks)));
+            ldmatrix_x4(a2, rowaddr + (lx ^ (uint32_t)(32 * ks + 32)));
             mma_bf16(s[mt], a, qf[2 * ks], qf[2 * ks + 1]);
             mma_bf16(s2, a2, qf[2 * ks + 2], qf[2 * ks + 3]);
         }
@@ -217,10 +224,11 @@ __device__ __forceinline__ void consume_stage(Acc &acc, const uint32_t (&qf)[16]
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt) {
         const uint32_t rowaddr = vbase + (mt * 16 + (mi >> 1) * 8 + rr) * kRowBytes;
+        const uint32_t lx = (uint32_t)((mi & 1) ^ rr) << 4;
 #pragma unroll
         for (int dt = 0; dt < 8; ++dt) {
             uint32_t a[4];
-            ldmatrix_x4_trans(a, rowaddr + (((2 * dt + (mi & 1)) ^ rr) << 4));
+            ldmatrix_x4_trans(a, rowaddr + (lx ^ (uint32_t)(32 * dt)));
             mma_bf16(acc.o[dt], a, pb[mt][0], pb[mt][1]);
         }
     }
@@ -579,6 +587,7 @@ cudaError_t set_attrs()
 bool sparse_mma_supported(const Params &p, hs2_dtype dt)
 {
     auto m8 = [](int64_t x) { return x % 8 == 0; };
+    if (p.ks_t * 2 > 0x7fffffffLL) return false;   // the row stride is used as a 32-bit multiplier
     return dt == HS2_BF16 && p.D == HD && p.G >= 1 && p.G <= 8 && m8(p.qs_b) && m8(p.qs_t) && m8(p.qs_h) &&
            m8(p.ks_b) && m8(p.ks_t) && m8(p.ks_h) && m8(p.os_b) && m8(p.os_t) && m8(p.os_h);
 }
