@@ -22,7 +22,10 @@ hs2_status cuda_fail(cudaError_t e)
 
 size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
 
-constexpr size_t kStripCapBytes = (size_t)1 << 30;   // default bound on the score strips of one launch
+#ifndef HS2_STRIP_CAP_MB
+#define HS2_STRIP_CAP_MB 1024
+#endif
+constexpr size_t kStripCapBytes = (size_t)HS2_STRIP_CAP_MB << 20;   // bound on the score strips of one launch
 
 // Validate the host-visible part of a problem and resolve defaults.
 hs2_status resolve(const hs2_problem *hp, bool need_tensors, Params *out)
@@ -187,16 +190,23 @@ hs2_status hs2_full_attn_select(const hs2_problem *hp, const void *Q, const void
     if (!want_sel && !scores_dbg) return HS2_OK;
 
     const int64_t rows = select_rows(p);
+    constexpr int64_t kMaxBlockRows = 262144;   // keeps the score kernels' grid.y inside its limit
     if (scores_dbg) {
         // scores for every visible key go straight to the caller's tensor; the selection reads them from there
-        e = launch_scores(p, dt, mma, aligned16(Q, K, V, O), Q, K, LSE, scores_dbg, p.Lk, 0, rows, true, st);
-        if (e != cudaSuccess) return cuda_fail(e);
-        if (want_sel && (e = launch_topk(p, scores_dbg, p.Lk, idx, 0, rows, st)) != cudaSuccess) return cuda_fail(e);
+        for (int64_t r0 = 0; r0 < rows; r0 += kMaxBlockRows) {
+            const int64_t n = rows - r0 < kMaxBlockRows ? rows - r0 : kMaxBlockRows;
+            float *dst = scores_dbg + r0 * p.Lk;
+            e = launch_scores(p, dt, mma, aligned16(Q, K, V, O), Q, K, LSE, dst, p.Lk, r0, n, true, st);
+            if (e != cudaSuccess) return cuda_fail(e);
+            if (want_sel && (e = launch_topk(p, dst, p.Lk, idx, r0, n, st)) != cudaSuccess) return cuda_fail(e);
+        }
         return HS2_OK;
     }
     // bounded strips: score a block of query rows into the workspace, select from it, move on
     const int64_t stride = (int64_t)(row_bytes / sizeof(float));
-    int64_t block = (int64_t)(ws_bytes / row_bytes);
+    int64_t block = (int64_t)((ws_bytes < kStripCapBytes ? ws_bytes : kStripCapBytes) / row_bytes);
+    if (block < 1) block = 1;
+    if (block > kMaxBlockRows) block = kMaxBlockRows;
     if (block > rows) block = rows;
     float *strip = (float *)ws;
     for (int64_t r0 = 0; r0 < rows; r0 += block) {

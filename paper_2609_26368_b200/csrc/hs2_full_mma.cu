@@ -246,13 +246,14 @@ template <int G>
 __global__ void __launch_bounds__(SC_WARPS * 32, 1)
 k_scores_mma(const Params p, const __nv_bfloat16 *__restrict__ Q, const __nv_bfloat16 *__restrict__ K,
              const float *__restrict__ LSE, float *__restrict__ out, int64_t out_stride, int64_t row0, int64_t n_rows,
-             int all_visible, int bg_first, int tiles_per_bg, int vec_ok)
+             int all_visible, int tile_first, int tiles_per_bg, int vec_ok)
 {
     extern __shared__ __align__(128) char smem[];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const int g = lane >> 2, t = lane & 3, mi = lane >> 3, rr = lane & 7;
-    const int bg = bg_first + blockIdx.y / tiles_per_bg;
-    const int qt = blockIdx.y % tiles_per_bg;
+    const int tile = tile_first + blockIdx.y;   // flattened (b, g, query tile)
+    const int bg = tile / tiles_per_bg;
+    const int qt = tile % tiles_per_bg;
     const int gkv = bg % p.Hkv, b = bg / p.Hkv;
     const int kvl = kvlen_of(p, b);
     const int iq0 = qt * SC_Q;                                // first query of the CTA
@@ -444,10 +445,13 @@ cudaError_t launch_scores_mma(const Params &p, const void *Q, const void *K, con
         k_fill<<<(unsigned)(fb < 148 * 16 ? fb : 148 * 16), 256, 0, st>>>(out, n, -INFINITY);
         count_launch();
     }
-    const int bg_first = (int)(row0 / p.Lq), bg_last = (int)((row0 + n_rows - 1) / p.Lq);
     const int tiles_per_bg = (p.Lq + SC_Q - 1) / SC_Q;
-    const int64_t gy = (int64_t)(bg_last - bg_first + 1) * tiles_per_bg;
-    if (gy > 65535) return cudaErrorInvalidConfiguration;
+    const int64_t last = row0 + n_rows - 1;
+    const int64_t t_first = (row0 / p.Lq) * tiles_per_bg + (row0 % p.Lq) / SC_Q;
+    const int64_t t_last = (last / p.Lq) * tiles_per_bg + (last % p.Lq) / SC_Q;
+    const int64_t gy = t_last - t_first + 1;
+    if (gy > 65535 || t_last > 0x7fffffffLL) return cudaErrorInvalidConfiguration;
+    const int bg_first = (int)t_first;
     dim3 grid((p.Lk + SC_CHUNK - 1) / SC_CHUNK, (unsigned)gy);
     const int vec_ok = (out_stride % 4 == 0) && (reinterpret_cast<uintptr_t>(out) % 16 == 0);
     const __nv_bfloat16 *q = (const __nv_bfloat16 *)Q, *k = (const __nv_bfloat16 *)K;

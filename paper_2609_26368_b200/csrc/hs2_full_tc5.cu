@@ -391,7 +391,7 @@ template <int G>
 __global__ void __launch_bounds__(kThreads, 2)
 k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, const Params p,
              const float *__restrict__ LSE, float *__restrict__ out, int64_t out_stride, int64_t row0, int64_t n_rows,
-             int all_visible, int bg_first, int tiles_per_bg)
+             int all_visible, int tile_first, int tiles_per_bg)
 {
     constexpr int TQ = 128 / G;          // queries per CTA
     constexpr int QPC = 32 / G > 0 ? 32 / G : 1;   // queries per 32-column chunk (G <= 32)
@@ -413,8 +413,9 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     int64_t *s_row = reinterpret_cast<int64_t *>(smem + kScOffRow);
 
     const int tid = threadIdx.x, warp = tid >> 5;
-    const int bg = bg_first + blockIdx.y / tiles_per_bg;
-    const int qt = blockIdx.y % tiles_per_bg;
+    const int tile = tile_first + blockIdx.y;   // flattened (b, g, query tile)
+    const int bg = tile / tiles_per_bg;
+    const int qt = tile % tiles_per_bg;
     const int gkv = bg % p.Hkv, b = bg / p.Hkv;
     const int kvl = kvlen_of(p, b);
     const int iq0 = qt * TQ;
@@ -627,13 +628,16 @@ cudaError_t launch_scores_tc5_g(const CUtensorMap &tmQ, const CUtensorMap &tmK, 
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
     constexpr int TQ = 128 / G;
-    const int bg_first = (int)(row0 / p.Lq), bg_last = (int)((row0 + n_rows - 1) / p.Lq);
     const int tiles_per_bg = (p.Lq + TQ - 1) / TQ;
-    const int64_t gy = (int64_t)(bg_last - bg_first + 1) * tiles_per_bg;
-    if (gy > 65535) return cudaErrorNotSupported;
+    // only the query tiles that intersect rows [row0, row0 + n_rows) of the flattened (b, g, i) index
+    const int64_t last = row0 + n_rows - 1;
+    const int64_t t_first = (row0 / p.Lq) * tiles_per_bg + (row0 % p.Lq) / TQ;
+    const int64_t t_last = (last / p.Lq) * tiles_per_bg + (last % p.Lq) / TQ;
+    const int64_t gy = t_last - t_first + 1;
+    if (gy > 65535 || t_last > 0x7fffffffLL) return cudaErrorNotSupported;
     dim3 grid((p.Lk + SC_KCHUNK - 1) / SC_KCHUNK, (unsigned)gy);
     k_scores_tc5<G><<<grid, kThreads, kScSmemBytes, st>>>(tmQ, tmK, p, LSE, out, out_stride, row0, n_rows, all_visible ? 1 : 0,
-                                                         bg_first, tiles_per_bg);
+                                                         (int)t_first, tiles_per_bg);
     count_launch();
     return cudaGetLastError();
 }
@@ -653,8 +657,7 @@ cudaError_t launch_scores_tc5(const Params &p, const void *Q, const void *K, con
     if (!make_map(&tmQ, Q, p.B, p.Lq, p.Hq, p.qs_b, p.qs_t, p.qs_h, 128 / p.G, p.G) ||
         !make_map(&tmK, K, p.B, p.Lk, p.Hkv, p.ks_b, p.ks_t, p.ks_h, 128))
         return cudaErrorNotSupported;
-    if ((int64_t)((row0 + n_rows - 1) / p.Lq - row0 / p.Lq + 1) * ((p.Lq + 128 / p.G - 1) / (128 / p.G)) > 65535)
-        return cudaErrorNotSupported;
+    if ((n_rows + p.Lq) / (128 / p.G) + 2 * (int64_t)p.B * p.Hkv > 65535) return cudaErrorNotSupported;   // grid.y bound
     if (all_visible) {   // keys a query cannot see read -inf
         const int64_t n = n_rows * out_stride;
         const int64_t fb = (n + 255) / 256;
