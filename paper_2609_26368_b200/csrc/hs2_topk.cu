@@ -11,6 +11,7 @@ namespace hs2 {
 namespace {
 
 constexpr int kItems = 4;                    // consecutive scores per thread per step
+constexpr unsigned kListCap = 2048;          // threshold-bin candidates kept in shared memory (cached variant)
 
 // float -> uint32 whose unsigned order is the float order; -0 is folded onto +0 first.
 __device__ __forceinline__ uint32_t order_key(float f)
@@ -66,9 +67,153 @@ __device__ __forceinline__ void pick_digit(const unsigned *hist, unsigned prefix
     }
 }
 
-// THREADS threads per row.  CACHED: the row (at most THREADS * ITEMS candidates) is read once into
-// registers and every later pass runs on them; otherwise the row is re-read for every pass.
-// Element order (and so the tie-break and the output order) is the key index in both cases.
+// ---- rows that fit in registers: THREADS x E candidates, read once ------------------------------
+// Thread t owns the E consecutive candidates E t .. E t + E - 1, so the ascending-index order of the
+// output is (thread, element) order and the ordered compaction needs a single block scan.  The radix
+// digits are taken below the common leading bits of the row's smallest and largest key, which makes
+// the first round spread the candidates over all 256 bins (log-probabilities share their top bits).
+template <int THREADS, int E, bool VEC>
+__global__ void __launch_bounds__(THREADS, THREADS <= 256 ? 3 : 1)
+k_topk_cached(const Params p, const float *__restrict__ scores, int64_t score_stride, int32_t *__restrict__ idx,
+              int64_t row0)
+{
+    constexpr int WARPS = THREADS / 32;
+    __shared__ unsigned hist[256];
+    __shared__ unsigned s_warp[WARPS];
+    __shared__ unsigned s_min[WARPS], s_max[WARPS];
+    __shared__ unsigned s_prefix, s_need, s_cnt;
+    __shared__ uint32_t s_list[kListCap];
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int64_t row = row0 + blockIdx.x;   // (b, g, i), i fastest
+    const int i = (int)(row % p.Lq);
+    const int b = (int)(row / ((int64_t)p.Lq * p.Hkv));
+    const int kvl = kvlen_of(p, b);
+    const int pos = pos_of(p, b, i);
+    const int nc = max(0, min(pos - p.w + 1, kvl));   // candidates are keys 0..nc-1
+    const int take = min(p.k, nc);
+    int32_t *out = idx + row * p.k;
+    const float *srow = scores + (int64_t)blockIdx.x * score_stride;
+
+    if (take == nc) {   // every candidate is kept: no need to look at the scores
+        for (int t = tid; t < p.k; t += THREADS) out[t] = t < nc ? t : -1;
+        return;
+    }
+    const int j0 = tid * E;
+    uint32_t key[E];
+    unsigned kmin = 0xffffffffu, kmax = 0u;
+#pragma unroll
+    for (int e4 = 0; e4 < E; e4 += 4) {
+        if (VEC && j0 + e4 + 4 <= nc) {
+            const float4 v = __ldg(reinterpret_cast<const float4 *>(srow + j0 + e4));
+            key[e4] = order_key(v.x); key[e4 + 1] = order_key(v.y); key[e4 + 2] = order_key(v.z); key[e4 + 3] = order_key(v.w);
+        } else {
+#pragma unroll
+            for (int e = e4; e < e4 + 4; ++e) key[e] = j0 + e < nc ? order_key(srow[j0 + e]) : 0u;
+        }
+#pragma unroll
+        for (int e = e4; e < e4 + 4; ++e)
+            if (j0 + e < nc) { kmin = min(kmin, key[e]); kmax = max(kmax, key[e]); }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        kmin = min(kmin, __shfl_xor_sync(0xffffffffu, kmin, o));
+        kmax = max(kmax, __shfl_xor_sync(0xffffffffu, kmax, o));
+    }
+    if (lane == 0) { s_min[warp] = kmin; s_max[warp] = kmax; }
+    __syncthreads();
+#pragma unroll
+    for (int w = 0; w < WARPS; ++w) { kmin = min(kmin, s_min[w]); kmax = max(kmax, s_max[w]); }
+
+    // bits above `hi` are equal in every candidate; resolve the rest 8 bits at a time
+    int hi = 32 - __clz(kmin ^ kmax);          // 0 when all candidates are equal
+    unsigned prefix = hi >= 32 ? 0u : (kmax >> hi);
+    unsigned need = (unsigned)take;
+    bool on_list = false;                      // later rounds run on the threshold bin's candidates only
+    unsigned n_list = 0;
+    while (hi > 0) {
+        const int w = min(8, hi), shift = hi - w;
+        const unsigned dmask = (1u << w) - 1u;
+        if (tid < 256) hist[tid] = 0;
+        if (THREADS < 256) for (int t = tid + THREADS; t < 256; t += THREADS) hist[t] = 0;
+        __syncthreads();
+        if (on_list) {
+            for (unsigned t = tid; t < n_list; t += THREADS) {
+                const uint32_t kk = s_list[t];
+                if ((kk >> hi) == prefix) atomicAdd(&hist[(kk >> shift) & dmask], 1u);
+            }
+        } else {
+#pragma unroll
+            for (int e = 0; e < E; ++e) {
+                const bool live = (j0 + e < nc) && (hi >= 32 || (key[e] >> hi) == prefix);
+                if (live) atomicAdd(&hist[(key[e] >> shift) & dmask], 1u);
+            }
+        }
+        __syncthreads();
+        if (warp == 0) pick_digit(hist, prefix, need, lane, &s_prefix, &s_need);
+        if (tid == 0) s_cnt = 0;
+        __syncthreads();
+        // pick_digit composes (prefix << 8) | digit; rebuild with the real digit width
+        const unsigned digit = s_prefix & 255u;
+        const unsigned in_bin = hist[digit];
+        prefix = (hi >= 32 ? 0u : (prefix << w)) | digit;
+        need = s_need;
+        hi = shift;
+        if (!on_list && hi > 0 && in_bin <= kListCap) {
+            // every candidate that can still be the take-th largest sits in this bin: collect them
+#pragma unroll
+            for (int e = 0; e < E; ++e)
+                if (j0 + e < nc && (key[e] >> hi) == prefix) s_list[atomicAdd(&s_cnt, 1u)] = key[e];
+            __syncthreads();
+            on_list = true;
+            n_list = s_cnt;
+        }
+    }
+    const uint32_t tau = hi == 0 && kmin == kmax ? kmax : prefix;   // key of the take-th largest candidate
+    const unsigned need_eq = need;                                   // equal keys kept, lowest indices first
+
+    // ---- ordered compaction with one block scan
+    unsigned n_gt = 0, n_eq = 0;
+#pragma unroll
+    for (int e = 0; e < E; ++e) {
+        const bool ok = j0 + e < nc;
+        n_gt += ok && key[e] > tau;
+        n_eq += ok && key[e] == tau;
+    }
+    const unsigned packed = (n_gt << 16) | n_eq;   // both totals stay below 65536 (rows <= 32768)
+    unsigned incl = packed;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const unsigned t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+    }
+    if (lane == 31) s_warp[warp] = incl;
+    __syncthreads();
+    unsigned wsum = lane < WARPS ? s_warp[lane] : 0u;
+    unsigned wincl = wsum;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const unsigned t = __shfl_up_sync(0xffffffffu, wincl, o);
+        if (lane >= o) wincl += t;
+    }
+    const unsigned excl = __shfl_sync(0xffffffffu, wincl - wsum, warp) + incl - packed;
+    unsigned gt_before = excl >> 16, eq_before = excl & 0xffffu;
+#pragma unroll
+    for (int e = 0; e < E; ++e) {
+        if (j0 + e >= nc) continue;
+        if (key[e] > tau) {
+            out[gt_before + min(eq_before, need_eq)] = j0 + e;
+            ++gt_before;
+        } else if (key[e] == tau) {
+            if (eq_before < need_eq) out[gt_before + eq_before] = j0 + e;
+            ++eq_before;
+        }
+    }
+    for (int t = take + tid; t < p.k; t += THREADS) out[t] = -1;
+}
+
+// ---- longer rows: re-read from memory for every pass -------------------------------------------
+// THREADS threads per row, kItems consecutive candidates per thread per step.
 template <int THREADS, int ITEMS, bool CACHED, bool VEC>
 __global__ void __launch_bounds__(THREADS)
 k_topk(const Params p, const float *__restrict__ scores, int64_t score_stride, int32_t *__restrict__ idx,
@@ -233,11 +378,13 @@ cudaError_t launch_topk(const Params &p, const float *scores, int64_t score_stri
     if (n_rows == 0 || p.k == 0) return cudaSuccess;
     const bool vec = (score_stride % 4 == 0) && (reinterpret_cast<uintptr_t>(scores) % 16 == 0);
     // no row is longer than Lk: short rows live in registers (read once), long rows are re-read per pass
-    if (p.Lk <= 256 * 32)
-        launch_variant<256, 32, true>(p, scores, score_stride, idx, row0, n_rows, vec, st);
-    else if (p.Lk <= 1024 * 32)
-        launch_variant<1024, 32, true>(p, scores, score_stride, idx, row0, n_rows, vec, st);
-    else
+    if (p.Lk <= 256 * 32) {
+        if (vec) k_topk_cached<256, 32, true><<<(unsigned)n_rows, 256, 0, st>>>(p, scores, score_stride, idx, row0);
+        else k_topk_cached<256, 32, false><<<(unsigned)n_rows, 256, 0, st>>>(p, scores, score_stride, idx, row0);
+    } else if (p.Lk <= 512 * 64) {
+        if (vec) k_topk_cached<512, 64, true><<<(unsigned)n_rows, 512, 0, st>>>(p, scores, score_stride, idx, row0);
+        else k_topk_cached<512, 64, false><<<(unsigned)n_rows, 512, 0, st>>>(p, scores, score_stride, idx, row0);
+    } else
         launch_variant<1024, kItems, false>(p, scores, score_stride, idx, row0, n_rows, vec, st);
     count_launch();
     return cudaGetLastError();
