@@ -369,7 +369,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2", choices=sorted(CONFIGS))
-    ap.add_argument("--cpu-rows", type=int, default=64, help="query rows of the CPU-oracle sample")
+    ap.add_argument("--cpu-rows", type=int, default=4096, help="query rows of the CPU-oracle sample (about 15 s of CPU work on cfg2)")
     ap.add_argument("--skip", default="", help="comma list of: block, decode64k, e2e, cpu")
     ap.add_argument("--decode-ctx", type=int, default=65536, help="context length of the decode section (profiling: 8192)")
     args = ap.parse_args()

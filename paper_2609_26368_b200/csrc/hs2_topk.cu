@@ -159,14 +159,19 @@ k_topk_cached(const Params p, const float *__restrict__ scores, int64_t score_st
         prefix = (hi >= 32 ? 0u : (prefix << w)) | digit;
         need = s_need;
         hi = shift;
-        if (!on_list && hi > 0 && in_bin <= kListCap) {
-            // every candidate that can still be the take-th largest sits in this bin: collect them
+        const bool collect = !on_list && hi > 0 && in_bin <= kListCap;
+        __syncthreads();   // every thread has read hist[digit] before the next round zeroes the histogram
+        if (collect) {
+            // every candidate that can still be the take-th largest sits in this bin (at most kListCap of them)
 #pragma unroll
             for (int e = 0; e < E; ++e)
-                if (j0 + e < nc && (key[e] >> hi) == prefix) s_list[atomicAdd(&s_cnt, 1u)] = key[e];
+                if (j0 + e < nc && (key[e] >> hi) == prefix) {
+                    const unsigned slot = atomicAdd(&s_cnt, 1u);
+                    if (slot < kListCap) s_list[slot] = key[e];
+                }
             __syncthreads();
             on_list = true;
-            n_list = s_cnt;
+            n_list = min(s_cnt, kListCap);
         }
     }
     const uint32_t tau = hi == 0 && kmin == kmax ? kmax : prefix;   // key of the take-th largest candidate

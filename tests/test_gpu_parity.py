@@ -87,6 +87,24 @@ def test_topk_adversarial_rows():
         _topk_case(scores, k, w, q_start=[Lk - 1 - len(rows) + 1])
 
 
+@pytest.mark.parametrize("Lk", [8192, 20000, 40000])
+def test_topk_threshold_bin_larger_than_the_shared_list(Lk):
+    """Few distinct values over long rows: the bin that holds the k-th value has thousands of members,
+    so the register kernels must fall back from their shared-memory candidate list (both variants),
+    and the streaming kernel sees heavy ties."""
+    g = torch.Generator().manual_seed(Lk)
+    rows = [
+        torch.randint(0, 3, (Lk,), generator=g).float() - 9.0,                  # three values
+        (torch.randn(Lk, generator=g) * 0.01).round() - 11.0,                    # almost everything equal
+        torch.where(torch.rand(Lk, generator=g) < 0.5, torch.tensor(-7.5), torch.tensor(-7.25)),
+        -8.0 - torch.rand(Lk, generator=g) * 2.0 ** -12,                         # differ only in the low mantissa bits
+        torch.randn(Lk, generator=g) - 10.0,
+    ]
+    scores = torch.stack(rows).view(1, 1, len(rows), Lk)
+    for k, w in [(1024, 128), (5, 0), (Lk // 2, 64)]:
+        _topk_case(scores, k, w, q_start=[Lk - len(rows)])
+
+
 def test_topk_edges_window_and_lengths():
     g = torch.Generator().manual_seed(9)
     s = torch.randn(1, 3, 1, 777, generator=g)
