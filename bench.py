@@ -35,6 +35,10 @@ import torch  # noqa: E402
 
 from gen import CONFIGS, make_inputs, sample_rows  # noqa: E402
 
+# dram__bytes_read.sum + dram__bytes_write.sum of one k_sparse_prefill launch, from the ncu capture
+# summarised in profiles/block_step_cfg2.md (bytes)
+NCU_DRAM_TRAFFIC = {"cfg2": 269.2e6}
+
 METRIC = "sparse-attn prefill tokens/s (hybrid block step: full-attn+select, sparse layers, decode step)"
 
 
@@ -436,7 +440,7 @@ def main():
         ach = gb / (sp_ms * 1e-3) / 1e9
         roofline = {"kernel": "k_sparse_prefill (hs2_sparse_attn_prefill)", "bound": "hbm", "achieved": round(ach, 1),
                     "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": round(ach / peaks["hbm_gbs"], 4),
-                    "traffic": None, "peak_source": peaks["source"], "algorithmic_bytes_per_launch": gb,
+                    "traffic": NCU_DRAM_TRAFFIC.get(wl.name), "peak_source": peaks["source"], "algorithmic_bytes_per_launch": gb,
                     "ms_per_launch": round(sp_ms, 4),
                     "tokens_per_s": round(tokens_per_step / (sp_ms * 1e-3), 1),
                     "note": "achieved counts gathered K/V rows (512 B per attended token per KV head); the cache of "
