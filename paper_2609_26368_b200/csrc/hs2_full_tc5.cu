@@ -269,26 +269,25 @@ k_full_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             if (!__all_sync(0xffffffffu, mbar_wait(bar(S_FULL0 + sb), (j >> 1) & 1, abort_flag))) { alive = false; break; }
             tc_fence_after();
             float s[64];
-            {
-                float lo[32], hi[32];
-                tmem_ld32(lane_base + sb * BN, lo);
-                tmem_ld32(lane_base + sb * BN + 32, hi);
-                tmem_wait_ld();
-#pragma unroll
-                for (int e = 0; e < 32; ++e) { s[e] = lo[e]; s[32 + e] = hi[e]; }
-            }
+            tmem_ld32(lane_base + sb * BN, *reinterpret_cast<float (*)[32]>(&s[0]));
+            tmem_ld32(lane_base + sb * BN + 32, *reinterpret_cast<float (*)[32]>(&s[32]));
+            tmem_wait_ld();
             tc_fence_before();
             mbar_arrive(bar(S_FREE0 + sb));
             const int j0 = j * BN;
-            const bool need_mask = (j0 + BN - 1 > pos0) || (j0 + BN > kvl);
-            float m_blk = -INFINITY;
+            // raw-score maximum; only tiles that touch the diagonal or the end of the cache pay for masking
+            float m_raw = -INFINITY;
+            if ((j0 + BN - 1 > pos0) || (j0 + BN > kvl)) {
 #pragma unroll
-            for (int e = 0; e < 64; ++e) {
-                float v = s[e] * p.scale_log2;
-                if (need_mask && (j0 + e > prow || j0 + e >= kvl)) v = -INFINITY;
-                s[e] = v;
-                m_blk = fmaxf(m_blk, v);
+                for (int e = 0; e < 64; ++e) {
+                    if (j0 + e > prow || j0 + e >= kvl) s[e] = -INFINITY;
+                    m_raw = fmaxf(m_raw, s[e]);
+                }
+            } else {
+#pragma unroll
+                for (int e = 0; e < 64; ++e) m_raw = fmaxf(m_raw, s[e]);
             }
+            const float m_blk = m_raw * p.scale_log2;                 // the scale is positive
             const bool need = m_blk > m_used + kRescaleThreshold;   // also true for the first finite block
             const float m_new = need ? m_blk : m_used;
             const float corr = need ? exp2f(m_used - m_new) : 1.f;  // 0 when nothing was accumulated yet
@@ -310,14 +309,17 @@ k_full_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             }
             l *= corr;
             m_used = m_new;
-            const float muse = m_used == -INFINITY ? 0.f : m_used;
+            const float neg_m = m_used == -INFINITY ? 0.f : -m_used;
             uint32_t pk[32];
+            float l0 = 0.f, l1 = 0.f;
 #pragma unroll
             for (int e = 0; e < 64; e += 2) {
-                const float p0 = exp2f(s[e] - muse), p1 = exp2f(s[e + 1] - muse);
-                l += p0 + p1;
+                const float p0 = exp2f(fmaf(s[e], p.scale_log2, neg_m));       // -inf stays -inf -> 0
+                const float p1 = exp2f(fmaf(s[e + 1], p.scale_log2, neg_m));
+                l0 += p0; l1 += p1;
                 pk[e >> 1] = pack_bf16(p0, p1);
             }
+            l += l0 + l1;
             char *prow_ptr = smem + kOffP + row * 128;
 #pragma unroll
             for (int c = 0; c < 8; ++c)   // 8 keys = one 16-byte chunk, chunk position XOR (row & 7)
