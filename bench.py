@@ -250,6 +250,55 @@ def time_steps(block, steps, warmup, world, timing=True, before=None, after=None
     return a.elapsed_time(b)
 
 
+def time_e2e(wl, device, rank, block0, steps, world):
+    """The same step fed from pinned host memory: every step copies its inputs host->device and its
+    outputs device->host inside the timed region.  Two device buffer sets and three streams let the
+    copies of neighbouring steps overlap the kernels (the user-level double buffering any server does)."""
+    blocks = [block0, Block(wl, device, rank)]
+    host_in = [t.cpu().pin_memory() for t in [block0.q_full, block0.k, block0.v] + block0.q_sparse]
+    host_out = [[torch.empty(t.shape, dtype=t.dtype, device="cpu").pin_memory() for t in b.output_tensors()] for b in blocks]
+    s_in, s_run, s_out = torch.cuda.Stream(), torch.cuda.Stream(), torch.cuda.Stream()
+    ev_in = [torch.cuda.Event() for _ in blocks]      # inputs of buffer set landed
+    ev_run = [torch.cuda.Event() for _ in blocks]     # kernels of buffer set finished
+    ev_out = [torch.cuda.Event() for _ in blocks]     # outputs of buffer set copied back
+
+    def run(n):
+        for it in range(n):
+            b = blocks[it & 1]
+            with torch.cuda.stream(s_in):
+                s_in.wait_event(ev_run[it & 1])           # the set's previous kernels no longer read the inputs
+                for d, h in zip([b.q_full, b.k, b.v] + b.q_sparse, host_in):
+                    d.copy_(h, non_blocking=True)
+                ev_in[it & 1].record(s_in)
+            with torch.cuda.stream(s_run):
+                s_run.wait_event(ev_in[it & 1])
+                s_run.wait_event(ev_out[it & 1])          # the set's previous outputs have left the device
+                b.step()
+                ev_run[it & 1].record(s_run)
+            with torch.cuda.stream(s_out):
+                s_out.wait_event(ev_run[it & 1])
+                for h, d in zip(host_out[it & 1], b.output_tensors()):
+                    h.copy_(d, non_blocking=True)
+                ev_out[it & 1].record(s_out)
+    run(2)
+    barrier(world)
+    a, e = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    a.record()                                         # default stream: everything before is done (synchronised)
+    for st in (s_in, s_run, s_out):
+        st.wait_event(a)
+    run(steps)
+    cur = torch.cuda.current_stream()
+    for st in (s_in, s_run, s_out):
+        done = torch.cuda.Event()
+        done.record(st)
+        cur.wait_event(done)
+    e.record()
+    torch.cuda.synchronize()
+    barrier(world)
+    del blocks[1]
+    return a.elapsed_time(e)
+
+
 # ------------------------------------------------------------------ decode at 64K context (cfg5)
 
 def bench_decode_64k(device, peaks, reps=5, burst=40, ctx=65536):
@@ -411,24 +460,14 @@ def main():
     # ---- end to end: pinned host inputs in, outputs back, every step
     e2e = None
     if "e2e" not in skip:
-        host_in = [t.cpu().pin_memory() for t in [block.q_full, block.k, block.v] + block.q_sparse]
-        dev_in = [block.q_full, block.k, block.v] + block.q_sparse
-        outs = block.output_tensors()
-        host_out = [torch.empty(t.shape, dtype=t.dtype, device="cpu").pin_memory() for t in outs]
-
-        def h2d():
-            for d, h in zip(dev_in, host_in):
-                d.copy_(h, non_blocking=True)
-
-        def d2h():
-            for h, d in zip(host_out, outs):
-                h.copy_(d, non_blocking=True)
-        ms_e2e = time_steps(block, args.steps, 1, world, timing=False, before=h2d, after=d2h)
+        ms_e2e = time_e2e(wl, device, rank, block, args.steps, world)
         ms_e2e = max_over_ranks(ms_e2e, world, device)
+        outs = block.output_tensors()
         e2e = {"value": round(world * tokens_per_step * args.steps / (ms_e2e * 1e-3), 1), "unit": "tokens/s",
                "h2d_bytes_per_step": int(block.input_bytes()),
                "d2h_bytes_per_step": int(sum(t.numel() * t.element_size() for t in outs)),
-               "ms_per_step": round(ms_e2e / args.steps, 3)}
+               "ms_per_step": round(ms_e2e / args.steps, 3),
+               "pipeline": "two device buffer sets; H2D of step n+1 and D2H of step n-1 overlap the kernels of step n"}
 
     if rank != 0:
         return
