@@ -377,21 +377,58 @@ void launch_variant(const Params &p, const float *scores, int64_t score_stride, 
         k_topk<THREADS, ITEMS, CACHED, false><<<(unsigned)n_rows, THREADS, 0, st>>>(p, scores, score_stride, idx, row0);
 }
 
+// one launch of the variant that fits rows of at most `max_nc` candidates
+void launch_rows(const Params &p, const float *scores, int64_t score_stride, int32_t *idx, int64_t row0, int64_t n_rows,
+                 int max_nc, bool vec, cudaStream_t st)
+{
+    if (n_rows <= 0) return;
+    if (max_nc <= 256 * 32) {
+        if (vec) k_topk_cached<256, 32, true><<<(unsigned)n_rows, 256, 0, st>>>(p, scores, score_stride, idx, row0);
+        else k_topk_cached<256, 32, false><<<(unsigned)n_rows, 256, 0, st>>>(p, scores, score_stride, idx, row0);
+    } else if (max_nc <= 512 * 64) {
+        if (vec) k_topk_cached<512, 64, true><<<(unsigned)n_rows, 512, 0, st>>>(p, scores, score_stride, idx, row0);
+        else k_topk_cached<512, 64, false><<<(unsigned)n_rows, 512, 0, st>>>(p, scores, score_stride, idx, row0);
+    } else {
+        launch_variant<1024, kItems, false>(p, scores, score_stride, idx, row0, n_rows, vec, st);
+    }
+    count_launch();
+}
+
 cudaError_t launch_topk(const Params &p, const float *scores, int64_t score_stride, int32_t *idx, int64_t row0,
                         int64_t n_rows, cudaStream_t st)
 {
     if (n_rows == 0 || p.k == 0) return cudaSuccess;
     const bool vec = (score_stride % 4 == 0) && (reinterpret_cast<uintptr_t>(scores) % 16 == 0);
-    // no row is longer than Lk: short rows live in registers (read once), long rows are re-read per pass
-    if (p.Lk <= 256 * 32) {
-        if (vec) k_topk_cached<256, 32, true><<<(unsigned)n_rows, 256, 0, st>>>(p, scores, score_stride, idx, row0);
-        else k_topk_cached<256, 32, false><<<(unsigned)n_rows, 256, 0, st>>>(p, scores, score_stride, idx, row0);
-    } else if (p.Lk <= 512 * 64) {
-        if (vec) k_topk_cached<512, 64, true><<<(unsigned)n_rows, 512, 0, st>>>(p, scores, score_stride, idx, row0);
-        else k_topk_cached<512, 64, false><<<(unsigned)n_rows, 512, 0, st>>>(p, scores, score_stride, idx, row0);
-    } else
-        launch_variant<1024, kItems, false>(p, scores, score_stride, idx, row0, n_rows, vec, st);
-    count_launch();
+    if (p.q_start || p.kv_lens || p.Lk <= 256 * 32) {
+        // positions live on the device (or every row is short): one variant sized for the longest possible row
+        launch_rows(p, scores, score_stride, idx, row0, n_rows, p.Lk, vec, st);
+        return cudaGetLastError();
+    }
+    // Positions are known on the host: query i of a sequence has min(max(Lk - Lq + i - w + 1, 0), Lk)
+    // candidates, growing with i.  Cut the row range where that count crosses a variant's capacity, so
+    // that the short rows at the start of each sequence run on the cheaper register-resident variants.
+    const int64_t caps[2] = {256 * 32, 512 * 64};
+    const int64_t base = (int64_t)p.Lk - p.Lq - p.w + 1;   // candidates of query 0 (before clamping)
+    int64_t r = row0;
+    const int64_t r_end = row0 + n_rows;
+    while (r < r_end) {
+        const int64_t bg = r / p.Lq;
+        const int64_t seg_end = (bg + 1) * p.Lq < r_end ? (bg + 1) * p.Lq : r_end;   // rows of one (sequence, KV head)
+        int64_t i = r - bg * p.Lq;
+        const int64_t i_end = seg_end - bg * p.Lq;
+        while (i < i_end) {
+            int64_t nc = base + i;
+            nc = nc < 0 ? 0 : (nc > p.Lk ? (int64_t)p.Lk : nc);
+            const int64_t cap = nc <= caps[0] ? caps[0] : (nc <= caps[1] ? caps[1] : (int64_t)p.Lk);
+            int64_t last = cap >= p.Lk ? i_end : cap - base + 1;   // base + q <= cap  <=>  q < last
+            if (last > i_end) last = i_end;
+            if (last <= i) last = i + 1;
+            const int64_t first_row = bg * p.Lq + i;
+            launch_rows(p, scores + (first_row - row0) * score_stride, score_stride, idx, first_row, last - i, (int)cap, vec, st);
+            i = last;
+        }
+        r = seg_end;
+    }
     return cudaGetLastError();
 }
 
