@@ -150,7 +150,7 @@ k_scores_generic(const Params p, const T *__restrict__ Q, const T *__restrict__ 
 {
     extern __shared__ float smem[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    const int64_t lr = (int64_t)blockIdx.x * kWarpsPerBlock + warp;
+    const int64_t lr = (int64_t)blockIdx.x * (blockDim.x >> 5) + warp;   // the launcher sizes the block to the shared memory
     if (lr >= n_rows) return;
     const int64_t row = row0 + lr;   // (b, g, i), i fastest
     const int i = (int)(row % p.Lq);
@@ -271,16 +271,21 @@ cudaError_t launch_scores_generic(const Params &p, hs2_dtype dt, const void *Q, 
                                   cudaStream_t st)
 {
     if (n_rows == 0) return cudaSuccess;
-    const unsigned blocks = (unsigned)((n_rows + kWarpsPerBlock - 1) / kWarpsPerBlock);
-    const size_t smem = sizeof(float) * kWarpsPerBlock * p.G * p.D;
+    // each warp keeps the G query vectors of its row in shared memory: fewer warps per block for large groups
+    const size_t per_warp = sizeof(float) * (size_t)p.G * p.D;
+    int warps = (int)((200 * 1024) / per_warp);
+    warps = warps < 1 ? 1 : (warps > kWarpsPerBlock ? kWarpsPerBlock : warps);
+    if (per_warp > 227 * 1024) return cudaErrorInvalidConfiguration;
+    const unsigned blocks = (unsigned)((n_rows + warps - 1) / warps);
+    const size_t smem = per_warp * warps;
     cudaError_t e;
     if (dt == HS2_F32) {
         if ((e = set_smem(k_scores_generic<float>, smem)) != cudaSuccess) return e;
-        k_scores_generic<float><<<blocks, kWarpsPerBlock * 32, smem, st>>>(p, (const float *)Q, (const float *)K, LSE,
-                                                                            out, out_stride, row0, n_rows, all_visible);
+        k_scores_generic<float><<<blocks, warps * 32, smem, st>>>(p, (const float *)Q, (const float *)K, LSE, out, out_stride,
+                                                                  row0, n_rows, all_visible);
     } else {
         if ((e = set_smem(k_scores_generic<__nv_bfloat16>, smem)) != cudaSuccess) return e;
-        k_scores_generic<__nv_bfloat16><<<blocks, kWarpsPerBlock * 32, smem, st>>>(
+        k_scores_generic<__nv_bfloat16><<<blocks, warps * 32, smem, st>>>(
             p, (const __nv_bfloat16 *)Q, (const __nv_bfloat16 *)K, LSE, out, out_stride, row0, n_rows, all_visible);
     }
     count_launch();

@@ -5,6 +5,8 @@
 // the value of the take-th largest score and how many candidates equal to it are still needed;
 // one ordered compaction pass then writes the kept indices in ascending key order, taking equal
 // scores from the lowest index upwards.  The result depends only on the score bits.
+#include <cooperative_groups.h>
+
 #include "hs2_common.cuh"
 
 namespace hs2 {
@@ -75,7 +77,7 @@ __device__ __forceinline__ void pick_digit(const unsigned *hist, unsigned prefix
 template <int THREADS, int E, bool VEC>
 __global__ void __launch_bounds__(THREADS, THREADS <= 256 ? 3 : 1)
 k_topk_cached(const Params p, const float *__restrict__ scores, int64_t score_stride, int32_t *__restrict__ idx,
-              int64_t row0)
+              int64_t row0, int nc_lo, int nc_hi)
 {
     constexpr int WARPS = THREADS / 32;
     __shared__ unsigned hist[256];
@@ -91,6 +93,7 @@ k_topk_cached(const Params p, const float *__restrict__ scores, int64_t score_st
     const int kvl = kvlen_of(p, b);
     const int pos = pos_of(p, b, i);
     const int nc = max(0, min(pos - p.w + 1, kvl));   // candidates are keys 0..nc-1
+    if (nc <= nc_lo || nc > nc_hi) return;   // this row belongs to another variant's launch
     const int take = min(p.k, nc);
     int32_t *out = idx + row * p.k;
     const float *srow = scores + (int64_t)blockIdx.x * score_stride;
@@ -217,12 +220,217 @@ k_topk_cached(const Params p, const float *__restrict__ scores, int64_t score_st
     for (int t = take + tid; t < p.k; t += THREADS) out[t] = -1;
 }
 
+// ---- rows of up to CL x 32768 candidates: one thread-block cluster per row ------------------------
+// Every CTA of the cluster keeps a 32768-candidate slice of the row in registers (read once).  Per
+// radix round each CTA histograms its slice, CTA 0 adds the histograms up through distributed shared
+// memory, picks the digit and publishes the decision; after the first round the threshold bin's
+// members are appended (remote shared-memory atomics) to a list in CTA 0, which finishes the search
+// alone.  The ordered compaction needs the totals of the lower-ranked CTAs, also read through DSMEM.
+template <int CL, bool VEC>
+__global__ void __cluster_dims__(CL, 1, 1) __launch_bounds__(512, 1)
+k_topk_cluster(const Params p, const float *__restrict__ scores, int64_t score_stride, int32_t *__restrict__ idx,
+               int64_t row0, int nc_lo, int nc_hi)
+{
+    namespace cg = cooperative_groups;
+    constexpr int THREADS = 512, E = 64, WARPS = THREADS / 32, SLICE = THREADS * E;
+    __shared__ unsigned hist[256];
+    __shared__ unsigned s_sum[256];
+    __shared__ unsigned s_warp[WARPS];
+    __shared__ unsigned s_min[WARPS], s_max[WARPS];
+    __shared__ unsigned s_mm[2];      // this CTA's min / max key
+    __shared__ unsigned s_tot[2];     // this CTA's number of keys above / equal to the threshold
+    __shared__ unsigned s_dec[3];     // CTA 0 publishes: digit, remaining need, size of the chosen bin
+    __shared__ unsigned s_prefix, s_need, s_cnt;
+    __shared__ uint32_t s_list[kListCap];
+
+    cg::cluster_group cluster = cg::this_cluster();
+    const unsigned rank = cluster.block_rank();
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int64_t row = row0 + blockIdx.x / CL;   // (b, g, i), i fastest
+    const int i = (int)(row % p.Lq);
+    const int b = (int)(row / ((int64_t)p.Lq * p.Hkv));
+    const int kvl = kvlen_of(p, b);
+    const int pos = pos_of(p, b, i);
+    const int nc = max(0, min(pos - p.w + 1, kvl));
+    if (nc <= nc_lo || nc > nc_hi) return;   // this row belongs to another variant's launch
+    const int take = min(p.k, nc);
+    int32_t *out = idx + row * p.k;
+    const float *srow = scores + (int64_t)(blockIdx.x / CL) * score_stride;
+
+    if (take == nc) {   // the same branch in every CTA of the cluster; no remote access on this path
+        for (int t = rank * THREADS + tid; t < p.k; t += CL * THREADS) out[t] = t < nc ? t : -1;
+        return;
+    }
+    const int j0 = rank * SLICE + tid * E;
+    uint32_t key[E];
+    unsigned kmin = 0xffffffffu, kmax = 0u;
+#pragma unroll
+    for (int e4 = 0; e4 < E; e4 += 4) {
+        if (VEC && j0 + e4 + 4 <= nc) {
+            const float4 v = __ldg(reinterpret_cast<const float4 *>(srow + j0 + e4));
+            key[e4] = order_key(v.x); key[e4 + 1] = order_key(v.y); key[e4 + 2] = order_key(v.z); key[e4 + 3] = order_key(v.w);
+        } else {
+#pragma unroll
+            for (int e = e4; e < e4 + 4; ++e) key[e] = j0 + e < nc ? order_key(srow[j0 + e]) : 0u;
+        }
+#pragma unroll
+        for (int e = e4; e < e4 + 4; ++e)
+            if (j0 + e < nc) { kmin = min(kmin, key[e]); kmax = max(kmax, key[e]); }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        kmin = min(kmin, __shfl_xor_sync(0xffffffffu, kmin, o));
+        kmax = max(kmax, __shfl_xor_sync(0xffffffffu, kmax, o));
+    }
+    if (lane == 0) { s_min[warp] = kmin; s_max[warp] = kmax; }
+    __syncthreads();
+    if (tid == 0) {
+        unsigned a = 0xffffffffu, c = 0u;
+        for (int w = 0; w < WARPS; ++w) { a = min(a, s_min[w]); c = max(c, s_max[w]); }
+        s_mm[0] = a; s_mm[1] = c;
+    }
+    cluster.sync();
+    kmin = 0xffffffffu; kmax = 0u;
+#pragma unroll
+    for (int r = 0; r < CL; ++r) {
+        const unsigned *mm = cluster.map_shared_rank(s_mm, r);
+        kmin = min(kmin, mm[0]); kmax = max(kmax, mm[1]);
+    }
+
+    int hi = 32 - __clz(kmin ^ kmax);
+    unsigned prefix = hi >= 32 ? 0u : (kmax >> hi);
+    unsigned need = (unsigned)take;
+    unsigned *cnt0 = cluster.map_shared_rank(&s_cnt, 0);
+    uint32_t *list0 = cluster.map_shared_rank(s_list, 0);
+    const unsigned *dec0 = cluster.map_shared_rank(s_dec, 0);
+    // Rounds on the register-resident slices (two cluster barriers each) until the threshold bin is small
+    // enough for the shared list; CTA 0 then finishes alone with CTA-local barriers only.
+    while (hi > 0) {
+        const int w = min(8, hi), shift = hi - w;
+        const unsigned dmask = (1u << w) - 1u;
+        if (tid < 256) hist[tid] = 0;
+        __syncthreads();
+#pragma unroll
+        for (int e = 0; e < E; ++e) {
+            const bool live = (j0 + e < nc) && (hi >= 32 || (key[e] >> hi) == prefix);
+            if (live) atomicAdd(&hist[(key[e] >> shift) & dmask], 1u);
+        }
+        cluster.sync();   // every CTA's histogram is complete
+        if (rank == 0) {
+            if (tid < 256) {
+                unsigned tsum = hist[tid];
+#pragma unroll
+                for (int r = 1; r < CL; ++r) tsum += cluster.map_shared_rank(hist, r)[tid];
+                s_sum[tid] = tsum;
+            }
+            __syncthreads();
+            if (warp == 0) pick_digit(s_sum, prefix, need, lane, &s_prefix, &s_need);
+            __syncthreads();
+            if (tid == 0) {
+                const unsigned digit = s_prefix & 255u;
+                s_dec[0] = digit; s_dec[1] = s_need; s_dec[2] = s_sum[digit];
+                s_cnt = 0;
+            }
+        }
+        cluster.sync();   // the decision is published (and every remote histogram read is over)
+        const unsigned digit = dec0[0], in_bin = dec0[2];
+        need = dec0[1];
+        prefix = (hi >= 32 ? 0u : (prefix << w)) | digit;
+        hi = shift;
+        if (hi > 0 && in_bin <= kListCap) {   // uniform over the cluster
+#pragma unroll
+            for (int e = 0; e < E; ++e)
+                if (j0 + e < nc && (key[e] >> hi) == prefix) {
+                    const unsigned slot = atomicAdd(cnt0, 1u);
+                    if (slot < kListCap) list0[slot] = key[e];
+                }
+            cluster.sync();   // the list is complete
+            if (rank == 0) {
+                const unsigned n_list = min(s_cnt, kListCap);
+                while (hi > 0) {
+                    const int w2 = min(8, hi), shift2 = hi - w2;
+                    const unsigned dmask2 = (1u << w2) - 1u;
+                    if (tid < 256) hist[tid] = 0;
+                    __syncthreads();
+                    for (unsigned t = tid; t < n_list; t += THREADS) {
+                        const uint32_t kk = s_list[t];
+                        if ((kk >> hi) == prefix) atomicAdd(&hist[(kk >> shift2) & dmask2], 1u);
+                    }
+                    __syncthreads();
+                    if (warp == 0) pick_digit(hist, prefix, need, lane, &s_prefix, &s_need);
+                    __syncthreads();
+                    prefix = (prefix << w2) | (s_prefix & 255u);
+                    need = s_need;
+                    hi = shift2;
+                    __syncthreads();   // s_prefix / hist are reused by the next round
+                }
+                if (tid == 0) { s_dec[0] = prefix; s_dec[1] = need; }
+            }
+            cluster.sync();   // the final threshold is published
+            prefix = dec0[0];
+            need = dec0[1];
+            hi = 0;
+        }
+        // CTA 0 overwrites s_dec only after a later cluster.sync, when every CTA has read it
+    }
+    const uint32_t tau = prefix;
+    const unsigned need_eq = need;
+
+    // ---- ordered compaction: block scan inside the CTA, totals of the lower-ranked CTAs through DSMEM
+    unsigned n_gt = 0, n_eq = 0;
+#pragma unroll
+    for (int e = 0; e < E; ++e) {
+        const bool ok = j0 + e < nc;
+        n_gt += ok && key[e] > tau;
+        n_eq += ok && key[e] == tau;
+    }
+    const unsigned packed = (n_gt << 16) | n_eq;   // per-CTA totals stay below 65536
+    unsigned incl = packed;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const unsigned t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+    }
+    if (lane == 31) s_warp[warp] = incl;
+    __syncthreads();
+    unsigned wsum = lane < WARPS ? s_warp[lane] : 0u;
+    unsigned wincl = wsum;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const unsigned t = __shfl_up_sync(0xffffffffu, wincl, o);
+        if (lane >= o) wincl += t;
+    }
+    const unsigned excl = __shfl_sync(0xffffffffu, wincl - wsum, warp) + incl - packed;
+    const unsigned cta_total = __shfl_sync(0xffffffffu, wincl, WARPS - 1);
+    if (tid == 0) { s_tot[0] = cta_total >> 16; s_tot[1] = cta_total & 0xffffu; }
+    cluster.sync();
+    unsigned gt_before = excl >> 16, eq_before = excl & 0xffffu;
+    for (unsigned r = 0; r < rank; ++r) {
+        const unsigned *tot = cluster.map_shared_rank(s_tot, r);
+        gt_before += tot[0]; eq_before += tot[1];
+    }
+#pragma unroll
+    for (int e = 0; e < E; ++e) {
+        if (j0 + e >= nc) continue;
+        if (key[e] > tau) {
+            out[gt_before + min(eq_before, need_eq)] = j0 + e;
+            ++gt_before;
+        } else if (key[e] == tau) {
+            if (eq_before < need_eq) out[gt_before + eq_before] = j0 + e;
+            ++eq_before;
+        }
+    }
+    if (rank == 0)
+        for (int t = take + tid; t < p.k; t += THREADS) out[t] = -1;
+    cluster.sync();   // nobody leaves while its shared memory may still be read by a neighbour
+}
+
 // ---- longer rows: re-read from memory for every pass -------------------------------------------
 // THREADS threads per row, kItems consecutive candidates per thread per step.
 template <int THREADS, int ITEMS, bool CACHED, bool VEC>
 __global__ void __launch_bounds__(THREADS)
 k_topk(const Params p, const float *__restrict__ scores, int64_t score_stride, int32_t *__restrict__ idx,
-       int64_t row0)
+       int64_t row0, int nc_lo, int nc_hi)
 {
     constexpr int WARPS = THREADS / 32;
     constexpr int CHUNK = THREADS * kItems;           // candidates per step
@@ -239,6 +447,7 @@ k_topk(const Params p, const float *__restrict__ scores, int64_t score_stride, i
     const int kvl = kvlen_of(p, b);
     const int pos = pos_of(p, b, i);
     const int nc = max(0, min(pos - p.w + 1, kvl));   // candidates are keys 0..nc-1
+    if (nc <= nc_lo || nc > nc_hi) return;   // this row belongs to another variant's launch
     const int take = min(p.k, nc);
     int32_t *out = idx + row * p.k;
     const float *srow = scores + (int64_t)blockIdx.x * score_stride;
@@ -367,29 +576,29 @@ k_topk(const Params p, const float *__restrict__ scores, int64_t score_stride, i
 
 }  // namespace
 
-template <int THREADS, int ITEMS, bool CACHED>
-void launch_variant(const Params &p, const float *scores, int64_t score_stride, int32_t *idx, int64_t row0, int64_t n_rows,
-                    bool vec, cudaStream_t st)
-{
-    if (vec)
-        k_topk<THREADS, ITEMS, CACHED, true><<<(unsigned)n_rows, THREADS, 0, st>>>(p, scores, score_stride, idx, row0);
-    else
-        k_topk<THREADS, ITEMS, CACHED, false><<<(unsigned)n_rows, THREADS, 0, st>>>(p, scores, score_stride, idx, row0);
-}
+// Variants by the number of candidates of a row: (lo, hi] -> kernel.  A launch covers every row of the
+// block; rows outside the variant's range leave at once, so each row is handled by exactly one launch
+// and the choice is per row even when the positions live on the device.
+struct TopkClass { int lo, hi; };
+constexpr TopkClass kClasses[6] = {{-1, 8192}, {8192, 32768}, {32768, 65536}, {65536, 131072}, {131072, 262144},
+                                   {262144, 0x7fffffff}};
 
-// one launch of the variant that fits rows of at most `max_nc` candidates
-void launch_rows(const Params &p, const float *scores, int64_t score_stride, int32_t *idx, int64_t row0, int64_t n_rows,
-                 int max_nc, bool vec, cudaStream_t st)
+template <bool VEC>
+void launch_class(int c, const Params &p, const float *scores, int64_t score_stride, int32_t *idx, int64_t row0,
+                  int64_t n_rows, cudaStream_t st)
 {
-    if (n_rows <= 0) return;
-    if (max_nc <= 256 * 32) {
-        if (vec) k_topk_cached<256, 32, true><<<(unsigned)n_rows, 256, 0, st>>>(p, scores, score_stride, idx, row0);
-        else k_topk_cached<256, 32, false><<<(unsigned)n_rows, 256, 0, st>>>(p, scores, score_stride, idx, row0);
-    } else if (max_nc <= 512 * 64) {
-        if (vec) k_topk_cached<512, 64, true><<<(unsigned)n_rows, 512, 0, st>>>(p, scores, score_stride, idx, row0);
-        else k_topk_cached<512, 64, false><<<(unsigned)n_rows, 512, 0, st>>>(p, scores, score_stride, idx, row0);
-    } else {
-        launch_variant<1024, kItems, false>(p, scores, score_stride, idx, row0, n_rows, vec, st);
+    const int lo = kClasses[c].lo, hi = kClasses[c].hi;
+    const unsigned n = (unsigned)n_rows;
+#ifdef HS2_TOPK_NO_CLUSTER
+    if (c >= 2 && c <= 4) c = 5;   // tuning builds: long rows on the streaming kernel
+#endif
+    switch (c) {
+        case 0: k_topk_cached<256, 32, VEC><<<n, 256, 0, st>>>(p, scores, score_stride, idx, row0, lo, hi); break;
+        case 1: k_topk_cached<512, 64, VEC><<<n, 512, 0, st>>>(p, scores, score_stride, idx, row0, lo, hi); break;
+        case 2: k_topk_cluster<2, VEC><<<n * 2, 512, 0, st>>>(p, scores, score_stride, idx, row0, lo, hi); break;
+        case 3: k_topk_cluster<4, VEC><<<n * 4, 512, 0, st>>>(p, scores, score_stride, idx, row0, lo, hi); break;
+        case 4: k_topk_cluster<8, VEC><<<n * 8, 512, 0, st>>>(p, scores, score_stride, idx, row0, lo, hi); break;
+        default: k_topk<1024, kItems, false, VEC><<<n, 1024, 0, st>>>(p, scores, score_stride, idx, row0, lo, hi); break;
     }
     count_launch();
 }
@@ -399,35 +608,22 @@ cudaError_t launch_topk(const Params &p, const float *scores, int64_t score_stri
 {
     if (n_rows == 0 || p.k == 0) return cudaSuccess;
     const bool vec = (score_stride % 4 == 0) && (reinterpret_cast<uintptr_t>(scores) % 16 == 0);
-    if (p.q_start || p.kv_lens || p.Lk <= 256 * 32) {
-        // positions live on the device (or every row is short): one variant sized for the longest possible row
-        launch_rows(p, scores, score_stride, idx, row0, n_rows, p.Lk, vec, st);
-        return cudaGetLastError();
+    // range of candidate counts that can occur in this block of rows
+    int64_t nc_min = 0, nc_max = p.Lk;
+    if (!p.q_start && !p.kv_lens) {
+        // host-known positions: query i has clamp(Lk - Lq + i - w + 1, 0, Lk) candidates, growing with i
+        const int64_t base = (int64_t)p.Lk - p.Lq - p.w + 1;
+        const int64_t i_first = row0 % p.Lq, i_last = (row0 + n_rows - 1) % p.Lq;
+        const bool wraps = (row0 / p.Lq) != ((row0 + n_rows - 1) / p.Lq);
+        const int64_t i_lo = wraps ? 0 : i_first, i_hi = wraps ? p.Lq - 1 : i_last;
+        auto clampnc = [&](int64_t v) { return v < 0 ? (int64_t)0 : (v > p.Lk ? (int64_t)p.Lk : v); };
+        nc_min = clampnc(base + i_lo);
+        nc_max = clampnc(base + i_hi);
     }
-    // Positions are known on the host: query i of a sequence has min(max(Lk - Lq + i - w + 1, 0), Lk)
-    // candidates, growing with i.  Cut the row range where that count crosses a variant's capacity, so
-    // that the short rows at the start of each sequence run on the cheaper register-resident variants.
-    const int64_t caps[2] = {256 * 32, 512 * 64};
-    const int64_t base = (int64_t)p.Lk - p.Lq - p.w + 1;   // candidates of query 0 (before clamping)
-    int64_t r = row0;
-    const int64_t r_end = row0 + n_rows;
-    while (r < r_end) {
-        const int64_t bg = r / p.Lq;
-        const int64_t seg_end = (bg + 1) * p.Lq < r_end ? (bg + 1) * p.Lq : r_end;   // rows of one (sequence, KV head)
-        int64_t i = r - bg * p.Lq;
-        const int64_t i_end = seg_end - bg * p.Lq;
-        while (i < i_end) {
-            int64_t nc = base + i;
-            nc = nc < 0 ? 0 : (nc > p.Lk ? (int64_t)p.Lk : nc);
-            const int64_t cap = nc <= caps[0] ? caps[0] : (nc <= caps[1] ? caps[1] : (int64_t)p.Lk);
-            int64_t last = cap >= p.Lk ? i_end : cap - base + 1;   // base + q <= cap  <=>  q < last
-            if (last > i_end) last = i_end;
-            if (last <= i) last = i + 1;
-            const int64_t first_row = bg * p.Lq + i;
-            launch_rows(p, scores + (first_row - row0) * score_stride, score_stride, idx, first_row, last - i, (int)cap, vec, st);
-            i = last;
-        }
-        r = seg_end;
+    for (int c = 0; c < 6; ++c) {
+        if (nc_max <= kClasses[c].lo || nc_min > kClasses[c].hi) continue;   // no row of the block falls in this class
+        if (vec) launch_class<true>(c, p, scores, score_stride, idx, row0, n_rows, st);
+        else launch_class<false>(c, p, scores, score_stride, idx, row0, n_rows, st);
     }
     return cudaGetLastError();
 }

@@ -87,7 +87,19 @@ def test_topk_adversarial_rows():
         _topk_case(scores, k, w, q_start=[Lk - 1 - len(rows) + 1])
 
 
-@pytest.mark.parametrize("Lk", [8192, 20000, 40000])
+@pytest.mark.parametrize("Lk,k,w", [(40000, 2048, 128), (70001, 4096, 256), (131072, 4096, 256), (200003, 1000, 17),
+                                     (262144, 4096, 0), (300000, 512, 64)])
+def test_topk_long_rows_cluster_and_streaming_variants(Lk, k, w):
+    """Rows beyond 32768 candidates: cluster kernels of 2, 4 and 8 CTAs, and the streaming kernel above that."""
+    g = torch.Generator().manual_seed(Lk)
+    s = torch.randn(1, 2, 6, Lk, generator=g) - 9.0
+    s[0, 0, 1] = (s[0, 0, 1] * 2).round() / 2                      # heavy ties
+    s[0, 1, 2] = -5.0                                              # all equal
+    _topk_case(s, k, w, q_start=[Lk - 6])
+    _topk_case(s, k, w, q_start=[Lk // 2])                         # rows that fall into a smaller variant
+
+
+@pytest.mark.parametrize("Lk", [8192, 20000, 40000, 100000])
 def test_topk_threshold_bin_larger_than_the_shared_list(Lk):
     """Few distinct values over long rows: the bin that holds the k-th value has thousands of members,
     so the register kernels must fall back from their shared-memory candidate list (both variants),
@@ -145,6 +157,24 @@ def test_small_block_every_row(name, over):
     for layer in range(len(run.qs)):
         out, lse = run.run_sparse(layer)
         run.check_sparse(out, lse, layer)
+
+
+def test_paper_native_shape_mqa64_dim256_with_sink():
+    """The attention shape of the paper's own model (Table 1: 64 query heads / 1 KV head, head dim 256,
+    128 forced local + 1024 global tokens, per-head sink bias in the sparse layers), scaled in length."""
+    wl = scaled("cfg2", q_len=1536, kv_len=1536, n_q_heads=64, n_kv_heads=1, head_dim=256, k_sel=1024, window=128,
+                n_needles=8)
+    run = BlockRun(make_inputs(wl)).run_full()
+    rows = [(0, i) for i in (0, 127, 128, 1151, 1152, 1300, 1535)]
+    run.check_full(rows=rows)
+    sink = torch.linspace(-2.0, 2.0, 64, device="cuda")
+    out, lse = run.run_sparse(0, sink=sink)
+    run.check_sparse(out, lse, 0, rows=rows, sink=sink)
+    q1 = run.qs[0][:, -1:].contiguous()
+    prob1 = hs2.Problem.from_tensors(q1, run.k, wl.k_sel, wl.window)
+    od, _ = hs2.hs2_sparse_attn_decode(prob1, q1, run.k, run.v, run.idx[:, :, -1:].contiguous(), sink=sink)
+    torch.cuda.synchronize()
+    assert (od.float() - out[:, -1:].float()).abs().max().item() <= 2e-2
 
 
 def test_ragged_lengths_offsets_strides_and_sink():
