@@ -177,6 +177,11 @@ int hs2_last_cuda_error(void);
  * window).  Sticky until the process exits.  Synchronises the current device.  Returns an hs2_status. */
 int hs2_device_error_flags(unsigned *flags);
 
+/* Tuning knob of hs2_full_attn_select: from which kv_len on the selection thresholds a sample of the scores
+ * and works on filtered candidate lists instead of complete score strips (default 65537; both ways give the
+ * same indices).  Returns the previous value; min_keys <= 0 only queries.  Process-wide. */
+int hs2_set_filter_min_keys(int min_keys);
+
 /* Number of kernels this library has launched in the process so far (all threads, all streams). */
 unsigned long long hs2_launch_count(void);
 

@@ -24,7 +24,7 @@ HS2_OP_FULL_ATTN_SELECT, HS2_OP_TOPK_SELECT, HS2_OP_SPARSE_ATTN_PREFILL, HS2_OP_
 
 EXPORTS = ["hs2_workspace_bytes", "hs2_full_attn_select", "hs2_topk_select", "hs2_sparse_attn_prefill",
            "hs2_sparse_attn_decode", "hs2_sparse_attn_decode_static", "hs2_status_string", "hs2_last_cuda_error",
-           "hs2_launch_count", "hs2_device_error_flags"]
+           "hs2_launch_count", "hs2_device_error_flags", "hs2_set_filter_min_keys"]
 
 
 class HS2Error(RuntimeError):
@@ -80,6 +80,11 @@ def hs2_device_error_flags() -> int:
     v = C.c_uint(0)
     _check(load_library().hs2_device_error_flags(C.byref(v)), "hs2_device_error_flags")
     return int(v.value)
+
+
+def hs2_set_filter_min_keys(min_keys: int) -> int:
+    """Tuning knob: kv_len from which the full layer's selection uses filtered candidate lists; returns the old value."""
+    return int(load_library().hs2_set_filter_min_keys(int(min_keys)))
 
 
 def hs2_launch_count() -> int:

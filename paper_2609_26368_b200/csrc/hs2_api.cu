@@ -75,6 +75,51 @@ size_t full_select_ws_bytes(const Params &p)
     return align_up(rows * row, 256);
 }
 
+// ---- filtered selection (sampled threshold -> ordered candidate lists -> select) ----
+constexpr int kFilterSamp = 8;              // every 8th key tile is scored for the threshold
+// The filtered path wins only when rows are long (measured: 131072 keys 485 ms vs 580 ms with strips, 32768
+// keys 67 ms vs 64 ms, 8192 keys 3.7 ms vs 2.1 ms): shorter contexts keep the strips.
+std::atomic<int> g_filter_min_keys{65537};
+constexpr size_t kFilterBigCap = (size_t)1 << 30;
+
+struct FilterPlan {
+    bool ok;
+    int cap;          // candidates kept per row
+    int ns_w;         // sampled scores per row (padded to whole tiles)
+    size_t per_row;   // bytes of the big region per row (sample strip, later the candidate lists)
+};
+
+FilterPlan filter_plan(const Params &p, hs2_dtype dt)
+{
+    FilterPlan f{};
+    // expected list length: samp * (r + 6 sqrt(r)) with r the threshold rank at the thinnest sampling (1/samp)
+    const double m = (double)p.k / kFilterSamp, r = m + 5.0 * sqrt(m) + 2.0;
+    const int want = (int)(kFilterSamp * (r + 6.0 * sqrt(r))) + 64;
+    f.cap = ((want > 1024 ? want : 1024) + 255) / 256 * 256;
+    f.ns_w = filter_sample_width(p, kFilterSamp);
+    f.per_row = align_up((size_t)f.ns_w * 4, 16);
+    if ((size_t)f.cap * 8 > f.per_row) f.per_row = (size_t)f.cap * 8;
+    f.ok = p.k > 0 && scores_filter_supported(p, dt) && f.cap <= 32768 && f.ns_w <= 32768 && p.Lk > f.cap &&
+           p.Lk >= g_filter_min_keys.load(std::memory_order_relaxed) && select_rows(p) >= 1024;
+    return f;
+}
+
+int64_t filter_block_rows(const FilterPlan &f, int64_t rows, size_t ws_bytes)
+{
+    const size_t budget = ws_bytes < kFilterBigCap + (size_t)(16 << 20) ? ws_bytes : kFilterBigCap + (size_t)(16 << 20);
+    if (budget < 4096) return 0;
+    int64_t r = (int64_t)((budget - 4096) / (f.per_row + 12));
+    return r > rows ? rows : r;
+}
+
+size_t filter_ws_bytes(const FilterPlan &f, int64_t rows)
+{
+    int64_t r = (int64_t)(kFilterBigCap / f.per_row);
+    if (r > rows) r = rows;
+    if (r < 1) r = 1;
+    return align_up((size_t)r * (f.per_row + 12) + 4096, 256);
+}
+
 bool ws_ok(const void *ws, size_t ws_bytes, size_t need)
 {
     if (need == 0) return true;
@@ -134,6 +179,11 @@ size_t hs2_workspace_bytes(const hs2_problem *hp, hs2_op op)
             if (resolve(hp, true, &p) != HS2_OK) return 0;
             {
                 size_t need = p.k > 0 ? full_select_ws_bytes(p) : 0;
+                const FilterPlan fp = filter_plan(p, hp->dtype);
+                if (fp.ok) {
+                    const size_t fneed = filter_ws_bytes(fp, select_rows(p));
+                    if (fneed > need) need = fneed;
+                }
                 if (p.Lq == 1 && sparse_mma_supported(p, hp->dtype)) {   // the decode-shaped layer may split over the keys
                     Params pd = p;
                     pd.k = 0; pd.w = p.Lk;
@@ -202,6 +252,37 @@ hs2_status hs2_full_attn_select(const hs2_problem *hp, const void *Q, const void
         }
         return HS2_OK;
     }
+    // Filtered path: a 1/8-sampled sweep gives every row a threshold that (with verification) lies below its
+    // k-th score; the main sweep then keeps only the (score, key) pairs at or above it, in key order, and the
+    // selection runs on those short lists.  Rows whose list came out too short or too long are redone exactly.
+    const FilterPlan fp = filter_plan(p, dt);
+    const bool al = aligned16(Q, K, V, O);
+    if (fp.ok && al && reinterpret_cast<uintptr_t>(ws) % 256 == 0) {
+        int64_t block = filter_block_rows(fp, rows, ws_bytes);
+        if (block > kMaxBlockRows) block = kMaxBlockRows;
+        if (block >= (rows < 1024 ? rows : 1024)) {
+            char *base = (char *)ws;
+            uint32_t *tau = (uint32_t *)base;
+            int *count = (int *)(base + (size_t)block * 4);
+            int *flag = (int *)(base + (size_t)block * 8);
+            char *big = base + align_up((size_t)block * 12, 256);
+            float *sample = (float *)big;
+            float *cand_a = (float *)big;
+            int32_t *cand_j = (int32_t *)(big + (size_t)block * fp.cap * 4);
+            bool usable = true;
+            for (int64_t r0 = 0; r0 < rows && usable; r0 += block) {
+                const int64_t n = rows - r0 < block ? rows - r0 : block;
+                e = launch_scores_sampled_tc5(p, Q, K, LSE, sample, fp.ns_w, r0, n, kFilterSamp, st);
+                if (e == cudaErrorNotSupported && r0 == 0) { usable = false; break; }   // nothing launched yet: use the strips
+                if (e != cudaSuccess) return cuda_fail(e);
+                if ((e = launch_filter_thresholds(p, sample, fp.ns_w, r0, n, kFilterSamp, fp.cap, tau, flag, st)) != cudaSuccess) return cuda_fail(e);
+                if ((e = launch_scores_filter_tc5(p, Q, K, LSE, r0, n, tau, cand_a, cand_j, count, fp.cap, st)) != cudaSuccess) return cuda_fail(e);
+                if ((e = launch_filter_select(p, cand_a, cand_j, count, fp.cap, idx, r0, n, flag, st)) != cudaSuccess) return cuda_fail(e);
+                if ((e = launch_select_recompute(p, Q, K, LSE, idx, r0, n, flag, st)) != cudaSuccess) return cuda_fail(e);
+            }
+            if (usable) return HS2_OK;
+        }
+    }
     // bounded strips: score a block of query rows into the workspace, select from it, move on
     const int64_t stride = (int64_t)(row_bytes / sizeof(float));
     int64_t block = (int64_t)((ws_bytes < kStripCapBytes ? ws_bytes : kStripCapBytes) / row_bytes);
@@ -211,7 +292,7 @@ hs2_status hs2_full_attn_select(const hs2_problem *hp, const void *Q, const void
     float *strip = (float *)ws;
     for (int64_t r0 = 0; r0 < rows; r0 += block) {
         const int64_t n = rows - r0 < block ? rows - r0 : block;
-        e = launch_scores(p, dt, mma, aligned16(Q, K, V, O), Q, K, LSE, strip, stride, r0, n, false, st);
+        e = launch_scores(p, dt, mma, al, Q, K, LSE, strip, stride, r0, n, false, st);
         if (e != cudaSuccess) return cuda_fail(e);
         if ((e = launch_topk(p, strip, stride, idx, r0, n, st)) != cudaSuccess) return cuda_fail(e);
     }
@@ -299,6 +380,13 @@ int hs2_device_error_flags(unsigned *flags)
     if (!flags) return HS2_ERR_INVALID_ARG;
     cudaError_t e = read_tc5_error(flags);
     return e == cudaSuccess ? HS2_OK : cuda_fail(e);
+}
+
+int hs2_set_filter_min_keys(int min_keys)
+{
+    const int old = g_filter_min_keys.load(std::memory_order_relaxed);
+    if (min_keys > 0) g_filter_min_keys.store(min_keys, std::memory_order_relaxed);
+    return old;
 }
 
 unsigned long long hs2_launch_count(void) { return g_launches.load(std::memory_order_relaxed); }

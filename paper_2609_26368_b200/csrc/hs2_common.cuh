@@ -77,6 +77,15 @@ cudaError_t launch_sparse_generic(const Params &p, hs2_dtype dt, const void *Q, 
 cudaError_t launch_topk(const Params &p, const float *scores, int64_t score_stride, int32_t *idx,
                         int64_t row0, int64_t n_rows, cudaStream_t st);
 
+// Filtered selection: thresholds from sampled strips, selection from candidate lists, exact redo of flagged rows.
+int filter_sample_width(const Params &p, int samp);
+cudaError_t launch_filter_thresholds(const Params &p, const float *sample, int64_t stride, int64_t row0, int64_t n_rows,
+                                     int samp, int cap, uint32_t *tau_key, int *flag, cudaStream_t st);
+cudaError_t launch_filter_select(const Params &p, const float *cand_a, const int32_t *cand_j, const int *count, int cap,
+                                 int32_t *idx, int64_t row0, int64_t n_rows, int *flag, cudaStream_t st);
+cudaError_t launch_select_recompute(const Params &p, const void *Q, const void *K, const float *LSE, int32_t *idx,
+                                    int64_t row0, int64_t n_rows, const int *flag, cudaStream_t st);
+
 // Tensor-core bf16 kernels (head_dim 128, group <= 8).
 bool sparse_mma_supported(const Params &p, hs2_dtype dt);
 cudaError_t launch_sparse_mma_prefill(const Params &p, const void *Q, const void *K, const void *V, const int32_t *idx,
@@ -105,6 +114,12 @@ cudaError_t launch_full_attn_tc5(const Params &p, const void *Q, const void *K, 
 bool scores_tc5_supported(const Params &p, hs2_dtype dt);
 cudaError_t launch_scores_tc5(const Params &p, const void *Q, const void *K, const float *LSE, float *out,
                               int64_t out_stride, int64_t row0, int64_t n_rows, bool all_visible, cudaStream_t st);
+bool scores_filter_supported(const Params &p, hs2_dtype dt);
+cudaError_t launch_scores_sampled_tc5(const Params &p, const void *Q, const void *K, const float *LSE, float *out,
+                                      int64_t out_stride, int64_t row0, int64_t n_rows, int samp, cudaStream_t st);
+cudaError_t launch_scores_filter_tc5(const Params &p, const void *Q, const void *K, const float *LSE, int64_t row0,
+                                     int64_t n_rows, const uint32_t *tau_key, float *cand_a, int32_t *cand_j, int *count,
+                                     int cap, cudaStream_t st);
 cudaError_t read_tc5_error(unsigned *out);
 
 }  // namespace hs2

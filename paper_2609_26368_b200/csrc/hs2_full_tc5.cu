@@ -385,18 +385,43 @@ constexpr uint32_t kScOffK = 32768;               // 2 stages x [2 halves][128 k
 constexpr uint32_t kScOffNl = kScOffK + 2 * 32768;   // float[128]: -LSE/scale per column
 constexpr uint32_t kScOffNq = kScOffNl + 512;     // int[128]: keys needed per query
 constexpr uint32_t kScOffRow = kScOffNq + 512;    // int64[128]: strip row of each query
-constexpr uint32_t kScOffBar = kScOffRow + 1024;
+constexpr uint32_t kScOffTau = kScOffRow + 1024;  // uint32[32]: filter threshold per query (filter mode)
+constexpr uint32_t kScOffCnt = kScOffTau + 128;   // int[2][4][32]: per-warp pass counts, two tile parities
+constexpr uint32_t kScOffBar = kScOffCnt + 1024;
 constexpr uint32_t kScSmemBytes = kScOffBar + kBarBytes + kAlignSlack;
 enum ScBar { SQ_FULL = 0, SK_FULL0, SK_FULL1, SK_EMPTY0, SK_EMPTY1, ACC_FULL0, ACC_FULL1, ACC_FREE0, ACC_FREE1, SC_N_BARS };
 
-template <int G>
+// What the sweep does with a score:
+//   SC_STRIP   write it to the strip row at its key position (keys split into chunks over blockIdx.x)
+//   SC_SAMPLE  only every `samp`-th key tile is computed; written compactly (tile t of the sample at 128 t)
+//   SC_FILTER  one CTA sweeps all keys of its queries in order and appends (score, key) of every score
+//              whose order key is >= the query's threshold to that query's candidate list, in key order
+enum { SC_STRIP = 0, SC_SAMPLE = 1, SC_FILTER = 2 };
+
+struct FilterBuf {
+    const uint32_t *tau_key;   // [rows of the block] threshold as order-preserving key
+    float *cand_a;             // [rows][cap]
+    int32_t *cand_j;           // [rows][cap]
+    int *count;                // [rows] candidates found (may exceed cap: then the row is redone elsewhere)
+    int cap;
+};
+
+__device__ __forceinline__ uint32_t order_key_f(float f)
+{
+    uint32_t u = __float_as_uint(f);
+    if (u == 0x80000000u) u = 0u;
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+
+template <int G, int MODE>
 __global__ void __launch_bounds__(kThreads, 2)
 k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, const Params p,
              const float *__restrict__ LSE, float *__restrict__ out, int64_t out_stride, int64_t row0, int64_t n_rows,
-             int all_visible, int tile_first, int tiles_per_bg)
+             int all_visible, int tile_first, int tiles_per_bg, int samp, FilterBuf fb)
 {
     constexpr int TQ = 128 / G;          // queries per CTA
     constexpr int QPC = 32 / G > 0 ? 32 / G : 1;   // queries per 32-column chunk (G <= 32)
+    static_assert(MODE != SC_FILTER || TQ <= 32, "filter mode keeps one counter per query in registers");
     extern __shared__ char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t pad = (1024u - (raw & 1023u)) & 1023u;
@@ -413,8 +438,10 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     float *s_nl = reinterpret_cast<float *>(smem + kScOffNl);
     int *s_nq = reinterpret_cast<int *>(smem + kScOffNq);
     int64_t *s_row = reinterpret_cast<int64_t *>(smem + kScOffRow);
+    uint32_t *s_tau = reinterpret_cast<uint32_t *>(smem + kScOffTau);
+    int *s_cntw = reinterpret_cast<int *>(smem + kScOffCnt);
 
-    const int tid = threadIdx.x, warp = tid >> 5;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int tile = tile_first + blockIdx.y;   // flattened (b, g, query tile)
     const int bg = tile / tiles_per_bg;
     const int qt = tile % tiles_per_bg;
@@ -430,10 +457,20 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         return max(0, min(all_visible ? pos + 1 : pos - p.w + 1, kvl));
     };
     const int limit = n_of(c_hi - 1);
-    const int key0 = blockIdx.x * SC_KCHUNK;
-    const int key_end = min(limit, key0 + SC_KCHUNK);
-    if (key0 >= key_end) return;
-    const int ntile = (key_end - key0 + 127) / 128;
+    // key tiles of this CTA: tile t of the loop is key tile (kt0 + t) * kstep
+    const int kstep = MODE == SC_SAMPLE ? samp : 1;
+    const int kt0 = MODE == SC_FILTER ? 0 : blockIdx.x * (SC_KCHUNK / 128);
+    const int tiles_total = (limit + 128 * kstep - 1) / (128 * kstep);   // key tiles (of this stride) that start below the limit
+    const int ntile = MODE == SC_FILTER ? tiles_total : min(SC_KCHUNK / 128, tiles_total - kt0);
+    if (MODE == SC_FILTER) {
+        if (blockIdx.x != 0) return;
+        if (ntile <= 0) {   // no candidates at all: the lists are empty
+            if (tid < TQ && iq0 + tid >= c_lo && iq0 + tid < c_hi) fb.count[bg_row0 + iq0 + tid - row0] = 0;
+            return;
+        }
+    } else if (ntile <= 0) {
+        return;
+    }
 
     if (tid < 128) {   // per-column constants
         const int t = tid / G, hh = tid % G;
@@ -442,7 +479,8 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         s_nl[tid] = ok ? -LSE[((int64_t)b * p.Hq + gkv * G + hh) * p.Lq + i] / p.scale : 0.f;
         if (hh == 0) {
             s_nq[t] = ok ? n_of(i) : 0;
-            s_row[t] = ok ? (bg_row0 + i - row0) : 0;
+            s_row[t] = ok ? (bg_row0 + i - row0) : -1;
+            if (MODE == SC_FILTER && t < 32) s_tau[t] = ok ? fb.tau_key[bg_row0 + i - row0] : 0xffffffffu;
         }
     }
     if (tid == 0) {
@@ -475,8 +513,9 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 issued = t + 1;
                 mbar_expect_tx(bar(SK_FULL0 + st), 32768);
                 const uint32_t kdst = sbase + kScOffK + st * 32768;
-                tma_load_4d(kdst, &tmK, bar(SK_FULL0 + st), 0, gkv, key0 + t * 128, b);
-                tma_load_4d(kdst + 16384, &tmK, bar(SK_FULL0 + st), 64, gkv, key0 + t * 128, b);
+                const int krow = (kt0 + t) * kstep * 128;
+                tma_load_4d(kdst, &tmK, bar(SK_FULL0 + st), 0, gkv, krow, b);
+                tma_load_4d(kdst + 16384, &tmK, bar(SK_FULL0 + st), 64, gkv, krow, b);
             }
             if (*abort_flag) {
                 for (int t = max(0, issued - 2); t < issued; ++t)
@@ -506,16 +545,29 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     } else {
         const int row = tid;   // key inside the tile = TMEM lane
         const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
+        int run[MODE == SC_FILTER ? TQ : 1];   // candidates appended so far, per query (filter mode)
+#pragma unroll
+        for (int q = 0; q < (MODE == SC_FILTER ? TQ : 1); ++q) run[q] = 0;
+        bool alive = true;
         for (int t = 0; t < ntile; ++t) {
             const int ab = t & 1;
-            if (!__all_sync(0xffffffffu, mbar_wait(bar(ACC_FULL0 + ab), (t >> 1) & 1, abort_flag))) break;
+            if (alive && !__all_sync(0xffffffffu, mbar_wait(bar(ACC_FULL0 + ab), (t >> 1) & 1, abort_flag))) alive = false;
+            if (MODE != SC_FILTER && !alive) break;
             tc_fence_after();
-            const int key = key0 + t * 128 + row;
+            const int key = (kt0 + t) * kstep * 128 + row;
+            const int col = MODE == SC_SAMPLE ? (kt0 + t) * 128 + row : key;
+            float aval[MODE == SC_FILTER ? TQ : 1];
+            unsigned passbits = 0;
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 float v[32];
-                tmem_ld32(lane_base + ab * 128 + c * 32, v);
-                tmem_wait_ld();
+                if (alive) {
+                    tmem_ld32(lane_base + ab * 128 + c * 32, v);
+                    tmem_wait_ld();
+                } else {
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) v[e] = 0.f;
+                }
                 const float4 *nl4 = reinterpret_cast<const float4 *>(s_nl + c * 32);
 #pragma unroll
                 for (int e4 = 0; e4 < 8; ++e4) {
@@ -528,11 +580,51 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
 #pragma unroll
                     for (int hh = 1; hh < G; ++hh) a = fmaxf(a, v[q * G + hh]);
                     const int tq = c * QPC + q;
-                    if (key < s_nq[tq]) out[s_row[tq] * out_stride + key] = a * p.scale;
+                    const float av = a * p.scale;
+                    if (MODE == SC_FILTER) {
+                        aval[tq] = av;
+                        const bool pass = alive && key < s_nq[tq] && order_key_f(av) >= s_tau[tq];
+                        passbits |= (pass ? 1u : 0u) << tq;
+                    } else {
+                        if (key < s_nq[tq]) out[s_row[tq] * out_stride + col] = av;
+                    }
                 }
             }
-            tc_fence_before();
-            mbar_arrive(bar(ACC_FREE0 + ab));
+            if (alive) {
+                tc_fence_before();
+                mbar_arrive(bar(ACC_FREE0 + ab));
+            }
+            if (MODE == SC_FILTER) {
+                // ordered append: keys of this tile in (warp, lane) order, after everything appended before
+                unsigned bal[TQ];
+                int *cw = s_cntw + ab * 4 * 32;
+#pragma unroll
+                for (int q = 0; q < TQ; ++q) {
+                    bal[q] = __ballot_sync(0xffffffffu, (passbits >> q) & 1u);
+                    if (lane == q) cw[warp * 32 + q] = __popc(bal[q]);
+                }
+                asm volatile("bar.sync 1, 128;\n" ::: "memory");   // the four epilogue warps, every tile, abort or not
+                const unsigned lt = (1u << lane) - 1u;
+#pragma unroll
+                for (int q = 0; q < TQ; ++q) {
+                    const int c0 = cw[q], c1 = cw[32 + q], c2 = cw[64 + q], c3 = cw[96 + q];
+                    const int before = warp == 0 ? 0 : (warp == 1 ? c0 : (warp == 2 ? c0 + c1 : c0 + c1 + c2));
+                    if ((passbits >> q) & 1u) {
+                        const int pos = run[q] + before + __popc(bal[q] & lt);
+                        if (pos < fb.cap) {
+                            const int64_t o = s_row[q] * fb.cap + pos;
+                            fb.cand_a[o] = aval[q];
+                            fb.cand_j[o] = key;
+                        }
+                    }
+                    run[q] += c0 + c1 + c2 + c3;
+                }
+            }
+        }
+        if (MODE == SC_FILTER) {
+#pragma unroll
+            for (int q = 0; q < TQ; ++q)
+                if (tid == q && s_row[q] >= 0) fb.count[s_row[q]] = alive ? run[q] : -1;   // -1: this CTA gave up
         }
     }
     __syncwarp();
@@ -617,16 +709,17 @@ cudaError_t launch_full_attn_tc5(const Params &p, const void *Q, const void *K, 
     return cudaGetLastError();
 }
 
-template <int G>
-cudaError_t launch_scores_tc5_g(const CUtensorMap &tmQ, const CUtensorMap &tmK, const Params &p, const float *LSE, float *out,
-                                int64_t out_stride, int64_t row0, int64_t n_rows, bool all_visible, cudaStream_t st)
+template <int G, int MODE>
+cudaError_t launch_sc(const CUtensorMap &tmQ, const CUtensorMap &tmK, const Params &p, const float *LSE, float *out,
+                      int64_t out_stride, int64_t row0, int64_t n_rows, bool all_visible, int samp, const FilterBuf &fb,
+                      cudaStream_t st)
 {
     static bool attr_set[64] = {};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (!(dev >= 0 && dev < 64 && attr_set[dev])) {
-        if ((e = cudaFuncSetAttribute(k_scores_tc5<G>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kScSmemBytes)) != cudaSuccess) return e;
+        if ((e = cudaFuncSetAttribute(k_scores_tc5<G, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kScSmemBytes)) != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
     constexpr int TQ = 128 / G;
@@ -637,11 +730,33 @@ cudaError_t launch_scores_tc5_g(const CUtensorMap &tmQ, const CUtensorMap &tmK, 
     const int64_t t_last = (last / p.Lq) * tiles_per_bg + (last % p.Lq) / TQ;
     const int64_t gy = t_last - t_first + 1;
     if (gy > 65535 || t_last > 0x7fffffffLL) return cudaErrorNotSupported;
-    dim3 grid((p.Lk + SC_KCHUNK - 1) / SC_KCHUNK, (unsigned)gy);
-    k_scores_tc5<G><<<grid, kThreads, kScSmemBytes, st>>>(tmQ, tmK, p, LSE, out, out_stride, row0, n_rows, all_visible ? 1 : 0,
-                                                         (int)t_first, tiles_per_bg);
+    const int key_tiles = (p.Lk + 128 * samp - 1) / (128 * samp);
+    const unsigned gx = MODE == SC_FILTER ? 1u : (unsigned)((key_tiles + SC_KCHUNK / 128 - 1) / (SC_KCHUNK / 128));
+    dim3 grid(gx, (unsigned)gy);
+    k_scores_tc5<G, MODE><<<grid, kThreads, kScSmemBytes, st>>>(tmQ, tmK, p, LSE, out, out_stride, row0, n_rows, all_visible ? 1 : 0,
+                                                               (int)t_first, tiles_per_bg, samp, fb);
     count_launch();
     return cudaGetLastError();
+}
+
+template <int MODE>
+cudaError_t launch_sc_mode(const Params &p, const void *Q, const void *K, const float *LSE, float *out, int64_t out_stride,
+                           int64_t row0, int64_t n_rows, bool all_visible, int samp, const FilterBuf &fb, cudaStream_t st)
+{
+    if (n_rows == 0) return cudaSuccess;
+    CUtensorMap tmQ, tmK;
+    if (!make_map(&tmQ, Q, p.B, p.Lq, p.Hq, p.qs_b, p.qs_t, p.qs_h, 128 / p.G, p.G) ||
+        !make_map(&tmK, K, p.B, p.Lk, p.Hkv, p.ks_b, p.ks_t, p.ks_h, 128))
+        return cudaErrorNotSupported;
+    if ((n_rows + p.Lq) / (128 / p.G) + 2 * (int64_t)p.B * p.Hkv > 65535) return cudaErrorNotSupported;   // grid.y bound
+    switch (p.G) {
+        case 1: if (MODE == SC_FILTER) return cudaErrorNotSupported; return launch_sc<1, MODE == SC_FILTER ? SC_STRIP : MODE>(tmQ, tmK, p, LSE, out, out_stride, row0, n_rows, all_visible, samp, fb, st);
+        case 2: if (MODE == SC_FILTER) return cudaErrorNotSupported; return launch_sc<2, MODE == SC_FILTER ? SC_STRIP : MODE>(tmQ, tmK, p, LSE, out, out_stride, row0, n_rows, all_visible, samp, fb, st);
+        case 4: return launch_sc<4, MODE>(tmQ, tmK, p, LSE, out, out_stride, row0, n_rows, all_visible, samp, fb, st);
+        case 8: return launch_sc<8, MODE>(tmQ, tmK, p, LSE, out, out_stride, row0, n_rows, all_visible, samp, fb, st);
+        case 16: return launch_sc<16, MODE>(tmQ, tmK, p, LSE, out, out_stride, row0, n_rows, all_visible, samp, fb, st);
+    }
+    return cudaErrorNotSupported;
 }
 
 bool scores_tc5_supported(const Params &p, hs2_dtype dt)
@@ -650,30 +765,42 @@ bool scores_tc5_supported(const Params &p, hs2_dtype dt)
     return g_ok && full_tc5_supported(p, dt);
 }
 
+// shape test only (no driver query): workspace sizes must not depend on the machine
+bool scores_filter_supported(const Params &p, hs2_dtype dt)
+{
+    auto m8 = [](int64_t x) { return x % 8 == 0 && x > 0; };
+    return (p.G == 4 || p.G == 8 || p.G == 16) && dt == HS2_BF16 && p.D == HD && m8(p.qs_b) && m8(p.qs_t) && m8(p.qs_h) &&
+           m8(p.ks_b) && m8(p.ks_t) && m8(p.ks_h) && (int64_t)p.B * p.Hq <= 65535;
+}
+
 // Returns cudaErrorNotSupported when the launch cannot be set up (the caller then takes the mma.sync sweep).
 cudaError_t launch_scores_tc5(const Params &p, const void *Q, const void *K, const float *LSE, float *out,
                               int64_t out_stride, int64_t row0, int64_t n_rows, bool all_visible, cudaStream_t st)
 {
     if (n_rows == 0) return cudaSuccess;
-    CUtensorMap tmQ, tmK;
-    if (!make_map(&tmQ, Q, p.B, p.Lq, p.Hq, p.qs_b, p.qs_t, p.qs_h, 128 / p.G, p.G) ||
-        !make_map(&tmK, K, p.B, p.Lk, p.Hkv, p.ks_b, p.ks_t, p.ks_h, 128))
-        return cudaErrorNotSupported;
-    if ((n_rows + p.Lq) / (128 / p.G) + 2 * (int64_t)p.B * p.Hkv > 65535) return cudaErrorNotSupported;   // grid.y bound
     if (all_visible) {   // keys a query cannot see read -inf
         const int64_t n = n_rows * out_stride;
         const int64_t fb = (n + 255) / 256;
         k_fill_tc5<<<(unsigned)(fb < 148 * 16 ? fb : 148 * 16), 256, 0, st>>>(out, n, -INFINITY);
         count_launch();
     }
-    switch (p.G) {
-        case 1: return launch_scores_tc5_g<1>(tmQ, tmK, p, LSE, out, out_stride, row0, n_rows, all_visible, st);
-        case 2: return launch_scores_tc5_g<2>(tmQ, tmK, p, LSE, out, out_stride, row0, n_rows, all_visible, st);
-        case 4: return launch_scores_tc5_g<4>(tmQ, tmK, p, LSE, out, out_stride, row0, n_rows, all_visible, st);
-        case 8: return launch_scores_tc5_g<8>(tmQ, tmK, p, LSE, out, out_stride, row0, n_rows, all_visible, st);
-        case 16: return launch_scores_tc5_g<16>(tmQ, tmK, p, LSE, out, out_stride, row0, n_rows, all_visible, st);
-    }
-    return cudaErrorNotSupported;
+    return launch_sc_mode<SC_STRIP>(p, Q, K, LSE, out, out_stride, row0, n_rows, all_visible, 1, FilterBuf{}, st);
+}
+
+// Scores of every `samp`-th key tile, written compactly: sampled tile t at columns 128 t .. 128 t + 127.
+cudaError_t launch_scores_sampled_tc5(const Params &p, const void *Q, const void *K, const float *LSE, float *out,
+                                      int64_t out_stride, int64_t row0, int64_t n_rows, int samp, cudaStream_t st)
+{
+    return launch_sc_mode<SC_SAMPLE>(p, Q, K, LSE, out, out_stride, row0, n_rows, false, samp, FilterBuf{}, st);
+}
+
+// Ordered candidate lists: every (score, key) whose order key is >= tau_key[row], in key order.
+cudaError_t launch_scores_filter_tc5(const Params &p, const void *Q, const void *K, const float *LSE, int64_t row0,
+                                     int64_t n_rows, const uint32_t *tau_key, float *cand_a, int32_t *cand_j, int *count,
+                                     int cap, cudaStream_t st)
+{
+    FilterBuf fb{tau_key, cand_a, cand_j, count, cap};
+    return launch_sc_mode<SC_FILTER>(p, Q, K, LSE, nullptr, 0, row0, n_rows, false, 1, fb, st);
 }
 
 // Device error word of the tcgen05 kernels (0 = no bounded wait ever ran out).  Synchronises the device.

@@ -74,10 +74,40 @@ __device__ __forceinline__ void pick_digit(const unsigned *hist, unsigned prefix
 // output is (thread, element) order and the ordered compaction needs a single block scan.  The radix
 // digits are taken below the common leading bits of the row's smallest and largest key, which makes
 // the first round spread the candidates over all 256 bins (log-probabilities share their top bits).
-template <int THREADS, int E, bool VEC>
+// What the register-resident select works on:
+//   SEL_ROW   a score row indexed by key (the plain entry point and the strip path)
+//   SEL_TAU   the sampled scores of a row: only the value at a given rank is wanted (the filter threshold)
+//   SEL_CAND  the filtered candidates of a row, in key order, with their key indices as payload
+enum { SEL_ROW = 0, SEL_TAU = 1, SEL_CAND = 2 };
+
+struct SelArgs {
+    int samp;                 // SEL_TAU: every samp-th key tile was scored
+    int cap;                  // candidate capacity per row (rows with at most cap keys keep every key)
+    uint32_t *tau_key;        // SEL_TAU out: [rows of the block]
+    int *flag;                // SEL_TAU: cleared; SEL_CAND: set when the row has to be redone exactly
+    const int *count;         // SEL_CAND: candidates found per row
+    const int32_t *payload;   // SEL_CAND: [rows][cap] key index of each candidate
+};
+
+// sampled scores of a row with n candidates: every samp-th tile of 128 keys, the last one possibly partial
+__host__ __device__ __forceinline__ int sample_size(int n, int samp)
+{
+    const int q = n / (samp * 128), rem = n - q * samp * 128;
+    return q * 128 + (rem < 128 ? rem : 128);
+}
+// Rank (from the top) of the sample whose value is a safe lower bound of the row's take-th largest score.
+// The sample holds n_s of the row's n keys; of the row's top `take` about take * n_s / n fall into it, and
+// the rank is put five standard deviations above that mean (short rows sample more than 1/samp of their keys).
+__device__ __forceinline__ int sample_rank(int take, int n, int n_s)
+{
+    const float m = (float)take * (float)n_s / (float)n;
+    return (int)(m + 5.f * sqrtf(m) + 2.f);
+}
+
+template <int THREADS, int E, bool VEC, int MODE>
 __global__ void __launch_bounds__(THREADS, THREADS <= 256 ? 3 : 1)
 k_topk_cached(const Params p, const float *__restrict__ scores, int64_t score_stride, int32_t *__restrict__ idx,
-              int64_t row0, int nc_lo, int nc_hi)
+              int64_t row0, int nc_lo, int nc_hi, SelArgs sa)
 {
     constexpr int WARPS = THREADS / 32;
     __shared__ unsigned hist[256];
@@ -92,15 +122,39 @@ k_topk_cached(const Params p, const float *__restrict__ scores, int64_t score_st
     const int b = (int)(row / ((int64_t)p.Lq * p.Hkv));
     const int kvl = kvlen_of(p, b);
     const int pos = pos_of(p, b, i);
-    const int nc = max(0, min(pos - p.w + 1, kvl));   // candidates are keys 0..nc-1
+    const int n_keys = max(0, min(pos - p.w + 1, kvl));   // the row's candidates are keys 0..n_keys-1
+    const int k_row = min(p.k, n_keys);                   // how many of them are selected
+    // what this launch selects from (nc entries) and how many (take)
+    int nc = n_keys, take = k_row;
+    if (MODE == SEL_TAU) {
+        nc = sample_size(n_keys, sa.samp);
+        take = n_keys > 0 ? min(nc, sample_rank(k_row, n_keys, nc)) : 0;
+    }
+    if (MODE == SEL_CAND) nc = sa.cap;   // one variant serves every row of this launch
     if (nc <= nc_lo || nc > nc_hi) return;   // this row belongs to another variant's launch
-    const int take = min(p.k, nc);
     int32_t *out = idx + row * p.k;
     const float *srow = scores + (int64_t)blockIdx.x * score_stride;
+    const int32_t *prow = MODE == SEL_CAND ? sa.payload + (int64_t)blockIdx.x * sa.cap : nullptr;
 
-    if (take == nc) {   // every candidate is kept: no need to look at the scores
-        for (int t = tid; t < p.k; t += THREADS) out[t] = t < nc ? t : -1;
-        return;
+    if (MODE == SEL_TAU) {
+        if (tid == 0) sa.flag[blockIdx.x] = 0;
+        if (n_keys <= sa.cap || take <= 0) {   // short row: every key is a candidate
+            if (tid == 0) sa.tau_key[blockIdx.x] = 0u;
+            return;
+        }
+    } else {
+        if (k_row == n_keys) {   // every candidate is kept: no need to look at the scores
+            for (int t = tid; t < p.k; t += THREADS) out[t] = t < n_keys ? t : -1;
+            return;
+        }
+        if (MODE == SEL_CAND) {
+            const int cnt = sa.count[blockIdx.x];
+            if (cnt < k_row || cnt > sa.cap) {   // the threshold was off (or the sweep gave up): redo this row exactly
+                if (tid == 0) sa.flag[blockIdx.x] = 1;
+                return;
+            }
+            nc = cnt;
+        }
     }
     const int j0 = tid * E;
     uint32_t key[E];
@@ -179,6 +233,10 @@ k_topk_cached(const Params p, const float *__restrict__ scores, int64_t score_st
     }
     const uint32_t tau = hi == 0 && kmin == kmax ? kmax : prefix;   // key of the take-th largest candidate
     const unsigned need_eq = need;                                   // equal keys kept, lowest indices first
+    if (MODE == SEL_TAU) {
+        if (tid == 0) sa.tau_key[blockIdx.x] = tau;
+        return;
+    }
 
     // ---- ordered compaction with one block scan
     unsigned n_gt = 0, n_eq = 0;
@@ -210,10 +268,10 @@ k_topk_cached(const Params p, const float *__restrict__ scores, int64_t score_st
     for (int e = 0; e < E; ++e) {
         if (j0 + e >= nc) continue;
         if (key[e] > tau) {
-            out[gt_before + min(eq_before, need_eq)] = j0 + e;
+            out[gt_before + min(eq_before, need_eq)] = MODE == SEL_CAND ? prow[j0 + e] : j0 + e;
             ++gt_before;
         } else if (key[e] == tau) {
-            if (eq_before < need_eq) out[gt_before + eq_before] = j0 + e;
+            if (eq_before < need_eq) out[gt_before + eq_before] = MODE == SEL_CAND ? prow[j0 + e] : j0 + e;
             ++eq_before;
         }
     }
@@ -593,8 +651,8 @@ void launch_class(int c, const Params &p, const float *scores, int64_t score_str
     if (c >= 2 && c <= 4) c = 5;   // tuning builds: long rows on the streaming kernel
 #endif
     switch (c) {
-        case 0: k_topk_cached<256, 32, VEC><<<n, 256, 0, st>>>(p, scores, score_stride, idx, row0, lo, hi); break;
-        case 1: k_topk_cached<512, 64, VEC><<<n, 512, 0, st>>>(p, scores, score_stride, idx, row0, lo, hi); break;
+        case 0: k_topk_cached<256, 32, VEC, SEL_ROW><<<n, 256, 0, st>>>(p, scores, score_stride, idx, row0, lo, hi, SelArgs{}); break;
+        case 1: k_topk_cached<512, 64, VEC, SEL_ROW><<<n, 512, 0, st>>>(p, scores, score_stride, idx, row0, lo, hi, SelArgs{}); break;
         case 2: k_topk_cluster<2, VEC><<<n * 2, 512, 0, st>>>(p, scores, score_stride, idx, row0, lo, hi); break;
         case 3: k_topk_cluster<4, VEC><<<n * 4, 512, 0, st>>>(p, scores, score_stride, idx, row0, lo, hi); break;
         case 4: k_topk_cluster<8, VEC><<<n * 8, 512, 0, st>>>(p, scores, score_stride, idx, row0, lo, hi); break;
@@ -625,6 +683,159 @@ cudaError_t launch_topk(const Params &p, const float *scores, int64_t score_stri
         if (vec) launch_class<true>(c, p, scores, score_stride, idx, row0, n_rows, st);
         else launch_class<false>(c, p, scores, score_stride, idx, row0, n_rows, st);
     }
+    return cudaGetLastError();
+}
+
+
+// ---- exact redo of flagged rows -------------------------------------------------------------------
+// The filtered pipeline marks a row when its candidate count came out below the number to select or
+// above the list capacity (the sampled threshold was off, which needs adversarially structured scores).
+// Such a row is selected here from scores recomputed on the fly, pass by pass (bf16 inputs, fp32 FMAs):
+// slow, but it needs no storage, no host round trip, and handles any number of rows.
+namespace {
+
+__global__ void __launch_bounds__(256)
+k_select_recompute(const Params p, const __nv_bfloat16 *__restrict__ Q, const __nv_bfloat16 *__restrict__ K,
+                   const float *__restrict__ LSE, int32_t *__restrict__ idx, int64_t row0, const int *__restrict__ flag)
+{
+    constexpr int THREADS = 256, WARPS = 8, D = 128;
+    extern __shared__ float sq[];                 // [G][128] queries, then [G] LSE
+    __shared__ unsigned hist[256];
+    __shared__ unsigned s_warp[WARPS];
+    __shared__ unsigned s_prefix, s_need, s_run_gt, s_run_eq;
+    if (!flag[blockIdx.x]) return;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int64_t row = row0 + blockIdx.x;
+    const int i = (int)(row % p.Lq);
+    const int g = (int)((row / p.Lq) % p.Hkv);
+    const int b = (int)(row / ((int64_t)p.Lq * p.Hkv));
+    const int kvl = kvlen_of(p, b);
+    const int pos = pos_of(p, b, i);
+    const int nc = max(0, min(pos - p.w + 1, kvl));
+    const int take = min(p.k, nc);
+    int32_t *out = idx + row * p.k;
+    float *slse = sq + p.G * D;
+    for (int e = tid; e < p.G * D; e += THREADS)
+        sq[e] = __bfloat162float(Q[b * p.qs_b + (int64_t)i * p.qs_t + (g * p.G + e / D) * p.qs_h + e % D]);
+    for (int e = tid; e < p.G; e += THREADS) slse[e] = LSE[((int64_t)b * p.Hq + g * p.G + e) * p.Lq + i];
+    __syncthreads();
+    const __nv_bfloat16 *kb = K + b * p.ks_b + g * p.ks_h;
+    auto key_of = [&](int j) -> uint32_t {   // order key of a[j] = max_h (scale <q_h, k_j> - LSE_h)
+        const uint4 *kr = reinterpret_cast<const uint4 *>(kb + (int64_t)j * p.ks_t);
+        float kf[D];
+#pragma unroll
+        for (int c = 0; c < D / 8; ++c) {
+            const uint4 v = __ldg(kr + c);
+            const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+#pragma unroll
+            for (int t = 0; t < 4; ++t) { kf[8 * c + 2 * t] = __uint_as_float(w[t] << 16); kf[8 * c + 2 * t + 1] = __uint_as_float(w[t] & 0xffff0000u); }
+        }
+        float best = -INFINITY;
+        for (int h = 0; h < p.G; ++h) {
+            float acc = 0.f;
+#pragma unroll
+            for (int d = 0; d < D; ++d) acc = fmaf(kf[d], sq[h * D + d], acc);
+            best = fmaxf(best, fmaf(acc, p.scale, -slse[h]));
+        }
+        return order_key(best);
+    };
+    unsigned prefix = 0, need = (unsigned)take;
+    for (int round = 0; round < 4; ++round) {
+        const int shift = 24 - 8 * round;
+        hist[tid] = 0;
+        __syncthreads();
+        for (int base = 0; base < nc; base += THREADS) {
+            const int j = base + tid;
+            const uint32_t kk = j < nc ? key_of(j) : 0u;
+            const bool live = j < nc && (round == 0 || (kk >> (shift + 8)) == prefix);
+            const unsigned digit = live ? ((kk >> shift) & 255u) : 256u;
+            const unsigned peers = __match_any_sync(0xffffffffu, digit);
+            if (live && lane == __ffs(peers) - 1) atomicAdd(&hist[digit], __popc(peers));
+        }
+        __syncthreads();
+        if (warp == 0) pick_digit(hist, prefix, need, lane, &s_prefix, &s_need);
+        __syncthreads();
+        prefix = s_prefix;
+        need = s_need;
+    }
+    const uint32_t tau = prefix;
+    const unsigned need_eq = need;
+    if (tid == 0) { s_run_gt = 0; s_run_eq = 0; }
+    __syncthreads();
+    for (int base = 0; base < nc; base += THREADS) {
+        const int j = base + tid;
+        const uint32_t kk = j < nc ? key_of(j) : 0u;
+        const unsigned gt = j < nc && kk > tau, eq = j < nc && kk == tau;
+        const unsigned bg = __ballot_sync(0xffffffffu, gt), be = __ballot_sync(0xffffffffu, eq);
+        if (lane == 0) s_warp[warp] = (__popc(bg) << 16) | __popc(be);
+        __syncthreads();
+        unsigned gt_before = s_run_gt, eq_before = s_run_eq, tot_gt = 0, tot_eq = 0;
+#pragma unroll
+        for (int w2 = 0; w2 < WARPS; ++w2) {
+            const unsigned c = s_warp[w2];
+            if (w2 < warp) { gt_before += c >> 16; eq_before += c & 0xffffu; }
+            tot_gt += c >> 16; tot_eq += c & 0xffffu;
+        }
+        const unsigned lt = (1u << lane) - 1u;
+        gt_before += __popc(bg & lt);
+        eq_before += __popc(be & lt);
+        if (gt) out[gt_before + min(eq_before, need_eq)] = j;
+        else if (eq && eq_before < need_eq) out[gt_before + eq_before] = j;
+        __syncthreads();
+        if (tid == 0) { s_run_gt += tot_gt; s_run_eq += tot_eq; }
+        __syncthreads();
+    }
+    for (int t = take + tid; t < p.k; t += THREADS) out[t] = -1;
+}
+
+}  // namespace
+
+int filter_sample_width(const Params &p, int samp)
+{
+    return ((p.Lk + 128 * samp - 1) / (128 * samp)) * 128;   // sampled scores per row, padded to whole tiles
+}
+
+// thresholds tau_key[row] from the sampled strips (row stride `stride` floats); clears flag[row]
+cudaError_t launch_filter_thresholds(const Params &p, const float *sample, int64_t stride, int64_t row0, int64_t n_rows,
+                                     int samp, int cap, uint32_t *tau_key, int *flag, cudaStream_t st)
+{
+    if (n_rows == 0) return cudaSuccess;
+    SelArgs sa{samp, cap, tau_key, flag, nullptr, nullptr};
+    const unsigned n = (unsigned)n_rows;
+    const int ns_max = filter_sample_width(p, samp);
+    // class by the size of the row's sample (every row is taken by exactly one launch)
+    k_topk_cached<256, 32, true, SEL_TAU><<<n, 256, 0, st>>>(p, sample, stride, nullptr, row0, -1, 8192, sa);
+    count_launch();
+    if (ns_max > 8192) {
+        k_topk_cached<512, 64, true, SEL_TAU><<<n, 512, 0, st>>>(p, sample, stride, nullptr, row0, 8192, 32768, sa);
+        count_launch();
+    }
+    return cudaGetLastError();
+}
+
+// final selection from the candidate lists; rows whose count is out of range get flag[row] = 1
+cudaError_t launch_filter_select(const Params &p, const float *cand_a, const int32_t *cand_j, const int *count, int cap,
+                                 int32_t *idx, int64_t row0, int64_t n_rows, int *flag, cudaStream_t st)
+{
+    if (n_rows == 0) return cudaSuccess;
+    SelArgs sa{1, cap, nullptr, flag, count, cand_j};
+    const unsigned n = (unsigned)n_rows;
+    if (cap <= 8192)
+        k_topk_cached<256, 32, true, SEL_CAND><<<n, 256, 0, st>>>(p, cand_a, cap, idx, row0, -1, 0x7fffffff, sa);
+    else
+        k_topk_cached<512, 64, true, SEL_CAND><<<n, 512, 0, st>>>(p, cand_a, cap, idx, row0, -1, 0x7fffffff, sa);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_select_recompute(const Params &p, const void *Q, const void *K, const float *LSE, int32_t *idx,
+                                    int64_t row0, int64_t n_rows, const int *flag, cudaStream_t st)
+{
+    if (n_rows == 0) return cudaSuccess;
+    const size_t smem = sizeof(float) * ((size_t)p.G * 128 + p.G);
+    k_select_recompute<<<(unsigned)n_rows, 256, smem, st>>>(p, (const __nv_bfloat16 *)Q, (const __nv_bfloat16 *)K, LSE, idx,
+                                                            row0, flag);
+    count_launch();
     return cudaGetLastError();
 }
 

@@ -48,7 +48,8 @@ def test_workspace_sizes_are_host_side(lib):
     assert hs2.hs2_workspace_bytes(p, binding.HS2_OP_TOPK_SELECT) == 0
     assert hs2.hs2_workspace_bytes(p, binding.HS2_OP_SPARSE_ATTN_PREFILL) == 0
     big = _prob(q_len=131072, kv_len=131072, n_q_heads=32, n_kv_heads=4, head_dim=128, dtype=torch.bfloat16)
-    assert hs2.hs2_workspace_bytes(big, binding.HS2_OP_FULL_ATTN_SELECT) == 1 << 30     # capped strips
+    n = hs2.hs2_workspace_bytes(big, binding.HS2_OP_FULL_ATTN_SELECT)                   # capped, whatever the path
+    assert (1 << 30) <= n <= (1 << 30) + (1 << 20)
     assert hs2.hs2_workspace_bytes(_prob(n_q_heads=3, n_kv_heads=2), binding.HS2_OP_FULL_ATTN_SELECT) == 0
 
 

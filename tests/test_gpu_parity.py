@@ -159,6 +159,65 @@ def test_small_block_every_row(name, over):
         run.check_sparse(out, lse, layer)
 
 
+def test_filtered_selection_equals_selection_on_the_full_score_rows():
+    """bf16 tensor-core path: without scores_dbg the layer thresholds a 1/8 sample, keeps ordered candidate lists
+    and selects from them; with scores_dbg it selects from complete score rows.  Same scores, same indices."""
+    old = hs2.hs2_set_filter_min_keys(1)          # force the filtered path on these small shapes
+    try:
+        _filtered_equals_full_rows()
+    finally:
+        hs2.hs2_set_filter_min_keys(old)
+
+
+def _filtered_equals_full_rows():
+    for over in (dict(q_len=4096, kv_len=4096, k_sel=256, window=64, n_needles=16),
+                 dict(q_len=700, kv_len=6000, k_sel=512, window=128, n_needles=16, batch=2),
+                 dict(q_len=1500, kv_len=3000, k_sel=300, window=0, n_q_heads=16, n_kv_heads=4, n_needles=8)):
+        inp = make_inputs(scaled("cfg2", **over))
+        a = BlockRun(inp).run_full(want_scores=True)
+        b = BlockRun(inp).run_full(want_scores=False)
+        assert torch.equal(a.idx, b.idx)
+        assert hs2.hs2_device_error_flags() == 0
+
+
+def test_filtered_selection_redoes_rows_whose_sample_misleads():
+    """Scores that depend on the key tile's phase defeat a tile-strided sample: the threshold comes out too
+    high (lists shorter than k) or too low (lists overflow).  Those rows must be redone exactly."""
+    old = hs2.hs2_set_filter_min_keys(1)
+    try:
+        _filtered_redo()
+    finally:
+        hs2.hs2_set_filter_min_keys(old)
+
+
+def _filtered_redo():
+    wl = scaled("cfg2", q_len=2048, kv_len=8192, k_sel=512, window=32, n_needles=4)
+    for sampled_high in (True, False):
+        inp = make_inputs(wl)
+        tile = (torch.arange(wl.kv_len) // 128) % 8 == 0                  # the key tiles the sample looks at
+        scale_rows = torch.where(tile == sampled_high, 3.0, 0.05).to(inp.k.dtype)
+        # keys of the favoured tiles line up with every query (large logits), the others are near zero
+        inp.k.mul_(scale_rows.view(1, -1, 1, 1))
+        run = BlockRun(inp)
+        n_rows = wl.batch * wl.n_kv_heads * wl.q_len
+        from paper_2609_26368_b200 import binding
+        ws = torch.zeros(hs2.hs2_workspace_bytes(run.prob, binding.HS2_OP_FULL_ATTN_SELECT), dtype=torch.uint8, device="cuda")
+        run.run_full(want_scores=False, ws=ws)
+        # white box: the workspace starts with threshold, count and flag words per row (one block here)
+        flags = ws[: 12 * n_rows].view(torch.int32)[2 * n_rows: 3 * n_rows]
+        assert int(flags.sum()) > n_rows // 4, "the adversarial rows were not sent to the exact redo"
+        rows = [(0, i) for i in (0, 600, 1500, 2047)]
+        run.check_full(rows=rows)
+        ref = BlockRun(inp).run_full(want_scores=True)
+        assert torch.equal(run.idx, ref.idx)
+    # and ordinary data does not need the redo at all
+    inp = make_inputs(wl)
+    run = BlockRun(inp)
+    ws = torch.zeros(hs2.hs2_workspace_bytes(run.prob, binding.HS2_OP_FULL_ATTN_SELECT), dtype=torch.uint8, device="cuda")
+    run.run_full(want_scores=False, ws=ws)
+    assert int(ws[: 12 * n_rows].view(torch.int32)[2 * n_rows: 3 * n_rows].sum()) == 0
+
+
 def test_paper_native_shape_mqa64_dim256_with_sink():
     """The attention shape of the paper's own model (Table 1: 64 query heads / 1 KV head, head dim 256,
     128 forced local + 1024 global tokens, per-head sink bias in the sparse layers), scaled in length."""
