@@ -386,7 +386,7 @@ constexpr uint32_t kScOffNl = kScOffK + 2 * 32768;   // float[128]: -LSE/scale p
 constexpr uint32_t kScOffNq = kScOffNl + 512;     // int[128]: keys needed per query
 constexpr uint32_t kScOffRow = kScOffNq + 512;    // int64[128]: strip row of each query
 constexpr uint32_t kScOffTau = kScOffRow + 1024;  // uint32[32]: filter threshold per query (filter mode)
-constexpr uint32_t kScOffCnt = kScOffTau + 128;   // int[2][4][32]: per-warp pass counts, two tile parities
+constexpr uint32_t kScOffCnt = kScOffTau + 128;   // int[32]: candidates appended per query (filter mode)
 constexpr uint32_t kScOffBar = kScOffCnt + 1024;
 constexpr uint32_t kScSmemBytes = kScOffBar + kBarBytes + kAlignSlack;
 enum ScBar { SQ_FULL = 0, SK_FULL0, SK_FULL1, SK_EMPTY0, SK_EMPTY1, ACC_FULL0, ACC_FULL1, ACC_FREE0, ACC_FREE1, SC_N_BARS };
@@ -394,8 +394,8 @@ enum ScBar { SQ_FULL = 0, SK_FULL0, SK_FULL1, SK_EMPTY0, SK_EMPTY1, ACC_FULL0, A
 // What the sweep does with a score:
 //   SC_STRIP   write it to the strip row at its key position (keys split into chunks over blockIdx.x)
 //   SC_SAMPLE  only every `samp`-th key tile is computed; written compactly (tile t of the sample at 128 t)
-//   SC_FILTER  one CTA sweeps all keys of its queries in order and appends (score, key) of every score
-//              whose order key is >= the query's threshold to that query's candidate list, in key order
+//   SC_FILTER  one CTA sweeps all keys of its queries and appends (score, key) of every score whose order key
+//              is >= the query's threshold to that query's candidate list (in no particular order)
 enum { SC_STRIP = 0, SC_SAMPLE = 1, SC_FILTER = 2 };
 
 struct FilterBuf {
@@ -442,7 +442,8 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     int *s_cntw = reinterpret_cast<int *>(smem + kScOffCnt);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int tile = tile_first + blockIdx.y;   // flattened (b, g, query tile)
+    // flattened (b, g, query tile); the filter sweep walks all keys per CTA, so its long tiles (late queries) go first
+    const int tile = tile_first + (MODE == SC_FILTER ? (int)(gridDim.y - 1 - blockIdx.y) : (int)blockIdx.y);
     const int bg = tile / tiles_per_bg;
     const int qt = tile % tiles_per_bg;
     const int gkv = bg % p.Hkv, b = bg / p.Hkv;
@@ -480,7 +481,10 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         if (hh == 0) {
             s_nq[t] = ok ? n_of(i) : 0;
             s_row[t] = ok ? (bg_row0 + i - row0) : -1;
-            if (MODE == SC_FILTER && t < 32) s_tau[t] = ok ? fb.tau_key[bg_row0 + i - row0] : 0xffffffffu;
+            if (MODE == SC_FILTER && t < 32) {
+                s_tau[t] = ok ? fb.tau_key[bg_row0 + i - row0] : 0xffffffffu;
+                s_cntw[t] = 0;
+            }
         }
     }
     if (tid == 0) {
@@ -545,9 +549,6 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     } else {
         const int row = tid;   // key inside the tile = TMEM lane
         const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
-        int run[MODE == SC_FILTER ? TQ : 1];   // candidates appended so far, per query (filter mode)
-#pragma unroll
-        for (int q = 0; q < (MODE == SC_FILTER ? TQ : 1); ++q) run[q] = 0;
         bool alive = true;
         for (int t = 0; t < ntile; ++t) {
             const int ab = t & 1;
@@ -595,36 +596,24 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 mbar_arrive(bar(ACC_FREE0 + ab));
             }
             if (MODE == SC_FILTER) {
-                // ordered append: keys of this tile in (warp, lane) order, after everything appended before
-                unsigned bal[TQ];
-                int *cw = s_cntw + ab * 4 * 32;
+                // append in no particular order: one shared-memory counter per query.  Only a few percent of the
+                // scores pass, so a plain atomic per passing element is cheaper than any warp-level aggregation.
 #pragma unroll
                 for (int q = 0; q < TQ; ++q) {
-                    bal[q] = __ballot_sync(0xffffffffu, (passbits >> q) & 1u);
-                    if (lane == q) cw[warp * 32 + q] = __popc(bal[q]);
-                }
-                asm volatile("bar.sync 1, 128;\n" ::: "memory");   // the four epilogue warps, every tile, abort or not
-                const unsigned lt = (1u << lane) - 1u;
-#pragma unroll
-                for (int q = 0; q < TQ; ++q) {
-                    const int c0 = cw[q], c1 = cw[32 + q], c2 = cw[64 + q], c3 = cw[96 + q];
-                    const int before = warp == 0 ? 0 : (warp == 1 ? c0 : (warp == 2 ? c0 + c1 : c0 + c1 + c2));
                     if ((passbits >> q) & 1u) {
-                        const int pos = run[q] + before + __popc(bal[q] & lt);
+                        const int pos = atomicAdd(&s_cntw[q], 1);
                         if (pos < fb.cap) {
                             const int64_t o = s_row[q] * fb.cap + pos;
                             fb.cand_a[o] = aval[q];
                             fb.cand_j[o] = key;
                         }
                     }
-                    run[q] += c0 + c1 + c2 + c3;
                 }
             }
         }
         if (MODE == SC_FILTER) {
-#pragma unroll
-            for (int q = 0; q < TQ; ++q)
-                if (tid == q && s_row[q] >= 0) fb.count[s_row[q]] = alive ? run[q] : -1;   // -1: this CTA gave up
+            asm volatile("bar.sync 1, 128;\n" ::: "memory");   // the four epilogue warps: all appends are counted
+            if (tid < TQ && s_row[tid] >= 0) fb.count[s_row[tid]] = (alive && !*abort_flag) ? s_cntw[tid] : -1;   // -1: gave up
         }
     }
     __syncwarp();

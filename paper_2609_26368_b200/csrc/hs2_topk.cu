@@ -74,6 +74,56 @@ __device__ __forceinline__ void pick_digit(const unsigned *hist, unsigned prefix
 // output is (thread, element) order and the ordered compaction needs a single block scan.  The radix
 // digits are taken below the common leading bits of the row's smallest and largest key, which makes
 // the first round spread the candidates over all 256 bins (log-probabilities share their top bits).
+
+// value of the `need`-th largest of list[0..n) (n >= need >= 1): four 8-bit rounds, CTA-wide, on a shared list
+template <int THREADS>
+__device__ __forceinline__ uint32_t select_on_list(const uint32_t *list, unsigned n, unsigned need, unsigned *hist,
+                                                   unsigned *s_prefix, unsigned *s_need, int tid, int lane, int warp)
+{
+    unsigned prefix = 0;
+    for (int round = 0; round < 4; ++round) {
+        const int shift = 24 - 8 * round;
+        if (tid < 256) hist[tid] = 0;
+        if (THREADS < 256) for (int t = tid + THREADS; t < 256; t += THREADS) hist[t] = 0;
+        __syncthreads();
+        for (unsigned t = tid; t < n; t += THREADS) {
+            const uint32_t kk = list[t];
+            if (round == 0 || (kk >> (shift + 8)) == prefix) atomicAdd(&hist[(kk >> shift) & 255u], 1u);
+        }
+        __syncthreads();
+        if (warp == 0) pick_digit(hist, prefix, need, lane, s_prefix, s_need);
+        __syncthreads();
+        prefix = *s_prefix;
+        need = *s_need;
+        __syncthreads();
+    }
+    return prefix;
+}
+
+// exclusive prefix of `v` over the CTA in thread order; *total receives the sum (s_warp: WARPS words)
+template <int WARPS>
+__device__ __forceinline__ unsigned block_excl_scan(unsigned v, unsigned *s_warp, int lane, int warp, unsigned *total)
+{
+    unsigned incl = v;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const unsigned t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+    }
+    __syncthreads();   // s_warp may still be read from an earlier use
+    if (lane == 31) s_warp[warp] = incl;
+    __syncthreads();
+    unsigned wsum = lane < WARPS ? s_warp[lane] : 0u;
+    unsigned wincl = wsum;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const unsigned t = __shfl_up_sync(0xffffffffu, wincl, o);
+        if (lane >= o) wincl += t;
+    }
+    *total = __shfl_sync(0xffffffffu, wincl, WARPS - 1);
+    return __shfl_sync(0xffffffffu, wincl - wsum, warp) + incl - v;
+}
+
 // What the register-resident select works on:
 //   SEL_ROW   a score row indexed by key (the plain entry point and the strip path)
 //   SEL_TAU   the sampled scores of a row: only the value at a given rank is wanted (the filter threshold)
@@ -235,6 +285,59 @@ k_topk_cached(const Params p, const float *__restrict__ scores, int64_t score_st
     const unsigned need_eq = need;                                   // equal keys kept, lowest indices first
     if (MODE == SEL_TAU) {
         if (tid == 0) sa.tau_key[blockIdx.x] = tau;
+        return;
+    }
+    if (MODE == SEL_CAND) {
+        // The candidates come in no particular order.  Kept: score above tau, or equal to tau and among the need_eq
+        // lowest key indices of the equal ones.  The kept keys are marked in a bitmap over the row's keys, which is
+        // then read out in ascending order.
+        extern __shared__ unsigned bitmap[];
+        unsigned my_eq = 0;
+#pragma unroll
+        for (int e = 0; e < E; ++e) my_eq += (j0 + e < nc) && key[e] == tau;
+        unsigned total_eq;
+        block_excl_scan<WARPS>(my_eq, s_warp, lane, warp, &total_eq);
+        uint32_t jmin = 0u;   // tied candidates are kept when ~index >= jmin
+        if (total_eq > need_eq) {
+            if (total_eq > kListCap) {   // thousands of exact ties at the threshold: leave the row to the exact redo
+                if (tid == 0) sa.flag[blockIdx.x] = 1;
+                return;
+            }
+            if (tid == 0) s_cnt = 0;
+            __syncthreads();
+#pragma unroll
+            for (int e = 0; e < E; ++e)
+                if (j0 + e < nc && key[e] == tau) s_list[atomicAdd(&s_cnt, 1u)] = ~(uint32_t)prow[j0 + e];
+            __syncthreads();
+            jmin = select_on_list<THREADS>(s_list, total_eq, need_eq, hist, &s_prefix, &s_need, tid, lane, warp);
+        }
+        const int nwords = (n_keys + 31) >> 5;
+        for (int wd = tid; wd < nwords; wd += THREADS) bitmap[wd] = 0u;
+        __syncthreads();
+#pragma unroll
+        for (int e = 0; e < E; ++e) {
+            if (j0 + e >= nc) continue;
+            if (key[e] > tau || key[e] == tau) {
+                const uint32_t j = (uint32_t)prow[j0 + e];
+                if (key[e] > tau || ~j >= jmin) atomicOr(&bitmap[j >> 5], 1u << (j & 31u));
+            }
+        }
+        __syncthreads();
+        const int per = (nwords + THREADS - 1) / THREADS;
+        const int w0 = tid * per, w1 = min(nwords, w0 + per);
+        unsigned mine = 0;
+        for (int wd = w0; wd < w1; ++wd) mine += __popc(bitmap[wd]);
+        unsigned total_sel;
+        unsigned posn = block_excl_scan<WARPS>(mine, s_warp, lane, warp, &total_sel);
+        for (int wd = w0; wd < w1; ++wd) {
+            unsigned bits = bitmap[wd];
+            while (bits) {
+                const int bpos = __ffs(bits) - 1;
+                bits &= bits - 1;
+                out[posn++] = wd * 32 + bpos;
+            }
+        }
+        for (int t = take + tid; t < p.k; t += THREADS) out[t] = -1;
         return;
     }
 
@@ -820,10 +923,11 @@ cudaError_t launch_filter_select(const Params &p, const float *cand_a, const int
     if (n_rows == 0) return cudaSuccess;
     SelArgs sa{1, cap, nullptr, flag, count, cand_j};
     const unsigned n = (unsigned)n_rows;
+    const size_t bm = (size_t)((p.Lk + 31) / 32) * 4;   // one bit per key of the row (at most 32 KB)
     if (cap <= 8192)
-        k_topk_cached<256, 32, true, SEL_CAND><<<n, 256, 0, st>>>(p, cand_a, cap, idx, row0, -1, 0x7fffffff, sa);
+        k_topk_cached<256, 32, true, SEL_CAND><<<n, 256, bm, st>>>(p, cand_a, cap, idx, row0, -1, 0x7fffffff, sa);
     else
-        k_topk_cached<512, 64, true, SEL_CAND><<<n, 512, 0, st>>>(p, cand_a, cap, idx, row0, -1, 0x7fffffff, sa);
+        k_topk_cached<512, 64, true, SEL_CAND><<<n, 512, bm, st>>>(p, cand_a, cap, idx, row0, -1, 0x7fffffff, sa);
     count_launch();
     return cudaGetLastError();
 }
