@@ -378,7 +378,10 @@ int hs2_last_cuda_error(void) { return g_last_cuda_error; }
 int hs2_device_error_flags(unsigned *flags)
 {
     if (!flags) return HS2_ERR_INVALID_ARG;
-    cudaError_t e = read_tc5_error(flags);
+    unsigned a = 0, b = 0;
+    cudaError_t e = read_tc5_error(&a);
+    if (e == cudaSuccess) e = read_sparse_error(&b);
+    *flags = a | (b << 8);   // bits 8.. : the sparse kernels
     return e == cudaSuccess ? HS2_OK : cuda_fail(e);
 }
 

@@ -121,5 +121,6 @@ cudaError_t launch_scores_filter_tc5(const Params &p, const void *Q, const void 
                                      int64_t n_rows, const uint32_t *tau_key, float *cand_a, int32_t *cand_j, int *count,
                                      int cap, cudaStream_t st);
 cudaError_t read_tc5_error(unsigned *out);
+cudaError_t read_sparse_error(unsigned *out);
 
 }  // namespace hs2

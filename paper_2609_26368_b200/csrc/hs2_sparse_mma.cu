@@ -37,20 +37,30 @@
 #ifndef HS2_SPD_WARPS
 #define HS2_SPD_WARPS 6
 #endif
+// 1: rows are fetched with one bulk async copy (TMA, 256 bytes) per row that completes on an mbarrier;
+// 0: sixteen 16-byte cp.async per row.
+#ifndef HS2_SP_BULK
+#define HS2_SP_BULK 0
+#endif
 
 namespace hs2 {
 namespace {
 
 constexpr int HD = 128;                      // head_dim
 constexpr int kRowBytes = HD * 2;            // one K or V row
+constexpr bool kBulk = HS2_SP_BULK != 0;
+// row pitch in shared memory: bulk copies cannot swizzle, so rows are padded by 16 bytes instead
+// (17 sixteen-byte units per row: eight consecutive rows hit eight different bank groups)
+constexpr int kPitch = kBulk ? kRowBytes + 16 : kRowBytes;
+__device__ unsigned g_sparse_error;          // bit 0: a bounded mbarrier wait ran out
 constexpr int kMaxSplits = 32;               // warp-level splits of one (sequence, KV head) in decode
 
 // KT key rows per pipeline stage (16 or 32), NSTAGE stages per warp, WARPS warps per CTA
 template <int KT_, int NSTAGE_, int WARPS_>
 struct Cfg {
     static constexpr int KT = KT_, NSTAGE = NSTAGE_, WARPS = WARPS_;
-    static constexpr int kStageBytes = 2 * KT * kRowBytes;                       // K tile then V tile
-    static constexpr int kWarpSmem = NSTAGE * kStageBytes + NSTAGE * 32 * 4;     // + key index of each staged row
+    static constexpr int kStageBytes = 2 * KT * kPitch;                          // K tile then V tile
+    static constexpr int kWarpSmem = NSTAGE * kStageBytes + NSTAGE * 32 * 4 + 64;   // + key index of each staged row + mbarriers
     static_assert(KT == 16 || KT == 32, "a stage holds 16 or 32 key rows");
     static_assert(NSTAGE >= 2, "double buffering at least");
 };
@@ -64,6 +74,27 @@ __device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, int sr
 }
 __device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::); }
 template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N)); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;\n" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;\n" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile("{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.b32 %0, 1, 0, p;\n}\n"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ void bulk_copy_row(uint32_t dst, const void *src, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], 256, [%2];\n"
+                 ::"r"(dst), "l"(src), "r"(bar) : "memory");
+}
 
 __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr)
 {
@@ -126,6 +157,23 @@ __device__ __forceinline__ int slot_key(const Params &p, const Item &it, int til
     return j;   // negative entries stay negative
 }
 
+// bulk variant: lane r < KT copies K row r, lane 16 + r copies V row r; void rows are not copied (the stage
+// buffers start zeroed and only ever receive real rows, so stale rows are finite and get probability 0)
+template <int KT>
+__device__ __forceinline__ void issue_stage_bulk(const Item &it, uint32_t stage_base, uint32_t bar, int j, int lane)
+{
+    static_assert(KT == 16, "the bulk variant maps one K and one V row to each lane");
+    const int r = lane & 15, hi = lane >> 4;
+    const int jr = __shfl_sync(0xffffffffu, j, r);
+    const unsigned valid = __ballot_sync(0xffffffffu, jr >= 0) & 0xffffu;
+    if (lane == 0) mbar_expect_tx(bar, __popc(valid) * 2u * kRowBytes);
+    __syncwarp();
+    if (jr >= 0) {
+        const char *src = (hi ? it.Vb : it.Kb) + (int64_t)jr * it.row_stride;
+        bulk_copy_row(stage_base + hi * KT * kPitch + r * kPitch, src, bar);
+    }
+}
+
 template <int KT>
 __device__ __forceinline__ void issue_stage(const Item &it, uint32_t stage_base, int j, int lane)
 {
@@ -161,13 +209,13 @@ __device__ __forceinline__ void consume_stage(Acc &acc, const uint32_t (&qf)[16]
         float s2[4] = {0.f, 0.f, 0.f, 0.f};
         s[mt][0] = s[mt][1] = s[mt][2] = s[mt][3] = 0.f;
         // chunk = 2 ks + (mi >> 1); (chunk ^ rr) << 4 = (32 ks) ^ lx with lx = ((mi >> 1) ^ rr) << 4
-        const uint32_t rowaddr = stage_base + (mt * 16 + (mi & 1) * 8 + rr) * kRowBytes;
-        const uint32_t lx = (uint32_t)((mi >> 1) ^ rr) << 4;
+        const uint32_t rowaddr = stage_base + (mt * 16 + (mi & 1) * 8 + rr) * kPitch;
+        const uint32_t lx = kBulk ? (uint32_t)(mi >> 1) << 4 : (uint32_t)((mi >> 1) ^ rr) << 4;   // padded rows need no swizzle
 #pragma unroll
         for (int ks = 0; ks < 8; ks += 2) {
             uint32_t a[4], a2[4];
-            ldmatrix_x4(a, rowaddr + (lx ^ (uint32_t)(32 * ks)));
-            ldmatrix_x4(a2, rowaddr + (lx ^ (uint32_t)(32 * ks + 32)));
+            ldmatrix_x4(a, rowaddr + (kBulk ? lx + (uint32_t)(32 * ks) : lx ^ (uint32_t)(32 * ks)));
+            ldmatrix_x4(a2, rowaddr + (kBulk ? lx + (uint32_t)(32 * ks + 32) : lx ^ (uint32_t)(32 * ks + 32)));
             mma_bf16(s[mt], a, qf[2 * ks], qf[2 * ks + 1]);
             mma_bf16(s2, a2, qf[2 * ks + 2], qf[2 * ks + 3]);
         }
@@ -220,15 +268,15 @@ __device__ __forceinline__ void consume_stage(Acc &acc, const uint32_t (&qf)[16]
         }
     }
     // O^T += V^T P^T : rows = output dimensions, contraction over the keys of the stage
-    const uint32_t vbase = stage_base + KT * kRowBytes;
+    const uint32_t vbase = stage_base + KT * kPitch;
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt) {
-        const uint32_t rowaddr = vbase + (mt * 16 + (mi >> 1) * 8 + rr) * kRowBytes;
-        const uint32_t lx = (uint32_t)((mi & 1) ^ rr) << 4;
+        const uint32_t rowaddr = vbase + (mt * 16 + (mi >> 1) * 8 + rr) * kPitch;
+        const uint32_t lx = kBulk ? (uint32_t)(mi & 1) << 4 : (uint32_t)((mi & 1) ^ rr) << 4;
 #pragma unroll
         for (int dt = 0; dt < 8; ++dt) {
             uint32_t a[4];
-            ldmatrix_x4_trans(a, rowaddr + (lx ^ (uint32_t)(32 * dt)));
+            ldmatrix_x4_trans(a, rowaddr + (kBulk ? lx + (uint32_t)(32 * dt) : lx ^ (uint32_t)(32 * dt)));
             mma_bf16(acc.o[dt], a, pb[mt][0], pb[mt][1]);
         }
     }
@@ -242,8 +290,20 @@ __device__ __forceinline__ void run_tiles(const Params &p, const Item &it, const
     constexpr int KT = C::KT, NSTAGE = C::NSTAGE, kStageBytes = C::kStageBytes;
     const uint32_t sbase = smem_u32(wsm);
     int *sj = reinterpret_cast<int *>(wsm + NSTAGE * kStageBytes);
+    const uint32_t bars = sbase + NSTAGE * kStageBytes + NSTAGE * 32 * 4;   // one mbarrier per stage (bulk variant)
+    if (kBulk) {
+        // zero the stage buffers once (void rows are never copied), set up the barriers
+        uint4 *z = reinterpret_cast<uint4 *>(wsm);
+        for (int e = lane; e < NSTAGE * kStageBytes / 16; e += 32) z[e] = make_uint4(0u, 0u, 0u, 0u);
+        if (lane == 0)
+            for (int s2 = 0; s2 < NSTAGE; ++s2) mbar_init(bars + 8 * s2, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;\n" ::: "memory");
+        __syncwarp();
+    }
     int next = t_begin;
     int jn = next < t_end ? slot_key<KT>(p, it, next, lane) : -1;
+    int n_issued = 0, n_done = 0;
     auto try_issue = [&](int stage) -> bool {
         while (next < t_end) {
             const int j = jn;
@@ -251,29 +311,51 @@ __device__ __forceinline__ void run_tiles(const Params &p, const Item &it, const
             if (next < t_end) jn = slot_key<KT>(p, it, next, lane);
             if (__ballot_sync(0xffffffffu, j >= 0)) {
                 sj[stage * 32 + lane] = j;
-                issue_stage<KT>(it, sbase + stage * kStageBytes, j, lane);
+                if (kBulk) issue_stage_bulk<KT>(it, sbase + stage * kStageBytes, bars + 8 * stage, j, lane);
+                else issue_stage<KT>(it, sbase + stage * kStageBytes, j, lane);
                 return true;
             }
         }
         return false;
     };
-    int n_issued = 0, n_done = 0;
 #pragma unroll
     for (int s = 0; s < NSTAGE - 1; ++s) {
         if (try_issue(n_issued % NSTAGE)) ++n_issued;
-        cp_async_commit();
+        if (!kBulk) cp_async_commit();
     }
+    bool gave_up = false;
     while (n_done < n_issued) {
-        cp_async_wait<NSTAGE - 2>();
+        const int stage = n_done % NSTAGE;
+        if (kBulk) {
+            // bounded wait for the stage's rows; the parity of a stage flips every NSTAGE tiles
+            const uint32_t parity = (uint32_t)(n_done / NSTAGE) & 1u;
+            bool ok = false;
+            for (uint32_t spin = 0; spin < (1u << 22) && !ok; ++spin) ok = mbar_try_wait(bars + 8 * stage, parity);
+            if (!__all_sync(0xffffffffu, ok)) {
+                if (lane == 0) atomicOr(&g_sparse_error, 1u);
+                gave_up = true;
+                break;
+            }
+        } else {
+            cp_async_wait<NSTAGE - 2>();
+        }
         __syncwarp();
         if (try_issue(n_issued % NSTAGE)) ++n_issued;
-        cp_async_commit();
-        const int stage = n_done % NSTAGE;
+        if (!kBulk) cp_async_commit();
         const unsigned mask = __ballot_sync(0xffffffffu, sj[stage * 32 + lane] >= 0);
         consume_stage<KT>(acc, qf, sbase + stage * kStageBytes, mask, p.scale_log2, lane);
         ++n_done;
     }
-    cp_async_wait<0>();
+    if (kBulk) {
+        if (gave_up) {   // let the copies that are still in flight land before the buffers are reused
+            for (int t = n_done; t < n_issued; ++t) {
+                const uint32_t parity = (uint32_t)(t / NSTAGE) & 1u;
+                for (uint32_t spin = 0; spin < (1u << 22) && !mbar_try_wait(bars + 8 * (t % NSTAGE), parity); ++spin) {}
+            }
+        }
+    } else {
+        cp_async_wait<0>();
+    }
     __syncwarp();
 }
 
@@ -735,5 +817,8 @@ cudaError_t launch_sparse_mma_decode_static(const Params &p, const void *Q, cons
     count_launch();
     return cudaGetLastError();
 }
+
+// device error word of the sparse kernels (bit 0: a bounded wait ran out); synchronises the device
+cudaError_t read_sparse_error(unsigned *out) { return cudaMemcpyFromSymbol(out, g_sparse_error, sizeof(unsigned)); }
 
 }  // namespace hs2
