@@ -177,6 +177,11 @@ int hs2_last_cuda_error(void);
  * window).  Sticky until the process exits.  Synchronises the current device.  Returns an hs2_status. */
 int hs2_device_error_flags(unsigned *flags);
 
+/* Testing knob: enabled = 0 makes hs2_full_attn_select use its mma.sync kernels (the path taken when TMA
+ * tensor maps cannot be built) instead of the tcgen05 ones; 1 restores the default; negative only queries.
+ * Returns the previous setting.  Process-wide. */
+int hs2_set_tcgen05_enabled(int enabled);
+
 /* Tuning knob of hs2_full_attn_select: from which kv_len on the selection thresholds a sample of the scores
  * and works on filtered candidate lists instead of complete score strips (default 65537; both ways give the
  * same indices).  Returns the previous value; min_keys <= 0 only queries.  Process-wide. */

@@ -24,7 +24,7 @@ HS2_OP_FULL_ATTN_SELECT, HS2_OP_TOPK_SELECT, HS2_OP_SPARSE_ATTN_PREFILL, HS2_OP_
 
 EXPORTS = ["hs2_workspace_bytes", "hs2_full_attn_select", "hs2_topk_select", "hs2_sparse_attn_prefill",
            "hs2_sparse_attn_decode", "hs2_sparse_attn_decode_static", "hs2_status_string", "hs2_last_cuda_error",
-           "hs2_launch_count", "hs2_device_error_flags", "hs2_set_filter_min_keys"]
+           "hs2_launch_count", "hs2_device_error_flags", "hs2_set_filter_min_keys", "hs2_set_tcgen05_enabled"]
 
 
 class HS2Error(RuntimeError):
@@ -85,6 +85,11 @@ def hs2_device_error_flags() -> int:
 def hs2_set_filter_min_keys(min_keys: int) -> int:
     """Tuning knob: kv_len from which the full layer's selection uses filtered candidate lists; returns the old value."""
     return int(load_library().hs2_set_filter_min_keys(int(min_keys)))
+
+
+def hs2_set_tcgen05_enabled(enabled: int) -> int:
+    """Testing knob: 0 routes the full layer through its mma.sync kernels; returns the previous setting."""
+    return int(load_library().hs2_set_tcgen05_enabled(int(enabled)))
 
 
 def hs2_launch_count() -> int:

@@ -80,6 +80,7 @@ constexpr int kFilterSamp = 8;              // every 8th key tile is scored for 
 // The filtered path wins only when rows are long (measured: 131072 keys 485 ms vs 580 ms with strips, 32768
 // keys 67 ms vs 64 ms, 8192 keys 3.7 ms vs 2.1 ms): shorter contexts keep the strips.
 std::atomic<int> g_filter_min_keys{65537};
+std::atomic<int> g_disable_tc5{0};          // testing knob: run the mma.sync kernels instead of the tcgen05 ones
 constexpr size_t kFilterBigCap = (size_t)1 << 30;
 
 struct FilterPlan {
@@ -99,7 +100,7 @@ FilterPlan filter_plan(const Params &p, hs2_dtype dt)
     f.ns_w = filter_sample_width(p, kFilterSamp);
     f.per_row = align_up((size_t)f.ns_w * 4, 16);
     if ((size_t)f.cap * 8 > f.per_row) f.per_row = (size_t)f.cap * 8;
-    f.ok = p.k > 0 && scores_filter_supported(p, dt) && f.cap <= 32768 && f.ns_w <= 32768 && p.Lk > f.cap &&
+    f.ok = p.k > 0 && !g_disable_tc5.load(std::memory_order_relaxed) && scores_filter_supported(p, dt) && f.cap <= 32768 && f.ns_w <= 32768 && p.Lk > f.cap &&
            p.Lk >= g_filter_min_keys.load(std::memory_order_relaxed) && select_rows(p) >= 1024;
     return f;
 }
@@ -146,7 +147,7 @@ cudaError_t launch_scores(const Params &p, hs2_dtype dt, bool mma, bool aligned,
 {
     cudaError_t e = cudaErrorNotSupported;
 #ifndef HS2_NO_TC5
-    if (aligned && scores_tc5_supported(p, dt)) e = launch_scores_tc5(p, Q, K, LSE, out, out_stride, row0, n_rows, all_visible, st);
+    if (aligned && !g_disable_tc5.load(std::memory_order_relaxed) && scores_tc5_supported(p, dt)) e = launch_scores_tc5(p, Q, K, LSE, out, out_stride, row0, n_rows, all_visible, st);
 #endif
     if (e == cudaErrorNotSupported)
         e = mma ? launch_scores_mma(p, Q, K, LSE, out, out_stride, row0, n_rows, all_visible, st)
@@ -231,7 +232,8 @@ hs2_status hs2_full_attn_select(const hs2_problem *hp, const void *Q, const void
     else {
         e = cudaErrorNotSupported;
 #ifndef HS2_NO_TC5
-        if (full_tc5_supported(p, dt) && aligned16(Q, K, V, O)) e = launch_full_attn_tc5(p, Q, K, V, O, LSE, st);
+        if (!g_disable_tc5.load(std::memory_order_relaxed) && full_tc5_supported(p, dt) && aligned16(Q, K, V, O))
+            e = launch_full_attn_tc5(p, Q, K, V, O, LSE, st);
 #endif
         if (e == cudaErrorNotSupported)
             e = mma ? launch_full_attn_mma(p, Q, K, V, O, LSE, st) : launch_full_attn_generic(p, dt, Q, K, V, O, LSE, st);
@@ -383,6 +385,13 @@ int hs2_device_error_flags(unsigned *flags)
     if (e == cudaSuccess) e = read_sparse_error(&b);
     *flags = a | (b << 8);   // bits 8.. : the sparse kernels
     return e == cudaSuccess ? HS2_OK : cuda_fail(e);
+}
+
+int hs2_set_tcgen05_enabled(int enabled)
+{
+    const int old = g_disable_tc5.load(std::memory_order_relaxed) ? 0 : 1;
+    if (enabled >= 0) g_disable_tc5.store(enabled ? 0 : 1, std::memory_order_relaxed);
+    return old;
 }
 
 int hs2_set_filter_min_keys(int min_keys)

@@ -218,6 +218,22 @@ def _filtered_redo():
     assert int(ws[: 12 * n_rows].view(torch.int32)[2 * n_rows: 3 * n_rows].sum()) == 0
 
 
+def test_mma_sync_fallback_kernels_of_the_full_layer():
+    """The mma.sync attention and score kernels are what runs when TMA tensor maps cannot be built."""
+    old = hs2.hs2_set_tcgen05_enabled(0)
+    try:
+        for over in (dict(q_len=333, kv_len=333, k_sel=48, window=13, n_needles=8),
+                     dict(q_len=200, kv_len=900, k_sel=64, window=16, n_q_heads=8, n_kv_heads=2, n_needles=8, batch=2)):
+            wl = scaled("cfg2", **over)
+            run = BlockRun(make_inputs(wl)).run_full(want_scores=True)
+            run.check_full(check_scores=True)
+            run.check_idx_bitexact_on_gpu_scores()
+            b = BlockRun(make_inputs(wl)).run_full(want_scores=False)
+            assert torch.equal(run.idx, b.idx)
+    finally:
+        hs2.hs2_set_tcgen05_enabled(old)
+
+
 def test_paper_native_shape_mqa64_dim256_with_sink():
     """The attention shape of the paper's own model (Table 1: 64 query heads / 1 KV head, head dim 256,
     128 forced local + 1024 global tokens, per-head sink bias in the sparse layers), scaled in length."""
