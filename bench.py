@@ -385,7 +385,8 @@ def run_reference(args, wl):
     import oracle
     oracle.build()
     inp = make_inputs(wl, "cpu")
-    rows = [(b, i) for b in range(wl.batch) for i in sample_rows(wl, args.cpu_rows)]
+    # a bounded sample per step, so that K steps end within a few minutes on the machine's host cores
+    rows = [(b, i) for b in range(wl.batch) for i in sample_rows(wl, min(args.cpu_rows, 1024))]
     for _ in range(min(args.warmup, 1)):
         oracle_sample_step(wl, inp, rows[:8])
     t0 = time.time()
