@@ -232,7 +232,7 @@ hs2_status hs2_full_attn_select(const hs2_problem *hp, const void *Q, const void
     else {
         e = cudaErrorNotSupported;
 #ifndef HS2_NO_TC5
-        if (!g_disable_tc5.load(std::memory_order_relaxed) && full_tc5_supported(p, dt) && aligned16(Q, K, V, O))
+        if (!g_disable_tc5.load(std::memory_order_relaxed) && full_attn_tc5_supported(p, dt) && aligned16(Q, K, V, O))
             e = launch_full_attn_tc5(p, Q, K, V, O, LSE, st);
 #endif
         if (e == cudaErrorNotSupported)

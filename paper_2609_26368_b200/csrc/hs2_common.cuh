@@ -108,7 +108,8 @@ cudaError_t launch_scores_mma(const Params &p, const void *Q, const void *K, con
                               int64_t out_stride, int64_t row0, int64_t n_rows, bool all_visible, cudaStream_t st);
 
 // tcgen05 / TMEM / TMA full attention (bf16, head_dim 128)
-bool full_tc5_supported(const Params &p, hs2_dtype dt);
+bool full_tc5_supported(const Params &p, hs2_dtype dt);        // head_dim 128: attention, score sweeps, filters
+bool full_attn_tc5_supported(const Params &p, hs2_dtype dt);   // the attention kernel alone: head_dim 128 or 256
 cudaError_t launch_full_attn_tc5(const Params &p, const void *Q, const void *K, const void *V, void *O, float *LSE,
                                  cudaStream_t st);
 bool scores_tc5_supported(const Params &p, hs2_dtype dt);

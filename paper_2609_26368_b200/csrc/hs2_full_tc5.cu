@@ -25,17 +25,25 @@ namespace {
 
 constexpr int BM = 128, BN = 64, HD = 128;
 constexpr int kThreads = 192;
-constexpr uint32_t kQBytes = 2 * BM * 128;        // two 64-dim halves
-constexpr uint32_t kKVStage = 2 * BN * 128;       // one K (or V) tile: two halves
-constexpr uint32_t kOffQ = 0;
-constexpr uint32_t kOffK = kOffQ + kQBytes;       // 2 stages
-constexpr uint32_t kOffV = kOffK + 2 * kKVStage;  // 2 stages
-constexpr uint32_t kOffP = kOffV + 2 * kKVStage;  // 128 rows x 64 keys bf16, K-major
-constexpr uint32_t kOffBar = kOffP + BM * 128;
 constexpr uint32_t kBarBytes = 128;
 constexpr uint32_t kAlignSlack = 896;             // the dynamic window is at least 128-byte aligned
-constexpr uint32_t kSmemBytes = kOffBar + kBarBytes + kAlignSlack;   // 115712 = (228 KB - 2 KB) / 2
-constexpr uint32_t kTmemCols = 256;
+constexpr uint32_t kTmemCols = 256;               // score kernels, attention at head_dim 128
+// shared-memory plan of the attention kernel for head_dim D (a multiple of 64): every operand tile is a set
+// of D/64 slices of [rows][64 dims] = 128-byte rows, each slice 128-byte swizzled
+template <int D>
+struct FaCfg {
+    static constexpr int NQ = D / 64;
+    static constexpr uint32_t kQBytes = NQ * BM * 128;
+    static constexpr uint32_t kKVStage = NQ * BN * 128;       // one K (or V) tile
+    static constexpr uint32_t kOffQ = 0;
+    static constexpr uint32_t kOffK = kOffQ + kQBytes;        // 2 stages
+    static constexpr uint32_t kOffV = kOffK + 2 * kKVStage;   // 2 stages
+    static constexpr uint32_t kOffP = kOffV + 2 * kKVStage;   // 128 rows x 64 keys bf16, K-major
+    static constexpr uint32_t kOffBar = kOffP + BM * 128;
+    static constexpr uint32_t kSmemBytes = kOffBar + kBarBytes + kAlignSlack;   // 115712 at D=128: two CTAs per SM
+    static constexpr uint32_t kTmem = D <= 128 ? 256 : 512;  // 2 x 64 score columns + D output columns, a power of two
+    static constexpr int kMinBlocks = D <= 128 ? 2 : 1;
+};
 constexpr uint32_t kSpinLimit = 1u << 22;
 constexpr float kRescaleThreshold = 8.f;          // log2 units
 
@@ -143,11 +151,16 @@ __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
     return *reinterpret_cast<uint32_t *>(&v);
 }
 
-__global__ void __launch_bounds__(kThreads, 2)
+template <int D>
+__global__ void __launch_bounds__(kThreads, FaCfg<D>::kMinBlocks)
 k_full_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
            const __grid_constant__ CUtensorMap tmV, const Params p, __nv_bfloat16 *__restrict__ O,
            float *__restrict__ LSE)
 {
+    using F = FaCfg<D>;
+    constexpr int NQ = F::NQ;
+    constexpr uint32_t kQBytes = F::kQBytes, kKVStage = F::kKVStage, kOffQ = F::kOffQ, kOffK = F::kOffK, kOffV = F::kOffV,
+                       kOffP = F::kOffP, kOffBar = F::kOffBar, kTmemFa = F::kTmem;
     extern __shared__ char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t pad = (1024u - (raw & 1023u)) & 1023u;
@@ -185,7 +198,7 @@ k_full_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
     if (warp == 5) {   // TMEM allocation is a warp-wide operation
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(tmem_slot)), "r"(kTmemFa) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
     }
     tc_fence_before();
@@ -197,8 +210,8 @@ k_full_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
         // ------------------------------------------------ TMA producer
         if (elect_one() && nblk > 0) {
             mbar_expect_tx(bar(Q_FULL), kQBytes);
-            tma_load_4d(sbase + kOffQ, &tmQ, bar(Q_FULL), 0, h, i0, b);
-            tma_load_4d(sbase + kOffQ + BM * 128, &tmQ, bar(Q_FULL), 64, h, i0, b);
+#pragma unroll
+            for (int sl = 0; sl < NQ; ++sl) tma_load_4d(sbase + kOffQ + sl * BM * 128, &tmQ, bar(Q_FULL), 64 * sl, h, i0, b);
             int issued = 0;
             for (int j = 0; j < nblk; ++j) {
                 const int st = j & 1;
@@ -206,10 +219,11 @@ k_full_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 issued = j + 1;
                 mbar_expect_tx(bar(KV_FULL0 + st), 2 * kKVStage);
                 const uint32_t kdst = sbase + kOffK + st * kKVStage, vdst = sbase + kOffV + st * kKVStage;
-                tma_load_4d(kdst, &tmK, bar(KV_FULL0 + st), 0, gkv, j * BN, b);
-                tma_load_4d(kdst + BN * 128, &tmK, bar(KV_FULL0 + st), 64, gkv, j * BN, b);
-                tma_load_4d(vdst, &tmV, bar(KV_FULL0 + st), 0, gkv, j * BN, b);
-                tma_load_4d(vdst + BN * 128, &tmV, bar(KV_FULL0 + st), 64, gkv, j * BN, b);
+#pragma unroll
+                for (int sl = 0; sl < NQ; ++sl) {
+                    tma_load_4d(kdst + sl * BN * 128, &tmK, bar(KV_FULL0 + st), 64 * sl, gkv, j * BN, b);
+                    tma_load_4d(vdst + sl * BN * 128, &tmV, bar(KV_FULL0 + st), 64 * sl, gkv, j * BN, b);
+                }
             }
             if (*abort_flag) {   // leaving early: let the copies already in flight land before the CTA goes away
                 for (int j = max(0, issued - 2); j < issued; ++j)
@@ -220,7 +234,7 @@ k_full_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
     } else if (warp == 5) {
         // ------------------------------------------------ MMA issuer
         if (elect_one() && nblk > 0) {
-            constexpr uint32_t idS = idesc(BM, BN, 0), idPV = idesc(BM, HD, 1);
+            constexpr uint32_t idS = idesc(BM, BN, 0), idPV = idesc(BM, D, 1);
             bool ok = mbar_wait(bar(Q_FULL), 0, abort_flag);
             auto issue_s = [&](int j) -> bool {
                 const int st = j & 1, ph = (j >> 1) & 1;
@@ -229,7 +243,7 @@ k_full_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 tc_fence_after();
                 const uint32_t qa = sbase + kOffQ, ka = sbase + kOffK + st * kKVStage;
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
+                for (int ks = 0; ks < D / 16; ++ks) {
                     const uint32_t off = (ks & 3) * 32;   // 16 dims = 32 bytes inside the swizzled 128-byte row
                     const uint64_t da = smem_desc(qa + (ks >> 2) * (BM * 128) + off, 16, 1024);
                     const uint64_t db = smem_desc(ka + (ks >> 2) * (BN * 128) + off, 16, 1024);
@@ -296,7 +310,7 @@ k_full_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 tc_fence_after();
                 if (__any_sync(0xffffffffu, need)) {   // rescale the O rows of this warp (a warp-wide TMEM access)
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) {
+                    for (int c = 0; c < D / 32; ++c) {
                         float o[32];
                         tmem_ld32(lane_base + 2 * BN + c * 32, o);
                         tmem_wait_ld();
@@ -336,7 +350,7 @@ k_full_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
         const float inv = l > 0.f ? 1.f / l : 0.f;
         __nv_bfloat16 *orow = O + b * p.os_b + (int64_t)i * p.os_t + h * p.os_h;
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
+        for (int c = 0; c < D / 32; ++c) {
             float o[32];
             if (have_o) {   // uniform across the warp except after an abort
                 tmem_ld32(lane_base + 2 * BN + c * 32, o);
@@ -366,7 +380,7 @@ k_full_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
     __syncthreads();
     if (warp == 5) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(kTmemFa) : "memory");
     }
 }
 
@@ -652,11 +666,11 @@ EncodeTiledFn encode_fn()
 
 // [B, L, H, 128] bf16 with element strides (sb, st, sh): box = 64 dims x `rows` tokens of one head, 128-byte swizzle
 bool make_map(CUtensorMap *tm, const void *base, int B, int L, int H, int64_t sb, int64_t st, int64_t sh, int rows,
-              int box_heads = 1)
+              int box_heads = 1, int D = HD)
 {
     EncodeTiledFn enc = encode_fn();
     if (!enc) return false;
-    const cuuint64_t dims[4] = {(cuuint64_t)HD, (cuuint64_t)H, (cuuint64_t)L, (cuuint64_t)B};
+    const cuuint64_t dims[4] = {(cuuint64_t)D, (cuuint64_t)H, (cuuint64_t)L, (cuuint64_t)B};
     const cuuint64_t strides[3] = {(cuuint64_t)sh * 2, (cuuint64_t)st * 2, (cuuint64_t)sb * 2};
     const cuuint32_t box[4] = {64, (cuuint32_t)box_heads, (cuuint32_t)rows, 1};
     const cuuint32_t estr[4] = {1, 1, 1, 1};
@@ -664,8 +678,6 @@ bool make_map(CUtensorMap *tm, const void *base, int B, int L, int H, int64_t sb
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_128B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
-
-bool g_attr_set[64] = {};
 
 }  // namespace
 
@@ -676,26 +688,44 @@ bool full_tc5_supported(const Params &p, hs2_dtype dt)
            m8(p.ks_h) && m8(p.os_b) && m8(p.os_t) && m8(p.os_h) && (int64_t)p.B * p.Hq <= 65535 && encode_fn() != nullptr;
 }
 
+// the attention kernel alone also covers head_dim 256 (the paper's own model shape, Table 1)
+bool full_attn_tc5_supported(const Params &p, hs2_dtype dt)
+{
+    if (p.D == HD) return full_tc5_supported(p, dt);
+    auto m8 = [](int64_t x) { return x % 8 == 0 && x > 0; };
+    return dt == HS2_BF16 && p.D == 256 && m8(p.qs_b) && m8(p.qs_t) && m8(p.qs_h) && m8(p.ks_b) && m8(p.ks_t) &&
+           m8(p.ks_h) && m8(p.os_b) && m8(p.os_t) && m8(p.os_h) && (int64_t)p.B * p.Hq <= 65535 && encode_fn() != nullptr;
+}
+
+template <int D>
+cudaError_t launch_fa(const Params &p, const void *Q, const void *K, const void *V, void *O, float *LSE, cudaStream_t st)
+{
+    CUtensorMap tmQ, tmK, tmV;
+    if (!make_map(&tmQ, Q, p.B, p.Lq, p.Hq, p.qs_b, p.qs_t, p.qs_h, BM, 1, D) ||
+        !make_map(&tmK, K, p.B, p.Lk, p.Hkv, p.ks_b, p.ks_t, p.ks_h, BN, 1, D) ||
+        !make_map(&tmV, V, p.B, p.Lk, p.Hkv, p.ks_b, p.ks_t, p.ks_h, BN, 1, D))
+        return cudaErrorNotSupported;
+    static bool attr_set[64] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (!(dev >= 0 && dev < 64 && attr_set[dev])) {
+        if ((e = cudaFuncSetAttribute(k_full_tc5<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FaCfg<D>::kSmemBytes)) != cudaSuccess) return e;
+        if (dev >= 0 && dev < 64) attr_set[dev] = true;
+    }
+    dim3 grid((p.Lq + BM - 1) / BM, p.B * p.Hq);
+    k_full_tc5<D><<<grid, kThreads, FaCfg<D>::kSmemBytes, st>>>(tmQ, tmK, tmV, p, (__nv_bfloat16 *)O, LSE);
+    count_launch();
+    return cudaGetLastError();
+}
+
 // Returns cudaErrorNotSupported when the tensor maps cannot be built (the caller then takes the mma.sync kernel).
 cudaError_t launch_full_attn_tc5(const Params &p, const void *Q, const void *K, const void *V, void *O, float *LSE,
                                  cudaStream_t st)
 {
-    CUtensorMap tmQ, tmK, tmV;
-    if (!make_map(&tmQ, Q, p.B, p.Lq, p.Hq, p.qs_b, p.qs_t, p.qs_h, BM) ||
-        !make_map(&tmK, K, p.B, p.Lk, p.Hkv, p.ks_b, p.ks_t, p.ks_h, BN) ||
-        !make_map(&tmV, V, p.B, p.Lk, p.Hkv, p.ks_b, p.ks_t, p.ks_h, BN))
-        return cudaErrorNotSupported;
-    int dev = 0;
-    cudaError_t e = cudaGetDevice(&dev);
-    if (e != cudaSuccess) return e;
-    if (!(dev >= 0 && dev < 64 && g_attr_set[dev])) {
-        if ((e = cudaFuncSetAttribute(k_full_tc5, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes)) != cudaSuccess) return e;
-        if (dev >= 0 && dev < 64) g_attr_set[dev] = true;
-    }
-    dim3 grid((p.Lq + BM - 1) / BM, p.B * p.Hq);
-    k_full_tc5<<<grid, kThreads, kSmemBytes, st>>>(tmQ, tmK, tmV, p, (__nv_bfloat16 *)O, LSE);
-    count_launch();
-    return cudaGetLastError();
+    if (p.D == 128) return launch_fa<128>(p, Q, K, V, O, LSE, st);
+    if (p.D == 256) return launch_fa<256>(p, Q, K, V, O, LSE, st);
+    return cudaErrorNotSupported;
 }
 
 template <int G, int MODE>
