@@ -394,15 +394,22 @@ k_full_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
 // warps 0-3 (thread = key) subtract LSE, take the group maximum and write 32 consecutive keys of a
 // strip row per warp instruction.
 constexpr int SC_KCHUNK = 4096;                   // keys per CTA
-constexpr uint32_t kScOffQ = 0;                   // [2 halves][128 (query, head) rows][128 B]
-constexpr uint32_t kScOffK = 32768;               // 2 stages x [2 halves][128 keys][128 B]
-constexpr uint32_t kScOffNl = kScOffK + 2 * 32768;   // float[128]: -LSE/scale per column
-constexpr uint32_t kScOffNq = kScOffNl + 512;     // int[128]: keys needed per query
-constexpr uint32_t kScOffRow = kScOffNq + 512;    // int64[128]: strip row of each query
-constexpr uint32_t kScOffTau = kScOffRow + 1024;  // uint32[32]: filter threshold per query (filter mode)
-constexpr uint32_t kScOffCnt = kScOffTau + 128;   // int[32]: candidates appended per query (filter mode)
-constexpr uint32_t kScOffBar = kScOffCnt + 1024;
-constexpr uint32_t kScSmemBytes = kScOffBar + kBarBytes + kAlignSlack;
+// shared-memory plan of the score sweep for head_dim D: Q and K tiles are D/64 slices of [128 rows][128 B]
+template <int D>
+struct ScCfg {
+    static constexpr int NQ = D / 64;
+    static constexpr uint32_t kSlice = 128 * 128;                 // one slice: 128 rows of 128 bytes
+    static constexpr uint32_t kOffQ = 0;                          // (query, head) rows
+    static constexpr uint32_t kOffK = NQ * kSlice;                // 2 stages of key rows
+    static constexpr uint32_t kOffNl = kOffK + 2 * NQ * kSlice;   // float[128]: -LSE/scale per column
+    static constexpr uint32_t kOffNq = kOffNl + 512;              // int[128]: keys needed per query
+    static constexpr uint32_t kOffRow = kOffNq + 512;             // int64[128]: strip row of each query
+    static constexpr uint32_t kOffTau = kOffRow + 1024;           // uint32[32]: filter threshold per query (filter mode)
+    static constexpr uint32_t kOffCnt = kOffTau + 128;            // int[32]: candidates appended per query (filter mode)
+    static constexpr uint32_t kOffBar = kOffCnt + 1024;
+    static constexpr uint32_t kSmemBytes = kOffBar + kBarBytes + kAlignSlack;
+    static constexpr int kMinBlocks = D <= 128 ? 2 : 1;
+};
 enum ScBar { SQ_FULL = 0, SK_FULL0, SK_FULL1, SK_EMPTY0, SK_EMPTY1, ACC_FULL0, ACC_FULL1, ACC_FREE0, ACC_FREE1, SC_N_BARS };
 
 // What the sweep does with a score:
@@ -427,15 +434,22 @@ __device__ __forceinline__ uint32_t order_key_f(float f)
     return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
 }
 
-template <int G, int MODE>
-__global__ void __launch_bounds__(kThreads, 2)
+template <int G, int MODE, int D>
+__global__ void __launch_bounds__(kThreads, ScCfg<D>::kMinBlocks)
 k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, const Params p,
              const float *__restrict__ LSE, float *__restrict__ out, int64_t out_stride, int64_t row0, int64_t n_rows,
              int all_visible, int tile_first, int tiles_per_bg, int samp, FilterBuf fb)
 {
-    constexpr int TQ = 128 / G;          // queries per CTA
-    constexpr int QPC = 32 / G > 0 ? 32 / G : 1;   // queries per 32-column chunk (G <= 32)
-    static_assert(MODE != SC_FILTER || TQ <= 32, "filter mode keeps one counter per query in registers");
+    using S = ScCfg<D>;
+    constexpr int NQ = S::NQ;
+    constexpr uint32_t kScOffQ = S::kOffQ, kScOffK = S::kOffK, kScOffNl = S::kOffNl, kScOffNq = S::kOffNq,
+                       kScOffRow = S::kOffRow, kScOffTau = S::kOffTau, kScOffCnt = S::kOffCnt, kScOffBar = S::kOffBar,
+                       kStage = NQ * S::kSlice;
+    constexpr int TQ = 128 / G;                    // queries per CTA
+    constexpr int QPC = G <= 32 ? 32 / G : 1;      // queries per 32-column chunk when a group fits a chunk
+    constexpr int CPQ = G <= 32 ? 1 : G / 32;      // 32-column chunks per query otherwise
+    static_assert(128 % G == 0 && (G <= 32 || G % 32 == 0), "the group's heads tile the 128 columns");
+    static_assert(MODE != SC_FILTER || TQ <= 32, "filter mode keeps one pass bit per query");
     extern __shared__ char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t pad = (1024u - (raw & 1023u)) & 1023u;
@@ -521,19 +535,19 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
 
     if (warp == 4) {
         if (elect_one()) {
-            mbar_expect_tx(bar(SQ_FULL), 32768);
-            tma_load_4d(sbase + kScOffQ, &tmQ, bar(SQ_FULL), 0, gkv * G, iq0, b);
-            tma_load_4d(sbase + kScOffQ + 16384, &tmQ, bar(SQ_FULL), 64, gkv * G, iq0, b);
+            mbar_expect_tx(bar(SQ_FULL), kStage);
+#pragma unroll
+            for (int sl = 0; sl < NQ; ++sl) tma_load_4d(sbase + kScOffQ + sl * S::kSlice, &tmQ, bar(SQ_FULL), 64 * sl, gkv * G, iq0, b);
             int issued = 0;
             for (int t = 0; t < ntile; ++t) {
                 const int st = t & 1;
                 if (!mbar_wait(bar(SK_EMPTY0 + st), ((t >> 1) & 1) ^ 1, abort_flag)) break;
                 issued = t + 1;
-                mbar_expect_tx(bar(SK_FULL0 + st), 32768);
-                const uint32_t kdst = sbase + kScOffK + st * 32768;
+                mbar_expect_tx(bar(SK_FULL0 + st), kStage);
+                const uint32_t kdst = sbase + kScOffK + st * kStage;
                 const int krow = (kt0 + t) * kstep * 128;
-                tma_load_4d(kdst, &tmK, bar(SK_FULL0 + st), 0, gkv, krow, b);
-                tma_load_4d(kdst + 16384, &tmK, bar(SK_FULL0 + st), 64, gkv, krow, b);
+#pragma unroll
+                for (int sl = 0; sl < NQ; ++sl) tma_load_4d(kdst + sl * S::kSlice, &tmK, bar(SK_FULL0 + st), 64 * sl, gkv, krow, b);
             }
             if (*abort_flag) {
                 for (int t = max(0, issued - 2); t < issued; ++t)
@@ -550,10 +564,10 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 if (!mbar_wait(bar(SK_FULL0 + st), ph, abort_flag)) break;
                 if (!mbar_wait(bar(ACC_FREE0 + st), ph ^ 1, abort_flag)) break;
                 tc_fence_after();
-                const uint32_t ka = sbase + kScOffK + st * 32768, qa = sbase + kScOffQ;
+                const uint32_t ka = sbase + kScOffK + st * kStage, qa = sbase + kScOffQ;
 #pragma unroll
-                for (int ks = 0; ks < 8; ++ks) {
-                    const uint32_t off = (ks >> 2) * 16384 + (ks & 3) * 32;
+                for (int ks = 0; ks < D / 16; ++ks) {
+                    const uint32_t off = (ks >> 2) * S::kSlice + (ks & 3) * 32;
                     umma(tmem + st * 128, smem_desc(ka + off, 16, 1024), smem_desc(qa + off, 16, 1024), id, ks > 0);
                 }
                 umma_commit(bar(SK_EMPTY0 + st));
@@ -573,6 +587,7 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             const int col = MODE == SC_SAMPLE ? (kt0 + t) * 128 + row : key;
             float aval[MODE == SC_FILTER ? TQ : 1];
             unsigned passbits = 0;
+            float carry = -INFINITY;   // running group maximum when a group spans several chunks
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 float v[32];
@@ -591,10 +606,17 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 }
 #pragma unroll
                 for (int q = 0; q < QPC; ++q) {
-                    float a = v[q * G];
+                    constexpr int W = G <= 32 ? G : 32;   // columns of this chunk that belong to one query
+                    float a = v[q * W];
 #pragma unroll
-                    for (int hh = 1; hh < G; ++hh) a = fmaxf(a, v[q * G + hh]);
-                    const int tq = c * QPC + q;
+                    for (int hh = 1; hh < W; ++hh) a = fmaxf(a, v[q * W + hh]);
+                    if (CPQ > 1) {
+                        carry = fmaxf(carry, a);
+                        if ((c + 1) % CPQ != 0) continue;   // more chunks of this query follow
+                        a = carry;
+                        carry = -INFINITY;
+                    }
+                    const int tq = CPQ > 1 ? c / CPQ : c * QPC + q;
                     const float av = a * p.scale;
                     if (MODE == SC_FILTER) {
                         aval[tq] = av;
@@ -728,7 +750,7 @@ cudaError_t launch_full_attn_tc5(const Params &p, const void *Q, const void *K, 
     return cudaErrorNotSupported;
 }
 
-template <int G, int MODE>
+template <int G, int MODE, int D>
 cudaError_t launch_sc(const CUtensorMap &tmQ, const CUtensorMap &tmK, const Params &p, const float *LSE, float *out,
                       int64_t out_stride, int64_t row0, int64_t n_rows, bool all_visible, int samp, const FilterBuf &fb,
                       cudaStream_t st)
@@ -738,7 +760,7 @@ cudaError_t launch_sc(const CUtensorMap &tmQ, const CUtensorMap &tmK, const Para
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (!(dev >= 0 && dev < 64 && attr_set[dev])) {
-        if ((e = cudaFuncSetAttribute(k_scores_tc5<G, MODE>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kScSmemBytes)) != cudaSuccess) return e;
+        if ((e = cudaFuncSetAttribute(k_scores_tc5<G, MODE, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ScCfg<D>::kSmemBytes)) != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
     constexpr int TQ = 128 / G;
@@ -752,7 +774,7 @@ cudaError_t launch_sc(const CUtensorMap &tmQ, const CUtensorMap &tmK, const Para
     const int key_tiles = (p.Lk + 128 * samp - 1) / (128 * samp);
     const unsigned gx = MODE == SC_FILTER ? 1u : (unsigned)((key_tiles + SC_KCHUNK / 128 - 1) / (SC_KCHUNK / 128));
     dim3 grid(gx, (unsigned)gy);
-    k_scores_tc5<G, MODE><<<grid, kThreads, kScSmemBytes, st>>>(tmQ, tmK, p, LSE, out, out_stride, row0, n_rows, all_visible ? 1 : 0,
+    k_scores_tc5<G, MODE, D><<<grid, kThreads, ScCfg<D>::kSmemBytes, st>>>(tmQ, tmK, p, LSE, out, out_stride, row0, n_rows, all_visible ? 1 : 0,
                                                                (int)t_first, tiles_per_bg, samp, fb);
     count_launch();
     return cudaGetLastError();
@@ -764,22 +786,34 @@ cudaError_t launch_sc_mode(const Params &p, const void *Q, const void *K, const 
 {
     if (n_rows == 0) return cudaSuccess;
     CUtensorMap tmQ, tmK;
-    if (!make_map(&tmQ, Q, p.B, p.Lq, p.Hq, p.qs_b, p.qs_t, p.qs_h, 128 / p.G, p.G) ||
-        !make_map(&tmK, K, p.B, p.Lk, p.Hkv, p.ks_b, p.ks_t, p.ks_h, 128))
+    if (!make_map(&tmQ, Q, p.B, p.Lq, p.Hq, p.qs_b, p.qs_t, p.qs_h, 128 / p.G, p.G, p.D) ||
+        !make_map(&tmK, K, p.B, p.Lk, p.Hkv, p.ks_b, p.ks_t, p.ks_h, 128, 1, p.D))
         return cudaErrorNotSupported;
     if ((n_rows + p.Lq) / (128 / p.G) + 2 * (int64_t)p.B * p.Hkv > 65535) return cudaErrorNotSupported;   // grid.y bound
-    switch (p.G) {
-        case 1: if (MODE == SC_FILTER) return cudaErrorNotSupported; return launch_sc<1, MODE == SC_FILTER ? SC_STRIP : MODE>(tmQ, tmK, p, LSE, out, out_stride, row0, n_rows, all_visible, samp, fb, st);
-        case 2: if (MODE == SC_FILTER) return cudaErrorNotSupported; return launch_sc<2, MODE == SC_FILTER ? SC_STRIP : MODE>(tmQ, tmK, p, LSE, out, out_stride, row0, n_rows, all_visible, samp, fb, st);
-        case 4: return launch_sc<4, MODE>(tmQ, tmK, p, LSE, out, out_stride, row0, n_rows, all_visible, samp, fb, st);
-        case 8: return launch_sc<8, MODE>(tmQ, tmK, p, LSE, out, out_stride, row0, n_rows, all_visible, samp, fb, st);
-        case 16: return launch_sc<16, MODE>(tmQ, tmK, p, LSE, out, out_stride, row0, n_rows, all_visible, samp, fb, st);
+    constexpr int M2 = MODE == SC_FILTER ? SC_STRIP : MODE;   // groups of 1 or 2 have no filter instantiation
+#define HS2_SC(G_, MODE_, D_) return launch_sc<G_, MODE_, D_>(tmQ, tmK, p, LSE, out, out_stride, row0, n_rows, all_visible, samp, fb, st)
+    if (p.D == 128) {
+        switch (p.G) {
+            case 1: if (MODE == SC_FILTER) return cudaErrorNotSupported; HS2_SC(1, M2, 128);
+            case 2: if (MODE == SC_FILTER) return cudaErrorNotSupported; HS2_SC(2, M2, 128);
+            case 4: HS2_SC(4, MODE, 128);
+            case 8: HS2_SC(8, MODE, 128);
+            case 16: HS2_SC(16, MODE, 128);
+        }
+    } else if (p.D == 256) {
+        if (MODE != SC_STRIP) return cudaErrorNotSupported;
+        switch (p.G) {
+            case 8: HS2_SC(8, M2, 256);
+            case 64: HS2_SC(64, M2, 256);
+        }
     }
+#undef HS2_SC
     return cudaErrorNotSupported;
 }
 
 bool scores_tc5_supported(const Params &p, hs2_dtype dt)
 {
+    if (p.D == 256) return (p.G == 8 || p.G == 64) && full_attn_tc5_supported(p, dt);
     const bool g_ok = p.G == 1 || p.G == 2 || p.G == 4 || p.G == 8 || p.G == 16;
     return g_ok && full_tc5_supported(p, dt);
 }

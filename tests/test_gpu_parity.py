@@ -144,6 +144,8 @@ SMALL = [
     ("cfg2", dict(q_len=200, kv_len=200, k_sel=40, window=0, n_needles=4)),              # no window
     ("cfg2", dict(q_len=150, kv_len=150, k_sel=16, window=4, n_q_heads=4, n_kv_heads=4, n_needles=4)),   # group of 1
     ("cfg2", dict(q_len=150, kv_len=150, k_sel=16, window=4, n_q_heads=16, n_kv_heads=1, n_needles=4)),  # MQA 16
+    ("cfg2", dict(q_len=300, kv_len=300, k_sel=64, window=16, n_q_heads=16, n_kv_heads=2, head_dim=256, n_needles=8)),
+    ("cfg2", dict(q_len=260, kv_len=700, k_sel=64, window=16, n_q_heads=64, n_kv_heads=1, head_dim=256, n_needles=8)),  # paper's shape
 ]
 
 
