@@ -324,9 +324,18 @@ hs2_status hs2_sparse_attn_prefill(const hs2_problem *hp, const void *Q, const v
     if (s != HS2_OK) return s;
     if ((s = check_device()) != HS2_OK) return s;
     cudaStream_t st = (cudaStream_t)cuda_stream;
-    cudaError_t e = (sparse_mma_supported(p, hp->dtype) && aligned16(Q, K, V, O))
-                        ? launch_sparse_mma_prefill(p, Q, K, V, idx, sink, O, LSE, st)
-                        : launch_sparse_generic(p, hp->dtype, Q, K, V, idx, sink, O, LSE, st);
+    cudaError_t e = cudaErrorNotSupported;
+    if (sparse_mma_supported(p, hp->dtype) && aligned16(Q, K, V, O)) {
+        e = launch_sparse_mma_prefill(p, Q, K, V, idx, sink, O, LSE, st);
+    } else {
+        // large head groups (the paper's 64 heads per KV head): the gather tile is a dense contraction
+        if (!g_disable_tc5.load(std::memory_order_relaxed) && sparse_tc5_supported(p, hp->dtype) && aligned16(Q, K, V, O))
+            e = launch_sparse_tc5(p, Q, K, V, idx, sink, O, LSE, st);
+        if (e == cudaErrorNotSupported) {
+            (void)cudaGetLastError();
+            e = launch_sparse_generic(p, hp->dtype, Q, K, V, idx, sink, O, LSE, st);
+        }
+    }
     return e == cudaSuccess ? HS2_OK : cuda_fail(e);
 }
 
@@ -380,10 +389,11 @@ int hs2_last_cuda_error(void) { return g_last_cuda_error; }
 int hs2_device_error_flags(unsigned *flags)
 {
     if (!flags) return HS2_ERR_INVALID_ARG;
-    unsigned a = 0, b = 0;
+    unsigned a = 0, b = 0, c = 0;
     cudaError_t e = read_tc5_error(&a);
     if (e == cudaSuccess) e = read_sparse_error(&b);
-    *flags = a | (b << 8);   // bits 8.. : the sparse kernels
+    if (e == cudaSuccess) e = read_sparse_tc5_error(&c);
+    *flags = a | (b << 8) | (c << 16);   // bits 8.. : the mma.sync sparse kernels, bits 16.. : the tcgen05 sparse kernel
     return e == cudaSuccess ? HS2_OK : cuda_fail(e);
 }
 

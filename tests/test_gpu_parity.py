@@ -254,6 +254,34 @@ def test_paper_native_shape_mqa64_dim256_with_sink():
     assert (od.float() - out[:, -1:].float()).abs().max().item() <= 2e-2
 
 
+def test_tcgen05_sparse_kernel_large_head_groups():
+    """Groups of more than 8 heads take the tensor-core gather kernel: odd group sizes, both head dims, ragged
+    lengths, sink, several KV heads; every row against the oracle and against the SIMT kernel."""
+    cases = [
+        dict(q_len=90, kv_len=500, k_sel=100, window=20, n_q_heads=96, n_kv_heads=2, head_dim=256, batch=2),   # G = 48
+        dict(q_len=70, kv_len=330, k_sel=64, window=64, n_q_heads=128, n_kv_heads=1, head_dim=128),            # G = 128
+        dict(q_len=150, kv_len=150, k_sel=7, window=3, n_q_heads=24, n_kv_heads=2, head_dim=128),              # one ragged tile
+        dict(q_len=64, kv_len=400, k_sel=0, window=130, n_q_heads=64, n_kv_heads=1, head_dim=256),             # window only
+    ]
+    for over in cases:
+        wl = scaled("cfg2", n_needles=4, **over)
+        run = BlockRun(make_inputs(wl)).run_full()
+        sink = torch.linspace(-1.5, 2.5, wl.n_q_heads, device="cuda")
+        for sk in (None, sink):
+            out, lse = run.run_sparse(0, sink=sk)
+            run.check_sparse(out, lse, 0, sink=sk)
+            old = hs2.hs2_set_tcgen05_enabled(0)
+            try:
+                out_g, lse_g = run.run_sparse(0, sink=sk)
+            finally:
+                hs2.hs2_set_tcgen05_enabled(old)
+            assert (out.float() - out_g.float()).abs().max().item() <= 2e-2
+            fin = torch.isfinite(lse_g)
+            assert torch.equal(torch.isfinite(lse), fin)
+            assert (lse[fin] - lse_g[fin]).abs().max().item() <= 2e-3
+    assert hs2.hs2_device_error_flags() == 0
+
+
 def test_ragged_lengths_offsets_strides_and_sink():
     wl = scaled("cfg2", batch=3, q_len=70, kv_len=400, k_sel=40, window=12, n_needles=4)
     inp = make_inputs(wl)
