@@ -3,16 +3,21 @@
 // paper's own models share one KV head among 64 query heads of dimension 256).
 //
 // With G = 64 heads per KV head every gathered key row is used by 64 heads, i.e. 64 flop per byte: the
-// gather tile is a dense contraction and belongs on tcgen05.  One CTA = one (sequence, KV head, query):
-//   rows of the MMA (M = 128, TMEM lane) = the G heads of the group (lanes >= G hold don't-care rows),
+// gather tile is a dense contraction and belongs on tcgen05.  Work item = one (sequence, KV head, sub-group
+// of up to 64 heads, query); persistent CTAs walk the items with all pipelines running across item boundaries.
+//   rows of the MMA (M = 128, TMEM lane) = the heads of the item (lanes >= 64 hold don't-care rows),
 //   columns = 64 gathered keys per tile.
-//   warps 5-7  gather producers: slot s of the virtual array [idx row | window] -> key index -> the key's
-//              K and V rows copied with 16-byte cp.async into the 128-byte-swizzled UMMA operand layout
-//              (void slots are zero filled), 2-stage ring, then a generic->async proxy fence and an
-//              mbarrier arrive per thread.  Q (G rows) arrives by TMA.
-//   warp 4     MMA issuer: S = Q K^T (M128 N64 K=D) into one of two TMEM buffers, O += P V (V MN-major).
-//   warps 0-3  one thread per head: online softmax in the base-2 domain exactly as in the full-attention
-//              kernel, void slots masked by a 64-bit validity word, optional sink logit in the denominator.
+//   gather warps  slot s of the virtual array [idx row | window] -> key index -> the key's K or V row copied
+//              with 16-byte cp.async into the 128-byte-swizzled UMMA operand layout (void slots are zero
+//              filled).  K and V have warp groups and rings of their own (K is released as soon as Q K^T has
+//              read it, V after P V); completion reaches the mbarrier without blocking the thread
+//              (cp.async.mbarrier.arrive).  The copy rate grows with the number of issuing warps, hence four
+//              warps per group at head_dim 256.  Q (the item's heads) arrives by TMA.
+//   MMA warp   S = Q K^T (M128 N64 K=D) into one of two TMEM buffers, O += P V (V as MN-major B operand).
+//   softmax    four warps, two threads per head (32 keys of the tile each; the row maximum is exchanged through
+//              shared memory): online softmax in the base-2 domain with a lazily rescaled accumulator as in
+//              the full-attention kernel, void slots masked, optional sink logit in the denominator; P is
+//              double buffered so that the exponentials of tile g+1 overlap P V of tile g.
 // Every mbarrier wait is bounded; a wait that runs out sets a device error word, the CTA drains its copies,
 // frees its TMEM and returns.
 #include <cuda.h>
@@ -29,32 +34,60 @@ namespace {
 using namespace tc5;
 
 constexpr int BM = 128, BN = 64;
-constexpr int kThreads = 256;
-constexpr int kFirstProducerWarp = 5;
-constexpr int kProducers = 96;
-constexpr uint32_t kBarBytes = 128;
+// Warps per gather group at head_dim 256.  Measured on the paper's shape (64 heads, 1152 keys per query): 2 -> 2.17 ms,
+// 3 -> 1.77 ms, 4 -> 1.60 ms, 5 -> 1.64 ms, 6 -> 2.28 ms (register cap forces spills).
+#ifndef HS2_SP_PWARPS
+#define HS2_SP_PWARPS 4
+#endif
+constexpr int kSubHeads = 64;              // heads per work item (a larger group is walked in sub-groups)
+constexpr uint32_t kBarBytes = 256;
 constexpr uint32_t kAlignSlack = 896;
 constexpr float kRescaleThreshold = 8.f;   // log2 units
 
+// Warp roles (the TMEM lanes 0-63 that hold the 64 heads are only reachable from warps with index % 4 in {0, 1}):
+//   0, 1, 4, 5  softmax: warp & 1 = TMEM lane quadrant (heads 0-31 / 32-63), warp >> 2 = column half of the tile
+//   2           MMA issuer (also owns the TMEM allocation)
+//   3, 6, 7..   gather producers: the first PW of them copy K, the next PW copy V
+__device__ __forceinline__ bool is_softmax_warp(int w) { return w < 6 && (w & 3) < 2; }
+__device__ __forceinline__ int producer_ordinal(int w) { return w == 3 ? 0 : w - 5; }
+
+// Shared-memory plan for head_dim D.  The MMA always reads 128 A rows per 64-dim slice of Q; rows past the 64
+// that are loaded alias whatever follows (the next slice or the K ring), which is harmless: they only produce
+// TMEM lanes that nobody reads.
 template <int D>
 struct SpCfg {
     static constexpr int NQ = D / 64;                           // 64-dim slices of an operand tile
     static constexpr int CH = D / 8;                            // 16-byte chunks per row
-    static constexpr uint32_t kQBytes = NQ * BM * 128;
+    static constexpr int KST = D == 256 ? 3 : 2;                // K ring depth (V ring: 2)
+    static constexpr int PW = D == 256 ? HS2_SP_PWARPS : 1;     // warps per gather group (one K group, one V group)
+    static constexpr int kThreads = (5 + 2 * PW) * 32;
+    static constexpr uint32_t kQSlice = kSubHeads * 128;
+    static constexpr uint32_t kQBytes = NQ * kQSlice;
     static constexpr uint32_t kKVStage = NQ * BN * 128;
     static constexpr uint32_t kOffQ = 0;
-    static constexpr uint32_t kOffK = kOffQ + kQBytes;
-    static constexpr uint32_t kOffV = kOffK + 2 * kKVStage;
-    static constexpr uint32_t kOffP = kOffV + 2 * kKVStage;     // 128 rows x 64 keys bf16
-    static constexpr uint32_t kOffKey = kOffP + BM * 128;       // int[2][64]: key index per slot of a stage
-    static constexpr uint32_t kOffMask = kOffKey + 512;         // uint32[2][2]: validity bits of a stage
-    static constexpr uint32_t kOffBar = kOffMask + 64;
+    // two P buffers of 64 real rows x 64 keys bf16, 8 KB apart; the 128 rows the MMA reads from the second one run
+    // on into the K ring (don't-care rows again)
+    static constexpr uint32_t kOffP = kOffQ + kQBytes;
+    static constexpr uint32_t kPStride = kSubHeads * 128;
+    static constexpr uint32_t kOffK = kOffP + 2 * kPStride;
+    static constexpr uint32_t kOffV = kOffK + KST * kKVStage;
+    static constexpr uint32_t kOffKey = kOffV + 2 * kKVStage;   // int[2 groups][2][64]: key index per slot of a tile
+    static constexpr uint32_t kOffMx = kOffKey + 4 * BN * 4;    // float[2 tiles][2 halves][64]: row maxima exchanged
+    static constexpr uint32_t kOffL = kOffMx + 4 * 64 * 4;      // float[2 halves][64]: row sums exchanged
+    static constexpr uint32_t kOffBar = kOffL + 2 * 64 * 4;
     static constexpr uint32_t kSmemBytes = kOffBar + kBarBytes + kAlignSlack;
     static constexpr uint32_t kTmem = D <= 128 ? 256 : 512;     // 2 x 64 score columns + D output columns
     static constexpr int kMinBlocks = D <= 128 ? 2 : 1;
+    static_assert(kOffQ + (NQ - 1) * kQSlice + BM * 128 <= kOffKey && kOffP + kPStride + BM * 128 <= kOffKey,
+                  "the 128 A rows the MMA reads stay inside the buffer");
+    static_assert(kSmemBytes <= 227 * 1024, "fits the shared memory of one SM");
 };
 
-enum Bar { Q_FULL = 0, KV_FULL0, KV_FULL1, KV_EMPTY0, KV_EMPTY1, S_FULL0, S_FULL1, S_FREE0, S_FREE1, P_FULL, PV_DONE, N_BARS };
+enum Bar {
+    Q_FULL = 0, Q_EMPTY, K_FULL0, K_FULL1, K_FULL2, K_EMPTY0, K_EMPTY1, K_EMPTY2, V_FULL0, V_FULL1, V_EMPTY0, V_EMPTY1,
+    S_FULL0, S_FULL1, S_FREE0, S_FREE1, P_FULL0, P_FULL1, PV_DONE0, PV_DONE1, O_FREE, N_BARS
+};
+static_assert(N_BARS * 8 + 8 <= kBarBytes, "barriers, TMEM slot and abort flag fit their block");
 
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag)
 {
@@ -62,27 +95,48 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
 }
 __device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, int src_bytes)
 {
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+    // .ca: measured a little faster than .cg here (the rows of a tile are touched once either way)
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
 }
-__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::: "memory"); }
-template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N) : "memory"); }
-// barrier over the producer threads that also ANDs a predicate (named barrier 1)
-__device__ __forceinline__ bool producers_all(bool pred)
+// the mbarrier receives one arrival from this thread once all its earlier cp.async copies have landed
+__device__ __forceinline__ void cp_async_arrive(uint32_t bar)
+{
+    asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];\n" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;\n" ::: "memory"); }
+// named barrier `id` over `count` threads that also ANDs a predicate
+__device__ __forceinline__ bool group_all(int id, int count, bool pred)
 {
     uint32_t out;
-    asm volatile("{\n .reg .pred p, q;\n setp.ne.b32 p, %1, 0;\n barrier.cta.red.and.pred q, 1, %2, p;\n selp.u32 %0, 1, 0, q;\n}\n"
-                 : "=r"(out) : "r"((uint32_t)pred), "n"(kProducers) : "memory");
+    asm volatile("{\n .reg .pred p, q;\n setp.ne.b32 p, %1, 0;\n barrier.cta.red.and.pred q, %2, %3, p;\n selp.u32 %0, 1, 0, q;\n}\n"
+                 : "=r"(out) : "r"((uint32_t)pred), "r"(id), "r"(count) : "memory");
     return out != 0;
 }
 
+// Slot s of the virtual slot array [idx row | window] of a query at position pos holds a key index or is void (-1).
+// slot_raw starts the fetch (an idx entry is a global load) and slot_fix applies the validity rules to it; callers
+// keep the raw value in a register for a whole tile so that the load's latency is never waited for.
+__device__ __forceinline__ int slot_raw(const Params &p, const int32_t *irow, int pos, int s)
+{
+    if (s < p.k) return irow ? __ldg(irow + s) : -1;
+    return s < p.k + p.w ? pos - p.w + 1 + (s - p.k) : -1;
+}
+__device__ __forceinline__ int slot_fix(const Params &p, int j, int pos, int kvl, int s)
+{
+    const int hi = s < p.k ? pos - p.w : pos;   // idx entries inside the window are void: the window slots cover them
+    return (j < 0 || j > hi || j >= kvl) ? -1 : j;
+}
+
+// Persistent: every CTA walks items blockIdx.x, blockIdx.x + gridDim.x, ...  All rings and phases are indexed by
+// the running tile number g = (items done by this CTA) * nblk + t, which every role computes for itself.
 template <int D>
-__global__ void __launch_bounds__(kThreads, SpCfg<D>::kMinBlocks)
+__global__ void __launch_bounds__(SpCfg<D>::kThreads, SpCfg<D>::kMinBlocks)
 k_sparse_tc5(const __grid_constant__ CUtensorMap tmQ, const Params p, const __nv_bfloat16 *__restrict__ K,
              const __nv_bfloat16 *__restrict__ V, const int32_t *__restrict__ idx, const float *__restrict__ sink,
-             __nv_bfloat16 *__restrict__ O, float *__restrict__ LSE)
+             __nv_bfloat16 *__restrict__ O, float *__restrict__ LSE, int64_t n_items, int n_sub)
 {
     using C = SpCfg<D>;
-    constexpr int NQ = C::NQ, CH = C::CH;
+    constexpr int NQ = C::NQ, CH = C::CH, KST = C::KST;
     constexpr uint32_t kKVStage = C::kKVStage;
     extern __shared__ char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -97,31 +151,44 @@ k_sparse_tc5(const __grid_constant__ CUtensorMap tmQ, const Params p, const __nv
     uint32_t *tmem_slot = reinterpret_cast<uint32_t *>(smem + C::kOffBar + N_BARS * 8);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + C::kOffBar + N_BARS * 8 + 4);
     int *s_key = reinterpret_cast<int *>(smem + C::kOffKey);
-    uint32_t *s_mask = reinterpret_cast<uint32_t *>(smem + C::kOffMask);
+    float *s_mx = reinterpret_cast<float *>(smem + C::kOffMx);
+    float *s_l = reinterpret_cast<float *>(smem + C::kOffL);
     auto bar = [&](int i) { return bars + 8u * i; };
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int64_t item = blockIdx.x;                 // (b, g, i) flattened
-    const int i = (int)(item % p.Lq);
-    const int bg = (int)(item / p.Lq);
-    const int gkv = bg % p.Hkv, b = bg / p.Hkv;
-    const int kvl = kvlen_of(p, b);
-    const int pos = pos_of(p, b, i);
     const int nblk = (p.k + p.w + BN - 1) / BN;      // tiles of the virtual slot array [idx row | window]
-    const int n_soft_warps = (p.G + 31) / 32;
+    // item -> (sequence, KV head, sub-group of heads, query, position)
+    struct Where { int b, gkv, sub, i, kvl, pos; };
+    auto where = [&](int64_t item) {
+        Where wq;
+        wq.i = (int)(item % p.Lq);
+        const int r = (int)(item / p.Lq);
+        wq.sub = r % n_sub;
+        const int bg = r / n_sub;
+        wq.gkv = bg % p.Hkv;
+        wq.b = bg / p.Hkv;
+        wq.kvl = kvlen_of(p, wq.b);
+        wq.pos = pos_of(p, wq.b, wq.i);
+        return wq;
+    };
+    auto irow_of = [&](const Where &wq) {
+        return (p.k > 0 && idx) ? idx + (((int64_t)wq.b * p.Hkv + wq.gkv) * p.Lq + wq.i) * p.k : (const int32_t *)nullptr;
+    };
+    const int box_heads = p.G < kSubHeads ? p.G : kSubHeads;
 
     if (tid == 0) {
         *abort_flag = 0;
-        mbar_init(bar(Q_FULL), 1);
-        mbar_init(bar(KV_FULL0), kProducers); mbar_init(bar(KV_FULL1), kProducers);
-        mbar_init(bar(KV_EMPTY0), 1); mbar_init(bar(KV_EMPTY1), 1);
-        mbar_init(bar(S_FULL0), 1); mbar_init(bar(S_FULL1), 1);
-        mbar_init(bar(S_FREE0), 32 * n_soft_warps); mbar_init(bar(S_FREE1), 32 * n_soft_warps);
-        mbar_init(bar(P_FULL), 32 * n_soft_warps);
-        mbar_init(bar(PV_DONE), 1);
+        mbar_init(bar(Q_FULL), 1); mbar_init(bar(Q_EMPTY), 1);
+        for (int s = 0; s < 3; ++s) { mbar_init(bar(K_FULL0 + s), 32 * C::PW); mbar_init(bar(K_EMPTY0 + s), 1); }
+        for (int s = 0; s < 2; ++s) {
+            mbar_init(bar(V_FULL0 + s), 32 * C::PW); mbar_init(bar(V_EMPTY0 + s), 1);
+            mbar_init(bar(S_FULL0 + s), 1); mbar_init(bar(S_FREE0 + s), 128);
+            mbar_init(bar(P_FULL0 + s), 128); mbar_init(bar(PV_DONE0 + s), 1);
+        }
+        mbar_init(bar(O_FREE), 128);
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
-    if (warp == 4) {
+    if (warp == 2) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(tmem_slot)), "r"(C::kTmem) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
     }
@@ -130,216 +197,274 @@ k_sparse_tc5(const __grid_constant__ CUtensorMap tmQ, const Params p, const __nv
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
 
-    if (warp >= kFirstProducerWarp) {
-        // ------------------------------------------------ gather producers
-        const int ptid = tid - kFirstProducerWarp * 32;
-        const char *Kb = reinterpret_cast<const char *>(K + b * p.ks_b + gkv * p.ks_h);
-        const char *Vb = reinterpret_cast<const char *>(V + b * p.ks_b + gkv * p.ks_h);
-        const int64_t row_bytes = p.ks_t * 2;
-        const int32_t *irow = (p.k > 0 && idx) ? idx + (((int64_t)b * p.Hkv + gkv) * p.Lq + i) * p.k : nullptr;
-        if (ptid == 0 && nblk > 0) {
-            mbar_expect_tx(bar(Q_FULL), (uint32_t)(NQ * p.G * 128));
+    if (is_softmax_warp(warp)) {
+        // ------------------------------------------------ softmax: two threads per head, 32 keys of a tile each
+        // Every thread of a quadrant pair executes the same sequence of pair barriers; a wait that runs out only
+        // marks the thread dead, and the next pair barrier then ends both loops together.
+        const int quad = warp & 1, half = warp >> 2;
+        const int row = 32 * quad + lane;
+        const int pair_bar = 3 + quad;
+        const uint32_t lane_base = tmem + ((uint32_t)(32 * quad) << 16);
+        const uint32_t o_col0 = 2 * BN + half * (D / 2);    // this thread's half of the output columns
+        bool alive = true, dead = false;
+        int n = 0;
+        for (int64_t item = blockIdx.x; item < n_items && alive; item += gridDim.x, ++n) {
+            const Where q = where(item);
+            const bool real = row < min(kSubHeads, p.G - kSubHeads * q.sub);
+            const int h = q.gkv * p.G + kSubHeads * q.sub + (real ? row : 0);
+            const int32_t *irow = irow_of(q);
+            float m_used = -INFINITY, l = 0.f;
+            if (sink && real) {   // Section 3.3 variant with a learnable sink logit: it only joins the denominator
+                m_used = sink[h] * kLog2e;
+                l = half == 0 ? 1.f : 0.f;
+            }
+            const int g0 = n * nblk;
+            // validity of this half's 32 slots is recomputed here (cheap, and no cross-warp visibility to argue
+            // about), one tile ahead so that the idx loads are off the critical path
+            int jn = slot_raw(p, irow, q.pos, 32 * half + lane);
+            for (int t = 0; t < nblk; ++t) {
+                const int g = g0 + t, sb = g & 1;
+                const uint32_t valid = __ballot_sync(0xffffffffu, slot_fix(p, jn, q.pos, q.kvl, t * BN + 32 * half + lane) >= 0);
+                if (t + 1 < nblk) jn = slot_raw(p, irow, q.pos, (t + 1) * BN + 32 * half + lane);
+                if (!dead && !__all_sync(0xffffffffu, mbar_wait(bar(S_FULL0 + sb), (g >> 1) & 1, abort_flag))) dead = true;
+                float s[32];
+                float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+                if (!dead) {
+                    tc_fence_after();
+                    tmem_ld32(lane_base + sb * BN + 32 * half, s);
+                    tmem_wait_ld();
+                    tc_fence_before();
+                    mbar_arrive(bar(S_FREE0 + sb));
+                    if (valid != 0xffffffffu) {
 #pragma unroll
-            for (int sl = 0; sl < NQ; ++sl) tma_load_4d(sbase + C::kOffQ + sl * BM * 128, &tmQ, bar(Q_FULL), 64 * sl, gkv * p.G, i, b);
-        }
-        int issued = 0, arrived = 0;   // tiles copied / tiles handed over
-        for (int t = 0; t < nblk; ++t) {
-            const int st = t & 1;
-            if (t > 0) {
-                // hand the previous tile to the tensor core BEFORE waiting for this stage to drain: the stage is
-                // released by P V of tile t-2, which the issuer orders after Q K^T of tile t-1
-                cp_async_wait<0>();
-                fence_proxy_async();
-                mbar_arrive(bar(KV_FULL0 + ((t - 1) & 1)));
-                arrived = t;
-            }
-            const bool ok = __all_sync(0xffffffffu, mbar_wait(bar(KV_EMPTY0 + st), ((t >> 1) & 1) ^ 1, abort_flag));
-            if (ok && ptid < BN) {   // warps 5 and 6: one slot each
-                const int s = t * BN + ptid;
-                int j = -1;
-                if (s < p.k) {
-                    j = irow ? __ldg(irow + s) : -1;
-                    if (j > pos - p.w || j >= kvl) j = -1;
-                } else if (s < p.k + p.w) {
-                    j = pos - p.w + 1 + (s - p.k);
-                    if (j > pos || j >= kvl) j = -1;
+                        for (int e = 0; e < 32; ++e)
+                            if (!((valid >> e) & 1u)) s[e] = -INFINITY;
+                    }
+#pragma unroll
+                    for (int e = 0; e < 32; e += 4) {
+                        mx0 = fmaxf(mx0, s[e]); mx1 = fmaxf(mx1, s[e + 1]); mx2 = fmaxf(mx2, s[e + 2]); mx3 = fmaxf(mx3, s[e + 3]);
+                    }
                 }
-                s_key[st * BN + ptid] = j;
-                const uint32_t m = __ballot_sync(0xffffffffu, j >= 0);
-                if (lane == 0) s_mask[st * 2 + (ptid >> 5)] = m;
+                float m_raw = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+                s_mx[((g & 1) * 2 + half) * 64 + row] = m_raw;
+                if (!group_all(pair_bar, 64, !dead)) { alive = false; break; }
+                m_raw = fmaxf(m_raw, s_mx[((g & 1) * 2 + (half ^ 1)) * 64 + row]);
+                const float m_blk = m_raw * p.scale_log2;
+                const bool need = m_blk > m_used + kRescaleThreshold;
+                const float m_new = need ? m_blk : m_used;
+                const float corr = need ? exp2f(m_used - m_new) : 1.f;
+                // P V of tile g-2 has read the P buffer this tile writes (two buffers, two barriers: a barrier's next
+                // completion always depends on this thread, so a parity wait can never be a phase behind)
+                if (g > 1 && !dead && !__all_sync(0xffffffffu, mbar_wait(bar(PV_DONE0 + sb), ((g - 2) >> 1) & 1, abort_flag))) dead = true;
+                if (t > 0 && __any_sync(0xffffffffu, need)) {   // rare: rescale the accumulator, after P V of tile g-1
+                    if (!dead && !__all_sync(0xffffffffu, mbar_wait(bar(PV_DONE0 + (sb ^ 1)), ((g - 1) >> 1) & 1, abort_flag))) dead = true;
+                    if (!dead) {
+                        tc_fence_after();
+#pragma unroll
+                        for (int cc = 0; cc < D / 64; ++cc) {
+                            float o[32];
+                            tmem_ld32(lane_base + o_col0 + cc * 32, o);
+                            tmem_wait_ld();
+#pragma unroll
+                            for (int e = 0; e < 32; ++e) o[e] *= corr;
+                            tmem_st32(lane_base + o_col0 + cc * 32, o);
+                        }
+                        tmem_wait_st();
+                    }
+                }
+                l *= corr;
+                m_used = m_new;
+                if (!dead) {
+                    const float neg_m = m_used == -INFINITY ? 0.f : -m_used;
+                    uint32_t pk[16];
+                    float l0 = 0.f, l1 = 0.f;
+#pragma unroll
+                    for (int e = 0; e < 32; e += 2) {
+                        const float p0 = exp2f(fmaf(s[e], p.scale_log2, neg_m));       // -inf stays -inf -> 0
+                        const float p1 = exp2f(fmaf(s[e + 1], p.scale_log2, neg_m));
+                        l0 += p0; l1 += p1;
+                        pk[e >> 1] = pack_bf16(p0, p1);
+                    }
+                    l += l0 + l1;
+                    char *prow_ptr = smem + C::kOffP + sb * C::kPStride + row * 128;
+#pragma unroll
+                    for (int c4 = 0; c4 < 4; ++c4)   // 8 keys = one 16-byte chunk, chunk position XOR (row & 7)
+                        *reinterpret_cast<uint4 *>(prow_ptr + (((half * 4 + c4) ^ (row & 7)) << 4)) =
+                            make_uint4(pk[4 * c4], pk[4 * c4 + 1], pk[4 * c4 + 2], pk[4 * c4 + 3]);
+                    fence_proxy_async();
+                    tc_fence_before();
+                    mbar_arrive(bar(P_FULL0 + sb));
+                }
             }
-            if (!producers_all(ok)) break;   // also publishes the key indices to the other producer threads
-            const uint32_t kdst = sbase + C::kOffK + st * kKVStage, vdst = sbase + C::kOffV + st * kKVStage;
-            for (int e = ptid; e < 2 * BN * CH; e += kProducers) {
-                const int isv = e / (BN * CH);
-                const int r = (e / CH) % BN, c = e % CH;
-                const int j = s_key[st * BN + r];
-                const char *src = (isv ? Vb : Kb) + (j >= 0 ? (int64_t)j * row_bytes + c * 16 : 0);
-                const uint32_t dst = (isv ? vdst : kdst) + (c >> 3) * (BN * 128) + r * 128 + (((c & 7) ^ (r & 7)) << 4);
-                cp_async16(dst, src, j >= 0 ? 16 : 0);
+            if (!alive) break;
+            // ---- epilogue of the item: both P V barriers (every completion is observed, none can lap a wait)
+            {
+                const int gl = g0 + nblk - 1;
+                if (!dead && gl > 0 && !__all_sync(0xffffffffu, mbar_wait(bar(PV_DONE0 + ((gl - 1) & 1)), ((gl - 1) >> 1) & 1, abort_flag))) dead = true;
+                if (!dead && !__all_sync(0xffffffffu, mbar_wait(bar(PV_DONE0 + (gl & 1)), (gl >> 1) & 1, abort_flag))) dead = true;
             }
-            cp_async_commit();
-            issued = t + 1;
+            s_l[half * 64 + row] = l;
+            if (!group_all(pair_bar, 64, !dead)) { alive = false; break; }
+            l += s_l[(half ^ 1) * 64 + row];
+            tc_fence_after();
+            const bool any = l > 0.f && m_used != -INFINITY;
+            const float inv = any ? 1.f / l : 0.f;
+            __nv_bfloat16 *orow = O + q.b * p.os_b + (int64_t)q.i * p.os_t + h * p.os_h + half * (D / 2);
+#pragma unroll
+            for (int cc = 0; cc < D / 64; ++cc) {
+                float o[32];
+                tmem_ld32(lane_base + o_col0 + cc * 32, o);
+                tmem_wait_ld();
+                if (cc == D / 64 - 1) {   // the accumulator may now be overwritten by the next item
+                    tc_fence_before();
+                    mbar_arrive(bar(O_FREE));
+                }
+                if (real) {
+#pragma unroll
+                    for (int q4 = 0; q4 < 4; ++q4) {
+                        uint4 v;
+                        v.x = pack_bf16(o[8 * q4 + 0] * inv, o[8 * q4 + 1] * inv);
+                        v.y = pack_bf16(o[8 * q4 + 2] * inv, o[8 * q4 + 3] * inv);
+                        v.z = pack_bf16(o[8 * q4 + 4] * inv, o[8 * q4 + 5] * inv);
+                        v.w = pack_bf16(o[8 * q4 + 6] * inv, o[8 * q4 + 7] * inv);
+                        *reinterpret_cast<uint4 *>(orow + cc * 32 + q4 * 8) = v;
+                    }
+                }
+            }
+            if (real && half == 0 && LSE) LSE[((int64_t)q.b * p.Hq + h) * p.Lq + q.i] = any ? (m_used + log2f(l)) * kLn2 : -INFINITY;
         }
-        cp_async_wait<0>();   // also on the abort path: nothing stays in flight
-        if (issued > arrived) {
-            fence_proxy_async();
-            mbar_arrive(bar(KV_FULL0 + ((issued - 1) & 1)));
-        }
-        if (ptid == 0 && nblk > 0 && *abort_flag)
-            for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait(bar(Q_FULL), 0); ++it) {}
-    } else if (warp == 4) {
+    } else if (warp == 2) {
         // ------------------------------------------------ MMA issuer
-        if (elect_one() && nblk > 0) {
+        if (elect_one()) {
             constexpr uint32_t idS = idesc(BM, BN, 0), idPV = idesc(BM, D, 1);
-            bool ok = mbar_wait(bar(Q_FULL), 0, abort_flag);
-            auto issue_s = [&](int j) -> bool {
-                const int st = j & 1, ph = (j >> 1) & 1;
-                if (!mbar_wait(bar(KV_FULL0 + st), ph, abort_flag)) return false;
-                if (!mbar_wait(bar(S_FREE0 + st), ph ^ 1, abort_flag)) return false;
-                tc_fence_after();
-                const uint32_t qa = sbase + C::kOffQ, ka = sbase + C::kOffK + st * kKVStage;
+            const uint64_t dq = smem_desc(sbase + C::kOffQ, 16, 1024);
+            bool ok = true;
+            int n = 0;
+            for (int64_t item = blockIdx.x; item < n_items && ok; item += gridDim.x, ++n) {
+                const int g0 = n * nblk;
+                auto issue_s = [&](int t) -> bool {
+                    const int g = g0 + t, ks = g % KST, sb = g & 1;
+                    if (!mbar_wait(bar(K_FULL0 + ks), (g / KST) & 1, abort_flag)) return false;
+                    if (!mbar_wait(bar(S_FREE0 + sb), ((g >> 1) & 1) ^ 1, abort_flag)) return false;
+                    fence_proxy_async();   // the gathered rows were written through the generic proxy
+                    tc_fence_after();
+                    const uint64_t dk = smem_desc(sbase + C::kOffK + ks * kKVStage, 16, 1024);
 #pragma unroll
-                for (int ks = 0; ks < D / 16; ++ks) {
-                    const uint32_t off = (ks & 3) * 32;
-                    const uint64_t da = smem_desc(qa + (ks >> 2) * (BM * 128) + off, 16, 1024);
-                    const uint64_t db = smem_desc(ka + (ks >> 2) * (BN * 128) + off, 16, 1024);
-                    umma(tmem + st * BN, da, db, idS, ks > 0);
-                }
-                umma_commit(bar(S_FULL0 + st));
-                return true;
-            };
-            ok = ok && issue_s(0);
-            for (int j = 0; ok && j < nblk; ++j) {
-                if (j + 1 < nblk && !issue_s(j + 1)) break;
-                if (!mbar_wait(bar(P_FULL), j & 1, abort_flag)) break;
-                tc_fence_after();
-                const int st = j & 1;
-                const uint32_t pa = sbase + C::kOffP, va = sbase + C::kOffV + st * kKVStage;
+                    for (int kk = 0; kk < D / 16; ++kk) {   // descriptor address field counts 16-byte units
+                        umma(tmem + sb * BN, dq + (((kk >> 2) * C::kQSlice + (kk & 3) * 32) >> 4),
+                             dk + (((kk >> 2) * (BN * 128) + (kk & 3) * 32) >> 4), idS, kk > 0);
+                    }
+                    umma_commit(bar(S_FULL0 + sb));
+                    umma_commit(bar(K_EMPTY0 + ks));
+                    if (t == nblk - 1) umma_commit(bar(Q_EMPTY));
+                    return true;
+                };
+                ok = mbar_wait(bar(Q_FULL), n & 1, abort_flag);
+                ok = ok && issue_s(0);
+                for (int t = 0; ok && t < nblk; ++t) {
+                    if (t + 1 < nblk && !issue_s(t + 1)) { ok = false; break; }
+                    const int g = g0 + t, vs = g & 1;
+                    if (!mbar_wait(bar(P_FULL0 + vs), (g >> 1) & 1, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(bar(V_FULL0 + vs), (g >> 1) & 1, abort_flag) ||
+                        (t == 0 && !mbar_wait(bar(O_FREE), (n & 1) ^ 1, abort_flag))) { ok = false; break; }
+                    fence_proxy_async();
+                    tc_fence_after();
+                    const uint64_t dp = smem_desc(sbase + C::kOffP + vs * C::kPStride, 16, 1024);
+                    // V: MN-major B operand, 64-dim slices BN*128 bytes apart (leading offset), 8-key groups 1024 bytes apart
+                    const uint64_t dv = smem_desc(sbase + C::kOffV + vs * kKVStage, BN * 128, 1024);
 #pragma unroll
-                for (int kk = 0; kk < 4; ++kk) {
-                    const uint64_t da = smem_desc(pa + kk * 32, 16, 1024);
-                    const uint64_t db = smem_desc(va + kk * 2048, BN * 128, 1024);
-                    umma(tmem + 2 * BN, da, db, idPV, (j > 0 || kk > 0) ? 1u : 0u);
+                    for (int kk = 0; kk < 4; ++kk) {   // 16 keys per instruction
+                        umma(tmem + 2 * BN, dp + ((kk * 32) >> 4), dv + ((kk * 2048) >> 4), idPV, (t > 0 || kk > 0) ? 1u : 0u);
+                    }
+                    umma_commit(bar(V_EMPTY0 + vs));
+                    umma_commit(bar(PV_DONE0 + vs));
                 }
-                umma_commit(bar(KV_EMPTY0 + st));
-                umma_commit(bar(PV_DONE));
             }
         }
-    } else if (warp < n_soft_warps) {
-        // ------------------------------------------------ softmax: one thread per head of the group
-        const int row = tid;
-        const bool real = row < p.G;
-        const int h = gkv * p.G + (real ? row : 0);
-        const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
-        float m_used = -INFINITY, l = 0.f;
-        if (sink && real) {   // Section 3.3 variant with a learnable sink logit: it only joins the denominator
-            m_used = sink[h] * kLog2e;
-            l = 1.f;
+    } else {
+        // ------------------------------------------------ gather producers: a K group and a V group of PW warps
+        // The groups run independently (own key records, own named barrier), so K can run KST tiles ahead of the
+        // tensor core while V waits for P V to release its stage.
+        // Thread -> one 16-byte chunk column c and every RPI-th row: a warp instruction copies whole key rows.
+        constexpr int GT = 32 * C::PW;                // threads per group
+        constexpr int RPI = GT / CH;                  // rows per iteration of the copy loop
+        constexpr int KPT = (BN + GT - 1) / GT;       // key records per thread
+        static_assert(GT % CH == 0, "a group's threads tile whole rows");
+        const int po = producer_ordinal(warp);
+        const int is_v = po / C::PW;
+        const int gtid = (po % C::PW) * 32 + lane;
+        const int c = gtid % CH, r0 = gtid / CH;
+        const uint32_t dst_c = (uint32_t)(c >> 3) * (BN * 128);
+        const int64_t row_bytes = p.ks_t * 2;
+        const __nv_bfloat16 *src_t = is_v ? V : K;
+        const uint32_t ring0 = sbase + (is_v ? C::kOffV : C::kOffK) + dst_c;
+        const int nst = is_v ? 2 : KST;
+        const int bar_full = is_v ? V_FULL0 : K_FULL0, bar_empty = is_v ? V_EMPTY0 : K_EMPTY0;
+        int *keys_base = s_key + is_v * 2 * BN;       // two records per group
+        // the key indices of a tile are fetched one tile ahead (the idx row is read from global memory, and that
+        // latency would otherwise sit in front of every tile's copies)
+        int j_next[KPT];
+#pragma unroll
+        for (int u = 0; u < KPT; ++u) j_next[u] = -1;
+        if ((int64_t)blockIdx.x < n_items) {
+            const Where q0 = where(blockIdx.x);
+#pragma unroll
+            for (int u = 0; u < KPT; ++u)
+                if (gtid + u * GT < BN) j_next[u] = slot_raw(p, irow_of(q0), q0.pos, gtid + u * GT);
         }
         bool alive = true;
-        for (int j = 0; j < nblk && alive; ++j) {
-            const int sb = j & 1;
-            if (!__all_sync(0xffffffffu, mbar_wait(bar(S_FULL0 + sb), (j >> 1) & 1, abort_flag))) { alive = false; break; }
-            // direct acquire of the producers' validity bits (the phase is complete already)
-            if (!__all_sync(0xffffffffu, mbar_wait(bar(KV_FULL0 + sb), (j >> 1) & 1, abort_flag))) { alive = false; break; }
-            tc_fence_after();
-            const uint32_t v0 = s_mask[sb * 2], v1 = s_mask[sb * 2 + 1];
-            float s[64];
-            tmem_ld32(lane_base + sb * BN, *reinterpret_cast<float (*)[32]>(&s[0]));
-            tmem_ld32(lane_base + sb * BN + 32, *reinterpret_cast<float (*)[32]>(&s[32]));
-            tmem_wait_ld();
-            tc_fence_before();
-            mbar_arrive(bar(S_FREE0 + sb));
-            float m_raw = -INFINITY;
-            if ((v0 & v1) != 0xffffffffu) {
+        int n = 0;
+        for (int64_t item = blockIdx.x; item < n_items && alive; item += gridDim.x, ++n) {
+            const Where q = where(item);
+            const bool more = item + gridDim.x < n_items;
+            const Where qn = where(more ? item + gridDim.x : item);
+            const int32_t *irow = irow_of(q), *irow_n = irow_of(qn);
+            const char *src0 = reinterpret_cast<const char *>(src_t + q.b * p.ks_b + q.gkv * p.ks_h) + c * 16;
+            if (!is_v && gtid == 0) {   // Q of this item, once the last Q K^T of the previous item has read the buffer
+                if (mbar_wait(bar(Q_EMPTY), (n & 1) ^ 1, abort_flag)) {
+                    mbar_expect_tx(bar(Q_FULL), (uint32_t)(NQ * box_heads * 128));
 #pragma unroll
-                for (int e = 0; e < 64; ++e) {
-                    if (!(((e < 32 ? v0 : v1) >> (e & 31)) & 1u)) s[e] = -INFINITY;
-                    m_raw = fmaxf(m_raw, s[e]);
+                    for (int sl = 0; sl < NQ; ++sl)
+                        tma_load_4d(sbase + C::kOffQ + sl * C::kQSlice, &tmQ, bar(Q_FULL), 64 * sl, q.gkv * p.G + kSubHeads * q.sub, q.i, q.b);
                 }
-            } else {
-#pragma unroll
-                for (int e = 0; e < 64; ++e) m_raw = fmaxf(m_raw, s[e]);
             }
-            const float m_blk = m_raw * p.scale_log2;
-            const bool need = m_blk > m_used + kRescaleThreshold;
-            const float m_new = need ? m_blk : m_used;
-            const float corr = need ? exp2f(m_used - m_new) : 1.f;
-            if (j > 0) {
-                if (!__all_sync(0xffffffffu, mbar_wait(bar(PV_DONE), (j - 1) & 1, abort_flag))) { alive = false; break; }
-                tc_fence_after();
-                if (__any_sync(0xffffffffu, need)) {
+            for (int t = 0; t < nblk; ++t) {
+                const int g = n * nblk + t;
+                const int st = g % nst;
+                int *keys = keys_base + (g & 1) * BN;   // double buffered: a thread is at most one barrier ahead
+                int j_mine[KPT];
 #pragma unroll
-                    for (int c = 0; c < D / 32; ++c) {
-                        float o[32];
-                        tmem_ld32(lane_base + 2 * BN + c * 32, o);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int e = 0; e < 32; ++e) o[e] *= corr;
-                        tmem_st32(lane_base + 2 * BN + c * 32, o);
+                for (int u = 0; u < KPT; ++u) {
+                    const int sl = gtid + u * GT;
+                    j_mine[u] = slot_fix(p, j_next[u], q.pos, q.kvl, t * BN + sl);
+                    if (sl < BN) {
+                        if (t + 1 < nblk) j_next[u] = slot_raw(p, irow, q.pos, (t + 1) * BN + sl);
+                        else if (more) j_next[u] = slot_raw(p, irow_n, qn.pos, sl);
                     }
-                    tmem_wait_st();
                 }
-            }
-            l *= corr;
-            m_used = m_new;
-            const float neg_m = m_used == -INFINITY ? 0.f : -m_used;
-            uint32_t pk[32];
-            float l0 = 0.f, l1 = 0.f;
+                const bool ok = __all_sync(0xffffffffu, mbar_wait(bar(bar_empty + st), ((g / nst) & 1) ^ 1, abort_flag));
 #pragma unroll
-            for (int e = 0; e < 64; e += 2) {
-                const float p0 = exp2f(fmaf(s[e], p.scale_log2, neg_m));
-                const float p1 = exp2f(fmaf(s[e + 1], p.scale_log2, neg_m));
-                l0 += p0; l1 += p1;
-                pk[e >> 1] = pack_bf16(p0, p1);
-            }
-            l += l0 + l1;
-            char *prow_ptr = smem + C::kOffP + row * 128;
-#pragma unroll
-            for (int c = 0; c < 8; ++c)
-                *reinterpret_cast<uint4 *>(prow_ptr + ((c ^ (row & 7)) << 4)) = make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
-            fence_proxy_async();
-            tc_fence_before();
-            mbar_arrive(bar(P_FULL));
-        }
-        // ------------------------------------------------ epilogue
-        bool have_o = alive && nblk > 0;
-        if (have_o) have_o = mbar_wait(bar(PV_DONE), (nblk - 1) & 1, abort_flag);
-        have_o = __all_sync(0xffffffffu, have_o);
-        tc_fence_after();
-        const bool any = l > 0.f && m_used != -INFINITY;
-        const float inv = any ? 1.f / l : 0.f;
-        __nv_bfloat16 *orow = O + b * p.os_b + (int64_t)i * p.os_t + h * p.os_h;
-#pragma unroll
-        for (int c = 0; c < D / 32; ++c) {
-            float o[32];
-            if (have_o) {
-                tmem_ld32(lane_base + 2 * BN + c * 32, o);
-                tmem_wait_ld();
-            } else {
-#pragma unroll
-                for (int e = 0; e < 32; ++e) o[e] = 0.f;
-            }
-            if (real) {
-#pragma unroll
-                for (int q4 = 0; q4 < 4; ++q4) {
-                    uint4 v;
-                    v.x = pack_bf16(o[8 * q4 + 0] * inv, o[8 * q4 + 1] * inv);
-                    v.y = pack_bf16(o[8 * q4 + 2] * inv, o[8 * q4 + 3] * inv);
-                    v.z = pack_bf16(o[8 * q4 + 4] * inv, o[8 * q4 + 5] * inv);
-                    v.w = pack_bf16(o[8 * q4 + 6] * inv, o[8 * q4 + 7] * inv);
-                    *reinterpret_cast<uint4 *>(orow + c * 32 + q4 * 8) = v;
+                for (int u = 0; u < KPT; ++u)
+                    if (gtid + u * GT < BN) keys[gtid + u * GT] = j_mine[u];
+                if (!group_all(1 + is_v, GT, ok)) { alive = false; break; }   // also publishes the key indices
+                const uint32_t dst0 = ring0 + st * kKVStage;
+#pragma unroll 4
+                for (int r = r0; r < BN; r += RPI) {
+                    const int j = keys[r];
+                    cp_async16(dst0 + r * 128 + (((c & 7) ^ (r & 7)) << 4), src0 + (j >= 0 ? (int64_t)j * row_bytes : 0), j >= 0 ? 16 : 0);
                 }
+                cp_async_arrive(bar(bar_full + st));
             }
         }
-        if (real && LSE) LSE[((int64_t)b * p.Hq + h) * p.Lq + i] = (have_o && any) ? (m_used + log2f(l)) * kLn2 : -INFINITY;
+        cp_async_wait_all();   // nothing of this thread stays in flight, also on the abort path
+        if (!is_v && gtid == 0 && *abort_flag)
+            for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait(bar(Q_FULL), (n - 1) & 1); ++it) {}
     }
     // ------------------------------------------------ teardown
     __syncwarp();
     tc_fence_before();
     __syncthreads();
-    if (warp == 4) {
+    if (warp == 2) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(C::kTmem) : "memory");
     }
@@ -349,20 +474,28 @@ template <int D>
 cudaError_t launch_sp(const Params &p, const void *Q, const void *K, const void *V, const int32_t *idx, const float *sink,
                       void *O, float *LSE, cudaStream_t st)
 {
+    using C = SpCfg<D>;
     CUtensorMap tmQ;
-    if (!make_tile_map(&tmQ, Q, p.B, p.Lq, p.Hq, p.qs_b, p.qs_t, p.qs_h, 1, p.G, D)) return cudaErrorNotSupported;
+    const int box_heads = p.G < kSubHeads ? p.G : kSubHeads;
+    if (!make_tile_map(&tmQ, Q, p.B, p.Lq, p.Hq, p.qs_b, p.qs_t, p.qs_h, 1, box_heads, D)) return cudaErrorNotSupported;
     static bool attr_set[64] = {};
+    static int n_sm[64] = {};
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
-    if (!(dev >= 0 && dev < 64 && attr_set[dev])) {
-        if ((e = cudaFuncSetAttribute(k_sparse_tc5<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SpCfg<D>::kSmemBytes)) != cudaSuccess) return e;
-        if (dev >= 0 && dev < 64) attr_set[dev] = true;
+    if (dev < 0 || dev >= 64) return cudaErrorNotSupported;
+    if (!attr_set[dev]) {
+        if ((e = cudaFuncSetAttribute(k_sparse_tc5<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::kSmemBytes)) != cudaSuccess) return e;
+        if ((e = cudaDeviceGetAttribute(&n_sm[dev], cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+        attr_set[dev] = true;
     }
-    const int64_t items = (int64_t)p.B * p.Hkv * p.Lq;
+    const int n_sub = (p.G + kSubHeads - 1) / kSubHeads;
+    const int64_t items = (int64_t)p.B * p.Hkv * n_sub * p.Lq;
     if (items <= 0) return cudaSuccess;
-    k_sparse_tc5<D><<<(unsigned)items, kThreads, SpCfg<D>::kSmemBytes, st>>>(
-        tmQ, p, (const __nv_bfloat16 *)K, (const __nv_bfloat16 *)V, idx, sink, (__nv_bfloat16 *)O, LSE);
+    const int64_t resident = (int64_t)n_sm[dev] * C::kMinBlocks;
+    const unsigned grid = (unsigned)(items < resident ? items : resident);
+    k_sparse_tc5<D><<<grid, C::kThreads, C::kSmemBytes, st>>>(
+        tmQ, p, (const __nv_bfloat16 *)K, (const __nv_bfloat16 *)V, idx, sink, (__nv_bfloat16 *)O, LSE, items, n_sub);
     count_launch();
     return cudaGetLastError();
 }
@@ -376,7 +509,7 @@ bool sparse_tc5_supported(const Params &p, hs2_dtype dt)
     if (p.ks_t * 2 > 0x7fffffffLL) return false;
     return dt == HS2_BF16 && (p.D == 128 || p.D == 256) && p.G > 8 && p.G <= 128 && m8(p.qs_b) && m8(p.qs_t) && m8(p.qs_h) &&
            m8(p.ks_b) && m8(p.ks_t) && m8(p.ks_h) && m8(p.os_b) && m8(p.os_t) && m8(p.os_h) &&
-           (int64_t)p.B * p.Hkv * p.Lq <= 0x7fffffffLL && p.k + p.w > 0 && tma_available();
+           (int64_t)p.B * p.Hkv * p.Lq * 2 <= 0x7fffffffLL && p.k + p.w > 0 && tma_available();
 }
 
 // Returns cudaErrorNotSupported when the tensor map cannot be built (the caller then takes the generic kernel).
