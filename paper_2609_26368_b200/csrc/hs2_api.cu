@@ -199,7 +199,8 @@ size_t hs2_workspace_bytes(const hs2_problem *hp, hs2_op op)
         case HS2_OP_SPARSE_ATTN_DECODE:
             if (resolve(hp, true, &p) != HS2_OK) return 0;
             if (p.Lq != 1) return 0;
-            return sparse_mma_supported(p, hp->dtype) ? sparse_mma_decode_ws_bytes(p) : 0;
+            if (sparse_mma_supported(p, hp->dtype)) return sparse_mma_decode_ws_bytes(p);
+            return sparse_tc5_supported_shape(p, hp->dtype) ? sparse_tc5_ws_bytes(p) : 0;
     }
     return 0;
 }
@@ -330,7 +331,7 @@ hs2_status hs2_sparse_attn_prefill(const hs2_problem *hp, const void *Q, const v
     } else {
         // large head groups (the paper's 64 heads per KV head): the gather tile is a dense contraction
         if (!g_disable_tc5.load(std::memory_order_relaxed) && sparse_tc5_supported(p, hp->dtype) && aligned16(Q, K, V, O))
-            e = launch_sparse_tc5(p, Q, K, V, idx, sink, O, LSE, st);
+            e = launch_sparse_tc5(p, Q, K, V, idx, sink, O, LSE, nullptr, 0, st);
         if (e == cudaErrorNotSupported) {
             (void)cudaGetLastError();
             e = launch_sparse_generic(p, hp->dtype, Q, K, V, idx, sink, O, LSE, st);
@@ -351,8 +352,20 @@ hs2_status hs2_sparse_attn_decode(const hs2_problem *hp, const void *Q, const vo
     if (mma && !ws_ok(ws, ws_bytes, sparse_mma_decode_ws_bytes(p))) return HS2_ERR_WORKSPACE_TOO_SMALL;
     if ((s = check_device()) != HS2_OK) return s;
     cudaStream_t st = (cudaStream_t)cuda_stream;
-    cudaError_t e = mma ? launch_sparse_mma_decode(p, Q, K, V, idx, sink, O, LSE, ws, ws_bytes, st)
-                        : launch_sparse_generic(p, hp->dtype, Q, K, V, idx, sink, O, LSE, st);
+    cudaError_t e = cudaErrorNotSupported;
+    if (mma) {
+        e = launch_sparse_mma_decode(p, Q, K, V, idx, sink, O, LSE, ws, ws_bytes, st);
+    } else {
+        // large head groups: the tcgen05 gather kernel, its keys split over CTAs when the scratch allows
+        if (!g_disable_tc5.load(std::memory_order_relaxed) && sparse_tc5_supported(p, hp->dtype) && aligned16(Q, K, V, O)) {
+            const bool ws_usable = ws != nullptr && (reinterpret_cast<uintptr_t>(ws) & 15u) == 0;
+            e = launch_sparse_tc5(p, Q, K, V, idx, sink, O, LSE, ws_usable ? ws : nullptr, ws_usable ? ws_bytes : 0, st);
+        }
+        if (e == cudaErrorNotSupported) {
+            (void)cudaGetLastError();
+            e = launch_sparse_generic(p, hp->dtype, Q, K, V, idx, sink, O, LSE, st);
+        }
+    }
     return e == cudaSuccess ? HS2_OK : cuda_fail(e);
 }
 

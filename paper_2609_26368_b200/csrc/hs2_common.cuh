@@ -122,9 +122,11 @@ cudaError_t launch_scores_filter_tc5(const Params &p, const void *Q, const void 
                                      int64_t n_rows, const uint32_t *tau_key, float *cand_a, int32_t *cand_j, int *count,
                                      int cap, cudaStream_t st);
 // tcgen05 sparse attention for large head groups (bf16, head_dim 128 or 256, 8 < group <= 128)
+bool sparse_tc5_supported_shape(const Params &p, hs2_dtype dt);   // the shape alone (no driver query)
 bool sparse_tc5_supported(const Params &p, hs2_dtype dt);
+size_t sparse_tc5_ws_bytes(const Params &p);   // scratch that lets few queries (decode) split their keys over CTAs
 cudaError_t launch_sparse_tc5(const Params &p, const void *Q, const void *K, const void *V, const int32_t *idx,
-                              const float *sink, void *O, float *LSE, cudaStream_t st);
+                              const float *sink, void *O, float *LSE, void *ws, size_t ws_bytes, cudaStream_t st);
 cudaError_t read_sparse_tc5_error(unsigned *out);
 cudaError_t read_tc5_error(unsigned *out);
 cudaError_t read_sparse_error(unsigned *out);

@@ -129,11 +129,15 @@ __device__ __forceinline__ int slot_fix(const Params &p, int j, int pos, int kvl
 
 // Persistent: every CTA walks items blockIdx.x, blockIdx.x + gridDim.x, ...  All rings and phases are indexed by
 // the running tile number g = (items done by this CTA) * nblk + t, which every role computes for itself.
+// With n_splits > 1 (few queries, e.g. decode) an item is one of n_splits runs of nblk tiles of a query's slot
+// array (slots past the array are void), and it leaves an unnormalised partial (running maximum, sum, fp32
+// accumulator) in part_ml / part_o for the combine kernel below.
 template <int D>
 __global__ void __launch_bounds__(SpCfg<D>::kThreads, SpCfg<D>::kMinBlocks)
 k_sparse_tc5(const __grid_constant__ CUtensorMap tmQ, const Params p, const __nv_bfloat16 *__restrict__ K,
              const __nv_bfloat16 *__restrict__ V, const int32_t *__restrict__ idx, const float *__restrict__ sink,
-             __nv_bfloat16 *__restrict__ O, float *__restrict__ LSE, int64_t n_items, int n_sub)
+             __nv_bfloat16 *__restrict__ O, float *__restrict__ LSE, int64_t n_items, int n_sub, int n_splits, int nblk,
+             float *__restrict__ part_ml, float *__restrict__ part_o)
 {
     using C = SpCfg<D>;
     constexpr int NQ = C::NQ, CH = C::CH, KST = C::KST;
@@ -156,11 +160,12 @@ k_sparse_tc5(const __grid_constant__ CUtensorMap tmQ, const Params p, const __nv
     auto bar = [&](int i) { return bars + 8u * i; };
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int nblk = (p.k + p.w + BN - 1) / BN;      // tiles of the virtual slot array [idx row | window]
     // item -> (sequence, KV head, sub-group of heads, query, position)
-    struct Where { int b, gkv, sub, i, kvl, pos; };
+    struct Where { int b, gkv, sub, i, kvl, pos, slot0; };
     auto where = [&](int64_t item) {
         Where wq;
+        wq.slot0 = (int)(item % n_splits) * nblk * BN;   // first slot of this run of tiles
+        item /= n_splits;
         wq.i = (int)(item % p.Lq);
         const int r = (int)(item / p.Lq);
         wq.sub = r % n_sub;
@@ -214,18 +219,19 @@ k_sparse_tc5(const __grid_constant__ CUtensorMap tmQ, const Params p, const __nv
             const int h = q.gkv * p.G + kSubHeads * q.sub + (real ? row : 0);
             const int32_t *irow = irow_of(q);
             float m_used = -INFINITY, l = 0.f;
-            if (sink && real) {   // Section 3.3 variant with a learnable sink logit: it only joins the denominator
+            if (sink && real && q.slot0 == 0) {   // Section 3.3 variant with a learnable sink logit: it only joins the denominator
                 m_used = sink[h] * kLog2e;
                 l = half == 0 ? 1.f : 0.f;
             }
             const int g0 = n * nblk;
             // validity of this half's 32 slots is recomputed here (cheap, and no cross-warp visibility to argue
             // about), one tile ahead so that the idx loads are off the critical path
-            int jn = slot_raw(p, irow, q.pos, 32 * half + lane);
+            const int my_slot = q.slot0 + 32 * half + lane;
+            int jn = slot_raw(p, irow, q.pos, my_slot);
             for (int t = 0; t < nblk; ++t) {
                 const int g = g0 + t, sb = g & 1;
-                const uint32_t valid = __ballot_sync(0xffffffffu, slot_fix(p, jn, q.pos, q.kvl, t * BN + 32 * half + lane) >= 0);
-                if (t + 1 < nblk) jn = slot_raw(p, irow, q.pos, (t + 1) * BN + 32 * half + lane);
+                const uint32_t valid = __ballot_sync(0xffffffffu, slot_fix(p, jn, q.pos, q.kvl, my_slot + t * BN) >= 0);
+                if (t + 1 < nblk) jn = slot_raw(p, irow, q.pos, my_slot + (t + 1) * BN);
                 if (!dead && !__all_sync(0xffffffffu, mbar_wait(bar(S_FULL0 + sb), (g >> 1) & 1, abort_flag))) dead = true;
                 float s[32];
                 float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
@@ -310,6 +316,7 @@ k_sparse_tc5(const __grid_constant__ CUtensorMap tmQ, const Params p, const __nv
             const bool any = l > 0.f && m_used != -INFINITY;
             const float inv = any ? 1.f / l : 0.f;
             __nv_bfloat16 *orow = O + q.b * p.os_b + (int64_t)q.i * p.os_t + h * p.os_h + half * (D / 2);
+            float *prow = n_splits > 1 ? part_o + (item * kSubHeads + row) * D + half * (D / 2) : nullptr;
 #pragma unroll
             for (int cc = 0; cc < D / 64; ++cc) {
                 float o[32];
@@ -319,7 +326,12 @@ k_sparse_tc5(const __grid_constant__ CUtensorMap tmQ, const Params p, const __nv
                     tc_fence_before();
                     mbar_arrive(bar(O_FREE));
                 }
-                if (real) {
+                if (n_splits > 1) {   // unnormalised partial, every row (rows past the group are never combined)
+#pragma unroll
+                    for (int q4 = 0; q4 < 8; ++q4)
+                        *reinterpret_cast<float4 *>(prow + cc * 32 + q4 * 4) =
+                            any ? make_float4(o[4 * q4], o[4 * q4 + 1], o[4 * q4 + 2], o[4 * q4 + 3]) : make_float4(0.f, 0.f, 0.f, 0.f);
+                } else if (real) {
 #pragma unroll
                     for (int q4 = 0; q4 < 4; ++q4) {
                         uint4 v;
@@ -331,7 +343,11 @@ k_sparse_tc5(const __grid_constant__ CUtensorMap tmQ, const Params p, const __nv
                     }
                 }
             }
-            if (real && half == 0 && LSE) LSE[((int64_t)q.b * p.Hq + h) * p.Lq + q.i] = any ? (m_used + log2f(l)) * kLn2 : -INFINITY;
+            if (n_splits > 1) {
+                if (half == 0) *reinterpret_cast<float2 *>(part_ml + (item * kSubHeads + row) * 2) = make_float2(any ? m_used : -INFINITY, any ? l : 0.f);
+            } else if (real && half == 0 && LSE) {
+                LSE[((int64_t)q.b * p.Hq + h) * p.Lq + q.i] = any ? (m_used + log2f(l)) * kLn2 : -INFINITY;
+            }
         }
     } else if (warp == 2) {
         // ------------------------------------------------ MMA issuer
@@ -410,7 +426,7 @@ k_sparse_tc5(const __grid_constant__ CUtensorMap tmQ, const Params p, const __nv
             const Where q0 = where(blockIdx.x);
 #pragma unroll
             for (int u = 0; u < KPT; ++u)
-                if (gtid + u * GT < BN) j_next[u] = slot_raw(p, irow_of(q0), q0.pos, gtid + u * GT);
+                if (gtid + u * GT < BN) j_next[u] = slot_raw(p, irow_of(q0), q0.pos, q0.slot0 + gtid + u * GT);
         }
         bool alive = true;
         int n = 0;
@@ -436,10 +452,10 @@ k_sparse_tc5(const __grid_constant__ CUtensorMap tmQ, const Params p, const __nv
 #pragma unroll
                 for (int u = 0; u < KPT; ++u) {
                     const int sl = gtid + u * GT;
-                    j_mine[u] = slot_fix(p, j_next[u], q.pos, q.kvl, t * BN + sl);
+                    j_mine[u] = slot_fix(p, j_next[u], q.pos, q.kvl, q.slot0 + t * BN + sl);
                     if (sl < BN) {
-                        if (t + 1 < nblk) j_next[u] = slot_raw(p, irow, q.pos, (t + 1) * BN + sl);
-                        else if (more) j_next[u] = slot_raw(p, irow_n, qn.pos, sl);
+                        if (t + 1 < nblk) j_next[u] = slot_raw(p, irow, q.pos, q.slot0 + (t + 1) * BN + sl);
+                        else if (more) j_next[u] = slot_raw(p, irow_n, qn.pos, qn.slot0 + sl);
                     }
                 }
                 const bool ok = __all_sync(0xffffffffu, mbar_wait(bar(bar_empty + st), ((g / nst) & 1) ^ 1, abort_flag));
@@ -470,9 +486,86 @@ k_sparse_tc5(const __grid_constant__ CUtensorMap tmQ, const Params p, const __nv
     }
 }
 
+constexpr int kMaxSplits = 16;
+
+// Combines the n_splits partials of every (query, head): one warp per pair.  Lane sp fetches the (maximum, sum) of
+// split sp, so all of them are in flight at once; the accumulator rows are then read with independent loads.
+template <int D>
+__global__ void __launch_bounds__(256)
+k_sparse_tc5_combine(const Params p, const float *__restrict__ part_ml, const float *__restrict__ part_o,
+                     __nv_bfloat16 *__restrict__ O, float *__restrict__ LSE, int n_sub, int n_splits, int64_t n_pairs)
+{
+    const int lane = threadIdx.x & 31;
+    const int64_t pair = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);   // (b, i, head)
+    if (pair >= n_pairs) return;
+    const int h = (int)(pair % p.Hq);
+    const int64_t bi = pair / p.Hq;
+    const int i = (int)(bi % p.Lq), b = (int)(bi / p.Lq);
+    const int gkv = h / p.G, hh = h % p.G;
+    const int sub = hh / kSubHeads, row = hh % kSubHeads;
+    const int64_t item0 = ((((int64_t)b * p.Hkv + gkv) * n_sub + sub) * p.Lq + i) * n_splits;
+    float2 ml = make_float2(-INFINITY, 0.f);
+    if (lane < n_splits) ml = *reinterpret_cast<const float2 *>(part_ml + ((item0 + lane) * kSubHeads + row) * 2);
+    const float m = warp_max(ml.x);
+    const float f_mine = ml.x == -INFINITY ? 0.f : exp2f(ml.x - m);
+    const float l = warp_sum(f_mine * ml.y);
+    constexpr int NV = D / 128;   // float4 per lane
+    float4 acc[NV];
+#pragma unroll
+    for (int u = 0; u < NV; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+    const float *po = part_o + (item0 * kSubHeads + row) * D + lane * 4;
+#pragma unroll 4
+    for (int sp = 0; sp < n_splits; ++sp) {
+        const float f = __shfl_sync(0xffffffffu, f_mine, sp);
+#pragma unroll
+        for (int u = 0; u < NV; ++u) {
+            const float4 v = *reinterpret_cast<const float4 *>(po + (int64_t)sp * kSubHeads * D + u * 128);
+            acc[u].x += f * v.x; acc[u].y += f * v.y; acc[u].z += f * v.z; acc[u].w += f * v.w;
+        }
+    }
+    const float inv = l > 0.f ? 1.f / l : 0.f;
+    __nv_bfloat16 *orow = O + b * p.os_b + (int64_t)i * p.os_t + h * p.os_h + lane * 4;
+#pragma unroll
+    for (int u = 0; u < NV; ++u) {
+        uint2 v;
+        v.x = pack_bf16(acc[u].x * inv, acc[u].y * inv);
+        v.y = pack_bf16(acc[u].z * inv, acc[u].w * inv);
+        *reinterpret_cast<uint2 *>(orow + u * 128) = v;
+    }
+    if (lane == 0 && LSE) LSE[((int64_t)b * p.Hq + h) * p.Lq + i] = l > 0.f ? (m + log2f(l)) * kLn2 : -INFINITY;
+}
+
+constexpr int kPlanSms = 148;   // the workspace is sized for this many SMs; a launch on another part adapts to what it got
+
+struct SplitPlan { int n_sub, n_splits, nblk; int64_t queries; };
+
+// Splits over the keys only when the queries alone cannot fill the SMs (decode, very short prefill chunks).
+SplitPlan plan_splits(const Params &p, int n_sm, bool allow_split)
+{
+    SplitPlan pl;
+    pl.n_sub = (p.G + kSubHeads - 1) / kSubHeads;
+    pl.queries = (int64_t)p.B * p.Hkv * pl.n_sub * p.Lq;
+    const int tiles = (p.k + p.w + BN - 1) / BN;
+    int ns = 1;
+    if (allow_split && pl.queries > 0 && pl.queries < n_sm) {
+        ns = (int)(n_sm / pl.queries);
+        if (ns > kMaxSplits) ns = kMaxSplits;
+        if (ns > tiles) ns = tiles;
+        if (ns < 1) ns = 1;
+    }
+    pl.nblk = (tiles + ns - 1) / ns;
+    pl.n_splits = (tiles + pl.nblk - 1) / pl.nblk;   // no run of tiles is entirely past the slot array
+    return pl;
+}
+size_t split_ws_bytes(const Params &p, const SplitPlan &pl)
+{
+    if (pl.n_splits <= 1) return 0;
+    return (size_t)pl.queries * pl.n_splits * kSubHeads * (p.D + 2) * sizeof(float);
+}
+
 template <int D>
 cudaError_t launch_sp(const Params &p, const void *Q, const void *K, const void *V, const int32_t *idx, const float *sink,
-                      void *O, float *LSE, cudaStream_t st)
+                      void *O, float *LSE, void *ws, size_t ws_bytes, bool allow_split, cudaStream_t st)
 {
     using C = SpCfg<D>;
     CUtensorMap tmQ;
@@ -489,13 +582,24 @@ cudaError_t launch_sp(const Params &p, const void *Q, const void *K, const void 
         if ((e = cudaDeviceGetAttribute(&n_sm[dev], cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
         attr_set[dev] = true;
     }
-    const int n_sub = (p.G + kSubHeads - 1) / kSubHeads;
-    const int64_t items = (int64_t)p.B * p.Hkv * n_sub * p.Lq;
+    SplitPlan pl = plan_splits(p, n_sm[dev] * C::kMinBlocks, allow_split && ws != nullptr);
+    if (split_ws_bytes(p, pl) > ws_bytes) pl = plan_splits(p, 1, false);   // scratch too small for this part: no split
+    const int64_t items = pl.queries * pl.n_splits;
     if (items <= 0) return cudaSuccess;
+    float *part_ml = reinterpret_cast<float *>(ws);
+    float *part_o = pl.n_splits > 1 ? part_ml + items * kSubHeads * 2 : nullptr;
     const int64_t resident = (int64_t)n_sm[dev] * C::kMinBlocks;
     const unsigned grid = (unsigned)(items < resident ? items : resident);
     k_sparse_tc5<D><<<grid, C::kThreads, C::kSmemBytes, st>>>(
-        tmQ, p, (const __nv_bfloat16 *)K, (const __nv_bfloat16 *)V, idx, sink, (__nv_bfloat16 *)O, LSE, items, n_sub);
+        tmQ, p, (const __nv_bfloat16 *)K, (const __nv_bfloat16 *)V, idx, sink, (__nv_bfloat16 *)O, LSE, items, pl.n_sub,
+        pl.n_splits, pl.nblk, part_ml, part_o);
+    count_launch();
+    if ((e = cudaGetLastError()) != cudaSuccess || pl.n_splits <= 1) return e;
+    const int64_t n_pairs = (int64_t)p.B * p.Lq * p.Hq;
+    // (a programmatic dependent launch of this kernel was measured: 23 -> 31 us per decode step at batch 16, so it is
+    // launched the plain way)
+    k_sparse_tc5_combine<D><<<(unsigned)((n_pairs + 7) / 8), 256, 0, st>>>(p, part_ml, part_o, (__nv_bfloat16 *)O, LSE, pl.n_sub,
+                                                                       pl.n_splits, n_pairs);
     count_launch();
     return cudaGetLastError();
 }
@@ -503,21 +607,29 @@ cudaError_t launch_sp(const Params &p, const void *Q, const void *K, const void 
 }  // namespace
 
 // bf16, head_dim 128 or 256, more than 8 and at most 128 query heads per KV head
-bool sparse_tc5_supported(const Params &p, hs2_dtype dt)
+bool sparse_tc5_supported_shape(const Params &p, hs2_dtype dt)
 {
     auto m8 = [](int64_t x) { return x % 8 == 0 && x > 0; };
     if (p.ks_t * 2 > 0x7fffffffLL) return false;
     return dt == HS2_BF16 && (p.D == 128 || p.D == 256) && p.G > 8 && p.G <= 128 && m8(p.qs_b) && m8(p.qs_t) && m8(p.qs_h) &&
            m8(p.ks_b) && m8(p.ks_t) && m8(p.ks_h) && m8(p.os_b) && m8(p.os_t) && m8(p.os_h) &&
-           (int64_t)p.B * p.Hkv * p.Lq * 2 <= 0x7fffffffLL && p.k + p.w > 0 && tma_available();
+           (int64_t)p.B * p.Hkv * p.Lq * 2 * kMaxSplits <= 0x7fffffffLL && p.k + p.w > 0;
+}
+bool sparse_tc5_supported(const Params &p, hs2_dtype dt) { return sparse_tc5_supported_shape(p, dt) && tma_available(); }
+
+// Scratch for splitting the keys of a query over several CTAs (sized for a 148-SM part; 0 when no split pays).
+size_t sparse_tc5_ws_bytes(const Params &p)
+{
+    return split_ws_bytes(p, plan_splits(p, kPlanSms * (p.D <= 128 ? 2 : 1), true));
 }
 
 // Returns cudaErrorNotSupported when the tensor map cannot be built (the caller then takes the generic kernel).
+// ws may be null: the keys of a query are then never split.
 cudaError_t launch_sparse_tc5(const Params &p, const void *Q, const void *K, const void *V, const int32_t *idx,
-                              const float *sink, void *O, float *LSE, cudaStream_t st)
+                              const float *sink, void *O, float *LSE, void *ws, size_t ws_bytes, cudaStream_t st)
 {
-    if (p.D == 128) return launch_sp<128>(p, Q, K, V, idx, sink, O, LSE, st);
-    if (p.D == 256) return launch_sp<256>(p, Q, K, V, idx, sink, O, LSE, st);
+    if (p.D == 128) return launch_sp<128>(p, Q, K, V, idx, sink, O, LSE, ws, ws_bytes, true, st);
+    if (p.D == 256) return launch_sp<256>(p, Q, K, V, idx, sink, O, LSE, ws, ws_bytes, true, st);
     return cudaErrorNotSupported;
 }
 

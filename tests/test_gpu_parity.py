@@ -279,6 +279,15 @@ def test_tcgen05_sparse_kernel_large_head_groups():
             fin = torch.isfinite(lse_g)
             assert torch.equal(torch.isfinite(lse), fin)
             assert (lse[fin] - lse_g[fin]).abs().max().item() <= 2e-3
+            # decode of the last position: few queries, so the keys of a query are split over CTAs and combined
+            q1 = run.qs[0][:, -1:].contiguous()
+            prob1 = hs2.Problem.from_tensors(q1, run.k, wl.k_sel, wl.window)
+            assert hs2.hs2_workspace_bytes(prob1, hs2.binding.HS2_OP_SPARSE_ATTN_DECODE) > 0 or wl.k_sel + wl.window <= 64
+            od, ld = hs2.hs2_sparse_attn_decode(prob1, q1, run.k, run.v, run.idx[:, :, -1:].contiguous(), sink=sk,
+                                                want_lse=True)
+            torch.cuda.synchronize()
+            assert (od.float() - out[:, -1:].float()).abs().max().item() <= 2e-2
+            assert (ld - lse[:, :, -1:]).abs().max().item() <= 2e-3
     assert hs2.hs2_device_error_flags() == 0
 
 
