@@ -354,6 +354,87 @@ def bench_decode_64k(device, peaks, reps=5, burst=40, ctx=65536):
             "l2": "%.1f GB cache, 4 rotating query/index sets (1.1 GB of gathered rows) > L2" % (2 * k.numel() * 2 / 1e9)}
 
 
+def bench_native(device, peaks, reps=5):
+    """The paper's own attention shape (Table 1: 64 query heads on one KV head, head_dim 256, 1024 selected + 128
+    window tokens): full layer with selection and sparse prefill at 8K, sparse decode at batch 64 and a 64K cache.
+    Reported beside the benchmark configurations; every kernel on this path is a tcgen05 kernel."""
+    import paper_2609_26368_b200 as hs2
+    from paper_2609_26368_b200 import binding
+    from gen.workloads import NATIVE
+
+    def med(fn, n=reps, warm=2):
+        for _ in range(warm):
+            fn()
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(n):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            fn()
+            b.record()
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b))
+        return statistics.median(ts)
+
+    out = {}
+    wl = NATIVE["native8k"]
+    inp = make_inputs(wl, device)
+    q, k, v = inp.q_full, inp.k, inp.v
+    prob = hs2.Problem.from_tensors(q, k, wl.k_sel, wl.window)
+    ws = torch.empty(max(256, hs2.hs2_workspace_bytes(prob, binding.HS2_OP_FULL_ATTN_SELECT)), dtype=torch.uint8, device=device)
+    O, LSE, idx, _ = hs2.hs2_full_attn_select(prob, q, k, v, ws=ws)
+    t_full = med(lambda: hs2.hs2_full_attn_select(prob, q, k, v, out=O, lse=LSE, idx=idx, ws=ws))
+    t_att = med(lambda: hs2.hs2_full_attn_select(prob, q, k, v, out=O, lse=LSE, want_idx=False, ws=ws))
+    osp = torch.empty_like(q)
+    t_sp = med(lambda: hs2.hs2_sparse_attn_prefill(prob, inp.q_sparse[0], k, v, idx, out=osp))
+    gb = gathered_kv_bytes(wl)
+    fl = full_attn_flops(wl)
+    out["prefill"] = {
+        "workload": "native8k: B=1, L=8192, 64q/1kv heads, D=256, bf16, k=1024, w=128",
+        "full_attn_select_ms": round(t_full, 3), "attention_only_ms": round(t_att, 3),
+        "attention_tflops": round(fl / (t_att * 1e-3) / 1e12, 1),
+        "attention_frac_of_bf16_peak": round(fl / (t_att * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"], 4),
+        "sparse_prefill_ms": round(t_sp, 3), "gathered_kv_bytes": gb,
+        "sparse_prefill_gbs": round(gb / (t_sp * 1e-3) / 1e9, 1),
+        "sparse_prefill_frac_of_hbm_peak": round(gb / (t_sp * 1e-3) / 1e9 / peaks["hbm_gbs"], 4),
+        "l2": "the 8 MB cache is L2 resident; Q, idx and O (100 MB) stream"}
+    del inp, q, k, v, O, LSE, idx, osp, ws
+    torch.cuda.empty_cache()
+
+    wl = NATIVE["native_decode"]
+    inp = make_inputs(wl, device)
+    k, v = inp.k, inp.v
+    prob = hs2.Problem.from_tensors(inp.q_full, k, wl.k_sel, wl.window)
+    ws_full = torch.empty(max(256, hs2.hs2_workspace_bytes(prob, binding.HS2_OP_FULL_ATTN_SELECT)), dtype=torch.uint8, device=device)
+    ws_dec = torch.empty(max(256, hs2.hs2_workspace_bytes(prob, binding.HS2_OP_SPARSE_ATTN_DECODE)), dtype=torch.uint8, device=device)
+    nset, burst = 4, 40
+    qfs = [inp.q_full] + [torch.randn_like(inp.q_full) for _ in range(nset - 1)]
+    idxs, t_full = [], []
+    for s in range(nset):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        _, _, idx, _ = hs2.hs2_full_attn_select(prob, qfs[s], k, v, ws=ws_full)
+        b.record()
+        torch.cuda.synchronize()
+        t_full.append(a.elapsed_time(b))
+        idxs.append(idx)
+    qss = [torch.randn_like(inp.q_full) for _ in range(nset)]
+    o1 = torch.empty_like(inp.q_full)
+
+    def run(n):
+        for it in range(n):
+            hs2.hs2_sparse_attn_decode(prob, qss[it % nset], k, v, idxs[it % nset], out=o1, ws=ws_dec)
+    us = med(lambda: run(burst), warm=1) / burst * 1e3
+    gb = gathered_kv_bytes(wl)
+    out["decode"] = {
+        "workload": "native_decode: B=64, ctx 65536, 64q/1kv heads, D=256, bf16, k=1024, w=128",
+        "sparse_decode_us_per_step": round(us, 2), "gathered_kv_bytes": gb,
+        "achieved_gbs": round(gb / (us * 1e-6) / 1e9, 1), "frac_of_hbm_peak": round(gb / (us * 1e-6) / 1e9 / peaks["hbm_gbs"], 4),
+        "full_attn_select_decode_ms": round(min(t_full[1:]), 3), "launches_back_to_back": burst,
+        "l2": "4.3 GB cache, 4 rotating query/index sets > L2"}
+    return out
+
+
 # ------------------------------------------------------------------ CPU oracle legs
 
 def oracle_sample_step(wl, inp_host, rows):
@@ -424,7 +505,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2", choices=sorted(CONFIGS))
     ap.add_argument("--cpu-rows", type=int, default=4096, help="query rows of the CPU-oracle sample (about 15 s of CPU work on cfg2)")
-    ap.add_argument("--skip", default="", help="comma list of: block, decode64k, e2e, cpu")
+    ap.add_argument("--skip", default="", help="comma list of: block, decode64k, native, e2e, cpu")
     ap.add_argument("--decode-ctx", type=int, default=65536, help="context length of the decode section (profiling: 8192)")
     args = ap.parse_args()
     wl = CONFIGS[args.workload]
@@ -507,6 +588,9 @@ def main():
         del block
         torch.cuda.empty_cache()
         line["decode_64k"] = bench_decode_64k(device, peaks, ctx=args.decode_ctx)
+    if "native" not in skip and world == 1:
+        torch.cuda.empty_cache()
+        line["paper_native_shape"] = bench_native(device, peaks)
     if "cpu" not in skip and world == 1:
         cb, _, _ = cpu_baseline(wl, args.cpu_rows)
         line["cpu_baseline"] = cb

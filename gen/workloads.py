@@ -169,6 +169,17 @@ CONFIGS: Dict[str, Workload] = {
 }
 
 
+# The attention shape of the paper's own models (Table 1): multi-query attention, 64 query heads sharing one KV head,
+# head_dim 256, 1024 selected + 128 window tokens.  Not benchmark configurations: measured beside them.
+NATIVE: Dict[str, Workload] = {
+    "native8k": _wl(11, name="native8k", batch=1, q_len=8192, kv_len=8192, n_q_heads=64, n_kv_heads=1, head_dim=256,
+                    dtype="bf16", k_sel=1024, window=128, n_sparse_layers=3, structure="needles_stratified"),
+    "native_decode": _wl(12, name="native_decode", batch=64, q_len=1, kv_len=65536, n_q_heads=64, n_kv_heads=1,
+                         head_dim=256, dtype="bf16", k_sel=1024, window=128, n_sparse_layers=3,
+                         structure="decode_needles"),
+}
+
+
 def scaled(name: str, **overrides) -> Workload:
     """A benchmark configuration with some fields replaced (small parity cases)."""
     return replace(CONFIGS[name], **overrides)

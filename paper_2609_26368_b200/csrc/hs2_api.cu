@@ -185,10 +185,12 @@ size_t hs2_workspace_bytes(const hs2_problem *hp, hs2_op op)
                     const size_t fneed = filter_ws_bytes(fp, select_rows(p));
                     if (fneed > need) need = fneed;
                 }
-                if (p.Lq == 1 && sparse_mma_supported(p, hp->dtype)) {   // the decode-shaped layer may split over the keys
+                if (p.Lq == 1) {   // the decode-shaped layer may split over the keys
                     Params pd = p;
                     pd.k = 0; pd.w = p.Lk;
-                    const size_t dec = sparse_mma_decode_ws_bytes(pd);
+                    const size_t dec = sparse_mma_supported(p, hp->dtype)         ? sparse_mma_decode_ws_bytes(pd)
+                                       : sparse_tc5_supported_shape(pd, hp->dtype) ? sparse_tc5_ws_bytes(pd)
+                                                                                   : 0;
                     if (dec > need) need = dec;
                 }
                 return need;
@@ -232,8 +234,14 @@ hs2_status hs2_full_attn_select(const hs2_problem *hp, const void *Q, const void
         e = launch_sparse_mma_decode(pd, Q, K, V, nullptr, nullptr, O, LSE, ws, ws_bytes, st);
     else {
         e = cudaErrorNotSupported;
+        // the same idea for large head groups: the tcgen05 gather kernel, keys split over CTAs through the scratch
+        if (p.Lq == 1 && !g_disable_tc5.load(std::memory_order_relaxed) && sparse_tc5_supported(pd, dt) && aligned16(Q, K, V, O)) {
+            const bool ws_usable = ws != nullptr && (reinterpret_cast<uintptr_t>(ws) & 15u) == 0;
+            e = launch_sparse_tc5(pd, Q, K, V, nullptr, nullptr, O, LSE, ws_usable ? ws : nullptr, ws_usable ? ws_bytes : 0, st);
+        }
 #ifndef HS2_NO_TC5
-        if (!g_disable_tc5.load(std::memory_order_relaxed) && full_attn_tc5_supported(p, dt) && aligned16(Q, K, V, O))
+        if (e == cudaErrorNotSupported && !g_disable_tc5.load(std::memory_order_relaxed) && full_attn_tc5_supported(p, dt) &&
+            aligned16(Q, K, V, O))
             e = launch_full_attn_tc5(p, Q, K, V, O, LSE, st);
 #endif
         if (e == cudaErrorNotSupported)
