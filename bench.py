@@ -522,8 +522,13 @@ def main():
     peaks = measured_peaks()
     warmup = max(args.warmup, 3)
 
-    if "block" in skip:      # decode-section only (used for profiling captures)
-        print(json.dumps({"decode_64k": bench_decode_64k(device, peaks, ctx=args.decode_ctx)}))
+    if "block" in skip:      # side sections only (used for profiling captures)
+        side = {}
+        if "decode64k" not in skip:
+            side["decode_64k"] = bench_decode_64k(device, peaks, ctx=args.decode_ctx)
+        if "native" not in skip:
+            side["paper_native_shape"] = bench_native(device, peaks)
+        print(json.dumps(side))
         return
     block = Block(wl, device, rank)
     tokens_per_step = wl.batch * wl.q_len
