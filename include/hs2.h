@@ -139,6 +139,20 @@ hs2_status hs2_sparse_attn_decode(const hs2_problem *p, const void *Q, const voi
                                   void *ws, size_t ws_bytes, void *cuda_stream);
 
 /*
+ * The two SA calls with the sigmoid output gate of the sparse layers fused into the store (Section 4.1:
+ * "all sparse and SWA layers use sigmoid output gates"): O = sigmoid(gate) * attention output, elementwise.
+ *   gate  in  the gate logits (the caller's projection of the layer input; not computed here): shape, dtype
+ *             and strides of O (p->o_stride).  Must not be NULL (use the ungated call instead).
+ * LSE is not affected by the gate.  Everything else as for the ungated calls.
+ */
+hs2_status hs2_sparse_attn_prefill_gated(const hs2_problem *p, const void *Q, const void *K, const void *V,
+                                         const int32_t *idx, const float *sink, const void *gate, void *O,
+                                         float *LSE, void *ws, size_t ws_bytes, void *cuda_stream);
+hs2_status hs2_sparse_attn_decode_gated(const hs2_problem *p, const void *Q, const void *K, const void *V,
+                                        const int32_t *idx, const float *sink, const void *gate, void *O,
+                                        float *LSE, void *ws, size_t ws_bytes, void *cuda_stream);
+
+/*
  * hs2_sparse_attn_decode for callers that cannot hand over a scratch buffer.  (The paper has no
  * counterpart to this call; it is a packaging variant of the decode operator above.)
  *

@@ -153,10 +153,12 @@ def select(scores, pos, kvlen, window: int, k_sel: int) -> np.ndarray:
 
 
 def sparse_attn(q, k, v, idx, window, rows=None, sink=None, scale=None, q_start=None, kv_lens=None,
-                want_member=False):
+                want_member=False, gate=None):
     """Sparse attention over (valid idx) U window for the listed rows.
 
     ``idx`` is ``[n, Hkv, k]`` aligned with ``rows``.  Returns ``(O [n,Hq,D], LSE [n,Hq], member)``.
+    ``gate`` (``[B, Lq, Hq, D]`` logits, optional) is the sigmoid output gate of the sparse layers
+    (Section 4.1): the attention output of a row is multiplied elementwise by 1 / (1 + exp(-gate)).
     """
     idx = np.ascontiguousarray(idx, dtype=np.int32)
     k_sel = idx.shape[-1]
@@ -172,4 +174,10 @@ def sparse_attn(q, k, v, idx, window, rows=None, sink=None, scale=None, q_start=
     sk = None if sink is None else np.ascontiguousarray(sink, dtype=np.float64)
     _get().hs2o_sparse_attn_rows(C.byref(prob.c), _ptr(prob.q), _ptr(prob.k), _ptr(vv), _ptr(idx), _ptr(sk),
                                  C.c_int(n), _ptr(rb), _ptr(ri), _ptr(O), _ptr(LSE), _ptr(member))
+    if gate is not None:
+        gg, code = _as_input(gate)                  # the exact input values, widened to fp64
+        if code == 1:                               # bf16 bit patterns: the upper half of an fp32
+            gg = (gg.astype(np.uint32) << 16).view(np.float32)
+        gg = gg.astype(np.float64).reshape(B, Lq, Hq, D)
+        O = O * (1.0 / (1.0 + np.exp(-gg[rb, ri])))
     return O, LSE, member

@@ -23,7 +23,8 @@ HS2_F32, HS2_BF16 = 0, 1
 HS2_OP_FULL_ATTN_SELECT, HS2_OP_TOPK_SELECT, HS2_OP_SPARSE_ATTN_PREFILL, HS2_OP_SPARSE_ATTN_DECODE = range(4)
 
 EXPORTS = ["hs2_workspace_bytes", "hs2_full_attn_select", "hs2_topk_select", "hs2_sparse_attn_prefill",
-           "hs2_sparse_attn_decode", "hs2_sparse_attn_decode_static", "hs2_status_string", "hs2_last_cuda_error",
+           "hs2_sparse_attn_decode", "hs2_sparse_attn_prefill_gated", "hs2_sparse_attn_decode_gated",
+           "hs2_sparse_attn_decode_static", "hs2_status_string", "hs2_last_cuda_error",
            "hs2_launch_count", "hs2_device_error_flags", "hs2_set_filter_min_keys", "hs2_set_tcgen05_enabled"]
 
 
@@ -68,8 +69,10 @@ def load_library():
         lib.hs2_sparse_attn_prefill.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         lib.hs2_sparse_attn_decode.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         lib.hs2_sparse_attn_decode_static.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp]
+        lib.hs2_sparse_attn_prefill_gated.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        lib.hs2_sparse_attn_decode_gated.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         for f in ("hs2_full_attn_select", "hs2_topk_select", "hs2_sparse_attn_prefill", "hs2_sparse_attn_decode",
-                  "hs2_sparse_attn_decode_static"):
+                  "hs2_sparse_attn_prefill_gated", "hs2_sparse_attn_decode_gated", "hs2_sparse_attn_decode_static"):
             getattr(lib, f).restype = C.c_int
         _lib = lib
     return _lib
@@ -213,7 +216,7 @@ def hs2_topk_select(prob: Problem, scores, *, idx=None, stream=None):
     return idx
 
 
-def _sparse(fn_name, op, prob, q, k, v, idx, sink, out, lse, want_lse, ws, stream):
+def _sparse(fn_name, op, prob, q, k, v, idx, sink, out, lse, want_lse, ws, stream, gate=None):
     _check_inputs(prob, q, k, v)
     dev = q.device
     if idx is not None:
@@ -226,24 +229,31 @@ def _sparse(fn_name, op, prob, q, k, v, idx, sink, out, lse, want_lse, ws, strea
         lse = torch.empty(prob.batch, prob.n_q_heads, prob.q_len, dtype=torch.float32, device=dev)
     ws = _workspace(prob, op, dev, ws)
     c = prob.c_struct(q, k, out)
-    st = getattr(load_library(), fn_name)(C.byref(c), _dp(q), _dp(k), _dp(v), _dp(idx), _dp(sink), _dp(out), _dp(lse),
-                                          _dp(ws), ws.numel(), _stream(stream))
+    if gate is not None:   # the gated entry point: gate logits laid out like the output
+        assert gate.is_cuda and gate.dtype == out.dtype and gate.shape == out.shape and gate.stride() == out.stride()
+        fn_name += "_gated"
+        st = getattr(load_library(), fn_name)(C.byref(c), _dp(q), _dp(k), _dp(v), _dp(idx), _dp(sink), _dp(gate), _dp(out),
+                                              _dp(lse), _dp(ws), ws.numel(), _stream(stream))
+    else:
+        st = getattr(load_library(), fn_name)(C.byref(c), _dp(q), _dp(k), _dp(v), _dp(idx), _dp(sink), _dp(out), _dp(lse),
+                                              _dp(ws), ws.numel(), _stream(stream))
     _check(st, fn_name)
     return out, lse
 
 
-def hs2_sparse_attn_prefill(prob: Problem, q, k, v, idx, *, sink=None, out=None, lse=None, want_lse=False,
+def hs2_sparse_attn_prefill(prob: Problem, q, k, v, idx, *, sink=None, gate=None, out=None, lse=None, want_lse=False,
                             ws=None, stream=None):
-    """SA layer, prefill: attention over (idx) U (forced window); returns ``(O, LSE | None)``."""
+    """SA layer, prefill: attention over (idx) U (forced window); returns ``(O, LSE | None)``.
+    With ``gate`` (logits shaped like the output) the output is multiplied by sigmoid(gate) in the kernel's store."""
     return _sparse("hs2_sparse_attn_prefill", HS2_OP_SPARSE_ATTN_PREFILL, prob, q, k, v, idx, sink, out, lse,
-                   want_lse, ws, stream)
+                   want_lse, ws, stream, gate)
 
 
-def hs2_sparse_attn_decode(prob: Problem, q, k, v, idx, *, sink=None, out=None, lse=None, want_lse=False,
+def hs2_sparse_attn_decode(prob: Problem, q, k, v, idx, *, sink=None, gate=None, out=None, lse=None, want_lse=False,
                            ws=None, stream=None):
     """SA layer, decode (q_len == 1, split over the attended set); returns ``(O, LSE | None)``."""
     return _sparse("hs2_sparse_attn_decode", HS2_OP_SPARSE_ATTN_DECODE, prob, q, k, v, idx, sink, out, lse,
-                   want_lse, ws, stream)
+                   want_lse, ws, stream, gate)
 
 
 def hs2_sparse_attn_decode_static(prob: Problem, q, k, v, idx, *, sink=None, out, lse=None, stream=None):

@@ -155,6 +155,9 @@ cudaError_t launch_scores(const Params &p, hs2_dtype dt, bool mma, bool aligned,
     return e;
 }
 
+// the gate is read with the 16-byte accesses of the output it scales
+bool gate_aligned(const void *gate) { return (reinterpret_cast<uintptr_t>(gate) & 15u) == 0; }
+
 hs2_status sparse_common(const hs2_problem *hp, const void *Q, const void *K, const void *V, const int32_t *idx,
                          void *O, Params *p)
 {
@@ -323,23 +326,69 @@ hs2_status hs2_topk_select(const hs2_problem *hp, const float *scores, int32_t *
     return e == cudaSuccess ? HS2_OK : cuda_fail(e);
 }
 
-hs2_status hs2_sparse_attn_prefill(const hs2_problem *hp, const void *Q, const void *K, const void *V,
-                                   const int32_t *idx, const float *sink, void *O, float *LSE, void *ws,
-                                   size_t ws_bytes, void *cuda_stream)
+static hs2_status sparse_prefill_impl(const hs2_problem *hp, const void *Q, const void *K, const void *V, const int32_t *idx,
+                                      const float *sink, const void *gate, void *O, float *LSE, void *ws, size_t ws_bytes,
+                                      void *cuda_stream)
 {
     (void)ws; (void)ws_bytes;
     Params p;
     hs2_status s = sparse_common(hp, Q, K, V, idx, O, &p);
     if (s != HS2_OK) return s;
+    p.gate = gate;
     if ((s = check_device()) != HS2_OK) return s;
     cudaStream_t st = (cudaStream_t)cuda_stream;
     cudaError_t e = cudaErrorNotSupported;
-    if (sparse_mma_supported(p, hp->dtype) && aligned16(Q, K, V, O)) {
+    if (sparse_mma_supported(p, hp->dtype) && aligned16(Q, K, V, O) && gate_aligned(gate)) {
         e = launch_sparse_mma_prefill(p, Q, K, V, idx, sink, O, LSE, st);
     } else {
         // large head groups (the paper's 64 heads per KV head): the gather tile is a dense contraction
-        if (!g_disable_tc5.load(std::memory_order_relaxed) && sparse_tc5_supported(p, hp->dtype) && aligned16(Q, K, V, O))
+        if (!g_disable_tc5.load(std::memory_order_relaxed) && sparse_tc5_supported(p, hp->dtype) && aligned16(Q, K, V, O) && gate_aligned(gate))
             e = launch_sparse_tc5(p, Q, K, V, idx, sink, O, LSE, nullptr, 0, st);
+        if (e == cudaErrorNotSupported) {
+            (void)cudaGetLastError();
+            e = launch_sparse_generic(p, hp->dtype, Q, K, V, idx, sink, O, LSE, st);
+        }
+    }
+    return e == cudaSuccess ? HS2_OK : cuda_fail(e);
+}
+
+hs2_status hs2_sparse_attn_prefill(const hs2_problem *hp, const void *Q, const void *K, const void *V,
+                                   const int32_t *idx, const float *sink, void *O, float *LSE, void *ws,
+                                   size_t ws_bytes, void *cuda_stream)
+{
+    return sparse_prefill_impl(hp, Q, K, V, idx, sink, nullptr, O, LSE, ws, ws_bytes, cuda_stream);
+}
+
+hs2_status hs2_sparse_attn_prefill_gated(const hs2_problem *hp, const void *Q, const void *K, const void *V,
+                                         const int32_t *idx, const float *sink, const void *gate, void *O, float *LSE,
+                                         void *ws, size_t ws_bytes, void *cuda_stream)
+{
+    if (!gate) return HS2_ERR_INVALID_ARG;
+    return sparse_prefill_impl(hp, Q, K, V, idx, sink, gate, O, LSE, ws, ws_bytes, cuda_stream);
+}
+
+static hs2_status sparse_decode_impl(const hs2_problem *hp, const void *Q, const void *K, const void *V, const int32_t *idx,
+                                     const float *sink, const void *gate, void *O, float *LSE, void *ws, size_t ws_bytes,
+                                     void *cuda_stream)
+{
+    Params p;
+    hs2_status s = sparse_common(hp, Q, K, V, idx, O, &p);
+    if (s != HS2_OK) return s;
+    p.gate = gate;
+    if (p.Lq != 1) return HS2_ERR_INVALID_ARG;
+    const bool mma = sparse_mma_supported(p, hp->dtype) && aligned16(Q, K, V, O) && gate_aligned(gate);
+    if (mma && !ws_ok(ws, ws_bytes, sparse_mma_decode_ws_bytes(p))) return HS2_ERR_WORKSPACE_TOO_SMALL;
+    if ((s = check_device()) != HS2_OK) return s;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    cudaError_t e = cudaErrorNotSupported;
+    if (mma) {
+        e = launch_sparse_mma_decode(p, Q, K, V, idx, sink, O, LSE, ws, ws_bytes, st);
+    } else {
+        // large head groups: the tcgen05 gather kernel, its keys split over CTAs when the scratch allows
+        if (!g_disable_tc5.load(std::memory_order_relaxed) && sparse_tc5_supported(p, hp->dtype) && aligned16(Q, K, V, O) && gate_aligned(gate)) {
+            const bool ws_usable = ws != nullptr && (reinterpret_cast<uintptr_t>(ws) & 15u) == 0;
+            e = launch_sparse_tc5(p, Q, K, V, idx, sink, O, LSE, ws_usable ? ws : nullptr, ws_usable ? ws_bytes : 0, st);
+        }
         if (e == cudaErrorNotSupported) {
             (void)cudaGetLastError();
             e = launch_sparse_generic(p, hp->dtype, Q, K, V, idx, sink, O, LSE, st);
@@ -352,29 +401,15 @@ hs2_status hs2_sparse_attn_decode(const hs2_problem *hp, const void *Q, const vo
                                   const int32_t *idx, const float *sink, void *O, float *LSE, void *ws,
                                   size_t ws_bytes, void *cuda_stream)
 {
-    Params p;
-    hs2_status s = sparse_common(hp, Q, K, V, idx, O, &p);
-    if (s != HS2_OK) return s;
-    if (p.Lq != 1) return HS2_ERR_INVALID_ARG;
-    const bool mma = sparse_mma_supported(p, hp->dtype) && aligned16(Q, K, V, O);
-    if (mma && !ws_ok(ws, ws_bytes, sparse_mma_decode_ws_bytes(p))) return HS2_ERR_WORKSPACE_TOO_SMALL;
-    if ((s = check_device()) != HS2_OK) return s;
-    cudaStream_t st = (cudaStream_t)cuda_stream;
-    cudaError_t e = cudaErrorNotSupported;
-    if (mma) {
-        e = launch_sparse_mma_decode(p, Q, K, V, idx, sink, O, LSE, ws, ws_bytes, st);
-    } else {
-        // large head groups: the tcgen05 gather kernel, its keys split over CTAs when the scratch allows
-        if (!g_disable_tc5.load(std::memory_order_relaxed) && sparse_tc5_supported(p, hp->dtype) && aligned16(Q, K, V, O)) {
-            const bool ws_usable = ws != nullptr && (reinterpret_cast<uintptr_t>(ws) & 15u) == 0;
-            e = launch_sparse_tc5(p, Q, K, V, idx, sink, O, LSE, ws_usable ? ws : nullptr, ws_usable ? ws_bytes : 0, st);
-        }
-        if (e == cudaErrorNotSupported) {
-            (void)cudaGetLastError();
-            e = launch_sparse_generic(p, hp->dtype, Q, K, V, idx, sink, O, LSE, st);
-        }
-    }
-    return e == cudaSuccess ? HS2_OK : cuda_fail(e);
+    return sparse_decode_impl(hp, Q, K, V, idx, sink, nullptr, O, LSE, ws, ws_bytes, cuda_stream);
+}
+
+hs2_status hs2_sparse_attn_decode_gated(const hs2_problem *hp, const void *Q, const void *K, const void *V,
+                                        const int32_t *idx, const float *sink, const void *gate, void *O, float *LSE,
+                                        void *ws, size_t ws_bytes, void *cuda_stream)
+{
+    if (!gate) return HS2_ERR_INVALID_ARG;
+    return sparse_decode_impl(hp, Q, K, V, idx, sink, gate, O, LSE, ws, ws_bytes, cuda_stream);
 }
 
 hs2_status hs2_sparse_attn_decode_static(const hs2_problem *hp, const void *Q, const void *K, const void *V,

@@ -21,7 +21,12 @@ struct Params {
     int64_t qs_b, qs_t, qs_h;   // element strides
     int64_t ks_b, ks_t, ks_h;
     int64_t os_b, os_t, os_h;
+    const void *gate;   // optional output-gate logits of the sparse layers: shape, dtype and strides of O; null = no gate
 };
+
+// sigmoid output gate of the sparse layers (Section 4.1): the attention output is multiplied elementwise by
+// sigmoid(gate logit)
+__device__ __forceinline__ float gate_of(float logit) { return 1.f / (1.f + __expf(-logit)); }
 
 // per-sequence geometry, clamped so that no later index arithmetic can leave the tensors
 __device__ __forceinline__ int kvlen_of(const Params &p, int b)

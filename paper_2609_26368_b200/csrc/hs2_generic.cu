@@ -92,13 +92,13 @@ __device__ __forceinline__ void fold_chunk(RowState &st, float t2, unsigned vali
 }
 
 template <typename T>
-__device__ __forceinline__ void write_row(const RowState &st, T *o, float *lse_out, int D, int lane)
+__device__ __forceinline__ void write_row(const RowState &st, T *o, float *lse_out, int D, int lane, const T *gate = nullptr)
 {
     const float inv = st.l > 0.f ? 1.f / st.l : 0.f;
 #pragma unroll
     for (int r = 0; r < kMaxDPerLane; ++r) {
         const int d = lane + 32 * r;
-        if (d < D) from_f32(o[d], st.acc[r] * inv);
+        if (d < D) from_f32(o[d], st.acc[r] * inv * (gate ? gate_of(to_f32(gate[d])) : 1.f));
     }
     if (lse_out && lane == 0) *lse_out = st.l > 0.f ? (st.m + log2f(st.l)) * kLn2 : -INFINITY;
 }
@@ -237,7 +237,8 @@ k_sparse_generic(const Params p, const T *__restrict__ Q, const T *__restrict__ 
             return vb + (int64_t)jt * p.ks_t;
         });
     }
-    write_row<T>(st, O + b * p.os_b + i * p.os_t + h * p.os_h, LSE ? LSE + row : nullptr, p.D, lane);
+    const int64_t o_off = b * p.os_b + i * p.os_t + h * p.os_h;
+    write_row<T>(st, O + o_off, LSE ? LSE + row : nullptr, p.D, lane, p.gate ? static_cast<const T *>(p.gate) + o_off : nullptr);
 }
 
 template <typename Kern>

@@ -424,8 +424,19 @@ __device__ __forceinline__ void store_output(const Params &p, const Acc &acc, __
     for (int v = lane; v < 8 * 16; v += 32) {
         const int head = v >> 4, c = v & 15;
         if (head < p.G) {
-            const uint4 val = *reinterpret_cast<const uint4 *>(so + head * kPitch + c * 8);
-            *reinterpret_cast<uint4 *>(O + b * p.os_b + i * p.os_t + (gkv * p.G + head) * p.os_h + c * 8) = val;
+            uint4 val = *reinterpret_cast<const uint4 *>(so + head * kPitch + c * 8);
+            const int64_t off = b * p.os_b + i * p.os_t + (gkv * p.G + head) * p.os_h + c * 8;
+            if (p.gate) {   // output gate: applied to the staged bf16 values, 8 at a time
+                const uint4 gv = *reinterpret_cast<const uint4 *>(static_cast<const __nv_bfloat16 *>(p.gate) + off);
+                __nv_bfloat162 *ov = reinterpret_cast<__nv_bfloat162 *>(&val);
+                const __nv_bfloat162 *gg = reinterpret_cast<const __nv_bfloat162 *>(&gv);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float2 o2 = __bfloat1622float2(ov[e]), g2 = __bfloat1622float2(gg[e]);
+                    ov[e] = __floats2bfloat162_rn(o2.x * gate_of(g2.x), o2.y * gate_of(g2.y));
+                }
+            }
+            *reinterpret_cast<uint4 *>(O + off) = val;
         }
     }
     if (LSE && g == 0) {

@@ -315,7 +315,9 @@ k_sparse_tc5(const __grid_constant__ CUtensorMap tmQ, const Params p, const __nv
             tc_fence_after();
             const bool any = l > 0.f && m_used != -INFINITY;
             const float inv = any ? 1.f / l : 0.f;
-            __nv_bfloat16 *orow = O + q.b * p.os_b + (int64_t)q.i * p.os_t + h * p.os_h + half * (D / 2);
+            const int64_t o_off = q.b * p.os_b + (int64_t)q.i * p.os_t + h * p.os_h + half * (D / 2);
+            __nv_bfloat16 *orow = O + o_off;
+            const __nv_bfloat16 *grow = p.gate ? static_cast<const __nv_bfloat16 *>(p.gate) + o_off : nullptr;
             float *prow = n_splits > 1 ? part_o + (item * kSubHeads + row) * D + half * (D / 2) : nullptr;
 #pragma unroll
             for (int cc = 0; cc < D / 64; ++cc) {
@@ -332,6 +334,19 @@ k_sparse_tc5(const __grid_constant__ CUtensorMap tmQ, const Params p, const __nv
                         *reinterpret_cast<float4 *>(prow + cc * 32 + q4 * 4) =
                             any ? make_float4(o[4 * q4], o[4 * q4 + 1], o[4 * q4 + 2], o[4 * q4 + 3]) : make_float4(0.f, 0.f, 0.f, 0.f);
                 } else if (real) {
+                    if (grow) {   // sigmoid output gate, before the single rounding to bf16
+#pragma unroll
+                        for (int q4 = 0; q4 < 4; ++q4) {
+                            const uint4 gv = *reinterpret_cast<const uint4 *>(grow + cc * 32 + q4 * 8);
+                            const __nv_bfloat162 *gg = reinterpret_cast<const __nv_bfloat162 *>(&gv);
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const float2 g2 = __bfloat1622float2(gg[e]);
+                                o[8 * q4 + 2 * e] *= gate_of(g2.x);
+                                o[8 * q4 + 2 * e + 1] *= gate_of(g2.y);
+                            }
+                        }
+                    }
 #pragma unroll
                     for (int q4 = 0; q4 < 4; ++q4) {
                         uint4 v;
@@ -524,9 +539,16 @@ k_sparse_tc5_combine(const Params p, const float *__restrict__ part_ml, const fl
         }
     }
     const float inv = l > 0.f ? 1.f / l : 0.f;
-    __nv_bfloat16 *orow = O + b * p.os_b + (int64_t)i * p.os_t + h * p.os_h + lane * 4;
+    const int64_t o_off = b * p.os_b + (int64_t)i * p.os_t + h * p.os_h + lane * 4;
+    __nv_bfloat16 *orow = O + o_off;
 #pragma unroll
     for (int u = 0; u < NV; ++u) {
+        if (p.gate) {
+            const uint2 gv = *reinterpret_cast<const uint2 *>(static_cast<const __nv_bfloat16 *>(p.gate) + o_off + u * 128);
+            const float2 g0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&gv.x));
+            const float2 g1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&gv.y));
+            acc[u].x *= gate_of(g0.x); acc[u].y *= gate_of(g0.y); acc[u].z *= gate_of(g1.x); acc[u].w *= gate_of(g1.y);
+        }
         uint2 v;
         v.x = pack_bf16(acc[u].x * inv, acc[u].y * inv);
         v.y = pack_bf16(acc[u].z * inv, acc[u].w * inv);

@@ -130,20 +130,21 @@ class BlockRun:
         got = gather_rows(self.idx, rows, "bgik").cpu().numpy()
         assert np.array_equal(got, want)
 
-    def run_sparse(self, layer=0, decode=False, sink=None, want_lse=True):
+    def run_sparse(self, layer=0, decode=False, sink=None, want_lse=True, gate=None):
         fn = hs2.hs2_sparse_attn_decode if decode else hs2.hs2_sparse_attn_prefill
-        out, lse = fn(self.prob, self.qs[layer], self.k, self.v, self.idx, sink=sink, want_lse=want_lse)
+        out, lse = fn(self.prob, self.qs[layer], self.k, self.v, self.idx, sink=sink, want_lse=want_lse, gate=gate)
         torch.cuda.synchronize()
         return out, lse
 
-    def check_sparse(self, out, lse, layer=0, rows=None, sink=None):
+    def check_sparse(self, out, lse, layer=0, rows=None, sink=None, gate=None):
         """Oracle sparse attention on the GPU's own indices (a legal tie swap must not pollute this check)."""
         wl = self.wl
         rows = rows_all(wl.batch, wl.q_len) if rows is None else rows
         idx_rows = gather_rows(self.idx, rows, "bgik").cpu().numpy()
         Oo, LSEo, _ = oracle.sparse_attn(to_host(self.qs[layer]), to_host(self.k), to_host(self.v), idx_rows,
                                          wl.window, rows=rows,
-                                         sink=None if sink is None else sink.cpu().numpy().astype(np.float64))
+                                         sink=None if sink is None else sink.cpu().numpy().astype(np.float64),
+                                         gate=None if gate is None else to_host(gate))
         dt = wl.torch_dtype
         assert_output_close(gather_rows(out, rows, "bihd"), Oo, dt, "sparse attention O")
         if lse is not None:

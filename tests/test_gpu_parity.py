@@ -291,6 +291,43 @@ def test_tcgen05_sparse_kernel_large_head_groups():
     assert hs2.hs2_device_error_flags() == 0
 
 
+def test_sigmoid_output_gate_in_every_sparse_kernel_family():
+    """The gated entry points (Section 4.1: sigmoid output gates in the sparse layers) against the oracle: SIMT fp32,
+    mma.sync (group of 8), tcgen05 (group of 64, head_dim 256), prefill and decode (split and unsplit)."""
+    cases = [
+        ("cfg1", dict(q_len=80, kv_len=200, k_sel=20, window=6)),
+        ("cfg2", dict(q_len=120, kv_len=500, k_sel=64, window=16, n_needles=4, batch=2)),
+        ("cfg2", dict(q_len=70, kv_len=400, k_sel=100, window=28, n_q_heads=64, n_kv_heads=1, head_dim=256, n_needles=4)),
+    ]
+    for name, over in cases:
+        wl = scaled(name, **over)
+        run = BlockRun(make_inputs(wl)).run_full()
+        g = torch.Generator(device="cuda").manual_seed(11)
+        gate = (torch.randn(run.qs[0].shape, device="cuda", generator=g) * 2.5).to(run.qs[0].dtype)
+        sink = torch.linspace(-1.0, 1.0, wl.n_q_heads, device="cuda")
+        out0, lse0 = run.run_sparse(0, sink=sink)
+        out, lse = run.run_sparse(0, sink=sink, gate=gate)
+        run.check_sparse(out, lse, 0, sink=sink, gate=gate)
+        assert torch.equal(lse, lse0)                     # the gate leaves LSE alone
+        # decode of the last position, gated
+        q1 = run.qs[0][:, -1:].contiguous()
+        g1 = gate[:, -1:].contiguous()
+        prob1 = hs2.Problem.from_tensors(q1, run.k, wl.k_sel, wl.window)
+        od, _ = hs2.hs2_sparse_attn_decode(prob1, q1, run.k, run.v, run.idx[:, :, -1:].contiguous(), sink=sink, gate=g1)
+        torch.cuda.synchronize()
+        tol = 1e-4 if wl.dtype == "f32" else 2e-2
+        assert (od.float() - out[:, -1:].float()).abs().max().item() <= tol
+    with pytest.raises(hs2.HS2Error):                     # the gated call needs a gate
+        lib = hs2.load_library()
+        c = run.prob.c_struct(run.qs[0], run.k, out)
+        import ctypes as C
+        st = lib.hs2_sparse_attn_prefill_gated(C.byref(c), run.qs[0].data_ptr(), run.k.data_ptr(), run.v.data_ptr(),
+                                               run.idx.data_ptr(), None, None, out.data_ptr(), None, None, 0, None)
+        if st != 0:
+            raise hs2.HS2Error(st, "hs2_sparse_attn_prefill_gated")
+    assert hs2.hs2_device_error_flags() == 0
+
+
 def test_ragged_lengths_offsets_strides_and_sink():
     wl = scaled("cfg2", batch=3, q_len=70, kv_len=400, k_sel=40, window=12, n_needles=4)
     inp = make_inputs(wl)

@@ -346,3 +346,28 @@ def test_fp32_and_bf16_inputs_are_read_exactly():
     a = oracle.full_attn_select(inp.q_full, inp.k, inp.v, wl.k_sel, wl.window, rows=rows)
     b = oracle.full_attn_select(inp.q_full.float(), inp.k.float(), inp.v.float(), wl.k_sel, wl.window, rows=rows)
     assert np.array_equal(a[0], b[0]) and np.array_equal(a[2], b[2])
+
+
+def test_output_gate_special_values_and_library_sigmoid():
+    """Sigmoid output gate of the sparse layers (Section 4.1): logit 0 halves the output exactly, a large logit
+    leaves it unchanged, a very negative one removes it, LSE is untouched, and a random gate agrees with torch's
+    own fp64 sigmoid applied to the ungated result."""
+    wl = scaled("cfg1", q_len=24, kv_len=24, k_sel=6, window=3)
+    inp = make_inputs(wl)
+    _, _, idx, _ = oracle.full_attn_select(inp.q_full, inp.k, inp.v, wl.k_sel, wl.window)
+    q = inp.q_sparse[0]
+    O0, L0, _ = oracle.sparse_attn(q, inp.k, inp.v, idx, wl.window)
+    for val, fac in ((0.0, 0.5), (40.0, 1.0), (-700.0, 0.0)):
+        g = torch.full(q.shape, val, dtype=torch.float32)
+        O1, L1, _ = oracle.sparse_attn(q, inp.k, inp.v, idx, wl.window, gate=g)
+        assert np.allclose(O1, O0 * fac, rtol=0, atol=1e-15)
+        assert np.array_equal(L1, L0)
+    g = torch.randn(q.shape, generator=torch.Generator().manual_seed(5), dtype=torch.float32) * 3
+    O2, _, _ = oracle.sparse_attn(q, inp.k, inp.v, idx, wl.window, gate=g)
+    B, Lq, Hq, D = q.shape
+    want = O0 * torch.sigmoid(g.double()).reshape(B * Lq, Hq, D).numpy()
+    assert np.abs(O2 - want).max() < 1e-14
+    gb = g.to(torch.bfloat16)                       # bf16 logits are read exactly
+    O3, _, _ = oracle.sparse_attn(q, inp.k, inp.v, idx, wl.window, gate=gb)
+    want = O0 * torch.sigmoid(gb.double()).reshape(B * Lq, Hq, D).numpy()
+    assert np.abs(O3 - want).max() < 1e-14
