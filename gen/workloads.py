@@ -280,3 +280,14 @@ def sample_rows(wl: Workload, n_rows: int = 64) -> List[int]:
         if r not in rows:
             rows.append(r)
     return sorted(rows)
+
+
+def quantize_kv_e4m3(x: torch.Tensor):
+    """Stand-in for the producer of an FP8 KV cache (outside the attention path): one fp32 scale per (token, KV head)
+    = amax / 448 (1 for an all-zero row), codes = x / scale rounded to the nearest e4m3 value by torch's own cast.
+    Returns ``(codes uint8 [B, L, Hkv, D], scales fp32 [B, L, Hkv])``."""
+    xf = x.float()
+    amax = xf.abs().amax(dim=-1)
+    scale = torch.where(amax > 0, amax / 448.0, torch.ones_like(amax)).float()
+    y = (xf / scale[..., None]).clamp(-448.0, 448.0).to(torch.float8_e4m3fn)
+    return y.view(torch.uint8).contiguous(), scale.contiguous()

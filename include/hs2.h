@@ -153,6 +153,25 @@ hs2_status hs2_sparse_attn_decode_gated(const hs2_problem *p, const void *Q, con
                                         float *LSE, void *ws, size_t ws_bytes, void *cuda_stream);
 
 /*
+ * The two SA calls on an FP8 KV cache (the storage format the paper's cost analysis of Section 4 assumes, "FP8
+ * KV-cache storage"; the paper gives no quantisation recipe, this is the usual one):
+ *   K8, V8   in  e4m3 codes (1 byte: sign, 4 exponent bits with bias 7, 3 mantissa bits; no infinities, the two
+ *                NaN codes are a caller error) [batch, kv_len, n_kv_heads, head_dim]; p->kv_stride counts codes
+ *                (= bytes), multiples of 16, or 0 for packed.
+ *   k_scale, v_scale  in  float [batch, kv_len, n_kv_heads], packed: the cache value is code * scale.
+ *   Q, O, LSE, idx, sink as for the bf16 calls; p->dtype describes Q and O and must be HS2_BF16.
+ * Covers head_dim 128 with n_q_heads / n_kv_heads <= 8 and 16-byte aligned tensors; anything else returns
+ * HS2_ERR_UNSUPPORTED.  V scales up to 255 are supported (probability x scale is carried in an f16 operand).
+ * No scratch is needed: decode runs one CTA per (sequence, KV head) whose warps split the attended set.
+ */
+hs2_status hs2_sparse_attn_prefill_fp8kv(const hs2_problem *p, const void *Q, const void *K8, const void *V8,
+                                         const float *k_scale, const float *v_scale, const int32_t *idx,
+                                         const float *sink, void *O, float *LSE, void *cuda_stream);
+hs2_status hs2_sparse_attn_decode_fp8kv(const hs2_problem *p, const void *Q, const void *K8, const void *V8,
+                                        const float *k_scale, const float *v_scale, const int32_t *idx,
+                                        const float *sink, void *O, float *LSE, void *cuda_stream);
+
+/*
  * hs2_sparse_attn_decode for callers that cannot hand over a scratch buffer.  (The paper has no
  * counterpart to this call; it is a packaging variant of the decode operator above.)
  *

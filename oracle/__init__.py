@@ -181,3 +181,25 @@ def sparse_attn(q, k, v, idx, window, rows=None, sink=None, scale=None, q_start=
         gg = gg.astype(np.float64).reshape(B, Lq, Hq, D)
         O = O * (1.0 / (1.0 + np.exp(-gg[rb, ri])))
     return O, LSE, member
+
+
+def decode_e4m3(codes):
+    """Value of every e4m3 code, from the format's definition: 1 sign bit, 4 exponent bits (bias 7), 3 mantissa
+    bits; exponent field 0 is subnormal (mantissa / 8 * 2^-6); there are no infinities, S.1111.111 is NaN."""
+    c = np.asarray(codes, dtype=np.uint8).astype(np.int64)
+    sign = np.where(c & 0x80, -1.0, 1.0)
+    e = (c >> 3) & 0xF
+    m = (c & 0x7).astype(np.float64)
+    val = np.where(e == 0, m / 8.0 * 2.0 ** -6, (1.0 + m / 8.0) * np.exp2((e - 7).astype(np.float64)))
+    val = np.where((e == 15) & ((c & 0x7) == 7), np.nan, val)
+    return sign * val
+
+
+def dequant_e4m3(codes, scales):
+    """FP8 cache contents: code value times the scale of its (token, KV head), as an fp32 array (the cache value is
+    defined as that product rounded to fp32)."""
+    if not isinstance(codes, np.ndarray):
+        codes = codes.detach().cpu().numpy()
+    if not isinstance(scales, np.ndarray):
+        scales = scales.detach().cpu().numpy()
+    return (decode_e4m3(codes) * scales.astype(np.float64)[..., None]).astype(np.float32)

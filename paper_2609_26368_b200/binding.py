@@ -24,6 +24,7 @@ HS2_OP_FULL_ATTN_SELECT, HS2_OP_TOPK_SELECT, HS2_OP_SPARSE_ATTN_PREFILL, HS2_OP_
 
 EXPORTS = ["hs2_workspace_bytes", "hs2_full_attn_select", "hs2_topk_select", "hs2_sparse_attn_prefill",
            "hs2_sparse_attn_decode", "hs2_sparse_attn_prefill_gated", "hs2_sparse_attn_decode_gated",
+           "hs2_sparse_attn_prefill_fp8kv", "hs2_sparse_attn_decode_fp8kv",
            "hs2_sparse_attn_decode_static", "hs2_status_string", "hs2_last_cuda_error",
            "hs2_launch_count", "hs2_device_error_flags", "hs2_set_filter_min_keys", "hs2_set_tcgen05_enabled"]
 
@@ -71,8 +72,11 @@ def load_library():
         lib.hs2_sparse_attn_decode_static.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp]
         lib.hs2_sparse_attn_prefill_gated.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         lib.hs2_sparse_attn_decode_gated.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        lib.hs2_sparse_attn_prefill_fp8kv.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+        lib.hs2_sparse_attn_decode_fp8kv.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         for f in ("hs2_full_attn_select", "hs2_topk_select", "hs2_sparse_attn_prefill", "hs2_sparse_attn_decode",
-                  "hs2_sparse_attn_prefill_gated", "hs2_sparse_attn_decode_gated", "hs2_sparse_attn_decode_static"):
+                  "hs2_sparse_attn_prefill_gated", "hs2_sparse_attn_decode_gated", "hs2_sparse_attn_decode_static",
+                  "hs2_sparse_attn_prefill_fp8kv", "hs2_sparse_attn_decode_fp8kv"):
             getattr(lib, f).restype = C.c_int
         _lib = lib
     return _lib
@@ -254,6 +258,44 @@ def hs2_sparse_attn_decode(prob: Problem, q, k, v, idx, *, sink=None, gate=None,
     """SA layer, decode (q_len == 1, split over the attended set); returns ``(O, LSE | None)``."""
     return _sparse("hs2_sparse_attn_decode", HS2_OP_SPARSE_ATTN_DECODE, prob, q, k, v, idx, sink, out, lse,
                    want_lse, ws, stream, gate)
+
+
+def _sparse_fp8(fn_name, prob, q, k8, v8, k_scale, v_scale, idx, sink, out, lse, want_lse, stream):
+    assert q.is_cuda and q.dtype == torch.bfloat16 and q.stride(-1) == 1
+    for t in (k8, v8):
+        assert t.is_cuda and t.dtype == torch.uint8 and t.stride(-1) == 1
+        assert tuple(t.shape) == (prob.batch, prob.kv_len, prob.n_kv_heads, prob.head_dim)
+    assert k8.stride() == v8.stride()
+    for t in (k_scale, v_scale):
+        assert t.is_cuda and t.dtype == torch.float32 and t.is_contiguous()
+        assert tuple(t.shape) == (prob.batch, prob.kv_len, prob.n_kv_heads)
+    if idx is not None:
+        assert idx.dtype == torch.int32 and idx.is_contiguous() and idx.is_cuda
+        assert tuple(idx.shape) == (prob.batch, prob.n_kv_heads, prob.q_len, prob.k_sel)
+    if sink is not None:
+        assert sink.dtype == torch.float32 and sink.is_cuda and sink.numel() == prob.n_q_heads
+    out = torch.empty_like(q) if out is None else out
+    if lse is None and want_lse:
+        lse = torch.empty(prob.batch, prob.n_q_heads, prob.q_len, dtype=torch.float32, device=q.device)
+    c = prob.c_struct(q, k8, out)
+    st = getattr(load_library(), fn_name)(C.byref(c), _dp(q), _dp(k8), _dp(v8), _dp(k_scale), _dp(v_scale), _dp(idx),
+                                          _dp(sink), _dp(out), _dp(lse), _stream(stream))
+    _check(st, fn_name)
+    return out, lse
+
+
+def hs2_sparse_attn_prefill_fp8kv(prob: Problem, q, k8, v8, k_scale, v_scale, idx, *, sink=None, out=None, lse=None,
+                                  want_lse=False, stream=None):
+    """SA layer, prefill, on an e4m3 cache (uint8 codes + fp32 scale per (token, KV head)); bf16 Q and O."""
+    return _sparse_fp8("hs2_sparse_attn_prefill_fp8kv", prob, q, k8, v8, k_scale, v_scale, idx, sink, out, lse, want_lse,
+                       stream)
+
+
+def hs2_sparse_attn_decode_fp8kv(prob: Problem, q, k8, v8, k_scale, v_scale, idx, *, sink=None, out=None, lse=None,
+                                 want_lse=False, stream=None):
+    """SA layer, decode (q_len == 1), on an e4m3 cache."""
+    return _sparse_fp8("hs2_sparse_attn_decode_fp8kv", prob, q, k8, v8, k_scale, v_scale, idx, sink, out, lse, want_lse,
+                       stream)
 
 
 def hs2_sparse_attn_decode_static(prob: Problem, q, k, v, idx, *, sink=None, out, lse=None, stream=None):

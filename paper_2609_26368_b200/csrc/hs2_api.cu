@@ -412,6 +412,37 @@ hs2_status hs2_sparse_attn_decode_gated(const hs2_problem *hp, const void *Q, co
     return sparse_decode_impl(hp, Q, K, V, idx, sink, gate, O, LSE, ws, ws_bytes, cuda_stream);
 }
 
+static hs2_status sparse_fp8_impl(const hs2_problem *hp, bool decode, const void *Q, const void *K8, const void *V8,
+                                  const float *k_scale, const float *v_scale, const int32_t *idx, const float *sink, void *O,
+                                  float *LSE, void *cuda_stream)
+{
+    Params p;
+    hs2_status s = sparse_common(hp, Q, K8, V8, idx, O, &p);
+    if (s != HS2_OK) return s;
+    if (!k_scale || !v_scale) return HS2_ERR_INVALID_ARG;
+    if (decode && p.Lq != 1) return HS2_ERR_INVALID_ARG;
+    if (!sparse_fp8_supported(p, hp->dtype) || !aligned16(Q, K8, V8, O)) return HS2_ERR_UNSUPPORTED;
+    if ((s = check_device()) != HS2_OK) return s;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    const cudaError_t e = decode ? launch_sparse_fp8_decode(p, Q, K8, V8, k_scale, v_scale, idx, sink, O, LSE, st)
+                                 : launch_sparse_fp8_prefill(p, Q, K8, V8, k_scale, v_scale, idx, sink, O, LSE, st);
+    return e == cudaSuccess ? HS2_OK : cuda_fail(e);
+}
+
+hs2_status hs2_sparse_attn_prefill_fp8kv(const hs2_problem *hp, const void *Q, const void *K8, const void *V8,
+                                         const float *k_scale, const float *v_scale, const int32_t *idx,
+                                         const float *sink, void *O, float *LSE, void *cuda_stream)
+{
+    return sparse_fp8_impl(hp, false, Q, K8, V8, k_scale, v_scale, idx, sink, O, LSE, cuda_stream);
+}
+
+hs2_status hs2_sparse_attn_decode_fp8kv(const hs2_problem *hp, const void *Q, const void *K8, const void *V8,
+                                        const float *k_scale, const float *v_scale, const int32_t *idx,
+                                        const float *sink, void *O, float *LSE, void *cuda_stream)
+{
+    return sparse_fp8_impl(hp, true, Q, K8, V8, k_scale, v_scale, idx, sink, O, LSE, cuda_stream);
+}
+
 hs2_status hs2_sparse_attn_decode_static(const hs2_problem *hp, const void *Q, const void *K, const void *V,
                                          const int32_t *idx, const float *sink, void *O, float *LSE,
                                          void *cuda_stream)

@@ -133,6 +133,14 @@ size_t sparse_tc5_ws_bytes(const Params &p);   // scratch that lets few queries 
 cudaError_t launch_sparse_tc5(const Params &p, const void *Q, const void *K, const void *V, const int32_t *idx,
                               const float *sink, void *O, float *LSE, void *ws, size_t ws_bytes, cudaStream_t st);
 cudaError_t read_sparse_tc5_error(unsigned *out);
+// FP8 (e4m3 + per-(token, KV head) scale) KV cache, bf16 queries: head_dim 128, group <= 8
+bool sparse_fp8_supported(const Params &p, hs2_dtype dt);
+cudaError_t launch_sparse_fp8_prefill(const Params &p, const void *Q, const void *K, const void *V, const float *ksc,
+                                      const float *vsc, const int32_t *idx, const float *sink, void *O, float *LSE,
+                                      cudaStream_t st);
+cudaError_t launch_sparse_fp8_decode(const Params &p, const void *Q, const void *K, const void *V, const float *ksc,
+                                     const float *vsc, const int32_t *idx, const float *sink, void *O, float *LSE,
+                                     cudaStream_t st);
 cudaError_t read_tc5_error(unsigned *out);
 cudaError_t read_sparse_error(unsigned *out);
 

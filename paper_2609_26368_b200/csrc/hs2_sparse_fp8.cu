@@ -1,0 +1,522 @@
+// Sparse attention over (reused top-k indices) U (forced window) on an FP8 KV cache: K and V stored as e4m3
+// codes with one fp32 scale per (token, KV head); Q and O stay bf16; head_dim 128, group <= 8.
+// (Section 3.3 for the operator; the paper's cost analysis of Section 4 assumes FP8 KV-cache storage.)
+//
+// The gather is bound by memory, so halving the bytes of a row is the whole point: a K or V row is 128 bytes
+// (+ 4 bytes of scale).  Structure as in the bf16 gather kernel - one warp per (query, KV head) item with a
+// private cp.async pipeline, keys on the MMA M dimension, heads on N - with these differences:
+//   * the stage holds the raw e4m3 rows (128-byte rows, 16-byte chunks XOR-swizzled by the row);
+//   * ldmatrix moves 16-bit units, i.e. PAIRS of codes.  For S^T = K Q^T a thread therefore receives four
+//     consecutive dims of a key per register; they are converted to two f16x2 registers (cvt e4m3x2 -> f16x2,
+//     exact) and used as k-slots (2t, 2t+1) and (2t+8, 2t+9) of an m16n8k16 f16 MMA - a permutation of the
+//     contraction index, matched by loading Q in the same order (four consecutive dims per thread);
+//   * for O^T = V^T P^T the transposing ldmatrix delivers, per register, codes (key 2t, dims 2g, 2g+1) and
+//     (key 2t+1, dims 2g, 2g+1); one byte permute makes them (dim 2g: keys 2t, 2t+1 | dim 2g+1: keys 2t, 2t+1),
+//     so MMA row g is dim 2g and row g+8 is dim 2g+1 of a 16-dim slice: the accumulator's dim order is a
+//     permutation that only the final store has to know;
+//   * the scales never touch the operands: the K scale multiplies the score row of its key, the V scale is
+//     folded into the probability of its key (times 2^8 to stay inside the normal range of f16; undone in the
+//     store).  The denominator sums the unscaled probabilities.
+// Decode: one CTA per (sequence, KV head), its warps split the attended set and merge through shared memory.
+#include <cuda_fp16.h>
+
+#include "hs2_common.cuh"
+
+#ifndef HS2_F8_WARPS
+#define HS2_F8_WARPS 12
+#endif
+#ifndef HS2_F8D_WARPS
+#define HS2_F8D_WARPS 8
+#endif
+
+namespace hs2 {
+namespace {
+
+constexpr int HD = 128;
+constexpr int KT = 16;                       // key rows per stage
+constexpr int NSTAGE = 2;
+constexpr int kRow = HD;                     // bytes of one e4m3 row
+constexpr int kTile = KT * kRow;             // one K or V tile of a stage
+constexpr int kStageBytes = 2 * kTile;
+// per warp: the stages, then per stage: key index of each row (32 ints), K scales (16), V scales (16)
+constexpr int kMetaBytes = 32 * 4 + 16 * 4 + 16 * 4;
+constexpr int kWarpSmem = NSTAGE * kStageBytes + NSTAGE * kMetaBytes;
+constexpr float kPShift = 256.f;             // probabilities x V scale are carried x 2^8 through the f16 operand
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void cp_async16(uint32_t dst, const void *src, int src_bytes)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;\n" ::"r"(dst), "l"(src), "r"(src_bytes));
+}
+__device__ __forceinline__ void cp_async4(uint32_t dst, const void *src, int src_bytes)
+{
+    asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;\n" ::"r"(dst), "l"(src), "r"(src_bytes));
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;\n" ::); }
+template <int N> __device__ __forceinline__ void cp_async_wait() { asm volatile("cp.async.wait_group %0;\n" ::"n"(N)); }
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], uint32_t addr)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t (&r)[4], uint32_t addr)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];\n"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a)
+{
+    uint32_t d;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;\n" : "=r"(d) : "r"(a));
+    return d;
+}
+__device__ __forceinline__ void mma_f16(float (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0, uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+// two e4m3 codes (low byte first) -> f16x2 (low half first); exact
+__device__ __forceinline__ uint32_t cvt_e4m3x2(uint32_t two_codes)
+{
+    uint32_t d;
+    asm("cvt.rn.f16x2.e4m3x2 %0, %1;\n" : "=r"(d) : "h"((unsigned short)two_codes));
+    return d;
+}
+__device__ __forceinline__ uint32_t pack_f16(float lo, float hi)
+{
+    __half2 v = __floats2half2_rn(lo, hi);
+    return *reinterpret_cast<uint32_t *>(&v);
+}
+__device__ __forceinline__ uint32_t pack_bf16(float lo, float hi)
+{
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+    return *reinterpret_cast<uint32_t *>(&v);
+}
+
+// Accumulators of one warp.  Thread (g = lane/4, t = lane%4) owns heads 2t and 2t+1 of the group:
+// o[dt][0..3] = O^T at (dim 16 dt + 2g, head 2t), (same dim, head 2t+1), (dim 16 dt + 2g + 1, head 2t),
+// (dim 16 dt + 2g + 1, head 2t+1), all times 2^8; m is replicated over g, l is this thread's partial sum.
+struct Acc {
+    float o[8][4];
+    float m[2], l[2];
+};
+
+struct Item {
+    const char *Kb, *Vb;          // first row of this (sequence, KV head)
+    const float *ksc, *vsc;       // its scales: element j * Hkv
+    int64_t row_stride;           // bytes between consecutive tokens
+    int sc_stride;                // floats between consecutive tokens' scales
+    const int32_t *irow;
+    int pos, kvl;
+};
+
+__device__ __forceinline__ Item make_item(const Params &p, const uint8_t *K, const uint8_t *V, const float *ksc, const float *vsc,
+                                          const int32_t *idx, int b, int gkv, int i)
+{
+    Item it;
+    const int64_t base = b * p.ks_b + gkv * p.ks_h;
+    it.Kb = reinterpret_cast<const char *>(K + base);
+    it.Vb = reinterpret_cast<const char *>(V + base);
+    it.ksc = ksc + (int64_t)b * p.Lk * p.Hkv + gkv;
+    it.vsc = vsc + (int64_t)b * p.Lk * p.Hkv + gkv;
+    it.row_stride = p.ks_t;
+    it.sc_stride = p.Hkv;
+    it.irow = idx ? idx + (((int64_t)b * p.Hkv + gkv) * p.Lq + i) * p.k : nullptr;
+    it.pos = pos_of(p, b, i);
+    it.kvl = kvlen_of(p, b);
+    return it;
+}
+
+// key index held by slot s of the virtual slot array [idx row | window], -1 when the slot is void
+__device__ __forceinline__ int slot_key(const Params &p, const Item &it, int tile, int lane)
+{
+    const int s = tile * KT + lane;
+    int j = -1;
+    if (lane < KT) {
+        if (s < p.k) {
+            j = it.irow ? __ldg(it.irow + s) : -1;
+            if (j > it.pos - p.w || j >= it.kvl) j = -1;
+        } else if (s < p.k + p.w) {
+            j = it.pos - p.w + 1 + (s - p.k);
+            if (j > it.pos || j >= it.kvl) j = -1;
+        }
+    }
+    return j;
+}
+
+// lane -> 16-byte chunk c (of 8) of rows r0 + (lane >> 3); lanes 0-15 also fetch the K scale of row `lane`,
+// lanes 16-31 the V scale of row `lane - 16`.  Void rows are zero filled, nothing is read for them.
+__device__ __forceinline__ void issue_stage(const Item &it, uint32_t stage_base, uint32_t meta_base, int j, int lane)
+{
+    const int c = lane & 7, hi = lane >> 3;
+    const char *kc = it.Kb + c * 16, *vc = it.Vb + c * 16;
+#pragma unroll
+    for (int r0 = 0; r0 < KT; r0 += 4) {
+        const int r = r0 + hi;
+        const int jr = __shfl_sync(0xffffffffu, j, r);
+        const uint32_t dst = stage_base + r * kRow + ((uint32_t)(c ^ (r & 7)) << 4);
+        const int64_t off = (int64_t)max(jr, 0) * it.row_stride;
+        const int nbytes = jr < 0 ? 0 : 16;
+        cp_async16(dst, kc + off, nbytes);
+        cp_async16(dst + kTile, vc + off, nbytes);
+    }
+    const int js = __shfl_sync(0xffffffffu, j, lane & 15);
+    const float *sp = (lane < 16 ? it.ksc : it.vsc) + (int64_t)max(js, 0) * it.sc_stride;
+    cp_async4(meta_base + 32 * 4 + lane * 4, sp, js < 0 ? 0 : 4);
+}
+
+__device__ __forceinline__ void consume_stage(Acc &acc, const uint32_t (&qf)[16], uint32_t stage_base, const float *sks,
+                                              const float *svs, unsigned mask, float scale_log2, int lane)
+{
+    const int g = lane >> 2;
+    const int mi = lane >> 3, rr = lane & 7;
+    float s[4] = {0.f, 0.f, 0.f, 0.f}, s2[4] = {0.f, 0.f, 0.f, 0.f};
+    // S^T = K Q^T : rows = keys, columns = heads.  One ldmatrix = 16 keys x 32 dims = two MMAs.
+    {
+        const uint32_t rowaddr = stage_base + ((mi & 1) * 8 + rr) * kRow;
+#pragma unroll
+        for (int q4 = 0; q4 < 4; ++q4) {
+            uint32_t a[4];
+            ldmatrix_x4(a, rowaddr + ((uint32_t)((2 * q4 + (mi >> 1)) ^ rr) << 4));
+            mma_f16(s, cvt_e4m3x2(a[0]), cvt_e4m3x2(a[1]), cvt_e4m3x2(a[0] >> 16), cvt_e4m3x2(a[1] >> 16), qf[4 * q4], qf[4 * q4 + 1]);
+            mma_f16(s2, cvt_e4m3x2(a[2]), cvt_e4m3x2(a[3]), cvt_e4m3x2(a[2] >> 16), cvt_e4m3x2(a[3] >> 16), qf[4 * q4 + 2], qf[4 * q4 + 3]);
+        }
+    }
+    // dequantise the score rows, online softmax in the base-2 domain; this thread: heads 2t+hh, keys g + 8 r
+    const float ks[2] = {sks[g] * scale_log2, sks[g + 8] * scale_log2};
+    const float vs[2] = {svs[g] * kPShift, svs[g + 8] * kPShift};
+    float mx[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+    for (int r = 0; r < 2; ++r) {
+        const bool ok = (mask >> (g + 8 * r)) & 1u;
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {
+            const float t2 = ok ? (s[2 * r + hh] + s2[2 * r + hh]) * ks[r] : -INFINITY;
+            s[2 * r + hh] = t2;
+            mx[hh] = fmaxf(mx[hh], t2);
+        }
+    }
+    float corr[2], muse[2];
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh) {
+        mx[hh] = fmaxf(mx[hh], __shfl_xor_sync(0xffffffffu, mx[hh], 4));
+        mx[hh] = fmaxf(mx[hh], __shfl_xor_sync(0xffffffffu, mx[hh], 8));
+        mx[hh] = fmaxf(mx[hh], __shfl_xor_sync(0xffffffffu, mx[hh], 16));
+        const float m_new = fmaxf(acc.m[hh], mx[hh]);
+        muse[hh] = m_new == -INFINITY ? 0.f : m_new;
+        corr[hh] = exp2f(acc.m[hh] - muse[hh]);
+        acc.m[hh] = m_new;
+        acc.l[hh] *= corr[hh];
+    }
+    float pv[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        pv[e] = exp2f(s[e] - muse[e & 1]);
+        acc.l[e & 1] += pv[e];
+    }
+    const uint32_t pb0 = movmatrix_trans(pack_f16(pv[0] * vs[0], pv[1] * vs[0]));   // keys 0..7
+    const uint32_t pb1 = movmatrix_trans(pack_f16(pv[2] * vs[1], pv[3] * vs[1]));   // keys 8..15
+    if (__any_sync(0xffffffffu, corr[0] != 1.f || corr[1] != 1.f)) {
+#pragma unroll
+        for (int dt = 0; dt < 8; ++dt) {
+            acc.o[dt][0] *= corr[0]; acc.o[dt][1] *= corr[1];
+            acc.o[dt][2] *= corr[0]; acc.o[dt][3] *= corr[1];
+        }
+    }
+    // O^T += V^T P^T : one transposing ldmatrix = 16 keys x 32 dims = two MMAs (16 dims each)
+    {
+        const uint32_t rowaddr = stage_base + kTile + ((mi & 1) * 8 + rr) * kRow;
+#pragma unroll
+        for (int dq = 0; dq < 4; ++dq) {
+            uint32_t a[4];
+            ldmatrix_x4_trans(a, rowaddr + ((uint32_t)((2 * dq + (mi >> 1)) ^ rr) << 4));
+#pragma unroll
+            for (int e = 0; e < 4; ++e) a[e] = __byte_perm(a[e], 0u, 0x3120);   // (dim 2g: keys 2t, 2t+1 | dim 2g+1: keys 2t, 2t+1)
+            mma_f16(acc.o[2 * dq], cvt_e4m3x2(a[0]), cvt_e4m3x2(a[0] >> 16), cvt_e4m3x2(a[1]), cvt_e4m3x2(a[1] >> 16), pb0, pb1);
+            mma_f16(acc.o[2 * dq + 1], cvt_e4m3x2(a[2]), cvt_e4m3x2(a[2] >> 16), cvt_e4m3x2(a[3]), cvt_e4m3x2(a[3] >> 16), pb0, pb1);
+        }
+    }
+}
+
+// Fold slot tiles [t_begin, t_end) of one item into acc with an NSTAGE-deep cp.async pipeline.
+__device__ __forceinline__ void run_tiles(const Params &p, const Item &it, const uint32_t (&qf)[16], Acc &acc, int t_begin,
+                                          int t_end, char *wsm, int lane)
+{
+    const uint32_t sbase = smem_u32(wsm);
+    char *meta = wsm + NSTAGE * kStageBytes;
+    const uint32_t mbase = sbase + NSTAGE * kStageBytes;
+    int next = t_begin;
+    int jn = next < t_end ? slot_key(p, it, next, lane) : -1;
+    int n_issued = 0, n_done = 0;
+    auto try_issue = [&](int stage) -> bool {
+        while (next < t_end) {
+            const int j = jn;
+            ++next;
+            if (next < t_end) jn = slot_key(p, it, next, lane);
+            if (__ballot_sync(0xffffffffu, j >= 0)) {   // all-void tiles are skipped
+                reinterpret_cast<int *>(meta + stage * kMetaBytes)[lane] = j;
+                issue_stage(it, sbase + stage * kStageBytes, mbase + stage * kMetaBytes, j, lane);
+                return true;
+            }
+        }
+        return false;
+    };
+#pragma unroll
+    for (int s = 0; s < NSTAGE - 1; ++s) {
+        if (try_issue(n_issued % NSTAGE)) ++n_issued;
+        cp_async_commit();
+    }
+    while (n_done < n_issued) {
+        const int stage = n_done % NSTAGE;
+        cp_async_wait<NSTAGE - 2>();
+        __syncwarp();
+        if (try_issue(n_issued % NSTAGE)) ++n_issued;
+        cp_async_commit();
+        const char *mt = meta + stage * kMetaBytes;
+        const unsigned mask = __ballot_sync(0xffffffffu, reinterpret_cast<const int *>(mt)[lane] >= 0);
+        consume_stage(acc, qf, sbase + stage * kStageBytes, reinterpret_cast<const float *>(mt + 32 * 4),
+                      reinterpret_cast<const float *>(mt + 32 * 4 + 16 * 4), mask, p.scale_log2, lane);
+        ++n_done;
+    }
+    cp_async_wait<0>();
+    __syncwarp();
+}
+
+// Q of head g in the contraction order of the K fragments: four consecutive dims per thread and 16-dim step.
+__device__ __forceinline__ void load_q_frags(const Params &p, const __nv_bfloat16 *Q, int b, int i, int gkv, int lane,
+                                             uint32_t (&qf)[16])
+{
+    const int g = lane >> 2, t = lane & 3;
+    if (g < p.G) {
+        const __nv_bfloat16 *q = Q + b * p.qs_b + i * p.qs_t + (gkv * p.G + g) * p.qs_h;
+#pragma unroll
+        for (int st = 0; st < 8; ++st) {   // dims 16 st + 4 t .. + 3
+            const uint2 raw = __ldg(reinterpret_cast<const uint2 *>(q + 16 * st + 4 * t));
+            const float2 lo = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&raw.x));
+            const float2 hi = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&raw.y));
+            qf[2 * st] = pack_f16(lo.x, lo.y);
+            qf[2 * st + 1] = pack_f16(hi.x, hi.y);
+        }
+    } else {
+#pragma unroll
+        for (int e = 0; e < 16; ++e) qf[e] = 0u;
+    }
+}
+
+__device__ __forceinline__ void init_acc(Acc &acc, const Params &p, const float *sink, int gkv, int lane, bool with_sink)
+{
+    const int g = lane >> 2, t = lane & 3;
+#pragma unroll
+    for (int dt = 0; dt < 8; ++dt) acc.o[dt][0] = acc.o[dt][1] = acc.o[dt][2] = acc.o[dt][3] = 0.f;
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh) {
+        const int head = 2 * t + hh;
+        float m = -INFINITY;
+        if (with_sink && sink && head < p.G) m = sink[gkv * p.G + head] * kLog2e;
+        acc.m[hh] = m;
+        acc.l[hh] = (m != -INFINITY && g == 0) ? 1.f : 0.f;
+    }
+}
+
+__device__ __forceinline__ void reduce_l(Acc &acc)
+{
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh) {
+        acc.l[hh] += __shfl_xor_sync(0xffffffffu, acc.l[hh], 4);
+        acc.l[hh] += __shfl_xor_sync(0xffffffffu, acc.l[hh], 8);
+        acc.l[hh] += __shfl_xor_sync(0xffffffffu, acc.l[hh], 16);
+    }
+}
+
+// Normalise and store one (query, KV head) result (staged through the warp's shared memory for 16-byte stores).
+__device__ __forceinline__ void store_output(const Params &p, const Acc &acc, __nv_bfloat16 *O, float *LSE, int b, int i,
+                                             int gkv, char *wsm, int lane)
+{
+    const int g = lane >> 2, t = lane & 3;
+    constexpr int kPitchO = HD + 8;   // bf16 elements per staged head row
+    __nv_bfloat16 *so = reinterpret_cast<__nv_bfloat16 *>(wsm);
+    float inv[2];
+#pragma unroll
+    for (int hh = 0; hh < 2; ++hh) inv[hh] = acc.l[hh] > 0.f ? (1.f / kPShift) / acc.l[hh] : 0.f;
+#pragma unroll
+    for (int dt = 0; dt < 8; ++dt)
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {   // dims 16 dt + 2g and + 1 of head 2t + hh are adjacent: one 4-byte store
+            const uint32_t two = pack_bf16(acc.o[dt][hh] * inv[hh], acc.o[dt][2 + hh] * inv[hh]);
+            *reinterpret_cast<uint32_t *>(so + (2 * t + hh) * kPitchO + 16 * dt + 2 * g) = two;
+        }
+    __syncwarp();
+#pragma unroll
+    for (int v = lane; v < 8 * 16; v += 32) {
+        const int head = v >> 4, c = v & 15;
+        if (head < p.G) {
+            const uint4 val = *reinterpret_cast<const uint4 *>(so + head * kPitchO + c * 8);
+            *reinterpret_cast<uint4 *>(O + b * p.os_b + i * p.os_t + (gkv * p.G + head) * p.os_h + c * 8) = val;
+        }
+    }
+    if (LSE && g == 0) {
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {
+            const int head = 2 * t + hh;
+            if (head < p.G)
+                LSE[((int64_t)b * p.Hq + gkv * p.G + head) * p.Lq + i] =
+                    acc.l[hh] > 0.f ? (acc.m[hh] + log2f(acc.l[hh])) * kLn2 : -INFINITY;
+        }
+    }
+}
+
+// ---------------------------------------------------------------- prefill: one warp per (b, g, i)
+__global__ void __launch_bounds__(HS2_F8_WARPS * 32)
+k_sparse_fp8_prefill(const Params p, const __nv_bfloat16 *__restrict__ Q, const uint8_t *__restrict__ K,
+                     const uint8_t *__restrict__ V, const float *__restrict__ ksc, const float *__restrict__ vsc,
+                     const int32_t *__restrict__ idx, const float *__restrict__ sink, __nv_bfloat16 *__restrict__ O,
+                     float *__restrict__ LSE)
+{
+    extern __shared__ __align__(128) char smem[];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t item = (int64_t)blockIdx.x * HS2_F8_WARPS + warp;   // (b, g, i), i fastest
+    if (item >= (int64_t)p.B * p.Hkv * p.Lq) return;
+    const int i = (int)(item % p.Lq);
+    const int gkv = (int)((item / p.Lq) % p.Hkv);
+    const int b = (int)(item / ((int64_t)p.Lq * p.Hkv));
+    char *wsm = smem + warp * kWarpSmem;
+    const Item it = make_item(p, K, V, ksc, vsc, idx, b, gkv, i);
+    uint32_t qf[16];
+    load_q_frags(p, Q, b, i, gkv, lane, qf);
+    Acc acc;
+    init_acc(acc, p, sink, gkv, lane, true);
+    run_tiles(p, it, qf, acc, 0, (p.k + p.w + KT - 1) / KT, wsm, lane);
+    reduce_l(acc);
+    store_output(p, acc, O, LSE, b, i, gkv, wsm, lane);
+}
+
+// ---------------------------------------------------------------- decode: one CTA per (sequence, KV head)
+__global__ void __launch_bounds__(HS2_F8D_WARPS * 32)
+k_sparse_fp8_decode(const Params p, const __nv_bfloat16 *__restrict__ Q, const uint8_t *__restrict__ K,
+                    const uint8_t *__restrict__ V, const float *__restrict__ ksc, const float *__restrict__ vsc,
+                    const int32_t *__restrict__ idx, const float *__restrict__ sink, __nv_bfloat16 *__restrict__ O,
+                    float *__restrict__ LSE)
+{
+    extern __shared__ __align__(128) char smem[];
+    constexpr int W = HS2_F8D_WARPS;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int bg = blockIdx.x;
+    const int gkv = bg % p.Hkv, b = bg / p.Hkv;
+    const int g = lane >> 2, t = lane & 3;
+    char *wsm = smem + warp * kWarpSmem;
+    float *sml = reinterpret_cast<float *>(smem + W * kWarpSmem);   // [W][16]: m then l per head
+    const Item it = make_item(p, K, V, ksc, vsc, idx, b, gkv, 0);
+    uint32_t qf[16];
+    load_q_frags(p, Q, b, 0, gkv, lane, qf);
+    Acc acc;
+    init_acc(acc, p, sink, gkv, lane, warp == 0);   // the sink joins the denominator once
+    const int n_tiles = (p.k + p.w + KT - 1) / KT;
+    const int per = (n_tiles + W - 1) / W;
+    run_tiles(p, it, qf, acc, warp * per, min(n_tiles, (warp + 1) * per), wsm, lane);
+    reduce_l(acc);
+    float4 *op = reinterpret_cast<float4 *>(wsm);   // the warp's own staging area: [8][32] float4
+#pragma unroll
+    for (int dt = 0; dt < 8; ++dt) op[dt * 32 + lane] = make_float4(acc.o[dt][0], acc.o[dt][1], acc.o[dt][2], acc.o[dt][3]);
+    if (g == 0) {
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) { sml[warp * 16 + 2 * t + hh] = acc.m[hh]; sml[warp * 16 + 8 + 2 * t + hh] = acc.l[hh]; }
+    }
+    __syncthreads();
+    if (warp != 0) return;
+    Acc tot;
+    float wgt[W][2];
+    tot.m[0] = tot.m[1] = -INFINITY;
+#pragma unroll
+    for (int s = 0; s < W; ++s)
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) tot.m[hh] = fmaxf(tot.m[hh], sml[s * 16 + 2 * t + hh]);
+    tot.l[0] = tot.l[1] = 0.f;
+#pragma unroll
+    for (int s = 0; s < W; ++s)
+#pragma unroll
+        for (int hh = 0; hh < 2; ++hh) {
+            const float ms = sml[s * 16 + 2 * t + hh];
+            wgt[s][hh] = ms == -INFINITY ? 0.f : exp2f(ms - tot.m[hh]);
+            tot.l[hh] += wgt[s][hh] * sml[s * 16 + 8 + 2 * t + hh];
+        }
+#pragma unroll
+    for (int dt = 0; dt < 8; ++dt) {
+        float4 a = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int s = 0; s < W; ++s) {
+            const float4 v = reinterpret_cast<const float4 *>(smem + s * kWarpSmem)[dt * 32 + lane];
+            a.x += wgt[s][0] * v.x; a.y += wgt[s][1] * v.y; a.z += wgt[s][0] * v.z; a.w += wgt[s][1] * v.w;
+        }
+        tot.o[dt][0] = a.x; tot.o[dt][1] = a.y; tot.o[dt][2] = a.z; tot.o[dt][3] = a.w;
+    }
+    __syncwarp();
+    // the output staging must not overlap the partials: it goes behind the per-warp areas
+    store_output(p, tot, O, LSE, b, 0, gkv, smem + W * kWarpSmem + W * 16 * 4, lane);
+}
+
+constexpr int kPrefillSmem = HS2_F8_WARPS * kWarpSmem;
+constexpr int kDecodeSmem = HS2_F8D_WARPS * kWarpSmem + HS2_F8D_WARPS * 16 * 4 + 8 * (HD + 8) * 2;
+static_assert(NSTAGE * kStageBytes >= 8 * 32 * 16, "a warp's stages hold its partial accumulator in decode");
+static_assert(NSTAGE * kStageBytes >= 8 * (HD + 8) * 2, "a warp's stages hold its staged output rows");
+
+template <class Kern>
+cudaError_t set_smem(Kern kern, int bytes, bool *done)
+{
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= 64) return cudaErrorNotSupported;
+    if (!done[dev]) {
+        if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes)) != cudaSuccess) return e;
+        done[dev] = true;
+    }
+    return cudaSuccess;
+}
+
+}  // namespace
+
+// bf16 queries, e4m3 cache with a scale per (token, KV head): head_dim 128, group <= 8; strides in bytes for the cache
+bool sparse_fp8_supported(const Params &p, hs2_dtype dt)
+{
+    auto m8 = [](int64_t x) { return x % 8 == 0; };
+    auto m16 = [](int64_t x) { return x % 16 == 0; };
+    if (p.ks_t > 0x7fffffffLL) return false;
+    return dt == HS2_BF16 && p.D == HD && p.G >= 1 && p.G <= 8 && m8(p.qs_b) && m8(p.qs_t) && m8(p.qs_h) && m16(p.ks_b) &&
+           m16(p.ks_t) && m16(p.ks_h) && m8(p.os_b) && m8(p.os_t) && m8(p.os_h);
+}
+
+cudaError_t launch_sparse_fp8_prefill(const Params &p, const void *Q, const void *K, const void *V, const float *ksc,
+                                      const float *vsc, const int32_t *idx, const float *sink, void *O, float *LSE,
+                                      cudaStream_t st)
+{
+    static bool done[64] = {};
+    cudaError_t e = set_smem(k_sparse_fp8_prefill, kPrefillSmem, done);
+    if (e != cudaSuccess) return e;
+    const int64_t items = (int64_t)p.B * p.Hkv * p.Lq;
+    if (items <= 0) return cudaSuccess;
+    const int64_t grid = (items + HS2_F8_WARPS - 1) / HS2_F8_WARPS;
+    if (grid > 0x7fffffffLL) return cudaErrorNotSupported;
+    k_sparse_fp8_prefill<<<(unsigned)grid, HS2_F8_WARPS * 32, kPrefillSmem, st>>>(
+        p, (const __nv_bfloat16 *)Q, (const uint8_t *)K, (const uint8_t *)V, ksc, vsc, idx, sink, (__nv_bfloat16 *)O, LSE);
+    count_launch();
+    return cudaGetLastError();
+}
+
+cudaError_t launch_sparse_fp8_decode(const Params &p, const void *Q, const void *K, const void *V, const float *ksc,
+                                     const float *vsc, const int32_t *idx, const float *sink, void *O, float *LSE,
+                                     cudaStream_t st)
+{
+    static bool done[64] = {};
+    cudaError_t e = set_smem(k_sparse_fp8_decode, kDecodeSmem, done);
+    if (e != cudaSuccess) return e;
+    const int64_t pairs = (int64_t)p.B * p.Hkv;
+    if (pairs <= 0) return cudaSuccess;
+    if (pairs > 0x7fffffffLL) return cudaErrorNotSupported;
+    k_sparse_fp8_decode<<<(unsigned)pairs, HS2_F8D_WARPS * 32, kDecodeSmem, st>>>(
+        p, (const __nv_bfloat16 *)Q, (const uint8_t *)K, (const uint8_t *)V, ksc, vsc, idx, sink, (__nv_bfloat16 *)O, LSE);
+    count_launch();
+    return cudaGetLastError();
+}
+
+}  // namespace hs2

@@ -328,6 +328,61 @@ def test_sigmoid_output_gate_in_every_sparse_kernel_family():
     assert hs2.hs2_device_error_flags() == 0
 
 
+def test_fp8_kv_cache_sparse_prefill_and_decode():
+    """Sparse attention on an e4m3 KV cache (codes + per-(token, KV head) scales) against the oracle run on the
+    dequantised cache: groups of 8, 4 and 1, ragged lengths, sink, a strided (fused K|V) cache, prefill and decode."""
+    from gen.workloads import quantize_kv_e4m3
+    cases = [
+        dict(q_len=150, kv_len=600, k_sel=100, window=24, batch=2),
+        dict(q_len=64, kv_len=300, k_sel=37, window=5, n_q_heads=8, n_kv_heads=2),
+        dict(q_len=40, kv_len=200, k_sel=0, window=50, n_q_heads=4, n_kv_heads=4),
+    ]
+    for ci, over in enumerate(cases):
+        wl = scaled("cfg2", n_needles=4, **over)
+        inp = make_inputs(wl)
+        run = BlockRun(inp).run_full()               # indices from the bf16 full layer
+        B, Lk, Hkv, D = inp.k.shape
+        k8, ksc = quantize_kv_e4m3(run.k)
+        v8, vsc = quantize_kv_e4m3(run.v)
+        if ci == 0:                                  # K and V as slices of one fused cache
+            fused = torch.empty(B, Lk, 2, Hkv, D, dtype=torch.uint8, device="cuda")
+            fused[:, :, 0].copy_(k8)
+            fused[:, :, 1].copy_(v8)
+            k8, v8 = fused[:, :, 0], fused[:, :, 1]
+        kv_lens = [Lk - 7 * b for b in range(wl.batch)]
+        kl_t = torch.tensor(kv_lens, dtype=torch.int32, device="cuda")
+        q = run.qs[0]
+        prob = hs2.Problem.from_tensors(q, k8, wl.k_sel, wl.window, kv_lens=kl_t)
+        sink = torch.linspace(-1.0, 1.5, wl.n_q_heads, device="cuda")
+        kd = oracle.dequant_e4m3(k8.contiguous(), ksc)
+        vd = oracle.dequant_e4m3(v8.contiguous(), vsc)
+        idx_rows = run.idx.permute(0, 2, 1, 3).reshape(B * wl.q_len, Hkv, wl.k_sel).cpu().numpy()
+        for sk in (None, sink):
+            out, lse = hs2.hs2_sparse_attn_prefill_fp8kv(prob, q, k8, v8, ksc, vsc, run.idx, sink=sk, want_lse=True)
+            torch.cuda.synchronize()
+            Oo, LSEo, _ = oracle.sparse_attn(q.float().cpu().numpy(), kd, vd, idx_rows, wl.window, kv_lens=kv_lens,
+                                             sink=None if sk is None else sk.cpu().numpy().astype(np.float64))
+            assert_output_close(out.reshape(-1, wl.n_q_heads, D), Oo, wl.torch_dtype, "fp8 sparse O")
+            l = lse.permute(0, 2, 1).reshape(B * wl.q_len, wl.n_q_heads).cpu().numpy()
+            fin = np.isfinite(LSEo)
+            assert np.array_equal(np.isfinite(l), fin) and np.abs(l[fin] - LSEo[fin]).max() <= TOL[wl.torch_dtype]["lse"]
+            q1 = q[:, -1:].contiguous()
+            prob1 = hs2.Problem.from_tensors(q1, k8, wl.k_sel, wl.window, kv_lens=kl_t)
+            od, ld = hs2.hs2_sparse_attn_decode_fp8kv(prob1, q1, k8, v8, ksc, vsc, run.idx[:, :, -1:].contiguous(), sink=sk,
+                                                      want_lse=True)
+            torch.cuda.synchronize()
+            assert (od.float() - out[:, -1:].float()).abs().max().item() <= 2e-2
+            assert (ld - lse[:, :, -1:]).abs().max().item() <= 2e-3
+    # shapes the FP8 kernels do not cover are refused, not mis-computed
+    wl = scaled("cfg2", q_len=16, kv_len=64, k_sel=8, window=4, n_q_heads=16, n_kv_heads=1, n_needles=4)
+    inp = make_inputs(wl, "cuda")
+    k8, ksc = quantize_kv_e4m3(inp.k)
+    prob = hs2.Problem.from_tensors(inp.q_full, k8, wl.k_sel, wl.window)
+    idx = torch.zeros(1, 1, 16, 8, dtype=torch.int32, device="cuda")
+    with pytest.raises(hs2.HS2Error):
+        hs2.hs2_sparse_attn_prefill_fp8kv(prob, inp.q_full, k8, k8, ksc, ksc, idx)
+
+
 def test_ragged_lengths_offsets_strides_and_sink():
     wl = scaled("cfg2", batch=3, q_len=70, kv_len=400, k_sel=40, window=12, n_needles=4)
     inp = make_inputs(wl)

@@ -371,3 +371,21 @@ def test_output_gate_special_values_and_library_sigmoid():
     O3, _, _ = oracle.sparse_attn(q, inp.k, inp.v, idx, wl.window, gate=gb)
     want = O0 * torch.sigmoid(gb.double()).reshape(B * Lq, Hq, D).numpy()
     assert np.abs(O3 - want).max() < 1e-14
+
+
+def test_e4m3_decoder_against_the_format_and_torch():
+    """The oracle's e4m3 decoder: landmark codes from the format definition, and all 256 codes against torch's
+    float8_e4m3fn -> float32 conversion."""
+    codes = np.arange(256, dtype=np.uint8)
+    val = oracle.decode_e4m3(codes)
+    assert val[0x00] == 0.0 and val[0x38] == 1.0 and val[0x7E] == 448.0 and val[0x01] == 2.0 ** -9 and val[0x08] == 2.0 ** -6
+    assert val[0xB8] == -1.0 and np.isnan(val[0x7F]) and np.isnan(val[0xFF])
+    ref = torch.arange(256, dtype=torch.uint8).view(torch.float8_e4m3fn).float().numpy().astype(np.float64)
+    ok = ~np.isnan(ref)
+    assert np.array_equal(np.isnan(val), ~ok) and np.array_equal(val[ok], ref[ok])
+    x = torch.randn(2, 5, 3, 16, generator=torch.Generator().manual_seed(3))
+    from gen.workloads import quantize_kv_e4m3
+    c8, sc = quantize_kv_e4m3(x)
+    deq = oracle.dequant_e4m3(c8, sc)
+    assert deq.dtype == np.float32 and np.abs(deq - x.numpy()).max() <= np.abs(x.numpy()).max() / 16 + 1e-6   # 3 mantissa bits
+    assert np.abs(deq).reshape(-1, 16).max(axis=1).max() <= np.abs(x.numpy()).max() * (1 + 1e-6)
