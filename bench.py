@@ -347,7 +347,30 @@ def bench_decode_64k(device, peaks, reps=5, burst=40, ctx=65536):
     us = statistics.median(per) * 1e3
     gb = gathered_kv_bytes(wl)
     ach = gb / (us * 1e-6) / 1e9
-    return {"workload": "cfg5: B=64, ctx %d, 32q/4kv, D=128, bf16, k=2048, w=128" % ctx,
+    # the same step on an e4m3 cache (codes + one fp32 scale per (token, KV head)): 264 B per attended token
+    from gen.workloads import quantize_kv_e4m3
+    k8, ksc = quantize_kv_e4m3(k)
+    v8, vsc = quantize_kv_e4m3(v)
+    prob8 = hs2.Problem.from_tensors(inp.q_full, k8, wl.k_sel, wl.window)
+
+    def run8(n):
+        for it in range(n):
+            hs2.hs2_sparse_attn_decode_fp8kv(prob8, qss[it % nset], k8, v8, ksc, vsc, idxs[it % nset], out=out)
+    run8(8)
+    torch.cuda.synchronize()
+    per8 = []
+    for _ in range(reps):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        run8(burst)
+        b.record()
+        torch.cuda.synchronize()
+        per8.append(a.elapsed_time(b) / burst)
+    us8 = statistics.median(per8) * 1e3
+    gb8 = gb / 512.0 * 264.0
+    fp8 = {"sparse_decode_us_per_step": round(us8, 2), "gathered_kv_bytes": gb8,
+           "achieved_gbs": round(gb8 / (us8 * 1e-6) / 1e9, 1), "frac": round(gb8 / (us8 * 1e-6) / 1e9 / peaks["hbm_gbs"], 4)}
+    return {"workload": "cfg5: B=64, ctx %d, 32q/4kv, D=128, bf16, k=2048, w=128" % ctx, "fp8_kv_cache": fp8,
             "sparse_decode_us_per_step": round(us, 2), "gathered_kv_bytes": gb,
             "achieved_gbs": round(ach, 1), "peak_gbs": peaks["hbm_gbs"], "frac": round(ach / peaks["hbm_gbs"], 4),
             "full_attn_select_decode_ms": round(min(t_full[1:]), 3), "launches_back_to_back": burst,

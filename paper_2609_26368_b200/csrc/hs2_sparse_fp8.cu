@@ -34,7 +34,10 @@ namespace {
 
 constexpr int HD = 128;
 constexpr int KT = 16;                       // key rows per stage
-constexpr int NSTAGE = 2;
+#ifndef HS2_F8_NSTAGE
+#define HS2_F8_NSTAGE 2
+#endif
+constexpr int NSTAGE = HS2_F8_NSTAGE;
 constexpr int kRow = HD;                     // bytes of one e4m3 row
 constexpr int kTile = KT * kRow;             // one K or V tile of a stage
 constexpr int kStageBytes = 2 * kTile;
