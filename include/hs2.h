@@ -74,6 +74,10 @@ typedef struct {
     int64_t q_stride[3];             /* elements: (batch, token, head); all 0 => packed */
     int64_t kv_stride[3];            /* shared by K and V */
     int64_t o_stride[3];
+    int32_t select_block;            /* selection granularity of hs2_full_attn_select / hs2_topk_select: 0 or 1 =
+                                        individual tokens (the paper's method); B > 1 = aligned blocks of B tokens,
+                                        the block-level variant the paper ablates against (Section 5, Ablation 1:
+                                        block size 64, 1024 tokens = 16 blocks); k_sel must then be a multiple of B */
 } hs2_problem;
 
 /* Bytes of scratch `op` needs for this problem (a host-side computation; 0 is a valid answer).
@@ -86,6 +90,9 @@ size_t hs2_workspace_bytes(const hs2_problem *p, hs2_op op);
  *
  *   O    out  attention output, same layout/dtype as Q
  *   LSE  out  log-sum-exp of the scaled logits per (batch, head, query), natural log; required
+ *   (With p->select_block = B > 1 the selection is block-level instead: the candidates of a row are cut into
+ *   aligned blocks [B m, B m + B); a block's score is the maximum a[j] over its candidate keys; the k_sel / B
+ *   best blocks (ties: lower block first) are kept and idx holds their candidate keys, ascending, -1 padded.)
  *   idx  out  [batch, n_kv_heads, q_len, k_sel] or NULL to skip the selection.  Row (b,g,i) holds the
  *             min(k_sel, pos-w+1) candidates with the highest group score
  *                 a[j] = max over the query heads h of group g of (scale*<q_h,k_j> - LSE_h)

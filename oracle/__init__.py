@@ -203,3 +203,26 @@ def dequant_e4m3(codes, scales):
     if not isinstance(scales, np.ndarray):
         scales = scales.detach().cpu().numpy()
     return (decode_e4m3(codes) * scales.astype(np.float64)[..., None]).astype(np.float32)
+
+
+def select_blocks(scores, pos, kvlen, window: int, k_sel: int, block: int) -> np.ndarray:
+    """Block-level selection (the variant of the paper's first ablation, Section 5) on given scores ``[n, Lk]``.
+
+    The candidates of a row are the keys 0 .. min(pos - window, kvlen - 1); they are cut into aligned blocks of
+    ``block`` keys (the last may be partial); a block scores the maximum over its candidates; the ``k_sel // block``
+    best blocks (ties: lower block first) are kept and their candidate keys listed ascending, -1 padded.
+    """
+    sc = np.asarray(scores, dtype=np.float64)
+    n, Lk = sc.shape
+    pos = np.broadcast_to(np.asarray(pos, dtype=np.int64), (n,))
+    kvlen = np.broadcast_to(np.asarray(kvlen, dtype=np.int64), (n,))
+    assert block >= 1 and k_sel % block == 0
+    idx = np.full((n, k_sel), -1, dtype=np.int32)
+    for r in range(n):
+        nk = int(max(0, min(pos[r] - window + 1, kvlen[r])))
+        nb = (nk + block - 1) // block
+        best = [max(sc[r, m * block:min(nk, (m + 1) * block)]) for m in range(nb)]
+        order = sorted(range(nb), key=lambda m: (-best[m], m))[:k_sel // block]
+        keys = [j for m in sorted(order) for j in range(m * block, min(nk, (m + 1) * block))]
+        idx[r, :len(keys)] = keys
+    return idx

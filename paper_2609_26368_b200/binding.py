@@ -40,7 +40,8 @@ class _CProblem(C.Structure):
                 ("head_dim", C.c_int32), ("q_len", C.c_int32), ("kv_len", C.c_int32),
                 ("k_sel", C.c_int32), ("window", C.c_int32), ("softmax_scale", C.c_float),
                 ("dtype", C.c_int), ("q_start", C.c_void_p), ("kv_lens", C.c_void_p),
-                ("q_stride", C.c_int64 * 3), ("kv_stride", C.c_int64 * 3), ("o_stride", C.c_int64 * 3)]
+                ("q_stride", C.c_int64 * 3), ("kv_stride", C.c_int64 * 3), ("o_stride", C.c_int64 * 3),
+                ("select_block", C.c_int32)]
 
 
 _lib = None
@@ -135,13 +136,14 @@ class Problem:
 
     def __init__(self, batch, q_len, kv_len, n_q_heads, n_kv_heads, head_dim, k_sel, window, dtype=torch.bfloat16,
                  softmax_scale: float = 0.0, q_start: Optional[torch.Tensor] = None,
-                 kv_lens: Optional[torch.Tensor] = None):
+                 kv_lens: Optional[torch.Tensor] = None, select_block: int = 0):
         self.batch, self.q_len, self.kv_len = int(batch), int(q_len), int(kv_len)
         self.n_q_heads, self.n_kv_heads, self.head_dim = int(n_q_heads), int(n_kv_heads), int(head_dim)
         self.k_sel, self.window = int(k_sel), int(window)
         self.dtype = dtype
         self.softmax_scale = float(softmax_scale)
         self.q_start, self.kv_lens = q_start, kv_lens
+        self.select_block = int(select_block)
         for t in (q_start, kv_lens):
             assert t is None or (t.dtype == torch.int32 and t.is_cuda and t.is_contiguous())
 
@@ -159,6 +161,7 @@ class Problem:
                       HS2_F32 if self.dtype == torch.float32 else HS2_BF16,
                       None if self.q_start is None else self.q_start.data_ptr(),
                       None if self.kv_lens is None else self.kv_lens.data_ptr())
+        c.select_block = self.select_block
         if q is not None:
             c.q_stride = _strides(q)
         if kv is not None:

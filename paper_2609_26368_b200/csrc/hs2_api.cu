@@ -38,6 +38,8 @@ hs2_status resolve(const hs2_problem *hp, bool need_tensors, Params *out)
     p.B = hp->batch; p.Hkv = hp->n_kv_heads; p.Lq = hp->q_len; p.Lk = hp->kv_len;
     p.k = hp->k_sel; p.w = hp->window;
     p.q_start = hp->q_start; p.kv_lens = hp->kv_lens;
+    p.blk = hp->select_block > 1 ? hp->select_block : 1;
+    if (hp->select_block < 0 || (p.blk > 1 && (hp->k_sel % p.blk != 0 || p.blk > 1024))) return HS2_ERR_INVALID_ARG;
     p.Hq = hp->n_q_heads; p.D = hp->head_dim;
     if (need_tensors) {
         if (hp->n_q_heads <= 0 || hp->n_q_heads % hp->n_kv_heads != 0 || hp->head_dim <= 0) return HS2_ERR_INVALID_ARG;
@@ -63,6 +65,13 @@ hs2_status resolve(const hs2_problem *hp, bool need_tensors, Params *out)
 }
 
 int64_t select_rows(const Params &p) { return (int64_t)p.B * p.Hkv * p.Lq; }
+
+// token-level top-k (Section 3.3) or the block-level variant of the paper's first ablation
+cudaError_t launch_select(const Params &p, const float *scores, int64_t stride, int32_t *idx, int64_t r0, int64_t n,
+                          cudaStream_t st)
+{
+    return p.blk > 1 ? launch_block_select(p, scores, stride, idx, r0, n, st) : launch_topk(p, scores, stride, idx, r0, n, st);
+}
 
 size_t strip_row_bytes(const Params &p) { return align_up((size_t)p.Lk * sizeof(float), 16); }
 
@@ -100,7 +109,7 @@ FilterPlan filter_plan(const Params &p, hs2_dtype dt)
     f.ns_w = filter_sample_width(p, kFilterSamp);
     f.per_row = align_up((size_t)f.ns_w * 4, 16);
     if ((size_t)f.cap * 8 > f.per_row) f.per_row = (size_t)f.cap * 8;
-    f.ok = p.k > 0 && !g_disable_tc5.load(std::memory_order_relaxed) && scores_filter_supported(p, dt) && f.cap <= 32768 && f.ns_w <= 32768 && p.Lk > f.cap &&
+    f.ok = p.k > 0 && p.blk == 1 && !g_disable_tc5.load(std::memory_order_relaxed) && scores_filter_supported(p, dt) && f.cap <= 32768 && f.ns_w <= 32768 && p.Lk > f.cap &&
            p.Lk >= g_filter_min_keys.load(std::memory_order_relaxed) && select_rows(p) >= 1024;
     return f;
 }
@@ -262,7 +271,7 @@ hs2_status hs2_full_attn_select(const hs2_problem *hp, const void *Q, const void
             float *dst = scores_dbg + r0 * p.Lk;
             e = launch_scores(p, dt, mma, aligned16(Q, K, V, O), Q, K, LSE, dst, p.Lk, r0, n, true, st);
             if (e != cudaSuccess) return cuda_fail(e);
-            if (want_sel && (e = launch_topk(p, dst, p.Lk, idx, r0, n, st)) != cudaSuccess) return cuda_fail(e);
+            if (want_sel && (e = launch_select(p, dst, p.Lk, idx, r0, n, st)) != cudaSuccess) return cuda_fail(e);
         }
         return HS2_OK;
     }
@@ -308,7 +317,7 @@ hs2_status hs2_full_attn_select(const hs2_problem *hp, const void *Q, const void
         const int64_t n = rows - r0 < block ? rows - r0 : block;
         e = launch_scores(p, dt, mma, al, Q, K, LSE, strip, stride, r0, n, false, st);
         if (e != cudaSuccess) return cuda_fail(e);
-        if ((e = launch_topk(p, strip, stride, idx, r0, n, st)) != cudaSuccess) return cuda_fail(e);
+        if ((e = launch_select(p, strip, stride, idx, r0, n, st)) != cudaSuccess) return cuda_fail(e);
     }
     return HS2_OK;
 }
@@ -322,7 +331,7 @@ hs2_status hs2_topk_select(const hs2_problem *hp, const float *scores, int32_t *
     if (s != HS2_OK) return s;
     if (p.k > 0 && (!scores || !idx)) return HS2_ERR_INVALID_ARG;
     if ((s = check_device()) != HS2_OK) return s;
-    cudaError_t e = launch_topk(p, scores, p.Lk, idx, 0, select_rows(p), (cudaStream_t)cuda_stream);
+    cudaError_t e = launch_select(p, scores, p.Lk, idx, 0, select_rows(p), (cudaStream_t)cuda_stream);
     return e == cudaSuccess ? HS2_OK : cuda_fail(e);
 }
 

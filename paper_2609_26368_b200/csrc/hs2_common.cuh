@@ -21,6 +21,7 @@ struct Params {
     int64_t qs_b, qs_t, qs_h;   // element strides
     int64_t ks_b, ks_t, ks_h;
     int64_t os_b, os_t, os_h;
+    int blk;            // selection granularity: 1 = tokens, B > 1 = aligned blocks of B tokens
     const void *gate;   // optional output-gate logits of the sparse layers: shape, dtype and strides of O; null = no gate
 };
 
@@ -78,6 +79,9 @@ cudaError_t launch_scores_generic(const Params &p, hs2_dtype dt, const void *Q, 
 cudaError_t launch_sparse_generic(const Params &p, hs2_dtype dt, const void *Q, const void *K, const void *V,
                                   const int32_t *idx, const float *sink, void *O, float *LSE, cudaStream_t st);
 
+// Block-level selection (p.blk > 1) over score rows [row0, row0+n_rows); `scores` points at row row0.
+cudaError_t launch_block_select(const Params &p, const float *scores, int64_t score_stride, int32_t *idx, int64_t row0,
+                                int64_t n_rows, cudaStream_t st);
 // Radix select over score rows [row0, row0+n_rows); `scores` points at row row0.
 cudaError_t launch_topk(const Params &p, const float *scores, int64_t score_stride, int32_t *idx,
                         int64_t row0, int64_t n_rows, cudaStream_t st);

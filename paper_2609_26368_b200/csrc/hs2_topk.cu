@@ -899,6 +899,118 @@ int filter_sample_width(const Params &p, int samp)
 }
 
 // thresholds tau_key[row] from the sampled strips (row stride `stride` floats); clears flag[row]
+// ---- block-level selection (the variant the paper ablates against: Section 5, Ablation 1) --------------------------
+// One warp per row.  The row's candidates 0..n-1 are cut into aligned blocks of p.blk keys (the last one may be
+// partial); a block's score is the maximum over its candidate keys; the k/blk best blocks (ties: lower block first)
+// are kept and their candidate keys written in ascending order.  The row is read once, coalesced; the block maxima
+// live in the warp's shared memory; the selection is k/blk rounds of a warp-wide argmax.
+constexpr int kBlkWarps = 8;
+
+__global__ void __launch_bounds__(kBlkWarps * 32)
+k_block_select(const Params p, const float *__restrict__ scores, int64_t score_stride, int32_t *__restrict__ idx, int64_t row0,
+               int64_t n_rows, int nb_max)
+{
+    extern __shared__ uint32_t s_blk[];   // [kBlkWarps][nb_max] block maxima as order-preserving keys; [kBlkWarps][k/blk] winners
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int64_t lr = (int64_t)blockIdx.x * kBlkWarps + warp;
+    if (lr >= n_rows) return;
+    const int64_t row = row0 + lr;
+    const int i = (int)(row % p.Lq);
+    const int b = (int)(row / ((int64_t)p.Lq * p.Hkv));
+    const int kvl = kvlen_of(p, b);
+    const int pos = pos_of(p, b, i);
+    const int n = max(0, min(pos - p.w + 1, kvl));
+    const int B = p.blk, kb = p.k / B;
+    const int nb = (n + B - 1) / B;
+    int32_t *out = idx + row * p.k;
+    uint32_t *bk = s_blk + (size_t)warp * nb_max;
+    int *win = reinterpret_cast<int *>(s_blk + (size_t)kBlkWarps * nb_max) + warp * kb;
+    const float *srow = scores + lr * score_stride;
+    const int take = min(kb, nb);
+    if (take < nb) {
+        // block maxima: lane l folds keys l, l + 32, ... of a block, then a warp maximum.  0 marks "already taken",
+        // and no real score maps to key 0 (the key of the NaN with all bits set)
+        for (int m = 0; m < nb; ++m) {
+            uint32_t best = 1u;
+            const int hi = min(n, (m + 1) * B);
+            for (int j = m * B + lane; j < hi; j += 32) best = max(best, max(order_key(srow[j]), 1u));
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) best = max(best, __shfl_xor_sync(0xffffffffu, best, o));
+            if (lane == 0) bk[m] = best;
+        }
+        __syncwarp();
+        for (int r = 0; r < take; ++r) {
+            // argmax with ties to the lower block: compare (key, ~block)
+            unsigned long long best = 0ull;
+            for (int m = lane; m < nb; m += 32) {
+                const unsigned long long c = ((unsigned long long)bk[m] << 32) | (uint32_t)(~m);
+                if (bk[m] != 0u && c > best) best = c;
+            }
+#pragma unroll
+            for (int o = 16; o > 0; o >>= 1) {
+                const unsigned long long t = __shfl_xor_sync(0xffffffffu, best, o);
+                best = t > best ? t : best;
+            }
+            const int m = (int)~(uint32_t)best;
+            if (lane == 0) { win[r] = m; bk[m] = 0u; }
+            __syncwarp();
+        }
+        // ascending block order: rank of each winner among the winners (take <= k / blk is small)
+        int mine[2] = {-1, -1}, rank[2] = {0, 0};
+        for (int u = 0; u < 2; ++u) {
+            const int r = lane + 32 * u;
+            if (r < take) {
+                mine[u] = win[r];
+                for (int q = 0; q < take; ++q) rank[u] += win[q] < mine[u];
+            }
+        }
+        __syncwarp();
+        if (take <= 64) {
+            for (int u = 0; u < 2; ++u)
+                if (mine[u] >= 0) win[rank[u]] = mine[u];
+        } else if (lane == 0) {   // many blocks per row: a plain insertion sort by one lane
+            for (int a = 1; a < take; ++a) {
+                const int v = win[a];
+                int c = a - 1;
+                while (c >= 0 && win[c] > v) { win[c + 1] = win[c]; --c; }
+                win[c + 1] = v;
+            }
+        }
+        __syncwarp();
+    }
+    // emit the candidate keys of the kept blocks, ascending; a partial last block gives fewer than B keys
+    int written = 0;
+    for (int r = 0; r < take; ++r) {
+        const int m = take < nb ? win[r] : r;
+        const int lo = m * B, hi = min(n, lo + B);
+        for (int j = lo + lane; j < hi; j += 32) out[written + (j - lo)] = j;
+        written += hi - lo;
+    }
+    for (int t = written + lane; t < p.k; t += 32) out[t] = -1;
+}
+
+cudaError_t launch_block_select(const Params &p, const float *scores, int64_t score_stride, int32_t *idx, int64_t row0,
+                                int64_t n_rows, cudaStream_t st)
+{
+    if (n_rows <= 0 || p.k <= 0) return cudaSuccess;
+    const int nb_max = (p.Lk + p.blk - 1) / p.blk;
+    const size_t smem = (size_t)kBlkWarps * (nb_max + p.k / p.blk) * sizeof(uint32_t);
+    if (smem > 200 * 1024) return cudaErrorNotSupported;
+    static bool done[64] = {};
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64 && !done[dev]) {
+        if ((e = cudaFuncSetAttribute(k_block_select, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024)) != cudaSuccess) return e;
+        done[dev] = true;
+    }
+    const int64_t grid = (n_rows + kBlkWarps - 1) / kBlkWarps;
+    if (grid > 0x7fffffffLL) return cudaErrorNotSupported;
+    k_block_select<<<(unsigned)grid, kBlkWarps * 32, smem, st>>>(p, scores, score_stride, idx, row0, n_rows, nb_max);
+    count_launch();
+    return cudaGetLastError();
+}
+
 cudaError_t launch_filter_thresholds(const Params &p, const float *sample, int64_t stride, int64_t row0, int64_t n_rows,
                                      int samp, int cap, uint32_t *tau_key, int *flag, cudaStream_t st)
 {

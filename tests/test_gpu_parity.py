@@ -383,6 +383,45 @@ def test_fp8_kv_cache_sparse_prefill_and_decode():
         hs2.hs2_sparse_attn_prefill_fp8kv(prob, inp.q_full, k8, k8, ksc, ksc, idx)
 
 
+def test_block_level_selection_variant():
+    """select_block = B (Section 5, Ablation 1: blocks of 64, 16 blocks) against the oracle: bit-exact on the GPU's
+    own fp32 scores, through hs2_topk_select on given scores (ties, partial last blocks, ragged lengths), and the
+    sparse layer consuming the block-structured index rows."""
+    rng = np.random.default_rng(3)
+    B_, Hkv, Lq, Lk, w = 2, 2, 50, 700, 9
+    sc = torch.tensor(np.round(rng.normal(size=(B_, Hkv, Lq, Lk)) * 4) / 4, dtype=torch.float32, device="cuda")
+    qs = torch.tensor([600, 37], dtype=torch.int32, device="cuda")
+    kl = torch.tensor([700, 90], dtype=torch.int32, device="cuda")
+    for blk, k in ((64, 256), (16, 48), (4, 64), (1, 30)):
+        prob = hs2.Problem(B_, Lq, Lk, 4, Hkv, 64, k, w, q_start=qs, kv_lens=kl, select_block=blk)
+        idx = hs2.hs2_topk_select(prob, sc)
+        torch.cuda.synchronize()
+        for b in range(B_):
+            pos = qs[b].item() + np.arange(Lq)
+            for g in range(Hkv):
+                want = oracle.select_blocks(sc[b, g].cpu().numpy(), pos, kl[b].item(), w, k, blk)
+                assert np.array_equal(idx[b, g].cpu().numpy(), want), (blk, b, g)
+    with pytest.raises(hs2.HS2Error):      # k must be a whole number of blocks
+        hs2.hs2_topk_select(hs2.Problem(B_, Lq, Lk, 4, Hkv, 64, 100, w, select_block=64), sc)
+    # the full layer in block mode, then a sparse layer on its indices
+    wl = scaled("cfg2", q_len=300, kv_len=900, k_sel=256, window=32, n_needles=8)
+    inp = make_inputs(wl, "cuda")
+    prob = hs2.Problem.from_tensors(inp.q_full, inp.k, wl.k_sel, wl.window, select_block=64)
+    O, LSE, idx, scores = hs2.hs2_full_attn_select(prob, inp.q_full, inp.k, inp.v, want_scores=True)
+    idx2 = hs2.hs2_full_attn_select(prob, inp.q_full, inp.k, inp.v)[2]      # strip path
+    torch.cuda.synchronize()
+    assert torch.equal(idx, idx2)
+    pos = wl.kv_len - wl.q_len + np.arange(wl.q_len)
+    for g in range(wl.n_kv_heads):
+        want = oracle.select_blocks(scores[0, g].cpu().numpy(), pos, wl.kv_len, wl.window, wl.k_sel, 64)
+        assert np.array_equal(idx[0, g].cpu().numpy(), want)
+    out, _ = hs2.hs2_sparse_attn_prefill(prob, inp.q_sparse[0], inp.k, inp.v, idx)
+    torch.cuda.synchronize()
+    idx_rows = idx.permute(0, 2, 1, 3).reshape(wl.q_len, wl.n_kv_heads, wl.k_sel).cpu().numpy()
+    Oo, _, _ = oracle.sparse_attn(to_host(inp.q_sparse[0]), to_host(inp.k), to_host(inp.v), idx_rows, wl.window)
+    assert_output_close(out.reshape(-1, wl.n_q_heads, wl.head_dim), Oo, wl.torch_dtype, "sparse O on block indices")
+
+
 def test_ragged_lengths_offsets_strides_and_sink():
     wl = scaled("cfg2", batch=3, q_len=70, kv_len=400, k_sel=40, window=12, n_needles=4)
     inp = make_inputs(wl)

@@ -389,3 +389,26 @@ def test_e4m3_decoder_against_the_format_and_torch():
     deq = oracle.dequant_e4m3(c8, sc)
     assert deq.dtype == np.float32 and np.abs(deq - x.numpy()).max() <= np.abs(x.numpy()).max() / 16 + 1e-6   # 3 mantissa bits
     assert np.abs(deq).reshape(-1, 16).max(axis=1).max() <= np.abs(x.numpy()).max() * (1 + 1e-6)
+
+
+def test_block_level_selection_reduces_to_token_level_and_matches_brute_force():
+    """Block-level selection (Section 5, Ablation 1): block size 1 is the token-level selection; for larger blocks
+    a block is kept iff fewer than k/B candidate blocks beat it (score, then lower index), and exactly the candidate
+    keys of the kept blocks are listed, ascending."""
+    rng = np.random.default_rng(7)
+    n, Lk, w = 40, 97, 5
+    sc = np.round(rng.normal(size=(n, Lk)) * 2) / 2          # many ties
+    pos = rng.integers(0, Lk + 10, size=n)
+    kvl = rng.integers(1, Lk + 1, size=n)
+    assert np.array_equal(oracle.select_blocks(sc, pos, kvl, w, 12, 1), oracle.select(sc, pos, kvl, w, 12))
+    for B, k in ((4, 12), (8, 16), (16, 64)):
+        idx = oracle.select_blocks(sc, pos, kvl, w, k, B)
+        for r in range(n):
+            nk = max(0, min(pos[r] - w + 1, kvl[r]))
+            nb = -(-nk // B)
+            bmax = [sc[r, m * B:min(nk, (m + 1) * B)].max() for m in range(nb)]
+            kept = {m for m in range(nb)
+                    if sum(1 for o in range(nb) if bmax[o] > bmax[m] or (bmax[o] == bmax[m] and o < m)) < k // B}
+            want = [j for m in sorted(kept) for j in range(m * B, min(nk, (m + 1) * B))]
+            got = [j for j in idx[r] if j >= 0]
+            assert got == want and all(j == -1 for j in idx[r, len(got):])
