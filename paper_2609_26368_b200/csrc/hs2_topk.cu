@@ -14,6 +14,7 @@ namespace {
 
 constexpr int kItems = 4;                    // consecutive scores per thread per step
 constexpr unsigned kListCap = 2048;          // threshold-bin candidates kept in shared memory (cached variant)
+constexpr int kStageOut = 4096;              // selected indices of a row staged in shared memory (cached variant)
 
 // float -> uint32 whose unsigned order is the float order; -0 is folded onto +0 first.
 __device__ __forceinline__ uint32_t order_key(float f)
@@ -270,6 +271,8 @@ k_topk_cached(const Params p, const float *__restrict__ scores, int64_t score_st
         __syncthreads();   // every thread has read hist[digit] before the next round zeroes the histogram
         if (collect) {
             // every candidate that can still be the take-th largest sits in this bin (at most kListCap of them)
+            // (one atomic per member on a single word looks wasteful, but a ballot-aggregated version was measured
+            // slower: 2.31 vs 2.18 ms for the whole full layer on the 8K benchmark)
 #pragma unroll
             for (int e = 0; e < E; ++e)
                 if (j0 + e < nc && (key[e] >> hi) == prefix) {
@@ -367,18 +370,28 @@ k_topk_cached(const Params p, const float *__restrict__ scores, int64_t score_st
     }
     const unsigned excl = __shfl_sync(0xffffffffu, wincl - wsum, warp) + incl - packed;
     unsigned gt_before = excl >> 16, eq_before = excl & 0xffffu;
+    // the kept indices are collected in shared memory (every thread owns a run of positions) and leave as one
+    // coalesced row; rows with more than kStageOut selected tokens write straight to global memory
+    extern __shared__ int s_out[];
+    const bool staged = p.k <= kStageOut;
+    int *dst = staged ? s_out : out;
 #pragma unroll
     for (int e = 0; e < E; ++e) {
         if (j0 + e >= nc) continue;
         if (key[e] > tau) {
-            out[gt_before + min(eq_before, need_eq)] = MODE == SEL_CAND ? prow[j0 + e] : j0 + e;
+            dst[gt_before + min(eq_before, need_eq)] = j0 + e;
             ++gt_before;
         } else if (key[e] == tau) {
-            if (eq_before < need_eq) out[gt_before + eq_before] = MODE == SEL_CAND ? prow[j0 + e] : j0 + e;
+            if (eq_before < need_eq) dst[gt_before + eq_before] = j0 + e;
             ++eq_before;
         }
     }
-    for (int t = take + tid; t < p.k; t += THREADS) out[t] = -1;
+    if (staged) {
+        __syncthreads();
+        for (int t = tid; t < p.k; t += THREADS) out[t] = t < take ? s_out[t] : -1;
+    } else {
+        for (int t = take + tid; t < p.k; t += THREADS) out[t] = -1;
+    }
 }
 
 // ---- rows of up to CL x 32768 candidates: one thread-block cluster per row ------------------------
@@ -750,12 +763,13 @@ void launch_class(int c, const Params &p, const float *scores, int64_t score_str
 {
     const int lo = kClasses[c].lo, hi = kClasses[c].hi;
     const unsigned n = (unsigned)n_rows;
+    const size_t stage = p.k <= kStageOut ? (size_t)p.k * sizeof(int) : 0;   // the register kernels stage their output row
 #ifdef HS2_TOPK_NO_CLUSTER
     if (c >= 2 && c <= 4) c = 5;   // tuning builds: long rows on the streaming kernel
 #endif
     switch (c) {
-        case 0: k_topk_cached<256, 32, VEC, SEL_ROW><<<n, 256, 0, st>>>(p, scores, score_stride, idx, row0, lo, hi, SelArgs{}); break;
-        case 1: k_topk_cached<512, 64, VEC, SEL_ROW><<<n, 512, 0, st>>>(p, scores, score_stride, idx, row0, lo, hi, SelArgs{}); break;
+        case 0: k_topk_cached<256, 32, VEC, SEL_ROW><<<n, 256, stage, st>>>(p, scores, score_stride, idx, row0, lo, hi, SelArgs{}); break;
+        case 1: k_topk_cached<512, 64, VEC, SEL_ROW><<<n, 512, stage, st>>>(p, scores, score_stride, idx, row0, lo, hi, SelArgs{}); break;
         case 2: k_topk_cluster<2, VEC><<<n * 2, 512, 0, st>>>(p, scores, score_stride, idx, row0, lo, hi); break;
         case 3: k_topk_cluster<4, VEC><<<n * 4, 512, 0, st>>>(p, scores, score_stride, idx, row0, lo, hi); break;
         case 4: k_topk_cluster<8, VEC><<<n * 8, 512, 0, st>>>(p, scores, score_stride, idx, row0, lo, hi); break;
