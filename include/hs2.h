@@ -206,6 +206,23 @@ hs2_status hs2_sparse_attn_decode_static(const hs2_problem *p, const void *Q, co
                                          const int32_t *idx, const float *sink, void *O, float *LSE,
                                          void *cuda_stream);
 
+/*
+ * Producer of the caches the calls above read (Section 3.2, KV Bridging: K_j = Proj^K_j(H_i), V_j = Proj^V_j(H_i);
+ * several layers fed from one hidden-state source are simply more output columns):  C = H W^T.
+ *   H       in  bf16 [n_tokens, d_model], row stride ldh (elements)
+ *   W       in  bf16 [n_out, d_model], row stride ldw: one row per output feature (a linear layer's weight)
+ *   C       out [n_tokens, n_out] with row stride ldc, so that it can be a cache [.., tokens, n_kv_heads, head_dim]
+ *               or a slice of a fused one.  scales == NULL: bf16 (ldc in elements).  scales != NULL: e4m3 codes
+ *               (ldc in bytes) and
+ *   scales  out float [n_tokens, n_out / 128], packed: one scale per token and group of 128 consecutive columns
+ *               (= one head of dim 128): amax / 448 (1 for an all-zero group); code = value / scale rounded to
+ *               nearest even.  This is the format hs2_sparse_attn_*_fp8kv reads.
+ * d_model % 64 == 0, n_out % 256 == 0, strides multiples of 8 elements (16 bytes for the e4m3 output), 16-byte
+ * aligned pointers; anything else returns HS2_ERR_UNSUPPORTED.  fp32 accumulation; no scratch.
+ */
+hs2_status hs2_kv_project(int64_t n_tokens, int32_t d_model, int32_t n_out, const void *H, int64_t ldh, const void *W,
+                          int64_t ldw, void *C, int64_t ldc, float *scales, void *cuda_stream);
+
 /* Static, never-NULL description of a status. */
 const char *hs2_status_string(hs2_status s);
 

@@ -226,3 +226,14 @@ def select_blocks(scores, pos, kvlen, window: int, k_sel: int, block: int) -> np
         keys = [j for m in sorted(order) for j in range(m * block, min(nk, (m + 1) * block))]
         idx[r, :len(keys)] = keys
     return idx
+
+
+def kv_project(h, w):
+    """KV-cache producer (Section 3.2, KV Bridging: K = Proj^K(H), V = Proj^V(H)): ``H [T, dm] @ W [N, dm]^T`` in fp64 on
+    the exact input values."""
+    def f64(x):
+        a, code = _as_input(x)
+        if code == 1:
+            a = (a.astype(np.uint32) << 16).view(np.float32)
+        return a.astype(np.float64)
+    return f64(h) @ f64(w).T

@@ -24,7 +24,7 @@ HS2_OP_FULL_ATTN_SELECT, HS2_OP_TOPK_SELECT, HS2_OP_SPARSE_ATTN_PREFILL, HS2_OP_
 
 EXPORTS = ["hs2_workspace_bytes", "hs2_full_attn_select", "hs2_topk_select", "hs2_sparse_attn_prefill",
            "hs2_sparse_attn_decode", "hs2_sparse_attn_prefill_gated", "hs2_sparse_attn_decode_gated",
-           "hs2_sparse_attn_prefill_fp8kv", "hs2_sparse_attn_decode_fp8kv",
+           "hs2_sparse_attn_prefill_fp8kv", "hs2_sparse_attn_decode_fp8kv", "hs2_kv_project",
            "hs2_sparse_attn_decode_static", "hs2_status_string", "hs2_last_cuda_error",
            "hs2_launch_count", "hs2_device_error_flags", "hs2_set_filter_min_keys", "hs2_set_tcgen05_enabled"]
 
@@ -73,6 +73,8 @@ def load_library():
         lib.hs2_sparse_attn_decode_static.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp]
         lib.hs2_sparse_attn_prefill_gated.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         lib.hs2_sparse_attn_decode_gated.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        lib.hs2_kv_project.argtypes = [C.c_int64, C.c_int32, C.c_int32, vp, C.c_int64, vp, C.c_int64, vp, C.c_int64, vp, vp]
+        lib.hs2_kv_project.restype = C.c_int
         lib.hs2_sparse_attn_prefill_fp8kv.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         lib.hs2_sparse_attn_decode_fp8kv.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         for f in ("hs2_full_attn_select", "hs2_topk_select", "hs2_sparse_attn_prefill", "hs2_sparse_attn_decode",
@@ -299,6 +301,26 @@ def hs2_sparse_attn_decode_fp8kv(prob: Problem, q, k8, v8, k_scale, v_scale, idx
     """SA layer, decode (q_len == 1), on an e4m3 cache."""
     return _sparse_fp8("hs2_sparse_attn_decode_fp8kv", prob, q, k8, v8, k_scale, v_scale, idx, sink, out, lse, want_lse,
                        stream)
+
+
+def hs2_kv_project(h, w, *, out=None, fp8=False, scales=None, stream=None):
+    """Cache producer: ``out[T, N] = h[T, dm] @ w[N, dm].T`` (bf16), or with ``fp8=True`` e4m3 codes (uint8) plus one
+    fp32 scale per (token, 128 columns).  ``out`` may be a strided 2-D view (e.g. a slice of a fused cache).
+    Returns ``out`` or ``(out, scales)``."""
+    assert h.is_cuda and w.is_cuda and h.dtype == torch.bfloat16 and w.dtype == torch.bfloat16
+    assert h.dim() == 2 and w.dim() == 2 and h.shape[1] == w.shape[1] and h.stride(1) == 1 and w.stride(1) == 1
+    T, dm = h.shape
+    N = w.shape[0]
+    if out is None:
+        out = torch.empty(T, N, dtype=torch.uint8 if fp8 else torch.bfloat16, device=h.device)
+    assert out.dim() == 2 and tuple(out.shape) == (T, N) and out.stride(1) == 1
+    assert out.dtype == (torch.uint8 if fp8 else torch.bfloat16)
+    if fp8 and scales is None:
+        scales = torch.empty(T, N // 128, dtype=torch.float32, device=h.device)
+    st = load_library().hs2_kv_project(T, dm, N, _dp(h), h.stride(0), _dp(w), w.stride(0), _dp(out), out.stride(0),
+                                       _dp(scales) if fp8 else None, _stream(stream))
+    _check(st, "hs2_kv_project")
+    return (out, scales) if fp8 else out
 
 
 def hs2_sparse_attn_decode_static(prob: Problem, q, k, v, idx, *, sink=None, out, lse=None, stream=None):

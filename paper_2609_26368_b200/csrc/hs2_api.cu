@@ -452,6 +452,23 @@ hs2_status hs2_sparse_attn_decode_fp8kv(const hs2_problem *hp, const void *Q, co
     return sparse_fp8_impl(hp, true, Q, K8, V8, k_scale, v_scale, idx, sink, O, LSE, cuda_stream);
 }
 
+hs2_status hs2_kv_project(int64_t n_tokens, int32_t d_model, int32_t n_out, const void *H, int64_t ldh, const void *W,
+                          int64_t ldw, void *C, int64_t ldc, float *scales, void *cuda_stream)
+{
+    if (n_tokens < 0 || d_model <= 0 || n_out <= 0 || !H || !W || !C) return HS2_ERR_INVALID_ARG;
+    if (n_tokens == 0) return HS2_OK;
+    if (!kv_project_supported(n_tokens, n_out, d_model, ldh, ldw, ldc, scales != nullptr) || !aligned16(H, W, C, C))
+        return HS2_ERR_UNSUPPORTED;
+    hs2_status s = check_device();
+    if (s != HS2_OK) return s;
+    const cudaError_t e = launch_kv_project(n_tokens, n_out, d_model, H, ldh, W, ldw, C, ldc, scales, (cudaStream_t)cuda_stream);
+    if (e == cudaErrorNotSupported) {
+        (void)cudaGetLastError();
+        return HS2_ERR_UNSUPPORTED;
+    }
+    return e == cudaSuccess ? HS2_OK : cuda_fail(e);
+}
+
 hs2_status hs2_sparse_attn_decode_static(const hs2_problem *hp, const void *Q, const void *K, const void *V,
                                          const int32_t *idx, const float *sink, void *O, float *LSE,
                                          void *cuda_stream)
@@ -485,11 +502,12 @@ int hs2_last_cuda_error(void) { return g_last_cuda_error; }
 int hs2_device_error_flags(unsigned *flags)
 {
     if (!flags) return HS2_ERR_INVALID_ARG;
-    unsigned a = 0, b = 0, c = 0;
+    unsigned a = 0, b = 0, c = 0, d = 0;
     cudaError_t e = read_tc5_error(&a);
     if (e == cudaSuccess) e = read_sparse_error(&b);
     if (e == cudaSuccess) e = read_sparse_tc5_error(&c);
-    *flags = a | (b << 8) | (c << 16);   // bits 8.. : the mma.sync sparse kernels, bits 16.. : the tcgen05 sparse kernel
+    if (e == cudaSuccess) e = read_kvproj_error(&d);
+    *flags = a | (b << 8) | (c << 16) | (d << 24);   // bits 8.. : the mma.sync sparse kernels, bits 16.. : the tcgen05 sparse kernel, bits 24.. : the KV projection
     return e == cudaSuccess ? HS2_OK : cuda_fail(e);
 }
 

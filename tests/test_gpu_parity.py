@@ -422,6 +422,51 @@ def test_block_level_selection_variant():
     assert_output_close(out.reshape(-1, wl.n_q_heads, wl.head_dim), Oo, wl.torch_dtype, "sparse O on block indices")
 
 
+def test_kv_projection_bf16_and_fp8_outputs():
+    """The cache producer C = H W^T (Section 3.2, KV Bridging) against the fp64 product: bf16 output into a slice of a
+    fused cache, and e4m3 codes + scales within the format's rounding bound; the FP8 caches it writes are then read
+    by the FP8 sparse kernel."""
+    g = torch.Generator(device="cuda").manual_seed(4)
+    T, dm, Hkv, D = 300, 320, 2, 128
+    N = 2 * Hkv * D                                         # K and V of one layer side by side
+    h = (torch.randn(T, dm, device="cuda", generator=g)).to(torch.bfloat16)
+    w = (torch.randn(N, dm, device="cuda", generator=g) / dm ** 0.5).to(torch.bfloat16)
+    want = oracle.kv_project(h.cpu(), w.cpu())
+    fused = torch.zeros(T, N + 64, dtype=torch.bfloat16, device="cuda")      # a wider row: strided output
+    out = hs2.hs2_kv_project(h, w, out=fused[:, :N])
+    torch.cuda.synchronize()
+    got = out.float().cpu().numpy().astype(np.float64)
+    assert np.all(np.abs(got - want) <= np.abs(want) * 2.0 ** -8 + 1e-5)
+    assert torch.count_nonzero(fused[:, N:]) == 0
+    c8, sc = hs2.hs2_kv_project(h, w, fp8=True)
+    torch.cuda.synchronize()
+    amax = np.abs(want).reshape(T, N // 128, 128).max(axis=2)
+    s_np = sc.cpu().numpy().astype(np.float64)
+    assert np.all(np.abs(s_np - amax / 448.0) <= 1e-4 * amax / 448.0 + 1e-12)
+    deq = oracle.dequant_e4m3(c8.cpu().numpy().reshape(T, N // 128, 128), s_np).astype(np.float64).reshape(T, N)
+    assert not np.isnan(deq).any()
+    s_full = np.repeat(s_np, 128, axis=1)
+    bound = np.maximum(np.abs(want) * 2.0 ** -4, s_full * 2.0 ** -10) * 1.01 + 1e-5
+    assert np.all(np.abs(deq - want) <= bound)
+    # the produced FP8 caches through the FP8 sparse kernel: [1, T, Hkv, D] K and V are column halves of the output
+    k8, v8 = c8[:, :Hkv * D].reshape(1, T, Hkv, D), c8[:, Hkv * D:].reshape(1, T, Hkv, D)
+    ksc, vsc = sc[:, :Hkv].reshape(1, T, Hkv).contiguous(), sc[:, Hkv:].reshape(1, T, Hkv).contiguous()
+    Lq, k_sel, win = 40, 32, 8
+    q = torch.randn(1, Lq, 8 * Hkv, D, device="cuda", generator=g).to(torch.bfloat16)
+    idx = torch.stack([torch.sort(torch.randperm(T - Lq - win, device="cuda", generator=g)[:k_sel]).values
+                       for _ in range(Hkv * Lq)]).to(torch.int32).reshape(1, Hkv, Lq, k_sel).contiguous()
+    prob = hs2.Problem.from_tensors(q, k8, k_sel, win)
+    o8, _ = hs2.hs2_sparse_attn_prefill_fp8kv(prob, q, k8, v8, ksc, vsc, idx)
+    torch.cuda.synchronize()
+    kd = oracle.dequant_e4m3(k8.contiguous(), ksc)
+    vd = oracle.dequant_e4m3(v8.contiguous(), vsc)
+    Oo, _, _ = oracle.sparse_attn(q.float().cpu().numpy(), kd, vd, idx.permute(0, 2, 1, 3).reshape(Lq, Hkv, k_sel).cpu().numpy(), win)
+    assert_output_close(o8.reshape(-1, 8 * Hkv, D), Oo, torch.bfloat16, "sparse O on the projected FP8 cache")
+    with pytest.raises(hs2.HS2Error):                       # n_out must be a multiple of 256
+        hs2.hs2_kv_project(h, w[:128])
+    assert hs2.hs2_device_error_flags() == 0
+
+
 def test_ragged_lengths_offsets_strides_and_sink():
     wl = scaled("cfg2", batch=3, q_len=70, kv_len=400, k_sel=40, window=12, n_needles=4)
     inp = make_inputs(wl)

@@ -412,3 +412,14 @@ def test_block_level_selection_reduces_to_token_level_and_matches_brute_force():
             want = [j for m in sorted(kept) for j in range(m * B, min(nk, (m + 1) * B))]
             got = [j for j in idx[r] if j >= 0]
             assert got == want and all(j == -1 for j in idx[r, len(got):])
+
+
+def test_kv_projection_is_the_plain_sum_of_products():
+    g = torch.Generator().manual_seed(2)
+    h = torch.randn(5, 7, generator=g).to(torch.bfloat16)
+    w = torch.randn(3, 7, generator=g).to(torch.bfloat16)
+    c = oracle.kv_project(h, w)
+    for t in range(5):
+        for n in range(3):
+            want = sum(float(h[t, d]) * float(w[n, d]) for d in range(7))
+            assert abs(c[t, n] - want) < 1e-12
