@@ -458,6 +458,41 @@ def bench_native(device, peaks, reps=5):
     return out
 
 
+def bench_kv_project(device, peaks, reps=7):
+    """The cache producer (Section 3.2, KV Bridging): C = H W^T for the paper's hidden size 2048 and four layers' K and V
+    projections (2048 output columns) over 32768 tokens; bf16 output and the quantising e4m3 output."""
+    import paper_2609_26368_b200 as hs2
+    T, dm, N = 32768, 2048, 2048
+    h = torch.randn(T, dm, device=device).to(torch.bfloat16)
+    w = (torch.randn(N, dm, device=device) / dm ** 0.5).to(torch.bfloat16)
+    out = torch.empty(T, N, dtype=torch.bfloat16, device=device)
+    o8 = torch.empty(T, N, dtype=torch.uint8, device=device)
+    sc = torch.empty(T, N // 128, dtype=torch.float32, device=device)
+
+    def med(fn):
+        for _ in range(3):
+            fn()
+        torch.cuda.synchronize()
+        ts = []
+        for _ in range(reps):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            fn()
+            b.record()
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b))
+        return statistics.median(ts)
+    fl = 2.0 * T * dm * N
+    t16 = med(lambda: hs2.hs2_kv_project(h, w, out=out))
+    t8 = med(lambda: hs2.hs2_kv_project(h, w, out=o8, fp8=True, scales=sc))
+    peak = peaks.get("bf16_tflops", peaks["bf16_tflops_sustained"])
+    return {"workload": "T=32768 tokens, d_model 2048, 2048 output columns, bf16 in, fp32 accumulate",
+            "bf16_out_us": round(t16 * 1e3, 1), "bf16_out_tflops": round(fl / t16 / 1e9, 1),
+            "e4m3_out_us": round(t8 * 1e3, 1), "e4m3_out_tflops": round(fl / t8 / 1e9, 1),
+            "peak_tflops_burst": peak, "frac_bf16_out": round(fl / t16 / 1e9 / peak, 4),
+            "frac_e4m3_out": round(fl / t8 / 1e9 / peak, 4), "l2": "A, B and C are 134 + 8 + 134 MB: larger than L2"}
+
+
 # ------------------------------------------------------------------ CPU oracle legs
 
 def oracle_sample_step(wl, inp_host, rows):
@@ -528,7 +563,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="cfg2", choices=sorted(CONFIGS))
     ap.add_argument("--cpu-rows", type=int, default=4096, help="query rows of the CPU-oracle sample (about 15 s of CPU work on cfg2)")
-    ap.add_argument("--skip", default="", help="comma list of: block, decode64k, native, e2e, cpu")
+    ap.add_argument("--skip", default="", help="comma list of: block, decode64k, native, kvproj, e2e, cpu")
     ap.add_argument("--decode-ctx", type=int, default=65536, help="context length of the decode section (profiling: 8192)")
     args = ap.parse_args()
     wl = CONFIGS[args.workload]
@@ -551,6 +586,8 @@ def main():
             side["decode_64k"] = bench_decode_64k(device, peaks, ctx=args.decode_ctx)
         if "native" not in skip:
             side["paper_native_shape"] = bench_native(device, peaks)
+        if "kvproj" not in skip:
+            side["kv_project"] = bench_kv_project(device, peaks)
         print(json.dumps(side))
         return
     block = Block(wl, device, rank)
@@ -619,6 +656,9 @@ def main():
     if "native" not in skip and world == 1:
         torch.cuda.empty_cache()
         line["paper_native_shape"] = bench_native(device, peaks)
+    if "kvproj" not in skip and world == 1:
+        torch.cuda.empty_cache()
+        line["kv_project"] = bench_kv_project(device, peaks)
     if "cpu" not in skip and world == 1:
         cb, _, _ = cpu_baseline(wl, args.cpu_rows)
         line["cpu_baseline"] = cb
