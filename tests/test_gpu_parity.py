@@ -467,6 +467,28 @@ def test_kv_projection_bf16_and_fp8_outputs():
     assert hs2.hs2_device_error_flags() == 0
 
 
+def test_union_mode_selection_is_the_full_layer_with_window_zero():
+    """The alternative reading of the budget (k counted over all visible tokens, window included): select with
+    window 0, attend with window w.  Selected tokens that fall inside the window are ignored by the sparse kernels
+    (they are covered by the window slots), exactly as the oracle's set semantics say."""
+    wl = scaled("cfg2", q_len=200, kv_len=500, k_sel=64, window=24, n_needles=8)
+    inp = make_inputs(wl, "cuda")
+    prob_sel = hs2.Problem.from_tensors(inp.q_full, inp.k, wl.k_sel, 0)
+    prob_att = hs2.Problem.from_tensors(inp.q_full, inp.k, wl.k_sel, wl.window)
+    _, _, idx, scores = hs2.hs2_full_attn_select(prob_sel, inp.q_full, inp.k, inp.v, want_scores=True)
+    out, _ = hs2.hs2_sparse_attn_prefill(prob_att, inp.q_sparse[0], inp.k, inp.v, idx)
+    torch.cuda.synchronize()
+    pos = wl.kv_len - wl.q_len + np.arange(wl.q_len)
+    for g in range(wl.n_kv_heads):       # bit-exact on the GPU's own scores, window 0: every visible key is a candidate
+        assert np.array_equal(idx[0, g].cpu().numpy(), oracle.select(scores[0, g].cpu().numpy(), pos, wl.kv_len, 0, wl.k_sel))
+    assert (idx[0, :, -1] > wl.kv_len - 1 - wl.window).any()      # some selected tokens do sit inside the window
+    idx_rows = idx.permute(0, 2, 1, 3).reshape(wl.q_len, wl.n_kv_heads, wl.k_sel).cpu().numpy()
+    Oo, _, member = oracle.sparse_attn(to_host(inp.q_sparse[0]), to_host(inp.k), to_host(inp.v), idx_rows, wl.window,
+                                       want_member=True)
+    assert_output_close(out.reshape(-1, wl.n_q_heads, wl.head_dim), Oo, wl.torch_dtype, "union-mode sparse O")
+    assert member.sum(axis=2).max() <= wl.k_sel + wl.window
+
+
 def test_ragged_lengths_offsets_strides_and_sink():
     wl = scaled("cfg2", batch=3, q_len=70, kv_len=400, k_sel=40, window=12, n_needles=4)
     inp = make_inputs(wl)
