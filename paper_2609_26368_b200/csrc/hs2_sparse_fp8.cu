@@ -28,6 +28,9 @@
 #ifndef HS2_F8D_WARPS
 #define HS2_F8D_WARPS 8
 #endif
+#ifndef HS2_F8D_MINB
+#define HS2_F8D_MINB 1
+#endif
 
 namespace hs2 {
 namespace {
@@ -395,7 +398,7 @@ k_sparse_fp8_prefill(const Params p, const __nv_bfloat16 *__restrict__ Q, const 
 }
 
 // ---------------------------------------------------------------- decode: one CTA per (sequence, KV head)
-__global__ void __launch_bounds__(HS2_F8D_WARPS * 32)
+__global__ void __launch_bounds__(HS2_F8D_WARPS * 32, HS2_F8D_MINB)
 k_sparse_fp8_decode(const Params p, const __nv_bfloat16 *__restrict__ Q, const uint8_t *__restrict__ K,
                     const uint8_t *__restrict__ V, const float *__restrict__ ksc, const float *__restrict__ vsc,
                     const int32_t *__restrict__ idx, const float *__restrict__ sink, __nv_bfloat16 *__restrict__ O,
