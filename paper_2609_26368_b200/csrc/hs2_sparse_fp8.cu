@@ -29,7 +29,7 @@
 #define HS2_F8D_WARPS 8
 #endif
 #ifndef HS2_F8D_MINB
-#define HS2_F8D_MINB 1
+#define HS2_F8D_MINB 2
 #endif
 
 namespace hs2 {
