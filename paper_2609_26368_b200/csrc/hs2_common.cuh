@@ -21,6 +21,8 @@ struct Params {
     int64_t qs_b, qs_t, qs_h;   // element strides
     int64_t ks_b, ks_t, ks_h;
     int64_t os_b, os_t, os_h;
+    int share;          // > 1: consecutive groups of `share` KV-head slots are one real KV head seen through sub-groups
+                        // of its query heads (K, V and idx are indexed by slot / share); 0 or 1: plain
     int blk;            // selection granularity: 1 = tokens, B > 1 = aligned blocks of B tokens
     const void *gate;   // optional output-gate logits of the sparse layers: shape, dtype and strides of O; null = no gate
 };

@@ -706,6 +706,7 @@ cudaError_t launch_sc_mode(const Params &p, const void *Q, const void *K, const 
         return cudaErrorNotSupported;
     if ((n_rows + p.Lq) / (128 / p.G) + 2 * (int64_t)p.B * p.Hkv > 65535) return cudaErrorNotSupported;   // grid.y bound
     constexpr int M2 = MODE == SC_FILTER ? SC_STRIP : MODE;   // groups of 1 or 2 have no filter instantiation
+    constexpr int M3 = SC_STRIP;                              // large groups and head_dim 256: strips only
 #define HS2_SC(G_, MODE_, D_) return launch_sc<G_, MODE_, D_>(tmQ, tmK, p, LSE, out, out_stride, row0, n_rows, all_visible, samp, fb, st)
     if (p.D == 128) {
         switch (p.G) {
@@ -714,12 +715,18 @@ cudaError_t launch_sc_mode(const Params &p, const void *Q, const void *K, const 
             case 4: HS2_SC(4, MODE, 128);
             case 8: HS2_SC(8, MODE, 128);
             case 16: HS2_SC(16, MODE, 128);
+            case 32: if (MODE != SC_STRIP) return cudaErrorNotSupported; HS2_SC(32, M3, 128);
+            case 64: if (MODE != SC_STRIP) return cudaErrorNotSupported; HS2_SC(64, M3, 128);
+            case 128: if (MODE != SC_STRIP) return cudaErrorNotSupported; HS2_SC(128, M3, 128);
         }
     } else if (p.D == 256) {
         if (MODE != SC_STRIP) return cudaErrorNotSupported;
         switch (p.G) {
-            case 8: HS2_SC(8, M2, 256);
-            case 64: HS2_SC(64, M2, 256);
+            case 8: HS2_SC(8, M3, 256);
+            case 16: HS2_SC(16, M3, 256);
+            case 32: HS2_SC(32, M3, 256);
+            case 64: HS2_SC(64, M3, 256);
+            case 128: HS2_SC(128, M3, 256);
         }
     }
 #undef HS2_SC
@@ -728,8 +735,8 @@ cudaError_t launch_sc_mode(const Params &p, const void *Q, const void *K, const 
 
 bool scores_tc5_supported(const Params &p, hs2_dtype dt)
 {
-    if (p.D == 256) return (p.G == 8 || p.G == 64) && full_attn_tc5_supported(p, dt);
-    const bool g_ok = p.G == 1 || p.G == 2 || p.G == 4 || p.G == 8 || p.G == 16;
+    if (p.D == 256) return (p.G == 8 || p.G == 16 || p.G == 32 || p.G == 64 || p.G == 128) && full_attn_tc5_supported(p, dt);
+    const bool g_ok = p.G == 1 || p.G == 2 || p.G == 4 || p.G == 8 || p.G == 16 || p.G == 32 || p.G == 64 || p.G == 128;
     return g_ok && full_tc5_supported(p, dt);
 }
 

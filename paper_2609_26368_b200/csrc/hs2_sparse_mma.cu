@@ -455,11 +455,14 @@ __device__ __forceinline__ Item make_item(const Params &p, const __nv_bfloat16 *
                                           const int32_t *idx, int b, int gkv, int i)
 {
     Item it;
-    const int64_t base = b * p.ks_b + gkv * p.ks_h;
+    // a group of 16 query heads runs as two sub-groups of 8: slot gkv of p.Hkv slots reads real KV head gkv / share
+    const int share = p.share > 1 ? p.share : 1;
+    const int g_real = gkv / share, hkv_real = p.Hkv / share;
+    const int64_t base = b * p.ks_b + g_real * p.ks_h;
     it.Kb = reinterpret_cast<const char *>(K + base);
     it.Vb = reinterpret_cast<const char *>(V + base);
     it.row_stride = p.ks_t * 2;
-    it.irow = idx ? idx + (((int64_t)b * p.Hkv + gkv) * p.Lq + i) * p.k : nullptr;
+    it.irow = idx ? idx + (((int64_t)b * hkv_real + g_real) * p.Lq + i) * p.k : nullptr;
     it.pos = pos_of(p, b, i);
     it.kvl = kvlen_of(p, b);
     return it;

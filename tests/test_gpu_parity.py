@@ -144,6 +144,8 @@ SMALL = [
     ("cfg2", dict(q_len=200, kv_len=200, k_sel=40, window=0, n_needles=4)),              # no window
     ("cfg2", dict(q_len=150, kv_len=150, k_sel=16, window=4, n_q_heads=4, n_kv_heads=4, n_needles=4)),   # group of 1
     ("cfg2", dict(q_len=150, kv_len=150, k_sel=16, window=4, n_q_heads=16, n_kv_heads=1, n_needles=4)),  # MQA 16
+    ("cfg2", dict(q_len=130, kv_len=420, k_sel=48, window=10, n_q_heads=48, n_kv_heads=3, n_needles=4, batch=2)),  # groups of 16
+    ("cfg2", dict(q_len=90, kv_len=300, k_sel=32, window=8, n_q_heads=64, n_kv_heads=2, n_needles=4)),   # groups of 32
     ("cfg2", dict(q_len=300, kv_len=300, k_sel=64, window=16, n_q_heads=16, n_kv_heads=2, head_dim=256, n_needles=8)),
     ("cfg2", dict(q_len=260, kv_len=700, k_sel=64, window=16, n_q_heads=64, n_kv_heads=1, head_dim=256, n_needles=8)),  # paper's shape
 ]
@@ -336,6 +338,7 @@ def test_fp8_kv_cache_sparse_prefill_and_decode():
         dict(q_len=150, kv_len=600, k_sel=100, window=24, batch=2),
         dict(q_len=64, kv_len=300, k_sel=37, window=5, n_q_heads=8, n_kv_heads=2),
         dict(q_len=40, kv_len=200, k_sel=0, window=50, n_q_heads=4, n_kv_heads=4),
+        dict(q_len=48, kv_len=260, k_sel=40, window=12, n_q_heads=32, n_kv_heads=2),     # groups of 16: two sub-groups of 8
     ]
     for ci, over in enumerate(cases):
         wl = scaled("cfg2", n_needles=4, **over)
@@ -374,7 +377,7 @@ def test_fp8_kv_cache_sparse_prefill_and_decode():
             assert (od.float() - out[:, -1:].float()).abs().max().item() <= 2e-2
             assert (ld - lse[:, :, -1:]).abs().max().item() <= 2e-3
     # shapes the FP8 kernels do not cover are refused, not mis-computed
-    wl = scaled("cfg2", q_len=16, kv_len=64, k_sel=8, window=4, n_q_heads=16, n_kv_heads=1, n_needles=4)
+    wl = scaled("cfg2", q_len=16, kv_len=64, k_sel=8, window=4, n_q_heads=24, n_kv_heads=1, n_needles=4)
     inp = make_inputs(wl, "cuda")
     k8, ksc = quantize_kv_e4m3(inp.k)
     prob = hs2.Problem.from_tensors(inp.q_full, k8, wl.k_sel, wl.window)
@@ -555,8 +558,9 @@ def test_malformed_indices_cannot_read_out_of_bounds():
 
 # ---------------------------------------------------------------- decode
 
-def test_decode_small_matches_oracle_and_prefill_last_row():
-    wl = scaled("cfg5", batch=5, kv_len=3000, k_sel=256, window=32, n_needles=8)
+@pytest.mark.parametrize("heads", [(32, 4), (64, 4)])      # groups of 8, and of 16 (two sub-groups of 8)
+def test_decode_small_matches_oracle_and_prefill_last_row(heads):
+    wl = scaled("cfg5", batch=5, kv_len=3000, k_sel=256, window=32, n_needles=8, n_q_heads=heads[0], n_kv_heads=heads[1])
     run = BlockRun(make_inputs(wl)).run_full(want_scores=True)
     run.check_full(check_scores=True)
     run.check_idx_bitexact_on_gpu_scores()
