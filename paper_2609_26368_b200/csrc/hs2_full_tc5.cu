@@ -411,7 +411,9 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         const int t = tid / G, hh = tid % G;
         const int i = iq0 + t;
         const bool ok = i >= c_lo && i < c_hi;
-        s_nl[tid] = ok ? -LSE[((int64_t)b * p.Hq + gkv * G + hh) * p.Lq + i] / p.scale : 0.f;
+        // G is the group size rounded up to a tile-able one; columns past the real group hold some other head's
+        // (or zero-filled) scores and are taken out of the maximum by -inf
+        s_nl[tid] = !ok ? 0.f : hh < p.G ? -LSE[((int64_t)b * p.Hq + gkv * p.G + hh) * p.Lq + i] / p.scale : -INFINITY;
         if (hh == 0) {
             s_nq[t] = ok ? n_of(i) : 0;
             s_row[t] = ok ? (bg_row0 + i - row0) : -1;
@@ -443,7 +445,7 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         if (elect_one()) {
             mbar_expect_tx(bar(SQ_FULL), kStage);
 #pragma unroll
-            for (int sl = 0; sl < NQ; ++sl) tma_load_4d(sbase + kScOffQ + sl * S::kSlice, &tmQ, bar(SQ_FULL), 64 * sl, gkv * G, iq0, b);
+            for (int sl = 0; sl < NQ; ++sl) tma_load_4d(sbase + kScOffQ + sl * S::kSlice, &tmQ, bar(SQ_FULL), 64 * sl, gkv * p.G, iq0, b);
             int issued = 0;
             for (int t = 0; t < ntile; ++t) {
                 const int st = t & 1;
@@ -695,21 +697,34 @@ cudaError_t launch_sc(const CUtensorMap &tmQ, const CUtensorMap &tmK, const Para
     return cudaGetLastError();
 }
 
+// smallest instantiated group size >= g (powers of two up to 128), 0 if there is none
+int padded_group(int g, int D)
+{
+    if (D != 128 && D != 256) return 0;
+    for (int c = 1; c <= 128; c *= 2)
+        if (c >= g) return c;
+    return 0;
+}
+
 template <int MODE>
 cudaError_t launch_sc_mode(const Params &p, const void *Q, const void *K, const float *LSE, float *out, int64_t out_stride,
                            int64_t row0, int64_t n_rows, bool all_visible, int samp, const FilterBuf &fb, cudaStream_t st)
 {
     if (n_rows == 0) return cudaSuccess;
     CUtensorMap tmQ, tmK;
-    if (!make_map(&tmQ, Q, p.B, p.Lq, p.Hq, p.qs_b, p.qs_t, p.qs_h, 128 / p.G, p.G, p.D) ||
+    // the kernel is instantiated for groups that tile its 128 columns; any other size runs as the next one up
+    // with the surplus columns masked (the sampled and filtered sweeps exist for exact sizes only)
+    const int gp = padded_group(p.G, p.D);
+    if (gp == 0 || (gp != p.G && MODE != SC_STRIP)) return cudaErrorNotSupported;
+    if (!make_map(&tmQ, Q, p.B, p.Lq, p.Hq, p.qs_b, p.qs_t, p.qs_h, 128 / gp, gp, p.D) ||
         !make_map(&tmK, K, p.B, p.Lk, p.Hkv, p.ks_b, p.ks_t, p.ks_h, 128, 1, p.D))
         return cudaErrorNotSupported;
-    if ((n_rows + p.Lq) / (128 / p.G) + 2 * (int64_t)p.B * p.Hkv > 65535) return cudaErrorNotSupported;   // grid.y bound
+    if ((n_rows + p.Lq) / (128 / gp) + 2 * (int64_t)p.B * p.Hkv > 65535) return cudaErrorNotSupported;   // grid.y bound
     constexpr int M2 = MODE == SC_FILTER ? SC_STRIP : MODE;   // groups of 1 or 2 have no filter instantiation
     constexpr int M3 = SC_STRIP;                              // large groups and head_dim 256: strips only
 #define HS2_SC(G_, MODE_, D_) return launch_sc<G_, MODE_, D_>(tmQ, tmK, p, LSE, out, out_stride, row0, n_rows, all_visible, samp, fb, st)
     if (p.D == 128) {
-        switch (p.G) {
+        switch (gp) {
             case 1: if (MODE == SC_FILTER) return cudaErrorNotSupported; HS2_SC(1, M2, 128);
             case 2: if (MODE == SC_FILTER) return cudaErrorNotSupported; HS2_SC(2, M2, 128);
             case 4: HS2_SC(4, MODE, 128);
@@ -721,7 +736,10 @@ cudaError_t launch_sc_mode(const Params &p, const void *Q, const void *K, const 
         }
     } else if (p.D == 256) {
         if (MODE != SC_STRIP) return cudaErrorNotSupported;
-        switch (p.G) {
+        switch (gp) {
+            case 1: HS2_SC(1, M3, 256);
+            case 2: HS2_SC(2, M3, 256);
+            case 4: HS2_SC(4, M3, 256);
             case 8: HS2_SC(8, M3, 256);
             case 16: HS2_SC(16, M3, 256);
             case 32: HS2_SC(32, M3, 256);
@@ -735,9 +753,8 @@ cudaError_t launch_sc_mode(const Params &p, const void *Q, const void *K, const 
 
 bool scores_tc5_supported(const Params &p, hs2_dtype dt)
 {
-    if (p.D == 256) return (p.G == 8 || p.G == 16 || p.G == 32 || p.G == 64 || p.G == 128) && full_attn_tc5_supported(p, dt);
-    const bool g_ok = p.G == 1 || p.G == 2 || p.G == 4 || p.G == 8 || p.G == 16 || p.G == 32 || p.G == 64 || p.G == 128;
-    return g_ok && full_tc5_supported(p, dt);
+    if (padded_group(p.G, p.D) == 0) return false;
+    return p.D == 256 ? full_attn_tc5_supported(p, dt) : full_tc5_supported(p, dt);
 }
 
 // shape test only (no driver query): workspace sizes must not depend on the machine

@@ -628,12 +628,13 @@ cudaError_t launch_sp(const Params &p, const void *Q, const void *K, const void 
 
 }  // namespace
 
-// bf16, head_dim 128 or 256, more than 8 and at most 128 query heads per KV head
+// bf16; head_dim 256 with up to 128 query heads per KV head, head_dim 128 with 9 to 128
 bool sparse_tc5_supported_shape(const Params &p, hs2_dtype dt)
 {
     auto m8 = [](int64_t x) { return x % 8 == 0 && x > 0; };
     if (p.ks_t * 2 > 0x7fffffffLL) return false;
-    return dt == HS2_BF16 && (p.D == 128 || p.D == 256) && p.G > 8 && p.G <= 128 && m8(p.qs_b) && m8(p.qs_t) && m8(p.qs_h) &&
+    // at head_dim 128 groups of up to 8 belong to the mma.sync gather kernel; at 256 this is the only tensor-core one
+    return dt == HS2_BF16 && (p.D == 256 || (p.D == 128 && p.G > 8)) && p.G >= 1 && p.G <= 128 && m8(p.qs_b) && m8(p.qs_t) && m8(p.qs_h) &&
            m8(p.ks_b) && m8(p.ks_t) && m8(p.ks_h) && m8(p.os_b) && m8(p.os_t) && m8(p.os_h) &&
            (int64_t)p.B * p.Hkv * p.Lq * 2 * kMaxSplits <= 0x7fffffffLL && p.k + p.w > 0;
 }

@@ -146,6 +146,10 @@ SMALL = [
     ("cfg2", dict(q_len=150, kv_len=150, k_sel=16, window=4, n_q_heads=16, n_kv_heads=1, n_needles=4)),  # MQA 16
     ("cfg2", dict(q_len=130, kv_len=420, k_sel=48, window=10, n_q_heads=48, n_kv_heads=3, n_needles=4, batch=2)),  # groups of 16
     ("cfg2", dict(q_len=90, kv_len=300, k_sel=32, window=8, n_q_heads=64, n_kv_heads=2, n_needles=4)),   # groups of 32
+    ("cfg2", dict(q_len=140, kv_len=380, k_sel=40, window=12, n_q_heads=24, n_kv_heads=2, n_needles=4)),  # groups of 12 (padded to 16)
+    ("cfg2", dict(q_len=100, kv_len=330, k_sel=40, window=12, n_q_heads=6, n_kv_heads=2, head_dim=256, n_needles=4)),  # groups of 3, dim 256
+    ("cfg2", dict(q_len=100, kv_len=330, k_sel=40, window=12, n_q_heads=3, n_kv_heads=3, head_dim=256, n_needles=4)),  # groups of 1, dim 256
+    ("cfg2", dict(q_len=70, kv_len=280, k_sel=40, window=12, n_q_heads=48, n_kv_heads=1, head_dim=256, n_needles=4)),  # group of 48, dim 256
     ("cfg2", dict(q_len=300, kv_len=300, k_sel=64, window=16, n_q_heads=16, n_kv_heads=2, head_dim=256, n_needles=8)),
     ("cfg2", dict(q_len=260, kv_len=700, k_sel=64, window=16, n_q_heads=64, n_kv_heads=1, head_dim=256, n_needles=8)),  # paper's shape
 ]
