@@ -8,9 +8,11 @@
 //   sparse layers - e4m3 codes plus one fp32 scale per (token, group of 128 columns = one head), quantised in the
 //   epilogue while the accumulator row is still in registers.
 //
-// One CTA = one 128 x 256 output tile: warp 4 feeds H and W tiles by TMA (64 k-columns per stage, 128-byte swizzle),
-// warp 5 issues tcgen05.mma (M128 N256 K16) into 256 TMEM columns, warps 0-3 (thread = output row) run the epilogue.
-// Two CTAs fit an SM, so one CTA's epilogue overlaps the other's main loop.  Every mbarrier wait is bounded.
+// Persistent CTAs (one per SM) walk the 128 x 256 output tiles, n-tiles fastest so that neighbouring CTAs share an H
+// tile in L2: warp 4 feeds H and W tiles by TMA (64 k-columns per stage, 128-byte swizzle, 4-stage ring that runs on
+// across tiles), warp 5 issues tcgen05.mma (M128 N256 K16) into one of two 256-column TMEM accumulators, warps 0-3
+// (thread = output row) run the epilogue of tile i while the tensor core is already on tile i+1.  Every mbarrier
+// wait is bounded.
 #include <cuda.h>
 
 #include "hs2_common.cuh"
@@ -25,9 +27,8 @@ namespace {
 using namespace tc5;
 
 constexpr int BM = 128, BN = 256, BK = 64;
-// TMA stages per CTA.  2 (two CTAs per SM) measured ahead of 4 (one CTA per SM): 221 vs 232 us at 32768 x 2048 x 2048.
 #ifndef HS2_KVP_STAGES
-#define HS2_KVP_STAGES 2
+#define HS2_KVP_STAGES 4
 #endif
 constexpr int kStages = HS2_KVP_STAGES;
 constexpr int kThreads = 192;
@@ -37,7 +38,8 @@ constexpr uint32_t kAlignSlack = 896;
 constexpr uint32_t kSmemBytes = kOffBar + 128 + kAlignSlack;
 constexpr int kQuantGroup = 128;      // columns that share a scale in the FP8 output (one head of dim 128)
 
-enum Bar { FULL0 = 0, EMPTY0 = kStages, ACC_FULL = 2 * kStages, N_BARS };
+enum Bar { FULL0 = 0, EMPTY0 = kStages, ACC_FULL0 = 2 * kStages, ACC_EMPTY0 = 2 * kStages + 2, N_BARS = 2 * kStages + 4 };
+constexpr uint32_t kTmemCols = 2 * BN;   // two accumulators
 
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag)
 {
@@ -52,7 +54,7 @@ __device__ __forceinline__ uint32_t cvt_f32x2_e4m3(float lo, float hi)
 }
 
 template <bool FP8>
-__global__ void __launch_bounds__(kThreads, kStages <= 2 ? 2 : 1)
+__global__ void __launch_bounds__(kThreads, 1)
 k_kv_project(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtensorMap tmW, int64_t T, int N, int dm,
              void *__restrict__ C, int64_t ldc, float *__restrict__ scales)
 {
@@ -71,18 +73,18 @@ k_kv_project(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CU
     auto bar = [&](int i) { return bars + 8u * i; };
 
     const int tid = threadIdx.x, warp = tid >> 5;
-    const int n0 = blockIdx.x * BN;
-    const int64_t m0 = (int64_t)blockIdx.y * BM;
     const int nk = dm / BK;
+    const int tiles_n = N / BN;
+    const int64_t n_tiles = ((T + BM - 1) / BM) * tiles_n;
 
     if (tid == 0) {
         *abort_flag = 0;
         for (int s = 0; s < kStages; ++s) { mbar_init(bar(FULL0 + s), 1); mbar_init(bar(EMPTY0 + s), 1); }
-        mbar_init(bar(ACC_FULL), 1);
+        for (int s = 0; s < 2; ++s) { mbar_init(bar(ACC_FULL0 + s), 1); mbar_init(bar(ACC_EMPTY0 + s), 128); }
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
     if (warp == 5) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(tmem_slot)), "r"((uint32_t)BN) : "memory");
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
     }
     tc_fence_before();
@@ -91,55 +93,75 @@ k_kv_project(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CU
     const uint32_t tmem = *tmem_slot;
 
     if (warp == 4) {
-        // ------------------------------------------------ TMA producer
+        // ------------------------------------------------ TMA producer: the stage ring runs on across tiles
         if (elect_one()) {
-            int issued = 0;
-            for (int kb = 0; kb < nk; ++kb) {
-                const int st = kb % kStages;
-                if (!mbar_wait(bar(EMPTY0 + st), ((kb / kStages) & 1) ^ 1, abort_flag)) break;
-                issued = kb + 1;
-                mbar_expect_tx(bar(FULL0 + st), kStage);
-                // tensors are described as [1, rows, 1, d_model]: coordinates (k, 0, row, 0)
-                tma_load_4d(sbase + st * kStage, &tmH, bar(FULL0 + st), kb * BK, 0, (int)m0, 0);
-                tma_load_4d(sbase + st * kStage + kABytes, &tmW, bar(FULL0 + st), kb * BK, 0, n0, 0);
+            int c = 0, issued = 0;   // k-blocks so far
+            bool ok = true;
+            for (int64_t tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x) {
+                const int n0 = (int)(tile % tiles_n) * BN;
+                const int m0 = (int)(tile / tiles_n) * BM;
+                for (int kb = 0; kb < nk; ++kb, ++c) {
+                    const int st = c % kStages;
+                    if (!mbar_wait(bar(EMPTY0 + st), ((c / kStages) & 1) ^ 1, abort_flag)) { ok = false; break; }
+                    issued = c + 1;
+                    mbar_expect_tx(bar(FULL0 + st), kStage);
+                    // tensors are described as [1, rows, 1, d_model]: coordinates (k, 0, row, 0)
+                    tma_load_4d(sbase + st * kStage, &tmH, bar(FULL0 + st), kb * BK, 0, m0, 0);
+                    tma_load_4d(sbase + st * kStage + kABytes, &tmW, bar(FULL0 + st), kb * BK, 0, n0, 0);
+                }
             }
             if (*abort_flag)   // leaving early: let the copies in flight land before the CTA goes away
-                for (int kb = max(0, issued - kStages); kb < issued; ++kb)
-                    for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait(bar(FULL0 + kb % kStages), (kb / kStages) & 1); ++it) {}
+                for (int k2 = max(0, issued - kStages); k2 < issued; ++k2)
+                    for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait(bar(FULL0 + k2 % kStages), (k2 / kStages) & 1); ++it) {}
         }
     } else if (warp == 5) {
         // ------------------------------------------------ MMA issuer
         if (elect_one()) {
             constexpr uint32_t id = idesc(BM, BN, 0);
             bool ok = true;
-            for (int kb = 0; kb < nk && ok; ++kb) {
-                const int st = kb % kStages;
-                if (!mbar_wait(bar(FULL0 + st), (kb / kStages) & 1, abort_flag)) { ok = false; break; }
+            int c = 0, i = 0;
+            for (int64_t tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++i) {
+                const int ab = i & 1;
+                if (!mbar_wait(bar(ACC_EMPTY0 + ab), ((i >> 1) & 1) ^ 1, abort_flag)) break;   // the epilogue has drained it
                 tc_fence_after();
-                const uint64_t da = smem_desc(sbase + st * kStage, 16, 1024);
-                const uint64_t db = smem_desc(sbase + st * kStage + kABytes, 16, 1024);
+                for (int kb = 0; kb < nk; ++kb, ++c) {
+                    const int st = c % kStages;
+                    if (!mbar_wait(bar(FULL0 + st), (c / kStages) & 1, abort_flag)) { ok = false; break; }
+                    tc_fence_after();
+                    const uint64_t da = smem_desc(sbase + st * kStage, 16, 1024);
+                    const uint64_t db = smem_desc(sbase + st * kStage + kABytes, 16, 1024);
 #pragma unroll
-                for (int kk = 0; kk < BK / 16; ++kk)   // the descriptor's address field counts 16-byte units
-                    umma(tmem, da + ((kk * 32) >> 4), db + ((kk * 32) >> 4), id, (kb > 0 || kk > 0) ? 1u : 0u);
-                umma_commit(bar(EMPTY0 + st));
+                    for (int kk = 0; kk < BK / 16; ++kk)   // the descriptor's address field counts 16-byte units
+                        umma(tmem + ab * BN, da + ((kk * 32) >> 4), db + ((kk * 32) >> 4), id, (kb > 0 || kk > 0) ? 1u : 0u);
+                    umma_commit(bar(EMPTY0 + st));
+                }
+                if (ok) umma_commit(bar(ACC_FULL0 + ab));
             }
-            if (ok) umma_commit(bar(ACC_FULL));
         }
     } else {
         // ------------------------------------------------ epilogue: one thread per output row (= token)
         const int row = tid;
-        const int64_t tok = m0 + row;
-        const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
-        bool ok = __all_sync(0xffffffffu, mbar_wait(bar(ACC_FULL), 0, abort_flag));
-        tc_fence_after();
-        if (ok) {
+        bool ok = true;
+        int i = 0;
+        for (int64_t tile = blockIdx.x; tile < n_tiles && ok; tile += gridDim.x, ++i) {
+            const int ab = i & 1;
+            const int n0 = (int)(tile % tiles_n) * BN;
+            const int64_t tok = (tile / tiles_n) * BM + row;
+            const uint32_t acc = tmem + ((uint32_t)(warp * 32) << 16) + ab * BN;
+            ok = __all_sync(0xffffffffu, mbar_wait(bar(ACC_FULL0 + ab), (i >> 1) & 1, abort_flag));
+            if (!ok) break;
+            tc_fence_after();
             if (!FP8) {
                 __nv_bfloat16 *crow = static_cast<__nv_bfloat16 *>(C) + tok * ldc + n0;
 #pragma unroll 1
                 for (int c = 0; c < BN / 32; ++c) {
                     float v[32];
-                    tmem_ld32(lane_base + c * 32, v);
+                    tmem_ld32(acc + c * 32, v);
                     tmem_wait_ld();
+                    if (c == BN / 32 - 1) {   // the accumulator may be overwritten by the tile after next
+                        tc_fence_before();
+                        mbar_arrive(bar(ACC_EMPTY0 + ab));
+                    }
                     if (tok < T) {
 #pragma unroll
                         for (int q4 = 0; q4 < 4; ++q4) {
@@ -161,7 +183,7 @@ k_kv_project(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CU
 #pragma unroll 1
                     for (int c = 0; c < kQuantGroup / 32; ++c) {
                         float v[32];
-                        tmem_ld32(lane_base + grp * kQuantGroup + c * 32, v);
+                        tmem_ld32(acc + grp * kQuantGroup + c * 32, v);
                         tmem_wait_ld();
 #pragma unroll
                         for (int e = 0; e < 32; ++e) amax = fmaxf(amax, fabsf(v[e]));
@@ -172,8 +194,12 @@ k_kv_project(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CU
 #pragma unroll 1
                     for (int c = 0; c < kQuantGroup / 32; ++c) {
                         float v[32];
-                        tmem_ld32(lane_base + grp * kQuantGroup + c * 32, v);
+                        tmem_ld32(acc + grp * kQuantGroup + c * 32, v);
                         tmem_wait_ld();
+                        if (grp == BN / kQuantGroup - 1 && c == kQuantGroup / 32 - 1) {
+                            tc_fence_before();
+                            mbar_arrive(bar(ACC_EMPTY0 + ab));
+                        }
                         if (tok < T) {
 #pragma unroll
                             for (int q4 = 0; q4 < 2; ++q4) {
@@ -197,7 +223,7 @@ k_kv_project(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CU
     __syncthreads();
     if (warp == 5) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"((uint32_t)BN) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(kTmemCols) : "memory");
     }
 }
 
@@ -219,7 +245,10 @@ cudaError_t launch(int64_t T, int N, int dm, const void *H, int64_t ldh, const v
         if ((e = cudaFuncSetAttribute(k_kv_project<FP8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kSmemBytes)) != cudaSuccess) return e;
         done[dev] = true;
     }
-    dim3 grid((unsigned)(N / BN), (unsigned)((T + BM - 1) / BM));
+    static int n_sm[64] = {};
+    if (n_sm[dev] == 0 && (e = cudaDeviceGetAttribute(&n_sm[dev], cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+    const int64_t n_tiles = ((T + BM - 1) / BM) * (N / BN);
+    const unsigned grid = (unsigned)(n_tiles < n_sm[dev] ? n_tiles : n_sm[dev]);
     k_kv_project<FP8><<<grid, kThreads, kSmemBytes, st>>>(tmH, tmW, T, N, dm, C, ldc, scales);
     count_launch();
     return cudaGetLastError();
@@ -229,7 +258,7 @@ cudaError_t launch(int64_t T, int N, int dm, const void *H, int64_t ldh, const v
 
 bool kv_project_supported(int64_t T, int N, int dm, int64_t ldh, int64_t ldw, int64_t ldc, bool fp8)
 {
-    return T > 0 && T <= 0x7fffffffLL && (T + BM - 1) / BM <= 65535 && N > 0 && N % BN == 0 && dm > 0 && dm % BK == 0 &&
+    return T > 0 && T <= 0x7fffff00LL && N > 0 && N % BN == 0 && dm > 0 && dm % BK == 0 &&
            ldh >= dm && ldw >= dm && ldc >= N && ldh % 8 == 0 && ldw % 8 == 0 && ldc % (fp8 ? 16 : 8) == 0;
 }
 
