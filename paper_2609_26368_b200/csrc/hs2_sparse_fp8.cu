@@ -137,21 +137,20 @@ __device__ __forceinline__ Item make_item(const Params &p, const uint8_t *K, con
     return it;
 }
 
-// key index held by slot s of the virtual slot array [idx row | window], -1 when the slot is void
-__device__ __forceinline__ int slot_key(const Params &p, const Item &it, int tile, int lane)
+// Slot s of the virtual slot array [idx row | window] holds a key index or is void (-1).  slot_raw starts the fetch
+// (an idx entry is a global load), slot_fix applies the validity rules when the value is used one tile later, so
+// that the load's latency is never waited for.
+__device__ __forceinline__ int slot_raw(const Params &p, const Item &it, int tile, int lane)
 {
     const int s = tile * KT + lane;
-    int j = -1;
-    if (lane < KT) {
-        if (s < p.k) {
-            j = it.irow ? __ldg(it.irow + s) : -1;
-            if (j > it.pos - p.w || j >= it.kvl) j = -1;
-        } else if (s < p.k + p.w) {
-            j = it.pos - p.w + 1 + (s - p.k);
-            if (j > it.pos || j >= it.kvl) j = -1;
-        }
-    }
-    return j;
+    if (lane >= KT) return -1;
+    if (s < p.k) return it.irow ? __ldg(it.irow + s) : -1;
+    return s < p.k + p.w ? it.pos - p.w + 1 + (s - p.k) : -1;
+}
+__device__ __forceinline__ int slot_fix(const Params &p, const Item &it, int tile, int lane, int j)
+{
+    const int hi = tile * KT + lane < p.k ? it.pos - p.w : it.pos;   // idx entries inside the window are void
+    return (j < 0 || j > hi || j >= it.kvl) ? -1 : j;
 }
 
 // lane -> 16-byte chunk c (of 8) of rows r0 + (lane >> 3); lanes 0-15 also fetch the K scale of row `lane`,
@@ -256,13 +255,13 @@ __device__ __forceinline__ void run_tiles(const Params &p, const Item &it, const
     char *meta = wsm + NSTAGE * kStageBytes;
     const uint32_t mbase = sbase + NSTAGE * kStageBytes;
     int next = t_begin;
-    int jn = next < t_end ? slot_key(p, it, next, lane) : -1;
+    int jn = next < t_end ? slot_raw(p, it, next, lane) : -1;
     int n_issued = 0, n_done = 0;
     auto try_issue = [&](int stage) -> bool {
         while (next < t_end) {
-            const int j = jn;
+            const int j = slot_fix(p, it, next, lane, jn);
             ++next;
-            if (next < t_end) jn = slot_key(p, it, next, lane);
+            if (next < t_end) jn = slot_raw(p, it, next, lane);
             if (__ballot_sync(0xffffffffu, j >= 0)) {   // all-void tiles are skipped
                 reinterpret_cast<int *>(meta + stage * kMetaBytes)[lane] = j;
                 issue_stage(it, sbase + stage * kStageBytes, mbase + stage * kMetaBytes, j, lane);

@@ -139,22 +139,22 @@ struct Item {
     int pos, kvl;
 };
 
-// key index held by slot s of the virtual slot array [idx row | window], -1 when the slot is void
+// Slot s of the virtual slot array [idx row | window] holds a key index or is void (-1).  slot_raw starts the fetch
+// (an idx entry is a global load), slot_fix applies the validity rules when the value is used one tile later, so
+// that the load's latency is never waited for.
 template <int KT>
-__device__ __forceinline__ int slot_key(const Params &p, const Item &it, int tile, int lane)
+__device__ __forceinline__ int slot_raw(const Params &p, const Item &it, int tile, int lane)
 {
     const int s = tile * KT + lane;
-    int j = -1;
-    if (lane < KT) {
-        if (s < p.k) {
-            j = __ldg(it.irow + s);
-            if (j > it.pos - p.w || j >= it.kvl) j = -1;
-        } else if (s < p.k + p.w) {
-            j = it.pos - p.w + 1 + (s - p.k);
-            if (j > it.pos || j >= it.kvl) j = -1;
-        }
-    }
-    return j;   // negative entries stay negative
+    if (lane >= KT) return -1;
+    if (s < p.k) return __ldg(it.irow + s);
+    return s < p.k + p.w ? it.pos - p.w + 1 + (s - p.k) : -1;
+}
+template <int KT>
+__device__ __forceinline__ int slot_fix(const Params &p, const Item &it, int tile, int lane, int j)
+{
+    const int hi = tile * KT + lane < p.k ? it.pos - p.w : it.pos;   // idx entries inside the window are void
+    return (j < 0 || j > hi || j >= it.kvl) ? -1 : j;
 }
 
 // bulk variant: lane r < KT copies K row r, lane 16 + r copies V row r; void rows are not copied (the stage
@@ -302,13 +302,13 @@ __device__ __forceinline__ void run_tiles(const Params &p, const Item &it, const
         __syncwarp();
     }
     int next = t_begin;
-    int jn = next < t_end ? slot_key<KT>(p, it, next, lane) : -1;
+    int jn = next < t_end ? slot_raw<KT>(p, it, next, lane) : -1;
     int n_issued = 0, n_done = 0;
     auto try_issue = [&](int stage) -> bool {
         while (next < t_end) {
-            const int j = jn;
+            const int j = slot_fix<KT>(p, it, next, lane, jn);
             ++next;
-            if (next < t_end) jn = slot_key<KT>(p, it, next, lane);
+            if (next < t_end) jn = slot_raw<KT>(p, it, next, lane);
             if (__ballot_sync(0xffffffffu, j >= 0)) {
                 sj[stage * 32 + lane] = j;
                 if (kBulk) issue_stage_bulk<KT>(it, sbase + stage * kStageBytes, bars + 8 * stage, j, lane);
