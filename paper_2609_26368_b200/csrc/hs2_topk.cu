@@ -208,8 +208,10 @@ k_topk_cached(const Params p, const float *__restrict__ scores, int64_t score_st
         }
     }
     const int j0 = tid * E;
+    const bool has = j0 < nc;   // threads (whole warps, on short rows) past the row's end skip every per-candidate loop
     uint32_t key[E];
     unsigned kmin = 0xffffffffu, kmax = 0u;
+    if (has)
 #pragma unroll
     for (int e4 = 0; e4 < E; e4 += 4) {
         if (VEC && j0 + e4 + 4 <= nc) {
@@ -250,10 +252,12 @@ k_topk_cached(const Params p, const float *__restrict__ scores, int64_t score_st
                 const uint32_t kk = s_list[t];
                 if ((kk >> hi) == prefix) atomicAdd(&hist[(kk >> shift) & dmask], 1u);
             }
-        } else {
+        } else if (has) {
 #pragma unroll
             for (int e = 0; e < E; ++e) {
-                const bool live = (j0 + e < nc) && (hi >= 32 || (key[e] >> hi) == prefix);
+                // slots past the row's end hold key 0, which is below every real key (the lowest, -inf, maps to
+                // 0x007fffff): counted or not, they sit at the very bottom of the lowest bin and are never reached
+                const bool live = hi >= 32 || (key[e] >> hi) == prefix;
                 if (live) atomicAdd(&hist[(key[e] >> shift) & dmask], 1u);
             }
         }
@@ -273,9 +277,10 @@ k_topk_cached(const Params p, const float *__restrict__ scores, int64_t score_st
             // every candidate that can still be the take-th largest sits in this bin (at most kListCap of them)
             // (one atomic per member on a single word looks wasteful, but a ballot-aggregated version was measured
             // slower: 2.31 vs 2.18 ms for the whole full layer on the 8K benchmark)
+            if (has)
 #pragma unroll
             for (int e = 0; e < E; ++e)
-                if (j0 + e < nc && (key[e] >> hi) == prefix) {
+                if ((key[e] >> hi) == prefix) {
                     const unsigned slot = atomicAdd(&s_cnt, 1u);
                     if (slot < kListCap) s_list[slot] = key[e];
                 }
@@ -346,11 +351,11 @@ k_topk_cached(const Params p, const float *__restrict__ scores, int64_t score_st
 
     // ---- ordered compaction with one block scan
     unsigned n_gt = 0, n_eq = 0;
+    if (has)
 #pragma unroll
-    for (int e = 0; e < E; ++e) {
-        const bool ok = j0 + e < nc;
-        n_gt += ok && key[e] > tau;
-        n_eq += ok && key[e] == tau;
+    for (int e = 0; e < E; ++e) {   // key 0 (past the end) is below tau
+        n_gt += key[e] > tau;
+        n_eq += key[e] == tau;
     }
     const unsigned packed = (n_gt << 16) | n_eq;   // both totals stay below 65536 (rows <= 32768)
     unsigned incl = packed;
@@ -375,9 +380,9 @@ k_topk_cached(const Params p, const float *__restrict__ scores, int64_t score_st
     extern __shared__ int s_out[];
     const bool staged = p.k <= kStageOut;
     int *dst = staged ? s_out : out;
+    if (has)
 #pragma unroll
     for (int e = 0; e < E; ++e) {
-        if (j0 + e >= nc) continue;
         if (key[e] > tau) {
             dst[gt_before + min(eq_before, need_eq)] = j0 + e;
             ++gt_before;
