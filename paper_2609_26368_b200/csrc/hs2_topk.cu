@@ -241,6 +241,7 @@ k_topk_cached(const Params p, const float *__restrict__ scores, int64_t score_st
     unsigned need = (unsigned)take;
     bool on_list = false;                      // later rounds run on the threshold bin's candidates only
     unsigned n_list = 0;
+    bool first = true;
     while (hi > 0) {
         const int w = min(8, hi), shift = hi - w;
         const unsigned dmask = (1u << w) - 1u;
@@ -257,7 +258,8 @@ k_topk_cached(const Params p, const float *__restrict__ scores, int64_t score_st
             for (int e = 0; e < E; ++e) {
                 // slots past the row's end hold key 0, which is below every real key (the lowest, -inf, maps to
                 // 0x007fffff): counted or not, they sit at the very bottom of the lowest bin and are never reached
-                const bool live = hi >= 32 || (key[e] >> hi) == prefix;
+                // (in the first round every candidate has the common prefix by construction)
+                const bool live = first || (key[e] >> hi) == prefix;
                 if (live) atomicAdd(&hist[(key[e] >> shift) & dmask], 1u);
             }
         }
@@ -271,6 +273,7 @@ k_topk_cached(const Params p, const float *__restrict__ scores, int64_t score_st
         prefix = (hi >= 32 ? 0u : (prefix << w)) | digit;
         need = s_need;
         hi = shift;
+        first = false;
         const bool collect = !on_list && hi > 0 && in_bin <= kListCap;
         __syncthreads();   // every thread has read hist[digit] before the next round zeroes the histogram
         if (collect) {
@@ -350,13 +353,16 @@ k_topk_cached(const Params p, const float *__restrict__ scores, int64_t score_st
     }
 
     // ---- ordered compaction with one block scan
-    unsigned n_gt = 0, n_eq = 0;
+    // which of this thread's candidates are above tau / equal to it (key 0, past the end, is below tau)
+    static_assert(E <= 64, "one 64-bit mask per thread");
+    unsigned long long m_gt = 0ull, m_eq = 0ull;
     if (has)
 #pragma unroll
-    for (int e = 0; e < E; ++e) {   // key 0 (past the end) is below tau
-        n_gt += key[e] > tau;
-        n_eq += key[e] == tau;
+    for (int e = 0; e < E; ++e) {
+        m_gt |= (unsigned long long)(key[e] > tau) << e;
+        m_eq |= (unsigned long long)(key[e] == tau) << e;
     }
+    const unsigned n_gt = __popcll(m_gt), n_eq = __popcll(m_eq);
     const unsigned packed = (n_gt << 16) | n_eq;   // both totals stay below 65536 (rows <= 32768)
     unsigned incl = packed;
 #pragma unroll
@@ -380,15 +386,21 @@ k_topk_cached(const Params p, const float *__restrict__ scores, int64_t score_st
     extern __shared__ int s_out[];
     const bool staged = p.k <= kStageOut;
     int *dst = staged ? s_out : out;
-    if (has)
-#pragma unroll
-    for (int e = 0; e < E; ++e) {
-        if (key[e] > tau) {
-            dst[gt_before + min(eq_before, need_eq)] = j0 + e;
-            ++gt_before;
-        } else if (key[e] == tau) {
-            if (eq_before < need_eq) dst[gt_before + eq_before] = j0 + e;
-            ++eq_before;
+    {
+        // of the equal ones this thread keeps those that are still among the first need_eq of the row
+        unsigned keep_eq = eq_before < need_eq ? min(n_eq, need_eq - eq_before) : 0u;
+        unsigned long long m_keep = m_gt;
+        while (keep_eq > 0) {   // rare: ties at the threshold
+            const unsigned long long low = m_eq & (0ull - m_eq);
+            m_keep |= low;
+            m_eq ^= low;
+            --keep_eq;
+        }
+        unsigned posn = gt_before + min(eq_before, need_eq);
+        while (m_keep) {   // ascending candidate index
+            const int e = __ffsll((long long)m_keep) - 1;
+            m_keep &= m_keep - 1;
+            dst[posn++] = j0 + e;
         }
     }
     if (staged) {
