@@ -163,7 +163,7 @@ k_topk_cached(const Params p, const float *__restrict__ scores, int64_t score_st
     constexpr int WARPS = THREADS / 32;
     __shared__ unsigned hist[256];
     __shared__ unsigned s_warp[WARPS];
-    __shared__ unsigned s_min[WARPS], s_max[WARPS];
+    __shared__ unsigned s_min[WARPS];   // per-warp partial of the row-wide reduction
     __shared__ unsigned s_prefix, s_need, s_cnt;
     __shared__ uint32_t s_list[kListCap];
 
@@ -210,34 +210,36 @@ k_topk_cached(const Params p, const float *__restrict__ scores, int64_t score_st
     const int j0 = tid * E;
     const bool has = j0 < nc;   // threads (whole warps, on short rows) past the row's end skip every per-candidate loop
     uint32_t key[E];
-    unsigned kmin = 0xffffffffu, kmax = 0u;
+    // which bits differ anywhere in the row: OR of (key ^ key of candidate 0), one logic op per candidate
+    const uint32_t ref = order_key(__ldg(srow));
+    unsigned diff = 0u;
     if (has)
 #pragma unroll
     for (int e4 = 0; e4 < E; e4 += 4) {
         if (VEC && j0 + e4 + 4 <= nc) {
             const float4 v = __ldg(reinterpret_cast<const float4 *>(srow + j0 + e4));
             key[e4] = order_key(v.x); key[e4 + 1] = order_key(v.y); key[e4 + 2] = order_key(v.z); key[e4 + 3] = order_key(v.w);
+#pragma unroll
+            for (int e = e4; e < e4 + 4; ++e) diff |= key[e] ^ ref;
         } else {
 #pragma unroll
-            for (int e = e4; e < e4 + 4; ++e) key[e] = j0 + e < nc ? order_key(srow[j0 + e]) : 0u;
+            for (int e = e4; e < e4 + 4; ++e) {
+                const bool ok = j0 + e < nc;
+                key[e] = ok ? order_key(srow[j0 + e]) : 0u;
+                if (ok) diff |= key[e] ^ ref;
+            }
         }
-#pragma unroll
-        for (int e = e4; e < e4 + 4; ++e)
-            if (j0 + e < nc) { kmin = min(kmin, key[e]); kmax = max(kmax, key[e]); }
     }
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        kmin = min(kmin, __shfl_xor_sync(0xffffffffu, kmin, o));
-        kmax = max(kmax, __shfl_xor_sync(0xffffffffu, kmax, o));
-    }
-    if (lane == 0) { s_min[warp] = kmin; s_max[warp] = kmax; }
+    for (int o = 16; o > 0; o >>= 1) diff |= __shfl_xor_sync(0xffffffffu, diff, o);
+    if (lane == 0) s_min[warp] = diff;
     __syncthreads();
 #pragma unroll
-    for (int w = 0; w < WARPS; ++w) { kmin = min(kmin, s_min[w]); kmax = max(kmax, s_max[w]); }
+    for (int w = 0; w < WARPS; ++w) diff |= s_min[w];
 
     // bits above `hi` are equal in every candidate; resolve the rest 8 bits at a time
-    int hi = 32 - __clz(kmin ^ kmax);          // 0 when all candidates are equal
-    unsigned prefix = hi >= 32 ? 0u : (kmax >> hi);
+    int hi = 32 - __clz(diff);                 // 0 when all candidates are equal
+    unsigned prefix = hi >= 32 ? 0u : (ref >> hi);
     unsigned need = (unsigned)take;
     bool on_list = false;                      // later rounds run on the threshold bin's candidates only
     unsigned n_list = 0;
@@ -292,7 +294,7 @@ k_topk_cached(const Params p, const float *__restrict__ scores, int64_t score_st
             n_list = min(s_cnt, kListCap);
         }
     }
-    const uint32_t tau = hi == 0 && kmin == kmax ? kmax : prefix;   // key of the take-th largest candidate
+    const uint32_t tau = diff == 0u ? ref : prefix;                  // key of the take-th largest candidate
     const unsigned need_eq = need;                                   // equal keys kept, lowest indices first
     if (MODE == SEL_TAU) {
         if (tid == 0) sa.tau_key[blockIdx.x] = tau;
