@@ -399,7 +399,7 @@ def test_block_level_selection_variant():
     sc = torch.tensor(np.round(rng.normal(size=(B_, Hkv, Lq, Lk)) * 4) / 4, dtype=torch.float32, device="cuda")
     qs = torch.tensor([600, 37], dtype=torch.int32, device="cuda")
     kl = torch.tensor([700, 90], dtype=torch.int32, device="cuda")
-    for blk, k in ((64, 256), (16, 48), (4, 64), (1, 30)):
+    for blk, k in ((64, 256), (16, 48), (4, 64), (4, 512), (1, 30)):     # (4, 512): more than 64 blocks per row
         prob = hs2.Problem(B_, Lq, Lk, 4, Hkv, 64, k, w, q_start=qs, kv_lens=kl, select_block=blk)
         idx = hs2.hs2_topk_select(prob, sc)
         torch.cuda.synchronize()
