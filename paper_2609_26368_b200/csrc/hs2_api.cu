@@ -84,6 +84,19 @@ size_t full_select_ws_bytes(const Params &p)
     return align_up(rows * row, 256);
 }
 
+// Decode-shaped full layer (one query per sequence) on the mma.sync gather kernel: the sweep over the cache keeps the
+// raw q.k products, so that the selection scores need no second pass over K.  Scratch: [sweep's own scratch][raw
+// products: B * Hq * Lk floats][score rows: B * Hkv rows].
+struct DecodeFusedPlan { size_t off_raw, off_strip, total; };
+DecodeFusedPlan decode_fused_plan(const Params &pd, size_t sweep_ws)
+{
+    DecodeFusedPlan f;
+    f.off_raw = align_up(sweep_ws, 256);
+    f.off_strip = f.off_raw + align_up((size_t)pd.B * pd.Hq * pd.Lk * sizeof(float), 256);
+    f.total = f.off_strip + align_up((size_t)pd.B * pd.Hkv * strip_row_bytes(pd), 256);
+    return f;
+}
+
 // ---- filtered selection (sampled threshold -> ordered candidate lists -> select) ----
 constexpr int kFilterSamp = 8;              // every 8th key tile is scored for the threshold
 // The filtered path wins only when rows are long (measured: 131072 keys 485 ms vs 580 ms with strips, 32768
@@ -212,7 +225,7 @@ size_t hs2_workspace_bytes(const hs2_problem *hp, hs2_op op)
                 if (p.Lq == 1) {   // the decode-shaped layer may split over the keys
                     Params pd = p;
                     pd.k = 0; pd.w = p.Lk;
-                    const size_t dec = sparse_mma_supported(p, hp->dtype)         ? sparse_mma_decode_ws_bytes(pd)
+                    const size_t dec = sparse_mma_supported(p, hp->dtype)         ? decode_fused_plan(pd, sparse_mma_decode_ws_bytes(pd)).total
                                        : sparse_tc5_supported_shape(pd, hp->dtype) ? sparse_tc5_ws_bytes(pd)
                                                                                    : 0;
                     if (dec > need) need = dec;
@@ -255,9 +268,24 @@ hs2_status hs2_full_attn_select(const hs2_problem *hp, const void *Q, const void
     Params pd = p;
     pd.k = 0; pd.w = p.Lk;
     if (as_decode && !ws_ok(ws, ws_bytes, sparse_mma_decode_ws_bytes(pd))) as_decode = false;
-    if (as_decode)
+    if (as_decode) {
+        const bool want_sel_now = idx != nullptr && p.k > 0 && !scores_dbg;
+        const DecodeFusedPlan fu = decode_fused_plan(pd, sparse_mma_decode_ws_bytes(pd));
+        if (want_sel_now && ws_bytes >= fu.total && (int64_t)p.B * p.Hkv <= 65535) {
+            float *raw = reinterpret_cast<float *>(static_cast<char *>(ws) + fu.off_raw);
+            float *strip = reinterpret_cast<float *>(static_cast<char *>(ws) + fu.off_strip);
+            e = launch_sparse_mma_decode(pd, Q, K, V, nullptr, nullptr, O, LSE, ws, ws_bytes, st, raw);
+            if (e == cudaSuccess) {
+                const int64_t stride = (int64_t)(strip_row_bytes(p) / sizeof(float));
+                if ((e = launch_scores_from_raw(p, raw, LSE, strip, stride, st)) != cudaSuccess) return cuda_fail(e);
+                if ((e = launch_select(p, strip, stride, idx, 0, select_rows(p), st)) != cudaSuccess) return cuda_fail(e);
+                return HS2_OK;
+            }
+            if (e != cudaErrorNotSupported) return cuda_fail(e);
+            (void)cudaGetLastError();
+        }
         e = launch_sparse_mma_decode(pd, Q, K, V, nullptr, nullptr, O, LSE, ws, ws_bytes, st);
-    else {
+    } else {
         e = cudaErrorNotSupported;
         // the same idea for large head groups: the tcgen05 gather kernel, keys split over CTAs through the scratch
         if (p.Lq == 1 && !g_disable_tc5.load(std::memory_order_relaxed) && sparse_tc5_supported(pd, dt) && aligned16(Q, K, V, O)) {

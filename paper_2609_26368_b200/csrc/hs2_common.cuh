@@ -102,9 +102,13 @@ bool sparse_mma_supported(const Params &p, hs2_dtype dt);
 cudaError_t launch_sparse_mma_prefill(const Params &p, const void *Q, const void *K, const void *V, const int32_t *idx,
                                       const float *sink, void *O, float *LSE, cudaStream_t st);
 size_t sparse_mma_decode_ws_bytes(const Params &p);
+// raw (optional): float [B * Hkv][G][Lk]; receives the unscaled q.k of every attended (head, key)
 cudaError_t launch_sparse_mma_decode(const Params &p, const void *Q, const void *K, const void *V, const int32_t *idx,
                                      const float *sink, void *O, float *LSE, void *ws, size_t ws_bytes,
-                                     cudaStream_t st);
+                                     cudaStream_t st, float *raw = nullptr);
+// group scores of a single-query layer from those raw products (rows = (b, g), row stride out_stride)
+cudaError_t launch_scores_from_raw(const Params &p, const float *raw, const float *LSE, float *out, int64_t out_stride,
+                                   cudaStream_t st);
 
 // Decode with the partials in a static device array of the library (no caller scratch).
 constexpr int kStaticDecodeMaxPairs = HS2_STATIC_DECODE_MAX_PAIRS;

@@ -137,6 +137,8 @@ struct Item {
     int64_t row_stride;       // bytes between consecutive tokens
     const int32_t *irow;      // idx row of this (query, KV head), or nullptr when k == 0
     int pos, kvl;
+    float *raw;               // optional: raw q.k of every (head, key) of this pair, [G][lk] (decode-shaped full layer)
+    int lk;
 };
 
 // Slot s of the virtual slot array [idx row | window] holds a key index or is void (-1).  slot_raw starts the fetch
@@ -197,7 +199,8 @@ __device__ __forceinline__ void issue_stage(const Item &it, uint32_t stage_base,
 
 template <int KT>
 __device__ __forceinline__ void consume_stage(Acc &acc, const uint32_t (&qf)[16], uint32_t stage_base, unsigned mask,
-                                              float scale_log2, int lane)
+                                              float scale_log2, int lane, float *raw = nullptr, int lk = 0, int G = 0,
+                                              const int *sjrow = nullptr)
 {
     const int g = lane >> 2;
     const int mi = lane >> 3, rr = lane & 7;
@@ -221,6 +224,22 @@ __device__ __forceinline__ void consume_stage(Acc &acc, const uint32_t (&qf)[16]
         }
 #pragma unroll
         for (int e = 0; e < 4; ++e) s[mt][e] += s2[e];
+    }
+    if (raw) {
+        // The decode-shaped full layer keeps the raw products: the selection scores need the final LSE, and reading
+        // them back (4 bytes per head and key) is far cheaper than sweeping K a second time.
+        const int t = lane & 3;
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+            for (int r = 0; r < 2; ++r) {
+                const int j = sjrow[mt * 16 + g + 8 * r];
+                if (j >= 0) {
+#pragma unroll
+                    for (int hh = 0; hh < 2; ++hh)
+                        if (2 * t + hh < G) raw[(int64_t)(2 * t + hh) * lk + j] = s[mt][2 * r + hh];
+                }
+            }
     }
     // online softmax, base-2 domain; this thread: heads 2t+hh, keys 16 mt + g + 8 r
     float mx[2] = {-INFINITY, -INFINITY};
@@ -343,7 +362,7 @@ __device__ __forceinline__ void run_tiles(const Params &p, const Item &it, const
         if (try_issue(n_issued % NSTAGE)) ++n_issued;
         if (!kBulk) cp_async_commit();
         const unsigned mask = __ballot_sync(0xffffffffu, sj[stage * 32 + lane] >= 0);
-        consume_stage<KT>(acc, qf, sbase + stage * kStageBytes, mask, p.scale_log2, lane);
+        consume_stage<KT>(acc, qf, sbase + stage * kStageBytes, mask, p.scale_log2, lane, it.raw, it.lk, p.G, sj + stage * 32);
         ++n_done;
     }
     if (kBulk) {
@@ -465,6 +484,8 @@ __device__ __forceinline__ Item make_item(const Params &p, const __nv_bfloat16 *
     it.irow = idx ? idx + (((int64_t)b * hkv_real + g_real) * p.Lq + i) * p.k : nullptr;
     it.pos = pos_of(p, b, i);
     it.kvl = kvlen_of(p, b);
+    it.raw = nullptr;
+    it.lk = p.Lk;
     return it;
 }
 
@@ -501,7 +522,8 @@ template <class C>
 __global__ void __launch_bounds__(C::WARPS * 32)
 k_sparse_decode_cta(const Params p, const __nv_bfloat16 *__restrict__ Q, const __nv_bfloat16 *__restrict__ K,
                     const __nv_bfloat16 *__restrict__ V, const int32_t *__restrict__ idx,
-                    const float *__restrict__ sink, __nv_bfloat16 *__restrict__ O, float *__restrict__ LSE)
+                    const float *__restrict__ sink, __nv_bfloat16 *__restrict__ O, float *__restrict__ LSE,
+                    float *__restrict__ raw)
 {
     extern __shared__ __align__(128) char smem[];
     constexpr int W = C::WARPS;
@@ -511,7 +533,8 @@ k_sparse_decode_cta(const Params p, const __nv_bfloat16 *__restrict__ Q, const _
     const int g = lane >> 2, t = lane & 3;
     char *wsm = smem + warp * C::kWarpSmem;
     float *sml = reinterpret_cast<float *>(smem + W * C::kWarpSmem);   // [W][16]: m then l per head
-    const Item it = make_item(p, K, V, idx, b, gkv, 0);
+    Item it = make_item(p, K, V, idx, b, gkv, 0);
+    if (raw) it.raw = raw + (int64_t)bg * p.G * p.Lk;
     uint32_t qf[16];
     load_q_frags(p, Q, b, 0, gkv, lane, qf);
     Acc acc;
@@ -573,7 +596,7 @@ __global__ void __launch_bounds__(C::WARPS * 32)
 k_sparse_decode_split(const Params p, const __nv_bfloat16 *__restrict__ Q, const __nv_bfloat16 *__restrict__ K,
                       const __nv_bfloat16 *__restrict__ V, const int32_t *__restrict__ idx,
                       const float *__restrict__ sink, __nv_bfloat16 *__restrict__ O, float *__restrict__ LSE,
-                      DecodeWs ws, int n_splits, int tiles_per_split)
+                      DecodeWs ws, int n_splits, int tiles_per_split, float *__restrict__ raw)
 {
     extern __shared__ __align__(128) char smem[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -584,7 +607,8 @@ k_sparse_decode_split(const Params p, const __nv_bfloat16 *__restrict__ Q, const
     const int gkv = bg % p.Hkv, b = bg / p.Hkv;
     const int g = lane >> 2, t = lane & 3;
     char *wsm = smem + warp * C::kWarpSmem;
-    const Item it = make_item(p, K, V, idx, b, gkv, 0);
+    Item it = make_item(p, K, V, idx, b, gkv, 0);
+    if (raw) it.raw = raw + (int64_t)bg * p.G * p.Lk;
     uint32_t qf[16];
     load_q_frags(p, Q, b, 0, gkv, lane, qf);
     Acc acc;
@@ -709,7 +733,8 @@ size_t sparse_mma_decode_ws_bytes(const Params &p)
 }
 
 cudaError_t launch_sparse_mma_decode(const Params &p, const void *Q, const void *K, const void *V, const int32_t *idx,
-                                     const float *sink, void *O, float *LSE, void *ws, size_t ws_bytes, cudaStream_t st)
+                                     const float *sink, void *O, float *LSE, void *ws, size_t ws_bytes, cudaStream_t st,
+                                     float *raw)
 {
     using C = DecodeCfg;
     cudaError_t e = set_attrs();
@@ -724,7 +749,7 @@ cudaError_t launch_sparse_mma_decode(const Params &p, const void *Q, const void 
     cta_path = false;   // tuning builds only
 #endif
     if (cta_path) {
-        k_sparse_decode_cta<C><<<bg, C::WARPS * 32, kDecodeCtaSmem, st>>>(p, q, k, v, idx, sink, (__nv_bfloat16 *)O, LSE);
+        k_sparse_decode_cta<C><<<bg, C::WARPS * 32, kDecodeCtaSmem, st>>>(p, q, k, v, idx, sink, (__nv_bfloat16 *)O, LSE, raw);
         count_launch();
     return cudaGetLastError();
     }
@@ -738,7 +763,7 @@ cudaError_t launch_sparse_mma_decode(const Params &p, const void *Q, const void 
     if (n_splits > (n_tiles + 1) / 2) n_splits = (n_tiles + 1) / 2 > 0 ? (n_tiles + 1) / 2 : 1;
     const int tiles_per_split = (n_tiles + n_splits - 1) / n_splits;
     n_splits = (n_tiles + tiles_per_split - 1) / tiles_per_split;
-    if (n_splits <= 1) return launch_sparse_mma_prefill(p, Q, K, V, idx, sink, O, LSE, st);
+    if (n_splits <= 1) return raw ? cudaErrorNotSupported : launch_sparse_mma_prefill(p, Q, K, V, idx, sink, O, LSE, st);
     DecodeWs w;
     char *base = (char *)ws;
     const size_t items = (size_t)bg * kMaxSplits;
@@ -750,7 +775,35 @@ cudaError_t launch_sparse_mma_decode(const Params &p, const void *Q, const void 
     const int64_t n_items = (int64_t)bg * n_splits;
     const unsigned blocks = (unsigned)((n_items + C::WARPS - 1) / C::WARPS);
     k_sparse_decode_split<C><<<blocks, C::WARPS * 32, C::WARPS * C::kWarpSmem, st>>>(
-        p, q, k, v, idx, sink, (__nv_bfloat16 *)O, LSE, w, n_splits, tiles_per_split);
+        p, q, k, v, idx, sink, (__nv_bfloat16 *)O, LSE, w, n_splits, tiles_per_split, raw);
+    count_launch();
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------- selection scores from the kept raw products
+// a[j] = max over the heads h of the group of (scale * raw[h][j] - LSE_h)   (Section 3.4), one thread per key
+__global__ void __launch_bounds__(256)
+k_scores_from_raw(const Params p, const float *__restrict__ raw, const float *__restrict__ LSE, float *__restrict__ out,
+                  int64_t out_stride)
+{
+    const int bg = blockIdx.y;
+    const int gkv = bg % p.Hkv, b = bg / p.Hkv;
+    const int j = blockIdx.x * 256 + threadIdx.x;
+    if (j >= p.Lk) return;
+    const float *r = raw + (int64_t)bg * p.G * p.Lk + j;
+    float a = -INFINITY;
+    for (int h = 0; h < p.G; ++h)
+        a = fmaxf(a, fmaf(p.scale, r[(int64_t)h * p.Lk], -LSE[(int64_t)b * p.Hq + gkv * p.G + h]));   // Lq == 1
+    out[(int64_t)bg * out_stride + j] = a;
+}
+
+cudaError_t launch_scores_from_raw(const Params &p, const float *raw, const float *LSE, float *out, int64_t out_stride,
+                                   cudaStream_t st)
+{
+    const int bg = p.B * p.Hkv;
+    if (bg <= 0 || bg > 65535 || p.Lq != 1) return cudaErrorNotSupported;
+    dim3 grid((unsigned)((p.Lk + 255) / 256), (unsigned)bg);
+    k_scores_from_raw<<<grid, 256, 0, st>>>(p, raw, LSE, out, out_stride);
     count_launch();
     return cudaGetLastError();
 }
@@ -827,7 +880,7 @@ cudaError_t launch_sparse_mma_decode_static(const Params &p, const void *Q, cons
     const unsigned blocks = (unsigned)((n_items + C::WARPS - 1) / C::WARPS);
     k_sparse_decode_split<C><<<blocks, C::WARPS * 32, C::WARPS * C::kWarpSmem, st>>>(
         p, (const __nv_bfloat16 *)Q, (const __nv_bfloat16 *)K, (const __nv_bfloat16 *)V, idx, sink, (__nv_bfloat16 *)O, LSE,
-        w, n_splits, tiles_per_split);
+        w, n_splits, tiles_per_split, nullptr);
     count_launch();
     return cudaGetLastError();
 }
