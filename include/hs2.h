@@ -13,6 +13,10 @@
  *   hs2_sparse_attn_prefill  SA layer: attention over (reused indices) U (forced window of the most
  *                            recent w tokens), K/V read from the FA layer's cache (Section 3.3).
  *   hs2_sparse_attn_decode   the SA layer for one new token per sequence (split over the KV set).
+ *   ..._gated                the two SA calls with the sigmoid output gate of the sparse layers fused in.
+ *   ..._fp8kv                the two SA calls on an e4m3 KV cache with per-token scales.
+ *   hs2_kv_project           the producer of those caches: the K/V projection of KV Bridging (Section 3.2),
+ *                            bf16 or quantised to the e4m3 cache format in its epilogue.
  *
  * Conventions
  *   - Every tensor pointer is a DEVICE pointer owned by the caller; `hs2_problem` itself is a
