@@ -87,10 +87,12 @@ size_t full_select_ws_bytes(const Params &p)
 // Decode-shaped full layer (one query per sequence) on the mma.sync gather kernel: the sweep over the cache keeps the
 // raw q.k products, so that the selection scores need no second pass over K.  Scratch: [sweep's own scratch][raw
 // products: B * Hq * Lk floats][score rows: B * Hkv rows].
-struct DecodeFusedPlan { size_t off_raw, off_strip, total; };
+struct DecodeFusedPlan { size_t off_raw, off_strip, total; bool ok; };
+constexpr size_t kRawCapBytes = (size_t)2 << 30;   // beyond this the layer sweeps K twice instead
 DecodeFusedPlan decode_fused_plan(const Params &pd, size_t sweep_ws)
 {
     DecodeFusedPlan f;
+    f.ok = (size_t)pd.B * pd.Hq * pd.Lk * sizeof(float) <= kRawCapBytes;
     f.off_raw = align_up(sweep_ws, 256);
     f.off_strip = f.off_raw + align_up((size_t)pd.B * pd.Hq * pd.Lk * sizeof(float), 256);
     f.total = f.off_strip + align_up((size_t)pd.B * pd.Hkv * strip_row_bytes(pd), 256);
@@ -225,7 +227,8 @@ size_t hs2_workspace_bytes(const hs2_problem *hp, hs2_op op)
                 if (p.Lq == 1) {   // the decode-shaped layer may split over the keys
                     Params pd = p;
                     pd.k = 0; pd.w = p.Lk;
-                    const size_t dec = sparse_mma_supported(p, hp->dtype)         ? decode_fused_plan(pd, sparse_mma_decode_ws_bytes(pd)).total
+                    const DecodeFusedPlan fu = decode_fused_plan(pd, sparse_mma_supported(p, hp->dtype) ? sparse_mma_decode_ws_bytes(pd) : 0);
+                    const size_t dec = sparse_mma_supported(p, hp->dtype)         ? (fu.ok ? fu.total : sparse_mma_decode_ws_bytes(pd))
                                        : sparse_tc5_supported_shape(pd, hp->dtype) ? sparse_tc5_ws_bytes(pd)
                                                                                    : 0;
                     if (dec > need) need = dec;
@@ -271,7 +274,7 @@ hs2_status hs2_full_attn_select(const hs2_problem *hp, const void *Q, const void
     if (as_decode) {
         const bool want_sel_now = idx != nullptr && p.k > 0 && !scores_dbg;
         const DecodeFusedPlan fu = decode_fused_plan(pd, sparse_mma_decode_ws_bytes(pd));
-        if (want_sel_now && ws_bytes >= fu.total && (int64_t)p.B * p.Hkv <= 65535) {
+        if (want_sel_now && fu.ok && ws_bytes >= fu.total && (int64_t)p.B * p.Hkv <= 65535) {
             float *raw = reinterpret_cast<float *>(static_cast<char *>(ws) + fu.off_raw);
             float *strip = reinterpret_cast<float *>(static_cast<char *>(ws) + fu.off_strip);
             e = launch_sparse_mma_decode(pd, Q, K, V, nullptr, nullptr, O, LSE, ws, ws_bytes, st, raw);
