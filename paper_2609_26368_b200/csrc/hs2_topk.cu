@@ -156,7 +156,7 @@ __device__ __forceinline__ int sample_rank(int take, int n, int n_s)
 }
 
 template <int THREADS, int E, bool VEC, int MODE>
-__global__ void __launch_bounds__(THREADS, THREADS <= 256 ? 3 : 1)
+__global__ void __launch_bounds__(THREADS, THREADS > 256 ? 1 : (E > 32 ? 2 : 3))
 k_topk_cached(const Params p, const float *__restrict__ scores, int64_t score_stride, int32_t *__restrict__ idx,
               int64_t row0, int nc_lo, int nc_hi, SelArgs sa)
 {
@@ -773,8 +773,10 @@ k_topk(const Params p, const float *__restrict__ scores, int64_t score_stride, i
 // block; rows outside the variant's range leave at once, so each row is handled by exactly one launch
 // and the choice is per row even when the positions live on the device.
 struct TopkClass { int lo, hi; };
-constexpr TopkClass kClasses[6] = {{-1, 8192}, {8192, 32768}, {32768, 65536}, {65536, 131072}, {131072, 262144},
-                                   {262144, 0x7fffffff}};
+constexpr int kNumClasses = 9;
+constexpr TopkClass kClasses[kNumClasses] = {{-1, 2048},      {2048, 4096},     {4096, 8192},        {8192, 16384},
+                                             {16384, 32768},  {32768, 65536},   {65536, 131072},     {131072, 262144},
+                                             {262144, 0x7fffffff}};
 
 template <bool VEC>
 void launch_class(int c, const Params &p, const float *scores, int64_t score_stride, int32_t *idx, int64_t row0,
@@ -784,14 +786,19 @@ void launch_class(int c, const Params &p, const float *scores, int64_t score_str
     const unsigned n = (unsigned)n_rows;
     const size_t stage = p.k <= kStageOut ? (size_t)p.k * sizeof(int) : 0;   // the register kernels stage their output row
 #ifdef HS2_TOPK_NO_CLUSTER
-    if (c >= 2 && c <= 4) c = 5;   // tuning builds: long rows on the streaming kernel
+    if (c >= 5 && c <= 7) c = 8;   // tuning builds: long rows on the streaming kernel
 #endif
+    // The register kernels pay a fixed price per warp and row (rounds, scans, barriers), so a row gets no more
+    // warps than its candidates fill: 32 (or 64) candidates per thread.
     switch (c) {
-        case 0: k_topk_cached<256, 32, VEC, SEL_ROW><<<n, 256, stage, st>>>(p, scores, score_stride, idx, row0, lo, hi, SelArgs{}); break;
-        case 1: k_topk_cached<512, 64, VEC, SEL_ROW><<<n, 512, stage, st>>>(p, scores, score_stride, idx, row0, lo, hi, SelArgs{}); break;
-        case 2: k_topk_cluster<2, VEC><<<n * 2, 512, 0, st>>>(p, scores, score_stride, idx, row0, lo, hi); break;
-        case 3: k_topk_cluster<4, VEC><<<n * 4, 512, 0, st>>>(p, scores, score_stride, idx, row0, lo, hi); break;
-        case 4: k_topk_cluster<8, VEC><<<n * 8, 512, 0, st>>>(p, scores, score_stride, idx, row0, lo, hi); break;
+        case 0: k_topk_cached<64, 32, VEC, SEL_ROW><<<n, 64, stage, st>>>(p, scores, score_stride, idx, row0, lo, hi, SelArgs{}); break;
+        case 1: k_topk_cached<128, 32, VEC, SEL_ROW><<<n, 128, stage, st>>>(p, scores, score_stride, idx, row0, lo, hi, SelArgs{}); break;
+        case 2: k_topk_cached<256, 32, VEC, SEL_ROW><<<n, 256, stage, st>>>(p, scores, score_stride, idx, row0, lo, hi, SelArgs{}); break;
+        case 3: k_topk_cached<256, 64, VEC, SEL_ROW><<<n, 256, stage, st>>>(p, scores, score_stride, idx, row0, lo, hi, SelArgs{}); break;
+        case 4: k_topk_cached<512, 64, VEC, SEL_ROW><<<n, 512, stage, st>>>(p, scores, score_stride, idx, row0, lo, hi, SelArgs{}); break;
+        case 5: k_topk_cluster<2, VEC><<<n * 2, 512, 0, st>>>(p, scores, score_stride, idx, row0, lo, hi); break;
+        case 6: k_topk_cluster<4, VEC><<<n * 4, 512, 0, st>>>(p, scores, score_stride, idx, row0, lo, hi); break;
+        case 7: k_topk_cluster<8, VEC><<<n * 8, 512, 0, st>>>(p, scores, score_stride, idx, row0, lo, hi); break;
         default: k_topk<1024, kItems, false, VEC><<<n, 1024, 0, st>>>(p, scores, score_stride, idx, row0, lo, hi); break;
     }
     count_launch();
@@ -814,7 +821,7 @@ cudaError_t launch_topk(const Params &p, const float *scores, int64_t score_stri
         nc_min = clampnc(base + i_lo);
         nc_max = clampnc(base + i_hi);
     }
-    for (int c = 0; c < 6; ++c) {
+    for (int c = 0; c < kNumClasses; ++c) {
         if (nc_max <= kClasses[c].lo || nc_min > kClasses[c].hi) continue;   // no row of the block falls in this class
         if (vec) launch_class<true>(c, p, scores, score_stride, idx, row0, n_rows, st);
         else launch_class<false>(c, p, scores, score_stride, idx, row0, n_rows, st);
