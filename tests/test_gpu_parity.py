@@ -59,7 +59,8 @@ def _topk_case(scores: torch.Tensor, k, w, q_start=None, kv_lens=None):
     assert np.array_equal(got.reshape(-1, k), want)
 
 
-@pytest.mark.parametrize("Lk,k,w", [(512, 64, 16), (1000, 100, 0), (4099, 257, 33), (9001, 1024, 128)])
+@pytest.mark.parametrize("Lk,k,w", [(512, 64, 16), (1000, 100, 0), (3000, 700, 5), (4099, 257, 33), (9001, 1024, 128),
+                                     (14000, 3000, 64), (30000, 2048, 128)])   # every row class of the register kernels
 def test_topk_random_scores(Lk, k, w):
     g = torch.Generator().manual_seed(Lk)
     _topk_case(torch.randn(2, 2, 37, Lk, generator=g), k, w, q_start=[Lk - 37, Lk // 2], kv_lens=[Lk, Lk - 5])
