@@ -70,6 +70,11 @@ __device__ __forceinline__ void pick_digit(const unsigned *hist, unsigned prefix
     }
 }
 
+#ifndef HS2_TOPK_RANKMAX
+#define HS2_TOPK_RANKMAX 64
+#endif
+constexpr unsigned kRankMax = HS2_TOPK_RANKMAX;           // a threshold bin this small is finished by ranking its members
+
 // ---- rows that fit in registers: THREADS x E candidates, read once ------------------------------
 // Thread t owns the E consecutive candidates E t .. E t + E - 1, so the ascending-index order of the
 // output is (thread, element) order and the ordered compaction needs a single block scan.  The radix
@@ -292,6 +297,24 @@ k_topk_cached(const Params p, const float *__restrict__ scores, int64_t score_st
             __syncthreads();
             on_list = true;
             n_list = min(s_cnt, kListCap);
+            if (n_list <= kRankMax && n_list <= (unsigned)THREADS) {   // one thread per member
+                // A short list is finished by ranking instead of more histogram rounds (four barriers each): member
+                // t is the answer when fewer than `need` members are above it and at least `need` are not below it.
+                if ((unsigned)tid < n_list) {
+                    const uint32_t kt = s_list[tid];
+                    unsigned gt = 0, eq = 0;
+                    for (unsigned u = 0; u < n_list; ++u) {
+                        const uint32_t v = s_list[u];
+                        gt += v > kt;
+                        eq += v == kt;
+                    }
+                    if (gt < need && need <= gt + eq) { s_prefix = kt; s_need = need - gt; }   // equal members write the same
+                }
+                __syncthreads();
+                prefix = s_prefix;   // the full key
+                need = s_need;
+                hi = 0;
+            }
         }
     }
     const uint32_t tau = diff == 0u ? ref : prefix;                  // key of the take-th largest candidate
