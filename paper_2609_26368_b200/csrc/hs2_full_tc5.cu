@@ -196,17 +196,18 @@ k_full_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             mbar_arrive(bar(S_FREE0 + sb));
             const int j0 = j * BN;
             // raw-score maximum; only tiles that touch the diagonal or the end of the cache pay for masking
-            float m_raw = -INFINITY;
             if ((j0 + BN - 1 > pos0) || (j0 + BN > kvl)) {
 #pragma unroll
-                for (int e = 0; e < 64; ++e) {
+                for (int e = 0; e < 64; ++e)
                     if (j0 + e > prow || j0 + e >= kvl) s[e] = -INFINITY;
-                    m_raw = fmaxf(m_raw, s[e]);
-                }
-            } else {
-#pragma unroll
-                for (int e = 0; e < 64; ++e) m_raw = fmaxf(m_raw, s[e]);
             }
+            // four independent chains: one chain of 64 dependent maxima is 250 cycles of latency per tile
+            float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+#pragma unroll
+            for (int e = 0; e < 64; e += 4) {
+                mx0 = fmaxf(mx0, s[e]); mx1 = fmaxf(mx1, s[e + 1]); mx2 = fmaxf(mx2, s[e + 2]); mx3 = fmaxf(mx3, s[e + 3]);
+            }
+            const float m_raw = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
             const float m_blk = m_raw * p.scale_log2;                 // the scale is positive
             const bool need = m_blk > m_used + kRescaleThreshold;   // also true for the first finite block
             const float m_new = need ? m_blk : m_used;
