@@ -300,7 +300,10 @@ k_full_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
 // Warp 4 feeds K tiles by TMA (2-stage ring), warp 5 issues the MMAs into two accumulator buffers,
 // warps 0-3 (thread = key) subtract LSE, take the group maximum and write 32 consecutive keys of a
 // strip row per warp instruction.
-constexpr int SC_KCHUNK = 4096;                   // keys per CTA
+#ifndef HS2_SC_KCHUNK
+#define HS2_SC_KCHUNK 4096
+#endif
+constexpr int SC_KCHUNK = HS2_SC_KCHUNK;                  // keys per CTA
 // shared-memory plan of the score sweep for head_dim D: Q and K tiles are D/64 slices of [128 rows][128 B]
 template <int D>
 struct ScCfg {
