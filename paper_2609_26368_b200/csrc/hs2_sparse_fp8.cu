@@ -36,7 +36,12 @@ namespace hs2 {
 namespace {
 
 constexpr int HD = 128;
-constexpr int KT = 16;                       // key rows per stage
+#ifndef HS2_F8_KT
+#define HS2_F8_KT 16
+#endif
+constexpr int KT = HS2_F8_KT;                // key rows per stage (32-row stages were measured: 47.8 vs 45.3 us per decode step)
+constexpr int MT = KT / 16;                  // 16-key MMA tiles per stage
+static_assert(KT == 16 || KT == 32, "a stage holds 16 or 32 key rows");
 #ifndef HS2_F8_NSTAGE
 #define HS2_F8_NSTAGE 2
 #endif
@@ -44,8 +49,8 @@ constexpr int NSTAGE = HS2_F8_NSTAGE;
 constexpr int kRow = HD;                     // bytes of one e4m3 row
 constexpr int kTile = KT * kRow;             // one K or V tile of a stage
 constexpr int kStageBytes = 2 * kTile;
-// per warp: the stages, then per stage: key index of each row (32 ints), K scales (16), V scales (16)
-constexpr int kMetaBytes = 32 * 4 + 16 * 4 + 16 * 4;
+// per warp: the stages, then per stage: key index of each row (32 ints), K scales (KT), V scales (KT)
+constexpr int kMetaBytes = 32 * 4 + 2 * KT * 4;
 constexpr int kWarpSmem = NSTAGE * kStageBytes + NSTAGE * kMetaBytes;
 constexpr float kPShift = 256.f;             // probabilities x V scale are carried x 2^8 through the f16 operand
 
@@ -153,8 +158,8 @@ __device__ __forceinline__ int slot_fix(const Params &p, const Item &it, int til
     return (j < 0 || j > hi || j >= it.kvl) ? -1 : j;
 }
 
-// lane -> 16-byte chunk c (of 8) of rows r0 + (lane >> 3); lanes 0-15 also fetch the K scale of row `lane`,
-// lanes 16-31 the V scale of row `lane - 16`.  Void rows are zero filled, nothing is read for them.
+// lane -> 16-byte chunk c (of 8) of rows r0 + (lane >> 3); the lanes also fetch the stage's scales.  Void rows are
+// zero filled, nothing is read for them.
 __device__ __forceinline__ void issue_stage(const Item &it, uint32_t stage_base, uint32_t meta_base, int j, int lane)
 {
     const int c = lane & 7, hi = lane >> 3;
@@ -169,9 +174,14 @@ __device__ __forceinline__ void issue_stage(const Item &it, uint32_t stage_base,
         cp_async16(dst, kc + off, nbytes);
         cp_async16(dst + kTile, vc + off, nbytes);
     }
-    const int js = __shfl_sync(0xffffffffu, j, lane & 15);
-    const float *sp = (lane < 16 ? it.ksc : it.vsc) + (int64_t)max(js, 0) * it.sc_stride;
-    cp_async4(meta_base + 32 * 4 + lane * 4, sp, js < 0 ? 0 : 4);
+    // the 2 * KT scales of the stage: K scales of rows 0..KT-1, then V scales
+#pragma unroll
+    for (int s0 = 0; s0 < 2 * KT; s0 += 32) {
+        const int sl = s0 + lane;
+        const int js = __shfl_sync(0xffffffffu, j, sl % KT);
+        const float *sp = (sl < KT ? it.ksc : it.vsc) + (int64_t)max(js, 0) * it.sc_stride;
+        cp_async4(meta_base + 32 * 4 + sl * 4, sp, js < 0 ? 0 : 4);
+    }
 }
 
 __device__ __forceinline__ void consume_stage(Acc &acc, const uint32_t (&qf)[16], uint32_t stage_base, const float *sks,
@@ -179,32 +189,39 @@ __device__ __forceinline__ void consume_stage(Acc &acc, const uint32_t (&qf)[16]
 {
     const int g = lane >> 2;
     const int mi = lane >> 3, rr = lane & 7;
-    float s[4] = {0.f, 0.f, 0.f, 0.f}, s2[4] = {0.f, 0.f, 0.f, 0.f};
+    float s[MT][4];
     // S^T = K Q^T : rows = keys, columns = heads.  One ldmatrix = 16 keys x 32 dims = two MMAs.
-    {
-        const uint32_t rowaddr = stage_base + ((mi & 1) * 8 + rr) * kRow;
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt) {
+        float s2[4] = {0.f, 0.f, 0.f, 0.f};
+        s[mt][0] = s[mt][1] = s[mt][2] = s[mt][3] = 0.f;
+        const uint32_t rowaddr = stage_base + (mt * 16 + (mi & 1) * 8 + rr) * kRow;
 #pragma unroll
         for (int q4 = 0; q4 < 4; ++q4) {
             uint32_t a[4];
             ldmatrix_x4(a, rowaddr + ((uint32_t)((2 * q4 + (mi >> 1)) ^ rr) << 4));
-            mma_f16(s, cvt_e4m3x2(a[0]), cvt_e4m3x2(a[1]), cvt_e4m3x2(a[0] >> 16), cvt_e4m3x2(a[1] >> 16), qf[4 * q4], qf[4 * q4 + 1]);
+            mma_f16(s[mt], cvt_e4m3x2(a[0]), cvt_e4m3x2(a[1]), cvt_e4m3x2(a[0] >> 16), cvt_e4m3x2(a[1] >> 16), qf[4 * q4], qf[4 * q4 + 1]);
             mma_f16(s2, cvt_e4m3x2(a[2]), cvt_e4m3x2(a[3]), cvt_e4m3x2(a[2] >> 16), cvt_e4m3x2(a[3] >> 16), qf[4 * q4 + 2], qf[4 * q4 + 3]);
         }
+#pragma unroll
+        for (int e = 0; e < 4; ++e) s[mt][e] += s2[e];
     }
-    // dequantise the score rows, online softmax in the base-2 domain; this thread: heads 2t+hh, keys g + 8 r
-    const float ks[2] = {sks[g] * scale_log2, sks[g + 8] * scale_log2};
-    const float vs[2] = {svs[g] * kPShift, svs[g + 8] * kPShift};
+    // dequantise the score rows, online softmax in the base-2 domain; this thread: heads 2t+hh, keys 16 mt + g + 8 r
     float mx[2] = {-INFINITY, -INFINITY};
 #pragma unroll
-    for (int r = 0; r < 2; ++r) {
-        const bool ok = (mask >> (g + 8 * r)) & 1u;
+    for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
-        for (int hh = 0; hh < 2; ++hh) {
-            const float t2 = ok ? (s[2 * r + hh] + s2[2 * r + hh]) * ks[r] : -INFINITY;
-            s[2 * r + hh] = t2;
-            mx[hh] = fmaxf(mx[hh], t2);
+        for (int r = 0; r < 2; ++r) {
+            const int row = mt * 16 + g + 8 * r;
+            const bool ok = (mask >> row) & 1u;
+            const float ks = sks[row] * scale_log2;
+#pragma unroll
+            for (int hh = 0; hh < 2; ++hh) {
+                const float t2 = ok ? s[mt][2 * r + hh] * ks : -INFINITY;
+                s[mt][2 * r + hh] = t2;
+                mx[hh] = fmaxf(mx[hh], t2);
+            }
         }
-    }
     float corr[2], muse[2];
 #pragma unroll
     for (int hh = 0; hh < 2; ++hh) {
@@ -217,14 +234,19 @@ __device__ __forceinline__ void consume_stage(Acc &acc, const uint32_t (&qf)[16]
         acc.m[hh] = m_new;
         acc.l[hh] *= corr[hh];
     }
-    float pv[4];
+    uint32_t pb[MT][2];
 #pragma unroll
-    for (int e = 0; e < 4; ++e) {
-        pv[e] = exp2f(s[e] - muse[e & 1]);
-        acc.l[e & 1] += pv[e];
+    for (int mt = 0; mt < MT; ++mt) {
+        float pv[4];
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            pv[e] = exp2f(s[mt][e] - muse[e & 1]);
+            acc.l[e & 1] += pv[e];
+        }
+        const float vs0 = svs[mt * 16 + g] * kPShift, vs1 = svs[mt * 16 + g + 8] * kPShift;
+        pb[mt][0] = movmatrix_trans(pack_f16(pv[0] * vs0, pv[1] * vs0));   // keys 16 mt + 0..7
+        pb[mt][1] = movmatrix_trans(pack_f16(pv[2] * vs1, pv[3] * vs1));   // keys 16 mt + 8..15
     }
-    const uint32_t pb0 = movmatrix_trans(pack_f16(pv[0] * vs[0], pv[1] * vs[0]));   // keys 0..7
-    const uint32_t pb1 = movmatrix_trans(pack_f16(pv[2] * vs[1], pv[3] * vs[1]));   // keys 8..15
     if (__any_sync(0xffffffffu, corr[0] != 1.f || corr[1] != 1.f)) {
 #pragma unroll
         for (int dt = 0; dt < 8; ++dt) {
@@ -233,16 +255,17 @@ __device__ __forceinline__ void consume_stage(Acc &acc, const uint32_t (&qf)[16]
         }
     }
     // O^T += V^T P^T : one transposing ldmatrix = 16 keys x 32 dims = two MMAs (16 dims each)
-    {
-        const uint32_t rowaddr = stage_base + kTile + ((mi & 1) * 8 + rr) * kRow;
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt) {
+        const uint32_t rowaddr = stage_base + kTile + (mt * 16 + (mi & 1) * 8 + rr) * kRow;
 #pragma unroll
         for (int dq = 0; dq < 4; ++dq) {
             uint32_t a[4];
             ldmatrix_x4_trans(a, rowaddr + ((uint32_t)((2 * dq + (mi >> 1)) ^ rr) << 4));
 #pragma unroll
             for (int e = 0; e < 4; ++e) a[e] = __byte_perm(a[e], 0u, 0x3120);   // (dim 2g: keys 2t, 2t+1 | dim 2g+1: keys 2t, 2t+1)
-            mma_f16(acc.o[2 * dq], cvt_e4m3x2(a[0]), cvt_e4m3x2(a[0] >> 16), cvt_e4m3x2(a[1]), cvt_e4m3x2(a[1] >> 16), pb0, pb1);
-            mma_f16(acc.o[2 * dq + 1], cvt_e4m3x2(a[2]), cvt_e4m3x2(a[2] >> 16), cvt_e4m3x2(a[3]), cvt_e4m3x2(a[3] >> 16), pb0, pb1);
+            mma_f16(acc.o[2 * dq], cvt_e4m3x2(a[0]), cvt_e4m3x2(a[0] >> 16), cvt_e4m3x2(a[1]), cvt_e4m3x2(a[1] >> 16), pb[mt][0], pb[mt][1]);
+            mma_f16(acc.o[2 * dq + 1], cvt_e4m3x2(a[2]), cvt_e4m3x2(a[2] >> 16), cvt_e4m3x2(a[3]), cvt_e4m3x2(a[3] >> 16), pb[mt][0], pb[mt][1]);
         }
     }
 }
@@ -284,7 +307,7 @@ __device__ __forceinline__ void run_tiles(const Params &p, const Item &it, const
         const char *mt = meta + stage * kMetaBytes;
         const unsigned mask = __ballot_sync(0xffffffffu, reinterpret_cast<const int *>(mt)[lane] >= 0);
         consume_stage(acc, qf, sbase + stage * kStageBytes, reinterpret_cast<const float *>(mt + 32 * 4),
-                      reinterpret_cast<const float *>(mt + 32 * 4 + 16 * 4), mask, p.scale_log2, lane);
+                      reinterpret_cast<const float *>(mt + 32 * 4 + KT * 4), mask, p.scale_log2, lane);
         ++n_done;
     }
     cp_async_wait<0>();
