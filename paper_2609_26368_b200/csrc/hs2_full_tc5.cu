@@ -297,13 +297,17 @@ k_full_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
 // One CTA = TQ = 128/G consecutive queries of one (sequence, KV head) x one chunk of keys.  The MMA
 // computes S^T = K Q^T: 128 keys on M (TMEM lane = key), the TQ x G (query, head) pairs on N = 128,
 // so the G heads of a query are adjacent TMEM columns of one lane and their maximum is thread local.
-// Warp 4 feeds K tiles by TMA (2-stage ring), warp 5 issues the MMAs into two accumulator buffers,
-// warps 0-3 (thread = key) subtract LSE, take the group maximum and write 32 consecutive keys of a
-// strip row per warp instruction.
+// Warp 8 feeds K tiles by TMA (2-stage ring), warp 9 issues the MMAs into two accumulator buffers,
+// warps 0-7 (thread = key; warps w and w+4 share the 32 TMEM lanes of quarter w and take 64 columns each)
+// subtract LSE, take the group maximum and write 32 consecutive keys of a strip row per warp instruction.
+// The epilogue is a chain of TMEM loads and short dependent arithmetic: eight warps per CTA hide its latency
+// where four left the tensor pipe waiting for a free accumulator.
 #ifndef HS2_SC_KCHUNK
 #define HS2_SC_KCHUNK 4096
 #endif
 constexpr int SC_KCHUNK = HS2_SC_KCHUNK;                  // keys per CTA
+constexpr int kScThreads = 320;                           // 8 epilogue warps + TMA warp + MMA warp
+constexpr int kScTmaWarp = 8, kScMmaWarp = 9;
 // shared-memory plan of the score sweep for head_dim D: Q and K tiles are D/64 slices of [128 rows][128 B]
 template <int D>
 struct ScCfg {
@@ -311,7 +315,8 @@ struct ScCfg {
     static constexpr uint32_t kSlice = 128 * 128;                 // one slice: 128 rows of 128 bytes
     static constexpr uint32_t kOffQ = 0;                          // (query, head) rows
     static constexpr uint32_t kOffK = NQ * kSlice;                // 2 stages of key rows
-    static constexpr uint32_t kOffNl = kOffK + 2 * NQ * kSlice;   // float[128]: -LSE/scale per column
+    static constexpr uint32_t kOffAug = kOffK + 2 * NQ * kSlice;  // one extra K step: [128][16] bf16 per operand, 32-byte swizzle
+    static constexpr uint32_t kOffNl = kOffAug + 2 * 4096;        // float[128]: -LSE/scale per column
     static constexpr uint32_t kOffNq = kOffNl + 512;              // int[128]: keys needed per query
     static constexpr uint32_t kOffRow = kOffNq + 512;             // int64[128]: strip row of each query
     static constexpr uint32_t kOffTau = kOffRow + 1024;           // uint32[32]: filter threshold per query (filter mode)
@@ -345,7 +350,7 @@ __device__ __forceinline__ uint32_t order_key_f(float f)
 }
 
 template <int G, int MODE, int D>
-__global__ void __launch_bounds__(kThreads, ScCfg<D>::kMinBlocks)
+__global__ void __launch_bounds__(kScThreads, ScCfg<D>::kMinBlocks)
 k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, const Params p,
              const float *__restrict__ LSE, float *__restrict__ out, int64_t out_stride, int64_t row0, int64_t n_rows,
              int all_visible, int tile_first, int tiles_per_bg, int samp, FilterBuf fb)
@@ -358,6 +363,10 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     constexpr int TQ = 128 / G;                    // queries per CTA
     constexpr int QPC = G <= 32 ? 32 / G : 1;      // queries per 32-column chunk when a group fits a chunk
     constexpr int CPQ = G <= 32 ? 1 : G / 32;      // 32-column chunks per query otherwise
+    constexpr int EW = G <= 64 ? 2 : 1;            // epilogue warps per TMEM lane quarter (a query's columns stay in one warp)
+    constexpr int CPW = 4 / EW;                    // 32-column chunks per epilogue warp
+    constexpr int TQW = TQ / EW;                   // queries per epilogue warp
+    constexpr int kEpiThreads = 128 * EW;
     static_assert(128 % G == 0 && (G <= 32 || G % 32 == 0), "the group's heads tile the 128 columns");
     static_assert(MODE != SC_FILTER || TQ <= 32, "filter mode keeps one pass bit per query");
     extern __shared__ char smem_raw[];
@@ -417,7 +426,23 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         const bool ok = i >= c_lo && i < c_hi;
         // G is the group size rounded up to a tile-able one; columns past the real group hold some other head's
         // (or zero-filled) scores and are taken out of the maximum by -inf
-        s_nl[tid] = !ok ? 0.f : hh < p.G ? -LSE[((int64_t)b * p.Hq + gkv * p.G + hh) * p.Lq + i] / p.scale : -INFINITY;
+        const float nl = !ok ? 0.f : hh < p.G ? -LSE[((int64_t)b * p.Hq + gkv * p.G + hh) * p.Lq + i] / p.scale : -INFINITY;
+        s_nl[tid] = nl;
+        // The subtraction of LSE rides on the tensor cores: one more K step whose key operand is all ones and whose
+        // (query, head) operand holds nl as three bf16 terms (hi + mid + lo carry 24 bits), the other 13 entries zero.
+        // Only the sum over a row's 16 entries matters, so the order of the two 16-byte chunks inside a row is free.
+        const bool fin = fabsf(nl) <= 3.0e38f;
+        const __nv_bfloat16 hi = __float2bfloat16_rn(nl);
+        const float r1 = fin ? nl - __bfloat162float(hi) : 0.f;
+        const __nv_bfloat16 mid = __float2bfloat16_rn(r1);
+        const __nv_bfloat16 lo = __float2bfloat16_rn(r1 - __bfloat162float(mid));
+        uint4 c0;
+        c0.x = (uint32_t)__bfloat16_as_ushort(hi) | ((uint32_t)__bfloat16_as_ushort(mid) << 16);
+        c0.y = (uint32_t)__bfloat16_as_ushort(lo);
+        c0.z = 0u; c0.w = 0u;
+        uint4 *qaug = reinterpret_cast<uint4 *>(smem + S::kOffAug + 4096 + tid * 32);
+        qaug[0] = c0;
+        qaug[1] = make_uint4(0u, 0u, 0u, 0u);
         if (hh == 0) {
             s_nq[t] = ok ? n_of(i) : 0;
             s_row[t] = ok ? (bg_row0 + i - row0) : -1;
@@ -427,16 +452,19 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             }
         }
     }
+    if (tid < 256)   // the all-ones key operand of the extra step
+        reinterpret_cast<uint4 *>(smem + S::kOffAug)[tid] = make_uint4(0x3f803f80u, 0x3f803f80u, 0x3f803f80u, 0x3f803f80u);
+    fence_proxy_async();   // the tensor cores read what these threads wrote
     if (tid == 0) {
         *abort_flag = 0;
         mbar_init(bar(SQ_FULL), 1);
         mbar_init(bar(SK_FULL0), 1); mbar_init(bar(SK_FULL1), 1);
         mbar_init(bar(SK_EMPTY0), 1); mbar_init(bar(SK_EMPTY1), 1);
         mbar_init(bar(ACC_FULL0), 1); mbar_init(bar(ACC_FULL1), 1);
-        mbar_init(bar(ACC_FREE0), 128); mbar_init(bar(ACC_FREE1), 128);
+        mbar_init(bar(ACC_FREE0), kEpiThreads); mbar_init(bar(ACC_FREE1), kEpiThreads);
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
-    if (warp == 5) {
+    if (warp == kScMmaWarp) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
     }
@@ -445,7 +473,7 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
 
-    if (warp == 4) {
+    if (warp == kScTmaWarp) {
         if (elect_one()) {
             mbar_expect_tx(bar(SQ_FULL), kStage);
 #pragma unroll
@@ -467,7 +495,7 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait(bar(SQ_FULL), 0); ++it) {}
             }
         }
-    } else if (warp == 5) {
+    } else if (warp == kScMmaWarp) {
         if (elect_one()) {
             constexpr uint32_t id = idesc(128, 128, 0);
             bool ok = mbar_wait(bar(SQ_FULL), 0, abort_flag);
@@ -482,13 +510,30 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                     const uint32_t off = (ks >> 2) * S::kSlice + (ks & 3) * 32;
                     umma(tmem + st * 128, smem_desc(ka + off, 16, 1024), smem_desc(qa + off, 16, 1024), id, ks > 0);
                 }
+                umma(tmem + st * 128, smem_desc_sw32(sbase + S::kOffAug, 256), smem_desc_sw32(sbase + S::kOffAug + 4096, 256), id, 1);   // - LSE / scale
                 umma_commit(bar(SK_EMPTY0 + st));
                 umma_commit(bar(ACC_FULL0 + st));
             }
         }
-    } else {
-        const int row = tid;   // key inside the tile = TMEM lane
-        const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
+    } else if (warp < 4 * EW) {
+        const int quarter = warp & 3, half = warp >> 2;
+        const int row = quarter * 32 + lane;   // key inside the tile = TMEM lane
+        const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16);
+        const int q_first = half * TQW;        // this warp's queries: q_first .. q_first + TQW - 1
+        const unsigned lt_mask = (1u << lane) - 1u;
+        // per-query constants in registers when a warp owns few queries (they are read once per score otherwise)
+        constexpr bool kHoist = TQW <= 8;
+        int nq_r[kHoist ? TQW : 1];
+        float *orow_r[kHoist && MODE != SC_FILTER ? TQW : 1];
+        uint32_t tau_r[kHoist && MODE == SC_FILTER ? TQW : 1];
+        if (kHoist) {
+#pragma unroll
+            for (int q = 0; q < TQW; ++q) {
+                nq_r[q] = s_nq[q_first + q];
+                if (MODE != SC_FILTER) orow_r[q] = out + s_row[q_first + q] * out_stride;   // never used when nq is 0
+                if (MODE == SC_FILTER) tau_r[q] = s_tau[q_first + q];
+            }
+        }
         bool alive = true;
         for (int t = 0; t < ntile; ++t) {
             const int ab = t & 1;
@@ -497,45 +542,45 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             tc_fence_after();
             const int key = (kt0 + t) * kstep * 128 + row;
             const int col = MODE == SC_SAMPLE ? (kt0 + t) * 128 + row : key;
-            float aval[MODE == SC_FILTER ? TQ : 1];
-            unsigned passbits = 0;
+            float aval[MODE == SC_FILTER ? TQW : 1];
+            unsigned passbits = 0;     // bit q: the score of query q_first + q passes the filter
             float carry = -INFINITY;   // running group maximum when a group spans several chunks
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
+            for (int c = 0; c < CPW; ++c) {
+                const int cc = half * CPW + c;   // 32-column chunk of the accumulator
                 float v[32];
                 if (alive) {
-                    tmem_ld32(lane_base + ab * 128 + c * 32, v);
+                    tmem_ld32(lane_base + ab * 128 + cc * 32, v);
                     tmem_wait_ld();
                 } else {
 #pragma unroll
                     for (int e = 0; e < 32; ++e) v[e] = 0.f;
-                }
-                const float4 *nl4 = reinterpret_cast<const float4 *>(s_nl + c * 32);
-#pragma unroll
-                for (int e4 = 0; e4 < 8; ++e4) {
-                    const float4 n4 = nl4[e4];
-                    v[4 * e4] += n4.x; v[4 * e4 + 1] += n4.y; v[4 * e4 + 2] += n4.z; v[4 * e4 + 3] += n4.w;
                 }
 #pragma unroll
                 for (int q = 0; q < QPC; ++q) {
                     constexpr int W = G <= 32 ? G : 32;   // columns of this chunk that belong to one query
                     float a = v[q * W];
 #pragma unroll
-                    for (int hh = 1; hh < W; ++hh) a = fmaxf(a, v[q * W + hh]);
+                    for (int hh = 1; hh + 1 < W; hh += 2) a = max3(a, v[q * W + hh], v[q * W + hh + 1]);
+                    if (W % 2 == 0 && W > 1) a = fmaxf(a, v[q * W + W - 1]);
                     if (CPQ > 1) {
                         carry = fmaxf(carry, a);
                         if ((c + 1) % CPQ != 0) continue;   // more chunks of this query follow
                         a = carry;
                         carry = -INFINITY;
                     }
-                    const int tq = CPQ > 1 ? c / CPQ : c * QPC + q;
+                    const int ql = CPQ > 1 ? c / CPQ : c * QPC + q;   // query inside this warp's set
+                    const int tq = q_first + ql;
                     const float av = a * p.scale;
+                    const int nq = kHoist ? nq_r[kHoist ? ql : 0] : s_nq[tq];
                     if (MODE == SC_FILTER) {
-                        aval[tq] = av;
-                        const bool pass = alive && key < s_nq[tq] && order_key_f(av) >= s_tau[tq];
-                        passbits |= (pass ? 1u : 0u) << tq;
-                    } else {
-                        if (key < s_nq[tq]) out[s_row[tq] * out_stride + col] = av;
+                        aval[ql] = av;
+                        const uint32_t tau = kHoist ? tau_r[kHoist ? ql : 0] : s_tau[tq];
+                        const bool pass = alive && key < nq && order_key_f(av) >= tau;
+                        passbits |= (pass ? 1u : 0u) << ql;
+                    } else if (key < nq) {
+                        if (kHoist) orow_r[kHoist ? ql : 0][col] = av;
+                        else out[s_row[tq] * out_stride + col] = av;
                     }
                 }
             }
@@ -544,30 +589,45 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 mbar_arrive(bar(ACC_FREE0 + ab));
             }
             if (MODE == SC_FILTER) {
-                // append in no particular order: one shared-memory counter per query.  Only a few percent of the
-                // scores pass, so a plain atomic per passing element is cheaper than any warp-level aggregation.
+                // Append in no particular order, one shared-memory counter per query.  Per warp and tile: one ballot
+                // per query, lane q reserves the warp's slots of query q with a single atomic (distinct addresses,
+                // one instruction), and every passing lane takes its rank inside the ballot.  A per-element atomic
+                // serialised the lanes of a query and cost one atomic round trip per query and tile.
+                if (__any_sync(0xffffffffu, passbits != 0u)) {
+                    unsigned masks[TQW];
+                    unsigned mine = 0u;
 #pragma unroll
-                for (int q = 0; q < TQ; ++q) {
-                    if ((passbits >> q) & 1u) {
-                        const int pos = atomicAdd(&s_cntw[q], 1);
-                        if (pos < fb.cap) {
-                            const int64_t o = s_row[q] * fb.cap + pos;
-                            fb.cand_a[o] = aval[q];
-                            fb.cand_j[o] = key;
+                    for (int q = 0; q < TQW; ++q) {
+                        masks[q] = __ballot_sync(0xffffffffu, (passbits >> q) & 1u);
+                        if (lane == q) mine = masks[q];
+                    }
+                    int base = 0;
+                    if (mine != 0u) base = atomicAdd(&s_cntw[q_first + lane], __popc(mine));
+#pragma unroll
+                    for (int q = 0; q < TQW; ++q) {
+                        if (masks[q] == 0u) continue;   // uniform
+                        const int bq = __shfl_sync(0xffffffffu, base, q);
+                        if ((passbits >> q) & 1u) {
+                            const int pos = bq + __popc(masks[q] & lt_mask);
+                            if (pos < fb.cap) {
+                                const int64_t o = s_row[q_first + q] * fb.cap + pos;
+                                fb.cand_a[o] = aval[q];
+                                fb.cand_j[o] = key;
+                            }
                         }
                     }
                 }
             }
         }
         if (MODE == SC_FILTER) {
-            asm volatile("bar.sync 1, 128;\n" ::: "memory");   // the four epilogue warps: all appends are counted
+            asm volatile("bar.sync 1, %0;\n" ::"n"(kEpiThreads) : "memory");   // the epilogue warps: all appends are counted
             if (tid < TQ && s_row[tid] >= 0) fb.count[s_row[tid]] = (alive && !*abort_flag) ? s_cntw[tid] : -1;   // -1: gave up
         }
     }
     __syncwarp();
     tc_fence_before();
     __syncthreads();
-    if (warp == 5) {
+    if (warp == kScMmaWarp) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(kTmemCols) : "memory");
     }
@@ -695,7 +755,7 @@ cudaError_t launch_sc(const CUtensorMap &tmQ, const CUtensorMap &tmK, const Para
     const int key_tiles = (p.Lk + 128 * samp - 1) / (128 * samp);
     const unsigned gx = MODE == SC_FILTER ? 1u : (unsigned)((key_tiles + SC_KCHUNK / 128 - 1) / (SC_KCHUNK / 128));
     dim3 grid(gx, (unsigned)gy);
-    k_scores_tc5<G, MODE, D><<<grid, kThreads, ScCfg<D>::kSmemBytes, st>>>(tmQ, tmK, p, LSE, out, out_stride, row0, n_rows, all_visible ? 1 : 0,
+    k_scores_tc5<G, MODE, D><<<grid, kScThreads, ScCfg<D>::kSmemBytes, st>>>(tmQ, tmK, p, LSE, out, out_stride, row0, n_rows, all_visible ? 1 : 0,
                                                                (int)t_first, tiles_per_bg, samp, fb);
     count_launch();
     return cudaGetLastError();

@@ -69,6 +69,24 @@ __device__ __forceinline__ uint64_t smem_desc(uint32_t addr, uint32_t lbo_bytes,
     d |= (uint64_t)2 << 61;    // SWIZZLE_128B
     return d;
 }
+// the same for a K-major operand of exactly 16 bf16 per row (one MMA K step) in the 32-byte swizzle: rows of 32
+// bytes, 8-row groups `sbo_bytes` (256 when packed) apart
+__device__ __forceinline__ uint64_t smem_desc_sw32(uint32_t addr, uint32_t sbo_bytes)
+{
+    uint64_t d = 0;
+    d |= (uint64_t)((addr >> 4) & 0x3fffu);
+    d |= (uint64_t)1 << 16;
+    d |= (uint64_t)((sbo_bytes >> 4) & 0x3fffu) << 32;
+    d |= (uint64_t)1 << 46;    // descriptor version
+    d |= (uint64_t)6 << 61;    // SWIZZLE_32B
+    return d;
+}
+__device__ __forceinline__ float max3(float a, float b, float c)
+{
+    float r;
+    asm("max.f32 %0, %1, %2, %3;\n" : "=f"(r) : "f"(a), "f"(b), "f"(c));
+    return r;
+}
 // instruction descriptor, kind::f16: bf16 x bf16 -> fp32, A K-major, B K-major (0) or MN-major (1)
 __host__ __device__ constexpr uint32_t idesc(int M, int N, int b_mn_major)
 {
