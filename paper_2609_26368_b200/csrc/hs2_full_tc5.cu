@@ -1,18 +1,23 @@
-// Full causal attention on the 5th-generation tensor cores (tcgen05 + TMEM), bf16, head_dim 128
+// Full causal attention on the 5th-generation tensor cores (tcgen05 + TMEM), bf16, head_dim 128 or 256
 // (Section 3.4: the full-attention layer; NoPE, Section 4.1).
 //
-// One CTA = 128 queries of one head (MMA M = 128), 192 threads, two CTAs per SM so that one CTA's
-// softmax overlaps the other's tensor work:
-//   warp 4   TMA producer: Q once, then K/V tiles of 64 keys into a 2-stage ring.  Every tile is a
-//            pair of 128-byte-swizzled halves ([rows][64 dims]), the canonical UMMA operand layout.
-//   warp 5   MMA issuer: S = Q K^T (M128 N64 K128, eight tcgen05.mma of K=16) into one of two S
-//            buffers in TMEM, and O += P V (M128 N128 K64, V as an MN-major B operand) into TMEM.
-//   warps 0-3 one thread per query row: tcgen05.ld of the S row, causal mask, online softmax in the
-//            base-2 domain with a lazily updated row maximum (O in TMEM is rescaled only when the
-//            maximum grows by more than 2^8), P written as bf16 into swizzled shared memory.
-// TMEM: columns 0-63 / 64-127 the two S buffers, 128-255 the O accumulator (fp32, lane = query row).
-// Every mbarrier wait is bounded; a wait that runs out sets a bit in a device error word, makes the
-// CTA abandon its loops, and the CTA still frees its TMEM before it returns.
+// One CTA = 128 queries of one head (MMA M = 128), 320 threads, two CTAs per SM at head_dim 128 so that one
+// CTA's softmax overlaps the other's tensor work:
+//   warp 8   TMA producer: Q once, then K/V tiles of 64 keys into a 2-stage ring.  Every tile is a set of
+//            128-byte-swizzled slices ([rows][64 dims]), the canonical UMMA operand layout.
+//   warp 9   MMA issuer: S = Q K^T (M128 N64 K=D) into one of two S buffers in TMEM, and O += P V
+//            (M128 N=D K64, P as the tensor-memory A operand, V as an MN-major B operand) into TMEM.
+//   warps 0-7 two threads per query row (warps w and w+4 share the 32 TMEM lanes of quarter w and take 32 keys
+//            of a tile each): tcgen05.ld of the half row, causal mask, the tile maximum agreed through shared
+//            memory and a named pair barrier, online softmax in the base-2 domain with a lazily updated row
+//            maximum (O in TMEM is rescaled only when the maximum grows by more than 2^8), P written as bf16
+//            pairs over the scores it came from (tcgen05.st).  Eight warps instead of four: the softmax is a
+//            chain of TMEM round trips and MUFU latencies, and four warps per scheduler hide it where two did not.
+// TMEM: columns 0-63 / 64-127 the two S buffers (P of a tile in the first 32 columns of its buffer), then the
+// O accumulator (fp32, lane = query row).
+// Every mbarrier wait is bounded; a wait that runs out sets a bit in a device error word, makes the CTA abandon
+// its loops (partners leave together through the predicate of their pair barrier), and the CTA still frees its
+// TMEM before it returns.
 #include <cuda.h>
 
 #include "hs2_common.cuh"
@@ -25,7 +30,6 @@ __device__ unsigned g_tc5_error;   // bit 0: an mbarrier wait ran out; bit 1: sh
 namespace {
 
 constexpr int BM = 128, BN = 64, HD = 128;
-constexpr int kThreads = 192;
 constexpr uint32_t kBarBytes = 128;
 constexpr uint32_t kAlignSlack = 896;             // the dynamic window is at least 128-byte aligned
 constexpr uint32_t kTmemCols = 256;               // score kernels, attention at head_dim 128
@@ -39,15 +43,24 @@ struct FaCfg {
     static constexpr uint32_t kOffQ = 0;
     static constexpr uint32_t kOffK = kOffQ + kQBytes;        // 2 stages
     static constexpr uint32_t kOffV = kOffK + 2 * kKVStage;   // 2 stages
-    static constexpr uint32_t kOffP = kOffV + 2 * kKVStage;   // 128 rows x 64 keys bf16, K-major
-    static constexpr uint32_t kOffBar = kOffP + BM * 128;
-    static constexpr uint32_t kSmemBytes = kOffBar + kBarBytes + kAlignSlack;   // 115712 at D=128: two CTAs per SM
+    static constexpr uint32_t kOffX = kOffV + 2 * kKVStage;   // exchange between the two threads of a row: 6 x 128 floats
+    static constexpr uint32_t kOffBar = kOffX + 6 * BM * 4;
+    static constexpr uint32_t kSmemBytes = kOffBar + kBarBytes + kAlignSlack;   // 102400 at D=128: two CTAs per SM
     static constexpr uint32_t kTmem = D <= 128 ? 256 : 512;  // 2 x 64 score columns + D output columns, a power of two
     static constexpr int kMinBlocks = D <= 128 ? 2 : 1;
+    template <int HV> static constexpr int threads() { return 128 * HV + 64; }   // softmax warps + TMA warp + MMA warp
 };
+// Threads per query row.  Measured on B200: at head_dim 128 (two CTAs per SM) and at head_dim 256 (one CTA per SM).
+#ifndef HS2_FA_HV128
+#define HS2_FA_HV128 1
+#endif
+#ifndef HS2_FA_HV256
+#define HS2_FA_HV256 1
+#endif
+template <int D> struct FaShape { static constexpr int HV = D <= 128 ? HS2_FA_HV128 : HS2_FA_HV256; };
 constexpr float kRescaleThreshold = 8.f;          // log2 units
 
-enum Bar { Q_FULL = 0, KV_FULL0, KV_FULL1, KV_EMPTY0, KV_EMPTY1, S_FULL0, S_FULL1, S_FREE0, S_FREE1, P_FULL, PV_DONE, N_BARS };
+enum Bar { Q_FULL = 0, K_FULL0, K_FULL1, V_FULL0, V_FULL1, S_FULL0, S_FULL1, S_FREE0, S_FREE1, P_FULL0, P_FULL1, PV_DONE0, PV_DONE1, N_BARS };
 
 using namespace tc5;
 
@@ -57,8 +70,8 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     return tc5::mbar_wait(bar, parity, abort_flag, &g_tc5_error);
 }
 
-template <int D>
-__global__ void __launch_bounds__(kThreads, FaCfg<D>::kMinBlocks)
+template <int D, int HV>
+__global__ void __launch_bounds__(FaCfg<D>::template threads<HV>(), FaCfg<D>::kMinBlocks)
 k_full_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
            const __grid_constant__ CUtensorMap tmV, const Params p, __nv_bfloat16 *__restrict__ O,
            float *__restrict__ LSE)
@@ -66,7 +79,10 @@ k_full_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
     using F = FaCfg<D>;
     constexpr int NQ = F::NQ;
     constexpr uint32_t kQBytes = F::kQBytes, kKVStage = F::kKVStage, kOffQ = F::kOffQ, kOffK = F::kOffK, kOffV = F::kOffV,
-                       kOffP = F::kOffP, kOffBar = F::kOffBar, kTmemFa = F::kTmem;
+                       kOffX = F::kOffX, kOffBar = F::kOffBar, kTmemFa = F::kTmem;
+    constexpr int kTmaWarp = 4 * HV, kMmaWarp = 4 * HV + 1;   // behind the softmax warps
+    constexpr int EPT = BN / HV;                              // scores per softmax thread and tile
+    constexpr int kSoftmaxThreads = 128 * HV;
     extern __shared__ char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t pad = (1024u - (raw & 1023u)) & 1023u;
@@ -81,7 +97,7 @@ k_full_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
     volatile int *abort_flag = reinterpret_cast<volatile int *>(smem + kOffBar + N_BARS * 8 + 4);
     auto bar = [&](int i) { return bars + 8u * i; };
 
-    const int tid = threadIdx.x, warp = tid >> 5;
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int mblk = gridDim.x - 1 - blockIdx.x;   // long rows first
     const int h = blockIdx.y % p.Hq, b = blockIdx.y / p.Hq;
     const int gkv = h / p.G;
@@ -95,15 +111,15 @@ k_full_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
     if (tid == 0) {
         *abort_flag = 0;
         mbar_init(bar(Q_FULL), 1);
-        mbar_init(bar(KV_FULL0), 1); mbar_init(bar(KV_FULL1), 1);
-        mbar_init(bar(KV_EMPTY0), 1); mbar_init(bar(KV_EMPTY1), 1);
+        mbar_init(bar(K_FULL0), 1); mbar_init(bar(K_FULL1), 1);
+        mbar_init(bar(V_FULL0), 1); mbar_init(bar(V_FULL1), 1);
         mbar_init(bar(S_FULL0), 1); mbar_init(bar(S_FULL1), 1);
-        mbar_init(bar(S_FREE0), 128); mbar_init(bar(S_FREE1), 128);
-        mbar_init(bar(P_FULL), 128);
-        mbar_init(bar(PV_DONE), 1);
+        mbar_init(bar(S_FREE0), kSoftmaxThreads); mbar_init(bar(S_FREE1), kSoftmaxThreads);
+        mbar_init(bar(P_FULL0), kSoftmaxThreads); mbar_init(bar(P_FULL1), kSoftmaxThreads);
+        mbar_init(bar(PV_DONE0), 1); mbar_init(bar(PV_DONE1), 1);
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
-    if (warp == 5) {   // TMEM allocation is a warp-wide operation
+    if (warp == kMmaWarp) {   // TMEM allocation is a warp-wide operation
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(tmem_slot)), "r"(kTmemFa) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
     }
@@ -112,39 +128,46 @@ k_full_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
     tc_fence_after();
     const uint32_t tmem = *tmem_slot;
 
-    if (warp == 4) {
+    if (warp == kTmaWarp) {
         // ------------------------------------------------ TMA producer
         if (elect_one() && nblk > 0) {
             mbar_expect_tx(bar(Q_FULL), kQBytes);
 #pragma unroll
             for (int sl = 0; sl < NQ; ++sl) tma_load_4d(sbase + kOffQ + sl * BM * 128, &tmQ, bar(Q_FULL), 64 * sl, h, i0, b);
-            int issued = 0;
+            // K and V travel in rings of their own (two stages each).  A K stage is free again as soon as Q K^T of the
+            // tile two back has run (the event S_FULL of that tile), a V stage when its P V has (PV_DONE): K runs a whole
+            // tile ahead of V, so the next scores are in tensor memory before the softmax asks for them.
+            int k_issued = 0, v_issued = 0;
             for (int j = 0; j < nblk; ++j) {
                 const int st = j & 1;
-                if (!mbar_wait(bar(KV_EMPTY0 + st), ((j >> 1) & 1) ^ 1, abort_flag)) break;
-                issued = j + 1;
-                mbar_expect_tx(bar(KV_FULL0 + st), 2 * kKVStage);
+                if (j >= 2 && !mbar_wait(bar(S_FULL0 + st), ((j - 2) >> 1) & 1, abort_flag)) break;
+                mbar_expect_tx(bar(K_FULL0 + st), kKVStage);
                 const uint32_t kdst = sbase + kOffK + st * kKVStage, vdst = sbase + kOffV + st * kKVStage;
 #pragma unroll
-                for (int sl = 0; sl < NQ; ++sl) {
-                    tma_load_4d(kdst + sl * BN * 128, &tmK, bar(KV_FULL0 + st), 64 * sl, gkv, j * BN, b);
-                    tma_load_4d(vdst + sl * BN * 128, &tmV, bar(KV_FULL0 + st), 64 * sl, gkv, j * BN, b);
-                }
+                for (int sl = 0; sl < NQ; ++sl) tma_load_4d(kdst + sl * BN * 128, &tmK, bar(K_FULL0 + st), 64 * sl, gkv, j * BN, b);
+                k_issued = j + 1;
+                if (j >= 2 && !mbar_wait(bar(PV_DONE0 + st), ((j - 2) >> 1) & 1, abort_flag)) break;
+                mbar_expect_tx(bar(V_FULL0 + st), kKVStage);
+#pragma unroll
+                for (int sl = 0; sl < NQ; ++sl) tma_load_4d(vdst + sl * BN * 128, &tmV, bar(V_FULL0 + st), 64 * sl, gkv, j * BN, b);
+                v_issued = j + 1;
             }
             if (*abort_flag) {   // leaving early: let the copies already in flight land before the CTA goes away
-                for (int j = max(0, issued - 2); j < issued; ++j)
-                    for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait(bar(KV_FULL0 + (j & 1)), (j >> 1) & 1); ++it) {}
+                for (int j = max(0, k_issued - 2); j < k_issued; ++j)
+                    for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait(bar(K_FULL0 + (j & 1)), (j >> 1) & 1); ++it) {}
+                for (int j = max(0, v_issued - 2); j < v_issued; ++j)
+                    for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait(bar(V_FULL0 + (j & 1)), (j >> 1) & 1); ++it) {}
                 for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait(bar(Q_FULL), 0); ++it) {}
             }
         }
-    } else if (warp == 5) {
+    } else if (warp == kMmaWarp) {
         // ------------------------------------------------ MMA issuer
         if (elect_one() && nblk > 0) {
             constexpr uint32_t idS = idesc(BM, BN, 0), idPV = idesc(BM, D, 1);
             bool ok = mbar_wait(bar(Q_FULL), 0, abort_flag);
             auto issue_s = [&](int j) -> bool {
                 const int st = j & 1, ph = (j >> 1) & 1;
-                if (!mbar_wait(bar(KV_FULL0 + st), ph, abort_flag)) return false;
+                if (!mbar_wait(bar(K_FULL0 + st), ph, abort_flag)) return false;
                 if (!mbar_wait(bar(S_FREE0 + st), ph ^ 1, abort_flag)) return false;
                 tc_fence_after();
                 const uint32_t qa = sbase + kOffQ, ka = sbase + kOffK + st * kKVStage;
@@ -161,106 +184,141 @@ k_full_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
             ok = ok && issue_s(0);
             for (int j = 0; ok && j < nblk; ++j) {
                 if (j + 1 < nblk && !issue_s(j + 1)) break;
-                if (!mbar_wait(bar(P_FULL), j & 1, abort_flag)) break;
-                tc_fence_after();
                 const int st = j & 1;
-                const uint32_t pa = sbase + kOffP, va = sbase + kOffV + st * kKVStage;
+                if (!mbar_wait(bar(V_FULL0 + st), (j >> 1) & 1, abort_flag)) break;
+                if (!mbar_wait(bar(P_FULL0 + st), (j >> 1) & 1, abort_flag)) break;
+                tc_fence_after();
+                const uint32_t va = sbase + kOffV + st * kKVStage;
 #pragma unroll
                 for (int kk = 0; kk < 4; ++kk) {   // 16 keys per instruction
-                    const uint64_t da = smem_desc(pa + kk * 32, 16, 1024);
+                    // P: in tensor memory, over the first 32 columns of the score buffer it was computed from
+                    // (16 keys = 8 columns of bf16 pairs); the in-order tensor pipe runs Q K^T of tile j+2, which
+                    // overwrites that buffer, after this instruction
                     // V: MN-major, 64-dim halves BN*128 bytes apart (leading offset), 8-key groups 1024 bytes apart
                     const uint64_t db = smem_desc(va + kk * 2048, BN * 128, 1024);
-                    umma(tmem + 2 * BN, da, db, idPV, (j > 0 || kk > 0) ? 1u : 0u);
+                    umma_ts(tmem + 2 * BN, tmem + st * BN + kk * 8, db, idPV, (j > 0 || kk > 0) ? 1u : 0u);
                 }
-                umma_commit(bar(KV_EMPTY0 + st));
-                umma_commit(bar(PV_DONE));
+                umma_commit(bar(PV_DONE0 + st));
             }
         }
     } else {
-        // ------------------------------------------------ softmax: one thread per query row
-        const int row = tid;                       // 0..127, TMEM lane
+        // ------------------------------------------------ softmax: HV threads per query row, BN / HV keys of a tile each
+        const int quarter = warp & 3, half = HV == 2 ? warp >> 2 : 0;
+        const int row = quarter * 32 + lane;       // 0..127, TMEM lane
         const int i = i0 + row;
         const int prow = pos0 + row;
-        const uint32_t lane_base = tmem + ((uint32_t)(warp * 32) << 16);
+        const uint32_t lane_base = tmem + ((uint32_t)(quarter * 32) << 16);
+        float *s_mx = reinterpret_cast<float *>(smem + kOffX);   // [tile parity][half][row] raw maximum of the half tile
+        float *s_l = s_mx + 4 * BM;                              // [half][row] partial denominators
+        const int pair_bar = 1 + quarter;          // named barrier of the two warps that share these 32 rows
+        constexpr int OCH = D / 32 / HV;           // 32-column chunks of the O row this thread rescales and stores
         float m_used = -INFINITY, l = 0.f;
-        bool alive = true;
-        for (int j = 0; j < nblk && alive; ++j) {
+        bool ok = true;
+        float s[EPT];
+        for (int j = 0; j < nblk; ++j) {
             const int sb = j & 1;
-            if (!__all_sync(0xffffffffu, mbar_wait(bar(S_FULL0 + sb), (j >> 1) & 1, abort_flag))) { alive = false; break; }
-            tc_fence_after();
-            float s[64];
-            tmem_ld32(lane_base + sb * BN, *reinterpret_cast<float (*)[32]>(&s[0]));
-            tmem_ld32(lane_base + sb * BN + 32, *reinterpret_cast<float (*)[32]>(&s[32]));
-            tmem_wait_ld();
-            tc_fence_before();
-            mbar_arrive(bar(S_FREE0 + sb));
-            const int j0 = j * BN;
-            // raw-score maximum; only tiles that touch the diagonal or the end of the cache pay for masking
-            if ((j0 + BN - 1 > pos0) || (j0 + BN > kvl)) {
-#pragma unroll
-                for (int e = 0; e < 64; ++e)
-                    if (j0 + e > prow || j0 + e >= kvl) s[e] = -INFINITY;
+            if (ok && !__all_sync(0xffffffffu, mbar_wait(bar(S_FULL0 + sb), (j >> 1) & 1, abort_flag))) ok = false;
+            float m_raw = -INFINITY;
+            if (ok) {   // this thread's scores into registers; the score buffer is then free for Q K^T of tile j+2
+                tc_fence_after();
+                if constexpr (EPT == 64) {
+                    tmem_ld32(lane_base + sb * BN, *reinterpret_cast<float (*)[32]>(&s[0]));
+                    tmem_ld32(lane_base + sb * BN + 32, *reinterpret_cast<float (*)[32]>(&s[32]));
+                } else {
+                    tmem_ld32(lane_base + sb * BN + half * 32, s);
+                }
+                tmem_wait_ld();
+                tc_fence_before();
+                mbar_arrive(bar(S_FREE0 + sb));
             }
-            // four independent chains: one chain of 64 dependent maxima is 250 cycles of latency per tile
-            float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
+            if (ok) {
+                const int j0 = j * BN + half * EPT;
+                // raw-score maximum; only tiles that touch the diagonal or the end of the cache pay for masking
+                if ((j0 + EPT - 1 > pos0) || (j0 + EPT > kvl)) {
 #pragma unroll
-            for (int e = 0; e < 64; e += 4) {
-                mx0 = fmaxf(mx0, s[e]); mx1 = fmaxf(mx1, s[e + 1]); mx2 = fmaxf(mx2, s[e + 2]); mx3 = fmaxf(mx3, s[e + 3]);
+                    for (int e = 0; e < EPT; ++e)
+                        if (j0 + e > prow || j0 + e >= kvl) s[e] = -INFINITY;
+                }
+                // four independent chains of 3-input maxima
+                float mx0 = s[0], mx1 = s[1], mx2 = s[2], mx3 = s[3];
+#pragma unroll
+                for (int e = 4; e + 8 <= EPT; e += 8) {
+                    mx0 = max3(mx0, s[e], s[e + 4]); mx1 = max3(mx1, s[e + 1], s[e + 5]);
+                    mx2 = max3(mx2, s[e + 2], s[e + 6]); mx3 = max3(mx3, s[e + 3], s[e + 7]);
+                }
+                mx0 = fmaxf(mx0, s[EPT - 4]); mx1 = fmaxf(mx1, s[EPT - 3]); mx2 = fmaxf(mx2, s[EPT - 2]); mx3 = fmaxf(mx3, s[EPT - 1]);
+                m_raw = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
             }
-            const float m_raw = fmaxf(fmaxf(mx0, mx1), fmaxf(mx2, mx3));
+            if (HV == 2) {
+                // the two halves of a row agree on the tile's maximum (and leave the loop together after a failed wait)
+                s_mx[((j & 1) * 2 + half) * BM + row] = m_raw;
+                if (!group_all(pair_bar, 64, ok)) { ok = false; break; }
+                m_raw = fmaxf(m_raw, s_mx[((j & 1) * 2 + (half ^ 1)) * BM + row]);
+            } else if (!ok) {
+                break;
+            }
             const float m_blk = m_raw * p.scale_log2;                 // the scale is positive
             const bool need = m_blk > m_used + kRescaleThreshold;   // also true for the first finite block
             const float m_new = need ? m_blk : m_used;
             const float corr = need ? exp2f(m_used - m_new) : 1.f;  // 0 when nothing was accumulated yet
-            if (j > 0) {
-                if (!__all_sync(0xffffffffu, mbar_wait(bar(PV_DONE), (j - 1) & 1, abort_flag))) { alive = false; break; }
-                tc_fence_after();
-                if (__any_sync(0xffffffffu, need)) {   // rescale the O rows of this warp (a warp-wide TMEM access)
-#pragma unroll
-                    for (int c = 0; c < D / 32; ++c) {
-                        float o[32];
-                        tmem_ld32(lane_base + 2 * BN + c * 32, o);
-                        tmem_wait_ld();
-#pragma unroll
-                        for (int e = 0; e < 32; ++e) o[e] *= corr;
-                        tmem_st32(lane_base + 2 * BN + c * 32, o);
-                    }
-                    tmem_wait_st();
+            // P of this tile goes to the score buffer it came from, which P V of tile j-2 has left (Q K^T of this tile
+            // ran behind it in the tensor pipe), so only a rescale of O has to wait for P V of tile j-1.  One barrier
+            // per tile parity: P V of tile j-3 is certainly complete here, so the awaited phase is never ambiguous.
+            if (j > 0 && __any_sync(0xffffffffu, need)) {
+                if (!__all_sync(0xffffffffu, mbar_wait(bar(PV_DONE0 + ((j - 1) & 1)), ((j - 1) >> 1) & 1, abort_flag))) {
+                    ok = false;
+                    if (HV == 2) continue;   // the partner learns at the next pair barrier
+                    break;
                 }
+                tc_fence_after();
+#pragma unroll
+                for (int c = 0; c < OCH; ++c) {   // this thread's columns of the O row (a warp-wide TMEM access)
+                    float o[32];
+                    const uint32_t oc = lane_base + 2 * BN + (half * OCH + c) * 32;
+                    tmem_ld32(oc, o);
+                    tmem_wait_ld();
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) o[e] *= corr;
+                    tmem_st32(oc, o);
+                }
+                tmem_wait_st();
             }
             l *= corr;
             m_used = m_new;
             const float neg_m = m_used == -INFINITY ? 0.f : -m_used;
-            uint32_t pk[32];
+            uint32_t pk[EPT / 2];
             float l0 = 0.f, l1 = 0.f;
 #pragma unroll
-            for (int e = 0; e < 64; e += 2) {
+            for (int e = 0; e < EPT; e += 2) {
                 const float p0 = exp2f(fmaf(s[e], p.scale_log2, neg_m));       // -inf stays -inf -> 0
                 const float p1 = exp2f(fmaf(s[e + 1], p.scale_log2, neg_m));
                 l0 += p0; l1 += p1;
                 pk[e >> 1] = pack_bf16(p0, p1);
             }
             l += l0 + l1;
-            char *prow_ptr = smem + kOffP + row * 128;
-#pragma unroll
-            for (int c = 0; c < 8; ++c)   // 8 keys = one 16-byte chunk, chunk position XOR (row & 7)
-                *reinterpret_cast<uint4 *>(prow_ptr + ((c ^ (row & 7)) << 4)) = make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]);
-            fence_proxy_async();
+            // P replaces the scores it came from
+            if constexpr (EPT == 64) tmem_st32u(lane_base + sb * BN, pk);
+            else tmem_st16u(lane_base + sb * BN + half * (EPT / 2), pk);
+            tmem_wait_st();
             tc_fence_before();
-            mbar_arrive(bar(P_FULL));
+            mbar_arrive(bar(P_FULL0 + sb));
         }
         // ------------------------------------------------ epilogue
-        bool have_o = alive && nblk > 0;
-        if (have_o) have_o = mbar_wait(bar(PV_DONE), (nblk - 1) & 1, abort_flag);
-        have_o = __all_sync(0xffffffffu, have_o);   // TMEM loads below are warp-wide
+        bool have_o = ok && nblk > 0;
+        if (have_o) have_o = __all_sync(0xffffffffu, mbar_wait(bar(PV_DONE0 + ((nblk - 1) & 1)), ((nblk - 1) >> 1) & 1, abort_flag));
+        if (HV == 2) {
+            s_l[half * BM + row] = l;
+            have_o = group_all(pair_bar, 64, have_o);
+            l += s_l[(half ^ 1) * BM + row];
+        }
         tc_fence_after();
         const float inv = l > 0.f ? 1.f / l : 0.f;
-        __nv_bfloat16 *orow = O + b * p.os_b + (int64_t)i * p.os_t + h * p.os_h;
+        __nv_bfloat16 *orow = O + b * p.os_b + (int64_t)i * p.os_t + h * p.os_h + half * (D / HV);
 #pragma unroll
-        for (int c = 0; c < D / 32; ++c) {
+        for (int c = 0; c < OCH; ++c) {
             float o[32];
-            if (have_o) {   // uniform across the warp except after an abort
-                tmem_ld32(lane_base + 2 * BN + c * 32, o);
+            if (have_o) {   // uniform across the warp
+                tmem_ld32(lane_base + 2 * BN + (half * OCH + c) * 32, o);
                 tmem_wait_ld();
             } else {
 #pragma unroll
@@ -278,14 +336,14 @@ k_full_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
                 }
             }
         }
-        if (i < p.Lq)
+        if (half == 0 && i < p.Lq)
             LSE[((int64_t)b * p.Hq + h) * p.Lq + i] = (have_o && l > 0.f) ? (m_used + log2f(l)) * kLn2 : -INFINITY;
     }
     // ------------------------------------------------ teardown: everybody arrives, then TMEM is returned
     __syncwarp();
     tc_fence_before();
     __syncthreads();
-    if (warp == 5) {
+    if (warp == kMmaWarp) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(kTmemFa) : "memory");
     }
@@ -713,11 +771,11 @@ cudaError_t launch_fa(const Params &p, const void *Q, const void *K, const void 
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (!(dev >= 0 && dev < 64 && attr_set[dev])) {
-        if ((e = cudaFuncSetAttribute(k_full_tc5<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FaCfg<D>::kSmemBytes)) != cudaSuccess) return e;
+        if ((e = cudaFuncSetAttribute(k_full_tc5<D, FaShape<D>::HV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FaCfg<D>::kSmemBytes)) != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
     dim3 grid((p.Lq + BM - 1) / BM, p.B * p.Hq);
-    k_full_tc5<D><<<grid, kThreads, FaCfg<D>::kSmemBytes, st>>>(tmQ, tmK, tmV, p, (__nv_bfloat16 *)O, LSE);
+    k_full_tc5<D, FaShape<D>::HV><<<grid, FaCfg<D>::template threads<FaShape<D>::HV>(), FaCfg<D>::kSmemBytes, st>>>(tmQ, tmK, tmV, p, (__nv_bfloat16 *)O, LSE);
     count_launch();
     return cudaGetLastError();
 }

@@ -104,15 +104,6 @@ __device__ __forceinline__ void cp_async_arrive(uint32_t bar)
     asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];\n" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;\n" ::: "memory"); }
-// named barrier `id` over `count` threads that also ANDs a predicate
-__device__ __forceinline__ bool group_all(int id, int count, bool pred)
-{
-    uint32_t out;
-    asm volatile("{\n .reg .pred p, q;\n setp.ne.b32 p, %1, 0;\n barrier.cta.red.and.pred q, %2, %3, p;\n selp.u32 %0, 1, 0, q;\n}\n"
-                 : "=r"(out) : "r"((uint32_t)pred), "r"(id), "r"(count) : "memory");
-    return out != 0;
-}
-
 // Slot s of the virtual slot array [idx row | window] of a query at position pos holds a key index or is void (-1).
 // slot_raw starts the fetch (an idx entry is a global load) and slot_fix applies the validity rules to it; callers
 // keep the raw value in a register for a whole tile so that the load's latency is never waited for.
