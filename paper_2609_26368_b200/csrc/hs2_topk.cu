@@ -1081,11 +1081,24 @@ cudaError_t launch_filter_thresholds(const Params &p, const float *sample, int64
     SelArgs sa{samp, cap, tau_key, flag, nullptr, nullptr};
     const unsigned n = (unsigned)n_rows;
     const int ns_max = filter_sample_width(p, samp);
-    // class by the size of the row's sample (every row is taken by exactly one launch)
-    k_topk_cached<256, 32, true, SEL_TAU><<<n, 256, 0, st>>>(p, sample, stride, nullptr, row0, -1, 8192, sa);
+    // class by the size of the row's sample (every row is taken by exactly one launch); as for whole rows, a sample
+    // gets no more warps than it fills
+    k_topk_cached<64, 32, true, SEL_TAU><<<n, 64, 0, st>>>(p, sample, stride, nullptr, row0, -1, 2048, sa);
     count_launch();
+    if (ns_max > 2048) {
+        k_topk_cached<128, 32, true, SEL_TAU><<<n, 128, 0, st>>>(p, sample, stride, nullptr, row0, 2048, 4096, sa);
+        count_launch();
+    }
+    if (ns_max > 4096) {
+        k_topk_cached<256, 32, true, SEL_TAU><<<n, 256, 0, st>>>(p, sample, stride, nullptr, row0, 4096, 8192, sa);
+        count_launch();
+    }
     if (ns_max > 8192) {
-        k_topk_cached<512, 64, true, SEL_TAU><<<n, 512, 0, st>>>(p, sample, stride, nullptr, row0, 8192, 32768, sa);
+        k_topk_cached<256, 64, true, SEL_TAU><<<n, 256, 0, st>>>(p, sample, stride, nullptr, row0, 8192, 16384, sa);
+        count_launch();
+    }
+    if (ns_max > 16384) {
+        k_topk_cached<512, 64, true, SEL_TAU><<<n, 512, 0, st>>>(p, sample, stride, nullptr, row0, 16384, 32768, sa);
         count_launch();
     }
     return cudaGetLastError();
