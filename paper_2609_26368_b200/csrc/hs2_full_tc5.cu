@@ -400,11 +400,12 @@ struct FilterBuf {
     int cap;
 };
 
-__device__ __forceinline__ uint32_t order_key_f(float f)
+// the float whose order key is `key`; the two sentinels of the filter thresholds map to values that make the
+// comparison `score >= threshold` come out right: key 0 (every score passes) -> -inf, key 0xffffffff (none) -> NaN
+__device__ __forceinline__ float key_to_float(uint32_t key)
 {
-    uint32_t u = __float_as_uint(f);
-    if (u == 0x80000000u) u = 0u;
-    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+    if (key == 0u) return -INFINITY;
+    return __uint_as_float((key & 0x80000000u) ? (key & 0x7fffffffu) : ~key);
 }
 
 template <int G, int MODE, int D>
@@ -583,13 +584,13 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         constexpr bool kHoist = TQW <= 8;
         int nq_r[kHoist ? TQW : 1];
         float *orow_r[kHoist && MODE != SC_FILTER ? TQW : 1];
-        uint32_t tau_r[kHoist && MODE == SC_FILTER ? TQW : 1];
+        float tau_r[kHoist && MODE == SC_FILTER ? TQW : 1];   // thresholds as floats: one compare per score
         if (kHoist) {
 #pragma unroll
             for (int q = 0; q < TQW; ++q) {
                 nq_r[q] = s_nq[q_first + q];
                 if (MODE != SC_FILTER) orow_r[q] = out + s_row[q_first + q] * out_stride;   // never used when nq is 0
-                if (MODE == SC_FILTER) tau_r[q] = s_tau[q_first + q];
+                if (MODE == SC_FILTER) tau_r[q] = key_to_float(s_tau[q_first + q]);
             }
         }
         bool alive = true;
@@ -633,8 +634,9 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                     const int nq = kHoist ? nq_r[kHoist ? ql : 0] : s_nq[tq];
                     if (MODE == SC_FILTER) {
                         aval[ql] = av;
-                        const uint32_t tau = kHoist ? tau_r[kHoist ? ql : 0] : s_tau[tq];
-                        const bool pass = alive && key < nq && order_key_f(av) >= tau;
+                        // (float order and key order agree: -0 and +0 are one key, NaN scores are a caller error)
+                        const float tau = kHoist ? tau_r[kHoist ? ql : 0] : key_to_float(s_tau[tq]);
+                        const bool pass = alive && key < nq && av >= tau;
                         passbits |= (pass ? 1u : 0u) << ql;
                     } else if (key < nq) {
                         if (kHoist) orow_r[kHoist ? ql : 0][col] = av;
