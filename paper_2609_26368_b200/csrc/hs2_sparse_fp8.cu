@@ -23,7 +23,7 @@
 #include "hs2_common.cuh"
 
 #ifndef HS2_F8_WARPS
-#define HS2_F8_WARPS 12
+#define HS2_F8_WARPS 20
 #endif
 #ifndef HS2_F8D_WARPS
 #define HS2_F8D_WARPS 8
@@ -45,6 +45,9 @@ static_assert(KT == 16 || KT == 32, "a stage holds 16 or 32 key rows");
 #ifndef HS2_F8_NSTAGE
 #define HS2_F8_NSTAGE 2
 #endif
+#ifndef HS2_F8_PNSTAGE
+#define HS2_F8_PNSTAGE 1    // stages per warp in the prefill kernel (one buffer and 20 warps measured best)
+#endif
 constexpr int NSTAGE = HS2_F8_NSTAGE;
 constexpr int kRow = HD;                     // bytes of one e4m3 row
 constexpr int kTile = KT * kRow;             // one K or V tile of a stage
@@ -52,6 +55,8 @@ constexpr int kStageBytes = 2 * kTile;
 // per warp: the stages, then per stage: key index of each row (32 ints), K scales (KT), V scales (KT)
 constexpr int kMetaBytes = 32 * 4 + 2 * KT * 4;
 constexpr int kWarpSmem = NSTAGE * kStageBytes + NSTAGE * kMetaBytes;
+constexpr int NSP = HS2_F8_PNSTAGE;
+constexpr int kWarpSmemP = NSP * kStageBytes + NSP * kMetaBytes;   // prefill
 constexpr float kPShift = 256.f;             // probabilities x V scale are carried x 2^8 through the f16 operand
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -270,13 +275,15 @@ __device__ __forceinline__ void consume_stage(Acc &acc, const uint32_t (&qf)[16]
     }
 }
 
-// Fold slot tiles [t_begin, t_end) of one item into acc with an NSTAGE-deep cp.async pipeline.
+// Fold slot tiles [t_begin, t_end) of one item into acc with an NS-deep cp.async pipeline.  NS = 1: fetch, wait, fold in
+// one buffer; the warp overlaps nothing by itself, but needs half the shared memory, so more warps are resident.
+template <int NS>
 __device__ __forceinline__ void run_tiles(const Params &p, const Item &it, const uint32_t (&qf)[16], Acc &acc, int t_begin,
                                           int t_end, char *wsm, int lane)
 {
     const uint32_t sbase = smem_u32(wsm);
-    char *meta = wsm + NSTAGE * kStageBytes;
-    const uint32_t mbase = sbase + NSTAGE * kStageBytes;
+    char *meta = wsm + NS * kStageBytes;
+    const uint32_t mbase = sbase + NS * kStageBytes;
     int next = t_begin;
     int jn = next < t_end ? slot_raw(p, it, next, lane) : -1;
     int n_issued = 0, n_done = 0;
@@ -293,16 +300,28 @@ __device__ __forceinline__ void run_tiles(const Params &p, const Item &it, const
         }
         return false;
     };
+    if (NS == 1) {
+        while (try_issue(0)) {
+            cp_async_commit();
+            cp_async_wait<0>();
+            __syncwarp();
+            const unsigned mask = __ballot_sync(0xffffffffu, reinterpret_cast<const int *>(meta)[lane] >= 0);
+            consume_stage(acc, qf, sbase, reinterpret_cast<const float *>(meta + 32 * 4),
+                          reinterpret_cast<const float *>(meta + 32 * 4 + KT * 4), mask, p.scale_log2, lane);
+            __syncwarp();   // every lane has read the buffer before the next tile's copies land in it
+        }
+        return;
+    }
 #pragma unroll
-    for (int s = 0; s < NSTAGE - 1; ++s) {
-        if (try_issue(n_issued % NSTAGE)) ++n_issued;
+    for (int s = 0; s < NS - 1; ++s) {
+        if (try_issue(n_issued % NS)) ++n_issued;
         cp_async_commit();
     }
     while (n_done < n_issued) {
-        const int stage = n_done % NSTAGE;
-        cp_async_wait<NSTAGE - 2>();
+        const int stage = n_done % NS;
+        cp_async_wait<(NS >= 2 ? NS - 2 : 0)>();
         __syncwarp();
-        if (try_issue(n_issued % NSTAGE)) ++n_issued;
+        if (try_issue(n_issued % NS)) ++n_issued;
         cp_async_commit();
         const char *mt = meta + stage * kMetaBytes;
         const unsigned mask = __ballot_sync(0xffffffffu, reinterpret_cast<const int *>(mt)[lane] >= 0);
@@ -411,13 +430,13 @@ k_sparse_fp8_prefill(const Params p, const __nv_bfloat16 *__restrict__ Q, const 
     const int i = (int)(item % p.Lq);
     const int gkv = (int)((item / p.Lq) % p.Hkv);
     const int b = (int)(item / ((int64_t)p.Lq * p.Hkv));
-    char *wsm = smem + warp * kWarpSmem;
+    char *wsm = smem + warp * kWarpSmemP;
     const Item it = make_item(p, K, V, ksc, vsc, idx, b, gkv, i);
     uint32_t qf[16];
     load_q_frags(p, Q, b, i, gkv, lane, qf);
     Acc acc;
     init_acc(acc, p, sink, gkv, lane, true);
-    run_tiles(p, it, qf, acc, 0, (p.k + p.w + KT - 1) / KT, wsm, lane);
+    run_tiles<NSP>(p, it, qf, acc, 0, (p.k + p.w + KT - 1) / KT, wsm, lane);
     reduce_l(acc);
     store_output(p, acc, O, LSE, b, i, gkv, wsm, lane);
 }
@@ -444,7 +463,7 @@ k_sparse_fp8_decode(const Params p, const __nv_bfloat16 *__restrict__ Q, const u
     init_acc(acc, p, sink, gkv, lane, warp == 0);   // the sink joins the denominator once
     const int n_tiles = (p.k + p.w + KT - 1) / KT;
     const int per = (n_tiles + W - 1) / W;
-    run_tiles(p, it, qf, acc, warp * per, min(n_tiles, (warp + 1) * per), wsm, lane);
+    run_tiles<NSTAGE>(p, it, qf, acc, warp * per, min(n_tiles, (warp + 1) * per), wsm, lane);
     reduce_l(acc);
     float4 *op = reinterpret_cast<float4 *>(wsm);   // the warp's own staging area: [8][32] float4
 #pragma unroll
@@ -486,10 +505,10 @@ k_sparse_fp8_decode(const Params p, const __nv_bfloat16 *__restrict__ Q, const u
     store_output(p, tot, O, LSE, b, 0, gkv, smem + W * kWarpSmem + W * 16 * 4, lane);
 }
 
-constexpr int kPrefillSmem = HS2_F8_WARPS * kWarpSmem;
+constexpr int kPrefillSmem = HS2_F8_WARPS * kWarpSmemP;
 constexpr int kDecodeSmem = HS2_F8D_WARPS * kWarpSmem + HS2_F8D_WARPS * 16 * 4 + 8 * (HD + 8) * 2;
 static_assert(NSTAGE * kStageBytes >= 8 * 32 * 16, "a warp's stages hold its partial accumulator in decode");
-static_assert(NSTAGE * kStageBytes >= 8 * (HD + 8) * 2, "a warp's stages hold its staged output rows");
+static_assert(NSTAGE * kStageBytes >= 8 * (HD + 8) * 2 && NSP * kStageBytes >= 8 * (HD + 8) * 2, "a warp's stages hold its staged output rows");
 
 template <class Kern>
 cudaError_t set_smem(Kern kern, int bytes, bool *done)

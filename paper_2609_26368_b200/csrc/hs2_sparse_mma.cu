@@ -23,10 +23,10 @@
 #define HS2_SP_KT 16
 #endif
 #ifndef HS2_SP_NSTAGE
-#define HS2_SP_NSTAGE 2
+#define HS2_SP_NSTAGE 1
 #endif
 #ifndef HS2_SP_WARPS
-#define HS2_SP_WARPS 12
+#define HS2_SP_WARPS 20
 #endif
 #ifndef HS2_SPD_KT
 #define HS2_SPD_KT 16
@@ -62,7 +62,7 @@ struct Cfg {
     static constexpr int kStageBytes = 2 * KT * kPitch;                          // K tile then V tile
     static constexpr int kWarpSmem = NSTAGE * kStageBytes + NSTAGE * 32 * 4 + 64;   // + key index of each staged row + mbarriers
     static_assert(KT == 16 || KT == 32, "a stage holds 16 or 32 key rows");
-    static_assert(NSTAGE >= 2, "double buffering at least");
+    static_assert(NSTAGE >= 1, "at least one buffer");
 };
 using PrefillCfg = Cfg<HS2_SP_KT, HS2_SP_NSTAGE, HS2_SP_WARPS>;
 using DecodeCfg = Cfg<HS2_SPD_KT, HS2_SPD_NSTAGE, HS2_SPD_WARPS>;
@@ -337,6 +337,19 @@ __device__ __forceinline__ void run_tiles(const Params &p, const Item &it, const
         }
         return false;
     };
+    if (NSTAGE == 1 && !kBulk) {
+        // one buffer per warp: fetch, wait, fold.  A warp overlaps nothing by itself; the other warps of the SM do,
+        // and a warp that needs half the shared memory lets twice as many of them be resident.
+        while (try_issue(0)) {
+            cp_async_commit();
+            cp_async_wait<0>();
+            __syncwarp();
+            const unsigned mask = __ballot_sync(0xffffffffu, sj[lane] >= 0);
+            consume_stage<KT>(acc, qf, sbase, mask, p.scale_log2, lane, it.raw, it.lk, p.G, sj);
+            __syncwarp();   // every lane has read the buffer before the next tile's copies land in it
+        }
+        return;
+    }
 #pragma unroll
     for (int s = 0; s < NSTAGE - 1; ++s) {
         if (try_issue(n_issued % NSTAGE)) ++n_issued;
@@ -356,7 +369,7 @@ __device__ __forceinline__ void run_tiles(const Params &p, const Item &it, const
                 break;
             }
         } else {
-            cp_async_wait<NSTAGE - 2>();
+            cp_async_wait<(NSTAGE >= 2 ? NSTAGE - 2 : 0)>();
         }
         __syncwarp();
         if (try_issue(n_issued % NSTAGE)) ++n_issued;
