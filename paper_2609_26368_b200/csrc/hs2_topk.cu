@@ -12,6 +12,9 @@
 namespace hs2 {
 namespace {
 
+#ifndef HS2_TOPK_LINEAR
+#define HS2_TOPK_LINEAR 1
+#endif
 constexpr int kItems = 4;                    // consecutive scores per thread per step
 constexpr unsigned kListCap = 2048;          // threshold-bin candidates kept in shared memory (cached variant)
 constexpr int kStageOut = 4096;              // selected indices of a row staged in shared memory (cached variant)
@@ -436,6 +439,208 @@ k_topk_cached(const Params p, const float *__restrict__ scores, int64_t score_st
     }
 }
 
+// ---- whole rows, first round on a linear scale -------------------------------------------------------
+// The scores of a row are logarithms of probabilities: as floats they spend their leading bits on the exponent,
+// and most candidates share one or two exponents, so a radix digit of the float key leaves a threshold bin with a
+// large share of the row (measured on the 8K benchmark: the rounds on that bin's members were 43 % of the select).
+// Any monotone map to bins narrows the search just as exactly, so the first round here bins the VALUES on a linear
+// scale between the row's smallest and largest score (4 bins per thread); the threshold bin's members - now a few
+// dozen - go to a shared list as order-preserving keys and the exact take-th largest is found there (by ranking
+// when the list is short, else by the radix select on the list).  The candidates stay in registers as floats;
+// key equality and float equality agree (-0 and +0 are one key; NaN scores are a caller error).  Slots past the
+// row's end hold -inf and, having the highest indices, lose every tie, so they can never be selected while
+// take <= candidates.  A row whose range is empty or not finite puts every candidate in one bin: slow, still exact.
+// v > t and v == t as 0/1, comparing denormals as they are (the file is compiled with flush-to-zero, which would
+// make every denormal score equal to zero in a plain comparison; the keys, and the oracle, tell them apart)
+__device__ __forceinline__ void compare_exact(float v, float t, unsigned &gt, unsigned &eq)
+{
+    asm("{\n .reg .pred p, q;\n setp.gt.f32 p, %2, %3;\n setp.eq.f32 q, %2, %3;\n selp.u32 %0, 1, 0, p;\n selp.u32 %1, 1, 0, q;\n}\n"
+        : "=r"(gt), "=r"(eq) : "f"(v), "f"(t));
+}
+
+template <int THREADS, int E, bool VEC>
+__global__ void __launch_bounds__(THREADS, THREADS > 256 ? 1 : (E > 32 ? 2 : 3))
+k_topk_linear(const Params p, const float *__restrict__ scores, int64_t score_stride, int32_t *__restrict__ idx,
+              int64_t row0, int nc_lo, int nc_hi)
+{
+    constexpr int WARPS = THREADS / 32;
+    constexpr int NBT = 4;                  // bins per thread
+    constexpr int NB = NBT * THREADS;       // bins of the first round
+    __shared__ unsigned hist[NB < 256 ? 256 : NB];
+    __shared__ unsigned s_warp[WARPS];
+    __shared__ float s_lo[WARPS], s_hi[WARPS];
+    __shared__ unsigned s_prefix, s_need, s_cnt, s_bin;
+    extern __shared__ int s_dyn[];          // [selected indices staged for the coalesced store][list: THREADS * E keys]
+
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int64_t row = row0 + blockIdx.x;   // (b, g, i), i fastest
+    const int i = (int)(row % p.Lq);
+    const int b = (int)(row / ((int64_t)p.Lq * p.Hkv));
+    const int kvl = kvlen_of(p, b);
+    const int pos = pos_of(p, b, i);
+    const int nc = max(0, min(pos - p.w + 1, kvl));   // the row's candidates are keys 0..nc-1
+    const int take = min(p.k, nc);                    // how many of them are selected
+    if (nc <= nc_lo || nc > nc_hi) return;            // this row belongs to another variant's launch
+    int32_t *out = idx + row * p.k;
+    const float *srow = scores + (int64_t)blockIdx.x * score_stride;
+    if (take == nc) {   // every candidate is kept: no need to look at the scores
+        for (int t = tid; t < p.k; t += THREADS) out[t] = t < nc ? t : -1;
+        return;
+    }
+    const bool staged = p.k <= kStageOut;
+    int *s_out = s_dyn;
+    uint32_t *s_list = reinterpret_cast<uint32_t *>(s_dyn + (staged ? p.k : 0));
+
+    const int j0 = tid * E;
+    const bool has = j0 < nc;   // threads (whole warps, on short rows) past the row's end skip every per-candidate loop
+    float val[E];
+    float vmin = INFINITY, vmax = -INFINITY;
+    if (has)
+#pragma unroll
+    for (int e4 = 0; e4 < E; e4 += 4) {
+        if (VEC && j0 + e4 + 4 <= nc) {
+            const float4 v = __ldg(reinterpret_cast<const float4 *>(srow + j0 + e4));
+            val[e4] = v.x; val[e4 + 1] = v.y; val[e4 + 2] = v.z; val[e4 + 3] = v.w;
+            vmin = fminf(fminf(vmin, v.x), fminf(v.y, fminf(v.z, v.w)));
+            vmax = fmaxf(fmaxf(vmax, v.x), fmaxf(v.y, fmaxf(v.z, v.w)));
+        } else {
+#pragma unroll
+            for (int e = e4; e < e4 + 4; ++e) {
+                const bool ok = j0 + e < nc;
+                val[e] = ok ? srow[j0 + e] : -INFINITY;
+                if (ok) { vmin = fminf(vmin, val[e]); vmax = fmaxf(vmax, val[e]); }
+            }
+        }
+    }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        vmin = fminf(vmin, __shfl_xor_sync(0xffffffffu, vmin, o));
+        vmax = fmaxf(vmax, __shfl_xor_sync(0xffffffffu, vmax, o));
+    }
+    if (lane == 0) { s_lo[warp] = vmin; s_hi[warp] = vmax; }
+#pragma unroll
+    for (int t = 0; t < NBT; ++t) hist[t * THREADS + tid] = 0u;
+    if (tid == 0) s_cnt = 0u;
+    __syncthreads();
+#pragma unroll
+    for (int w = 0; w < WARPS; ++w) { vmin = fminf(vmin, s_lo[w]); vmax = fmaxf(vmax, s_hi[w]); }
+    // bin(v) = clamp(floor(v * c + d), 0, NB - 1) with one fused multiply-add: monotone in v, and the same
+    // instruction in both passes gives the same bin
+    const float range = vmax - vmin;
+    const bool flat = !(range > 0.f) || !(range < 3.0e38f);
+    const float c = flat ? 0.f : (float)NB / range;
+    const float d = flat ? 0.f : -vmin * c;
+    auto bin_of = [&](float v) {
+        const int bb = __float2int_rd(__fmaf_rn(v, c, d));
+        return (unsigned)min(max(bb, 0), NB - 1);
+    };
+    if (has)
+#pragma unroll
+    for (int e = 0; e < E; ++e) atomicAdd(&hist[bin_of(val[e])], 1u);
+    __syncthreads();
+    // from the top: the bin at which the running count reaches `take`.  Thread t owns bins NB-1-NBT*t-e.
+    unsigned mine = 0;
+#pragma unroll
+    for (int e = 0; e < NBT; ++e) mine += hist[NB - 1 - NBT * tid - e];
+    unsigned total;
+    const unsigned before = block_excl_scan<WARPS>(mine, s_warp, lane, warp, &total);
+    if (before < (unsigned)take && (unsigned)take <= before + mine) {
+        unsigned cum = before;
+#pragma unroll
+        for (int e = 0; e < NBT; ++e) {
+            const unsigned cnt = hist[NB - 1 - NBT * tid - e];
+            if (cum < (unsigned)take && (unsigned)take <= cum + cnt) { s_bin = NB - 1 - NBT * tid - e; s_need = (unsigned)take - cum; }
+            cum += cnt;
+        }
+    }
+    __syncthreads();
+    const unsigned tbin = s_bin;
+    unsigned need = s_need;
+    // the threshold bin's members, as keys
+    if (has)
+#pragma unroll
+    for (int e = 0; e < E; ++e)
+        if (bin_of(val[e]) == tbin) s_list[atomicAdd(&s_cnt, 1u)] = order_key(val[e]);
+    __syncthreads();
+    const unsigned n_list = s_cnt;
+    uint32_t tau;
+    if (n_list <= kRankMax && n_list <= (unsigned)THREADS) {   // one thread per member
+        if ((unsigned)tid < n_list) {
+            const uint32_t kt = s_list[tid];
+            unsigned gt = 0, eq = 0;
+            for (unsigned u = 0; u < n_list; ++u) {
+                const uint32_t v = s_list[u];
+                gt += v > kt;
+                eq += v == kt;
+            }
+            if (gt < need && need <= gt + eq) { s_prefix = kt; s_need = need - gt; }   // equal members write the same
+        }
+        __syncthreads();
+        tau = s_prefix;
+        need = s_need;
+    } else {
+        tau = select_on_list<THREADS>(s_list, n_list, need, hist, &s_prefix, &s_need, tid, lane, warp);
+        need = s_need;
+    }
+    const unsigned need_eq = need;   // equal keys kept, lowest indices first
+    const float tau_f = __uint_as_float((tau & 0x80000000u) ? (tau & 0x7fffffffu) : ~tau);
+
+    // ---- ordered compaction with one block scan
+    static_assert(E <= 64, "one 64-bit mask per thread");
+    unsigned long long m_gt = 0ull, m_eq = 0ull;
+    if (has)
+#pragma unroll
+    for (int e = 0; e < E; ++e) {
+        unsigned gt, eq;
+        compare_exact(val[e], tau_f, gt, eq);
+        m_gt |= (unsigned long long)gt << e;
+        m_eq |= (unsigned long long)eq << e;
+    }
+    const unsigned n_gt = __popcll(m_gt), n_eq = __popcll(m_eq);
+    const unsigned packed = (n_gt << 16) | n_eq;   // both totals stay below 65536 (rows <= 32768)
+    unsigned incl = packed;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const unsigned t = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += t;
+    }
+    __syncthreads();   // s_warp was read by the scan above
+    if (lane == 31) s_warp[warp] = incl;
+    __syncthreads();
+    unsigned wsum = lane < WARPS ? s_warp[lane] : 0u;
+    unsigned wincl = wsum;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const unsigned t = __shfl_up_sync(0xffffffffu, wincl, o);
+        if (lane >= o) wincl += t;
+    }
+    const unsigned excl = __shfl_sync(0xffffffffu, wincl - wsum, warp) + incl - packed;
+    const unsigned gt_before = excl >> 16, eq_before = excl & 0xffffu;
+    int *dst = staged ? s_out : out;
+    {
+        unsigned keep_eq = eq_before < need_eq ? min(n_eq, need_eq - eq_before) : 0u;
+        unsigned long long m_keep = m_gt;
+        while (keep_eq > 0) {   // rare: ties at the threshold
+            const unsigned long long low = m_eq & (0ull - m_eq);
+            m_keep |= low;
+            m_eq ^= low;
+            --keep_eq;
+        }
+        unsigned posn = gt_before + min(eq_before, need_eq);
+        while (m_keep) {   // ascending candidate index
+            const int e = __ffsll((long long)m_keep) - 1;
+            m_keep &= m_keep - 1;
+            dst[posn++] = j0 + e;
+        }
+    }
+    if (staged) {
+        __syncthreads();
+        for (int t = tid; t < p.k; t += THREADS) out[t] = t < take ? s_out[t] : -1;
+    } else {
+        for (int t = take + tid; t < p.k; t += THREADS) out[t] = -1;
+    }
+}
+
 // ---- rows of up to CL x 32768 candidates: one thread-block cluster per row ------------------------
 // Every CTA of the cluster keeps a 32768-candidate slice of the row in registers (read once).  Per
 // radix round each CTA histograms its slice, CTA 0 adds the histograms up through distributed shared
@@ -813,6 +1018,34 @@ void launch_class(int c, const Params &p, const float *scores, int64_t score_str
 #endif
     // The register kernels pay a fixed price per warp and row (rounds, scans, barriers), so a row gets no more
     // warps than its candidates fill: 32 (or 64) candidates per thread.
+#if HS2_TOPK_LINEAR
+    if (c <= 4) {   // register-resident rows: first round on a linear scale, the threshold bin's members in a shared list
+        auto go = [&](auto kern, int threads, int e) {
+            const size_t smem = stage + (size_t)threads * e * sizeof(uint32_t);
+            if (smem > 32 * 1024) {   // static shared memory counts against the 48 KB default too
+                static bool attr_set[5][64] = {};   // per row class: the kernels share one function type, hence one lambda body
+                int dev = 0;
+                if (cudaGetDevice(&dev) != cudaSuccess) return;
+                if (!(dev >= 0 && dev < 64 && attr_set[c][dev])) {
+                    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             (int)(kStageOut * sizeof(int) + (size_t)threads * e * sizeof(uint32_t))) != cudaSuccess)
+                        return;
+                    if (dev >= 0 && dev < 64) attr_set[c][dev] = true;
+                }
+            }
+            kern<<<n, threads, smem, st>>>(p, scores, score_stride, idx, row0, lo, hi);
+        };
+        switch (c) {
+            case 0: go(k_topk_linear<64, 32, VEC>, 64, 32); break;
+            case 1: go(k_topk_linear<128, 32, VEC>, 128, 32); break;
+            case 2: go(k_topk_linear<256, 32, VEC>, 256, 32); break;
+            case 3: go(k_topk_linear<256, 64, VEC>, 256, 64); break;
+            default: go(k_topk_linear<512, 64, VEC>, 512, 64); break;
+        }
+        count_launch();
+        return;
+    }
+#endif
     switch (c) {
         case 0: k_topk_cached<64, 32, VEC, SEL_ROW><<<n, 64, stage, st>>>(p, scores, score_stride, idx, row0, lo, hi, SelArgs{}); break;
         case 1: k_topk_cached<128, 32, VEC, SEL_ROW><<<n, 128, stage, st>>>(p, scores, score_stride, idx, row0, lo, hi, SelArgs{}); break;
