@@ -458,6 +458,13 @@ __device__ __forceinline__ void compare_exact(float v, float t, unsigned &gt, un
         : "=r"(gt), "=r"(eq) : "f"(v), "f"(t));
 }
 
+__device__ __forceinline__ unsigned ge_exact(float v, float t)
+{
+    unsigned r;
+    asm("{\n .reg .pred p;\n setp.ge.f32 p, %1, %2;\n selp.u32 %0, 1, 0, p;\n}\n" : "=r"(r) : "f"(v), "f"(t));
+    return r;
+}
+
 template <int THREADS, int E, bool VEC>
 __global__ void __launch_bounds__(THREADS, THREADS > 256 ? 1 : (E > 32 ? 2 : 3))
 k_topk_linear(const Params p, const float *__restrict__ scores, int64_t score_stride, int32_t *__restrict__ idx,
@@ -469,7 +476,7 @@ k_topk_linear(const Params p, const float *__restrict__ scores, int64_t score_st
     __shared__ unsigned hist[NB < 256 ? 256 : NB];
     __shared__ unsigned s_warp[WARPS];
     __shared__ float s_lo[WARPS], s_hi[WARPS];
-    __shared__ unsigned s_prefix, s_need, s_cnt, s_bin;
+    __shared__ unsigned s_prefix, s_need, s_cnt, s_bin, s_eq;
     extern __shared__ int s_dyn[];          // [selected indices staged for the coalesced store][list: THREADS * E keys]
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
@@ -530,10 +537,8 @@ k_topk_linear(const Params p, const float *__restrict__ scores, int64_t score_st
     const bool flat = !(range > 0.f) || !(range < 3.0e38f);
     const float c = flat ? 0.f : (float)NB / range;
     const float d = flat ? 0.f : -vmin * c;
-    auto bin_of = [&](float v) {
-        const int bb = __float2int_rd(__fmaf_rn(v, c, d));
-        return (unsigned)min(max(bb, 0), NB - 1);
-    };
+    // (the conversion to unsigned saturates: negative values, -inf and NaN give bin 0)
+    auto bin_of = [&](float v) { return min(__float2uint_rd(__fmaf_rn(v, c, d)), (unsigned)(NB - 1)); };
     if (has)
 #pragma unroll
     for (int e = 0; e < E; ++e) atomicAdd(&hist[bin_of(val[e])], 1u);
@@ -557,14 +562,23 @@ k_topk_linear(const Params p, const float *__restrict__ scores, int64_t score_st
     const unsigned tbin = s_bin;
     unsigned need = s_need;
     // the threshold bin's members, as keys
+    // (bin_of(v) == tbin as a range test on the same fused multiply-add: floor(x) == tbin; the clamped ends are open:
+    // nothing is below -inf, and no comparison with NaN holds, so bin 0 takes NaN and -inf, the last bin +inf)
+    const float x_lo = tbin == 0u ? -INFINITY : (float)tbin;
+    const float x_hi = tbin == (unsigned)(NB - 1) ? __uint_as_float(0x7fc00000u) : (float)(tbin + 1u);
     if (has)
 #pragma unroll
-    for (int e = 0; e < E; ++e)
-        if (bin_of(val[e]) == tbin) s_list[atomicAdd(&s_cnt, 1u)] = order_key(val[e]);
+    for (int e = 0; e < E; ++e) {
+        const float x = __fmaf_rn(val[e], c, d);
+        if (!(x < x_lo) && !(x >= x_hi)) s_list[atomicAdd(&s_cnt, 1u)] = order_key(val[e]);
+    }
     __syncthreads();
     const unsigned n_list = s_cnt;
     uint32_t tau;
     if (n_list <= kRankMax && n_list <= (unsigned)THREADS) {   // one thread per member
+        // A short list is finished by ranking: member t is the answer when fewer than `need` members are above it and
+        // at least `need` are not below it.  (Sharing a member among several threads, so that lists up to THREADS
+        // members rank too, was measured slower: short lists are the rule and the extra bookkeeping hits them all.)
         if ((unsigned)tid < n_list) {
             const uint32_t kt = s_list[tid];
             unsigned gt = 0, eq = 0;
@@ -573,7 +587,7 @@ k_topk_linear(const Params p, const float *__restrict__ scores, int64_t score_st
                 gt += v > kt;
                 eq += v == kt;
             }
-            if (gt < need && need <= gt + eq) { s_prefix = kt; s_need = need - gt; }   // equal members write the same
+            if (gt < need && need <= gt + eq) { s_prefix = kt; s_need = need - gt; s_eq = eq; }   // equal members write the same
         }
         __syncthreads();
         tau = s_prefix;
@@ -581,8 +595,11 @@ k_topk_linear(const Params p, const float *__restrict__ scores, int64_t score_st
     } else {
         tau = select_on_list<THREADS>(s_list, n_list, need, hist, &s_prefix, &s_need, tid, lane, warp);
         need = s_need;
+        if (tid == 0) s_eq = hist[tau & 255u];   // the last round's histogram: members equal to tau in all 32 bits
+        __syncthreads();
     }
     const unsigned need_eq = need;   // equal keys kept, lowest indices first
+    const bool all_ties = s_eq == need_eq;   // (the usual case: one candidate has the threshold value) every tie is kept
     const float tau_f = __uint_as_float((tau & 0x80000000u) ? (tau & 0x7fffffffu) : ~tau);
 
     // ---- ordered compaction with one block scan
@@ -591,10 +608,14 @@ k_topk_linear(const Params p, const float *__restrict__ scores, int64_t score_st
     if (has)
 #pragma unroll
     for (int e = 0; e < E; ++e) {
-        unsigned gt, eq;
-        compare_exact(val[e], tau_f, gt, eq);
-        m_gt |= (unsigned long long)gt << e;
-        m_eq |= (unsigned long long)eq << e;
+        if (all_ties) {   // uniform: the kept candidates are simply those >= tau
+            m_gt |= (unsigned long long)ge_exact(val[e], tau_f) << e;
+        } else {
+            unsigned gt, eq;
+            compare_exact(val[e], tau_f, gt, eq);
+            m_gt |= (unsigned long long)gt << e;
+            m_eq |= (unsigned long long)eq << e;
+        }
     }
     const unsigned n_gt = __popcll(m_gt), n_eq = __popcll(m_eq);
     const unsigned packed = (n_gt << 16) | n_eq;   // both totals stay below 65536 (rows <= 32768)
