@@ -12,6 +12,9 @@
 namespace hs2 {
 namespace {
 
+#ifndef HS2_TOPK_NBT
+#define HS2_TOPK_NBT 4
+#endif
 #ifndef HS2_TOPK_LINEAR
 #define HS2_TOPK_LINEAR 1
 #endif
@@ -471,7 +474,7 @@ k_topk_linear(const Params p, const float *__restrict__ scores, int64_t score_st
               int64_t row0, int nc_lo, int nc_hi)
 {
     constexpr int WARPS = THREADS / 32;
-    constexpr int NBT = 4;                  // bins per thread
+    constexpr int NBT = HS2_TOPK_NBT;       // bins per thread
     constexpr int NB = NBT * THREADS;       // bins of the first round
     __shared__ unsigned hist[NB < 256 ? 256 : NB];
     __shared__ unsigned s_warp[WARPS];
