@@ -74,7 +74,7 @@ template <int D, int HV>
 __global__ void __launch_bounds__(FaCfg<D>::template threads<HV>(), FaCfg<D>::kMinBlocks)
 k_full_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK,
            const __grid_constant__ CUtensorMap tmV, const Params p, __nv_bfloat16 *__restrict__ O,
-           float *__restrict__ LSE)
+           float *__restrict__ LSE, int head_major)
 {
     using F = FaCfg<D>;
     constexpr int NQ = F::NQ;
@@ -98,8 +98,17 @@ k_full_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
     auto bar = [&](int i) { return bars + 8u * i; };
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int mblk = gridDim.x - 1 - blockIdx.x;   // long rows first
-    const int h = blockIdx.y % p.Hq, b = blockIdx.y / p.Hq;
+    // One-dimensional grid; CTAs start in order of their index.  head_major = 0: (sequence, head) fastest and the query
+    // tile descending, so ALL heads' longest tiles run first and the last CTAs to start are the shortest ones.  (With
+    // the heads as the slow index every head's long tiles start in turn - on the 8K benchmark the last head's
+    // 130-microsecond tile at 460 of 590 microseconds, and SMs finished between 479 and 593.)  head_major = 1: one
+    // head after the other, long tiles first within a head: the CTAs in flight then share one KV head, which is worth
+    // more than the tail once the cache no longer fits L2 and the kernel runs for a hundred waves.
+    const int n_bh = p.B * p.Hq;
+    const int n_mblk = (int)(gridDim.x / n_bh);
+    const int mblk = n_mblk - 1 - (int)(head_major ? blockIdx.x % n_mblk : blockIdx.x / n_bh);
+    const int bh = (int)(head_major ? blockIdx.x / n_mblk : blockIdx.x % n_bh);
+    const int h = bh % p.Hq, b = bh / p.Hq;
     const int gkv = h / p.G;
     const int i0 = mblk * BM;
     const int kvl = kvlen_of(p, b);
@@ -776,8 +785,11 @@ cudaError_t launch_fa(const Params &p, const void *Q, const void *K, const void 
         if ((e = cudaFuncSetAttribute(k_full_tc5<D, FaShape<D>::HV>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)FaCfg<D>::kSmemBytes)) != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
-    dim3 grid((p.Lq + BM - 1) / BM, p.B * p.Hq);
-    k_full_tc5<D, FaShape<D>::HV><<<grid, FaCfg<D>::template threads<FaShape<D>::HV>(), FaCfg<D>::kSmemBytes, st>>>(tmQ, tmK, tmV, p, (__nv_bfloat16 *)O, LSE);
+    dim3 grid((unsigned)(((p.Lq + BM - 1) / BM) * (p.B * p.Hq)));
+    // the whole cache of the call against the L2 (126 MB on B200; the test is a fixed 96 MB so that it is the same everywhere)
+    const int64_t kv_bytes = (int64_t)p.B * p.Hkv * p.Lk * D * 2 * 2;
+    const int head_major = kv_bytes > ((int64_t)96 << 20) ? 1 : 0;
+    k_full_tc5<D, FaShape<D>::HV><<<grid, FaCfg<D>::template threads<FaShape<D>::HV>(), FaCfg<D>::kSmemBytes, st>>>(tmQ, tmK, tmV, p, (__nv_bfloat16 *)O, LSE, head_major);
     count_launch();
     return cudaGetLastError();
 }
