@@ -61,7 +61,8 @@ typedef enum {
     HS2_OP_FULL_ATTN_SELECT = 0,
     HS2_OP_TOPK_SELECT = 1,
     HS2_OP_SPARSE_ATTN_PREFILL = 2,
-    HS2_OP_SPARSE_ATTN_DECODE = 3
+    HS2_OP_SPARSE_ATTN_DECODE = 3,
+    HS2_OP_FULL_ATTN_SELECT_FP8KV = 4
 } hs2_op;
 
 typedef struct {
@@ -181,6 +182,23 @@ hs2_status hs2_sparse_attn_prefill_fp8kv(const hs2_problem *p, const void *Q, co
 hs2_status hs2_sparse_attn_decode_fp8kv(const hs2_problem *p, const void *Q, const void *K8, const void *V8,
                                         const float *k_scale, const float *v_scale, const int32_t *idx,
                                         const float *sink, void *O, float *LSE, void *cuda_stream);
+
+/*
+ * The decode step of the full-attention layer on the FP8 cache (Section 3.4, with the cache storage that the cost
+ * analysis of Section 4 assumes): one query per sequence attends to its whole context, and the layer selects the
+ * k_sel tokens outside the window from the same scores, exactly as hs2_full_attn_select does on a bf16 cache.
+ *   Q [B,1,Hq,D] bf16; K8, V8, k_scale, v_scale: the cache as described above for the sparse calls; O [B,1,Hq,D] bf16;
+ *   LSE [B,Hq,1] fp32; idx [B,Hkv,1,k_sel] int32 or NULL (attention only).  All device pointers.
+ *   ws: with idx, at least hs2_workspace_bytes(p, HS2_OP_FULL_ATTN_SELECT_FP8KV) bytes, 256-byte aligned (the
+ *   dequantised q.k products of every head and key, 4 bytes each, and one score row per (sequence, KV head));
+ *   HS2_ERR_WORKSPACE_TOO_SMALL otherwise.  Without idx no scratch is needed.
+ *   Covers q_len == 1, head_dim 128, groups of at most 8 query heads, 16-byte aligned tensors, products that fit
+ *   2 GiB; anything else returns HS2_ERR_UNSUPPORTED and launches nothing.  (A prefill-shaped full layer attends to
+ *   the bf16 K and V it has just produced, so there is no FP8 variant of it.)
+ */
+hs2_status hs2_full_attn_select_fp8kv(const hs2_problem *p, const void *Q, const void *K8, const void *V8,
+                                      const float *k_scale, const float *v_scale, void *O, float *LSE, int32_t *idx,
+                                      void *ws, size_t ws_bytes, void *cuda_stream);
 
 /*
  * hs2_sparse_attn_decode for callers that cannot hand over a scratch buffer.  (The paper has no

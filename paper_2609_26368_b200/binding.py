@@ -21,10 +21,11 @@ HS2_OK, HS2_ERR_INVALID_ARG, HS2_ERR_UNSUPPORTED, HS2_ERR_WORKSPACE_TOO_SMALL, H
 HS2_STATIC_DECODE_MAX_PAIRS = 64
 HS2_F32, HS2_BF16 = 0, 1
 HS2_OP_FULL_ATTN_SELECT, HS2_OP_TOPK_SELECT, HS2_OP_SPARSE_ATTN_PREFILL, HS2_OP_SPARSE_ATTN_DECODE = range(4)
+HS2_OP_FULL_ATTN_SELECT_FP8KV = 4
 
 EXPORTS = ["hs2_workspace_bytes", "hs2_full_attn_select", "hs2_topk_select", "hs2_sparse_attn_prefill",
            "hs2_sparse_attn_decode", "hs2_sparse_attn_prefill_gated", "hs2_sparse_attn_decode_gated",
-           "hs2_sparse_attn_prefill_fp8kv", "hs2_sparse_attn_decode_fp8kv", "hs2_kv_project",
+           "hs2_sparse_attn_prefill_fp8kv", "hs2_sparse_attn_decode_fp8kv", "hs2_full_attn_select_fp8kv", "hs2_kv_project",
            "hs2_sparse_attn_decode_static", "hs2_status_string", "hs2_last_cuda_error",
            "hs2_launch_count", "hs2_device_error_flags", "hs2_set_filter_min_keys", "hs2_set_tcgen05_enabled"]
 
@@ -77,6 +78,7 @@ def load_library():
         lib.hs2_kv_project.restype = C.c_int
         lib.hs2_sparse_attn_prefill_fp8kv.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         lib.hs2_sparse_attn_decode_fp8kv.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
+        lib.hs2_full_attn_select_fp8kv.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         for f in ("hs2_full_attn_select", "hs2_topk_select", "hs2_sparse_attn_prefill", "hs2_sparse_attn_decode",
                   "hs2_sparse_attn_prefill_gated", "hs2_sparse_attn_decode_gated", "hs2_sparse_attn_decode_static",
                   "hs2_sparse_attn_prefill_fp8kv", "hs2_sparse_attn_decode_fp8kv"):
@@ -287,6 +289,31 @@ def _sparse_fp8(fn_name, prob, q, k8, v8, k_scale, v_scale, idx, sink, out, lse,
                                           _dp(sink), _dp(out), _dp(lse), _stream(stream))
     _check(st, fn_name)
     return out, lse
+
+
+def hs2_full_attn_select_fp8kv(prob: Problem, q, k8, v8, k_scale, v_scale, *, out=None, lse=None, idx=None, want_idx=True,
+                               ws=None, stream=None):
+    """FA layer, decode step (one query per sequence), on an e4m3 cache: returns ``(O, LSE, idx | None)``."""
+    assert q.is_cuda and q.dtype == torch.bfloat16 and q.stride(-1) == 1
+    for t in (k8, v8):
+        assert t.is_cuda and t.dtype == torch.uint8 and t.stride(-1) == 1
+        assert tuple(t.shape) == (prob.batch, prob.kv_len, prob.n_kv_heads, prob.head_dim)
+    assert k8.stride() == v8.stride()
+    for t in (k_scale, v_scale):
+        assert t.is_cuda and t.dtype == torch.float32 and t.is_contiguous()
+        assert tuple(t.shape) == (prob.batch, prob.kv_len, prob.n_kv_heads)
+    dev = q.device
+    out = torch.empty_like(q) if out is None else out
+    lse = torch.empty(prob.batch, prob.n_q_heads, prob.q_len, dtype=torch.float32, device=dev) if lse is None else lse
+    if idx is None and want_idx:
+        idx = torch.empty(prob.batch, prob.n_kv_heads, prob.q_len, prob.k_sel, dtype=torch.int32, device=dev)
+    if idx is not None:
+        ws = _workspace(prob, HS2_OP_FULL_ATTN_SELECT_FP8KV, dev, ws)
+    c = prob.c_struct(q, k8, out)
+    st = load_library().hs2_full_attn_select_fp8kv(C.byref(c), _dp(q), _dp(k8), _dp(v8), _dp(k_scale), _dp(v_scale), _dp(out),
+                                                   _dp(lse), _dp(idx), _dp(ws), 0 if ws is None else ws.numel(), _stream(stream))
+    _check(st, "hs2_full_attn_select_fp8kv")
+    return out, lse, idx
 
 
 def hs2_sparse_attn_prefill_fp8kv(prob: Problem, q, k8, v8, k_scale, v_scale, idx, *, sink=None, out=None, lse=None,

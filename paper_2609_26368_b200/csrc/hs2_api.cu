@@ -238,6 +238,15 @@ size_t hs2_workspace_bytes(const hs2_problem *hp, hs2_op op)
         case HS2_OP_TOPK_SELECT:
         case HS2_OP_SPARSE_ATTN_PREFILL:
             return 0;
+        case HS2_OP_FULL_ATTN_SELECT_FP8KV:
+            if (resolve(hp, true, &p) != HS2_OK) return 0;
+            if (p.Lq != 1 || p.k == 0) return 0;
+            {
+                Params pd = p;
+                pd.k = 0; pd.w = p.Lk;
+                const DecodeFusedPlan fu = decode_fused_plan(pd, 0);
+                return fu.ok ? fu.total : 0;
+            }
         case HS2_OP_SPARSE_ATTN_DECODE:
             if (resolve(hp, true, &p) != HS2_OK) return 0;
             if (p.Lq != 1) return 0;
@@ -499,6 +508,39 @@ hs2_status hs2_sparse_attn_decode_fp8kv(const hs2_problem *hp, const void *Q, co
                                         const float *sink, void *O, float *LSE, void *cuda_stream)
 {
     return sparse_fp8_impl(hp, true, Q, K8, V8, k_scale, v_scale, idx, sink, O, LSE, cuda_stream);
+}
+
+hs2_status hs2_full_attn_select_fp8kv(const hs2_problem *hp, const void *Q, const void *K8, const void *V8,
+                                      const float *k_scale, const float *v_scale, void *O, float *LSE, int32_t *idx,
+                                      void *ws, size_t ws_bytes, void *cuda_stream)
+{
+    Params p;
+    hs2_status s = resolve(hp, true, &p);
+    if (s != HS2_OK) return s;
+    if (!Q || !K8 || !V8 || !k_scale || !v_scale || !O || !LSE) return HS2_ERR_INVALID_ARG;
+    // One query per sequence only: a prefill-shaped full layer attends to the bf16 K and V it has just produced; it
+    // is the decode step that reads the quantised cache.
+    if (p.Lq != 1) return HS2_ERR_UNSUPPORTED;
+    Params pd = p;   // a sweep over the whole cache: the gather kernel with no index list and a window that covers the context
+    pd.k = 0; pd.w = p.Lk;
+    if (!sparse_fp8_supported(pd, hp->dtype) || !aligned16(Q, K8, V8, O) || (int64_t)p.B * p.Hkv > 65535) return HS2_ERR_UNSUPPORTED;
+    const bool want_sel = idx != nullptr && p.k > 0;
+    const DecodeFusedPlan fu = decode_fused_plan(pd, 0);
+    if (want_sel) {
+        if (!fu.ok) return HS2_ERR_UNSUPPORTED;   // the raw products of this problem would not fit the scratch cap
+        if (!ws_ok(ws, ws_bytes, fu.total)) return HS2_ERR_WORKSPACE_TOO_SMALL;
+    }
+    if ((s = check_device()) != HS2_OK) return s;
+    cudaStream_t st = (cudaStream_t)cuda_stream;
+    float *raw = want_sel ? reinterpret_cast<float *>(static_cast<char *>(ws) + fu.off_raw) : nullptr;
+    cudaError_t e = launch_sparse_fp8_decode(pd, Q, K8, V8, k_scale, v_scale, nullptr, nullptr, O, LSE, st, raw);
+    if (e != cudaSuccess) return cuda_fail(e);
+    if (!want_sel) return HS2_OK;
+    float *strip = reinterpret_cast<float *>(static_cast<char *>(ws) + fu.off_strip);
+    const int64_t stride = (int64_t)(strip_row_bytes(p) / sizeof(float));
+    if ((e = launch_scores_from_raw(p, raw, LSE, strip, stride, st)) != cudaSuccess) return cuda_fail(e);
+    if ((e = launch_select(p, strip, stride, idx, 0, select_rows(p), st)) != cudaSuccess) return cuda_fail(e);
+    return HS2_OK;
 }
 
 hs2_status hs2_kv_project(int64_t n_tokens, int32_t d_model, int32_t n_out, const void *H, int64_t ldh, const void *W,

@@ -150,7 +150,7 @@ cudaError_t launch_sparse_fp8_prefill(const Params &p, const void *Q, const void
                                       cudaStream_t st);
 cudaError_t launch_sparse_fp8_decode(const Params &p, const void *Q, const void *K, const void *V, const float *ksc,
                                      const float *vsc, const int32_t *idx, const float *sink, void *O, float *LSE,
-                                     cudaStream_t st);
+                                     cudaStream_t st, float *raw = nullptr);
 // KV-cache producer: C[T, N] = H[T, dm] W[N, dm]^T, bf16 out or e4m3 codes + scale per (token, 128 columns)
 bool kv_project_supported(int64_t T, int N, int dm, int64_t ldh, int64_t ldw, int64_t ldc, bool fp8);
 cudaError_t launch_kv_project(int64_t T, int N, int dm, const void *H, int64_t ldh, const void *W, int64_t ldw, void *C,

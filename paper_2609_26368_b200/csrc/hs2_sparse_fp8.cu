@@ -125,6 +125,8 @@ struct Item {
     int sc_stride;                // floats between consecutive tokens' scales
     const int32_t *irow;
     int pos, kvl;
+    float *raw;                   // decode-shaped full layer: dequantised q.k of every (head, key) goes here, or null
+    int lk;
 };
 
 __device__ __forceinline__ Item make_item(const Params &p, const uint8_t *K, const uint8_t *V, const float *ksc, const float *vsc,
@@ -144,6 +146,8 @@ __device__ __forceinline__ Item make_item(const Params &p, const uint8_t *K, con
     it.irow = idx ? idx + (((int64_t)b * hkv_real + g_real) * p.Lq + i) * p.k : nullptr;
     it.pos = pos_of(p, b, i);
     it.kvl = kvlen_of(p, b);
+    it.raw = nullptr;
+    it.lk = 0;
     return it;
 }
 
@@ -190,7 +194,8 @@ __device__ __forceinline__ void issue_stage(const Item &it, uint32_t stage_base,
 }
 
 __device__ __forceinline__ void consume_stage(Acc &acc, const uint32_t (&qf)[16], uint32_t stage_base, const float *sks,
-                                              const float *svs, unsigned mask, float scale_log2, int lane)
+                                              const float *svs, unsigned mask, float scale_log2, int lane,
+                                              float *raw = nullptr, int lk = 0, int G = 0, const int *sjrow = nullptr)
 {
     const int g = lane >> 2;
     const int mi = lane >> 3, rr = lane & 7;
@@ -210,6 +215,24 @@ __device__ __forceinline__ void consume_stage(Acc &acc, const uint32_t (&qf)[16]
         }
 #pragma unroll
         for (int e = 0; e < 4; ++e) s[mt][e] += s2[e];
+    }
+    if (raw) {
+        // The decode-shaped full layer keeps the dequantised products: the selection scores need the final LSE, and
+        // reading them back (4 bytes per head and key) is far cheaper than sweeping K a second time.
+        const int t = lane & 3;
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+            for (int r = 0; r < 2; ++r) {
+                const int row = mt * 16 + g + 8 * r;
+                const int j = sjrow[row];
+                if (j >= 0) {
+                    const float ks = sks[row];
+#pragma unroll
+                    for (int hh = 0; hh < 2; ++hh)
+                        if (2 * t + hh < G) raw[(int64_t)(2 * t + hh) * lk + j] = s[mt][2 * r + hh] * ks;
+                }
+            }
     }
     // dequantise the score rows, online softmax in the base-2 domain; this thread: heads 2t+hh, keys 16 mt + g + 8 r
     float mx[2] = {-INFINITY, -INFINITY};
@@ -307,7 +330,8 @@ __device__ __forceinline__ void run_tiles(const Params &p, const Item &it, const
             __syncwarp();
             const unsigned mask = __ballot_sync(0xffffffffu, reinterpret_cast<const int *>(meta)[lane] >= 0);
             consume_stage(acc, qf, sbase, reinterpret_cast<const float *>(meta + 32 * 4),
-                          reinterpret_cast<const float *>(meta + 32 * 4 + KT * 4), mask, p.scale_log2, lane);
+                          reinterpret_cast<const float *>(meta + 32 * 4 + KT * 4), mask, p.scale_log2, lane, it.raw, it.lk, p.G,
+                          reinterpret_cast<const int *>(meta));
             __syncwarp();   // every lane has read the buffer before the next tile's copies land in it
         }
         return;
@@ -326,7 +350,8 @@ __device__ __forceinline__ void run_tiles(const Params &p, const Item &it, const
         const char *mt = meta + stage * kMetaBytes;
         const unsigned mask = __ballot_sync(0xffffffffu, reinterpret_cast<const int *>(mt)[lane] >= 0);
         consume_stage(acc, qf, sbase + stage * kStageBytes, reinterpret_cast<const float *>(mt + 32 * 4),
-                      reinterpret_cast<const float *>(mt + 32 * 4 + KT * 4), mask, p.scale_log2, lane);
+                      reinterpret_cast<const float *>(mt + 32 * 4 + KT * 4), mask, p.scale_log2, lane, it.raw, it.lk, p.G,
+                      reinterpret_cast<const int *>(mt));
         ++n_done;
     }
     cp_async_wait<0>();
@@ -446,7 +471,7 @@ __global__ void __launch_bounds__(HS2_F8D_WARPS * 32, HS2_F8D_MINB)
 k_sparse_fp8_decode(const Params p, const __nv_bfloat16 *__restrict__ Q, const uint8_t *__restrict__ K,
                     const uint8_t *__restrict__ V, const float *__restrict__ ksc, const float *__restrict__ vsc,
                     const int32_t *__restrict__ idx, const float *__restrict__ sink, __nv_bfloat16 *__restrict__ O,
-                    float *__restrict__ LSE)
+                    float *__restrict__ LSE, float *__restrict__ raw)
 {
     extern __shared__ __align__(128) char smem[];
     constexpr int W = HS2_F8D_WARPS;
@@ -456,7 +481,8 @@ k_sparse_fp8_decode(const Params p, const __nv_bfloat16 *__restrict__ Q, const u
     const int g = lane >> 2, t = lane & 3;
     char *wsm = smem + warp * kWarpSmem;
     float *sml = reinterpret_cast<float *>(smem + W * kWarpSmem);   // [W][16]: m then l per head
-    const Item it = make_item(p, K, V, ksc, vsc, idx, b, gkv, 0);
+    Item it = make_item(p, K, V, ksc, vsc, idx, b, gkv, 0);
+    if (raw) { it.raw = raw + (int64_t)bg * p.G * p.Lk; it.lk = p.Lk; }
     uint32_t qf[16];
     load_q_frags(p, Q, b, 0, gkv, lane, qf);
     Acc acc;
@@ -555,7 +581,7 @@ cudaError_t launch_sparse_fp8_prefill(const Params &p, const void *Q, const void
 
 cudaError_t launch_sparse_fp8_decode(const Params &p, const void *Q, const void *K, const void *V, const float *ksc,
                                      const float *vsc, const int32_t *idx, const float *sink, void *O, float *LSE,
-                                     cudaStream_t st)
+                                     cudaStream_t st, float *raw)
 {
     static bool done[64] = {};
     cudaError_t e = set_smem(k_sparse_fp8_decode, kDecodeSmem, done);
@@ -564,7 +590,7 @@ cudaError_t launch_sparse_fp8_decode(const Params &p, const void *Q, const void 
     if (pairs <= 0) return cudaSuccess;
     if (pairs > 0x7fffffffLL) return cudaErrorNotSupported;
     k_sparse_fp8_decode<<<(unsigned)pairs, HS2_F8D_WARPS * 32, kDecodeSmem, st>>>(
-        p, (const __nv_bfloat16 *)Q, (const uint8_t *)K, (const uint8_t *)V, ksc, vsc, idx, sink, (__nv_bfloat16 *)O, LSE);
+        p, (const __nv_bfloat16 *)Q, (const uint8_t *)K, (const uint8_t *)V, ksc, vsc, idx, sink, (__nv_bfloat16 *)O, LSE, raw);
     count_launch();
     return cudaGetLastError();
 }

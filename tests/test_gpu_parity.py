@@ -6,7 +6,7 @@ import torch
 import oracle
 import paper_2609_26368_b200 as hs2
 from gen import CONFIGS, make_inputs, scaled
-from parity import BlockRun, TOL, assert_output_close, to_host
+from parity import BlockRun, TOL, assert_output_close, check_idx_against_oracle, rows_all, to_host
 
 pytestmark = pytest.mark.gpu
 
@@ -389,6 +389,53 @@ def test_fp8_kv_cache_sparse_prefill_and_decode():
     idx = torch.zeros(1, 1, 16, 8, dtype=torch.int32, device="cuda")
     with pytest.raises(hs2.HS2Error):
         hs2.hs2_sparse_attn_prefill_fp8kv(prob, inp.q_full, k8, k8, ksc, ksc, idx)
+
+
+def test_fp8_kv_cache_full_layer_decode_step():
+    """The full-attention layer's decode step on the e4m3 cache: O, LSE and the selected indices against the oracle
+    run on the dequantised cache (groups of 8, 4 and 1, ragged lengths, a strided cache, several key tiles per warp)."""
+    from gen.workloads import quantize_kv_e4m3
+    cases = [
+        dict(kv_len=3000, k_sel=200, window=32, batch=3),
+        dict(kv_len=700, k_sel=64, window=16, n_q_heads=8, n_kv_heads=2, batch=2),
+        dict(kv_len=450, k_sel=100, window=0, n_q_heads=4, n_kv_heads=4, batch=1),
+    ]
+    for ci, over in enumerate(cases):
+        wl = scaled("cfg5", q_len=1, n_needles=6, **over)
+        inp = make_inputs(wl, "cuda")
+        B, Lk, Hkv, D = inp.k.shape
+        k8, ksc = quantize_kv_e4m3(inp.k)
+        v8, vsc = quantize_kv_e4m3(inp.v)
+        if ci == 0:                                  # K and V as slices of one fused cache
+            fused = torch.empty(B, Lk, 2, Hkv, D, dtype=torch.uint8, device="cuda")
+            fused[:, :, 0].copy_(k8)
+            fused[:, :, 1].copy_(v8)
+            k8, v8 = fused[:, :, 0], fused[:, :, 1]
+        kv_lens = [Lk - 11 * b for b in range(wl.batch)]
+        kl_t = torch.tensor(kv_lens, dtype=torch.int32, device="cuda")
+        q = inp.q_full
+        prob = hs2.Problem.from_tensors(q, k8, wl.k_sel, wl.window, kv_lens=kl_t)
+        O, LSE, idx = hs2.hs2_full_attn_select_fp8kv(prob, q, k8, v8, ksc, vsc)
+        torch.cuda.synchronize()
+        kd = torch.from_numpy(oracle.dequant_e4m3(k8.contiguous(), ksc))
+        vd = torch.from_numpy(oracle.dequant_e4m3(v8.contiguous(), vsc))
+        rows = rows_all(B, 1)
+        Oo, LSEo, idxo, sco = oracle.full_attn_select(q.float().cpu(), kd, vd, wl.k_sel, wl.window, rows=rows,
+                                                      want_scores=True, kv_lens=kv_lens)
+        assert_output_close(O.reshape(-1, wl.n_q_heads, D), Oo, wl.torch_dtype, "fp8 full attention O")
+        l = LSE.permute(0, 2, 1).reshape(B, wl.n_q_heads).cpu().numpy().astype(np.float64)
+        assert np.abs(l - LSEo).max() <= TOL[wl.torch_dtype]["lse"]
+        check_idx_against_oracle(idx.permute(0, 2, 1, 3).reshape(B, Hkv, wl.k_sel).cpu().numpy(), idxo, sco)
+        # attention only: no scratch, same O
+        O2, _, none = hs2.hs2_full_attn_select_fp8kv(prob, q, k8, v8, ksc, vsc, want_idx=False)
+        assert none is None and torch.equal(O, O2)
+    # more than one query per sequence is refused
+    wl = scaled("cfg2", q_len=4, kv_len=64, k_sel=8, window=4, n_needles=4)
+    inp = make_inputs(wl, "cuda")
+    k8, ksc = quantize_kv_e4m3(inp.k)
+    prob = hs2.Problem.from_tensors(inp.q_full, k8, wl.k_sel, wl.window)
+    with pytest.raises(hs2.HS2Error):
+        hs2.hs2_full_attn_select_fp8kv(prob, inp.q_full, k8, k8, ksc, ksc)
 
 
 def test_block_level_selection_variant():
