@@ -7,10 +7,10 @@
 //   * one warp owns one (query, KV head) item (prefill) or one split of it (decode) and runs its own
 //     cp.async pipeline: NSTAGE stages of KT key rows (K and V), 16-byte copies, rows placed in
 //     shared memory with an XOR swizzle so that ldmatrix is conflict free; no CTA-wide barriers.
-//     Prefill (cache mostly in L2) runs with ONE buffer per warp - fetch, wait, fold - and 20 warps per
-//     SM: the latency of a warp's fetch is covered by the other warps, and the halved shared memory is
-//     what lets them be resident (measured 1.23 ms against 1.47 ms with two stages and 12 warps on the
-//     8K benchmark).  Decode (cache in HBM, few tiles per warp) keeps two stages;
+//     Prefill (cache mostly in L2) runs with ONE buffer per warp - fetch, wait, fold: the latency of a
+//     warp's fetch is covered by the other warps.  Measured on the 8K benchmark: two stages of 16 rows x
+//     12 warps 1.47 ms; one buffer of 16 rows x 20 warps 1.23 ms; one buffer of 32 rows x 12 warps
+//     1.19 ms (the default).  Decode (cache in HBM, few tiles per warp) keeps two stages of 16 rows;
 //   * the G x keys products go through tensor cores only because plain FMAs could not keep up with
 //     the memory system at 8 flop/byte: S^T = K Q^T with the keys on the MMA M dimension and the
 //     (padded to 8) heads on N, so nothing of the m16n8k16 tile is wasted; P^T is re-laid out for the
@@ -24,13 +24,13 @@
 
 // Tuning knobs (compile time): key rows per stage, pipeline depth, warps per CTA; prefill and decode.
 #ifndef HS2_SP_KT
-#define HS2_SP_KT 16
+#define HS2_SP_KT 32
 #endif
 #ifndef HS2_SP_NSTAGE
 #define HS2_SP_NSTAGE 1
 #endif
 #ifndef HS2_SP_WARPS
-#define HS2_SP_WARPS 20
+#define HS2_SP_WARPS 12
 #endif
 #ifndef HS2_SPD_KT
 #define HS2_SPD_KT 16
@@ -334,7 +334,7 @@ __device__ __forceinline__ void run_tiles(const Params &p, const Item &it, const
             if (next < t_end) jn = slot_raw<KT>(p, it, next, lane);
             if (__ballot_sync(0xffffffffu, j >= 0)) {
                 sj[stage * 32 + lane] = j;
-                if (kBulk) issue_stage_bulk<KT>(it, sbase + stage * kStageBytes, bars + 8 * stage, j, lane);
+                if constexpr (kBulk) issue_stage_bulk<KT>(it, sbase + stage * kStageBytes, bars + 8 * stage, j, lane);
                 else issue_stage<KT>(it, sbase + stage * kStageBytes, j, lane);
                 return true;
             }
