@@ -468,8 +468,11 @@ __device__ __forceinline__ unsigned ge_exact(float v, float t)
     return r;
 }
 
+#ifndef HS2_TOPK_MINB32
+#define HS2_TOPK_MINB32 4
+#endif
 template <int THREADS, int E, bool VEC>
-__global__ void __launch_bounds__(THREADS, THREADS > 256 ? 1 : (E > 32 ? 2 : 3))
+__global__ void __launch_bounds__(THREADS, THREADS > 256 ? 1 : (E > 32 ? 2 : (HS2_TOPK_MINB32 * 256 / THREADS)))
 k_topk_linear(const Params p, const float *__restrict__ scores, int64_t score_stride, int32_t *__restrict__ idx,
               int64_t row0, int nc_lo, int nc_hi)
 {
