@@ -474,7 +474,7 @@ __device__ __forceinline__ unsigned ge_exact(float v, float t)
 template <int THREADS, int E, bool VEC>
 __global__ void __launch_bounds__(THREADS, THREADS > 256 ? 1 : (E > 32 ? 2 : (HS2_TOPK_MINB32 * 256 / THREADS)))
 k_topk_linear(const Params p, const float *__restrict__ scores, int64_t score_stride, int32_t *__restrict__ idx,
-              int64_t row0, int nc_lo, int nc_hi)
+              int64_t row0, int nc_lo, int nc_hi, int64_t n_rows, int i_first)
 {
     constexpr int WARPS = THREADS / 32;
     constexpr int NBT = HS2_TOPK_NBT;       // bins per thread
@@ -486,7 +486,12 @@ k_topk_linear(const Params p, const float *__restrict__ scores, int64_t score_st
     extern __shared__ int s_dyn[];          // [selected indices staged for the coalesced store][list: THREADS * E keys]
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    const int64_t row = row0 + blockIdx.x;   // (b, g, i), i fastest
+    // i_first < 0: one CTA per row of the block.  Otherwise (positions known on the host) the grid covers only the
+    // queries whose candidate count falls into this launch's class: x = query offset from i_first, y = (sequence,
+    // KV head) from the block's first one; a launch then starts no CTAs that would leave at once.
+    const int64_t row = i_first < 0 ? row0 + blockIdx.x : (row0 / p.Lq + blockIdx.y) * p.Lq + i_first + blockIdx.x;   // (b, g, i), i fastest
+    if (row < row0 || row >= row0 + n_rows) return;
+    const int64_t local = row - row0;
     const int i = (int)(row % p.Lq);
     const int b = (int)(row / ((int64_t)p.Lq * p.Hkv));
     const int kvl = kvlen_of(p, b);
@@ -495,7 +500,7 @@ k_topk_linear(const Params p, const float *__restrict__ scores, int64_t score_st
     const int take = min(p.k, nc);                    // how many of them are selected
     if (nc <= nc_lo || nc > nc_hi) return;            // this row belongs to another variant's launch
     int32_t *out = idx + row * p.k;
-    const float *srow = scores + (int64_t)blockIdx.x * score_stride;
+    const float *srow = scores + local * score_stride;
     if (take == nc) {   // every candidate is kept: no need to look at the scores
         for (int t = tid; t < p.k; t += THREADS) out[t] = t < nc ? t : -1;
         return;
@@ -1047,29 +1052,45 @@ void launch_class(int c, const Params &p, const float *scores, int64_t score_str
     // warps than its candidates fill: 32 (or 64) candidates per thread.
 #if HS2_TOPK_LINEAR
     if (c <= 4) {   // register-resident rows: first round on a linear scale, the threshold bin's members in a shared list
-        auto go = [&](auto kern, int threads, int e) {
+        auto go = [&](auto kern, int threads, int e) -> bool {   // false: nothing was launched
             const size_t smem = stage + (size_t)threads * e * sizeof(uint32_t);
             if (smem > 32 * 1024) {   // static shared memory counts against the 48 KB default too
                 static bool attr_set[5][64] = {};   // per row class: the kernels share one function type, hence one lambda body
                 int dev = 0;
-                if (cudaGetDevice(&dev) != cudaSuccess) return;
+                if (cudaGetDevice(&dev) != cudaSuccess) return false;
                 if (!(dev >= 0 && dev < 64 && attr_set[c][dev])) {
                     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
                                              (int)(kStageOut * sizeof(int) + (size_t)threads * e * sizeof(uint32_t))) != cudaSuccess)
-                        return;
+                        return false;
                     if (dev >= 0 && dev < 64) attr_set[c][dev] = true;
                 }
             }
-            kern<<<n, threads, smem, st>>>(p, scores, score_stride, idx, row0, lo, hi);
+            // the queries of this class, when the candidate count is a known function of the query index
+            if (!p.q_start && !p.kv_lens) {
+                const int64_t base = (int64_t)p.Lk - p.Lq - p.w + 1;   // candidates of query i: clamp(base + i, 0, Lk)
+                int64_t i_lo = lo < 0 ? 0 : (int64_t)lo + 1 - base, i_hi = hi >= p.Lk ? (int64_t)p.Lq - 1 : (int64_t)hi - base;
+                if (i_lo < 0) i_lo = 0;
+                if (i_hi > p.Lq - 1) i_hi = p.Lq - 1;
+                if (i_hi < i_lo) return false;
+                const int64_t n_bg = (row0 + n_rows - 1) / p.Lq - row0 / p.Lq + 1;
+                if (n_bg <= 65535) {
+                    kern<<<dim3((unsigned)(i_hi - i_lo + 1), (unsigned)n_bg), threads, smem, st>>>(p, scores, score_stride, idx, row0, lo, hi,
+                                                                                          n_rows, (int)i_lo);
+                    return true;
+                }
+            }
+            kern<<<n, threads, smem, st>>>(p, scores, score_stride, idx, row0, lo, hi, n_rows, -1);
+            return true;
         };
+        bool launched = false;
         switch (c) {
-            case 0: go(k_topk_linear<64, 32, VEC>, 64, 32); break;
-            case 1: go(k_topk_linear<128, 32, VEC>, 128, 32); break;
-            case 2: go(k_topk_linear<256, 32, VEC>, 256, 32); break;
-            case 3: go(k_topk_linear<256, 64, VEC>, 256, 64); break;
-            default: go(k_topk_linear<512, 64, VEC>, 512, 64); break;
+            case 0: launched = go(k_topk_linear<64, 32, VEC>, 64, 32); break;
+            case 1: launched = go(k_topk_linear<128, 32, VEC>, 128, 32); break;
+            case 2: launched = go(k_topk_linear<256, 32, VEC>, 256, 32); break;
+            case 3: launched = go(k_topk_linear<256, 64, VEC>, 256, 64); break;
+            default: launched = go(k_topk_linear<512, 64, VEC>, 512, 64); break;
         }
-        count_launch();
+        if (launched) count_launch();
         return;
     }
 #endif
