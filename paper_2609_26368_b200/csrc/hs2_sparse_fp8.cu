@@ -23,7 +23,7 @@
 #include "hs2_common.cuh"
 
 #ifndef HS2_F8_WARPS
-#define HS2_F8_WARPS 20
+#define HS2_F8_WARPS 16
 #endif
 #ifndef HS2_F8D_WARPS
 #define HS2_F8D_WARPS 8
@@ -39,9 +39,12 @@ constexpr int HD = 128;
 #ifndef HS2_F8_KT
 #define HS2_F8_KT 16
 #endif
-constexpr int KT = HS2_F8_KT;                // key rows per stage (32-row stages were measured: 47.8 vs 45.3 us per decode step)
-constexpr int MT = KT / 16;                  // 16-key MMA tiles per stage
-static_assert(KT == 16 || KT == 32, "a stage holds 16 or 32 key rows");
+#ifndef HS2_F8_PKT
+#define HS2_F8_PKT 32
+#endif
+constexpr int KTD = HS2_F8_KT;               // key rows per stage, decode (32-row stages were measured: 47.8 vs 45.3 us per step)
+constexpr int KTP = HS2_F8_PKT;              // key rows per buffer, prefill
+static_assert((KTD == 16 || KTD == 32) && (KTP == 16 || KTP == 32), "a stage holds 16 or 32 key rows");
 #ifndef HS2_F8_NSTAGE
 #define HS2_F8_NSTAGE 2
 #endif
@@ -50,13 +53,16 @@ static_assert(KT == 16 || KT == 32, "a stage holds 16 or 32 key rows");
 #endif
 constexpr int NSTAGE = HS2_F8_NSTAGE;
 constexpr int kRow = HD;                     // bytes of one e4m3 row
-constexpr int kTile = KT * kRow;             // one K or V tile of a stage
-constexpr int kStageBytes = 2 * kTile;
-// per warp: the stages, then per stage: key index of each row (32 ints), K scales (KT), V scales (KT)
-constexpr int kMetaBytes = 32 * 4 + 2 * KT * 4;
-constexpr int kWarpSmem = NSTAGE * kStageBytes + NSTAGE * kMetaBytes;
+// a stage of KT rows: the K tile, the V tile; per stage also: key index of each row (32 ints), K scales (KT), V scales (KT)
+template <int KT> struct Stage {
+    static constexpr int MT = KT / 16;               // 16-key MMA tiles per stage
+    static constexpr int kTile = KT * kRow;          // one K or V tile
+    static constexpr int kStageBytes = 2 * kTile;
+    static constexpr int kMetaBytes = 32 * 4 + 2 * KT * 4;
+};
+constexpr int kWarpSmem = NSTAGE * (Stage<KTD>::kStageBytes + Stage<KTD>::kMetaBytes);   // decode
 constexpr int NSP = HS2_F8_PNSTAGE;
-constexpr int kWarpSmemP = NSP * kStageBytes + NSP * kMetaBytes;   // prefill
+constexpr int kWarpSmemP = NSP * (Stage<KTP>::kStageBytes + Stage<KTP>::kMetaBytes);     // prefill
 constexpr float kPShift = 256.f;             // probabilities x V scale are carried x 2^8 through the f16 operand
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -154,6 +160,7 @@ __device__ __forceinline__ Item make_item(const Params &p, const uint8_t *K, con
 // Slot s of the virtual slot array [idx row | window] holds a key index or is void (-1).  slot_raw starts the fetch
 // (an idx entry is a global load), slot_fix applies the validity rules when the value is used one tile later, so
 // that the load's latency is never waited for.
+template <int KT>
 __device__ __forceinline__ int slot_raw(const Params &p, const Item &it, int tile, int lane)
 {
     const int s = tile * KT + lane;
@@ -161,6 +168,7 @@ __device__ __forceinline__ int slot_raw(const Params &p, const Item &it, int til
     if (s < p.k) return it.irow ? __ldg(it.irow + s) : -1;
     return s < p.k + p.w ? it.pos - p.w + 1 + (s - p.k) : -1;
 }
+template <int KT>
 __device__ __forceinline__ int slot_fix(const Params &p, const Item &it, int tile, int lane, int j)
 {
     const int hi = tile * KT + lane < p.k ? it.pos - p.w : it.pos;   // idx entries inside the window are void
@@ -169,8 +177,10 @@ __device__ __forceinline__ int slot_fix(const Params &p, const Item &it, int til
 
 // lane -> 16-byte chunk c (of 8) of rows r0 + (lane >> 3); the lanes also fetch the stage's scales.  Void rows are
 // zero filled, nothing is read for them.
+template <int KT>
 __device__ __forceinline__ void issue_stage(const Item &it, uint32_t stage_base, uint32_t meta_base, int j, int lane)
 {
+    constexpr int kTile = Stage<KT>::kTile;
     const int c = lane & 7, hi = lane >> 3;
     const char *kc = it.Kb + c * 16, *vc = it.Vb + c * 16;
 #pragma unroll
@@ -193,10 +203,12 @@ __device__ __forceinline__ void issue_stage(const Item &it, uint32_t stage_base,
     }
 }
 
+template <int KT>
 __device__ __forceinline__ void consume_stage(Acc &acc, const uint32_t (&qf)[16], uint32_t stage_base, const float *sks,
                                               const float *svs, unsigned mask, float scale_log2, int lane,
                                               float *raw = nullptr, int lk = 0, int G = 0, const int *sjrow = nullptr)
 {
+    constexpr int MT = Stage<KT>::MT, kTile = Stage<KT>::kTile;
     const int g = lane >> 2;
     const int mi = lane >> 3, rr = lane & 7;
     float s[MT][4];
@@ -300,24 +312,25 @@ __device__ __forceinline__ void consume_stage(Acc &acc, const uint32_t (&qf)[16]
 
 // Fold slot tiles [t_begin, t_end) of one item into acc with an NS-deep cp.async pipeline.  NS = 1: fetch, wait, fold in
 // one buffer; the warp overlaps nothing by itself, but needs half the shared memory, so more warps are resident.
-template <int NS>
+template <int NS, int KT>
 __device__ __forceinline__ void run_tiles(const Params &p, const Item &it, const uint32_t (&qf)[16], Acc &acc, int t_begin,
                                           int t_end, char *wsm, int lane)
 {
+    constexpr int kStageBytes = Stage<KT>::kStageBytes, kMetaBytes = Stage<KT>::kMetaBytes;
     const uint32_t sbase = smem_u32(wsm);
     char *meta = wsm + NS * kStageBytes;
     const uint32_t mbase = sbase + NS * kStageBytes;
     int next = t_begin;
-    int jn = next < t_end ? slot_raw(p, it, next, lane) : -1;
+    int jn = next < t_end ? slot_raw<KT>(p, it, next, lane) : -1;
     int n_issued = 0, n_done = 0;
     auto try_issue = [&](int stage) -> bool {
         while (next < t_end) {
-            const int j = slot_fix(p, it, next, lane, jn);
+            const int j = slot_fix<KT>(p, it, next, lane, jn);
             ++next;
-            if (next < t_end) jn = slot_raw(p, it, next, lane);
+            if (next < t_end) jn = slot_raw<KT>(p, it, next, lane);
             if (__ballot_sync(0xffffffffu, j >= 0)) {   // all-void tiles are skipped
                 reinterpret_cast<int *>(meta + stage * kMetaBytes)[lane] = j;
-                issue_stage(it, sbase + stage * kStageBytes, mbase + stage * kMetaBytes, j, lane);
+                issue_stage<KT>(it, sbase + stage * kStageBytes, mbase + stage * kMetaBytes, j, lane);
                 return true;
             }
         }
@@ -329,7 +342,7 @@ __device__ __forceinline__ void run_tiles(const Params &p, const Item &it, const
             cp_async_wait<0>();
             __syncwarp();
             const unsigned mask = __ballot_sync(0xffffffffu, reinterpret_cast<const int *>(meta)[lane] >= 0);
-            consume_stage(acc, qf, sbase, reinterpret_cast<const float *>(meta + 32 * 4),
+            consume_stage<KT>(acc, qf, sbase, reinterpret_cast<const float *>(meta + 32 * 4),
                           reinterpret_cast<const float *>(meta + 32 * 4 + KT * 4), mask, p.scale_log2, lane, it.raw, it.lk, p.G,
                           reinterpret_cast<const int *>(meta));
             __syncwarp();   // every lane has read the buffer before the next tile's copies land in it
@@ -349,7 +362,7 @@ __device__ __forceinline__ void run_tiles(const Params &p, const Item &it, const
         cp_async_commit();
         const char *mt = meta + stage * kMetaBytes;
         const unsigned mask = __ballot_sync(0xffffffffu, reinterpret_cast<const int *>(mt)[lane] >= 0);
-        consume_stage(acc, qf, sbase + stage * kStageBytes, reinterpret_cast<const float *>(mt + 32 * 4),
+        consume_stage<KT>(acc, qf, sbase + stage * kStageBytes, reinterpret_cast<const float *>(mt + 32 * 4),
                       reinterpret_cast<const float *>(mt + 32 * 4 + KT * 4), mask, p.scale_log2, lane, it.raw, it.lk, p.G,
                       reinterpret_cast<const int *>(mt));
         ++n_done;
@@ -461,7 +474,7 @@ k_sparse_fp8_prefill(const Params p, const __nv_bfloat16 *__restrict__ Q, const 
     load_q_frags(p, Q, b, i, gkv, lane, qf);
     Acc acc;
     init_acc(acc, p, sink, gkv, lane, true);
-    run_tiles<NSP>(p, it, qf, acc, 0, (p.k + p.w + KT - 1) / KT, wsm, lane);
+    run_tiles<NSP, KTP>(p, it, qf, acc, 0, (p.k + p.w + KTP - 1) / KTP, wsm, lane);
     reduce_l(acc);
     store_output(p, acc, O, LSE, b, i, gkv, wsm, lane);
 }
@@ -487,9 +500,9 @@ k_sparse_fp8_decode(const Params p, const __nv_bfloat16 *__restrict__ Q, const u
     load_q_frags(p, Q, b, 0, gkv, lane, qf);
     Acc acc;
     init_acc(acc, p, sink, gkv, lane, warp == 0);   // the sink joins the denominator once
-    const int n_tiles = (p.k + p.w + KT - 1) / KT;
+    const int n_tiles = (p.k + p.w + KTD - 1) / KTD;
     const int per = (n_tiles + W - 1) / W;
-    run_tiles<NSTAGE>(p, it, qf, acc, warp * per, min(n_tiles, (warp + 1) * per), wsm, lane);
+    run_tiles<NSTAGE, KTD>(p, it, qf, acc, warp * per, min(n_tiles, (warp + 1) * per), wsm, lane);
     reduce_l(acc);
     float4 *op = reinterpret_cast<float4 *>(wsm);   // the warp's own staging area: [8][32] float4
 #pragma unroll
@@ -533,8 +546,9 @@ k_sparse_fp8_decode(const Params p, const __nv_bfloat16 *__restrict__ Q, const u
 
 constexpr int kPrefillSmem = HS2_F8_WARPS * kWarpSmemP;
 constexpr int kDecodeSmem = HS2_F8D_WARPS * kWarpSmem + HS2_F8D_WARPS * 16 * 4 + 8 * (HD + 8) * 2;
-static_assert(NSTAGE * kStageBytes >= 8 * 32 * 16, "a warp's stages hold its partial accumulator in decode");
-static_assert(NSTAGE * kStageBytes >= 8 * (HD + 8) * 2 && NSP * kStageBytes >= 8 * (HD + 8) * 2, "a warp's stages hold its staged output rows");
+static_assert(NSTAGE * Stage<KTD>::kStageBytes >= 8 * 32 * 16, "a warp's stages hold its partial accumulator in decode");
+static_assert(NSTAGE * Stage<KTD>::kStageBytes >= 8 * (HD + 8) * 2 && NSP * Stage<KTP>::kStageBytes >= 8 * (HD + 8) * 2,
+              "a warp's stages hold its staged output rows");
 
 template <class Kern>
 cudaError_t set_smem(Kern kern, int bytes, bool *done)
