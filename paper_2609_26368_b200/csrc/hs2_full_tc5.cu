@@ -3,7 +3,7 @@
 //
 // One CTA = 128 queries of one head (MMA M = 128), 320 threads, two CTAs per SM at head_dim 128 so that one
 // CTA's softmax overlaps the other's tensor work:
-//   warp 8   TMA producer: Q once, then K/V tiles of 64 keys into a 2-stage ring.  Every tile is a set of
+//   warp 8   TMA producer: Q once, then K and V tiles of 64 keys, each into a 2-stage ring of its own.  Every tile is a set of
 //            128-byte-swizzled slices ([rows][64 dims]), the canonical UMMA operand layout.
 //   warp 9   MMA issuer: S = Q K^T (M128 N64 K=D) into one of two S buffers in TMEM, and O += P V
 //            (M128 N=D K64, P as the tensor-memory A operand, V as an MN-major B operand) into TMEM.

@@ -17,7 +17,10 @@
 //   * the scales never touch the operands: the K scale multiplies the score row of its key, the V scale is
 //     folded into the probability of its key (times 2^8 to stay inside the normal range of f16; undone in the
 //     store).  The denominator sums the unscaled probabilities.
-// Decode: one CTA per (sequence, KV head), its warps split the attended set and merge through shared memory.
+// Prefill: one buffer of 32 rows per warp (fetch, wait, fold) and 16 warps per SM, as in the bf16 kernel - whose
+// warps need twice the shared memory, so that only 12 of them fit.  Decode: one CTA per (sequence, KV head), its
+// warps split the attended set (two stages of 16 rows each) and merge through shared memory; with a pointer for them
+// it also leaves the dequantised q.k of every (head, key) behind, for the selection of the full layer's decode step.
 #include <cuda_fp16.h>
 
 #include "hs2_common.cuh"
