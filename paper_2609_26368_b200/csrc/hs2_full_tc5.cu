@@ -1,18 +1,19 @@
 // Full causal attention on the 5th-generation tensor cores (tcgen05 + TMEM), bf16, head_dim 128 or 256
 // (Section 3.4: the full-attention layer; NoPE, Section 4.1).
 //
-// One CTA = 128 queries of one head (MMA M = 128), 320 threads, two CTAs per SM at head_dim 128 so that one
-// CTA's softmax overlaps the other's tensor work:
-//   warp 8   TMA producer: Q once, then K and V tiles of 64 keys, each into a 2-stage ring of its own.  Every tile is a set of
-//            128-byte-swizzled slices ([rows][64 dims]), the canonical UMMA operand layout.
-//   warp 9   MMA issuer: S = Q K^T (M128 N64 K=D) into one of two S buffers in TMEM, and O += P V
+// One CTA = 128 queries of one head (MMA M = 128), 128 HV + 64 threads (HV = threads per query row, 1 by default),
+// two CTAs per SM at head_dim 128 so that one CTA's softmax overlaps the other's tensor work:
+//   softmax warps (the first 4 HV warps): HV = 1: one thread per query row; HV = 2: warps w and w+4 share the 32 TMEM
+//            lanes of quarter w and take 32 keys of a tile each, the tile maximum agreed through shared memory and a
+//            named pair barrier (measured slower than HV = 1: the barrier and the doubled per-tile overhead cost more
+//            than the extra warps hide).  tcgen05.ld of the row, causal mask, online softmax in the base-2 domain
+//            with a lazily updated row maximum (O in TMEM is rescaled only when the maximum grows by more than 2^8,
+//            and only then does a softmax thread wait for P V of the previous tile), P written as bf16 pairs over
+//            the scores it came from (tcgen05.st).
+//   next warp TMA producer: Q once, then K and V tiles of 64 keys, each into a 2-stage ring of its own.  Every tile
+//            is a set of 128-byte-swizzled slices ([rows][64 dims]), the canonical UMMA operand layout.
+//   last warp MMA issuer: S = Q K^T (M128 N64 K=D) into one of two S buffers in TMEM, and O += P V
 //            (M128 N=D K64, P as the tensor-memory A operand, V as an MN-major B operand) into TMEM.
-//   warps 0-7 two threads per query row (warps w and w+4 share the 32 TMEM lanes of quarter w and take 32 keys
-//            of a tile each): tcgen05.ld of the half row, causal mask, the tile maximum agreed through shared
-//            memory and a named pair barrier, online softmax in the base-2 domain with a lazily updated row
-//            maximum (O in TMEM is rescaled only when the maximum grows by more than 2^8), P written as bf16
-//            pairs over the scores it came from (tcgen05.st).  Eight warps instead of four: the softmax is a
-//            chain of TMEM round trips and MUFU latencies, and four warps per scheduler hide it where two did not.
 // TMEM: columns 0-63 / 64-127 the two S buffers (P of a tile in the first 32 columns of its buffer), then the
 // O accumulator (fp32, lane = query row).
 // Every mbarrier wait is bounded; a wait that runs out sets a bit in a device error word, makes the CTA abandon
