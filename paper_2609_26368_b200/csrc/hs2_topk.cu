@@ -361,7 +361,8 @@ k_topk_cached(const Params p, const float *__restrict__ scores, int64_t score_st
             if (j0 + e >= nc) continue;
             if (key[e] > tau || key[e] == tau) {
                 const uint32_t j = (uint32_t)prow[j0 + e];
-                if (key[e] > tau || ~j >= jmin) atomicOr(&bitmap[j >> 5], 1u << (j & 31u));
+                // (the sweep only writes keys below n_keys; the range test keeps a damaged list from writing outside the bitmap)
+                if (j < (uint32_t)n_keys && (key[e] > tau || ~j >= jmin)) atomicOr(&bitmap[j >> 5], 1u << (j & 31u));
             }
         }
         __syncthreads();
