@@ -595,12 +595,16 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         int nq_r[kHoist ? TQW : 1];
         float *orow_r[kHoist && MODE != SC_FILTER ? TQW : 1];
         float tau_r[kHoist && MODE == SC_FILTER ? TQW : 1];   // thresholds as floats: one compare per score
+        int rb_r[kHoist && MODE == SC_FILTER ? TQW : 1];      // first slot of the query's candidate list (the lists of a block hold < 2^28 entries)
         if (kHoist) {
 #pragma unroll
             for (int q = 0; q < TQW; ++q) {
                 nq_r[q] = s_nq[q_first + q];
                 if (MODE != SC_FILTER) orow_r[q] = out + s_row[q_first + q] * out_stride;   // never used when nq is 0
-                if (MODE == SC_FILTER) tau_r[q] = key_to_float(s_tau[q_first + q]);
+                if (MODE == SC_FILTER) {
+                    tau_r[q] = key_to_float(s_tau[q_first + q]);
+                    rb_r[q] = (int)(s_row[q_first + q] * fb.cap);
+                }
             }
         }
         bool alive = true;
@@ -680,7 +684,7 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                         if ((passbits >> q) & 1u) {
                             const int pos = bq + __popc(masks[q] & lt_mask);
                             if (pos < fb.cap) {
-                                const int64_t o = s_row[q_first + q] * fb.cap + pos;
+                                const int64_t o = kHoist ? (int64_t)(rb_r[kHoist ? q : 0] + pos) : s_row[q_first + q] * fb.cap + pos;
                                 fb.cand_a[o] = aval[q];
                                 fb.cand_j[o] = key;
                             }
