@@ -472,10 +472,13 @@ __device__ __forceinline__ unsigned ge_exact(float v, float t)
 #ifndef HS2_TOPK_MINB32
 #define HS2_TOPK_MINB32 4
 #endif
+#ifndef HS2_TOPK_ROWS
+#define HS2_TOPK_ROWS 1    // rows per CTA of the linear kernel (consecutive queries of one (sequence, KV head))
+#endif
+// one row of k_topk_linear; every exit is taken by the whole CTA
 template <int THREADS, int E, bool VEC>
-__global__ void __launch_bounds__(THREADS, THREADS > 256 ? 1 : (E > 32 ? 2 : (HS2_TOPK_MINB32 * 256 / THREADS)))
-k_topk_linear(const Params p, const float *__restrict__ scores, int64_t score_stride, int32_t *__restrict__ idx,
-              int64_t row0, int nc_lo, int nc_hi, int64_t n_rows, int i_first)
+__device__ __forceinline__ void topk_linear_row(const Params &p, const float *__restrict__ scores, int64_t score_stride,
+                                                int32_t *__restrict__ idx, int64_t row0, int nc_lo, int nc_hi, int64_t row)
 {
     constexpr int WARPS = THREADS / 32;
     constexpr int NBT = HS2_TOPK_NBT;       // bins per thread
@@ -487,11 +490,6 @@ k_topk_linear(const Params p, const float *__restrict__ scores, int64_t score_st
     extern __shared__ int s_dyn[];          // [selected indices staged for the coalesced store][list: THREADS * E keys]
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    // i_first < 0: one CTA per row of the block.  Otherwise (positions known on the host) the grid covers only the
-    // queries whose candidate count falls into this launch's class: x = query offset from i_first, y = (sequence,
-    // KV head) from the block's first one; a launch then starts no CTAs that would leave at once.
-    const int64_t row = i_first < 0 ? row0 + blockIdx.x : (row0 / p.Lq + blockIdx.y) * p.Lq + i_first + blockIdx.x;   // (b, g, i), i fastest
-    if (row < row0 || row >= row0 + n_rows) return;
     const int64_t local = row - row0;
     const int i = (int)(row % p.Lq);
     const int b = (int)(row / ((int64_t)p.Lq * p.Hkv));
@@ -671,6 +669,31 @@ k_topk_linear(const Params p, const float *__restrict__ scores, int64_t score_st
         for (int t = tid; t < p.k; t += THREADS) out[t] = t < take ? s_out[t] : -1;
     } else {
         for (int t = take + tid; t < p.k; t += THREADS) out[t] = -1;
+    }
+}
+
+template <int THREADS, int E, bool VEC>
+__global__ void __launch_bounds__(THREADS, THREADS > 256 ? 1 : (E > 32 ? 2 : (HS2_TOPK_MINB32 * 256 / THREADS)))
+k_topk_linear(const Params p, const float *__restrict__ scores, int64_t score_stride, int32_t *__restrict__ idx,
+              int64_t row0, int nc_lo, int nc_hi, int64_t n_rows, int i_first)
+{
+    // i_first < 0: the CTAs walk the rows of the block in order.  Otherwise (positions known on the host) the grid covers
+    // only the queries whose candidate count falls into this launch's class: x = query offset from i_first, y =
+    // (sequence, KV head) from the block's first one; a launch then starts no CTAs that would leave at once.  A CTA
+    // takes HS2_TOPK_ROWS consecutive rows, which spreads the cost of starting it.
+    constexpr int R = HS2_TOPK_ROWS;
+#pragma unroll 1
+    for (int rr = 0; rr < R; ++rr) {
+        const int64_t x = (int64_t)blockIdx.x * R + rr;
+        int64_t row;
+        if (i_first < 0) {
+            row = row0 + x;
+        } else {
+            if (i_first + x >= p.Lq) break;
+            row = (row0 / p.Lq + blockIdx.y) * p.Lq + i_first + x;
+        }
+        if (row >= row0 && row < row0 + n_rows) topk_linear_row<THREADS, E, VEC>(p, scores, score_stride, idx, row0, nc_lo, nc_hi, row);
+        if (R > 1) __syncthreads();   // the next row reuses the shared arrays
     }
 }
 
@@ -1075,12 +1098,12 @@ void launch_class(int c, const Params &p, const float *scores, int64_t score_str
                 if (i_hi < i_lo) return false;
                 const int64_t n_bg = (row0 + n_rows - 1) / p.Lq - row0 / p.Lq + 1;
                 if (n_bg <= 65535) {
-                    kern<<<dim3((unsigned)(i_hi - i_lo + 1), (unsigned)n_bg), threads, smem, st>>>(p, scores, score_stride, idx, row0, lo, hi,
-                                                                                          n_rows, (int)i_lo);
+                    kern<<<dim3((unsigned)((i_hi - i_lo + HS2_TOPK_ROWS) / HS2_TOPK_ROWS), (unsigned)n_bg), threads, smem, st>>>(
+                        p, scores, score_stride, idx, row0, lo, hi, n_rows, (int)i_lo);
                     return true;
                 }
             }
-            kern<<<n, threads, smem, st>>>(p, scores, score_stride, idx, row0, lo, hi, n_rows, -1);
+            kern<<<(n + HS2_TOPK_ROWS - 1) / HS2_TOPK_ROWS, threads, smem, st>>>(p, scores, score_stride, idx, row0, lo, hi, n_rows, -1);
             return true;
         };
         bool launched = false;
