@@ -243,6 +243,17 @@ def test_mma_sync_fallback_kernels_of_the_full_layer():
         hs2.hs2_set_tcgen05_enabled(old)
 
 
+def test_full_layer_on_a_cache_larger_than_l2():
+    """A cache above 96 MB switches the attention kernel to its head-major CTA order (and chunks the score strips);
+    queries at the end of a 50K context, sampled rows against the oracle."""
+    wl = scaled("cfg2", q_len=384, kv_len=50176, k_sel=96, window=32, n_needles=8)
+    run = BlockRun(make_inputs(wl)).run_full()
+    rows = [(0, i) for i in (0, 1, 127, 128, 129, 255, 300, 383)]
+    run.check_full(rows=rows)
+    out, lse = run.run_sparse(0)
+    run.check_sparse(out, lse, 0, rows=rows)
+
+
 def test_paper_native_shape_mqa64_dim256_with_sink():
     """The attention shape of the paper's own model (Table 1: 64 query heads / 1 KV head, head dim 256,
     128 forced local + 1024 global tokens, per-head sink bias in the sparse layers), scaled in length."""
