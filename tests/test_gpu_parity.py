@@ -64,6 +64,8 @@ def _topk_case(scores: torch.Tensor, k, w, q_start=None, kv_lens=None):
 def test_topk_random_scores(Lk, k, w):
     g = torch.Generator().manual_seed(Lk)
     _topk_case(torch.randn(2, 2, 37, Lk, generator=g), k, w, q_start=[Lk - 37, Lk // 2], kv_lens=[Lk, Lk - 5])
+    # positions known on the host: every class launch covers only its own queries
+    _topk_case(torch.randn(1, 2, 61, Lk, generator=g) * 3.0 - 9.0, k, w)
 
 
 def test_topk_adversarial_rows():
