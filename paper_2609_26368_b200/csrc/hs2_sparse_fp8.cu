@@ -52,7 +52,7 @@ static_assert((KTD == 16 || KTD == 32) && (KTP == 16 || KTP == 32), "a stage hol
 #define HS2_F8_NSTAGE 2
 #endif
 #ifndef HS2_F8_PNSTAGE
-#define HS2_F8_PNSTAGE 1    // stages per warp in the prefill kernel (one buffer and 20 warps measured best)
+#define HS2_F8_PNSTAGE 1    // stages per warp in the prefill kernel (one buffer of 32 rows and 16 warps measured best)
 #endif
 constexpr int NSTAGE = HS2_F8_NSTAGE;
 constexpr int kRow = HD;                     // bytes of one e4m3 row
