@@ -37,7 +37,7 @@ from gen import CONFIGS, make_inputs, sample_rows  # noqa: E402
 
 # dram__bytes_read.sum + dram__bytes_write.sum of one k_sparse_prefill launch, from the ncu capture
 # summarised in profiles/block_step_cfg2.md (bytes)
-NCU_DRAM_TRAFFIC = {"cfg2": 269.2e6}
+NCU_DRAM_TRAFFIC = {"cfg2": 268.1e6}
 
 METRIC = "sparse-attn prefill tokens/s (hybrid block step: full-attn+select, sparse layers, decode step)"
 
