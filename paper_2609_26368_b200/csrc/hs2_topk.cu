@@ -475,6 +475,10 @@ __device__ __forceinline__ unsigned ge_exact(float v, float t)
 #ifndef HS2_TOPK_ROWS
 #define HS2_TOPK_ROWS 1    // rows per CTA of the linear kernel (consecutive queries of one (sequence, KV head))
 #endif
+#ifndef HS2_TOPK_WIDE
+#define HS2_TOPK_WIDE 1    // rows of 8193..16384 candidates: 32 per thread on 512 threads, two CTAs per SM (4 % faster than 64 per
+                           // thread on 256; the same step for the longest class, 1024 threads, measured 5 % slower)
+#endif
 // one row of k_topk_linear; every exit is taken by the whole CTA
 template <int THREADS, int E, bool VEC>
 __device__ __forceinline__ void topk_linear_row(const Params &p, const float *__restrict__ scores, int64_t score_stride,
@@ -673,7 +677,7 @@ __device__ __forceinline__ void topk_linear_row(const Params &p, const float *__
 }
 
 template <int THREADS, int E, bool VEC>
-__global__ void __launch_bounds__(THREADS, THREADS > 256 ? 1 : (E > 32 ? 2 : (HS2_TOPK_MINB32 * 256 / THREADS)))
+__global__ void __launch_bounds__(THREADS, THREADS > 256 ? (THREADS == 512 && E <= 32 ? 2 : 1) : (E > 32 ? 2 : (HS2_TOPK_MINB32 * 256 / THREADS)))
 k_topk_linear(const Params p, const float *__restrict__ scores, int64_t score_stride, int32_t *__restrict__ idx,
               int64_t row0, int nc_lo, int nc_hi, int64_t n_rows, int i_first)
 {
@@ -1111,7 +1115,11 @@ void launch_class(int c, const Params &p, const float *scores, int64_t score_str
             case 0: launched = go(k_topk_linear<64, 32, VEC>, 64, 32); break;
             case 1: launched = go(k_topk_linear<128, 32, VEC>, 128, 32); break;
             case 2: launched = go(k_topk_linear<256, 32, VEC>, 256, 32); break;
+#if HS2_TOPK_WIDE
+            case 3: launched = go(k_topk_linear<512, 32, VEC>, 512, 32); break;
+#else
             case 3: launched = go(k_topk_linear<256, 64, VEC>, 256, 64); break;
+#endif
             default: launched = go(k_topk_linear<512, 64, VEC>, 512, 64); break;
         }
         if (launched) count_launch();
