@@ -68,8 +68,8 @@ def test_topk_random_scores(Lk, k, w):
     _topk_case(torch.randn(1, 2, 61, Lk, generator=g) * 3.0 - 9.0, k, w)
 
 
-def test_topk_adversarial_rows():
-    Lk = 2500
+@pytest.mark.parametrize("Lk", [2500, 12000, 20000])   # 128, 512 and 512 x 64 thread classes
+def test_topk_adversarial_rows(Lk):
     g = torch.Generator().manual_seed(5)
     rows = [
         torch.zeros(Lk),                                                   # all equal: lowest indices win
