@@ -54,11 +54,22 @@ __device__ __forceinline__ int producer_ordinal(int w) { return w == 3 ? 0 : w -
 // Shared-memory plan for head_dim D.  The MMA always reads 128 A rows per 64-dim slice of Q; rows past the 64
 // that are loaded alias whatever follows (the next slice or the K ring), which is harmless: they only produce
 // TMEM lanes that nobody reads.
+#ifndef HS2_SPTC5_PTMEM
+#define HS2_SPTC5_PTMEM 1   // P as a tensor-memory operand of P V (0: through shared memory)
+#endif
+#ifndef HS2_SPTC5_VST3
+#define HS2_SPTC5_VST3 1    // three V stages at head_dim 256 (needs P in tensor memory)
+#endif
+
 template <int D>
 struct SpCfg {
     static constexpr int NQ = D / 64;                           // 64-dim slices of an operand tile
     static constexpr int CH = D / 8;                            // 16-byte chunks per row
-    static constexpr int KST = D == 256 ? 3 : 2;                // K ring depth (V ring: 2)
+    static constexpr int KST = D == 256 ? 3 : 2;                // K ring depth
+    // V ring depth: with P in tensor memory its 16 KB of shared memory, and most of the alignment slack, buy a third
+    // V stage at head_dim 256 (the layout then fills the 227 KB to the byte)
+    static constexpr int VST = (D == 256 && HS2_SPTC5_PTMEM && HS2_SPTC5_VST3) ? 3 : 2;
+    static constexpr uint32_t kSlack = VST == 3 ? 256 : kAlignSlack;
     static constexpr int PW = D == 256 ? HS2_SP_PWARPS : 1;     // warps per gather group (one K group, one V group)
     static constexpr int kThreads = (5 + 2 * PW) * 32;
     static constexpr uint32_t kQSlice = kSubHeads * 128;
@@ -69,22 +80,22 @@ struct SpCfg {
     // on into the K ring (don't-care rows again)
     static constexpr uint32_t kOffP = kOffQ + kQBytes;
     static constexpr uint32_t kPStride = kSubHeads * 128;
-    static constexpr uint32_t kOffK = kOffP + 2 * kPStride;
+    static constexpr uint32_t kOffK = kOffP + (HS2_SPTC5_PTMEM ? 0 : 2 * kPStride);
     static constexpr uint32_t kOffV = kOffK + KST * kKVStage;
-    static constexpr uint32_t kOffKey = kOffV + 2 * kKVStage;   // int[2 groups][2][64]: key index per slot of a tile
+    static constexpr uint32_t kOffKey = kOffV + VST * kKVStage;   // int[2 groups][2][64]: key index per slot of a tile
     static constexpr uint32_t kOffMx = kOffKey + 4 * BN * 4;    // float[2 tiles][2 halves][64]: row maxima exchanged
     static constexpr uint32_t kOffL = kOffMx + 4 * 64 * 4;      // float[2 halves][64]: row sums exchanged
     static constexpr uint32_t kOffBar = kOffL + 2 * 64 * 4;
-    static constexpr uint32_t kSmemBytes = kOffBar + kBarBytes + kAlignSlack;
+    static constexpr uint32_t kSmemBytes = kOffBar + kBarBytes + kSlack;
     static constexpr uint32_t kTmem = D <= 128 ? 256 : 512;     // 2 x 64 score columns + D output columns
     static constexpr int kMinBlocks = D <= 128 ? 2 : 1;
-    static_assert(kOffQ + (NQ - 1) * kQSlice + BM * 128 <= kOffKey && kOffP + kPStride + BM * 128 <= kOffKey,
+    static_assert(kOffQ + (NQ - 1) * kQSlice + BM * 128 <= kOffKey && (HS2_SPTC5_PTMEM || kOffP + kPStride + BM * 128 <= kOffKey),
                   "the 128 A rows the MMA reads stay inside the buffer");
     static_assert(kSmemBytes <= 227 * 1024, "fits the shared memory of one SM");
 };
 
 enum Bar {
-    Q_FULL = 0, Q_EMPTY, K_FULL0, K_FULL1, K_FULL2, K_EMPTY0, K_EMPTY1, K_EMPTY2, V_FULL0, V_FULL1, V_EMPTY0, V_EMPTY1,
+    Q_FULL = 0, Q_EMPTY, K_FULL0, K_FULL1, K_FULL2, K_EMPTY0, K_EMPTY1, K_EMPTY2, V_FULL0, V_FULL1, V_FULL2, V_EMPTY0, V_EMPTY1, V_EMPTY2,
     S_FULL0, S_FULL1, S_FREE0, S_FREE1, P_FULL0, P_FULL1, PV_DONE0, PV_DONE1, O_FREE, N_BARS
 };
 static_assert(N_BARS * 8 + 8 <= kBarBytes, "barriers, TMEM slot and abort flag fit their block");
@@ -136,7 +147,7 @@ k_sparse_tc5(const __grid_constant__ CUtensorMap tmQ, const Params p, const __nv
     extern __shared__ char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
     const uint32_t pad = (1024u - (raw & 1023u)) & 1023u;
-    if (pad > kAlignSlack) {
+    if (pad > C::kSlack) {
         if (threadIdx.x == 0) atomicOr(&g_sptc5_error, 2u);
         return;
     }
@@ -175,9 +186,11 @@ k_sparse_tc5(const __grid_constant__ CUtensorMap tmQ, const Params p, const __nv
     if (tid == 0) {
         *abort_flag = 0;
         mbar_init(bar(Q_FULL), 1); mbar_init(bar(Q_EMPTY), 1);
-        for (int s = 0; s < 3; ++s) { mbar_init(bar(K_FULL0 + s), 32 * C::PW); mbar_init(bar(K_EMPTY0 + s), 1); }
-        for (int s = 0; s < 2; ++s) {
+        for (int s = 0; s < 3; ++s) {
+            mbar_init(bar(K_FULL0 + s), 32 * C::PW); mbar_init(bar(K_EMPTY0 + s), 1);
             mbar_init(bar(V_FULL0 + s), 32 * C::PW); mbar_init(bar(V_EMPTY0 + s), 1);
+        }
+        for (int s = 0; s < 2; ++s) {
             mbar_init(bar(S_FULL0 + s), 1); mbar_init(bar(S_FREE0 + s), 128);
             mbar_init(bar(P_FULL0 + s), 128); mbar_init(bar(PV_DONE0 + s), 1);
         }
@@ -283,12 +296,19 @@ k_sparse_tc5(const __grid_constant__ CUtensorMap tmQ, const Params p, const __nv
                         pk[e >> 1] = pack_bf16(p0, p1);
                     }
                     l += l0 + l1;
+#if HS2_SPTC5_PTMEM
+                    // P replaces the scores it came from: bf16 pairs over the first 32 columns of the score buffer, this
+                    // half's 32 keys in 16 of them (the partner has read its scores: it passed the pair barrier above)
+                    tmem_st16u(lane_base + sb * BN + 16 * half, pk);
+                    tmem_wait_st();
+#else
                     char *prow_ptr = smem + C::kOffP + sb * C::kPStride + row * 128;
 #pragma unroll
                     for (int c4 = 0; c4 < 4; ++c4)   // 8 keys = one 16-byte chunk, chunk position XOR (row & 7)
                         *reinterpret_cast<uint4 *>(prow_ptr + (((half * 4 + c4) ^ (row & 7)) << 4)) =
                             make_uint4(pk[4 * c4], pk[4 * c4 + 1], pk[4 * c4 + 2], pk[4 * c4 + 3]);
                     fence_proxy_async();
+#endif
                     tc_fence_before();
                     mbar_arrive(bar(P_FULL0 + sb));
                 }
@@ -385,21 +405,29 @@ k_sparse_tc5(const __grid_constant__ CUtensorMap tmQ, const Params p, const __nv
                 ok = ok && issue_s(0);
                 for (int t = 0; ok && t < nblk; ++t) {
                     if (t + 1 < nblk && !issue_s(t + 1)) { ok = false; break; }
-                    const int g = g0 + t, vs = g & 1;
-                    if (!mbar_wait(bar(P_FULL0 + vs), (g >> 1) & 1, abort_flag)) { ok = false; break; }
-                    if (!mbar_wait(bar(V_FULL0 + vs), (g >> 1) & 1, abort_flag) ||
+                    const int g = g0 + t, pb = g & 1, vs = g % C::VST;   // P / score buffer, V stage
+                    if (!mbar_wait(bar(P_FULL0 + pb), (g >> 1) & 1, abort_flag)) { ok = false; break; }
+                    if (!mbar_wait(bar(V_FULL0 + vs), (g / C::VST) & 1, abort_flag) ||
                         (t == 0 && !mbar_wait(bar(O_FREE), (n & 1) ^ 1, abort_flag))) { ok = false; break; }
                     fence_proxy_async();
                     tc_fence_after();
-                    const uint64_t dp = smem_desc(sbase + C::kOffP + vs * C::kPStride, 16, 1024);
+#if !HS2_SPTC5_PTMEM
+                    const uint64_t dp = smem_desc(sbase + C::kOffP + pb * C::kPStride, 16, 1024);
+#endif
                     // V: MN-major B operand, 64-dim slices BN*128 bytes apart (leading offset), 8-key groups 1024 bytes apart
                     const uint64_t dv = smem_desc(sbase + C::kOffV + vs * kKVStage, BN * 128, 1024);
 #pragma unroll
                     for (int kk = 0; kk < 4; ++kk) {   // 16 keys per instruction
+#if HS2_SPTC5_PTMEM
+                        // P: tensor-memory A operand, 16 keys = 8 columns of bf16 pairs; the in-order tensor pipe runs
+                        // Q K^T of tile g+2, which overwrites that score buffer, after this instruction
+                        umma_ts(tmem + 2 * BN, tmem + pb * BN + kk * 8, dv + ((kk * 2048) >> 4), idPV, (t > 0 || kk > 0) ? 1u : 0u);
+#else
                         umma(tmem + 2 * BN, dp + ((kk * 32) >> 4), dv + ((kk * 2048) >> 4), idPV, (t > 0 || kk > 0) ? 1u : 0u);
+#endif
                     }
                     umma_commit(bar(V_EMPTY0 + vs));
-                    umma_commit(bar(PV_DONE0 + vs));
+                    umma_commit(bar(PV_DONE0 + pb));
                 }
             }
         }
@@ -420,11 +448,11 @@ k_sparse_tc5(const __grid_constant__ CUtensorMap tmQ, const Params p, const __nv
         const int64_t row_bytes = p.ks_t * 2;
         const __nv_bfloat16 *src_t = is_v ? V : K;
         const uint32_t ring0 = sbase + (is_v ? C::kOffV : C::kOffK) + dst_c;
-        const int nst = is_v ? 2 : KST;
+        const int nst = is_v ? C::VST : KST;
         const int bar_full = is_v ? V_FULL0 : K_FULL0, bar_empty = is_v ? V_EMPTY0 : K_EMPTY0;
         int *keys_base = s_key + is_v * 2 * BN;       // two records per group
         // the key indices of a tile are fetched one tile ahead (the idx row is read from global memory, and that
-        // latency would otherwise sit in front of every tile's copies)
+        // latency would otherwise sit in front of every tile's copies; three and five tiles ahead measured the same)
         int j_next[KPT];
 #pragma unroll
         for (int u = 0; u < KPT; ++u) j_next[u] = -1;
