@@ -90,6 +90,22 @@ def test_topk_adversarial_rows(Lk):
         _topk_case(scores, k, w, q_start=[Lk - 1 - len(rows) + 1])
 
 
+def test_topk_longest_register_class_with_prefetched_rows():
+    """Positions known on the host and rows of 16385..32768 candidates: one CTA takes consecutive queries and fetches the
+    next row during the current one; rows whose threshold bin holds (nearly) the whole row push the list into the
+    prefetch buffer, so the row after them is read the plain way."""
+    Lk, Lq = 24000, 40
+    g = torch.Generator().manual_seed(77)
+    s = torch.randn(1, 2, Lq, Lk, generator=g) * 2.0 - 10.0
+    s[0, 0, 3] = -4.0                                              # all equal: the list holds the whole row
+    s[0, 0, 4] = (s[0, 0, 4] * 2).round() / 2                      # heavy ties
+    s[0, 0, 17, : Lk // 2] = -7.5                                  # half of the row in one bin
+    s[0, 1, 20:23] = 0.0
+    s[0, 1, 30] = torch.where(torch.arange(Lk) % 3 == 0, torch.tensor(-1.0), torch.tensor(-1.0e-41))   # denormals against a flat rest
+    for k, w in [(2048, 128), (1000, 0), (4096, 333), (5000, 64)]:    # staged and unstaged output rows
+        _topk_case(s, k, w)
+
+
 @pytest.mark.parametrize("Lk,k,w", [(40000, 2048, 128), (70001, 4096, 256), (131072, 4096, 256), (200003, 1000, 17),
                                      (262144, 4096, 0), (300000, 512, 64)])
 def test_topk_long_rows_cluster_and_streaming_variants(Lk, k, w):
