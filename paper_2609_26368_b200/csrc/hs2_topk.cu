@@ -475,6 +475,9 @@ __device__ __forceinline__ unsigned ge_exact(float v, float t)
 #ifndef HS2_TOPK_ROWS
 #define HS2_TOPK_ROWS 1    // rows per CTA of the linear kernel (consecutive queries of one (sequence, KV head))
 #endif
+#ifndef HS2_TOPK_STAGE
+#define HS2_TOPK_STAGE 1      // rows reach the registers through a coalesced copy into shared memory
+#endif
 #ifndef HS2_TOPK_PRE
 #define HS2_TOPK_PRE 1        // longest register class: the next row streams into shared memory during the current one
 #endif
@@ -542,6 +545,27 @@ __device__ __forceinline__ bool topk_linear_row(const Params &p, const float *__
 
     const int j0 = tid * E;
     const bool has = j0 < nc;   // threads (whole warps, on short rows) past the row's end skip every per-candidate loop
+    constexpr int CPT = E / 4;  // 16-byte chunks per thread
+#if HS2_TOPK_STAGE
+    // A thread's candidates are E consecutive floats, so its own 16-byte loads would sit E * 4 bytes apart between
+    // lanes: 32 cache lines per warp instruction.  Instead consecutive lanes copy consecutive chunks into the (still
+    // unused) list, chunk c at slot c + c / CPT, and every thread then reads its chunks at a pitch of CPT + 1 slots:
+    // both sides are free of bank conflicts.
+    float *s_stage = reinterpret_cast<float *>(s_dyn + (((staged ? p.k : 0) + 3) & ~3));
+    const bool from_stage = VEC && !PRE;
+    if (from_stage) {
+#pragma unroll
+        for (int it = 0; it < CPT; ++it) {
+            const int c = it * THREADS + tid;
+            if (4 * c + 4 <= nc) topk_cp_async16(s_stage + (c + c / CPT) * 4, srow + 4 * c);
+        }
+        topk_cp_async_wait_all();
+        __syncthreads();
+    }
+#else
+    constexpr bool from_stage = false;
+    float *s_stage = nullptr;
+#endif
     float val[E];
     float vmin = INFINITY, vmax = -INFINITY;
     if (has)
@@ -549,6 +573,7 @@ __device__ __forceinline__ bool topk_linear_row(const Params &p, const float *__
     for (int e4 = 0; e4 < E; e4 += 4) {
         if (VEC && j0 + e4 + 4 <= nc) {
             const float4 v = (PRE && have_pre) ? *reinterpret_cast<const float4 *>(s_pre + (17 * tid + (e4 >> 2)) * 4)
+                             : from_stage      ? *reinterpret_cast<const float4 *>(s_stage + ((CPT + 1) * tid + (e4 >> 2)) * 4)
                                                : __ldg(reinterpret_cast<const float4 *>(srow + j0 + e4));
             val[e4] = v.x; val[e4 + 1] = v.y; val[e4 + 2] = v.z; val[e4 + 3] = v.w;
             vmin = fminf(fminf(vmin, v.x), fminf(v.y, fminf(v.z, v.w)));
@@ -1171,14 +1196,15 @@ void launch_class(int c, const Params &p, const float *scores, int64_t score_str
 #if HS2_TOPK_LINEAR
     if (c <= 4) {   // register-resident rows: first round on a linear scale, the threshold bin's members in a shared list
         auto go = [&](auto kern, int threads, int e) -> bool {   // false: nothing was launched
-            const size_t smem = stage + (size_t)threads * e * sizeof(uint32_t);
+            // (+ one 16-byte slot per thread and the alignment of the staged row, which passes through the list's memory)
+            const size_t smem = stage + (size_t)threads * e * sizeof(uint32_t) + (size_t)threads * 16 + 16;
             if (smem > 32 * 1024) {   // static shared memory counts against the 48 KB default too
                 static bool attr_set[5][64] = {};   // per row class: the kernels share one function type, hence one lambda body
                 int dev = 0;
                 if (cudaGetDevice(&dev) != cudaSuccess) return false;
                 if (!(dev >= 0 && dev < 64 && attr_set[c][dev])) {
                     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)(kStageOut * sizeof(int) + (size_t)threads * e * sizeof(uint32_t))) != cudaSuccess)
+                                             (int)(kStageOut * sizeof(int) + (size_t)threads * e * sizeof(uint32_t) + (size_t)threads * 16 + 16)) != cudaSuccess)
                         return false;
                     if (dev >= 0 && dev < 64) attr_set[c][dev] = true;
                 }
