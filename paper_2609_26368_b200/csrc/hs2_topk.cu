@@ -478,12 +478,6 @@ __device__ __forceinline__ unsigned ge_exact(float v, float t)
 #ifndef HS2_TOPK_STAGE
 #define HS2_TOPK_STAGE 1      // rows reach the registers through a coalesced copy into shared memory
 #endif
-#ifndef HS2_TOPK_PRE
-#define HS2_TOPK_PRE 1        // longest register class: the next row streams into shared memory during the current one
-#endif
-#ifndef HS2_TOPK_PRE_ROWS
-#define HS2_TOPK_PRE_ROWS 16  // consecutive queries per CTA of that variant
-#endif
 #ifndef HS2_TOPK_WIDE
 #define HS2_TOPK_WIDE 1    // rows of 8193..16384 candidates: 32 per thread on 512 threads, two CTAs per SM (4 % faster than 64 per
                            // thread on 256; the same step for the longest class, 1024 threads, measured 5 % slower)
@@ -497,19 +491,10 @@ __device__ __forceinline__ void topk_cp_async_wait_all()
     asm volatile("cp.async.commit_group;\n cp.async.wait_group 0;\n" ::: "memory");
 }
 
-// Candidates the list of the prefetching variant holds by itself; a longer list runs on into the prefetch buffer
-constexpr int kPreListCap = 12288;
-
-// one row of k_topk_linear; every exit is taken by the whole CTA.
-// PRE (rows of one block taken in order by one CTA): the row's 16-byte chunks may already sit in shared memory
-// (`have_pre`, chunk c of the row at s_pre[(c + c / 16) * 4], in flight until waited for), and the chunks of
-// the next row (`next_srow`, `next_nc` candidates; none when next_nc <= 0) are fetched into the same buffer while
-// this row's rounds run.  Returns whether that prefetch stands (false: none was issued, or the list needed the room).
-template <int THREADS, int E, bool VEC, bool PRE = false>
-__device__ __forceinline__ bool topk_linear_row(const Params &p, const float *__restrict__ scores, int64_t score_stride,
-                                                int32_t *__restrict__ idx, int64_t row0, int nc_lo, int nc_hi, int64_t row,
-                                                float *s_pre = nullptr, bool have_pre = false,
-                                                const float *next_srow = nullptr, int next_nc = 0)
+// one row of k_topk_linear; every exit is taken by the whole CTA
+template <int THREADS, int E, bool VEC>
+__device__ __forceinline__ void topk_linear_row(const Params &p, const float *__restrict__ scores, int64_t score_stride,
+                                                int32_t *__restrict__ idx, int64_t row0, int nc_lo, int nc_hi, int64_t row)
 {
     constexpr int WARPS = THREADS / 32;
     constexpr int NBT = HS2_TOPK_NBT;       // bins per thread
@@ -521,10 +506,6 @@ __device__ __forceinline__ bool topk_linear_row(const Params &p, const float *__
     extern __shared__ int s_dyn[];          // [selected indices staged for the coalesced store][list: THREADS * E keys]
 
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    if (PRE && have_pre) {   // this row's chunks were fetched during the previous row
-        topk_cp_async_wait_all();
-        __syncthreads();
-    }
     const int64_t local = row - row0;
     const int i = (int)(row % p.Lq);
     const int b = (int)(row / ((int64_t)p.Lq * p.Hkv));
@@ -532,12 +513,12 @@ __device__ __forceinline__ bool topk_linear_row(const Params &p, const float *__
     const int pos = pos_of(p, b, i);
     const int nc = max(0, min(pos - p.w + 1, kvl));   // the row's candidates are keys 0..nc-1
     const int take = min(p.k, nc);                    // how many of them are selected
-    if (nc <= nc_lo || nc > nc_hi) return false;      // this row belongs to another variant's launch
+    if (nc <= nc_lo || nc > nc_hi) return;            // this row belongs to another variant's launch
     int32_t *out = idx + row * p.k;
     const float *srow = scores + local * score_stride;
     if (take == nc) {   // every candidate is kept: no need to look at the scores
         for (int t = tid; t < p.k; t += THREADS) out[t] = t < nc ? t : -1;
-        return false;
+        return;
     }
     const bool staged = p.k <= kStageOut;
     int *s_out = s_dyn;
@@ -550,10 +531,10 @@ __device__ __forceinline__ bool topk_linear_row(const Params &p, const float *__
     // A thread's candidates are E consecutive floats, so its own 16-byte loads would sit E * 4 bytes apart between
     // lanes: 32 cache lines per warp instruction.  Instead consecutive lanes copy consecutive chunks into the (still
     // unused) list, chunk c at slot c + c / CPT, and every thread then reads its chunks at a pitch of CPT + 1 slots:
-    // both sides are free of bank conflicts.
+    // both sides are free of bank conflicts.  (Fetching the NEXT row this way during the current one, a CTA taking
+    // 16 consecutive queries, was also built: no faster than this, so the load's cost was its access pattern.)
     float *s_stage = reinterpret_cast<float *>(s_dyn + (((staged ? p.k : 0) + 3) & ~3));
-    const bool from_stage = VEC && !PRE;
-    if (from_stage) {
+    if (VEC) {
 #pragma unroll
         for (int it = 0; it < CPT; ++it) {
             const int c = it * THREADS + tid;
@@ -562,6 +543,7 @@ __device__ __forceinline__ bool topk_linear_row(const Params &p, const float *__
         topk_cp_async_wait_all();
         __syncthreads();
     }
+    constexpr bool from_stage = VEC;
 #else
     constexpr bool from_stage = false;
     float *s_stage = nullptr;
@@ -572,9 +554,8 @@ __device__ __forceinline__ bool topk_linear_row(const Params &p, const float *__
 #pragma unroll
     for (int e4 = 0; e4 < E; e4 += 4) {
         if (VEC && j0 + e4 + 4 <= nc) {
-            const float4 v = (PRE && have_pre) ? *reinterpret_cast<const float4 *>(s_pre + (17 * tid + (e4 >> 2)) * 4)
-                             : from_stage      ? *reinterpret_cast<const float4 *>(s_stage + ((CPT + 1) * tid + (e4 >> 2)) * 4)
-                                               : __ldg(reinterpret_cast<const float4 *>(srow + j0 + e4));
+            const float4 v = from_stage ? *reinterpret_cast<const float4 *>(s_stage + ((CPT + 1) * tid + (e4 >> 2)) * 4)
+                                        : __ldg(reinterpret_cast<const float4 *>(srow + j0 + e4));
             val[e4] = v.x; val[e4 + 1] = v.y; val[e4 + 2] = v.z; val[e4 + 3] = v.w;
             vmin = fminf(fminf(vmin, v.x), fminf(v.y, fminf(v.z, v.w)));
             vmax = fmaxf(fmaxf(vmax, v.x), fmaxf(v.y, fmaxf(v.z, v.w)));
@@ -597,17 +578,6 @@ __device__ __forceinline__ bool topk_linear_row(const Params &p, const float *__
     for (int t = 0; t < NBT; ++t) hist[t * THREADS + tid] = 0u;
     if (tid == 0) s_cnt = 0u;
     __syncthreads();
-    bool pre_ok = false;
-    if (PRE && VEC && next_nc > 0) {   // every thread has taken its chunks out of the buffer: fetch the next row's
-        // consecutive lanes copy consecutive chunks (coalesced); chunk c lands in slot c + c / 16, so that the owner
-        // of chunks 16 t .. 16 t + 15 reads them at a pitch of 17 slots, free of bank conflicts
-#pragma unroll
-        for (int it = 0; it < E / 4; ++it) {
-            const int c = it * THREADS + tid;
-            if (4 * c + 4 <= next_nc) topk_cp_async16(s_pre + (c + (c >> 4)) * 4, next_srow + 4 * c);
-        }
-        pre_ok = true;
-    }
 #pragma unroll
     for (int w = 0; w < WARPS; ++w) { vmin = fminf(vmin, s_lo[w]); vmax = fmaxf(vmax, s_hi[w]); }
     // bin(v) = clamp(floor(v * c + d), 0, NB - 1) with one fused multiply-add: monotone in v, and the same
@@ -640,11 +610,6 @@ __device__ __forceinline__ bool topk_linear_row(const Params &p, const float *__
     __syncthreads();
     const unsigned tbin = s_bin;
     unsigned need = s_need;
-    if (PRE && pre_ok && hist[tbin] > (unsigned)kPreListCap) {   // (uniform) the list will run on into the prefetch buffer
-        topk_cp_async_wait_all();
-        __syncthreads();
-        pre_ok = false;
-    }
     // the threshold bin's members, as keys
     // (bin_of(v) == tbin as a range test on the same fused multiply-add: floor(x) == tbin; the clamped ends are open:
     // nothing is below -inf, and no comparison with NaN holds, so bin 0 takes NaN and -inf, the last bin +inf)
@@ -744,7 +709,6 @@ __device__ __forceinline__ bool topk_linear_row(const Params &p, const float *__
     } else {
         for (int t = take + tid; t < p.k; t += THREADS) out[t] = -1;
     }
-    return pre_ok;
 }
 
 template <int THREADS, int E, bool VEC>
@@ -770,50 +734,6 @@ k_topk_linear(const Params p, const float *__restrict__ scores, int64_t score_st
         if (row >= row0 && row < row0 + n_rows) topk_linear_row<THREADS, E, VEC>(p, scores, score_stride, idx, row0, nc_lo, nc_hi, row);
         if (R > 1) __syncthreads();   // the next row reuses the shared arrays
     }
-}
-
-// The same for the longest class with the next row's fetch overlapped: a CTA takes `rows_per_cta` consecutive queries of
-// one (sequence, KV head), and while it works on one row the next one streams into shared memory (a single CTA of this
-// size is resident per SM, so nothing else would cover the load).  Dynamic shared memory: [staged output][list of
-// kPreListCap keys][prefetch buffer of 17 slots of 16 bytes per thread, 16-byte aligned]; a list that outgrows its part runs on into
-// the buffer, after the fetch has been waited for and given up.
-template <int THREADS, int E, bool VEC>
-__global__ void __launch_bounds__(THREADS, 1)
-k_topk_linear_pre(const Params p, const float *__restrict__ scores, int64_t score_stride, int32_t *__restrict__ idx,
-                  int64_t row0, int nc_lo, int nc_hi, int64_t n_rows, int i_first, int rows_per_cta)
-{
-    extern __shared__ int s_dyn_pre[];
-    const int stage_ints = p.k <= kStageOut ? p.k : 0;
-    float *s_pre = reinterpret_cast<float *>(s_dyn_pre + ((stage_ints + kPreListCap + 3) & ~3));
-    auto row_of = [&](int64_t x) { return (row0 / p.Lq + blockIdx.y) * p.Lq + i_first + x; };
-    auto nc_of = [&](int64_t row) {
-        const int i = (int)(row % p.Lq);
-        const int b = (int)(row / ((int64_t)p.Lq * p.Hkv));
-        return max(0, min(pos_of(p, b, i) - p.w + 1, kvlen_of(p, b)));
-    };
-    bool have = false;
-#pragma unroll 1
-    for (int rr = 0; rr < rows_per_cta; ++rr) {
-        const int64_t x = (int64_t)blockIdx.x * rows_per_cta + rr;
-        if (i_first + x >= p.Lq) break;
-        const int64_t row = row_of(x);
-        // the next row of this CTA, when it exists, belongs to this launch and has something to select
-        int next_nc = 0;
-        const float *next_srow = nullptr;
-        if (rr + 1 < rows_per_cta && i_first + x + 1 < p.Lq && row + 1 >= row0 && row + 1 < row0 + n_rows) {
-            const int nn = nc_of(row + 1);
-            if (nn > nc_lo && nn <= nc_hi && min(p.k, nn) < nn) {
-                next_nc = nn;
-                next_srow = scores + (row + 1 - row0) * score_stride;
-            }
-        }
-        if (row >= row0 && row < row0 + n_rows)
-            have = topk_linear_row<THREADS, E, VEC, true>(p, scores, score_stride, idx, row0, nc_lo, nc_hi, row, s_pre, have, next_srow, next_nc);
-        else
-            have = false;
-        __syncthreads();   // the next row reuses the shared arrays
-    }
-    if (have) topk_cp_async_wait_all();   // nothing stays in flight when the CTA leaves
 }
 
 // ---- rows of up to CL x 32768 candidates: one thread-block cluster per row ------------------------
@@ -1227,34 +1147,6 @@ void launch_class(int c, const Params &p, const float *scores, int64_t score_str
             return true;
         };
         bool launched = false;
-#if HS2_TOPK_PRE
-        // the longest class, positions known on the host, aligned rows: consecutive queries per CTA, next row prefetched
-        if (c == 4 && VEC && !p.q_start && !p.kv_lens) {
-            const int64_t base = (int64_t)p.Lk - p.Lq - p.w + 1;
-            int64_t i_lo = (int64_t)lo + 1 - base, i_hi = hi >= p.Lk ? (int64_t)p.Lq - 1 : (int64_t)hi - base;
-            if (i_lo < 0) i_lo = 0;
-            if (i_hi > p.Lq - 1) i_hi = p.Lq - 1;
-            const int64_t n_bg = (row0 + n_rows - 1) / p.Lq - row0 / p.Lq + 1;
-            const size_t smem = ((size_t)(p.k <= kStageOut ? p.k : 0) + kPreListCap + 4 + 512 * 68) * sizeof(int);
-            static bool pre_attr[64] = {};
-            int dev = 0;
-            if (i_hi >= i_lo && n_bg <= 65535 && cudaGetDevice(&dev) == cudaSuccess && dev >= 0 && dev < 64) {
-                bool ok = pre_attr[dev];
-                if (!ok) {
-                    const size_t smem_max = ((size_t)kStageOut + kPreListCap + 4 + 512 * 68) * sizeof(int);
-                    ok = cudaFuncSetAttribute(k_topk_linear_pre<512, 64, VEC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem_max) == cudaSuccess;
-                    pre_attr[dev] = ok;
-                }
-                if (ok) {
-                    const int R = HS2_TOPK_PRE_ROWS;
-                    k_topk_linear_pre<512, 64, VEC><<<dim3((unsigned)((i_hi - i_lo + R) / R), (unsigned)n_bg), 512, smem, st>>>(
-                        p, scores, score_stride, idx, row0, lo, hi, n_rows, (int)i_lo, R);
-                    count_launch();
-                    return;
-                }
-            }
-        }
-#endif
         switch (c) {
             case 0: launched = go(k_topk_linear<64, 32, VEC>, 64, 32); break;
             case 1: launched = go(k_topk_linear<128, 32, VEC>, 128, 32); break;

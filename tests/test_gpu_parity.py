@@ -90,10 +90,10 @@ def test_topk_adversarial_rows(Lk):
         _topk_case(scores, k, w, q_start=[Lk - 1 - len(rows) + 1])
 
 
-def test_topk_longest_register_class_with_prefetched_rows():
-    """Positions known on the host and rows of 16385..32768 candidates: one CTA takes consecutive queries and fetches the
-    next row during the current one; rows whose threshold bin holds (nearly) the whole row push the list into the
-    prefetch buffer, so the row after them is read the plain way."""
+def test_topk_host_known_positions_adversarial_rows_in_the_longest_register_class():
+    """Positions known on the host (every class launch covers only its own queries) and rows of 16385..32768 candidates
+    that are staged through the shared list's memory: rows whose threshold bin holds (nearly) the whole row then fill
+    that list completely; ties, flat rows, denormals; staged and unstaged output rows."""
     Lk, Lq = 24000, 40
     g = torch.Generator().manual_seed(77)
     s = torch.randn(1, 2, Lq, Lk, generator=g) * 2.0 - 10.0
