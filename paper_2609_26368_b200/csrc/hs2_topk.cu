@@ -166,6 +166,22 @@ __device__ __forceinline__ int sample_rank(int take, int n, int n_s)
     return (int)(m + 5.f * sqrtf(m) + 2.f);
 }
 
+__device__ __forceinline__ void topk_cp_async16(void *dst, const void *src)
+{
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"((uint32_t)__cvta_generic_to_shared(dst)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void topk_cp_async_wait_all()
+{
+    asm volatile("cp.async.commit_group;\n cp.async.wait_group 0;\n" ::: "memory");
+}
+
+#ifndef HS2_TOPK_STAGE
+#define HS2_TOPK_STAGE 1      // rows reach the registers through a coalesced copy into shared memory
+#endif
+// dynamic shared memory of the two selects of the filtered path: [bitmap (candidate select only)][staged row]
+__host__ __device__ inline size_t cached_bitmap_bytes(int Lk) { return ((size_t)((Lk + 31) / 32) * 4 + 15) & ~(size_t)15; }
+constexpr size_t cached_stage_bytes(int threads, int e) { return (size_t)threads * (e + 4) * 4; }
+
 template <int THREADS, int E, bool VEC, int MODE>
 __global__ void __launch_bounds__(THREADS, THREADS > 256 ? 1 : (E > 32 ? 2 : 3))
 k_topk_cached(const Params p, const float *__restrict__ scores, int64_t score_stride, int32_t *__restrict__ idx,
@@ -221,6 +237,24 @@ k_topk_cached(const Params p, const float *__restrict__ scores, int64_t score_st
     const int j0 = tid * E;
     const bool has = j0 < nc;   // threads (whole warps, on short rows) past the row's end skip every per-candidate loop
     uint32_t key[E];
+    // The two selects of the filtered path bring the row in through shared memory: consecutive lanes copy consecutive
+    // 16-byte chunks (chunk c to slot c + c / CPT), every thread reads its own chunks at a pitch of CPT + 1 slots.
+    // A thread's own loads would sit E * 4 bytes apart between lanes, 32 cache lines per warp instruction.
+    constexpr int CPT = E / 4;
+    constexpr bool kStaged = HS2_TOPK_STAGE && VEC && MODE != SEL_ROW;
+    extern __shared__ __align__(16) unsigned char s_cached_dyn[];
+    float *s_stage = reinterpret_cast<float *>(s_cached_dyn + (MODE == SEL_CAND ? cached_bitmap_bytes(p.Lk) : 0));
+    auto stage_in = [&](const void *src_row) {   // whole chunks of the first nc 4-byte entries of a row
+        const float *src = static_cast<const float *>(src_row);
+#pragma unroll
+        for (int it = 0; it < CPT; ++it) {
+            const int c = it * THREADS + tid;
+            if (4 * c + 4 <= nc) topk_cp_async16(s_stage + (c + c / CPT) * 4, src + 4 * c);
+        }
+        topk_cp_async_wait_all();
+        __syncthreads();
+    };
+    if (kStaged) stage_in(srow);
     // which bits differ anywhere in the row: OR of (key ^ key of candidate 0), one logic op per candidate
     const uint32_t ref = order_key(__ldg(srow));
     unsigned diff = 0u;
@@ -228,7 +262,8 @@ k_topk_cached(const Params p, const float *__restrict__ scores, int64_t score_st
 #pragma unroll
     for (int e4 = 0; e4 < E; e4 += 4) {
         if (VEC && j0 + e4 + 4 <= nc) {
-            const float4 v = __ldg(reinterpret_cast<const float4 *>(srow + j0 + e4));
+            const float4 v = kStaged ? *reinterpret_cast<const float4 *>(s_stage + ((CPT + 1) * tid + (e4 >> 2)) * 4)
+                                     : __ldg(reinterpret_cast<const float4 *>(srow + j0 + e4));
             key[e4] = order_key(v.x); key[e4 + 1] = order_key(v.y); key[e4 + 2] = order_key(v.z); key[e4 + 3] = order_key(v.w);
 #pragma unroll
             for (int e = e4; e < e4 + 4; ++e) diff |= key[e] ^ ref;
@@ -333,7 +368,14 @@ k_topk_cached(const Params p, const float *__restrict__ scores, int64_t score_st
         // The candidates come in no particular order.  Kept: score above tau, or equal to tau and among the need_eq
         // lowest key indices of the equal ones.  The kept keys are marked in a bitmap over the row's keys, which is
         // then read out in ascending order.
-        extern __shared__ unsigned bitmap[];
+        unsigned *bitmap = reinterpret_cast<unsigned *>(s_cached_dyn);
+        // the key indices of the candidates come in the same way (every thread has its scores in registers by now)
+        __syncthreads();
+        if (kStaged) stage_in(prow);
+        auto pay = [&](int e) -> int32_t {
+            if (kStaged && j0 + (e & ~3) + 4 <= nc) return reinterpret_cast<const int32_t *>(s_stage)[((CPT + 1) * tid + (e >> 2)) * 4 + (e & 3)];
+            return prow[j0 + e];
+        };
         unsigned my_eq = 0;
 #pragma unroll
         for (int e = 0; e < E; ++e) my_eq += (j0 + e < nc) && key[e] == tau;
@@ -349,7 +391,7 @@ k_topk_cached(const Params p, const float *__restrict__ scores, int64_t score_st
             __syncthreads();
 #pragma unroll
             for (int e = 0; e < E; ++e)
-                if (j0 + e < nc && key[e] == tau) s_list[atomicAdd(&s_cnt, 1u)] = ~(uint32_t)prow[j0 + e];
+                if (j0 + e < nc && key[e] == tau) s_list[atomicAdd(&s_cnt, 1u)] = ~(uint32_t)pay(e);
             __syncthreads();
             jmin = select_on_list<THREADS>(s_list, total_eq, need_eq, hist, &s_prefix, &s_need, tid, lane, warp);
         }
@@ -360,7 +402,7 @@ k_topk_cached(const Params p, const float *__restrict__ scores, int64_t score_st
         for (int e = 0; e < E; ++e) {
             if (j0 + e >= nc) continue;
             if (key[e] > tau || key[e] == tau) {
-                const uint32_t j = (uint32_t)prow[j0 + e];
+                const uint32_t j = (uint32_t)pay(e);
                 // (the sweep only writes keys below n_keys; the range test keeps a damaged list from writing outside the bitmap)
                 if (j < (uint32_t)n_keys && (key[e] > tau || ~j >= jmin)) atomicOr(&bitmap[j >> 5], 1u << (j & 31u));
             }
@@ -475,22 +517,10 @@ __device__ __forceinline__ unsigned ge_exact(float v, float t)
 #ifndef HS2_TOPK_ROWS
 #define HS2_TOPK_ROWS 1    // rows per CTA of the linear kernel (consecutive queries of one (sequence, KV head))
 #endif
-#ifndef HS2_TOPK_STAGE
-#define HS2_TOPK_STAGE 1      // rows reach the registers through a coalesced copy into shared memory
-#endif
 #ifndef HS2_TOPK_WIDE
 #define HS2_TOPK_WIDE 1    // rows of 8193..16384 candidates: 32 per thread on 512 threads, two CTAs per SM (4 % faster than 64 per
                            // thread on 256; the same step for the longest class, 1024 threads, measured 5 % slower)
 #endif
-__device__ __forceinline__ void topk_cp_async16(void *dst, const void *src)
-{
-    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;\n" ::"r"((uint32_t)__cvta_generic_to_shared(dst)), "l"(src) : "memory");
-}
-__device__ __forceinline__ void topk_cp_async_wait_all()
-{
-    asm volatile("cp.async.commit_group;\n cp.async.wait_group 0;\n" ::: "memory");
-}
-
 // one row of k_topk_linear; every exit is taken by the whole CTA
 template <int THREADS, int E, bool VEC>
 __device__ __forceinline__ void topk_linear_row(const Params &p, const float *__restrict__ scores, int64_t score_stride,
@@ -1432,24 +1462,23 @@ cudaError_t launch_filter_thresholds(const Params &p, const float *sample, int64
     const int ns_max = filter_sample_width(p, samp);
     // class by the size of the row's sample (every row is taken by exactly one launch); as for whole rows, a sample
     // gets no more warps than it fills
-    k_topk_cached<64, 32, true, SEL_TAU><<<n, 64, 0, st>>>(p, sample, stride, nullptr, row0, -1, 2048, sa);
-    count_launch();
-    if (ns_max > 2048) {
-        k_topk_cached<128, 32, true, SEL_TAU><<<n, 128, 0, st>>>(p, sample, stride, nullptr, row0, 2048, 4096, sa);
+    // (dynamic shared memory: the staged sample row; above 48 KB it has to be asked for)
+    auto go = [&](auto kern, int threads, int e, int lo, int hi) -> cudaError_t {
+        const size_t smem = HS2_TOPK_STAGE ? cached_stage_bytes(threads, e) : 0;
+        if (smem > 48 * 1024) {
+            const cudaError_t e2 = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e2 != cudaSuccess) return e2;
+        }
+        kern<<<n, threads, smem, st>>>(p, sample, stride, nullptr, row0, lo, hi, sa);
         count_launch();
-    }
-    if (ns_max > 4096) {
-        k_topk_cached<256, 32, true, SEL_TAU><<<n, 256, 0, st>>>(p, sample, stride, nullptr, row0, 4096, 8192, sa);
-        count_launch();
-    }
-    if (ns_max > 8192) {
-        k_topk_cached<256, 64, true, SEL_TAU><<<n, 256, 0, st>>>(p, sample, stride, nullptr, row0, 8192, 16384, sa);
-        count_launch();
-    }
-    if (ns_max > 16384) {
-        k_topk_cached<512, 64, true, SEL_TAU><<<n, 512, 0, st>>>(p, sample, stride, nullptr, row0, 16384, 32768, sa);
-        count_launch();
-    }
+        return cudaSuccess;
+    };
+    cudaError_t e = go(k_topk_cached<64, 32, true, SEL_TAU>, 64, 32, -1, 2048);
+    if (e == cudaSuccess && ns_max > 2048) e = go(k_topk_cached<128, 32, true, SEL_TAU>, 128, 32, 2048, 4096);
+    if (e == cudaSuccess && ns_max > 4096) e = go(k_topk_cached<256, 32, true, SEL_TAU>, 256, 32, 4096, 8192);
+    if (e == cudaSuccess && ns_max > 8192) e = go(k_topk_cached<256, 64, true, SEL_TAU>, 256, 64, 8192, 16384);
+    if (e == cudaSuccess && ns_max > 16384) e = go(k_topk_cached<512, 64, true, SEL_TAU>, 512, 64, 16384, 32768);
+    if (e != cudaSuccess) return e;
     return cudaGetLastError();
 }
 
@@ -1460,12 +1489,19 @@ cudaError_t launch_filter_select(const Params &p, const float *cand_a, const int
     if (n_rows == 0) return cudaSuccess;
     SelArgs sa{1, cap, nullptr, flag, count, cand_j};
     const unsigned n = (unsigned)n_rows;
-    const size_t bm = (size_t)((p.Lk + 31) / 32) * 4;   // one bit per key of the row (at most 32 KB)
-    if (cap <= 8192)
-        k_topk_cached<256, 32, true, SEL_CAND><<<n, 256, bm, st>>>(p, cand_a, cap, idx, row0, -1, 0x7fffffff, sa);
-    else
-        k_topk_cached<512, 64, true, SEL_CAND><<<n, 512, bm, st>>>(p, cand_a, cap, idx, row0, -1, 0x7fffffff, sa);
-    count_launch();
+    const size_t bm = cached_bitmap_bytes(p.Lk);   // one bit per key of the row (at most 32 KB), then the staged row
+    auto go = [&](auto kern, int threads, int e) -> cudaError_t {
+        const size_t smem = bm + (HS2_TOPK_STAGE ? cached_stage_bytes(threads, e) : 0);
+        if (smem > 48 * 1024) {
+            const cudaError_t e2 = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+            if (e2 != cudaSuccess) return e2;
+        }
+        kern<<<n, threads, smem, st>>>(p, cand_a, cap, idx, row0, -1, 0x7fffffff, sa);
+        count_launch();
+        return cudaSuccess;
+    };
+    const cudaError_t e = cap <= 8192 ? go(k_topk_cached<256, 32, true, SEL_CAND>, 256, 32) : go(k_topk_cached<512, 64, true, SEL_CAND>, 512, 64);
+    if (e != cudaSuccess) return e;
     return cudaGetLastError();
 }
 
