@@ -810,10 +810,25 @@ k_topk_cluster(const Params p, const float *__restrict__ scores, int64_t score_s
     const int j0 = rank * SLICE + tid * E;
     uint32_t key[E];
     unsigned kmin = 0xffffffffu, kmax = 0u;
+    // the slice comes in through shared memory, as in the register kernels: coalesced 16-byte copies, chunk c of the
+    // slice to slot c + c / 16, each thread reading its own 16 chunks at a pitch of 17 slots
+    extern __shared__ __align__(16) float s_cl_stage[];
+    constexpr bool kStaged = HS2_TOPK_STAGE && VEC;
+    if (kStaged) {
+#pragma unroll
+        for (int it = 0; it < E / 4; ++it) {
+            const int c = it * THREADS + tid;
+            const int jg = (int)rank * SLICE + 4 * c;
+            if (jg + 4 <= nc) topk_cp_async16(s_cl_stage + (c + c / (E / 4)) * 4, srow + jg);
+        }
+        topk_cp_async_wait_all();
+        __syncthreads();
+    }
 #pragma unroll
     for (int e4 = 0; e4 < E; e4 += 4) {
         if (VEC && j0 + e4 + 4 <= nc) {
-            const float4 v = __ldg(reinterpret_cast<const float4 *>(srow + j0 + e4));
+            const float4 v = kStaged ? *reinterpret_cast<const float4 *>(s_cl_stage + ((E / 4 + 1) * tid + (e4 >> 2)) * 4)
+                                     : __ldg(reinterpret_cast<const float4 *>(srow + j0 + e4));
             key[e4] = order_key(v.x); key[e4 + 1] = order_key(v.y); key[e4 + 2] = order_key(v.z); key[e4 + 3] = order_key(v.w);
         } else {
 #pragma unroll
@@ -1198,9 +1213,17 @@ void launch_class(int c, const Params &p, const float *scores, int64_t score_str
         case 2: k_topk_cached<256, 32, VEC, SEL_ROW><<<n, 256, stage, st>>>(p, scores, score_stride, idx, row0, lo, hi, SelArgs{}); break;
         case 3: k_topk_cached<256, 64, VEC, SEL_ROW><<<n, 256, stage, st>>>(p, scores, score_stride, idx, row0, lo, hi, SelArgs{}); break;
         case 4: k_topk_cached<512, 64, VEC, SEL_ROW><<<n, 512, stage, st>>>(p, scores, score_stride, idx, row0, lo, hi, SelArgs{}); break;
-        case 5: k_topk_cluster<2, VEC><<<n * 2, 512, 0, st>>>(p, scores, score_stride, idx, row0, lo, hi); break;
-        case 6: k_topk_cluster<4, VEC><<<n * 4, 512, 0, st>>>(p, scores, score_stride, idx, row0, lo, hi); break;
-        case 7: k_topk_cluster<8, VEC><<<n * 8, 512, 0, st>>>(p, scores, score_stride, idx, row0, lo, hi); break;
+        case 5: case 6: case 7: {   // (dynamic shared memory: the staged slice of the row)
+            const size_t smem = (HS2_TOPK_STAGE && VEC) ? cached_stage_bytes(512, 64) : 0;
+            auto go = [&](auto kern, unsigned cl) {
+                if (smem > 48 * 1024 && cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return;
+                kern<<<n * cl, 512, smem, st>>>(p, scores, score_stride, idx, row0, lo, hi);
+            };
+            if (c == 5) go(k_topk_cluster<2, VEC>, 2u);
+            else if (c == 6) go(k_topk_cluster<4, VEC>, 4u);
+            else go(k_topk_cluster<8, VEC>, 8u);
+            break;
+        }
         default: k_topk<1024, kItems, false, VEC><<<n, 1024, 0, st>>>(p, scores, score_stride, idx, row0, lo, hi); break;
     }
     count_launch();
