@@ -29,9 +29,12 @@
  *   - Query i of sequence b sits at absolute position pos = q_start[b] + i and sees keys
  *     0 .. min(pos, kv_lens[b]-1).  The forced window is [pos-w+1, pos] (the token itself counts);
  *     selection candidates are keys 0 .. pos-w.
- *   - The library allocates no memory, keeps no state between calls, enqueues its work on the
- *     given CUDA stream and returns without synchronising.  Scratch comes from the caller
- *     (`ws`, at least hs2_workspace_bytes() bytes, 256-byte aligned).
+ *   - The library allocates no memory, enqueues its work on the given CUDA stream and returns
+ *     without synchronising.  Scratch comes from the caller (`ws`, at least hs2_workspace_bytes()
+ *     bytes, 256-byte aligned).  No result of one call depends on an earlier call; what the process
+ *     does keep is listed at the end of this file: two dispatch knobs (hs2_set_tcgen05_enabled,
+ *     hs2_set_filter_min_keys), per-device caches of device attributes, a sticky device error word,
+ *     a launch counter, and the built-in scratch array of hs2_sparse_attn_decode_static.
  *   - Argument errors are found on the host before anything is launched and reported through the
  *     status; nothing throws, aborts or traps.  There is no CPU fallback: without a CUDA device
  *     every compute entry point returns HS2_ERR_CUDA.
@@ -90,8 +93,8 @@ typedef struct {
 size_t hs2_workspace_bytes(const hs2_problem *p, hs2_op op);
 
 /*
- * FA layer of a hybrid block (Section 3.4: the full-attention layers "serve as indexers, using
- * exact attention scores"; Section 3.3: top-k over individual tokens, outside the forced window).
+ * FA layer of a hybrid block (Section 3.4: the full-attention layers are the indexers, their own exact
+ * attention scores rank the tokens; Section 3.3: top-k over individual tokens, outside the forced window).
  *
  *   O    out  attention output, same layout/dtype as Q
  *   LSE  out  log-sum-exp of the scaled logits per (batch, head, query), natural log; required
@@ -126,8 +129,8 @@ hs2_status hs2_topk_select(const hs2_problem *p, const float *scores, int32_t *i
                            void *ws, size_t ws_bytes, void *cuda_stream);
 
 /*
- * SA layer, prefill (Section 3.3: the window "is always selected, followed by the highest-scoring
- * tokens outside the window. Both selected sets are read from the full-attention KV cache").
+ * SA layer, prefill (Section 3.3: the recent window is always part of the attended set, the k best-scoring
+ * tokens outside it come from the FA layer's selection, and K/V of both are read from the FA layer's cache).
  *   Q     in  this SA layer's own queries; K, V: the FA layer's cache; idx: the FA layer's indices.
  *   An idx entry is ignored when it is negative, greater than pos-w (inside the window or in the
  *   future) or >= kv_lens[b]; the attended set is the union with the window and no entry can cause
@@ -151,8 +154,8 @@ hs2_status hs2_sparse_attn_decode(const hs2_problem *p, const void *Q, const voi
                                   void *ws, size_t ws_bytes, void *cuda_stream);
 
 /*
- * The two SA calls with the sigmoid output gate of the sparse layers fused into the store (Section 4.1:
- * "all sparse and SWA layers use sigmoid output gates"): O = sigmoid(gate) * attention output, elementwise.
+ * The two SA calls with the sigmoid output gate of the sparse layers fused into the store (Section 4.1 gives the
+ * sparse and the sliding-window layers such gates): O = sigmoid(gate) * attention output, elementwise.
  *   gate  in  the gate logits (the caller's projection of the layer input; not computed here): shape, dtype
  *             and strides of O (p->o_stride).  Must not be NULL (use the ungated call instead).
  * LSE is not affected by the gate.  Everything else as for the ungated calls.
@@ -165,8 +168,8 @@ hs2_status hs2_sparse_attn_decode_gated(const hs2_problem *p, const void *Q, con
                                         float *LSE, void *ws, size_t ws_bytes, void *cuda_stream);
 
 /*
- * The two SA calls on an FP8 KV cache (the storage format the paper's cost analysis of Section 4 assumes, "FP8
- * KV-cache storage"; the paper gives no quantisation recipe, this is the usual one):
+ * The two SA calls on an FP8 KV cache (the storage format the paper's cost analysis of Section 4 assumes; the
+ * paper gives no quantisation recipe, this is the usual one):
  *   K8, V8   in  e4m3 codes (1 byte: sign, 4 exponent bits with bias 7, 3 mantissa bits; no infinities, the two
  *                NaN codes are a caller error) [batch, kv_len, n_kv_heads, head_dim]; p->kv_stride counts codes
  *                (= bytes), multiples of 16, or 0 for packed.
@@ -213,10 +216,12 @@ hs2_status hs2_full_attn_select_fp8kv(const hs2_problem *p, const void *Q, const
  *
  *   - Same arguments and results as hs2_sparse_attn_decode, minus `ws`.  The call allocates nothing
  *     and frees nothing, on the host or on the device.
- *   - Limit: batch * n_kv_heads <= HS2_STATIC_DECODE_MAX_PAIRS (64); a larger problem returns
- *     HS2_ERR_STATIC_SCRATCH and launches nothing.  It covers what the tensor-core decode kernel
- *     covers (bf16, head_dim 128, group <= 8, 16-byte aligned tensors); anything else returns
- *     HS2_ERR_UNSUPPORTED.
+ *   - Limit: at most HS2_STATIC_DECODE_MAX_PAIRS (64) units of work, a unit being one (sequence,
+ *     KV head) with up to 8 query heads: batch * n_kv_heads <= 64 for groups of up to 8 heads; a
+ *     group of 16 heads runs as two units, so batch * n_kv_heads <= 32 there.  A larger problem
+ *     returns HS2_ERR_STATIC_SCRATCH and launches nothing.  It covers what the tensor-core decode
+ *     kernel covers (bf16, head_dim 128, groups of up to 8 or of 16 heads, 16-byte aligned tensors);
+ *     anything else returns HS2_ERR_UNSUPPORTED.
  *   - The first call on each device looks up the array's device address; make that first call
  *     outside any stream capture.
  *   - All calls on a device share the one array, which still holds the previous call's data: the
@@ -251,9 +256,15 @@ const char *hs2_status_string(hs2_status s);
 /* The cudaError_t (as int) behind the calling thread's most recent HS2_ERR_CUDA, 0 if none. */
 int hs2_last_cuda_error(void);
 
-/* Reads the library's device error word into *flags (0 = fine; bit 0: a bounded wait inside a kernel
- * ran out and that kernel abandoned its work; bit 1: a kernel refused a misaligned shared-memory
- * window).  Sticky until the process exits.  Synchronises the current device.  Returns an hs2_status. */
+/* Reads the library's device error word into *flags (0 = fine).  One byte per kernel family:
+ *   bits  0-7   full-attention and score-sweep kernels (tcgen05)
+ *   bits  8-15  sparse-attention kernels on mma.sync (bf16 and FP8 cache)
+ *   bits 16-23  sparse-attention kernel on tcgen05
+ *   bits 24-31  KV projection
+ * Within a byte, bit 0: a bounded wait inside a kernel ran out and that kernel abandoned its work (its
+ * output is then incomplete); bit 1: a kernel refused a misaligned shared-memory window.  Test
+ * `flags != 0`, not single bits.  Sticky until the process exits.  Synchronises the current device.
+ * Returns an hs2_status. */
 int hs2_device_error_flags(unsigned *flags);
 
 /* Testing knob: enabled = 0 makes hs2_full_attn_select use its mma.sync kernels (the path taken when TMA
@@ -262,8 +273,11 @@ int hs2_device_error_flags(unsigned *flags);
 int hs2_set_tcgen05_enabled(int enabled);
 
 /* Tuning knob of hs2_full_attn_select: from which kv_len on the selection thresholds a sample of the scores
- * and works on filtered candidate lists instead of complete score strips (default 65537; both ways give the
- * same indices).  Returns the previous value; min_keys <= 0 only queries.  Process-wide. */
+ * and works on filtered candidate lists instead of complete score strips.  Both ways select from the same
+ * tensor-core scores and give the same indices, with one exception: a row whose filtered list came out unusable
+ * is redone from scores recomputed with fp32 FMAs, which can order two keys differently when their scores agree
+ * to within rounding (inside the 1e-3 near-tie band).  Returns the previous value; min_keys <= 0 only queries.
+ * Process-wide, read at the start of each call: set it before calls start on other threads. */
 int hs2_set_filter_min_keys(int min_keys);
 
 /* Number of kernels this library has launched in the process so far (all threads, all streams). */

@@ -354,7 +354,8 @@ def hs2_sparse_attn_decode_static(prob: Problem, q, k, v, idx, *, sink=None, out
     """Decode for callers that may not allocate: the split kernel's partials live in a fixed
     8.5 MB array inside the library, so no workspace is passed and nothing is allocated - here
     included, which is why ``out`` (and ``lse``, if wanted) must be given.  Limit:
-    ``batch * n_kv_heads <= 64``.  Calls on one device share that array: keep them ordered on the GPU.
+    ``batch * n_kv_heads <= 64`` for groups of up to 8 query heads per KV head, ``<= 32`` for groups of 16 (which
+    run as two sub-groups of 8).  Calls on one device share that array: keep them ordered on the GPU.
     """
     _check_inputs(prob, q, k, v)
     assert out is not None and out.is_cuda and out.shape == q.shape and out.dtype == q.dtype

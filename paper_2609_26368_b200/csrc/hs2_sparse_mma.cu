@@ -18,6 +18,7 @@
 //   * online softmax in the base-2 domain with warp shuffles across the 8 key rows of a fragment.
 // Decode splits the attended set of one (sequence, KV head) over several warps; each writes an
 // un-normalised partial (m, l, O) and the last one to arrive (an atomic ticket, nobody waits) merges.
+#include <atomic>
 #include <mutex>
 
 #include "hs2_common.cuh"
@@ -684,18 +685,22 @@ size_t ws_tickets_bytes(const Params &p) { return ((size_t)p.B * p.Hkv * sizeof(
 
 constexpr int kDecodeCtaSmem = DecodeCfg::WARPS * DecodeCfg::kWarpSmem + DecodeCfg::WARPS * 16 * 4 + 8 * (HD + 8) * 2;
 
-int g_sm_count = 0;
+// SM count per device ordinal (0 = not asked yet); relaxed atomics: concurrent first calls write the same value
+std::atomic<int> g_sm_count[64];
 cudaError_t sm_count(int *n)
 {
-    if (g_sm_count == 0) {
-        int dev = 0, v = 0;
-        cudaError_t e = cudaGetDevice(&dev);
-        if (e != cudaSuccess) return e;
-        e = cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev);
-        if (e != cudaSuccess) return e;
-        g_sm_count = v;
+    int dev = 0, v = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    const bool cached = dev >= 0 && dev < 64;
+    if (cached && (v = g_sm_count[dev].load(std::memory_order_relaxed)) > 0) {
+        *n = v;
+        return cudaSuccess;
     }
-    *n = g_sm_count;
+    e = cudaDeviceGetAttribute(&v, cudaDevAttrMultiProcessorCount, dev);
+    if (e != cudaSuccess) return e;
+    if (cached) g_sm_count[dev].store(v, std::memory_order_relaxed);
+    *n = v;
     return cudaSuccess;
 }
 

@@ -1147,8 +1147,8 @@ constexpr TopkClass kClasses[kNumClasses] = {{-1, 2048},      {2048, 4096},     
                                              {262144, 0x7fffffff}};
 
 template <bool VEC>
-void launch_class(int c, const Params &p, const float *scores, int64_t score_stride, int32_t *idx, int64_t row0,
-                  int64_t n_rows, cudaStream_t st)
+cudaError_t launch_class(int c, const Params &p, const float *scores, int64_t score_stride, int32_t *idx, int64_t row0,
+                         int64_t n_rows, cudaStream_t st)
 {
     const int lo = kClasses[c].lo, hi = kClasses[c].hi;
     const unsigned n = (unsigned)n_rows;
@@ -1160,16 +1160,17 @@ void launch_class(int c, const Params &p, const float *scores, int64_t score_str
     // warps than its candidates fill: 32 (or 64) candidates per thread.
 #if HS2_TOPK_LINEAR
     if (c <= 4) {   // register-resident rows: first round on a linear scale, the threshold bin's members in a shared list
-        auto go = [&](auto kern, int threads, int e) -> bool {   // false: nothing was launched
+        cudaError_t err = cudaSuccess;
+        auto go = [&](auto kern, int threads, int e) -> bool {   // false: nothing was launched (err says whether that is a failure)
             // (+ one 16-byte slot per thread and the alignment of the staged row, which passes through the list's memory)
             const size_t smem = stage + (size_t)threads * e * sizeof(uint32_t) + (size_t)threads * 16 + 16;
             if (smem > 32 * 1024) {   // static shared memory counts against the 48 KB default too
                 static bool attr_set[5][64] = {};   // per row class: the kernels share one function type, hence one lambda body
                 int dev = 0;
-                if (cudaGetDevice(&dev) != cudaSuccess) return false;
+                if ((err = cudaGetDevice(&dev)) != cudaSuccess) return false;
                 if (!(dev >= 0 && dev < 64 && attr_set[c][dev])) {
-                    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             (int)(kStageOut * sizeof(int) + (size_t)threads * e * sizeof(uint32_t) + (size_t)threads * 16 + 16)) != cudaSuccess)
+                    if ((err = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                                    (int)(kStageOut * sizeof(int) + (size_t)threads * e * sizeof(uint32_t) + (size_t)threads * 16 + 16))) != cudaSuccess)
                         return false;
                     if (dev >= 0 && dev < 64) attr_set[c][dev] = true;
                 }
@@ -1204,7 +1205,7 @@ void launch_class(int c, const Params &p, const float *scores, int64_t score_str
             default: launched = go(k_topk_linear<512, 64, VEC>, 512, 64); break;
         }
         if (launched) count_launch();
-        return;
+        return err;
     }
 #endif
     switch (c) {
@@ -1215,18 +1216,28 @@ void launch_class(int c, const Params &p, const float *scores, int64_t score_str
         case 4: k_topk_cached<512, 64, VEC, SEL_ROW><<<n, 512, stage, st>>>(p, scores, score_stride, idx, row0, lo, hi, SelArgs{}); break;
         case 5: case 6: case 7: {   // (dynamic shared memory: the staged slice of the row)
             const size_t smem = (HS2_TOPK_STAGE && VEC) ? cached_stage_bytes(512, 64) : 0;
-            auto go = [&](auto kern, unsigned cl) {
-                if (smem > 48 * 1024 && cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem) != cudaSuccess) return;
+            auto go = [&](auto kern, unsigned cl) -> cudaError_t {
+                if (smem > 48 * 1024) {
+                    static bool attr_set[3][64] = {};   // per cluster size and device ordinal
+                    int dev = 0;
+                    cudaError_t e = cudaGetDevice(&dev);
+                    if (e != cudaSuccess) return e;
+                    if (!(dev >= 0 && dev < 64 && attr_set[c - 5][dev])) {
+                        if ((e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem)) != cudaSuccess) return e;
+                        if (dev >= 0 && dev < 64) attr_set[c - 5][dev] = true;
+                    }
+                }
                 kern<<<n * cl, 512, smem, st>>>(p, scores, score_stride, idx, row0, lo, hi);
+                return cudaSuccess;
             };
-            if (c == 5) go(k_topk_cluster<2, VEC>, 2u);
-            else if (c == 6) go(k_topk_cluster<4, VEC>, 4u);
-            else go(k_topk_cluster<8, VEC>, 8u);
+            const cudaError_t e = c == 5 ? go(k_topk_cluster<2, VEC>, 2u) : c == 6 ? go(k_topk_cluster<4, VEC>, 4u) : go(k_topk_cluster<8, VEC>, 8u);
+            if (e != cudaSuccess) return e;   // nothing was launched: the rows of this class would stay unwritten
             break;
         }
         default: k_topk<1024, kItems, false, VEC><<<n, 1024, 0, st>>>(p, scores, score_stride, idx, row0, lo, hi); break;
     }
     count_launch();
+    return cudaSuccess;
 }
 
 cudaError_t launch_topk(const Params &p, const float *scores, int64_t score_stride, int32_t *idx, int64_t row0,
@@ -1248,8 +1259,9 @@ cudaError_t launch_topk(const Params &p, const float *scores, int64_t score_stri
     }
     for (int c = 0; c < kNumClasses; ++c) {
         if (nc_max <= kClasses[c].lo || nc_min > kClasses[c].hi) continue;   // no row of the block falls in this class
-        if (vec) launch_class<true>(c, p, scores, score_stride, idx, row0, n_rows, st);
-        else launch_class<false>(c, p, scores, score_stride, idx, row0, n_rows, st);
+        const cudaError_t e = vec ? launch_class<true>(c, p, scores, score_stride, idx, row0, n_rows, st)
+                                  : launch_class<false>(c, p, scores, score_stride, idx, row0, n_rows, st);
+        if (e != cudaSuccess) return e;
     }
     return cudaGetLastError();
 }

@@ -150,3 +150,20 @@ class BlockRun:
         if lse is not None:
             l = gather_rows(lse, rows, "bhi").cpu().numpy().astype(np.float64)
             assert np.abs(l - LSEo).max() <= TOL[dt]["lse"], "sparse LSE max-abs %.3e" % np.abs(l - LSEo).max()
+
+    def check_decode(self, out1, lse1, layer=0, sink=None, gate=None):
+        """A decode call on the last query of every sequence against the oracle itself (not against the GPU's prefill
+        row): sparse attention of row q_len-1 on the GPU's own indices, max-abs and mean-abs.  `out1` [B,1,Hq,D],
+        `lse1` [B,Hq,1] or None, `gate` the prefill-shaped gate tensor or None."""
+        wl = self.wl
+        rows = [(b, wl.q_len - 1) for b in range(wl.batch)]
+        idx_rows = gather_rows(self.idx, rows, "bgik").cpu().numpy()
+        Oo, LSEo, _ = oracle.sparse_attn(to_host(self.qs[layer]), to_host(self.k), to_host(self.v), idx_rows,
+                                         wl.window, rows=rows,
+                                         sink=None if sink is None else sink.cpu().numpy().astype(np.float64),
+                                         gate=None if gate is None else to_host(gate))
+        dt = wl.torch_dtype
+        assert_output_close(out1[:, 0], Oo, dt, "sparse decode O")
+        if lse1 is not None:
+            l = lse1[:, :, 0].cpu().numpy().astype(np.float64)
+            assert np.abs(l - LSEo).max() <= TOL[dt]["lse"], "decode LSE max-abs %.3e" % np.abs(l - LSEo).max()

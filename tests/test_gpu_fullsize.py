@@ -49,11 +49,11 @@ def test_cfg2_full_size_sampled():
 
 
 def test_cfg3_full_size_sampled():
-    _run_block("cfg3", 48)
+    _run_block("cfg3", 64)
 
 
 def test_cfg4_full_size_sampled():
-    _run_block("cfg4", 32, layers=[0, 2])
+    _run_block("cfg4", 64)
 
 
 def test_cfg5_decode_full_size_every_sequence():

@@ -339,6 +339,47 @@ def test_decode_equals_last_row_of_prefill():
     np.testing.assert_allclose(Osd, Osp, atol=0)
 
 
+def test_sparse_attention_with_causal_offsets_and_ragged_cache_lengths():
+    """`q_start` / `kv_lens`: the sparse row is the library attention under an explicit mask built from
+    the definition - key j is attended iff j < kv_lens[b] and (j in the forced window [pos-w+1, pos] or j a listed
+    index <= pos - w), pos = q_start[b] + i.  The second sequence's cache length cuts its windows (and, for its last
+    queries, removes the query's own token), the third has queries whose window is cut to nothing but one key."""
+    B, Lq, Lk, Hq, Hkv, D, w, k = 3, 7, 48, 4, 2, 16, 6, 5
+    q, kk, v = _rand((B, Lq, Hq, D), 31), _rand((B, Lk, Hkv, D), 32), _rand((B, Lk, Hkv, D), 33)
+    q_start, kv_lens = [41, 20, 9], [48, 23, 11]      # seq 1: pos 20..26 vs 23 keys; seq 2: pos 9..15 vs 11 keys
+    rng = np.random.default_rng(5)
+    rows = [(b, i) for b in range(B) for i in range(Lq)]
+    # listed indices: random keys of the whole tensor extent, so some are in the window, in the future or past the
+    # ragged end (all of which the definition drops); no duplicates inside a row
+    idx = np.stack([np.stack([np.sort(rng.choice(Lk, size=k, replace=False)) for _ in range(Hkv)]) for _ in rows])
+    idx = idx.astype(np.int32)
+    idx[3, 0, 1] = -1
+    O, LSE, mem = oracle.sparse_attn(q, kk, v, idx, w, rows=rows, scale=0.37, q_start=q_start, kv_lens=kv_lens,
+                                     want_member=True)
+    G = Hq // Hkv
+    cut_window = cut_self = 0
+    for r, (b, i) in enumerate(rows):
+        pos = q_start[b] + i
+        for g in range(Hkv):
+            mask = torch.zeros(Lk, dtype=torch.bool)
+            for j in range(Lk):
+                listed = j in idx[r, g].tolist() and j <= pos - w
+                in_window = pos - w + 1 <= j <= pos
+                mask[j] = (listed or in_window) and j < kv_lens[b]
+            assert np.array_equal(mem[r, g].astype(bool), mask.numpy())
+            assert mask.any()
+            cut_window += int(pos - w + 1 < kv_lens[b] <= pos)
+            cut_self += int(kv_lens[b] <= pos)
+            hs = slice(g * G, (g + 1) * G)
+            ref = _sdpa(q[b:b + 1, i:i + 1, hs], kk[b:b + 1, :, g:g + 1], v[b:b + 1, :, g:g + 1], mask[None, :],
+                        scale=0.37)
+            np.testing.assert_allclose(O[r, hs], ref[0, 0], rtol=0, atol=1e-12)
+            logits = 0.37 * torch.einsum("hd,jd->hj", q[b, i, hs].double(), kk[b, :, g].double())
+            lse = torch.logsumexp(logits.masked_fill(~mask[None, :], float("-inf")), dim=-1).numpy()
+            np.testing.assert_allclose(LSE[r, hs], lse, rtol=0, atol=1e-12)
+    assert cut_window >= 8 and cut_self >= 8          # the ragged end really cuts windows in this case
+
+
 def test_fp32_and_bf16_inputs_are_read_exactly():
     """bf16 bit patterns are widened exactly: the same values given as fp32 produce the same result."""
     wl, inp = _inputs_small()
