@@ -2,19 +2,26 @@
 """Benchmark of the hybrid sparse-attention hot path on B200.
 
 One *step* is one pass of the whole path over one batch of synthetic input of the chosen
-workload (default: the L=8192 prefill configuration, "cfg2"):
+workload (default: the largest single-GPU prefill configuration, "cfg4": L=131072, one full layer and
+three sparse layers; the two smaller prefill configurations are timed briefly as side sections):
 
     hs2_full_attn_select          full-attention layer + token-level top-k indices
     hs2_sparse_attn_prefill  x n  the sparse layers that reuse the cache and the indices
     hs2_full_attn_select (Lq=1) + hs2_sparse_attn_decode   one decode step on the same cache
 
 The JSON line's `value` is tokens/s of that step with inputs resident in HBM; `roofline` describes
-the sparse-prefill kernel (gathered K/V bytes per launch over its CUDA-event duration, against the
-measured HBM peak); `decode_64k` times the split-KV decode kernel on the 64K-context configuration;
+the sparse-prefill kernel: gathered K/V bytes per launch over its CUDA-event duration against the
+measured HBM peak (`frac`, which exceeds 1 when a KV head's cache is L2 resident) and against a gather
+ceiling measured in the same run (`frac_l2`: the same rows fetched by a kernel that does nothing else);
+`decode_64k` times the split-KV decode kernel on the 64K-context configuration;
 `e2e` repeats the step with pinned host inputs/outputs copied inside the timed region;
 `cpu_baseline` is the CPU oracle on a bounded sample of the same workload.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload cfg2]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--workload cfg4]
+
+`--gpus N` with N > 1 started as a plain process re-executes itself under torch.distributed.run with
+one rank per GPU (independent replicas of the workload; NCCL only for the barrier and the reduction
+of the timings).
 """
 from __future__ import annotations
 
@@ -35,9 +42,11 @@ import torch  # noqa: E402
 
 from gen import CONFIGS, make_inputs, sample_rows  # noqa: E402
 
-# dram__bytes_read.sum + dram__bytes_write.sum of one k_sparse_prefill launch, from the ncu capture
-# summarised in profiles/block_step_cfg2.md (bytes)
-NCU_DRAM_TRAFFIC = {"cfg2": 268.1e6}
+# dram__bytes_read.sum + dram__bytes_write.sum of one k_sparse_prefill launch (bytes): RECORDED from ncu captures,
+# not measured by this program.  Each entry names the summary under profiles/ that holds the capture's command.
+NCU_DRAM_TRAFFIC = {
+    "cfg2": (268.1e6, "profiles/block_step_cfg2.md"),
+}
 
 METRIC = "sparse-attn prefill tokens/s (hybrid block step: full-attn+select, sparse layers, decode step)"
 
@@ -74,6 +83,24 @@ def full_attn_flops(wl) -> float:
     q0 = wl.kv_len - wl.q_len
     pairs = sum(min(q0 + i + 1, wl.kv_len) for i in range(wl.q_len))
     return 4.0 * wl.head_dim * wl.batch * wl.n_q_heads * pairs
+
+
+def sparse_attn_flops(wl) -> float:
+    """4 * D flops per (query head, attended key) pair of one sparse layer."""
+    return 4.0 * wl.head_dim * attended_tokens(wl) * wl.batch * wl.n_q_heads
+
+
+def oracle_row_flops(wl) -> float:
+    """Average multiply-adds x 2 of one oracle query row (all heads): full attention + the sparse layers."""
+    return full_attn_flops(wl) / (wl.batch * wl.q_len) + wl.n_sparse_layers * sparse_attn_flops(wl) / (wl.batch * wl.q_len)
+
+
+def tensor_peak_for(ms: float, peaks):
+    """Which measured bf16 peak a tensor-core kernel of this duration is held against: the burst figure for a kernel
+    of a few milliseconds (it finishes before the power cap bites), the sustained one for longer kernels."""
+    if ms < 5.0:
+        return peaks["bf16_tflops"], "burst"
+    return peaks["bf16_tflops_sustained"], "sustained"
 
 
 # ------------------------------------------------------------------ clocks
@@ -187,6 +214,26 @@ class Block:
                 self._timed("sparse_attn_decode", lambda: hs2.hs2_sparse_attn_decode(
                     self.prob1, q, self.k, self.v, self.idx1, out=self.O1_sparse[l], ws=self.ws_dec), timing)
 
+    def gather_ceiling_ms(self, reps=3):
+        """Duration of the bare row gather of one sparse layer (hs2_probe_gather: the same rows in the same order,
+        nothing else), best of the two load modes, median of `reps` after one warm-up each.  Needs self.idx."""
+        best = None
+        word = torch.zeros(1, dtype=torch.int32, device=self.dev)
+        for mode in (0, 1):
+            self.hs2.hs2_probe_gather(self.prob, self.k, self.v, self.idx, mode=mode, sink_word=word)
+            ts = []
+            for _ in range(reps):
+                a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                a.record()
+                self.hs2.hs2_probe_gather(self.prob, self.k, self.v, self.idx, mode=mode, sink_word=word)
+                b.record()
+                torch.cuda.synchronize()
+                ts.append(a.elapsed_time(b))
+            t = statistics.median(ts)
+            if best is None or t < best[0]:
+                best = (t, mode)
+        return best
+
     def kernel_means(self):
         return {k: sum(a.elapsed_time(b) for a, b in v) / len(v) for k, v in self.kernel_ms.items()}
 
@@ -196,6 +243,19 @@ class Block:
 
     def output_tensors(self):
         return [self.O_full] + self.O_sparse
+
+
+def respawn_under_torchrun(n_gpus):
+    """`bench.py --gpus N` started as a plain process: run the same command line as N ranks, one per GPU."""
+    import socket
+    s = socket.socket()
+    s.bind(("127.0.0.1", 0))
+    port = s.getsockname()[1]
+    s.close()
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", "--nproc-per-node", str(n_gpus),
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    sys.stdout.flush()
+    os.execv(sys.executable, cmd)
 
 
 def dist_setup(n_gpus):
@@ -441,7 +501,8 @@ def bench_native(device, peaks, reps=5):
         "workload": "native8k: B=1, L=8192, 64q/1kv heads, D=256, bf16, k=1024, w=128",
         "full_attn_select_ms": round(t_full, 3), "attention_only_ms": round(t_att, 3),
         "attention_tflops": round(fl / (t_att * 1e-3) / 1e12, 1),
-        "attention_frac_of_bf16_peak": round(fl / (t_att * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"], 4),
+        "attention_frac_of_bf16_peak": round(fl / (t_att * 1e-3) / 1e12 / tensor_peak_for(t_att, peaks)[0], 4),
+        "attention_peak_kind": tensor_peak_for(t_att, peaks)[1],
         "sparse_prefill_ms": round(t_sp, 3), "gathered_kv_bytes": gb,
         "sparse_prefill_gbs": round(gb / (t_sp * 1e-3) / 1e9, 1),
         "sparse_prefill_frac_of_hbm_peak": round(gb / (t_sp * 1e-3) / 1e9 / peaks["hbm_gbs"], 4),
@@ -528,17 +589,35 @@ def oracle_sample_step(wl, inp_host, rows):
         oracle.sparse_attn(q, inp_host.k, inp_host.v, idx, wl.window, rows=rows)
 
 
+def host_inputs(wl):
+    """The workload's tensors in host memory (drawn on the GPU when there is one: the generator is counter based, and
+    the large configurations take minutes to draw on the host cores)."""
+    if torch.cuda.is_available():
+        from dataclasses import replace as _r
+        inp = make_inputs(wl, "cuda")
+        out = _r(inp, q_full=inp.q_full.cpu(), k=inp.k.cpu(), v=inp.v.cpu(), q_sparse=[q.cpu() for q in inp.q_sparse])
+        del inp
+        torch.cuda.empty_cache()
+        return out
+    return make_inputs(wl, "cpu")
+
+
+def rows_for_flops(wl, flops):
+    n = int(flops / oracle_row_flops(wl))
+    return max(8, min(n, wl.q_len))
+
+
 def cpu_baseline(wl, n_rows):
     import oracle
     oracle.build()
-    inp = make_inputs(wl, "cpu")
-    rows = [(b, i) for b in range(wl.batch) for i in sample_rows(wl, n_rows)]
+    inp = host_inputs(wl)
+    rows = [(b, i) for b in range(wl.batch) for i in sample_rows(wl, max(1, n_rows // wl.batch))]
     t0 = time.time()
     oracle_sample_step(wl, inp, rows)
     dt = time.time() - t0
     return {"value": round(len(rows) / dt, 3), "unit": "tokens/s", "cores": oracle.num_threads(), "kind": "oracle",
             "sample": "%d query rows of %s (budget edges + seeded uniform), all heads, full-attn+select+%d sparse "
-                      "layer(s), %.1f s" % (len(rows), wl.name, len(inp.q_sparse), dt)}, inp, rows
+                      "layer(s), %.1f s" % (len(rows), wl.name, len(inp.q_sparse), dt)}
 
 
 def run_reference(args, wl):
@@ -548,9 +627,11 @@ def run_reference(args, wl):
         return
     import oracle
     oracle.build()
-    inp = make_inputs(wl, "cpu")
-    # a bounded sample per step, so that K steps end within a few minutes on the machine's host cores
-    rows = [(b, i) for b in range(wl.batch) for i in sample_rows(wl, min(args.cpu_rows, 1024))]
+    inp = host_inputs(wl)
+    # a bounded sample per step (about 5e10 flops, two to three seconds on 16 cores), so that K steps end within a
+    # few minutes on the machine's host cores
+    n = args.cpu_rows if args.cpu_rows > 0 else rows_for_flops(wl, 5e10)
+    rows = [(b, i) for b in range(wl.batch) for i in sample_rows(wl, max(1, min(n, 1024) // wl.batch))]
     for _ in range(min(args.warmup, 1)):
         oracle_sample_step(wl, inp, rows[:8])
     t0 = time.time()
@@ -571,11 +652,74 @@ def run_reference(args, wl):
 
 
 def workload_config(wl, n_gpus):
+    step_mb = (2 + 2 * wl.n_sparse_layers) * wl.batch * wl.q_len * wl.n_q_heads * wl.head_dim * 2 / 1e6 \
+        + wl.batch * wl.n_kv_heads * wl.q_len * wl.k_sel * 4 / 1e6
     return {"workload": "%s: B=%d, L=%d, %dq/%dkv heads, D=%d, %s, k=%d, w=%d, 1 full + %d sparse layer(s) + 1 decode step"
                         % (wl.name, wl.batch, wl.q_len, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, wl.dtype,
                            wl.k_sel, wl.window, wl.n_sparse_layers),
             "structure": wl.structure, "sharding": "replica per GPU, no collective in the path (x%d)" % n_gpus,
-            "l2": "inputs larger than L2: every step streams Q, idx and O of several hundred MB"}
+            "l2": "inputs larger than L2: every step streams %.0f MB of Q, O and idx; the K/V cache of one KV head "
+                  "(%.1f MB) is L2 resident while its queries run" % (step_mb, 2 * wl.kv_len * wl.head_dim * 2 / 1e6)}
+
+
+# ------------------------------------------------------------------ roofline of the sparse-prefill kernel
+
+def sparse_roofline(wl, block, sp_ms, peaks):
+    """`frac`: gathered K/V bytes at the HBM peak, as the benchmark defines it (above 1 when the cache is L2
+    resident).  `frac_l2`: against the bare gather of the same rows measured now.  `binding_limit`: the slowest of
+    (recorded DRAM traffic at the HBM peak, flops at the bf16 peak, the measured gather) over the kernel's time."""
+    gb = gathered_kv_bytes(wl)
+    ach = gb / (sp_ms * 1e-3) / 1e9
+    tokens = wl.batch * wl.q_len
+    traffic, traffic_src = NCU_DRAM_TRAFFIC.get(wl.name, (None, None))
+    probe_ms, probe_mode = block.gather_ceiling_ms()
+    tpeak, which = tensor_peak_for(sp_ms, peaks)
+    t_tensor = sparse_attn_flops(wl) / (tpeak * 1e12) * 1e3
+    t_dram = traffic / (peaks["hbm_gbs"] * 1e9) * 1e3 if traffic else None
+    limits = {"gather_ms": round(probe_ms, 4), "tensor_ms": round(t_tensor, 4),
+              "dram_ms": None if t_dram is None else round(t_dram, 4)}
+    limit = max(v for v in (probe_ms, t_tensor, t_dram) if v is not None)
+    return {"kernel": "k_sparse_prefill (hs2_sparse_attn_prefill)", "bound": "hbm", "achieved": round(ach, 1),
+            "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": round(ach / peaks["hbm_gbs"], 4),
+            "traffic": traffic, "traffic_source": None if traffic is None else
+            "recorded ncu capture (%s), not measured in this run" % traffic_src,
+            "peak_source": peaks["source"], "algorithmic_bytes_per_launch": gb, "ms_per_launch": round(sp_ms, 4),
+            "tokens_per_s": round(tokens / (sp_ms * 1e-3), 1),
+            "l2_gather_ceiling": {"ms": round(probe_ms, 4), "gbs": round(gb / (probe_ms * 1e-3) / 1e9, 1),
+                                  "loads": "past L1" if probe_mode == 0 else "through L1",
+                                  "how": "hs2_probe_gather on the same K, V and idx: every attended row fetched in the "
+                                         "attention kernel's item order, no arithmetic, full occupancy"},
+            "frac_l2": round(probe_ms / sp_ms, 4),
+            "binding_limit": dict(limits, frac=round(limit / sp_ms, 4), tensor_peak=which),
+            "note": "achieved counts gathered K/V rows (512 B per attended token per KV head); one KV head's cache is "
+                    "L2 resident in prefill, so frac (of the HBM peak) exceeds 1 and is no measure of distance to a "
+                    "limit; frac_l2 is"}
+
+
+def full_layer_summary(wl, fa_ms, peaks):
+    fl = full_attn_flops(wl)
+    tpeak, which = tensor_peak_for(fa_ms, peaks)
+    return {"ms": round(fa_ms, 3), "effective_tflops": round(fl / (fa_ms * 1e-3) / 1e12, 2),
+            "peak_tflops": tpeak, "peak_kind": which, "frac": round(fl / (fa_ms * 1e-3) / 1e12 / tpeak, 4),
+            "note": "causal QK^T+PV flops only; score sweep and top-k are not credited"}
+
+
+def side_block(name, device, rank, peaks, world, steps=5):
+    """A smaller prefill configuration, timed briefly with the same step (side section of the JSON line)."""
+    wl = CONFIGS[name]
+    block = Block(wl, device, rank)
+    ms = time_steps(block, steps, 3, world)
+    km = block.kernel_means()
+    out = {"workload": workload_config(wl, world)["workload"], "ms_per_step": round(ms / steps, 4),
+           "tokens_per_s": round(wl.batch * wl.q_len * steps / (ms * 1e-3), 1),
+           "kernel_ms": {k: round(v, 4) for k, v in km.items()}}
+    if km.get("sparse_attn_prefill"):
+        out["roofline"] = sparse_roofline(wl, block, km["sparse_attn_prefill"], peaks)
+    if km.get("full_attn_select"):
+        out["full_attn_select"] = full_layer_summary(wl, km["full_attn_select"], peaks)
+    del block
+    torch.cuda.empty_cache()
+    return out
 
 
 # ------------------------------------------------------------------ main
@@ -586,13 +730,16 @@ def main():
     ap.add_argument("--steps", type=int, default=10)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=sorted(CONFIGS))
-    ap.add_argument("--cpu-rows", type=int, default=4096, help="query rows of the CPU-oracle sample (about 15 s of CPU work on cfg2)")
-    ap.add_argument("--skip", default="", help="comma list of: block, decode64k, native, kvproj, e2e, cpu")
+    ap.add_argument("--workload", default="cfg4", choices=sorted(CONFIGS))
+    ap.add_argument("--cpu-rows", type=int, default=0,
+                    help="query rows of the CPU-oracle sample (0: as many as about 3.5e11 oracle flops, 10-20 s)")
+    ap.add_argument("--skip", default="", help="comma list of: block, small, decode64k, native, kvproj, e2e, cpu")
     ap.add_argument("--decode-ctx", type=int, default=65536, help="context length of the decode section (profiling: 8192)")
     args = ap.parse_args()
     wl = CONFIGS[args.workload]
     skip = set(s for s in args.skip.split(",") if s)
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        respawn_under_torchrun(args.gpus)
     if args.impl == "reference":
         run_reference(args, wl)
         return
@@ -629,6 +776,11 @@ def main():
     kmeans = block.kernel_means()
     value = world * tokens_per_step * args.steps / (ms * 1e-3)
 
+    # ---- roofline of the sparse-prefill kernel (the metric's kernel), with the gather ceiling measured now
+    roofline = None
+    if rank == 0 and kmeans.get("sparse_attn_prefill"):
+        roofline = sparse_roofline(wl, block, kmeans["sparse_attn_prefill"], peaks)
+
     # ---- end to end: pinned host inputs in, outputs back, every step
     e2e = None
     if "e2e" not in skip:
@@ -644,28 +796,10 @@ def main():
 
     if rank != 0:
         return
-    # ---- roofline of the sparse-prefill kernel (the metric's kernel)
-    gb = gathered_kv_bytes(wl)
-    sp_ms = kmeans.get("sparse_attn_prefill")
-    roofline = None
-    if sp_ms:
-        ach = gb / (sp_ms * 1e-3) / 1e9
-        roofline = {"kernel": "k_sparse_prefill (hs2_sparse_attn_prefill)", "bound": "hbm", "achieved": round(ach, 1),
-                    "peak": peaks["hbm_gbs"], "unit": "GB/s", "frac": round(ach / peaks["hbm_gbs"], 4),
-                    "traffic": NCU_DRAM_TRAFFIC.get(wl.name), "peak_source": peaks["source"], "algorithmic_bytes_per_launch": gb,
-                    "ms_per_launch": round(sp_ms, 4),
-                    "tokens_per_s": round(tokens_per_step / (sp_ms * 1e-3), 1),
-                    "note": "achieved counts gathered K/V rows (512 B per attended token per KV head); the cache of "
-                            "this workload is L2 resident, so the fraction of the HBM peak can exceed 1"}
-    fa_ms = kmeans.get("full_attn_select")
     kernels = {k: round(v, 4) for k, v in kmeans.items()}
     extra = {}
-    if fa_ms:
-        fl = full_attn_flops(wl)
-        extra["full_attn_select"] = {"ms": round(fa_ms, 3), "effective_tflops": round(fl / (fa_ms * 1e-3) / 1e12, 2),
-                                     "peak_tflops": peaks["bf16_tflops_sustained"],
-                                     "frac": round(fl / (fa_ms * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"], 4),
-                                     "note": "causal QK^T+PV flops only; score sweep and top-k are not credited"}
+    if kmeans.get("full_attn_select"):
+        extra["full_attn_select"] = full_layer_summary(wl, kmeans["full_attn_select"], peaks)
     line = {
         "metric": METRIC, "value": round(value, 1), "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
         "warmup": warmup, "ms_per_step": round(ms / args.steps, 4), "higher_is_better": True, "scaling": "weak",
@@ -675,9 +809,13 @@ def main():
     line.update(extra)
     if e2e:
         line["e2e"] = e2e
+    del block
+    torch.cuda.empty_cache()
+    if "small" not in skip and world == 1:
+        for name in ("cfg2", "cfg3"):
+            if name != wl.name:
+                line[name] = side_block(name, device, rank, peaks, world)
     if "decode64k" not in skip and world == 1:
-        del block
-        torch.cuda.empty_cache()
         line["decode_64k"] = bench_decode_64k(device, peaks, ctx=args.decode_ctx)
     if "native" not in skip and world == 1:
         torch.cuda.empty_cache()
@@ -686,8 +824,9 @@ def main():
         torch.cuda.empty_cache()
         line["kv_project"] = bench_kv_project(device, peaks)
     if "cpu" not in skip and world == 1:
-        cb, _, _ = cpu_baseline(wl, args.cpu_rows)
-        line["cpu_baseline"] = cb
+        torch.cuda.empty_cache()
+        n = args.cpu_rows if args.cpu_rows > 0 else rows_for_flops(wl, 3.5e11)
+        line["cpu_baseline"] = cpu_baseline(wl, n)
     print(json.dumps(line))
 
 

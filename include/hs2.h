@@ -250,6 +250,20 @@ hs2_status hs2_sparse_attn_decode_static(const hs2_problem *p, const void *Q, co
 hs2_status hs2_kv_project(int64_t n_tokens, int32_t d_model, int32_t n_out, const void *H, int64_t ldh, const void *W,
                           int64_t ldw, void *C, int64_t ldc, float *scales, void *cuda_stream);
 
+/*
+ * Measurement aid for hs2_sparse_attn_prefill (the gather of Section 3.3; no counterpart in the paper): performs
+ * only the row fetches of that call - the same work items in the same order, the same slot array [idx row | forced
+ * window] with the same validity rules, every attended K row and V row loaded with 16-byte loads - and no
+ * arithmetic.  Its duration is what the memory system needs to deliver the rows to the SMs: the ceiling for the
+ * attention call's gather on this problem, whether the cache sits in L2 or in HBM.
+ *   p, K, V, idx  as for hs2_sparse_attn_prefill (bf16, head_dim 128, 16-byte aligned K and V; else
+ *                 HS2_ERR_UNSUPPORTED).  Q and O are not touched.
+ *   mode          0: loads that bypass L1 (what the attention kernel's copies do); 1: loads through L1.
+ *   sink_word     device, one unsigned the caller zeroes; it only keeps the loads observable.
+ */
+hs2_status hs2_probe_gather(const hs2_problem *p, const void *K, const void *V, const int32_t *idx, int mode,
+                            unsigned *sink_word, void *cuda_stream);
+
 /* Static, never-NULL description of a status. */
 const char *hs2_status_string(hs2_status s);
 

@@ -26,7 +26,7 @@ HS2_OP_FULL_ATTN_SELECT_FP8KV = 4
 EXPORTS = ["hs2_workspace_bytes", "hs2_full_attn_select", "hs2_topk_select", "hs2_sparse_attn_prefill",
            "hs2_sparse_attn_decode", "hs2_sparse_attn_prefill_gated", "hs2_sparse_attn_decode_gated",
            "hs2_sparse_attn_prefill_fp8kv", "hs2_sparse_attn_decode_fp8kv", "hs2_full_attn_select_fp8kv", "hs2_kv_project",
-           "hs2_sparse_attn_decode_static", "hs2_status_string", "hs2_last_cuda_error",
+           "hs2_sparse_attn_decode_static", "hs2_probe_gather", "hs2_status_string", "hs2_last_cuda_error",
            "hs2_launch_count", "hs2_device_error_flags", "hs2_set_filter_min_keys", "hs2_set_tcgen05_enabled"]
 
 
@@ -79,6 +79,8 @@ def load_library():
         lib.hs2_sparse_attn_prefill_fp8kv.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         lib.hs2_sparse_attn_decode_fp8kv.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         lib.hs2_full_attn_select_fp8kv.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
+        lib.hs2_probe_gather.argtypes = [pp, vp, vp, vp, C.c_int, vp, vp]
+        lib.hs2_probe_gather.restype = C.c_int
         for f in ("hs2_full_attn_select", "hs2_topk_select", "hs2_sparse_attn_prefill", "hs2_sparse_attn_decode",
                   "hs2_sparse_attn_prefill_gated", "hs2_sparse_attn_decode_gated", "hs2_sparse_attn_decode_static",
                   "hs2_sparse_attn_prefill_fp8kv", "hs2_sparse_attn_decode_fp8kv"):
@@ -348,6 +350,18 @@ def hs2_kv_project(h, w, *, out=None, fp8=False, scales=None, stream=None):
                                        _dp(scales) if fp8 else None, _stream(stream))
     _check(st, "hs2_kv_project")
     return (out, scales) if fp8 else out
+
+
+def hs2_probe_gather(prob: Problem, k, v, idx, *, mode=0, sink_word=None, stream=None):
+    """Measurement aid: only the K/V row fetches of ``hs2_sparse_attn_prefill`` on this problem (same items, same
+    order, same validity rules), no arithmetic.  ``mode`` 0 loads past L1, 1 through it.  Returns ``sink_word``."""
+    assert k.is_cuda and v.is_cuda and k.dtype == torch.bfloat16
+    if sink_word is None:
+        sink_word = torch.zeros(1, dtype=torch.int32, device=k.device)
+    c = prob.c_struct(None, k, None)
+    st = load_library().hs2_probe_gather(C.byref(c), _dp(k), _dp(v), _dp(idx), int(mode), _dp(sink_word), _stream(stream))
+    _check(st, "hs2_probe_gather")
+    return sink_word
 
 
 def hs2_sparse_attn_decode_static(prob: Problem, q, k, v, idx, *, sink=None, out, lse=None, stream=None):

@@ -13,7 +13,7 @@ _ROOT = os.path.dirname(_HERE)
 CSRC = os.path.join(_HERE, "csrc")
 LIB = os.path.join(_HERE, "libhs2.so")
 SOURCES = ["hs2_api.cu", "hs2_generic.cu", "hs2_topk.cu", "hs2_sparse_mma.cu", "hs2_full_mma.cu", "hs2_full_tc5.cu",
-           "hs2_sparse_tc5.cu", "hs2_sparse_fp8.cu", "hs2_kvproj.cu"]
+           "hs2_sparse_tc5.cu", "hs2_sparse_fp8.cu", "hs2_kvproj.cu", "hs2_probe.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--use_fast_math", "-I" + os.path.join(_ROOT, "include")]
 

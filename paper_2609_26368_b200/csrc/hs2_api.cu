@@ -576,6 +576,25 @@ hs2_status hs2_sparse_attn_decode_static(const hs2_problem *hp, const void *Q, c
     return e == cudaSuccess ? HS2_OK : cuda_fail(e);
 }
 
+hs2_status hs2_probe_gather(const hs2_problem *hp, const void *K, const void *V, const int32_t *idx, int mode,
+                            unsigned *sink_word, void *cuda_stream)
+{
+    Params p;
+    hs2_status s = resolve(hp, true, &p);
+    if (s != HS2_OK) return s;
+    if (!K || !V || !sink_word || (p.k > 0 && !idx) || (mode != 0 && mode != 1)) return HS2_ERR_INVALID_ARG;
+    if (hp->dtype != HS2_BF16 || p.D != 128 || p.ks_t % 8 || p.ks_h % 8 || p.ks_b % 8 ||
+        (reinterpret_cast<uintptr_t>(K) | reinterpret_cast<uintptr_t>(V)) % 16)
+        return HS2_ERR_UNSUPPORTED;
+    if ((s = check_device()) != HS2_OK) return s;
+    const cudaError_t e = launch_probe_gather(p, K, V, idx, mode, sink_word, (cudaStream_t)cuda_stream);
+    if (e == cudaErrorNotSupported) {
+        (void)cudaGetLastError();
+        return HS2_ERR_UNSUPPORTED;
+    }
+    return e == cudaSuccess ? HS2_OK : cuda_fail(e);
+}
+
 const char *hs2_status_string(hs2_status s)
 {
     switch (s) {

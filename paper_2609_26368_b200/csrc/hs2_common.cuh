@@ -156,6 +156,9 @@ bool kv_project_supported(int64_t T, int N, int dm, int64_t ldh, int64_t ldw, in
 cudaError_t launch_kv_project(int64_t T, int N, int dm, const void *H, int64_t ldh, const void *W, int64_t ldw, void *C,
                               int64_t ldc, float *scales, cudaStream_t st);
 cudaError_t read_kvproj_error(unsigned *out);
+// the row fetches of the sparse prefill and nothing else (measurement aid); mode 0: L2 loads, 1: through L1
+cudaError_t launch_probe_gather(const Params &p, const void *K, const void *V, const int32_t *idx, int mode,
+                                unsigned *out, cudaStream_t st);
 cudaError_t read_tc5_error(unsigned *out);
 cudaError_t read_sparse_error(unsigned *out);
 

@@ -92,6 +92,15 @@ def test_unsupported_and_null_and_workspace_errors(lib):
         binding.HS2_ERR_INVALID_ARG
 
 
+def test_gather_probe_argument_checks(lib):
+    one = C.c_void_p(256)
+    bf = _prob(head_dim=128, dtype=torch.bfloat16).c_struct()
+    assert lib.hs2_probe_gather(C.byref(bf), one, one, one, 0, None, None) == binding.HS2_ERR_INVALID_ARG   # no sink word
+    assert lib.hs2_probe_gather(C.byref(bf), one, one, one, 2, one, None) == binding.HS2_ERR_INVALID_ARG    # mode 0 or 1
+    assert lib.hs2_probe_gather(C.byref(bf), one, one, None, 0, one, None) == binding.HS2_ERR_INVALID_ARG   # idx needed
+    assert lib.hs2_probe_gather(C.byref(_prob().c_struct()), one, one, one, 0, one, None) == binding.HS2_ERR_UNSUPPORTED
+
+
 @pytest.mark.skipif(torch.cuda.is_available(), reason="checks the no-GPU behaviour")
 def test_no_gpu_means_an_error_not_a_fallback(lib):
     one = C.c_void_p(256)

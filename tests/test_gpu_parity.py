@@ -638,6 +638,24 @@ def test_malformed_indices_cannot_read_out_of_bounds():
     run.check_sparse(out, lse, 0)
 
 
+def test_gather_probe_runs_on_the_attention_calls_arguments():
+    """hs2_probe_gather (the bare row fetches of the sparse prefill, a measurement aid) accepts what the attention call
+    accepts - ragged lengths, malformed indices - touches neither indices nor cache, and sets no error."""
+    wl = scaled("cfg2", q_len=300, kv_len=700, k_sel=96, window=24, n_needles=4, batch=2)
+    run = BlockRun(make_inputs(wl)).run_full()
+    idx = run.idx.clone()
+    idx[0, 0, 5, :4] = torch.tensor([-1, 10 ** 6, 699, 3], dtype=torch.int32, device="cuda")   # void, past the cache, in the window, fine
+    kv_lens = torch.tensor([700, 333], dtype=torch.int32, device="cuda")
+    prob = hs2.Problem.from_tensors(run.q, run.k, wl.k_sel, wl.window, kv_lens=kv_lens)
+    k0, v0, i0 = run.k.clone(), run.v.clone(), idx.clone()
+    for mode in (0, 1):
+        word = hs2.hs2_probe_gather(prob, run.k, run.v, idx, mode=mode)
+        torch.cuda.synchronize()
+        assert int(word.item()) in (0, 1, 2)
+    assert torch.equal(run.k, k0) and torch.equal(run.v, v0) and torch.equal(idx, i0)
+    assert hs2.hs2_device_error_flags() == 0
+
+
 # ---------------------------------------------------------------- decode
 
 @pytest.mark.parametrize("heads", [(32, 4), (64, 4)])      # groups of 8, and of 16 (two sub-groups of 8)
