@@ -735,8 +735,17 @@ def main():
                     help="query rows of the CPU-oracle sample (0: as many as about 3.5e11 oracle flops, 10-20 s)")
     ap.add_argument("--skip", default="", help="comma list of: block, small, decode64k, native, kvproj, e2e, cpu")
     ap.add_argument("--decode-ctx", type=int, default=65536, help="context length of the decode section (profiling: 8192)")
+    ap.add_argument("--profile-len", type=int, default=0,
+                    help="profiling captures only: shorten the workload to this many tokens (same heads, k and w); "
+                         "the printed line is then no benchmark result")
+    ap.add_argument("--filter-min-keys", type=int, default=0,
+                    help="profiling captures only: context length from which the full layer's selection uses the "
+                         "filtered path (hs2_set_filter_min_keys); 0 keeps the library's default")
     args = ap.parse_args()
     wl = CONFIGS[args.workload]
+    if args.profile_len > 0:
+        from dataclasses import replace
+        wl = replace(wl, q_len=args.profile_len, kv_len=args.profile_len, name="%s_len%d" % (wl.name, args.profile_len))
     skip = set(s for s in args.skip.split(",") if s)
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
         respawn_under_torchrun(args.gpus)
@@ -747,6 +756,8 @@ def main():
         raise SystemExit("bench.py needs a CUDA device: the hs2 library has no CPU path")
     import paper_2609_26368_b200 as hs2
     hs2.load_library()
+    if args.filter_min_keys > 0:
+        hs2.hs2_set_filter_min_keys(args.filter_min_keys)
     rank, world, local = dist_setup(args.gpus)
     device = torch.device("cuda", local if world > 1 else 0)
     peaks = measured_peaks()

@@ -100,10 +100,11 @@ DecodeFusedPlan decode_fused_plan(const Params &pd, size_t sweep_ws)
 }
 
 // ---- filtered selection (sampled threshold -> ordered candidate lists -> select) ----
-constexpr int kFilterSamp = 8;              // every 8th key tile is scored for the threshold
-// The filtered path wins only when rows are long (measured: 131072 keys 485 ms vs 580 ms with strips, 32768
-// keys 67 ms vs 64 ms, 8192 keys 3.7 ms vs 2.1 ms): shorter contexts keep the strips.
-std::atomic<int> g_filter_min_keys{65537};
+constexpr int kFilterSamp = 16;             // every 16th key tile is scored for the threshold (every 8th: 6 ms more at 128K)
+// The filtered path wins when rows are long (measured, full layer with selection, filtered vs strips: 2 x 32768 keys
+// 35.0 vs 38.0 ms, 2 x 24576 keys 20.9 vs 21.5 ms, 2 x 16384 keys 10.3 vs 8.9 ms, 8192 keys 1.57 vs 1.12 ms): shorter
+// contexts keep the strips.
+std::atomic<int> g_filter_min_keys{24576};
 std::atomic<int> g_disable_tc5{0};          // testing knob: run the mma.sync kernels instead of the tcgen05 ones
 constexpr size_t kFilterBigCap = (size_t)1 << 30;
 
@@ -117,9 +118,12 @@ struct FilterPlan {
 FilterPlan filter_plan(const Params &p, hs2_dtype dt)
 {
     FilterPlan f{};
-    // expected list length: samp * (r + 6 sqrt(r)) with r the threshold rank at the thinnest sampling (1/samp)
+    // expected list length: samp * r with r the threshold rank at the thinnest sampling (1/samp), standard deviation
+    // samp * sqrt(r).  The list is kept as four sub-lists (one per quarter of a key tile), each a quarter of the
+    // list give or take the binomial split: capacity = mean + 6 standard deviations per sub-list.
     const double m = (double)p.k / kFilterSamp, r = m + 5.0 * sqrt(m) + 2.0;
-    const int want = (int)(kFilterSamp * (r + 6.0 * sqrt(r))) + 64;
+    const double mean = kFilterSamp * r, sd_sub = sqrt(kFilterSamp * kFilterSamp * r / 16.0 + 3.0 * mean / 16.0);
+    const int want = (int)(mean + 4.0 * 6.0 * sd_sub) + 64;
     f.cap = ((want > 1024 ? want : 1024) + 255) / 256 * 256;
     f.ns_w = filter_sample_width(p, kFilterSamp);
     f.per_row = align_up((size_t)f.ns_w * 4, 16);
@@ -133,7 +137,7 @@ int64_t filter_block_rows(const FilterPlan &f, int64_t rows, size_t ws_bytes)
 {
     const size_t budget = ws_bytes < kFilterBigCap + (size_t)(16 << 20) ? ws_bytes : kFilterBigCap + (size_t)(16 << 20);
     if (budget < 4096) return 0;
-    int64_t r = (int64_t)((budget - 4096) / (f.per_row + 12));
+    int64_t r = (int64_t)((budget - 4096) / (f.per_row + 24));
     return r > rows ? rows : r;
 }
 
@@ -142,7 +146,7 @@ size_t filter_ws_bytes(const FilterPlan &f, int64_t rows)
     int64_t r = (int64_t)(kFilterBigCap / f.per_row);
     if (r > rows) r = rows;
     if (r < 1) r = 1;
-    return align_up((size_t)r * (f.per_row + 12) + 4096, 256);
+    return align_up((size_t)r * (f.per_row + 24) + 4096, 256);
 }
 
 bool ws_ok(const void *ws, size_t ws_bytes, size_t need)
@@ -339,9 +343,9 @@ hs2_status hs2_full_attn_select(const hs2_problem *hp, const void *Q, const void
         if (block >= (rows < 1024 ? rows : 1024)) {
             char *base = (char *)ws;
             uint32_t *tau = (uint32_t *)base;
-            int *count = (int *)(base + (size_t)block * 4);
-            int *flag = (int *)(base + (size_t)block * 8);
-            char *big = base + align_up((size_t)block * 12, 256);
+            int *flag = (int *)(base + (size_t)block * 4);
+            int *count = (int *)(base + (size_t)block * 8);   // four sub-list counts per row
+            char *big = base + align_up((size_t)block * 24, 256);
             float *sample = (float *)big;
             float *cand_a = (float *)big;
             int32_t *cand_j = (int32_t *)(big + (size_t)block * fp.cap * 4);

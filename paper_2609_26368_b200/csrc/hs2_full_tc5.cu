@@ -399,15 +399,17 @@ enum ScBar { SQ_FULL = 0, SK_FULL0, SK_FULL1, SK_EMPTY0, SK_EMPTY1, ACC_FULL0, A
 //   SC_STRIP   write it to the strip row at its key position (keys split into chunks over blockIdx.x)
 //   SC_SAMPLE  only every `samp`-th key tile is computed; written compactly (tile t of the sample at 128 t)
 //   SC_FILTER  one CTA sweeps all keys of its queries and appends (score, key) of every score whose order key
-//              is >= the query's threshold to that query's candidate list (in no particular order)
+//              is >= the query's threshold to that query's candidate list (in no particular order).  A list is four
+//              sub-lists, one per quarter of a key tile (keys 32 q .. 32 q + 31 of every 128): the one warp that
+//              owns a (query, quarter) counts its sub-list in a register, so appending needs no atomic
 enum { SC_STRIP = 0, SC_SAMPLE = 1, SC_FILTER = 2 };
 
 struct FilterBuf {
     const uint32_t *tau_key;   // [rows of the block] threshold as order-preserving key
-    float *cand_a;             // [rows][cap]
-    int32_t *cand_j;           // [rows][cap]
-    int *count;                // [rows] candidates found (may exceed cap: then the row is redone elsewhere)
-    int cap;
+    float *cand_a;             // [rows][4][cap / 4]
+    int32_t *cand_j;           // [rows][4][cap / 4]
+    int *count;                // [rows][4] candidates found per sub-list (may exceed cap / 4: then the row is redone elsewhere; -1: gave up)
+    int cap;                   // multiple of 4
 };
 
 // the float whose order key is `key`; the two sentinels of the filter thresholds map to values that make the
@@ -455,7 +457,6 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     int *s_nq = reinterpret_cast<int *>(smem + kScOffNq);
     int64_t *s_row = reinterpret_cast<int64_t *>(smem + kScOffRow);
     uint32_t *s_tau = reinterpret_cast<uint32_t *>(smem + kScOffTau);
-    int *s_cntw = reinterpret_cast<int *>(smem + kScOffCnt);
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     // flattened (b, g, query tile); the filter sweep walks all keys per CTA, so its long tiles (late queries) go first
@@ -482,7 +483,7 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     if (MODE == SC_FILTER) {
         if (blockIdx.x != 0) return;
         if (ntile <= 0) {   // no candidates at all: the lists are empty
-            if (tid < TQ && iq0 + tid >= c_lo && iq0 + tid < c_hi) fb.count[bg_row0 + iq0 + tid - row0] = 0;
+            if (tid < 4 * TQ && iq0 + tid / 4 >= c_lo && iq0 + tid / 4 < c_hi) fb.count[(bg_row0 + iq0 + tid / 4 - row0) * 4 + (tid & 3)] = 0;
             return;
         }
     } else if (ntile <= 0) {
@@ -517,7 +518,6 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             s_row[t] = ok ? (bg_row0 + i - row0) : -1;
             if (MODE == SC_FILTER && t < 32) {
                 s_tau[t] = ok ? fb.tau_key[bg_row0 + i - row0] : 0xffffffffu;
-                s_cntw[t] = 0;
             }
         }
     }
@@ -595,7 +595,13 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         int nq_r[kHoist ? TQW : 1];
         float *orow_r[kHoist && MODE != SC_FILTER ? TQW : 1];
         float tau_r[kHoist && MODE == SC_FILTER ? TQW : 1];   // thresholds as floats: one compare per score
-        int rb_r[kHoist && MODE == SC_FILTER ? TQW : 1];      // first slot of the query's candidate list (the lists of a block hold < 2^28 entries)
+        int rb_r[kHoist && MODE == SC_FILTER ? TQW : 1];      // first slot of this warp's sub-list of the query's candidates (the lists of a block hold < 2^28 entries)
+        int cnt_r[MODE == SC_FILTER ? TQW : 1];               // entries this warp has appended per query (warp-uniform)
+        const int capq = MODE == SC_FILTER ? fb.cap >> 2 : 0;
+        if (MODE == SC_FILTER) {
+#pragma unroll
+            for (int q = 0; q < TQW; ++q) cnt_r[q] = 0;
+        }
         if (kHoist) {
 #pragma unroll
             for (int q = 0; q < TQW; ++q) {
@@ -603,7 +609,7 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 if (MODE != SC_FILTER) orow_r[q] = out + s_row[q_first + q] * out_stride;   // never used when nq is 0
                 if (MODE == SC_FILTER) {
                     tau_r[q] = key_to_float(s_tau[q_first + q]);
-                    rb_r[q] = (int)(s_row[q_first + q] * fb.cap);
+                    rb_r[q] = (int)(s_row[q_first + q] * fb.cap) + quarter * capq;
                 }
             }
         }
@@ -663,39 +669,33 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 mbar_arrive(bar(ACC_FREE0 + ab));
             }
             if (MODE == SC_FILTER) {
-                // Append in no particular order, one shared-memory counter per query.  Per warp and tile: one ballot
-                // per query, lane q reserves the warp's slots of query q with a single atomic (distinct addresses,
-                // one instruction), and every passing lane takes its rank inside the ballot.  A per-element atomic
-                // serialised the lanes of a query and cost one atomic round trip per query and tile.
+                // Append in no particular order.  This warp is the only writer of its sub-list of every query it owns,
+                // so the fill counts live in registers (the same in every lane): per query one ballot, a rank inside
+                // it, two stores.  The queries are independent of one another - no atomic, no shared memory, no
+                // dependent chain from one query to the next (an atomic per (query, warp, tile) on a shared counter
+                // plus a shuffle of its result made the eight appends one long latency chain).
                 if (__any_sync(0xffffffffu, passbits != 0u)) {
-                    unsigned masks[TQW];
-                    unsigned mine = 0u;
 #pragma unroll
                     for (int q = 0; q < TQW; ++q) {
-                        masks[q] = __ballot_sync(0xffffffffu, (passbits >> q) & 1u);
-                        if (lane == q) mine = masks[q];
-                    }
-                    int base = 0;
-                    if (mine != 0u) base = atomicAdd(&s_cntw[q_first + lane], __popc(mine));
-#pragma unroll
-                    for (int q = 0; q < TQW; ++q) {
-                        if (masks[q] == 0u) continue;   // uniform
-                        const int bq = __shfl_sync(0xffffffffu, base, q);
-                        if ((passbits >> q) & 1u) {
-                            const int pos = bq + __popc(masks[q] & lt_mask);
-                            if (pos < fb.cap) {
-                                const int64_t o = kHoist ? (int64_t)(rb_r[kHoist ? q : 0] + pos) : s_row[q_first + q] * fb.cap + pos;
-                                fb.cand_a[o] = aval[q];
-                                fb.cand_j[o] = key;
-                            }
+                        const bool mine = (passbits >> q) & 1u;
+                        const unsigned m = __ballot_sync(0xffffffffu, mine);
+                        const int pos = cnt_r[q] + __popc(m & lt_mask);
+                        if (mine && pos < capq) {
+                            const int64_t o = kHoist ? (int64_t)(rb_r[kHoist ? q : 0] + pos)
+                                                     : s_row[q_first + q] * fb.cap + quarter * capq + pos;
+                            fb.cand_a[o] = aval[q];
+                            fb.cand_j[o] = key;
                         }
+                        cnt_r[q] += __popc(m);
                     }
                 }
             }
         }
         if (MODE == SC_FILTER) {
-            asm volatile("bar.sync 1, %0;\n" ::"n"(kEpiThreads) : "memory");   // the epilogue warps: all appends are counted
-            if (tid < TQ && s_row[tid] >= 0) fb.count[s_row[tid]] = (alive && !*abort_flag) ? s_cntw[tid] : -1;   // -1: gave up
+            const bool fine = alive && !*abort_flag;   // otherwise the sweep gave up: -1 sends the row to the exact redo
+#pragma unroll
+            for (int q = 0; q < TQW; ++q)
+                if (lane == (q & 31) && s_row[q_first + q] >= 0) fb.count[s_row[q_first + q] * 4 + quarter] = fine ? cnt_r[q] : -1;
         }
     }
     __syncwarp();

@@ -139,7 +139,8 @@ __device__ __forceinline__ unsigned block_excl_scan(unsigned v, unsigned *s_warp
 // What the register-resident select works on:
 //   SEL_ROW   a score row indexed by key (the plain entry point and the strip path)
 //   SEL_TAU   the sampled scores of a row: only the value at a given rank is wanted (the filter threshold)
-//   SEL_CAND  the filtered candidates of a row, in key order, with their key indices as payload
+//   SEL_CAND  the filtered candidates of a row (four sub-lists of cap / 4 slots, each filled from its start, in no
+//             particular order), with their key indices as payload
 enum { SEL_ROW = 0, SEL_TAU = 1, SEL_CAND = 2 };
 
 struct SelArgs {
@@ -147,7 +148,7 @@ struct SelArgs {
     int cap;                  // candidate capacity per row (rows with at most cap keys keep every key)
     uint32_t *tau_key;        // SEL_TAU out: [rows of the block]
     int *flag;                // SEL_TAU: cleared; SEL_CAND: set when the row has to be redone exactly
-    const int *count;         // SEL_CAND: candidates found per row
+    const int *count;         // SEL_CAND: [rows][4] candidates found per sub-list (-1: the sweep gave up)
     const int32_t *payload;   // SEL_CAND: [rows][cap] key index of each candidate
 };
 
@@ -225,17 +226,31 @@ k_topk_cached(const Params p, const float *__restrict__ scores, int64_t score_st
             for (int t = tid; t < p.k; t += THREADS) out[t] = t < n_keys ? t : -1;
             return;
         }
-        if (MODE == SEL_CAND) {
-            const int cnt = sa.count[blockIdx.x];
-            if (cnt < k_row || cnt > sa.cap) {   // the threshold was off (or the sweep gave up): redo this row exactly
-                if (tid == 0) sa.flag[blockIdx.x] = 1;
-                return;
-            }
-            nc = cnt;
-        }
     }
     const int j0 = tid * E;
-    const bool has = j0 < nc;   // threads (whole warps, on short rows) past the row's end skip every per-candidate loop
+    int nv = min(max(nc - j0, 0), E);   // this thread's slots 0 .. nv-1 hold candidates
+    int ref_slot = 0;                   // a slot that holds a candidate
+    if (MODE == SEL_CAND) {
+        // all cap slots are loaded; sub-list s occupies slots [s capq, s capq + count[s]).  capq is a multiple of E, so
+        // the E slots of a thread lie in one sub-list.
+        const int capq = sa.cap >> 2;
+        int total = 0;
+        bool bad = false;
+#pragma unroll
+        for (int sub = 3; sub >= 0; --sub) {
+            const int c = sa.count[(int64_t)blockIdx.x * 4 + sub];
+            bad |= c < 0 || c > capq;
+            total += c;
+            if (c > 0) ref_slot = sub * capq;
+            if (j0 / capq == sub) nv = min(max(c - (j0 - sub * capq), 0), E);
+        }
+        if (bad || total < k_row) {   // the threshold was off (or the sweep gave up): redo this row exactly
+            if (tid == 0) sa.flag[blockIdx.x] = 1;
+            return;
+        }
+        if (j0 >= sa.cap) nv = 0;
+    }
+    const bool has = nv > 0;   // threads (whole warps, on short rows) past the row's end skip every per-candidate loop
     uint32_t key[E];
     // The two selects of the filtered path bring the row in through shared memory: consecutive lanes copy consecutive
     // 16-byte chunks (chunk c to slot c + c / CPT), every thread reads its own chunks at a pitch of CPT + 1 slots.
@@ -256,7 +271,7 @@ k_topk_cached(const Params p, const float *__restrict__ scores, int64_t score_st
     };
     if (kStaged) stage_in(srow);
     // which bits differ anywhere in the row: OR of (key ^ key of candidate 0), one logic op per candidate
-    const uint32_t ref = order_key(__ldg(srow));
+    const uint32_t ref = order_key(__ldg(srow + ref_slot));
     unsigned diff = 0u;
     if (has)
 #pragma unroll
@@ -266,15 +281,22 @@ k_topk_cached(const Params p, const float *__restrict__ scores, int64_t score_st
                                      : __ldg(reinterpret_cast<const float4 *>(srow + j0 + e4));
             key[e4] = order_key(v.x); key[e4 + 1] = order_key(v.y); key[e4 + 2] = order_key(v.z); key[e4 + 3] = order_key(v.w);
 #pragma unroll
-            for (int e = e4; e < e4 + 4; ++e) diff |= key[e] ^ ref;
+            for (int e = e4; e < e4 + 4; ++e) {
+                if (MODE == SEL_CAND && e >= nv) key[e] = 0u;   // a slot past the sub-list's fill
+                else diff |= key[e] ^ ref;
+            }
         } else {
 #pragma unroll
             for (int e = e4; e < e4 + 4; ++e) {
-                const bool ok = j0 + e < nc;
+                const bool ok = e < nv;
                 key[e] = ok ? order_key(srow[j0 + e]) : 0u;
                 if (ok) diff |= key[e] ^ ref;
             }
         }
+    }
+    else {
+#pragma unroll
+        for (int e = 0; e < E; ++e) key[e] = 0u;
     }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) diff |= __shfl_xor_sync(0xffffffffu, diff, o);
@@ -378,7 +400,7 @@ k_topk_cached(const Params p, const float *__restrict__ scores, int64_t score_st
         };
         unsigned my_eq = 0;
 #pragma unroll
-        for (int e = 0; e < E; ++e) my_eq += (j0 + e < nc) && key[e] == tau;
+        for (int e = 0; e < E; ++e) my_eq += (e < nv) && key[e] == tau;
         unsigned total_eq;
         block_excl_scan<WARPS>(my_eq, s_warp, lane, warp, &total_eq);
         uint32_t jmin = 0u;   // tied candidates are kept when ~index >= jmin
@@ -391,7 +413,7 @@ k_topk_cached(const Params p, const float *__restrict__ scores, int64_t score_st
             __syncthreads();
 #pragma unroll
             for (int e = 0; e < E; ++e)
-                if (j0 + e < nc && key[e] == tau) s_list[atomicAdd(&s_cnt, 1u)] = ~(uint32_t)pay(e);
+                if (e < nv && key[e] == tau) s_list[atomicAdd(&s_cnt, 1u)] = ~(uint32_t)pay(e);
             __syncthreads();
             jmin = select_on_list<THREADS>(s_list, total_eq, need_eq, hist, &s_prefix, &s_need, tid, lane, warp);
         }
@@ -400,7 +422,7 @@ k_topk_cached(const Params p, const float *__restrict__ scores, int64_t score_st
         __syncthreads();
 #pragma unroll
         for (int e = 0; e < E; ++e) {
-            if (j0 + e >= nc) continue;
+            if (e >= nv) continue;
             if (key[e] > tau || key[e] == tau) {
                 const uint32_t j = (uint32_t)pay(e);
                 // (the sweep only writes keys below n_keys; the range test keeps a damaged list from writing outside the bitmap)
@@ -1488,54 +1510,358 @@ cudaError_t launch_block_select(const Params &p, const float *scores, int64_t sc
     return cudaGetLastError();
 }
 
+// ---- the two selects of the filtered path --------------------------------------------------------------------------
+// Both want one thing first: the value at a given rank from the top of an unordered set (the threshold from a row's
+// sampled scores; the k-th best of a row's candidate list).  Order does not matter for that, so the values are read
+// strided - thread t takes entries t, t + THREADS, ... - which is coalesced without any staging and gives every
+// thread the same share whatever the set's size.  The rank is found as in k_topk_linear: one round of bins on a
+// linear scale between the set's smallest and largest value, then an exact ranking of the threshold bin's members.
+namespace {
+
+constexpr int kCandList = 4096;   // words of the candidate select's list (later its staged output row)
+
+struct RankOut {
+    uint32_t tau;       // order key of the value at rank `take` from the top
+    unsigned need_eq;   // how many of the entries equal to it belong to the top `take`
+    unsigned n_eq;      // how many entries equal it
+    bool ok;            // false: the threshold bin has more members than the list holds (nothing else is valid then)
+};
+
+// val[0 .. nv) are this thread's live entries; `take` >= 1 and at most the number of live entries of the CTA.
+// hist: 4 * THREADS words; s_list: list_cap words; every thread of the CTA must call.
+// BOTTOM: the wanted rank lies in the lower part of the set and the set thins out towards the top (a candidate list:
+// everything above a threshold, most of it to be kept).  Bins between the smallest and the largest value would then
+// put the dense lower part, where the answer is, into a few bins; instead the bins span twice the distance from the
+// smallest value to the mean (n_live entries in all) and the last bin takes everything above.  Any monotone map to
+// bins is exact; the choice only decides how many members the threshold bin has.
+template <int THREADS, int E, bool BOTTOM>
+__device__ __forceinline__ RankOut rank_from_top(const float (&val)[E], int nv, unsigned take, unsigned n_live, unsigned *hist,
+                                                 uint32_t *s_list, unsigned list_cap, float *s_lo, float *s_hi, unsigned *s_warp,
+                                                 unsigned *s_misc, int tid, int lane, int warp)
+{
+    constexpr int WARPS = THREADS / 32;
+    constexpr int NBT = 4, NB = NBT * THREADS;
+    unsigned &s_prefix = s_misc[0], &s_need = s_misc[1], &s_cnt = s_misc[2], &s_bin = s_misc[3], &s_eq = s_misc[4];
+    float vmin = INFINITY, vmax = -INFINITY;   // with BOTTOM, vmax carries the sum instead
+    if (BOTTOM) vmax = 0.f;
+#pragma unroll
+    for (int e = 0; e < E; ++e)
+        if (e < nv) { vmin = fminf(vmin, val[e]); vmax = BOTTOM ? vmax + val[e] : fmaxf(vmax, val[e]); }
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) {
+        vmin = fminf(vmin, __shfl_xor_sync(0xffffffffu, vmin, o));
+        const float t = __shfl_xor_sync(0xffffffffu, vmax, o);
+        vmax = BOTTOM ? vmax + t : fmaxf(vmax, t);
+    }
+    __syncthreads();   // the shared arrays may still be in use by an earlier phase of the caller
+    if (lane == 0) { s_lo[warp] = vmin; s_hi[warp] = vmax; }
+#pragma unroll
+    for (int t = 0; t < NBT; ++t) hist[t * THREADS + tid] = 0u;
+    if (tid == 0) s_cnt = 0u;
+    __syncthreads();
+    vmin = s_lo[0]; vmax = s_hi[0];
+#pragma unroll
+    for (int w = 1; w < WARPS; ++w) { vmin = fminf(vmin, s_lo[w]); vmax = BOTTOM ? vmax + s_hi[w] : fmaxf(vmax, s_hi[w]); }
+    const float range = BOTTOM ? 2.f * (vmax / (float)n_live - vmin) : vmax - vmin;
+    const bool flat = !(range > 0.f) || !(range < 3.0e38f);
+    const float c = flat ? 0.f : (float)NB / range;
+    const float d = flat ? 0.f : -vmin * c;
+    auto bin_of = [&](float v) { return min(__float2uint_rd(__fmaf_rn(v, c, d)), (unsigned)(NB - 1)); };
+#pragma unroll
+    for (int e = 0; e < E; ++e)
+        if (e < nv) atomicAdd(&hist[bin_of(val[e])], 1u);
+    __syncthreads();
+    unsigned mine = 0;
+#pragma unroll
+    for (int e = 0; e < NBT; ++e) mine += hist[NB - 1 - NBT * tid - e];
+    unsigned total;
+    const unsigned before = block_excl_scan<WARPS>(mine, s_warp, lane, warp, &total);
+    if (before < take && take <= before + mine) {
+        unsigned cum = before;
+#pragma unroll
+        for (int e = 0; e < NBT; ++e) {
+            const unsigned cnt = hist[NB - 1 - NBT * tid - e];
+            if (cum < take && take <= cum + cnt) { s_bin = NB - 1 - NBT * tid - e; s_need = take - cum; }
+            cum += cnt;
+        }
+    }
+    __syncthreads();
+    const unsigned tbin = s_bin;
+    unsigned need = s_need;
+    const float x_lo = tbin == 0u ? -INFINITY : (float)tbin;
+    const float x_hi = tbin == (unsigned)(NB - 1) ? __uint_as_float(0x7fc00000u) : (float)(tbin + 1u);
+#pragma unroll
+    for (int e = 0; e < E; ++e)
+        if (e < nv) {
+            const float x = __fmaf_rn(val[e], c, d);
+            if (!(x < x_lo) && !(x >= x_hi)) {
+                const unsigned slot = atomicAdd(&s_cnt, 1u);
+                if (slot < list_cap) s_list[slot] = order_key(val[e]);
+            }
+        }
+    __syncthreads();
+    const unsigned n_list = s_cnt;
+    RankOut r;
+    r.ok = n_list <= list_cap;
+    if (!r.ok) {
+        r.tau = 0u; r.need_eq = 0u; r.n_eq = 0u;
+        return r;
+    }
+    if (n_list <= kRankMax && n_list <= (unsigned)THREADS) {
+        if ((unsigned)tid < n_list) {
+            const uint32_t kt = s_list[tid];
+            unsigned gt = 0, eq = 0;
+            for (unsigned u = 0; u < n_list; ++u) {
+                const uint32_t v = s_list[u];
+                gt += v > kt;
+                eq += v == kt;
+            }
+            if (gt < need && need <= gt + eq) { s_prefix = kt; s_need = need - gt; s_eq = eq; }
+        }
+        __syncthreads();
+        r.tau = s_prefix;
+    } else {
+        r.tau = select_on_list<THREADS>(s_list, n_list, need, hist, &s_prefix, &s_need, tid, lane, warp);
+        if (tid == 0) s_eq = hist[r.tau & 255u];   // the last round's histogram: members equal to tau in all 32 bits
+        __syncthreads();
+    }
+    r.need_eq = s_need;
+    r.n_eq = s_eq;
+    return r;
+}
+
+// Threshold of a row from its sampled scores: the value at rank sample_rank() of the sample (see there).
+// One CTA per row; a launch takes the rows whose sample size lies in (ns_lo, ns_hi].
+template <int THREADS, int E>
+__global__ void __launch_bounds__(THREADS, E >= 64 ? 1 : (THREADS > 256 ? 2 : (E > 16 ? 3 : 1024 / THREADS)))
+k_sample_tau(const Params p, const float *__restrict__ sample, int64_t stride, int64_t row0, int ns_lo, int ns_hi, int samp,
+             int cap, uint32_t *__restrict__ tau_key, int *__restrict__ flag)
+{
+    constexpr int WARPS = THREADS / 32;
+    __shared__ unsigned hist[4 * THREADS];
+    __shared__ unsigned s_warp[WARPS];
+    __shared__ float s_lo[WARPS], s_hi[WARPS];
+    __shared__ unsigned s_misc[8];
+    extern __shared__ uint32_t s_tau_list[];   // THREADS * E keys
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int64_t row = row0 + blockIdx.x;
+    const int i = (int)(row % p.Lq);
+    const int b = (int)(row / ((int64_t)p.Lq * p.Hkv));
+    const int n_keys = max(0, min(pos_of(p, b, i) - p.w + 1, kvlen_of(p, b)));
+    const int k_row = min(p.k, n_keys);
+    const int nc = sample_size(n_keys, samp);
+    if (nc <= ns_lo || nc > ns_hi) return;   // another class's row
+    const int take = n_keys > 0 ? min(nc, sample_rank(k_row, n_keys, nc)) : 0;
+    if (tid == 0) flag[blockIdx.x] = 0;
+    if (n_keys <= cap || take <= 0) {   // short row: every key is a candidate
+        if (tid == 0) tau_key[blockIdx.x] = 0u;
+        return;
+    }
+    const float *srow = sample + (int64_t)blockIdx.x * stride;
+    float val[E];
+    const int nv = nc > tid ? min(E, (nc - tid + THREADS - 1) / THREADS) : 0;
+#pragma unroll
+    for (int e = 0; e < E; ++e) val[e] = e < nv ? __ldg(srow + tid + THREADS * e) : 0.f;
+    const RankOut r = rank_from_top<THREADS, E, false>(val, nv, (unsigned)take, (unsigned)nc, hist, s_tau_list, (unsigned)(THREADS * E), s_lo,
+                                                       s_hi, s_warp, s_misc, tid, lane, warp);
+    if (tid == 0) tau_key[blockIdx.x] = r.tau;
+}
+
+// Final selection of a row from its candidate list (four sub-lists, see the score sweep): the k best by (score
+// descending, key ascending), written in ascending key order.  Thread groups of THREADS / 4 take one sub-list each,
+// strided.  The kept keys are marked in a bitmap over the row's keys, which is then read out in order.
+// Rows whose list is unusable (a sub-list overflowed or was abandoned, fewer candidates than wanted) are flagged for
+// the exact redo.
+template <int THREADS, int E>
+__global__ void __launch_bounds__(THREADS, THREADS > 256 ? 1 : (E > 16 ? 3 : 4))
+k_cand_select(const Params p, const float *__restrict__ cand_a, const int32_t *__restrict__ cand_j, const int *__restrict__ count,
+              int cap, int32_t *__restrict__ idx, int64_t row0, int *__restrict__ flag)
+{
+    constexpr int WARPS = THREADS / 32, TG = THREADS / 4;
+    __shared__ unsigned hist[4 * THREADS];
+    __shared__ unsigned s_warp[WARPS];
+    __shared__ float s_lo[WARPS], s_hi[WARPS];
+    __shared__ unsigned s_misc[8];
+    extern __shared__ __align__(16) unsigned char s_cs_dyn[];   // [bitmap over the row's keys][list / staged output][key indices]
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int64_t row = row0 + blockIdx.x;
+    const int i = (int)(row % p.Lq);
+    const int b = (int)(row / ((int64_t)p.Lq * p.Hkv));
+    const int n_keys = max(0, min(pos_of(p, b, i) - p.w + 1, kvlen_of(p, b)));
+    const int k_row = min(p.k, n_keys);
+    int32_t *out = idx + row * p.k;
+    if (k_row == n_keys) {   // every candidate is kept: no need to look at the scores
+        for (int t = tid; t < p.k; t += THREADS) out[t] = t < n_keys ? t : -1;
+        return;
+    }
+    const int capq = cap >> 2;
+    int total = 0, mine_cnt = 0;
+    bool bad = false;
+#pragma unroll
+    for (int sub = 0; sub < 4; ++sub) {
+        const int c = count[(int64_t)blockIdx.x * 4 + sub];
+        bad |= c < 0 || c > capq;
+        total += c;
+        if (tid / TG == sub) mine_cnt = c;
+    }
+    if (bad || total < k_row) {   // the threshold was off (or the sweep gave up): redo this row exactly
+        if (tid == 0) flag[blockIdx.x] = 1;
+        return;
+    }
+    unsigned *bitmap = reinterpret_cast<unsigned *>(s_cs_dyn);
+    uint32_t *s_list = reinterpret_cast<uint32_t *>(s_cs_dyn + cached_bitmap_bytes(p.Lk));   // kCandList words
+    int32_t *s_pay = reinterpret_cast<int32_t *>(s_list + kCandList);                         // THREADS * E key indices
+    const int l = tid % TG;
+    const int64_t base = (int64_t)blockIdx.x * cap + (tid / TG) * capq + l;   // this thread's entries: base + TG * e
+    const int nv = mine_cnt > l ? min(E, (mine_cnt - l + TG - 1) / TG) : 0;
+    float val[E];
+#pragma unroll
+    for (int e = 0; e < E; ++e) val[e] = e < nv ? __ldg(cand_a + base + TG * e) : 0.f;
+    // the key indices are wanted only after the threshold is known: they travel to shared memory meanwhile (each
+    // thread reads back only what it copied itself, so its own wait is all the ordering that takes)
+#pragma unroll
+    for (int e = 0; e < E; ++e)
+        if (e < nv)
+            asm volatile("cp.async.ca.shared.global [%0], [%1], 4;\n" ::"r"((uint32_t)__cvta_generic_to_shared(s_pay + e * THREADS + tid)),
+                         "l"(cand_j + base + TG * e) : "memory");
+    asm volatile("cp.async.commit_group;\n" ::: "memory");
+    const int nwords = (n_keys + 31) >> 5;
+    for (int wd = tid; wd < nwords; wd += THREADS) bitmap[wd] = 0u;   // (rank_from_top's barriers order this before the marking)
+    const RankOut r = rank_from_top<THREADS, E, true>(val, nv, (unsigned)k_row, (unsigned)total, hist, s_list, (unsigned)kCandList, s_lo,
+                                                      s_hi, s_warp, s_misc, tid, lane, warp);
+    asm volatile("cp.async.wait_group 0;\n" ::: "memory");
+    if (!r.ok || r.n_eq > (unsigned)kCandList) {   // thousands of candidates within one bin of the threshold: the exact redo takes the row
+        if (tid == 0) flag[blockIdx.x] = 1;
+        return;
+    }
+    const float tau_f = __uint_as_float((r.tau & 0x80000000u) ? (r.tau & 0x7fffffffu) : ~r.tau);
+    uint32_t jmin = 0u;   // of the candidates equal to the threshold, those with ~key >= jmin are kept
+    if (r.n_eq > r.need_eq) {   // ties at the threshold, not all of them wanted: the lowest keys win
+        __syncthreads();
+        if (tid == 0) s_misc[2] = 0u;
+        __syncthreads();
+#pragma unroll
+        for (int e = 0; e < E; ++e)
+            if (e < nv && order_key(val[e]) == r.tau) s_list[atomicAdd(&s_misc[2], 1u)] = ~(uint32_t)s_pay[e * THREADS + tid];
+        __syncthreads();
+        jmin = select_on_list<THREADS>(s_list, r.n_eq, r.need_eq, hist, &s_misc[0], &s_misc[1], tid, lane, warp);
+    }
+    // mark the kept keys (the comparison must see denormal scores as they are)
+#pragma unroll
+    for (int e = 0; e < E; ++e)
+        if (e < nv && ge_exact(val[e], tau_f)) {
+            const uint32_t j = (uint32_t)s_pay[e * THREADS + tid];
+            // (the sweep only writes keys below n_keys; the range test keeps a damaged list from writing outside the bitmap)
+            if (j < (uint32_t)n_keys && (jmin == 0u || ~j >= jmin || order_key(val[e]) != r.tau)) atomicOr(&bitmap[j >> 5], 1u << (j & 31u));
+        }
+    __syncthreads();
+    // Read the bitmap out in ascending key order.  A warp takes a contiguous run of words, its lanes consecutive words
+    // (no bank conflicts); the position of a word's first kept key is the warp's base plus a shuffle scan of the counts.
+    const int per_warp = ((nwords + WARPS - 1) / WARPS + 31) & ~31;
+    const int wbeg = warp * per_warp;
+    unsigned kept = 0;
+    for (int wd = wbeg + lane; wd < min(nwords, wbeg + per_warp); wd += 32) kept += __popc(bitmap[wd]);
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) kept += __shfl_xor_sync(0xffffffffu, kept, o);
+    __syncthreads();   // s_warp may still be read by an earlier scan
+    if (lane == 0) s_warp[warp] = kept;
+    __syncthreads();
+    unsigned run = 0, total_sel = 0;
+#pragma unroll
+    for (int w = 0; w < WARPS; ++w) {
+        if (w < warp) run += s_warp[w];
+        total_sel += s_warp[w];
+    }
+    const bool staged = k_row <= kCandList;   // the list's memory is free now: the row leaves as coalesced stores
+    int32_t *dst = staged ? reinterpret_cast<int32_t *>(s_list) : out;
+    for (int w0 = wbeg; w0 < min(nwords, wbeg + per_warp); w0 += 32) {   // uniform per warp
+        const int wd = w0 + lane;
+        unsigned bits = wd < nwords ? bitmap[wd] : 0u;
+        const unsigned c = __popc(bits);
+        unsigned incl = c;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const unsigned t = __shfl_up_sync(0xffffffffu, incl, o);
+            if (lane >= o) incl += t;
+        }
+        unsigned posn = run + incl - c;
+        run += __shfl_sync(0xffffffffu, incl, 31);
+        while (bits) {
+            const int bpos = __ffs(bits) - 1;
+            bits &= bits - 1;
+            if (posn < (unsigned)p.k) dst[posn] = wd * 32 + bpos;
+            ++posn;
+        }
+    }
+    if (staged) {
+        __syncthreads();
+        for (int t = tid; t < p.k; t += THREADS) out[t] = t < k_row ? dst[t] : -1;
+    } else {
+        for (int t = k_row + tid; t < p.k; t += THREADS) out[t] = -1;
+    }
+    // a list with a repeated key (never written by the sweep) would select fewer keys than wanted: leave such a row to the redo
+    if (total_sel != (unsigned)k_row && tid == 0) flag[blockIdx.x] = 1;
+}
+
+}  // namespace
+
 cudaError_t launch_filter_thresholds(const Params &p, const float *sample, int64_t stride, int64_t row0, int64_t n_rows,
                                      int samp, int cap, uint32_t *tau_key, int *flag, cudaStream_t st)
 {
     if (n_rows == 0) return cudaSuccess;
-    SelArgs sa{samp, cap, tau_key, flag, nullptr, nullptr};
     const unsigned n = (unsigned)n_rows;
-    const int ns_max = filter_sample_width(p, samp);
-    // class by the size of the row's sample (every row is taken by exactly one launch); as for whole rows, a sample
-    // gets no more warps than it fills
-    // (dynamic shared memory: the staged sample row; above 48 KB it has to be asked for)
+    // sample sizes that occur among the rows of this block (known on the host when the positions are)
+    int ns_min = 0, ns_max = filter_sample_width(p, samp);
+    if (!p.q_start && !p.kv_lens && row0 / p.Lq == (row0 + n_rows - 1) / p.Lq) {
+        auto nk = [&](int64_t i) { const int64_t v = (int64_t)p.Lk - p.Lq + i - p.w + 1; return (int)(v < 0 ? 0 : (v > p.Lk ? p.Lk : v)); };
+        ns_min = sample_size(nk(row0 % p.Lq), samp);
+        ns_max = sample_size(nk((row0 + n_rows - 1) % p.Lq), samp);
+    }
+    // class by the size of the row's sample (every row is taken by exactly one launch); a sample gets no more warps
+    // than it fills.  Classes that no row of the block falls into are not launched.
     auto go = [&](auto kern, int threads, int e, int lo, int hi) -> cudaError_t {
-        const size_t smem = HS2_TOPK_STAGE ? cached_stage_bytes(threads, e) : 0;
-        if (smem > 48 * 1024) {
+        if (ns_max <= lo || ns_min > hi) return cudaSuccess;
+        const size_t smem = (size_t)threads * e * sizeof(uint32_t);
+        if (smem > 24 * 1024) {   // static shared memory counts against the 48 KB default too
             const cudaError_t e2 = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
             if (e2 != cudaSuccess) return e2;
         }
-        kern<<<n, threads, smem, st>>>(p, sample, stride, nullptr, row0, lo, hi, sa);
+        kern<<<n, threads, smem, st>>>(p, sample, stride, row0, lo, hi, samp, cap, tau_key, flag);
         count_launch();
         return cudaSuccess;
     };
-    cudaError_t e = go(k_topk_cached<64, 32, true, SEL_TAU>, 64, 32, -1, 2048);
-    if (e == cudaSuccess && ns_max > 2048) e = go(k_topk_cached<128, 32, true, SEL_TAU>, 128, 32, 2048, 4096);
-    if (e == cudaSuccess && ns_max > 4096) e = go(k_topk_cached<256, 32, true, SEL_TAU>, 256, 32, 4096, 8192);
-    if (e == cudaSuccess && ns_max > 8192) e = go(k_topk_cached<256, 64, true, SEL_TAU>, 256, 64, 8192, 16384);
-    if (e == cudaSuccess && ns_max > 16384) e = go(k_topk_cached<512, 64, true, SEL_TAU>, 512, 64, 16384, 32768);
+    cudaError_t e = go(k_sample_tau<64, 16>, 64, 16, -1, 1024);
+    if (e == cudaSuccess) e = go(k_sample_tau<128, 16>, 128, 16, 1024, 2048);
+    if (e == cudaSuccess) e = go(k_sample_tau<256, 16>, 256, 16, 2048, 4096);
+    if (e == cudaSuccess) e = go(k_sample_tau<256, 32>, 256, 32, 4096, 8192);
+    if (e == cudaSuccess) e = go(k_sample_tau<512, 32>, 512, 32, 8192, 16384);
+    if (e == cudaSuccess) e = go(k_sample_tau<512, 64>, 512, 64, 16384, 32768);
     if (e != cudaSuccess) return e;
     return cudaGetLastError();
 }
 
-// final selection from the candidate lists; rows whose count is out of range get flag[row] = 1
+// final selection from the candidate lists; rows whose lists are unusable get flag[row] = 1
 cudaError_t launch_filter_select(const Params &p, const float *cand_a, const int32_t *cand_j, const int *count, int cap,
                                  int32_t *idx, int64_t row0, int64_t n_rows, int *flag, cudaStream_t st)
 {
     if (n_rows == 0) return cudaSuccess;
-    SelArgs sa{1, cap, nullptr, flag, count, cand_j};
     const unsigned n = (unsigned)n_rows;
-    const size_t bm = cached_bitmap_bytes(p.Lk);   // one bit per key of the row (at most 32 KB), then the staged row
+    const size_t bm = cached_bitmap_bytes(p.Lk);   // one bit per key of the row, then the list (later the staged output row)
     auto go = [&](auto kern, int threads, int e) -> cudaError_t {
-        const size_t smem = bm + (HS2_TOPK_STAGE ? cached_stage_bytes(threads, e) : 0);
-        if (smem > 48 * 1024) {
+        const size_t smem = bm + (size_t)kCandList * sizeof(uint32_t) + (size_t)threads * e * sizeof(int32_t);
+        if (smem > 24 * 1024) {   // static shared memory counts against the 48 KB default too
             const cudaError_t e2 = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
             if (e2 != cudaSuccess) return e2;
         }
-        kern<<<n, threads, smem, st>>>(p, cand_a, cap, idx, row0, -1, 0x7fffffff, sa);
+        kern<<<n, threads, smem, st>>>(p, cand_a, cand_j, count, cap, idx, row0, flag);
         count_launch();
         return cudaSuccess;
     };
-    const cudaError_t e = cap <= 8192 ? go(k_topk_cached<256, 32, true, SEL_CAND>, 256, 32) : go(k_topk_cached<512, 64, true, SEL_CAND>, 512, 64);
+    // a thread group of THREADS / 4 takes one sub-list of cap / 4 slots, E slots per thread
+    cudaError_t e;
+    if (cap <= 4096) e = go(k_cand_select<256, 16>, 256, 16);
+    else if (cap <= 8192) e = go(k_cand_select<256, 32>, 256, 32);
+    else e = go(k_cand_select<512, 64>, 512, 64);
     if (e != cudaSuccess) return e;
     return cudaGetLastError();
 }

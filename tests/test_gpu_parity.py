@@ -221,7 +221,7 @@ def _filtered_redo():
     wl = scaled("cfg2", q_len=2048, kv_len=8192, k_sel=512, window=32, n_needles=4)
     for sampled_high in (True, False):
         inp = make_inputs(wl)
-        tile = (torch.arange(wl.kv_len) // 128) % 8 == 0                  # the key tiles the sample looks at
+        tile = (torch.arange(wl.kv_len) // 128) % 16 == 0                 # the key tiles the sample looks at
         scale_rows = torch.where(tile == sampled_high, 3.0, 0.05).to(inp.k.dtype)
         # keys of the favoured tiles line up with every query (large logits), the others are near zero
         inp.k.mul_(scale_rows.view(1, -1, 1, 1))
@@ -230,19 +230,31 @@ def _filtered_redo():
         from paper_2609_26368_b200 import binding
         ws = torch.zeros(hs2.hs2_workspace_bytes(run.prob, binding.HS2_OP_FULL_ATTN_SELECT), dtype=torch.uint8, device="cuda")
         run.run_full(want_scores=False, ws=ws)
-        # white box: the workspace starts with threshold, count and flag words per row (one block here)
-        flags = ws[: 12 * n_rows].view(torch.int32)[2 * n_rows: 3 * n_rows]
+        # white box: the workspace starts with one threshold word and one flag word per row (one block here)
+        flags = ws[: 8 * n_rows].view(torch.int32)[n_rows: 2 * n_rows]
         assert int(flags.sum()) > n_rows // 4, "the adversarial rows were not sent to the exact redo"
         rows = [(0, i) for i in (0, 600, 1500, 2047)]
         run.check_full(rows=rows)
         ref = BlockRun(inp).run_full(want_scores=True)
-        assert torch.equal(run.idx, ref.idx)
+        # Rows that were not redone select from the same tensor-core scores as the strip path: bit-equal.  A redone row
+        # is selected from scores recomputed with fp32 FMAs, so it may swap keys whose scores agree to within rounding:
+        # every key in the symmetric difference must lie in the near-tie band around the row's k-th score.
+        differ = (run.idx != ref.idx).any(-1).reshape(-1)
+        assert not bool((differ & (flags == 0)).any()), "a row that was not redone differs from the strip path"
+        sc = ref.scores.reshape(n_rows, wl.kv_len)
+        for r in torch.nonzero(differ).flatten().tolist()[:256]:
+            a, b = run.idx.reshape(n_rows, -1)[r], ref.idx.reshape(n_rows, -1)[r]
+            a, b = a[a >= 0], b[b >= 0]
+            assert a.numel() == b.numel() and bool((a[1:] > a[:-1]).all())
+            tau = sc[r, b.long()].min()
+            sym = torch.tensor(sorted(set(a.tolist()) ^ set(b.tolist())), device="cuda")
+            assert bool(((sc[r, sym] - tau).abs() <= 1e-3).all()), "row %d: swap outside the near-tie band" % r
     # and ordinary data does not need the redo at all
     inp = make_inputs(wl)
     run = BlockRun(inp)
     ws = torch.zeros(hs2.hs2_workspace_bytes(run.prob, binding.HS2_OP_FULL_ATTN_SELECT), dtype=torch.uint8, device="cuda")
     run.run_full(want_scores=False, ws=ws)
-    assert int(ws[: 12 * n_rows].view(torch.int32)[2 * n_rows: 3 * n_rows].sum()) == 0
+    assert int(ws[: 8 * n_rows].view(torch.int32)[n_rows: 2 * n_rows].sum()) == 0
 
 
 def test_mma_sync_fallback_kernels_of_the_full_layer():
@@ -270,6 +282,18 @@ def test_full_layer_on_a_cache_larger_than_l2():
     run.check_full(rows=rows)
     out, lse = run.run_sparse(0)
     run.check_sparse(out, lse, 0, rows=rows)
+
+
+def test_filtered_selection_on_a_context_of_70k_keys():
+    """Contexts from 65537 keys on take the filtered selection by default; between 65537 and about 90000 keys its
+    candidate select needs the opt-in to more than 48 KB of shared memory for static plus dynamic together."""
+    wl = scaled("cfg2", q_len=512, kv_len=70016, k_sel=1024, window=64, n_needles=8)
+    run = BlockRun(make_inputs(wl)).run_full()
+    rows = [(0, i) for i in (0, 1, 255, 256, 511)]
+    run.check_full(rows=rows)
+    ref = BlockRun(run.inp).run_full(want_scores=True)
+    assert torch.equal(run.idx, ref.idx)
+    assert hs2.hs2_device_error_flags() == 0
 
 
 def test_paper_native_shape_mqa64_dim256_with_sink():
