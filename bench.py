@@ -373,7 +373,7 @@ def time_e2e(wl, device, rank, block0, steps, world):
 
 # ------------------------------------------------------------------ decode at 64K context (cfg5)
 
-def bench_decode_64k(device, peaks, reps=5, burst=40, ctx=65536):
+def bench_decode_64k(device, peaks, reps=5, burst=40, ctx=65536, batch=0):
     """Split-KV sparse decode on the 64K-context configuration; indices from the full layer's scores.
 
     The cache (8.6 GB) is far above L2; consecutive launches rotate over four query/index sets so
@@ -383,6 +383,8 @@ def bench_decode_64k(device, peaks, reps=5, burst=40, ctx=65536):
     from paper_2609_26368_b200 import binding
     from dataclasses import replace
     wl = replace(CONFIGS["cfg5"], kv_len=ctx)
+    if batch > 0:
+        wl = replace(wl, batch=batch)
     inp = make_inputs(wl, device)
     k, v = inp.k, inp.v
     B, _, Hq, D = inp.q_full.shape
@@ -455,7 +457,7 @@ def bench_decode_64k(device, peaks, reps=5, burst=40, ctx=65536):
            "achieved_gbs": round(gb8 / (us8 * 1e-6) / 1e9, 1), "frac": round(gb8 / (us8 * 1e-6) / 1e9 / peaks["hbm_gbs"], 4),
            "full_attn_select_decode_ms": round(min(t_full8[1:]), 3), "cache_sweep_gb": round(sweep8, 2),
            "cache_sweep_ms_at_hbm_peak": round(sweep8 / peaks["hbm_gbs"] * 1e3, 3)}
-    return {"workload": "cfg5: B=64, ctx %d, 32q/4kv, D=128, bf16, k=2048, w=128" % ctx, "fp8_kv_cache": fp8,
+    return {"workload": "cfg5: B=%d, ctx %d, 32q/4kv, D=128, bf16, k=2048, w=128" % (wl.batch, ctx), "fp8_kv_cache": fp8,
             "sparse_decode_us_per_step": round(us, 2), "gathered_kv_bytes": gb,
             "achieved_gbs": round(ach, 1), "peak_gbs": peaks["hbm_gbs"], "frac": round(ach / peaks["hbm_gbs"], 4),
             "full_attn_select_decode_ms": round(min(t_full[1:]), 3), "launches_back_to_back": burst,
@@ -735,6 +737,7 @@ def main():
                     help="query rows of the CPU-oracle sample (0: as many as about 3.5e11 oracle flops, 10-20 s)")
     ap.add_argument("--skip", default="", help="comma list of: block, small, decode64k, native, kvproj, e2e, cpu")
     ap.add_argument("--decode-ctx", type=int, default=65536, help="context length of the decode section (profiling: 8192)")
+    ap.add_argument("--decode-batch", type=int, default=0, help="profiling captures only: batch of the decode section (default 64)")
     ap.add_argument("--profile-len", type=int, default=0,
                     help="profiling captures only: shorten the workload to this many tokens (same heads, k and w); "
                          "the printed line is then no benchmark result")
@@ -766,7 +769,7 @@ def main():
     if "block" in skip:      # side sections only (used for profiling captures)
         side = {}
         if "decode64k" not in skip:
-            side["decode_64k"] = bench_decode_64k(device, peaks, ctx=args.decode_ctx)
+            side["decode_64k"] = bench_decode_64k(device, peaks, ctx=args.decode_ctx, batch=args.decode_batch)
         if "native" not in skip:
             side["paper_native_shape"] = bench_native(device, peaks)
         if "kvproj" not in skip:
@@ -827,7 +830,7 @@ def main():
             if name != wl.name:
                 line[name] = side_block(name, device, rank, peaks, world)
     if "decode64k" not in skip and world == 1:
-        line["decode_64k"] = bench_decode_64k(device, peaks, ctx=args.decode_ctx)
+        line["decode_64k"] = bench_decode_64k(device, peaks, ctx=args.decode_ctx, batch=args.decode_batch)
     if "native" not in skip and world == 1:
         torch.cuda.empty_cache()
         line["paper_native_shape"] = bench_native(device, peaks)

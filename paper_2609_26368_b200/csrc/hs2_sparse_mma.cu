@@ -47,6 +47,11 @@
 #ifndef HS2_SP_BULK
 #define HS2_SP_BULK 0
 #endif
+// 1: the prefill kernel fetches the K rows and the V rows of a tile as separate copy groups and overlaps each with the
+// other half's arithmetic inside the warp; 0: one fetch, one wait, one fold per tile.
+#ifndef HS2_SP_OVERLAP
+#define HS2_SP_OVERLAP 0
+#endif
 
 namespace hs2 {
 namespace {
@@ -202,16 +207,29 @@ __device__ __forceinline__ void issue_stage(const Item &it, uint32_t stage_base,
     }
 }
 
+// one tensor's rows of a tile (K into the first half of a stage, V into the second): the overlapped prefill loop
+// fetches the two halves at different times
 template <int KT>
-__device__ __forceinline__ void consume_stage(Acc &acc, const uint32_t (&qf)[16], uint32_t stage_base, unsigned mask,
-                                              float scale_log2, int lane, float *raw = nullptr, int lk = 0, int G = 0,
-                                              const int *sjrow = nullptr)
+__device__ __forceinline__ void issue_rows(const char *tensor_base, int rs, uint32_t dst_base, int j, int lane)
 {
-    const int g = lane >> 2;
+    const int c = lane & 15, hi = lane >> 4;
+    const uint32_t cx = (uint32_t)(c ^ hi);
+    const uint32_t dst_lane = dst_base + hi * kRowBytes;
+    const char *tc = tensor_base + c * 16;
+#pragma unroll
+    for (int r0 = 0; r0 < KT; r0 += 2) {
+        const int jr = __shfl_sync(0xffffffffu, j, r0 + hi);
+        const uint32_t dst = dst_lane + r0 * kRowBytes + ((cx ^ (uint32_t)(r0 & 6)) << 4);
+        cp_async16(dst, tc + (int64_t)max(jr, 0) * rs, jr < 0 ? 0 : 16);   // void rows are zero filled, nothing is read
+    }
+}
+
+// S^T = K Q^T of one stage: rows = keys, columns = heads.  Two accumulator chains per tile keep the tensor pipe busy.
+template <int KT>
+__device__ __forceinline__ void stage_scores(float (&s)[KT / 16][4], const uint32_t (&qf)[16], uint32_t stage_base, int lane)
+{
     const int mi = lane >> 3, rr = lane & 7;
     constexpr int MT = KT / 16;
-    float s[MT][4];
-    // S^T = K Q^T : rows = keys, columns = heads.  Two accumulator chains per tile keep the tensor pipe busy.
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt) {
         float s2[4] = {0.f, 0.f, 0.f, 0.f};
@@ -230,23 +248,16 @@ __device__ __forceinline__ void consume_stage(Acc &acc, const uint32_t (&qf)[16]
 #pragma unroll
         for (int e = 0; e < 4; ++e) s[mt][e] += s2[e];
     }
-    if (raw) {
-        // The decode-shaped full layer keeps the raw products: the selection scores need the final LSE, and reading
-        // them back (4 bytes per head and key) is far cheaper than sweeping K a second time.
-        const int t = lane & 3;
-#pragma unroll
-        for (int mt = 0; mt < MT; ++mt)
-#pragma unroll
-            for (int r = 0; r < 2; ++r) {
-                const int j = sjrow[mt * 16 + g + 8 * r];
-                if (j >= 0) {
-#pragma unroll
-                    for (int hh = 0; hh < 2; ++hh)
-                        if (2 * t + hh < G) raw[(int64_t)(2 * t + hh) * lk + j] = s[mt][2 * r + hh];
-                }
-            }
-    }
-    // online softmax, base-2 domain; this thread: heads 2t+hh, keys 16 mt + g + 8 r
+}
+
+// online softmax of one stage in the base-2 domain; this thread: heads 2t+hh, keys 16 mt + g + 8 r.  Leaves the
+// probabilities as the bf16 B operand of the second product and rescales the accumulator when a maximum moved.
+template <int KT>
+__device__ __forceinline__ void stage_softmax(Acc &acc, float (&s)[KT / 16][4], uint32_t (&pb)[KT / 16][2], unsigned mask,
+                                              float scale_log2, int lane)
+{
+    const int g = lane >> 2;
+    constexpr int MT = KT / 16;
     float mx[2] = {-INFINITY, -INFINITY};
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt)
@@ -272,7 +283,6 @@ __device__ __forceinline__ void consume_stage(Acc &acc, const uint32_t (&qf)[16]
         acc.m[hh] = m_new;
         acc.l[hh] *= corr[hh];
     }
-    uint32_t pb[MT][2];
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt) {
         float pv[4];
@@ -291,8 +301,14 @@ __device__ __forceinline__ void consume_stage(Acc &acc, const uint32_t (&qf)[16]
             acc.o[dt][2] *= corr[0]; acc.o[dt][3] *= corr[1];
         }
     }
-    // O^T += V^T P^T : rows = output dimensions, contraction over the keys of the stage
-    const uint32_t vbase = stage_base + KT * kPitch;
+}
+
+// O^T += V^T P^T : rows = output dimensions, contraction over the keys of the stage (vbase: the stage's V rows)
+template <int KT>
+__device__ __forceinline__ void stage_pv(Acc &acc, const uint32_t (&pb)[KT / 16][2], uint32_t vbase, int lane)
+{
+    const int mi = lane >> 3, rr = lane & 7;
+    constexpr int MT = KT / 16;
 #pragma unroll
     for (int mt = 0; mt < MT; ++mt) {
         const uint32_t rowaddr = vbase + (mt * 16 + (mi >> 1) * 8 + rr) * kPitch;
@@ -304,6 +320,35 @@ __device__ __forceinline__ void consume_stage(Acc &acc, const uint32_t (&qf)[16]
             mma_bf16(acc.o[dt], a, pb[mt][0], pb[mt][1]);
         }
     }
+}
+
+template <int KT>
+__device__ __forceinline__ void consume_stage(Acc &acc, const uint32_t (&qf)[16], uint32_t stage_base, unsigned mask,
+                                              float scale_log2, int lane, float *raw = nullptr, int lk = 0, int G = 0,
+                                              const int *sjrow = nullptr)
+{
+    constexpr int MT = KT / 16;
+    float s[MT][4];
+    stage_scores<KT>(s, qf, stage_base, lane);
+    if (raw) {
+        // The decode-shaped full layer keeps the raw products: the selection scores need the final LSE, and reading
+        // them back (4 bytes per head and key) is far cheaper than sweeping K a second time.
+        const int g = lane >> 2, t = lane & 3;
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+            for (int r = 0; r < 2; ++r) {
+                const int j = sjrow[mt * 16 + g + 8 * r];
+                if (j >= 0) {
+#pragma unroll
+                    for (int hh = 0; hh < 2; ++hh)
+                        if (2 * t + hh < G) raw[(int64_t)(2 * t + hh) * lk + j] = s[mt][2 * r + hh];
+                }
+            }
+    }
+    uint32_t pb[MT][2];
+    stage_softmax<KT>(acc, s, pb, mask, scale_log2, lane);
+    stage_pv<KT>(acc, pb, stage_base + KT * kPitch, lane);
 }
 
 // Fold slot tiles [t_begin, t_end) of one item into acc with an NSTAGE-deep cp.async pipeline.
@@ -342,9 +387,56 @@ __device__ __forceinline__ void run_tiles(const Params &p, const Item &it, const
         }
         return false;
     };
+    if (HS2_SP_OVERLAP && NSTAGE == 1 && !kBulk && !it.raw) {
+        // Built and measured, not the default (HS2_SP_OVERLAP=1): 72.5 vs 68.5 ms per layer at 128K, 18.7 vs 17.6 ms at
+        // 2 x 32K, 1.18 vs 1.14 ms at 8K.  The other warps of the SM already cover a warp's fetch; two waits and half-sized
+        // copy bursts per tile cost more than the overlap inside one warp returns.
+        // One buffer per warp, its K half and its V half fetched at different times so that most of each fetch hides
+        // behind the other half's arithmetic:
+        //   V(t) is issued, K(t) awaited, S = K Q^T; K(t+1) is issued into the K half just read; softmax;
+        //   V(t) awaited, O += P V.  Two copy groups are in flight at any time and each wait leaves the younger one.
+        constexpr int MT = KT / 16;
+        const int rs = (int)it.row_stride;
+        auto next_tile = [&](int &j) -> bool {   // the next tile with a live slot
+            while (next < t_end) {
+                j = slot_fix<KT>(p, it, next, lane, jn);
+                ++next;
+                if (next < t_end) jn = slot_raw<KT>(p, it, next, lane);
+                if (__ballot_sync(0xffffffffu, j >= 0)) return true;
+            }
+            return false;
+        };
+        int jc;
+        if (!next_tile(jc)) return;
+        issue_rows<KT>(it.Kb, rs, sbase, jc, lane);
+        cp_async_commit();
+        while (true) {
+            issue_rows<KT>(it.Vb, rs, sbase + KT * kRowBytes, jc, lane);
+            cp_async_commit();
+            const unsigned mask = __ballot_sync(0xffffffffu, jc >= 0);
+            cp_async_wait<1>();   // K(t) has landed; V(t) may still be on its way
+            __syncwarp();
+            float s[MT][4];
+            stage_scores<KT>(s, qf, sbase, lane);
+            __syncwarp();         // every lane has read the K half before the next tile's rows land in it
+            int jnext = -1;
+            const bool more = next_tile(jnext);
+            if (more) issue_rows<KT>(it.Kb, rs, sbase, jnext, lane);
+            cp_async_commit();    // (an empty group after the last tile keeps the counting uniform)
+            uint32_t pb[MT][2];
+            stage_softmax<KT>(acc, s, pb, mask, p.scale_log2, lane);
+            cp_async_wait<1>();   // V(t) has landed; K(t+1) may still be on its way
+            __syncwarp();
+            stage_pv<KT>(acc, pb, sbase + KT * kRowBytes, lane);
+            __syncwarp();         // every lane has read the V half before the next tile's rows land in it
+            if (!more) break;
+            jc = jnext;
+        }
+        cp_async_wait<0>();
+        return;
+    }
     if (NSTAGE == 1 && !kBulk) {
-        // one buffer per warp: fetch, wait, fold.  A warp overlaps nothing by itself; the other warps of the SM do,
-        // and a warp that needs half the shared memory lets twice as many of them be resident.
+        // one buffer per warp: fetch, wait, fold (the variant that also keeps the raw products)
         while (try_issue(0)) {
             cp_async_commit();
             cp_async_wait<0>();

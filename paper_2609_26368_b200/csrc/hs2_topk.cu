@@ -1542,11 +1542,14 @@ __device__ __forceinline__ RankOut rank_from_top(const float (&val)[E], int nv, 
     constexpr int WARPS = THREADS / 32;
     constexpr int NBT = 4, NB = NBT * THREADS;
     unsigned &s_prefix = s_misc[0], &s_need = s_misc[1], &s_cnt = s_misc[2], &s_bin = s_misc[3], &s_eq = s_misc[4];
+    const int nvw = __reduce_max_sync(0xffffffffu, nv);   // the unrolled per-entry loops stop at the warp's longest thread
     float vmin = INFINITY, vmax = -INFINITY;   // with BOTTOM, vmax carries the sum instead
     if (BOTTOM) vmax = 0.f;
 #pragma unroll
-    for (int e = 0; e < E; ++e)
+    for (int e = 0; e < E; ++e) {
+        if (e >= nvw) break;
         if (e < nv) { vmin = fminf(vmin, val[e]); vmax = BOTTOM ? vmax + val[e] : fmaxf(vmax, val[e]); }
+    }
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) {
         vmin = fminf(vmin, __shfl_xor_sync(0xffffffffu, vmin, o));
@@ -1568,8 +1571,10 @@ __device__ __forceinline__ RankOut rank_from_top(const float (&val)[E], int nv, 
     const float d = flat ? 0.f : -vmin * c;
     auto bin_of = [&](float v) { return min(__float2uint_rd(__fmaf_rn(v, c, d)), (unsigned)(NB - 1)); };
 #pragma unroll
-    for (int e = 0; e < E; ++e)
+    for (int e = 0; e < E; ++e) {
+        if (e >= nvw) break;
         if (e < nv) atomicAdd(&hist[bin_of(val[e])], 1u);
+    }
     __syncthreads();
     unsigned mine = 0;
 #pragma unroll
@@ -1591,7 +1596,8 @@ __device__ __forceinline__ RankOut rank_from_top(const float (&val)[E], int nv, 
     const float x_lo = tbin == 0u ? -INFINITY : (float)tbin;
     const float x_hi = tbin == (unsigned)(NB - 1) ? __uint_as_float(0x7fc00000u) : (float)(tbin + 1u);
 #pragma unroll
-    for (int e = 0; e < E; ++e)
+    for (int e = 0; e < E; ++e) {
+        if (e >= nvw) break;
         if (e < nv) {
             const float x = __fmaf_rn(val[e], c, d);
             if (!(x < x_lo) && !(x >= x_hi)) {
@@ -1599,6 +1605,7 @@ __device__ __forceinline__ RankOut rank_from_top(const float (&val)[E], int nv, 
                 if (slot < list_cap) s_list[slot] = order_key(val[e]);
             }
         }
+    }
     __syncthreads();
     const unsigned n_list = s_cnt;
     RankOut r;
@@ -1714,6 +1721,7 @@ k_cand_select(const Params p, const float *__restrict__ cand_a, const int32_t *_
     const int l = tid % TG;
     const int64_t base = (int64_t)blockIdx.x * cap + (tid / TG) * capq + l;   // this thread's entries: base + TG * e
     const int nv = mine_cnt > l ? min(E, (mine_cnt - l + TG - 1) / TG) : 0;
+    const int nvw = __reduce_max_sync(0xffffffffu, nv);   // the unrolled per-entry loops stop at the warp's longest thread
     float val[E];
 #pragma unroll
     for (int e = 0; e < E; ++e) val[e] = e < nv ? __ldg(cand_a + base + TG * e) : 0.f;
@@ -1721,7 +1729,7 @@ k_cand_select(const Params p, const float *__restrict__ cand_a, const int32_t *_
     // thread reads back only what it copied itself, so its own wait is all the ordering that takes)
 #pragma unroll
     for (int e = 0; e < E; ++e)
-        if (e < nv)
+        if (e < nv && e < nvw)
             asm volatile("cp.async.ca.shared.global [%0], [%1], 4;\n" ::"r"((uint32_t)__cvta_generic_to_shared(s_pay + e * THREADS + tid)),
                          "l"(cand_j + base + TG * e) : "memory");
     asm volatile("cp.async.commit_group;\n" ::: "memory");
@@ -1748,12 +1756,14 @@ k_cand_select(const Params p, const float *__restrict__ cand_a, const int32_t *_
     }
     // mark the kept keys (the comparison must see denormal scores as they are)
 #pragma unroll
-    for (int e = 0; e < E; ++e)
+    for (int e = 0; e < E; ++e) {
+        if (e >= nvw) break;
         if (e < nv && ge_exact(val[e], tau_f)) {
             const uint32_t j = (uint32_t)s_pay[e * THREADS + tid];
             // (the sweep only writes keys below n_keys; the range test keeps a damaged list from writing outside the bitmap)
             if (j < (uint32_t)n_keys && (jmin == 0u || ~j >= jmin || order_key(val[e]) != r.tau)) atomicOr(&bitmap[j >> 5], 1u << (j & 31u));
         }
+    }
     __syncthreads();
     // Read the bitmap out in ascending key order.  A warp takes a contiguous run of words, its lanes consecutive words
     // (no bank conflicts); the position of a word's first kept key is the warp's base plus a shuffle scan of the counts.
