@@ -46,6 +46,8 @@ from gen import CONFIGS, make_inputs, sample_rows  # noqa: E402
 # not measured by this program.  Each entry names the summary under profiles/ that holds the capture's command.
 NCU_DRAM_TRAFFIC = {
     "cfg2": (268.1e6, "profiles/block_step_cfg2.md"),
+    "cfg4": (15.659e9, "profiles/sparse_prefill_dram_traffic.md"),
+    "cfg4_len32768": (2.750e9, "profiles/sparse_prefill_dram_traffic.md"),
 }
 
 METRIC = "sparse-attn prefill tokens/s (hybrid block step: full-attn+select, sparse layers, decode step)"
