@@ -499,6 +499,12 @@ def bench_native(device, peaks, reps=5):
     t_att = med(lambda: hs2.hs2_full_attn_select(prob, q, k, v, out=O, lse=LSE, want_idx=False, ws=ws))
     osp = torch.empty_like(q)
     t_sp = med(lambda: hs2.hs2_sparse_attn_prefill(prob, inp.q_sparse[0], k, v, idx, out=osp))
+    # the same layer on the e4m3 cache (codes + one fp32 scale per (token, KV head)): 520 B per attended token
+    from gen.workloads import quantize_kv_e4m3
+    k8, ksc = quantize_kv_e4m3(k)
+    v8, vsc = quantize_kv_e4m3(v)
+    prob8 = hs2.Problem.from_tensors(q, k8, wl.k_sel, wl.window)
+    t_sp8 = med(lambda: hs2.hs2_sparse_attn_prefill_fp8kv(prob8, inp.q_sparse[0], k8, v8, ksc, vsc, idx, out=osp))
     gb = gathered_kv_bytes(wl)
     fl = full_attn_flops(wl)
     out["prefill"] = {
@@ -510,8 +516,10 @@ def bench_native(device, peaks, reps=5):
         "sparse_prefill_ms": round(t_sp, 3), "gathered_kv_bytes": gb,
         "sparse_prefill_gbs": round(gb / (t_sp * 1e-3) / 1e9, 1),
         "sparse_prefill_frac_of_hbm_peak": round(gb / (t_sp * 1e-3) / 1e9 / peaks["hbm_gbs"], 4),
+        "fp8_kv_cache": {"sparse_prefill_ms": round(t_sp8, 3), "gathered_kv_bytes": gb / 1024.0 * 520.0,
+                         "frac_of_hbm_peak": round(gb / 1024.0 * 520.0 / (t_sp8 * 1e-3) / 1e9 / peaks["hbm_gbs"], 4)},
         "l2": "the 8 MB cache is L2 resident; Q, idx and O (100 MB) stream"}
-    del inp, q, k, v, O, LSE, idx, osp, ws
+    del inp, q, k, v, O, LSE, idx, osp, ws, k8, v8, ksc, vsc
     torch.cuda.empty_cache()
 
     wl = NATIVE["native_decode"]
@@ -539,6 +547,18 @@ def bench_native(device, peaks, reps=5):
             hs2.hs2_sparse_attn_decode(prob, qss[it % nset], k, v, idxs[it % nset], out=o1, ws=ws_dec)
     us = med(lambda: run(burst), warm=1) / burst * 1e3
     gb = gathered_kv_bytes(wl)
+    k8, ksc = quantize_kv_e4m3(k)
+    v8, vsc = quantize_kv_e4m3(v)
+    prob8 = hs2.Problem.from_tensors(inp.q_full, k8, wl.k_sel, wl.window)
+
+    def run8(n):
+        for it in range(n):
+            hs2.hs2_sparse_attn_decode_fp8kv(prob8, qss[it % nset], k8, v8, ksc, vsc, idxs[it % nset], out=o1)
+    us8 = med(lambda: run8(burst), warm=1) / burst * 1e3
+    out["decode_fp8_kv_cache"] = {
+        "sparse_decode_us_per_step": round(us8, 2), "gathered_kv_bytes": gb / 1024.0 * 520.0,
+        "frac_of_hbm_peak": round(gb / 1024.0 * 520.0 / (us8 * 1e-6) / 1e9 / peaks["hbm_gbs"], 4),
+        "note": "the FP8 entry point takes no scratch, so the keys of a sequence are not split over CTAs"}
     out["decode"] = {
         "workload": "native_decode: B=64, ctx 65536, 64q/1kv heads, D=256, bf16, k=1024, w=128",
         "sparse_decode_us_per_step": round(us, 2), "gathered_kv_bytes": gb,

@@ -175,9 +175,13 @@ hs2_status hs2_sparse_attn_decode_gated(const hs2_problem *p, const void *Q, con
  *                (= bytes), multiples of 16, or 0 for packed.
  *   k_scale, v_scale  in  float [batch, kv_len, n_kv_heads], packed: the cache value is code * scale.
  *   Q, O, LSE, idx, sink as for the bf16 calls; p->dtype describes Q and O and must be HS2_BF16.
- * Covers head_dim 128 with n_q_heads / n_kv_heads <= 8 and 16-byte aligned tensors; anything else returns
- * HS2_ERR_UNSUPPORTED.  V scales up to 255 are supported (probability x scale is carried in an f16 operand).
- * No scratch is needed: decode runs one CTA per (sequence, KV head) whose warps split the attended set.
+ * Covers head_dim 128 and 256 with up to 128 query heads per KV head (the paper's own shape, 64 heads on one KV
+ * head at head_dim 256, included) and 16-byte aligned tensors; anything else returns HS2_ERR_UNSUPPORTED.  At
+ * head_dim 128 with groups of up to 8 (or 16) heads the codes are converted on their way into the mma.sync
+ * operands and V scales up to 255 are supported (probability x scale is carried in an f16 operand); every other
+ * shape runs on the tcgen05 gather kernel, whose gather warps dequantise into bf16 operands.
+ * No scratch is needed: decode runs one CTA per (sequence, KV head); on the tcgen05 kernel the keys of a
+ * sequence are therefore not split over CTAs.
  */
 hs2_status hs2_sparse_attn_prefill_fp8kv(const hs2_problem *p, const void *Q, const void *K8, const void *V8,
                                          const float *k_scale, const float *v_scale, const int32_t *idx,

@@ -491,12 +491,25 @@ static hs2_status sparse_fp8_impl(const hs2_problem *hp, bool decode, const void
     if (s != HS2_OK) return s;
     if (!k_scale || !v_scale) return HS2_ERR_INVALID_ARG;
     if (decode && p.Lq != 1) return HS2_ERR_INVALID_ARG;
-    split_into_subgroups(&p, hp->dtype);
-    if (!sparse_fp8_supported(p, hp->dtype) || !aligned16(Q, K8, V8, O)) return HS2_ERR_UNSUPPORTED;
+    if (!aligned16(Q, K8, V8, O)) return HS2_ERR_UNSUPPORTED;
+    Params pm = p;   // the mma.sync kernel's view: a group of 16 as two sub-groups of 8
+    split_into_subgroups(&pm, hp->dtype);
+    const bool mma = sparse_fp8_supported(pm, hp->dtype);
+    // larger head groups and head_dim 256 (the paper's own shape): the tcgen05 gather kernel, dequantising as it gathers
+    const bool tc5 = !mma && !g_disable_tc5.load(std::memory_order_relaxed) && sparse_tc5_fp8_supported(p, hp->dtype);
+    if (!mma && !tc5) return HS2_ERR_UNSUPPORTED;
     if ((s = check_device()) != HS2_OK) return s;
     cudaStream_t st = (cudaStream_t)cuda_stream;
-    const cudaError_t e = decode ? launch_sparse_fp8_decode(p, Q, K8, V8, k_scale, v_scale, idx, sink, O, LSE, st)
-                                 : launch_sparse_fp8_prefill(p, Q, K8, V8, k_scale, v_scale, idx, sink, O, LSE, st);
+    cudaError_t e;
+    if (mma)
+        e = decode ? launch_sparse_fp8_decode(pm, Q, K8, V8, k_scale, v_scale, idx, sink, O, LSE, st)
+                   : launch_sparse_fp8_prefill(pm, Q, K8, V8, k_scale, v_scale, idx, sink, O, LSE, st);
+    else
+        e = launch_sparse_tc5_fp8(p, Q, K8, V8, k_scale, v_scale, idx, sink, O, LSE, nullptr, 0, st);   // no scratch: keys never split
+    if (e == cudaErrorNotSupported) {
+        (void)cudaGetLastError();
+        return HS2_ERR_UNSUPPORTED;
+    }
     return e == cudaSuccess ? HS2_OK : cuda_fail(e);
 }
 

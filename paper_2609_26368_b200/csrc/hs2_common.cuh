@@ -142,6 +142,11 @@ bool sparse_tc5_supported(const Params &p, hs2_dtype dt);
 size_t sparse_tc5_ws_bytes(const Params &p);   // scratch that lets few queries (decode) split their keys over CTAs
 cudaError_t launch_sparse_tc5(const Params &p, const void *Q, const void *K, const void *V, const int32_t *idx,
                               const float *sink, void *O, float *LSE, void *ws, size_t ws_bytes, cudaStream_t st);
+// the same kernel on an e4m3 cache with per-(token, KV head) scales (bf16 queries; any group up to 128, head_dim 128 or 256)
+bool sparse_tc5_fp8_supported(const Params &p, hs2_dtype dt);
+cudaError_t launch_sparse_tc5_fp8(const Params &p, const void *Q, const void *K8, const void *V8, const float *ksc,
+                                  const float *vsc, const int32_t *idx, const float *sink, void *O, float *LSE, void *ws,
+                                  size_t ws_bytes, cudaStream_t st);
 cudaError_t read_sparse_tc5_error(unsigned *out);
 // FP8 (e4m3 + per-(token, KV head) scale) KV cache, bf16 queries: head_dim 128, group <= 8
 bool sparse_fp8_supported(const Params &p, hs2_dtype dt);

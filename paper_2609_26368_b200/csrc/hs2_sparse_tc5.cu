@@ -61,14 +61,16 @@ __device__ __forceinline__ int producer_ordinal(int w) { return w == 3 ? 0 : w -
 #define HS2_SPTC5_VST3 1    // three V stages at head_dim 256 (needs P in tensor memory)
 #endif
 
-template <int D>
+// F8: the cache holds e4m3 codes with one fp32 scale per (token, KV head); the gather warps dequantise the codes into
+// the bf16 operand layout, the softmax applies the scales (see the kernel).
+template <int D, bool F8 = false>
 struct SpCfg {
     static constexpr int NQ = D / 64;                           // 64-dim slices of an operand tile
     static constexpr int CH = D / 8;                            // 16-byte chunks per row
     static constexpr int KST = D == 256 ? 3 : 2;                // K ring depth
     // V ring depth: with P in tensor memory its 16 KB of shared memory, and most of the alignment slack, buy a third
     // V stage at head_dim 256 (the layout then fills the 227 KB to the byte)
-    static constexpr int VST = (D == 256 && HS2_SPTC5_PTMEM && HS2_SPTC5_VST3) ? 3 : 2;
+    static constexpr int VST = (D == 256 && HS2_SPTC5_PTMEM && HS2_SPTC5_VST3 && !F8) ? 3 : 2;   // (the FP8 variant's register loads need the room less)
     static constexpr uint32_t kSlack = VST == 3 ? 256 : kAlignSlack;
     static constexpr int PW = D == 256 ? HS2_SP_PWARPS : 1;     // warps per gather group (one K group, one V group)
     static constexpr int kThreads = (5 + 2 * PW) * 32;
@@ -85,7 +87,8 @@ struct SpCfg {
     static constexpr uint32_t kOffKey = kOffV + VST * kKVStage;   // int[2 groups][2][64]: key index per slot of a tile
     static constexpr uint32_t kOffMx = kOffKey + 4 * BN * 4;    // float[2 tiles][2 halves][64]: row maxima exchanged
     static constexpr uint32_t kOffL = kOffMx + 4 * 64 * 4;      // float[2 halves][64]: row sums exchanged
-    static constexpr uint32_t kOffBar = kOffL + 2 * 64 * 4;
+    static constexpr uint32_t kOffSc = kOffL + 2 * 64 * 4;      // FP8: float[4 softmax warps][K scale, V scale][32 keys]
+    static constexpr uint32_t kOffBar = kOffSc + (F8 ? 4 * 2 * 32 * 4 : 0);
     static constexpr uint32_t kSmemBytes = kOffBar + kBarBytes + kSlack;
     static constexpr uint32_t kTmem = D <= 128 ? 256 : 512;     // 2 x 64 score columns + D output columns
     static constexpr int kMinBlocks = D <= 128 ? 2 : 1;
@@ -115,6 +118,21 @@ __device__ __forceinline__ void cp_async_arrive(uint32_t bar)
     asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];\n" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;\n" ::: "memory"); }
+// two e4m3 codes (low byte first) -> two bf16 (exact: e4m3 has 3 mantissa bits and a range bf16 covers)
+__device__ __forceinline__ uint32_t e4m3x2_to_bf16x2(uint32_t two_codes)
+{
+    uint32_t h2;
+    asm("cvt.rn.f16x2.e4m3x2 %0, %1;\n" : "=r"(h2) : "h"((unsigned short)two_codes));
+    const float2 f = __half22float2(*reinterpret_cast<const __half2 *>(&h2));
+    return pack_bf16(f.x, f.y);
+}
+__device__ __forceinline__ uint4 ld_codes16(const char *p)
+{
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];\n" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+
 // Slot s of the virtual slot array [idx row | window] of a query at position pos holds a key index or is void (-1).
 // slot_raw starts the fetch (an idx entry is a global load) and slot_fix applies the validity rules to it; callers
 // keep the raw value in a register for a whole tile so that the load's latency is never waited for.
@@ -134,14 +152,15 @@ __device__ __forceinline__ int slot_fix(const Params &p, int j, int pos, int kvl
 // With n_splits > 1 (few queries, e.g. decode) an item is one of n_splits runs of nblk tiles of a query's slot
 // array (slots past the array are void), and it leaves an unnormalised partial (running maximum, sum, fp32
 // accumulator) in part_ml / part_o for the combine kernel below.
-template <int D>
-__global__ void __launch_bounds__(SpCfg<D>::kThreads, SpCfg<D>::kMinBlocks)
-k_sparse_tc5(const __grid_constant__ CUtensorMap tmQ, const Params p, const __nv_bfloat16 *__restrict__ K,
-             const __nv_bfloat16 *__restrict__ V, const int32_t *__restrict__ idx, const float *__restrict__ sink,
+template <int D, bool F8>
+__global__ void __launch_bounds__(SpCfg<D, F8>::kThreads, SpCfg<D, F8>::kMinBlocks)
+k_sparse_tc5(const __grid_constant__ CUtensorMap tmQ, const Params p, const void *__restrict__ K,
+             const void *__restrict__ V, const float *__restrict__ ksc, const float *__restrict__ vsc,
+             const int32_t *__restrict__ idx, const float *__restrict__ sink,
              __nv_bfloat16 *__restrict__ O, float *__restrict__ LSE, int64_t n_items, int n_sub, int n_splits, int nblk,
              float *__restrict__ part_ml, float *__restrict__ part_o)
 {
-    using C = SpCfg<D>;
+    using C = SpCfg<D, F8>;
     constexpr int NQ = C::NQ, CH = C::CH, KST = C::KST;
     constexpr uint32_t kKVStage = C::kKVStage;
     extern __shared__ char smem_raw[];
@@ -232,10 +251,43 @@ k_sparse_tc5(const __grid_constant__ CUtensorMap tmQ, const Params p, const __nv
             // about), one tile ahead so that the idx loads are off the critical path
             const int my_slot = q.slot0 + 32 * half + lane;
             int jn = slot_raw(p, irow, q.pos, my_slot);
+            // FP8 cache: this lane's slot also tells it which key's scales the tile needs.  The key index is kept a tile
+            // further ahead (jn2) so that the scales of tile t+1 can be requested while tile t is worked on; they
+            // reach the other threads of the warp through a warp-private patch of shared memory.
+            float ks_cur = 0.f, vs_cur = 0.f;
+            int jn2 = -1;
+            float *my_sc = reinterpret_cast<float *>(smem + C::kOffSc) + ((warp & 1) + 2 * (warp >> 2)) * 64;
+            if (F8) {
+                const int j0 = slot_fix(p, jn, q.pos, q.kvl, my_slot);
+                if (j0 >= 0) {
+                    const int64_t so = ((int64_t)q.b * p.Lk + j0) * p.Hkv + q.gkv;
+                    ks_cur = __ldg(ksc + so);
+                    vs_cur = __ldg(vsc + so);
+                }
+                if (nblk > 1) jn2 = slot_raw(p, irow, q.pos, my_slot + BN);
+            }
             for (int t = 0; t < nblk; ++t) {
                 const int g = g0 + t, sb = g & 1;
                 const uint32_t valid = __ballot_sync(0xffffffffu, slot_fix(p, jn, q.pos, q.kvl, my_slot + t * BN) >= 0);
-                if (t + 1 < nblk) jn = slot_raw(p, irow, q.pos, my_slot + (t + 1) * BN);
+                if (!F8) {
+                    if (t + 1 < nblk) jn = slot_raw(p, irow, q.pos, my_slot + (t + 1) * BN);
+                } else {
+                    __syncwarp();   // the previous tile's scales have been read by every lane
+                    my_sc[lane] = ks_cur;
+                    my_sc[32 + lane] = vs_cur;
+                    jn = jn2;       // raw entry of tile t+1, fetched a tile ago
+                    ks_cur = 0.f; vs_cur = 0.f;
+                    if (t + 1 < nblk) {
+                        const int j1 = slot_fix(p, jn, q.pos, q.kvl, my_slot + (t + 1) * BN);
+                        if (j1 >= 0) {
+                            const int64_t so = ((int64_t)q.b * p.Lk + j1) * p.Hkv + q.gkv;
+                            ks_cur = __ldg(ksc + so);
+                            vs_cur = __ldg(vsc + so);
+                        }
+                        if (t + 2 < nblk) jn2 = slot_raw(p, irow, q.pos, my_slot + (t + 2) * BN);
+                    }
+                    __syncwarp();
+                }
                 if (!dead && !__all_sync(0xffffffffu, mbar_wait(bar(S_FULL0 + sb), (g >> 1) & 1, abort_flag))) dead = true;
                 float s[32];
                 float mx0 = -INFINITY, mx1 = -INFINITY, mx2 = -INFINITY, mx3 = -INFINITY;
@@ -245,6 +297,13 @@ k_sparse_tc5(const __grid_constant__ CUtensorMap tmQ, const Params p, const __nv
                     tmem_wait_ld();
                     tc_fence_before();
                     mbar_arrive(bar(S_FREE0 + sb));
+                    if (F8) {   // the K scale of a key multiplies its score (void slots: 0 * 0, masked below)
+#pragma unroll
+                        for (int e4 = 0; e4 < 32; e4 += 4) {
+                            const float4 kq = *reinterpret_cast<const float4 *>(my_sc + e4);
+                            s[e4] *= kq.x; s[e4 + 1] *= kq.y; s[e4 + 2] *= kq.z; s[e4 + 3] *= kq.w;
+                        }
+                    }
                     if (valid != 0xffffffffu) {
 #pragma unroll
                         for (int e = 0; e < 32; ++e)
@@ -293,7 +352,12 @@ k_sparse_tc5(const __grid_constant__ CUtensorMap tmQ, const Params p, const __nv
                         const float p0 = exp2f(fmaf(s[e], p.scale_log2, neg_m));       // -inf stays -inf -> 0
                         const float p1 = exp2f(fmaf(s[e + 1], p.scale_log2, neg_m));
                         l0 += p0; l1 += p1;
-                        pk[e >> 1] = pack_bf16(p0, p1);
+                        if (F8) {   // the V scale of a key rides on its probability into P V; the row sum stays unscaled
+                            const float2 vq = *reinterpret_cast<const float2 *>(my_sc + 32 + e);
+                            pk[e >> 1] = pack_bf16(p0 * vq.x, p1 * vq.y);
+                        } else {
+                            pk[e >> 1] = pack_bf16(p0, p1);
+                        }
                     }
                     l += l0 + l1;
 #if HS2_SPTC5_PTMEM
@@ -445,8 +509,11 @@ k_sparse_tc5(const __grid_constant__ CUtensorMap tmQ, const Params p, const __nv
         const int gtid = (po % C::PW) * 32 + lane;
         const int c = gtid % CH, r0 = gtid / CH;
         const uint32_t dst_c = (uint32_t)(c >> 3) * (BN * 128);
-        const int64_t row_bytes = p.ks_t * 2;
-        const __nv_bfloat16 *src_t = is_v ? V : K;
+        const int64_t row_bytes = p.ks_t * (F8 ? 1 : 2);
+        const char *src_t = static_cast<const char *>(is_v ? V : K);
+        // FP8: a thread takes one 16-byte run of codes (16 elements = two bf16 chunks) of every RPI8-th row
+        constexpr int CH8 = D / 16, RPI8 = GT / CH8;
+        const int c8 = gtid % CH8, r8 = gtid / CH8;
         const uint32_t ring0 = sbase + (is_v ? C::kOffV : C::kOffK) + dst_c;
         const int nst = is_v ? C::VST : KST;
         const int bar_full = is_v ? V_FULL0 : K_FULL0, bar_empty = is_v ? V_EMPTY0 : K_EMPTY0;
@@ -469,7 +536,7 @@ k_sparse_tc5(const __grid_constant__ CUtensorMap tmQ, const Params p, const __nv
             const bool more = item + gridDim.x < n_items;
             const Where qn = where(more ? item + gridDim.x : item);
             const int32_t *irow = irow_of(q), *irow_n = irow_of(qn);
-            const char *src0 = reinterpret_cast<const char *>(src_t + q.b * p.ks_b + q.gkv * p.ks_h) + c * 16;
+            const char *src0 = src_t + (q.b * p.ks_b + q.gkv * p.ks_h) * (F8 ? 1 : 2) + (F8 ? c8 : c) * 16;
             if (!is_v && gtid == 0) {   // Q of this item, once the last Q K^T of the previous item has read the buffer
                 if (mbar_wait(bar(Q_EMPTY), (n & 1) ^ 1, abort_flag)) {
                     mbar_expect_tx(bar(Q_FULL), (uint32_t)(NQ * box_heads * 128));
@@ -497,13 +564,45 @@ k_sparse_tc5(const __grid_constant__ CUtensorMap tmQ, const Params p, const __nv
                 for (int u = 0; u < KPT; ++u)
                     if (gtid + u * GT < BN) keys[gtid + u * GT] = j_mine[u];
                 if (!group_all(1 + is_v, GT, ok)) { alive = false; break; }   // also publishes the key indices
-                const uint32_t dst0 = ring0 + st * kKVStage;
+                if (!F8) {
+                    const uint32_t dst0 = ring0 + st * kKVStage;
 #pragma unroll 4
-                for (int r = r0; r < BN; r += RPI) {
-                    const int j = keys[r];
-                    cp_async16(dst0 + r * 128 + (((c & 7) ^ (r & 7)) << 4), src0 + (j >= 0 ? (int64_t)j * row_bytes : 0), j >= 0 ? 16 : 0);
+                    for (int r = r0; r < BN; r += RPI) {
+                        const int j = keys[r];
+                        cp_async16(dst0 + r * 128 + (((c & 7) ^ (r & 7)) << 4), src0 + (j >= 0 ? (int64_t)j * row_bytes : 0), j >= 0 ? 16 : 0);
+                    }
+                    cp_async_arrive(bar(bar_full + st));
+                } else {
+                    // codes -> registers (eight rows in flight per thread) -> bf16 -> the two 16-byte chunks of the
+                    // swizzled operand row; void slots are written as zeros
+                    const uint32_t dst8 = sbase + (is_v ? C::kOffV : C::kOffK) + st * kKVStage + (uint32_t)(c8 >> 2) * (BN * 128);
+                    constexpr int NIT = BN / RPI8, BATCH = NIT < 8 ? NIT : 8;
+#pragma unroll 1
+                    for (int i0 = 0; i0 < NIT; i0 += BATCH) {
+                        uint4 code[BATCH];
+#pragma unroll
+                        for (int u = 0; u < BATCH; ++u) {
+                            const int j = keys[r8 + (i0 + u) * RPI8];
+                            code[u] = j >= 0 ? ld_codes16(src0 + (int64_t)j * row_bytes) : make_uint4(0u, 0u, 0u, 0u);
+                        }
+#pragma unroll
+                        for (int u = 0; u < BATCH; ++u) {
+                            const int r = r8 + (i0 + u) * RPI8;
+                            const uint32_t w[4] = {code[u].x, code[u].y, code[u].z, code[u].w};
+                            uint32_t o[8];
+#pragma unroll
+                            for (int k4 = 0; k4 < 4; ++k4) {
+                                o[2 * k4] = e4m3x2_to_bf16x2(w[k4]);
+                                o[2 * k4 + 1] = e4m3x2_to_bf16x2(w[k4] >> 16);
+                            }
+                            const uint32_t row_dst = dst8 + r * 128;
+                            const int cb = (2 * c8) & 7;   // chunk inside the 64-dim slice: cb and cb + 1
+                            asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};\n" ::"r"(row_dst + ((cb ^ (r & 7)) << 4)), "r"(o[0]), "r"(o[1]), "r"(o[2]), "r"(o[3]) : "memory");
+                            asm volatile("st.shared.v4.b32 [%0], {%1,%2,%3,%4};\n" ::"r"(row_dst + (((cb + 1) ^ (r & 7)) << 4)), "r"(o[4]), "r"(o[5]), "r"(o[6]), "r"(o[7]) : "memory");
+                        }
+                    }
+                    mbar_arrive(bar(bar_full + st));   // (release: this thread's stores are visible to whoever observes the phase)
                 }
-                cp_async_arrive(bar(bar_full + st));
             }
         }
         cp_async_wait_all();   // nothing of this thread stays in flight, also on the abort path
@@ -604,11 +703,12 @@ size_t split_ws_bytes(const Params &p, const SplitPlan &pl)
     return (size_t)pl.queries * pl.n_splits * kSubHeads * (p.D + 2) * sizeof(float);
 }
 
-template <int D>
-cudaError_t launch_sp(const Params &p, const void *Q, const void *K, const void *V, const int32_t *idx, const float *sink,
-                      void *O, float *LSE, void *ws, size_t ws_bytes, bool allow_split, cudaStream_t st)
+template <int D, bool F8>
+cudaError_t launch_sp(const Params &p, const void *Q, const void *K, const void *V, const float *ksc, const float *vsc,
+                      const int32_t *idx, const float *sink, void *O, float *LSE, void *ws, size_t ws_bytes, bool allow_split,
+                      cudaStream_t st)
 {
-    using C = SpCfg<D>;
+    using C = SpCfg<D, F8>;
     CUtensorMap tmQ;
     const int box_heads = p.G < kSubHeads ? p.G : kSubHeads;
     if (!make_tile_map(&tmQ, Q, p.B, p.Lq, p.Hq, p.qs_b, p.qs_t, p.qs_h, 1, box_heads, D)) return cudaErrorNotSupported;
@@ -619,7 +719,7 @@ cudaError_t launch_sp(const Params &p, const void *Q, const void *K, const void 
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= 64) return cudaErrorNotSupported;
     if (!attr_set[dev]) {
-        if ((e = cudaFuncSetAttribute(k_sparse_tc5<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::kSmemBytes)) != cudaSuccess) return e;
+        if ((e = cudaFuncSetAttribute(k_sparse_tc5<D, F8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)C::kSmemBytes)) != cudaSuccess) return e;
         if ((e = cudaDeviceGetAttribute(&n_sm[dev], cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
         attr_set[dev] = true;
     }
@@ -631,9 +731,8 @@ cudaError_t launch_sp(const Params &p, const void *Q, const void *K, const void 
     float *part_o = pl.n_splits > 1 ? part_ml + items * kSubHeads * 2 : nullptr;
     const int64_t resident = (int64_t)n_sm[dev] * C::kMinBlocks;
     const unsigned grid = (unsigned)(items < resident ? items : resident);
-    k_sparse_tc5<D><<<grid, C::kThreads, C::kSmemBytes, st>>>(
-        tmQ, p, (const __nv_bfloat16 *)K, (const __nv_bfloat16 *)V, idx, sink, (__nv_bfloat16 *)O, LSE, items, pl.n_sub,
-        pl.n_splits, pl.nblk, part_ml, part_o);
+    k_sparse_tc5<D, F8><<<grid, C::kThreads, C::kSmemBytes, st>>>(
+        tmQ, p, K, V, ksc, vsc, idx, sink, (__nv_bfloat16 *)O, LSE, items, pl.n_sub, pl.n_splits, pl.nblk, part_ml, part_o);
     count_launch();
     if ((e = cudaGetLastError()) != cudaSuccess || pl.n_splits <= 1) return e;
     const int64_t n_pairs = (int64_t)p.B * p.Lq * p.Hq;
@@ -670,8 +769,28 @@ size_t sparse_tc5_ws_bytes(const Params &p)
 cudaError_t launch_sparse_tc5(const Params &p, const void *Q, const void *K, const void *V, const int32_t *idx,
                               const float *sink, void *O, float *LSE, void *ws, size_t ws_bytes, cudaStream_t st)
 {
-    if (p.D == 128) return launch_sp<128>(p, Q, K, V, idx, sink, O, LSE, ws, ws_bytes, true, st);
-    if (p.D == 256) return launch_sp<256>(p, Q, K, V, idx, sink, O, LSE, ws, ws_bytes, true, st);
+    if (p.D == 128) return launch_sp<128, false>(p, Q, K, V, nullptr, nullptr, idx, sink, O, LSE, ws, ws_bytes, true, st);
+    if (p.D == 256) return launch_sp<256, false>(p, Q, K, V, nullptr, nullptr, idx, sink, O, LSE, ws, ws_bytes, true, st);
+    return cudaErrorNotSupported;
+}
+
+// The same on an e4m3 cache (codes + one fp32 scale per (token, KV head)); bf16 queries and outputs.  The strides of
+// `p` for K and V count codes.  ws as above (null: the keys of a query are never split).
+bool sparse_tc5_fp8_supported(const Params &p, hs2_dtype dt)
+{
+    auto m8 = [](int64_t x) { return x % 8 == 0 && x > 0; };
+    auto m16 = [](int64_t x) { return x % 16 == 0 && x > 0; };
+    if (p.ks_t > 0x7fffffffLL) return false;
+    return dt == HS2_BF16 && (p.D == 256 || p.D == 128) && p.G >= 1 && p.G <= 128 && m8(p.qs_b) && m8(p.qs_t) && m8(p.qs_h) &&
+           m16(p.ks_b) && m16(p.ks_t) && m16(p.ks_h) && m8(p.os_b) && m8(p.os_t) && m8(p.os_h) &&
+           (int64_t)p.B * p.Hkv * p.Lq * 2 * kMaxSplits <= 0x7fffffffLL && p.k + p.w > 0 && tma_available();
+}
+cudaError_t launch_sparse_tc5_fp8(const Params &p, const void *Q, const void *K8, const void *V8, const float *ksc,
+                                  const float *vsc, const int32_t *idx, const float *sink, void *O, float *LSE, void *ws,
+                                  size_t ws_bytes, cudaStream_t st)
+{
+    if (p.D == 128) return launch_sp<128, true>(p, Q, K8, V8, ksc, vsc, idx, sink, O, LSE, ws, ws_bytes, true, st);
+    if (p.D == 256) return launch_sp<256, true>(p, Q, K8, V8, ksc, vsc, idx, sink, O, LSE, ws, ws_bytes, true, st);
     return cudaErrorNotSupported;
 }
 

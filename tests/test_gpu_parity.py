@@ -436,13 +436,60 @@ def test_fp8_kv_cache_sparse_prefill_and_decode():
             ldh = ld[:, :, 0].cpu().numpy()
             assert np.abs(ldh - LSEo[last]).max() <= TOL[wl.torch_dtype]["lse"]
     # shapes the FP8 kernels do not cover are refused, not mis-computed
-    wl = scaled("cfg2", q_len=16, kv_len=64, k_sel=8, window=4, n_q_heads=24, n_kv_heads=1, n_needles=4)
+    wl = scaled("cfg2", q_len=16, kv_len=64, k_sel=8, window=4, n_q_heads=4, n_kv_heads=1, head_dim=64, n_needles=4)
     inp = make_inputs(wl, "cuda")
     k8, ksc = quantize_kv_e4m3(inp.k)
     prob = hs2.Problem.from_tensors(inp.q_full, k8, wl.k_sel, wl.window)
     idx = torch.zeros(1, 1, 16, 8, dtype=torch.int32, device="cuda")
     with pytest.raises(hs2.HS2Error):
         hs2.hs2_sparse_attn_prefill_fp8kv(prob, inp.q_full, k8, k8, ksc, ksc, idx)
+
+
+def test_fp8_kv_cache_on_large_head_groups_and_head_dim_256():
+    """The e4m3 cache at the paper's own attention shape (Table 1: 64 query heads on one KV head, head_dim 256; the cost
+    analysis of Section 4 assumes FP8 storage) and on other shapes of the tensor-core gather kernel, which dequantises
+    while it gathers: prefill every row and the decode step against the oracle on the dequantised cache."""
+    from gen.workloads import quantize_kv_e4m3
+    cases = [
+        dict(q_len=192, kv_len=640, k_sel=128, window=32, n_q_heads=64, n_kv_heads=1, head_dim=256),            # the paper's shape
+        dict(q_len=90, kv_len=500, k_sel=100, window=20, n_q_heads=96, n_kv_heads=2, head_dim=256, batch=2),    # G = 48, two KV heads
+        dict(q_len=150, kv_len=330, k_sel=64, window=64, n_q_heads=24, n_kv_heads=2, head_dim=128),             # G = 12, head_dim 128
+        dict(q_len=64, kv_len=400, k_sel=0, window=130, n_q_heads=128, n_kv_heads=1, head_dim=128),             # window only, two sub-groups
+        dict(q_len=70, kv_len=300, k_sel=37, window=9, n_q_heads=8, n_kv_heads=2, head_dim=256),                # small group at head_dim 256
+    ]
+    for over in cases:
+        wl = scaled("cfg2", n_needles=4, **over)
+        inp = make_inputs(wl)
+        run = BlockRun(inp).run_full()               # indices from the bf16 full layer
+        B, Lk, Hkv, D = inp.k.shape
+        k8, ksc = quantize_kv_e4m3(run.k)
+        v8, vsc = quantize_kv_e4m3(run.v)
+        kv_lens = [Lk - 11 * b for b in range(wl.batch)]
+        kl_t = torch.tensor(kv_lens, dtype=torch.int32, device="cuda")
+        q = run.qs[0]
+        prob = hs2.Problem.from_tensors(q, k8, wl.k_sel, wl.window, kv_lens=kl_t)
+        sink = torch.linspace(-1.0, 1.5, wl.n_q_heads, device="cuda")
+        kd = oracle.dequant_e4m3(k8, ksc)
+        vd = oracle.dequant_e4m3(v8, vsc)
+        idx_rows = run.idx.permute(0, 2, 1, 3).reshape(B * wl.q_len, Hkv, wl.k_sel).cpu().numpy()
+        for sk in (None, sink):
+            out, lse = hs2.hs2_sparse_attn_prefill_fp8kv(prob, q, k8, v8, ksc, vsc, run.idx, sink=sk, want_lse=True)
+            torch.cuda.synchronize()
+            Oo, LSEo, _ = oracle.sparse_attn(q.float().cpu().numpy(), kd, vd, idx_rows, wl.window, kv_lens=kv_lens,
+                                             sink=None if sk is None else sk.cpu().numpy().astype(np.float64))
+            assert_output_close(out.reshape(-1, wl.n_q_heads, D), Oo, wl.torch_dtype, "fp8 sparse O (tensor-core gather)")
+            l = lse.permute(0, 2, 1).reshape(B * wl.q_len, wl.n_q_heads).cpu().numpy()
+            fin = np.isfinite(LSEo)
+            assert np.array_equal(np.isfinite(l), fin) and np.abs(l[fin] - LSEo[fin]).max() <= TOL[wl.torch_dtype]["lse"]
+            q1 = q[:, -1:].contiguous()
+            prob1 = hs2.Problem.from_tensors(q1, k8, wl.k_sel, wl.window, kv_lens=kl_t)
+            od, ld = hs2.hs2_sparse_attn_decode_fp8kv(prob1, q1, k8, v8, ksc, vsc, run.idx[:, :, -1:].contiguous(), sink=sk,
+                                                      want_lse=True)
+            torch.cuda.synchronize()
+            last = [b * wl.q_len + wl.q_len - 1 for b in range(B)]
+            assert_output_close(od[:, 0], Oo[last], wl.torch_dtype, "fp8 sparse decode O (tensor-core gather)")
+            assert np.abs(ld[:, :, 0].cpu().numpy() - LSEo[last]).max() <= TOL[wl.torch_dtype]["lse"]
+    assert hs2.hs2_device_error_flags() == 0
 
 
 def test_fp8_kv_cache_full_layer_decode_step():
