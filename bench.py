@@ -558,7 +558,7 @@ def bench_native(device, peaks, reps=5):
     out["decode_fp8_kv_cache"] = {
         "sparse_decode_us_per_step": round(us8, 2), "gathered_kv_bytes": gb / 1024.0 * 520.0,
         "frac_of_hbm_peak": round(gb / 1024.0 * 520.0 / (us8 * 1e-6) / 1e9 / peaks["hbm_gbs"], 4),
-        "note": "the FP8 entry point takes no scratch, so the keys of a sequence are not split over CTAs"}
+        "note": "the FP8 entry point takes no scratch: the splits of a sequence merge inside a thread-block cluster"}
     out["decode"] = {
         "workload": "native_decode: B=64, ctx 65536, 64q/1kv heads, D=256, bf16, k=1024, w=128",
         "sparse_decode_us_per_step": round(us, 2), "gathered_kv_bytes": gb,

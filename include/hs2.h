@@ -180,8 +180,8 @@ hs2_status hs2_sparse_attn_decode_gated(const hs2_problem *p, const void *Q, con
  * head_dim 128 with groups of up to 8 (or 16) heads the codes are converted on their way into the mma.sync
  * operands and V scales up to 255 are supported (probability x scale is carried in an f16 operand); every other
  * shape runs on the tcgen05 gather kernel, whose gather warps dequantise into bf16 operands.
- * No scratch is needed: decode runs one CTA per (sequence, KV head); on the tcgen05 kernel the keys of a
- * sequence are therefore not split over CTAs.
+ * No scratch is needed: decode runs one CTA per (sequence, KV head) on the mma.sync kernel; on the tcgen05 kernel
+ * the CTAs that split a sequence's keys form a thread-block cluster and merge through distributed shared memory.
  */
 hs2_status hs2_sparse_attn_prefill_fp8kv(const hs2_problem *p, const void *Q, const void *K8, const void *V8,
                                          const float *k_scale, const float *v_scale, const int32_t *idx,

@@ -57,6 +57,9 @@ __device__ __forceinline__ int producer_ordinal(int w) { return w == 3 ? 0 : w -
 #ifndef HS2_SPTC5_PTMEM
 #define HS2_SPTC5_PTMEM 1   // P as a tensor-memory operand of P V (0: through shared memory)
 #endif
+#ifndef HS2_SPTC5_CLUSTER
+#define HS2_SPTC5_CLUSTER 1   // split queries merge inside a thread-block cluster (0: through scratch and a second kernel)
+#endif
 #ifndef HS2_SPTC5_VST3
 #define HS2_SPTC5_VST3 1    // three V stages at head_dim 256 (needs P in tensor memory)
 #endif
@@ -90,6 +93,11 @@ struct SpCfg {
     static constexpr uint32_t kOffSc = kOffL + 2 * 64 * 4;      // FP8: float[4 softmax warps][K scale, V scale][32 keys]
     static constexpr uint32_t kOffBar = kOffSc + (F8 ? 4 * 2 * 32 * 4 : 0);
     static constexpr uint32_t kSmemBytes = kOffBar + kBarBytes + kSlack;
+    // cluster merge: a CTA's unnormalised partial (64 rows of D floats, 16 bytes of padding per row, then maximum and
+    // sum per row) lies in its K/V rings, which are idle by then
+    static constexpr uint32_t kPartPitch = (D + 4) * 4;
+    static constexpr uint32_t kOffPartMl = kOffK + kSubHeads * kPartPitch;
+    static_assert(kOffPartMl + kSubHeads * 8 <= kOffKey, "the partial fits the K and V rings");
     static constexpr uint32_t kTmem = D <= 128 ? 256 : 512;     // 2 x 64 score columns + D output columns
     static constexpr int kMinBlocks = D <= 128 ? 2 : 1;
     static_assert(kOffQ + (NQ - 1) * kQSlice + BM * 128 <= kOffKey && (HS2_SPTC5_PTMEM || kOffP + kPStride + BM * 128 <= kOffKey),
@@ -118,6 +126,31 @@ __device__ __forceinline__ void cp_async_arrive(uint32_t bar)
     asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];\n" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;\n" ::: "memory"); }
+// ---- thread-block clusters: the CTAs that share one query's keys merge their partial results through each other's
+// ---- shared memory (plain loads from a peer's window; no multicast anywhere)
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release.aligned;\n barrier.cluster.wait.acquire.aligned;\n" ::: "memory");
+}
+__device__ __forceinline__ uint32_t peer_smem(uint32_t addr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;\n" : "=r"(r) : "r"(addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ float4 ld_peer4(uint32_t addr)
+{
+    float4 v;
+    asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];\n" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ float2 ld_peer2(uint32_t addr)
+{
+    float2 v;
+    asm volatile("ld.shared::cluster.v2.f32 {%0,%1}, [%2];\n" : "=f"(v.x), "=f"(v.y) : "r"(addr) : "memory");
+    return v;
+}
+
 // two e4m3 codes (low byte first) -> two bf16 (exact: e4m3 has 3 mantissa bits and a range bf16 covers)
 __device__ __forceinline__ uint32_t e4m3x2_to_bf16x2(uint32_t two_codes)
 {
@@ -151,7 +184,10 @@ __device__ __forceinline__ int slot_fix(const Params &p, int j, int pos, int kvl
 // the running tile number g = (items done by this CTA) * nblk + t, which every role computes for itself.
 // With n_splits > 1 (few queries, e.g. decode) an item is one of n_splits runs of nblk tiles of a query's slot
 // array (slots past the array are void), and it leaves an unnormalised partial (running maximum, sum, fp32
-// accumulator) in part_ml / part_o for the combine kernel below.
+// accumulator) in part_ml / part_o for the combine kernel below - or, when part_o is null, the n_splits CTAs of a
+// query are one thread-block cluster (launched so: the grid is exactly the items, the cluster is the query) and merge
+// through distributed shared memory: every CTA parks its partial in its own, by then idle, K/V rings, and after a
+// cluster barrier CTA c reads column slice c of every peer's partial, merges and stores it.  No scratch, one launch.
 template <int D, bool F8>
 __global__ void __launch_bounds__(SpCfg<D, F8>::kThreads, SpCfg<D, F8>::kMinBlocks)
 k_sparse_tc5(const __grid_constant__ CUtensorMap tmQ, const Params p, const void *__restrict__ K,
@@ -393,7 +429,9 @@ k_sparse_tc5(const __grid_constant__ CUtensorMap tmQ, const Params p, const void
             const int64_t o_off = q.b * p.os_b + (int64_t)q.i * p.os_t + h * p.os_h + half * (D / 2);
             __nv_bfloat16 *orow = O + o_off;
             const __nv_bfloat16 *grow = p.gate ? static_cast<const __nv_bfloat16 *>(p.gate) + o_off : nullptr;
-            float *prow = n_splits > 1 ? part_o + (item * kSubHeads + row) * D + half * (D / 2) : nullptr;
+            const bool by_cluster = n_splits > 1 && part_o == nullptr;
+            float *prow = (n_splits > 1 && !by_cluster) ? part_o + (item * kSubHeads + row) * D + half * (D / 2) : nullptr;
+            float *srow = reinterpret_cast<float *>(smem + C::kOffK + row * C::kPartPitch) + half * (D / 2);
 #pragma unroll
             for (int cc = 0; cc < D / 64; ++cc) {
                 float o[32];
@@ -404,9 +442,10 @@ k_sparse_tc5(const __grid_constant__ CUtensorMap tmQ, const Params p, const void
                     mbar_arrive(bar(O_FREE));
                 }
                 if (n_splits > 1) {   // unnormalised partial, every row (rows past the group are never combined)
+                    float *dstp = by_cluster ? srow : prow;
 #pragma unroll
                     for (int q4 = 0; q4 < 8; ++q4)
-                        *reinterpret_cast<float4 *>(prow + cc * 32 + q4 * 4) =
+                        *reinterpret_cast<float4 *>(dstp + cc * 32 + q4 * 4) =
                             any ? make_float4(o[4 * q4], o[4 * q4 + 1], o[4 * q4 + 2], o[4 * q4 + 3]) : make_float4(0.f, 0.f, 0.f, 0.f);
                 } else if (real) {
                     if (grow) {   // sigmoid output gate, before the single rounding to bf16
@@ -434,7 +473,8 @@ k_sparse_tc5(const __grid_constant__ CUtensorMap tmQ, const Params p, const void
                 }
             }
             if (n_splits > 1) {
-                if (half == 0) *reinterpret_cast<float2 *>(part_ml + (item * kSubHeads + row) * 2) = make_float2(any ? m_used : -INFINITY, any ? l : 0.f);
+                float *mlp = by_cluster ? reinterpret_cast<float *>(smem + C::kOffPartMl) + row * 2 : part_ml + (item * kSubHeads + row) * 2;
+                if (half == 0) *reinterpret_cast<float2 *>(mlp) = make_float2(any ? m_used : -INFINITY, any ? l : 0.f);
             } else if (real && half == 0 && LSE) {
                 LSE[((int64_t)q.b * p.Hq + h) * p.Lq + q.i] = any ? (m_used + log2f(l)) * kLn2 : -INFINITY;
             }
@@ -609,6 +649,63 @@ k_sparse_tc5(const __grid_constant__ CUtensorMap tmQ, const Params p, const void
         if (!is_v && gtid == 0 && *abort_flag)
             for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait(bar(Q_FULL), (n - 1) & 1); ++it) {}
     }
+    // ------------------------------------------------ cluster merge (every thread of every CTA of the cluster comes here,
+    // whatever happened before: a CTA that gave up still arrives, its partial is then not valid and the error word says so)
+    if (n_splits > 1 && part_o == nullptr) {
+        __syncwarp();
+        cluster_sync_all();   // all partials are parked
+        if (is_softmax_warp(warp) && (int64_t)blockIdx.x < n_items) {
+            uint32_t my_rank;
+            asm volatile("mov.u32 %0, %%cluster_ctarank;\n" : "=r"(my_rank));
+            const Where q = where(blockIdx.x);
+            const int quad = warp & 1, half = warp >> 2;
+            const int row = 32 * quad + lane;
+            const bool real = row < min(kSubHeads, p.G - kSubHeads * q.sub);
+            const int h = q.gkv * p.G + kSubHeads * q.sub + (real ? row : 0);
+            const int W = D / n_splits, Wt = W / 2;            // this CTA's column slice, this thread's half of it
+            const int col0 = (int)my_rank * W + half * Wt;
+            float m = -INFINITY;
+            for (int r = 0; r < n_splits; ++r)
+                m = fmaxf(m, ld_peer2(peer_smem(sbase + C::kOffPartMl + row * 8, r)).x);
+            float l = 0.f;
+            float4 acc[D / 16];                                // Wt / 4 <= D / 16 entries are used
+#pragma unroll
+            for (int u = 0; u < D / 16; ++u) acc[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int r = 0; r < n_splits; ++r) {
+                const float2 ml = ld_peer2(peer_smem(sbase + C::kOffPartMl + row * 8, r));
+                const float f = ml.x == -INFINITY ? 0.f : exp2f(ml.x - m);
+                l += f * ml.y;
+                const uint32_t src = peer_smem(sbase + C::kOffK + row * C::kPartPitch + col0 * 4, r);
+#pragma unroll
+                for (int u = 0; u < D / 16; ++u)
+                    if (4 * u < Wt) {
+                        const float4 v = ld_peer4(src + u * 16);
+                        acc[u].x += f * v.x; acc[u].y += f * v.y; acc[u].z += f * v.z; acc[u].w += f * v.w;
+                    }
+            }
+            if (real) {
+                const float inv = l > 0.f ? 1.f / l : 0.f;
+                const int64_t o_off = q.b * p.os_b + (int64_t)q.i * p.os_t + h * p.os_h + col0;
+#pragma unroll
+                for (int u = 0; u < D / 16; ++u)
+                    if (4 * u < Wt) {
+                        if (p.gate) {
+                            const uint2 gv = *reinterpret_cast<const uint2 *>(static_cast<const __nv_bfloat16 *>(p.gate) + o_off + u * 4);
+                            const float2 g0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&gv.x));
+                            const float2 g1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&gv.y));
+                            acc[u].x *= gate_of(g0.x); acc[u].y *= gate_of(g0.y); acc[u].z *= gate_of(g1.x); acc[u].w *= gate_of(g1.y);
+                        }
+                        uint2 v;
+                        v.x = pack_bf16(acc[u].x * inv, acc[u].y * inv);
+                        v.y = pack_bf16(acc[u].z * inv, acc[u].w * inv);
+                        *reinterpret_cast<uint2 *>(O + o_off + u * 4) = v;
+                    }
+                if (my_rank == 0 && half == 0 && LSE) LSE[((int64_t)q.b * p.Hq + h) * p.Lq + q.i] = l > 0.f ? (m + log2f(l)) * kLn2 : -INFINITY;
+            }
+        }
+        __syncwarp();
+        cluster_sync_all();   // nobody leaves (and frees its shared memory) while a peer still reads it
+    }
     // ------------------------------------------------ teardown
     __syncwarp();
     tc_fence_before();
@@ -723,14 +820,46 @@ cudaError_t launch_sp(const Params &p, const void *Q, const void *K, const void 
         if ((e = cudaDeviceGetAttribute(&n_sm[dev], cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
         attr_set[dev] = true;
     }
-    SplitPlan pl = plan_splits(p, n_sm[dev] * C::kMinBlocks, allow_split && ws != nullptr);
-    if (split_ws_bytes(p, pl) > ws_bytes) pl = plan_splits(p, 1, false);   // scratch too small for this part: no split
+    // Few queries: the keys of a query are split over CTAs.  The splits of a query are a thread-block cluster that merges
+    // through distributed shared memory (no scratch, one launch) when their number can be a power of two up to 8;
+    // otherwise, with scratch, partials go through global memory and a second kernel combines them.
+    SplitPlan pl = plan_splits(p, n_sm[dev] * C::kMinBlocks, allow_split && (ws != nullptr || HS2_SPTC5_CLUSTER));
+    bool by_cluster = false;
+    if (HS2_SPTC5_CLUSTER && pl.n_splits > 1) {
+        const int tiles = (p.k + p.w + BN - 1) / BN;
+        int c = 8;
+        while (c > pl.n_splits) c >>= 1;          // largest power of two within the planned split and the cluster limit
+        pl.nblk = (tiles + c - 1) / c;            // (runs past the slot array are void and merge as nothing)
+        pl.n_splits = c;
+        by_cluster = true;
+    } else if (split_ws_bytes(p, pl) > ws_bytes) {
+        pl = plan_splits(p, 1, false);            // scratch too small for this part: no split
+    }
     const int64_t items = pl.queries * pl.n_splits;
     if (items <= 0) return cudaSuccess;
-    float *part_ml = reinterpret_cast<float *>(ws);
-    float *part_o = pl.n_splits > 1 ? part_ml + items * kSubHeads * 2 : nullptr;
+    float *part_ml = by_cluster ? nullptr : reinterpret_cast<float *>(ws);
+    float *part_o = (pl.n_splits > 1 && !by_cluster) ? part_ml + items * kSubHeads * 2 : nullptr;
     const int64_t resident = (int64_t)n_sm[dev] * C::kMinBlocks;
-    const unsigned grid = (unsigned)(items < resident ? items : resident);
+    const unsigned grid = (unsigned)(by_cluster ? items : (items < resident ? items : resident));
+    if (by_cluster) {
+        if (items > 0x7fffffffLL) return cudaErrorNotSupported;
+        cudaLaunchConfig_t cfg = {};
+        cfg.gridDim = dim3(grid);
+        cfg.blockDim = dim3(C::kThreads);
+        cfg.dynamicSmemBytes = C::kSmemBytes;
+        cfg.stream = st;
+        cudaLaunchAttribute at[1];
+        at[0].id = cudaLaunchAttributeClusterDimension;
+        at[0].val.clusterDim.x = (unsigned)pl.n_splits;
+        at[0].val.clusterDim.y = 1;
+        at[0].val.clusterDim.z = 1;
+        cfg.attrs = at;
+        cfg.numAttrs = 1;
+        e = cudaLaunchKernelEx(&cfg, k_sparse_tc5<D, F8>, tmQ, p, K, V, ksc, vsc, idx, sink, (__nv_bfloat16 *)O, LSE, items, pl.n_sub,
+                               pl.n_splits, pl.nblk, (float *)nullptr, (float *)nullptr);
+        count_launch();
+        return e != cudaSuccess ? e : cudaGetLastError();
+    }
     k_sparse_tc5<D, F8><<<grid, C::kThreads, C::kSmemBytes, st>>>(
         tmQ, p, K, V, ksc, vsc, idx, sink, (__nv_bfloat16 *)O, LSE, items, pl.n_sub, pl.n_splits, pl.nblk, part_ml, part_o);
     count_launch();
