@@ -362,36 +362,46 @@ k_full_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
 
 // ---------------------------------------------------------------- selection scores on tcgen05
 // a[i][j] = max over the heads h of the group of (scale <q_h(i), k_j> - LSE_h(i))   (Section 3.4)
-// One CTA = TQ = 128/G consecutive queries of one (sequence, KV head) x one chunk of keys.  The MMA
-// computes S^T = K Q^T: 128 keys on M (TMEM lane = key), the TQ x G (query, head) pairs on N = 128,
+// One CTA = TQ = NC/G consecutive queries of one (sequence, KV head) x one chunk of keys.  The MMA
+// computes S^T = K Q^T: 128 keys on M (TMEM lane = key), the TQ x G (query, head) pairs on N = NC columns,
 // so the G heads of a query are adjacent TMEM columns of one lane and their maximum is thread local.
 // Warp 8 feeds K tiles by TMA (2-stage ring), warp 9 issues the MMAs into two accumulator buffers,
 // warps 0-7 (thread = key; warps w and w+4 share the 32 TMEM lanes of quarter w and take 64 columns each)
 // subtract LSE, take the group maximum and write 32 consecutive keys of a strip row per warp instruction.
 // The epilogue is a chain of TMEM loads and short dependent arithmetic: eight warps per CTA hide its latency
 // where four left the tensor pipe waiting for a free accumulator.
+#ifndef HS2_SC_WIDE
+#define HS2_SC_WIDE 1   // 256-column CTAs of the score sweep for head_dim 128 and groups of 8 or 16 (0: 128 columns everywhere)
+#endif
 #ifndef HS2_SC_KCHUNK
 #define HS2_SC_KCHUNK 4096
 #endif
 constexpr int SC_KCHUNK = HS2_SC_KCHUNK;                  // keys per CTA
-constexpr int kScThreads = 320;                           // 8 epilogue warps + TMA warp + MMA warp
-constexpr int kScTmaWarp = 8, kScMmaWarp = 9;
+// NC = 128 columns: 8 epilogue warps, two CTAs per SM (tensor memory: 2 x 2 x 128 columns).  NC = 256 (head_dim 128):
+// 16 epilogue warps, one CTA per SM with all of tensor memory.  An M128 N128 K16 instruction reads 8 KB of operands in
+// the 64 cycles it takes - the whole bandwidth of shared memory, which the TMA writes of the key tiles want too; at
+// N = 256 it is 12 KB per 128 cycles, and a key tile is loaded once per 256 columns instead of once per 128.
 // shared-memory plan of the score sweep for head_dim D: Q and K tiles are D/64 slices of [128 rows][128 B]
-template <int D>
+template <int D, int NC = 128>
 struct ScCfg {
     static constexpr int NQ = D / 64;
-    static constexpr uint32_t kSlice = 128 * 128;                 // one slice: 128 rows of 128 bytes
+    static constexpr int kTmaWarp = NC / 16, kMmaWarp = NC / 16 + 1;   // after the (up to) NC / 16 epilogue warps
+    static constexpr int kThreads = (NC / 16 + 2) * 32;
+    static constexpr uint32_t kTmem = 2 * NC;                     // two accumulator buffers
+    static constexpr uint32_t kSlice = 128 * 128;                 // one slice of a key tile: 128 rows of 128 bytes
+    static constexpr uint32_t kSliceQ = NC * 128;                 // one slice of the (query, head) rows
     static constexpr uint32_t kOffQ = 0;                          // (query, head) rows
-    static constexpr uint32_t kOffK = NQ * kSlice;                // 2 stages of key rows
-    static constexpr uint32_t kOffAug = kOffK + 2 * NQ * kSlice;  // one extra K step: [128][16] bf16 per operand, 32-byte swizzle
-    static constexpr uint32_t kOffNl = kOffAug + 2 * 4096;        // float[128]: -LSE/scale per column
-    static constexpr uint32_t kOffNq = kOffNl + 512;              // int[128]: keys needed per query
-    static constexpr uint32_t kOffRow = kOffNq + 512;             // int64[128]: strip row of each query
-    static constexpr uint32_t kOffTau = kOffRow + 1024;           // uint32[32]: filter threshold per query (filter mode)
+    static constexpr uint32_t kOffK = NQ * kSliceQ;               // 2 stages of key rows
+    static constexpr uint32_t kOffAug = kOffK + 2 * NQ * kSlice;  // one extra K step: [128][16] and [NC][16] bf16, 32-byte swizzle
+    static constexpr uint32_t kOffNl = kOffAug + 4096 + NC * 32;  // float[NC]: -LSE/scale per column
+    static constexpr uint32_t kOffNq = kOffNl + NC * 4;           // int[NC]: keys needed per query
+    static constexpr uint32_t kOffRow = kOffNq + NC * 4;          // int64[NC]: strip row of each query
+    static constexpr uint32_t kOffTau = kOffRow + NC * 8;         // uint32[32]: filter threshold per query (filter mode)
     static constexpr uint32_t kOffCnt = kOffTau + 128;            // int[32]: candidates appended per query (filter mode)
     static constexpr uint32_t kOffBar = kOffCnt + 1024;
     static constexpr uint32_t kSmemBytes = kOffBar + kBarBytes + kAlignSlack;
-    static constexpr int kMinBlocks = D <= 128 ? 2 : 1;
+    static constexpr int kMinBlocks = (D <= 128 && NC == 128) ? 2 : 1;
+    static_assert(kSmemBytes <= 227 * 1024, "fits the shared memory of one SM");
 };
 enum ScBar { SQ_FULL = 0, SK_FULL0, SK_FULL1, SK_EMPTY0, SK_EMPTY1, ACC_FULL0, ACC_FULL1, ACC_FREE0, ACC_FREE1, SC_N_BARS };
 
@@ -420,25 +430,26 @@ __device__ __forceinline__ float key_to_float(uint32_t key)
     return __uint_as_float((key & 0x80000000u) ? (key & 0x7fffffffu) : ~key);
 }
 
-template <int G, int MODE, int D>
-__global__ void __launch_bounds__(kScThreads, ScCfg<D>::kMinBlocks)
+template <int G, int MODE, int D, int NC>
+__global__ void __launch_bounds__(ScCfg<D, NC>::kThreads, ScCfg<D, NC>::kMinBlocks)
 k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmK, const Params p,
              const float *__restrict__ LSE, float *__restrict__ out, int64_t out_stride, int64_t row0, int64_t n_rows,
              int all_visible, int tile_first, int tiles_per_bg, int samp, FilterBuf fb)
 {
-    using S = ScCfg<D>;
+    using S = ScCfg<D, NC>;
+    constexpr int kScTmaWarp = S::kTmaWarp, kScMmaWarp = S::kMmaWarp;
     constexpr int NQ = S::NQ;
     constexpr uint32_t kScOffQ = S::kOffQ, kScOffK = S::kOffK, kScOffNl = S::kOffNl, kScOffNq = S::kOffNq,
                        kScOffRow = S::kOffRow, kScOffTau = S::kOffTau, kScOffCnt = S::kOffCnt, kScOffBar = S::kOffBar,
-                       kStage = NQ * S::kSlice;
-    constexpr int TQ = 128 / G;                    // queries per CTA
+                       kStage = NQ * S::kSlice, kStageQ = NQ * S::kSliceQ;
+    constexpr int TQ = NC / G;                     // queries per CTA
     constexpr int QPC = G <= 32 ? 32 / G : 1;      // queries per 32-column chunk when a group fits a chunk
     constexpr int CPQ = G <= 32 ? 1 : G / 32;      // 32-column chunks per query otherwise
-    constexpr int EW = G <= 64 ? 2 : 1;            // epilogue warps per TMEM lane quarter (a query's columns stay in one warp)
-    constexpr int CPW = 4 / EW;                    // 32-column chunks per epilogue warp
+    constexpr int EW = NC / (G <= 64 ? 64 : G);    // epilogue warps per TMEM lane quarter (a query's columns stay in one warp)
+    constexpr int CPW = NC / 32 / EW;              // 32-column chunks per epilogue warp
     constexpr int TQW = TQ / EW;                   // queries per epilogue warp
     constexpr int kEpiThreads = 128 * EW;
-    static_assert(128 % G == 0 && (G <= 32 || G % 32 == 0), "the group's heads tile the 128 columns");
+    static_assert(NC % G == 0 && (G <= 32 || G % 32 == 0), "the group's heads tile the columns");
     static_assert(MODE != SC_FILTER || TQ <= 32, "filter mode keeps one pass bit per query");
     extern __shared__ char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -490,7 +501,7 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         return;
     }
 
-    if (tid < 128) {   // per-column constants
+    if (tid < NC) {   // per-column constants
         const int t = tid / G, hh = tid % G;
         const int i = iq0 + t;
         const bool ok = i >= c_lo && i < c_hi;
@@ -521,7 +532,7 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             }
         }
     }
-    if (tid < 256)   // the all-ones key operand of the extra step
+    if (tid < 256)   // the all-ones key operand of the extra step (128 rows of 32 bytes)
         reinterpret_cast<uint4 *>(smem + S::kOffAug)[tid] = make_uint4(0x3f803f80u, 0x3f803f80u, 0x3f803f80u, 0x3f803f80u);
     fence_proxy_async();   // the tensor cores read what these threads wrote
     if (tid == 0) {
@@ -534,7 +545,7 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
     }
     if (warp == kScMmaWarp) {
-        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(tmem_slot)), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;\n" ::"r"(smem_u32(tmem_slot)), "r"(S::kTmem) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;\n" ::: "memory");
     }
     tc_fence_before();
@@ -544,9 +555,9 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
 
     if (warp == kScTmaWarp) {
         if (elect_one()) {
-            mbar_expect_tx(bar(SQ_FULL), kStage);
+            mbar_expect_tx(bar(SQ_FULL), kStageQ);
 #pragma unroll
-            for (int sl = 0; sl < NQ; ++sl) tma_load_4d(sbase + kScOffQ + sl * S::kSlice, &tmQ, bar(SQ_FULL), 64 * sl, gkv * p.G, iq0, b);
+            for (int sl = 0; sl < NQ; ++sl) tma_load_4d(sbase + kScOffQ + sl * S::kSliceQ, &tmQ, bar(SQ_FULL), 64 * sl, gkv * p.G, iq0, b);
             int issued = 0;
             for (int t = 0; t < ntile; ++t) {
                 const int st = t & 1;
@@ -566,7 +577,7 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         }
     } else if (warp == kScMmaWarp) {
         if (elect_one()) {
-            constexpr uint32_t id = idesc(128, 128, 0);
+            constexpr uint32_t id = idesc(128, NC, 0);
             bool ok = mbar_wait(bar(SQ_FULL), 0, abort_flag);
             for (int t = 0; ok && t < ntile; ++t) {
                 const int st = t & 1, ph = (t >> 1) & 1;
@@ -576,10 +587,10 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 const uint32_t ka = sbase + kScOffK + st * kStage, qa = sbase + kScOffQ;
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks) {
-                    const uint32_t off = (ks >> 2) * S::kSlice + (ks & 3) * 32;
-                    umma(tmem + st * 128, smem_desc(ka + off, 16, 1024), smem_desc(qa + off, 16, 1024), id, ks > 0);
+                    const uint32_t off = (ks >> 2) * S::kSlice + (ks & 3) * 32, offq = (ks >> 2) * S::kSliceQ + (ks & 3) * 32;
+                    umma(tmem + st * NC, smem_desc(ka + off, 16, 1024), smem_desc(qa + offq, 16, 1024), id, ks > 0);
                 }
-                umma(tmem + st * 128, smem_desc_sw32(sbase + S::kOffAug, 256), smem_desc_sw32(sbase + S::kOffAug + 4096, 256), id, 1);   // - LSE / scale
+                umma(tmem + st * NC, smem_desc_sw32(sbase + S::kOffAug, 256), smem_desc_sw32(sbase + S::kOffAug + 4096, 256), id, 1);   // - LSE / scale
                 umma_commit(bar(SK_EMPTY0 + st));
                 umma_commit(bar(ACC_FULL0 + st));
             }
@@ -629,8 +640,12 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 const int cc = half * CPW + c;   // 32-column chunk of the accumulator
                 float v[32];
                 if (alive) {
-                    tmem_ld32(lane_base + ab * 128 + cc * 32, v);
+                    tmem_ld32(lane_base + ab * NC + cc * 32, v);
                     tmem_wait_ld();
+                    if (c == CPW - 1) {   // the last chunk is in registers: the accumulator goes back to the tensor core
+                        tc_fence_before();   // before the arithmetic on it, not after
+                        mbar_arrive(bar(ACC_FREE0 + ab));
+                    }
                 } else {
 #pragma unroll
                     for (int e = 0; e < 32; ++e) v[e] = 0.f;
@@ -663,10 +678,6 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                         else out[s_row[tq] * out_stride + col] = av;
                     }
                 }
-            }
-            if (alive) {
-                tc_fence_before();
-                mbar_arrive(bar(ACC_FREE0 + ab));
             }
             if (MODE == SC_FILTER) {
                 // Append in no particular order.  This warp is the only writer of its sub-list of every query it owns,
@@ -703,7 +714,7 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     __syncthreads();
     if (warp == kScMmaWarp) {
         tc_fence_after();
-        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(kTmemCols) : "memory");
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;\n" ::"r"(tmem), "r"(S::kTmem) : "memory");
     }
 }
 
@@ -808,7 +819,7 @@ cudaError_t launch_full_attn_tc5(const Params &p, const void *Q, const void *K, 
     return cudaErrorNotSupported;
 }
 
-template <int G, int MODE, int D>
+template <int G, int MODE, int D, int NC = 128>
 cudaError_t launch_sc(const CUtensorMap &tmQ, const CUtensorMap &tmK, const Params &p, const float *LSE, float *out,
                       int64_t out_stride, int64_t row0, int64_t n_rows, bool all_visible, int samp, const FilterBuf &fb,
                       cudaStream_t st)
@@ -818,10 +829,10 @@ cudaError_t launch_sc(const CUtensorMap &tmQ, const CUtensorMap &tmK, const Para
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (!(dev >= 0 && dev < 64 && attr_set[dev])) {
-        if ((e = cudaFuncSetAttribute(k_scores_tc5<G, MODE, D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ScCfg<D>::kSmemBytes)) != cudaSuccess) return e;
+        if ((e = cudaFuncSetAttribute(k_scores_tc5<G, MODE, D, NC>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)ScCfg<D, NC>::kSmemBytes)) != cudaSuccess) return e;
         if (dev >= 0 && dev < 64) attr_set[dev] = true;
     }
-    constexpr int TQ = 128 / G;
+    constexpr int TQ = NC / G;
     const int tiles_per_bg = (p.Lq + TQ - 1) / TQ;
     // only the query tiles that intersect rows [row0, row0 + n_rows) of the flattened (b, g, i) index
     const int64_t last = row0 + n_rows - 1;
@@ -832,7 +843,7 @@ cudaError_t launch_sc(const CUtensorMap &tmQ, const CUtensorMap &tmK, const Para
     const int key_tiles = (p.Lk + 128 * samp - 1) / (128 * samp);
     const unsigned gx = MODE == SC_FILTER ? 1u : (unsigned)((key_tiles + SC_KCHUNK / 128 - 1) / (SC_KCHUNK / 128));
     dim3 grid(gx, (unsigned)gy);
-    k_scores_tc5<G, MODE, D><<<grid, kScThreads, ScCfg<D>::kSmemBytes, st>>>(tmQ, tmK, p, LSE, out, out_stride, row0, n_rows, all_visible ? 1 : 0,
+    k_scores_tc5<G, MODE, D, NC><<<grid, ScCfg<D, NC>::kThreads, ScCfg<D, NC>::kSmemBytes, st>>>(tmQ, tmK, p, LSE, out, out_stride, row0, n_rows, all_visible ? 1 : 0,
                                                                (int)t_first, tiles_per_bg, samp, fb);
     count_launch();
     return cudaGetLastError();
@@ -857,13 +868,22 @@ cudaError_t launch_sc_mode(const Params &p, const void *Q, const void *K, const 
     // with the surplus columns masked (the sampled and filtered sweeps exist for exact sizes only)
     const int gp = padded_group(p.G, p.D);
     if (gp == 0 || (gp != p.G && MODE != SC_STRIP)) return cudaErrorNotSupported;
-    if (!make_map(&tmQ, Q, p.B, p.Lq, p.Hq, p.qs_b, p.qs_t, p.qs_h, 128 / gp, gp, p.D) ||
+    // head_dim 128, groups of 8 and 16: 256 (query, head) columns per CTA (see ScCfg); everything else 128
+    const bool wide = HS2_SC_WIDE && p.D == 128 && (gp == 8 || gp == 16);
+    const int ncol = wide ? 256 : 128;
+    if (!make_map(&tmQ, Q, p.B, p.Lq, p.Hq, p.qs_b, p.qs_t, p.qs_h, ncol / gp, gp, p.D) ||
         !make_map(&tmK, K, p.B, p.Lk, p.Hkv, p.ks_b, p.ks_t, p.ks_h, 128, 1, p.D))
         return cudaErrorNotSupported;
-    if ((n_rows + p.Lq) / (128 / gp) + 2 * (int64_t)p.B * p.Hkv > 65535) return cudaErrorNotSupported;   // grid.y bound
+    if ((n_rows + p.Lq) / (ncol / gp) + 2 * (int64_t)p.B * p.Hkv > 65535) return cudaErrorNotSupported;   // grid.y bound
     constexpr int M2 = MODE == SC_FILTER ? SC_STRIP : MODE;   // groups of 1 or 2 have no filter instantiation
     constexpr int M3 = SC_STRIP;                              // large groups and head_dim 256: strips only
 #define HS2_SC(G_, MODE_, D_) return launch_sc<G_, MODE_, D_>(tmQ, tmK, p, LSE, out, out_stride, row0, n_rows, all_visible, samp, fb, st)
+#if HS2_SC_WIDE
+    if (wide) {
+        if (gp == 8) return launch_sc<8, MODE, 128, 256>(tmQ, tmK, p, LSE, out, out_stride, row0, n_rows, all_visible, samp, fb, st);
+        return launch_sc<16, MODE, 128, 256>(tmQ, tmK, p, LSE, out, out_stride, row0, n_rows, all_visible, samp, fb, st);
+    }
+#endif
     if (p.D == 128) {
         switch (gp) {
             case 1: if (MODE == SC_FILTER) return cudaErrorNotSupported; HS2_SC(1, M2, 128);
