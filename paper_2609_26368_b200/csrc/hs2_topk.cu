@@ -136,22 +136,6 @@ __device__ __forceinline__ unsigned block_excl_scan(unsigned v, unsigned *s_warp
     return __shfl_sync(0xffffffffu, wincl - wsum, warp) + incl - v;
 }
 
-// What the register-resident select works on:
-//   SEL_ROW   a score row indexed by key (the plain entry point and the strip path)
-//   SEL_TAU   the sampled scores of a row: only the value at a given rank is wanted (the filter threshold)
-//   SEL_CAND  the filtered candidates of a row (four sub-lists of cap / 4 slots, each filled from its start, in no
-//             particular order), with their key indices as payload
-enum { SEL_ROW = 0, SEL_TAU = 1, SEL_CAND = 2 };
-
-struct SelArgs {
-    int samp;                 // SEL_TAU: every samp-th key tile was scored
-    int cap;                  // candidate capacity per row (rows with at most cap keys keep every key)
-    uint32_t *tau_key;        // SEL_TAU out: [rows of the block]
-    int *flag;                // SEL_TAU: cleared; SEL_CAND: set when the row has to be redone exactly
-    const int *count;         // SEL_CAND: [rows][4] candidates found per sub-list (-1: the sweep gave up)
-    const int32_t *payload;   // SEL_CAND: [rows][cap] key index of each candidate
-};
-
 // sampled scores of a row with n candidates: every samp-th tile of 128 keys, the last one possibly partial
 __host__ __device__ __forceinline__ int sample_size(int n, int samp)
 {
@@ -183,10 +167,10 @@ __device__ __forceinline__ void topk_cp_async_wait_all()
 __host__ __device__ inline size_t cached_bitmap_bytes(int Lk) { return ((size_t)((Lk + 31) / 32) * 4 + 15) & ~(size_t)15; }
 constexpr size_t cached_stage_bytes(int threads, int e) { return (size_t)threads * (e + 4) * 4; }
 
-template <int THREADS, int E, bool VEC, int MODE>
+template <int THREADS, int E, bool VEC>
 __global__ void __launch_bounds__(THREADS, THREADS > 256 ? 1 : (E > 32 ? 2 : 3))
 k_topk_cached(const Params p, const float *__restrict__ scores, int64_t score_stride, int32_t *__restrict__ idx,
-              int64_t row0, int nc_lo, int nc_hi, SelArgs sa)
+              int64_t row0, int nc_lo, int nc_hi)
 {
     constexpr int WARPS = THREADS / 32;
     __shared__ unsigned hist[256];
@@ -203,88 +187,30 @@ k_topk_cached(const Params p, const float *__restrict__ scores, int64_t score_st
     const int pos = pos_of(p, b, i);
     const int n_keys = max(0, min(pos - p.w + 1, kvl));   // the row's candidates are keys 0..n_keys-1
     const int k_row = min(p.k, n_keys);                   // how many of them are selected
-    // what this launch selects from (nc entries) and how many (take)
-    int nc = n_keys, take = k_row;
-    if (MODE == SEL_TAU) {
-        nc = sample_size(n_keys, sa.samp);
-        take = n_keys > 0 ? min(nc, sample_rank(k_row, n_keys, nc)) : 0;
-    }
-    if (MODE == SEL_CAND) nc = sa.cap;   // one variant serves every row of this launch
+    const int nc = n_keys, take = k_row;
     if (nc <= nc_lo || nc > nc_hi) return;   // this row belongs to another variant's launch
     int32_t *out = idx + row * p.k;
     const float *srow = scores + (int64_t)blockIdx.x * score_stride;
-    const int32_t *prow = MODE == SEL_CAND ? sa.payload + (int64_t)blockIdx.x * sa.cap : nullptr;
 
-    if (MODE == SEL_TAU) {
-        if (tid == 0) sa.flag[blockIdx.x] = 0;
-        if (n_keys <= sa.cap || take <= 0) {   // short row: every key is a candidate
-            if (tid == 0) sa.tau_key[blockIdx.x] = 0u;
-            return;
-        }
-    } else {
-        if (k_row == n_keys) {   // every candidate is kept: no need to look at the scores
-            for (int t = tid; t < p.k; t += THREADS) out[t] = t < n_keys ? t : -1;
-            return;
-        }
+    if (k_row == n_keys) {   // every candidate is kept: no need to look at the scores
+        for (int t = tid; t < p.k; t += THREADS) out[t] = t < n_keys ? t : -1;
+        return;
     }
     const int j0 = tid * E;
-    int nv = min(max(nc - j0, 0), E);   // this thread's slots 0 .. nv-1 hold candidates
-    int ref_slot = 0;                   // a slot that holds a candidate
-    if (MODE == SEL_CAND) {
-        // all cap slots are loaded; sub-list s occupies slots [s capq, s capq + count[s]).  capq is a multiple of E, so
-        // the E slots of a thread lie in one sub-list.
-        const int capq = sa.cap >> 2;
-        int total = 0;
-        bool bad = false;
-#pragma unroll
-        for (int sub = 3; sub >= 0; --sub) {
-            const int c = sa.count[(int64_t)blockIdx.x * 4 + sub];
-            bad |= c < 0 || c > capq;
-            total += c;
-            if (c > 0) ref_slot = sub * capq;
-            if (j0 / capq == sub) nv = min(max(c - (j0 - sub * capq), 0), E);
-        }
-        if (bad || total < k_row) {   // the threshold was off (or the sweep gave up): redo this row exactly
-            if (tid == 0) sa.flag[blockIdx.x] = 1;
-            return;
-        }
-        if (j0 >= sa.cap) nv = 0;
-    }
+    const int nv = min(max(nc - j0, 0), E);   // this thread's slots 0 .. nv-1 hold candidates
     const bool has = nv > 0;   // threads (whole warps, on short rows) past the row's end skip every per-candidate loop
     uint32_t key[E];
-    // The two selects of the filtered path bring the row in through shared memory: consecutive lanes copy consecutive
-    // 16-byte chunks (chunk c to slot c + c / CPT), every thread reads its own chunks at a pitch of CPT + 1 slots.
-    // A thread's own loads would sit E * 4 bytes apart between lanes, 32 cache lines per warp instruction.
-    constexpr int CPT = E / 4;
-    constexpr bool kStaged = HS2_TOPK_STAGE && VEC && MODE != SEL_ROW;
-    extern __shared__ __align__(16) unsigned char s_cached_dyn[];
-    float *s_stage = reinterpret_cast<float *>(s_cached_dyn + (MODE == SEL_CAND ? cached_bitmap_bytes(p.Lk) : 0));
-    auto stage_in = [&](const void *src_row) {   // whole chunks of the first nc 4-byte entries of a row
-        const float *src = static_cast<const float *>(src_row);
-#pragma unroll
-        for (int it = 0; it < CPT; ++it) {
-            const int c = it * THREADS + tid;
-            if (4 * c + 4 <= nc) topk_cp_async16(s_stage + (c + c / CPT) * 4, src + 4 * c);
-        }
-        topk_cp_async_wait_all();
-        __syncthreads();
-    };
-    if (kStaged) stage_in(srow);
     // which bits differ anywhere in the row: OR of (key ^ key of candidate 0), one logic op per candidate
-    const uint32_t ref = order_key(__ldg(srow + ref_slot));
+    const uint32_t ref = order_key(__ldg(srow));
     unsigned diff = 0u;
     if (has)
 #pragma unroll
     for (int e4 = 0; e4 < E; e4 += 4) {
         if (VEC && j0 + e4 + 4 <= nc) {
-            const float4 v = kStaged ? *reinterpret_cast<const float4 *>(s_stage + ((CPT + 1) * tid + (e4 >> 2)) * 4)
-                                     : __ldg(reinterpret_cast<const float4 *>(srow + j0 + e4));
+            const float4 v = __ldg(reinterpret_cast<const float4 *>(srow + j0 + e4));
             key[e4] = order_key(v.x); key[e4 + 1] = order_key(v.y); key[e4 + 2] = order_key(v.z); key[e4 + 3] = order_key(v.w);
 #pragma unroll
-            for (int e = e4; e < e4 + 4; ++e) {
-                if (MODE == SEL_CAND && e >= nv) key[e] = 0u;   // a slot past the sub-list's fill
-                else diff |= key[e] ^ ref;
-            }
+            for (int e = e4; e < e4 + 4; ++e) diff |= key[e] ^ ref;
         } else {
 #pragma unroll
             for (int e = e4; e < e4 + 4; ++e) {
@@ -382,71 +308,6 @@ k_topk_cached(const Params p, const float *__restrict__ scores, int64_t score_st
     }
     const uint32_t tau = diff == 0u ? ref : prefix;                  // key of the take-th largest candidate
     const unsigned need_eq = need;                                   // equal keys kept, lowest indices first
-    if (MODE == SEL_TAU) {
-        if (tid == 0) sa.tau_key[blockIdx.x] = tau;
-        return;
-    }
-    if (MODE == SEL_CAND) {
-        // The candidates come in no particular order.  Kept: score above tau, or equal to tau and among the need_eq
-        // lowest key indices of the equal ones.  The kept keys are marked in a bitmap over the row's keys, which is
-        // then read out in ascending order.
-        unsigned *bitmap = reinterpret_cast<unsigned *>(s_cached_dyn);
-        // the key indices of the candidates come in the same way (every thread has its scores in registers by now)
-        __syncthreads();
-        if (kStaged) stage_in(prow);
-        auto pay = [&](int e) -> int32_t {
-            if (kStaged && j0 + (e & ~3) + 4 <= nc) return reinterpret_cast<const int32_t *>(s_stage)[((CPT + 1) * tid + (e >> 2)) * 4 + (e & 3)];
-            return prow[j0 + e];
-        };
-        unsigned my_eq = 0;
-#pragma unroll
-        for (int e = 0; e < E; ++e) my_eq += (e < nv) && key[e] == tau;
-        unsigned total_eq;
-        block_excl_scan<WARPS>(my_eq, s_warp, lane, warp, &total_eq);
-        uint32_t jmin = 0u;   // tied candidates are kept when ~index >= jmin
-        if (total_eq > need_eq) {
-            if (total_eq > kListCap) {   // thousands of exact ties at the threshold: leave the row to the exact redo
-                if (tid == 0) sa.flag[blockIdx.x] = 1;
-                return;
-            }
-            if (tid == 0) s_cnt = 0;
-            __syncthreads();
-#pragma unroll
-            for (int e = 0; e < E; ++e)
-                if (e < nv && key[e] == tau) s_list[atomicAdd(&s_cnt, 1u)] = ~(uint32_t)pay(e);
-            __syncthreads();
-            jmin = select_on_list<THREADS>(s_list, total_eq, need_eq, hist, &s_prefix, &s_need, tid, lane, warp);
-        }
-        const int nwords = (n_keys + 31) >> 5;
-        for (int wd = tid; wd < nwords; wd += THREADS) bitmap[wd] = 0u;
-        __syncthreads();
-#pragma unroll
-        for (int e = 0; e < E; ++e) {
-            if (e >= nv) continue;
-            if (key[e] > tau || key[e] == tau) {
-                const uint32_t j = (uint32_t)pay(e);
-                // (the sweep only writes keys below n_keys; the range test keeps a damaged list from writing outside the bitmap)
-                if (j < (uint32_t)n_keys && (key[e] > tau || ~j >= jmin)) atomicOr(&bitmap[j >> 5], 1u << (j & 31u));
-            }
-        }
-        __syncthreads();
-        const int per = (nwords + THREADS - 1) / THREADS;
-        const int w0 = tid * per, w1 = min(nwords, w0 + per);
-        unsigned mine = 0;
-        for (int wd = w0; wd < w1; ++wd) mine += __popc(bitmap[wd]);
-        unsigned total_sel;
-        unsigned posn = block_excl_scan<WARPS>(mine, s_warp, lane, warp, &total_sel);
-        for (int wd = w0; wd < w1; ++wd) {
-            unsigned bits = bitmap[wd];
-            while (bits) {
-                const int bpos = __ffs(bits) - 1;
-                bits &= bits - 1;
-                out[posn++] = wd * 32 + bpos;
-            }
-        }
-        for (int t = take + tid; t < p.k; t += THREADS) out[t] = -1;
-        return;
-    }
 
     // ---- ordered compaction with one block scan
     // which of this thread's candidates are above tau / equal to it (key 0, past the end, is below tau)
@@ -1231,11 +1092,11 @@ cudaError_t launch_class(int c, const Params &p, const float *scores, int64_t sc
     }
 #endif
     switch (c) {
-        case 0: k_topk_cached<64, 32, VEC, SEL_ROW><<<n, 64, stage, st>>>(p, scores, score_stride, idx, row0, lo, hi, SelArgs{}); break;
-        case 1: k_topk_cached<128, 32, VEC, SEL_ROW><<<n, 128, stage, st>>>(p, scores, score_stride, idx, row0, lo, hi, SelArgs{}); break;
-        case 2: k_topk_cached<256, 32, VEC, SEL_ROW><<<n, 256, stage, st>>>(p, scores, score_stride, idx, row0, lo, hi, SelArgs{}); break;
-        case 3: k_topk_cached<256, 64, VEC, SEL_ROW><<<n, 256, stage, st>>>(p, scores, score_stride, idx, row0, lo, hi, SelArgs{}); break;
-        case 4: k_topk_cached<512, 64, VEC, SEL_ROW><<<n, 512, stage, st>>>(p, scores, score_stride, idx, row0, lo, hi, SelArgs{}); break;
+        case 0: k_topk_cached<64, 32, VEC><<<n, 64, stage, st>>>(p, scores, score_stride, idx, row0, lo, hi); break;
+        case 1: k_topk_cached<128, 32, VEC><<<n, 128, stage, st>>>(p, scores, score_stride, idx, row0, lo, hi); break;
+        case 2: k_topk_cached<256, 32, VEC><<<n, 256, stage, st>>>(p, scores, score_stride, idx, row0, lo, hi); break;
+        case 3: k_topk_cached<256, 64, VEC><<<n, 256, stage, st>>>(p, scores, score_stride, idx, row0, lo, hi); break;
+        case 4: k_topk_cached<512, 64, VEC><<<n, 512, stage, st>>>(p, scores, score_stride, idx, row0, lo, hi); break;
         case 5: case 6: case 7: {   // (dynamic shared memory: the staged slice of the row)
             const size_t smem = (HS2_TOPK_STAGE && VEC) ? cached_stage_bytes(512, 64) : 0;
             auto go = [&](auto kern, unsigned cl) -> cudaError_t {
