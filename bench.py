@@ -38,6 +38,12 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 if ROOT not in sys.path:
     sys.path.insert(0, ROOT)
 
+# torch.distributed.run sets OMP_NUM_THREADS=1 for its ranks; the CPU-oracle arm runs on rank 0 alone and is meant to use
+# the machine's host cores, so it takes them back before any OpenMP runtime reads the variable
+if "reference" in sys.argv and os.environ.get("RANK", "0") == "0" and os.environ.get("OMP_NUM_THREADS") == "1" \
+        and "TORCHELASTIC_RUN_ID" in os.environ:
+    os.environ["OMP_NUM_THREADS"] = str(os.cpu_count() or 1)
+
 import torch  # noqa: E402
 
 from gen import CONFIGS, make_inputs, sample_rows  # noqa: E402
