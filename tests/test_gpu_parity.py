@@ -207,6 +207,32 @@ def _filtered_equals_full_rows():
         assert hs2.hs2_device_error_flags() == 0
 
 
+def test_filtered_selection_breaks_ties_at_the_threshold_by_key_index():
+    """Every key row appears twice (keys 2j and 2j+1 are equal), so every score appears twice and about half of the rows
+    have a tied pair straddling the k-th place: the candidate select must keep the lower key of the pair, as the
+    selection from complete score rows and the oracle's ordering do."""
+    old = hs2.hs2_set_filter_min_keys(1)
+    try:
+        wl = scaled("cfg2", q_len=1024, kv_len=4096, k_sel=255, window=32, n_needles=4)
+        inp = make_inputs(wl)
+        inp.k[:, 1::2] = inp.k[:, 0::2]
+        a = BlockRun(inp).run_full(want_scores=True)           # complete rows, the same tensor-core scores
+        b = BlockRun(inp).run_full(want_scores=False)          # sampled threshold, candidate lists, candidate select
+        assert torch.equal(a.idx, b.idx)
+        a.check_idx_bitexact_on_gpu_scores(rows=[(0, i) for i in range(0, wl.q_len, 37)])
+        # the case really has straddling pairs: rows whose last kept key (by score) has an unkept twin
+        sc = a.scores[0, 0]                                    # [Lq, Lk]
+        kept = torch.zeros_like(sc, dtype=torch.bool)
+        rows = torch.arange(wl.q_len, device="cuda").unsqueeze(1).expand(-1, wl.k_sel)
+        kept[rows, a.idx[0, 0].long()] = True
+        twins = kept[:, 0::2] != kept[:, 1::2]
+        assert int(twins.any(dim=1).sum()) > wl.q_len // 8
+        assert bool((kept[:, 0::2] | ~kept[:, 1::2]).all())    # never the higher key of a pair without the lower one
+        assert hs2.hs2_device_error_flags() == 0
+    finally:
+        hs2.hs2_set_filter_min_keys(old)
+
+
 def test_filtered_selection_redoes_rows_whose_sample_misleads():
     """Scores that depend on the key tile's phase defeat a tile-strided sample: the threshold comes out too
     high (lists shorter than k) or too low (lists overflow).  Those rows must be redone exactly."""
