@@ -7,6 +7,7 @@ import torch
 
 import paper_2609_26368_b200 as hs2
 from gen import CONFIGS, make_inputs, sample_rows
+from gen.workloads import NATIVE
 from parity import BlockRun
 
 pytestmark = pytest.mark.gpu
@@ -30,7 +31,7 @@ def _index_properties(run, stride=1):
 
 
 def _run_block(name, n_rows, layers=None):
-    wl = CONFIGS[name]
+    wl = CONFIGS[name] if name in CONFIGS else NATIVE[name]
     inp = make_inputs(wl, "cuda")
     run = BlockRun(inp).run_full()
     rows = [(b, i) for b in range(wl.batch) for i in sample_rows(wl, n_rows)]
@@ -58,3 +59,14 @@ def test_cfg4_full_size_sampled():
 
 def test_cfg5_decode_full_size_every_sequence():
     _run_block("cfg5", 1)
+
+
+def test_native8k_full_size_sampled():
+    """The paper's own attention shape (64 query heads on one KV head, head_dim 256) as bench.py times it: every kernel
+    of the block on tcgen05."""
+    _run_block("native8k", 64)
+
+
+def test_native_decode_full_size_every_sequence():
+    """Decode at the paper's shape, batch 64 on a 64K-token cache: the splits of a sequence merge inside a cluster."""
+    _run_block("native_decode", 1, layers=[0])
