@@ -561,8 +561,11 @@ def bench_native(device, peaks, reps=5):
         for it in range(n):
             hs2.hs2_sparse_attn_decode_fp8kv(prob8, qss[it % nset], k8, v8, ksc, vsc, idxs[it % nset], out=o1)
     us8 = med(lambda: run8(burst), warm=1) / burst * 1e3
+    ws8 = torch.empty(max(256, hs2.hs2_workspace_bytes(prob8, binding.HS2_OP_FULL_ATTN_SELECT_FP8KV)), dtype=torch.uint8, device=device)
+    t_full8 = med(lambda: hs2.hs2_full_attn_select_fp8kv(prob8, qfs[0], k8, v8, ksc, vsc, ws=ws8), n=4, warm=1)
     out["decode_fp8_kv_cache"] = {
         "sparse_decode_us_per_step": round(us8, 2), "gathered_kv_bytes": gb / 1024.0 * 520.0,
+        "full_attn_select_decode_ms": round(t_full8, 3),
         "frac_of_hbm_peak": round(gb / 1024.0 * 520.0 / (us8 * 1e-6) / 1e9 / peaks["hbm_gbs"], 4),
         "note": "the FP8 entry point takes no scratch: the splits of a sequence merge inside a thread-block cluster"}
     out["decode"] = {

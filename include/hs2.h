@@ -199,9 +199,10 @@ hs2_status hs2_sparse_attn_decode_fp8kv(const hs2_problem *p, const void *Q, con
  *   ws: with idx, at least hs2_workspace_bytes(p, HS2_OP_FULL_ATTN_SELECT_FP8KV) bytes, 256-byte aligned (the
  *   dequantised q.k products of every head and key, 4 bytes each, and one score row per (sequence, KV head));
  *   HS2_ERR_WORKSPACE_TOO_SMALL otherwise.  Without idx no scratch is needed.
- *   Covers q_len == 1, head_dim 128, groups of at most 8 query heads, 16-byte aligned tensors, products that fit
- *   2 GiB; anything else returns HS2_ERR_UNSUPPORTED and launches nothing.  (A prefill-shaped full layer attends to
- *   the bf16 K and V it has just produced, so there is no FP8 variant of it.)
+ *   Covers q_len == 1, 16-byte aligned tensors, head_dim 128 or 256 with up to 128 query heads per KV head (at
+ *   head_dim 128 and groups of at most 8 the cache is swept once and the products kept, which must fit 2 GiB; other
+ *   shapes sweep K a second time for the scores); anything else returns HS2_ERR_UNSUPPORTED and launches nothing.
+ *   (A prefill-shaped full layer attends to the bf16 K and V it has just produced, so there is no FP8 variant of it.)
  */
 hs2_status hs2_full_attn_select_fp8kv(const hs2_problem *p, const void *Q, const void *K8, const void *V8,
                                       const float *k_scale, const float *v_scale, void *O, float *LSE, int32_t *idx,

@@ -248,6 +248,8 @@ size_t hs2_workspace_bytes(const hs2_problem *hp, hs2_op op)
             {
                 Params pd = p;
                 pd.k = 0; pd.w = p.Lk;
+                if (!sparse_fp8_supported(pd, hp->dtype))   // large groups / head_dim 256: one score row per (sequence, KV head)
+                    return sparse_tc5_fp8_supported(pd, hp->dtype) ? align_up((size_t)p.B * p.Hkv * strip_row_bytes(p), 256) : 0;
                 const DecodeFusedPlan fu = decode_fused_plan(pd, 0);
                 return fu.ok ? fu.total : 0;
             }
@@ -540,8 +542,30 @@ hs2_status hs2_full_attn_select_fp8kv(const hs2_problem *hp, const void *Q, cons
     if (p.Lq != 1) return HS2_ERR_UNSUPPORTED;
     Params pd = p;   // a sweep over the whole cache: the gather kernel with no index list and a window that covers the context
     pd.k = 0; pd.w = p.Lk;
-    if (!sparse_fp8_supported(pd, hp->dtype) || !aligned16(Q, K8, V8, O) || (int64_t)p.B * p.Hkv > 65535) return HS2_ERR_UNSUPPORTED;
+    if (!aligned16(Q, K8, V8, O) || (int64_t)p.B * p.Hkv > 65535) return HS2_ERR_UNSUPPORTED;
     const bool want_sel = idx != nullptr && p.k > 0;
+    if (!sparse_fp8_supported(pd, hp->dtype)) {
+        // Larger head groups and head_dim 256 (the paper's own shape): the attention sweeps the cache on the tcgen05
+        // gather kernel (the CTAs that split a sequence merge inside a cluster, no scratch), a second pass over the K
+        // codes gives the selection scores once the LSE is known, the top-k runs on those rows.
+        if (g_disable_tc5.load(std::memory_order_relaxed) || !sparse_tc5_fp8_supported(pd, hp->dtype) || p.blk > 1) return HS2_ERR_UNSUPPORTED;
+        const size_t need = want_sel ? align_up((size_t)p.B * p.Hkv * strip_row_bytes(p), 256) : 0;
+        if (!ws_ok(ws, ws_bytes, need)) return HS2_ERR_WORKSPACE_TOO_SMALL;
+        if ((s = check_device()) != HS2_OK) return s;
+        cudaStream_t st2 = (cudaStream_t)cuda_stream;
+        cudaError_t e2 = launch_sparse_tc5_fp8(pd, Q, K8, V8, k_scale, v_scale, nullptr, nullptr, O, LSE, nullptr, 0, st2);
+        if (e2 == cudaErrorNotSupported) {
+            (void)cudaGetLastError();
+            return HS2_ERR_UNSUPPORTED;
+        }
+        if (e2 != cudaSuccess) return cuda_fail(e2);
+        if (!want_sel) return HS2_OK;
+        float *strip2 = static_cast<float *>(ws);
+        const int64_t stride2 = (int64_t)(strip_row_bytes(p) / sizeof(float));
+        if ((e2 = launch_scores_fp8_decode(p, Q, K8, k_scale, LSE, strip2, stride2, st2)) != cudaSuccess) return cuda_fail(e2);
+        if ((e2 = launch_select(p, strip2, stride2, idx, 0, select_rows(p), st2)) != cudaSuccess) return cuda_fail(e2);
+        return HS2_OK;
+    }
     const DecodeFusedPlan fu = decode_fused_plan(pd, 0);
     if (want_sel) {
         if (!fu.ok) return HS2_ERR_UNSUPPORTED;   // the raw products of this problem would not fit the scratch cap

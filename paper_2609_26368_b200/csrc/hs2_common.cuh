@@ -156,6 +156,9 @@ cudaError_t launch_sparse_fp8_prefill(const Params &p, const void *Q, const void
 cudaError_t launch_sparse_fp8_decode(const Params &p, const void *Q, const void *K, const void *V, const float *ksc,
                                      const float *vsc, const int32_t *idx, const float *sink, void *O, float *LSE,
                                      cudaStream_t st, float *raw = nullptr);
+// selection scores of a one-query layer on the FP8 cache (any group up to 128, head_dim 128 or 256), rows = (b, g)
+cudaError_t launch_scores_fp8_decode(const Params &p, const void *Q, const void *K8, const float *ksc, const float *LSE,
+                                     float *out, int64_t out_stride, cudaStream_t st);
 // KV-cache producer: C[T, N] = H[T, dm] W[N, dm]^T, bf16 out or e4m3 codes + scale per (token, 128 columns)
 bool kv_project_supported(int64_t T, int N, int dm, int64_t ldh, int64_t ldw, int64_t ldc, bool fp8);
 cudaError_t launch_kv_project(int64_t T, int N, int dm, const void *H, int64_t ldh, const void *W, int64_t ldw, void *C,

@@ -570,6 +570,121 @@ cudaError_t set_smem(Kern kern, int bytes, bool *done)
 }  // namespace
 
 // bf16 queries, e4m3 cache with a scale per (token, KV head): head_dim 128, group <= 8; strides in bytes for the cache
+// ---------------------------------------------------------------- selection scores of a one-query layer on the FP8 cache
+// a[j] = max over the heads h of the group of (scale * k_scale[j] * <q_h, code_j> - LSE_h)   (Section 3.4), for one
+// query per sequence, any group of up to 128 heads, head_dim 128 or 256: the second pass of the full layer's decode step
+// on shapes whose first pass (attention, LSE) runs on the tcgen05 gather kernel.  Memory-bound: every key's codes are
+// read once.  A warp takes 16 consecutive keys against all heads: the key codes go from global memory straight into
+// MMA A fragments (a thread reads 16 consecutive bytes of a row: four consecutive dims for each of four k-steps, a
+// permutation of the contraction index that the query fragments in shared memory follow), cvt e4m3x2 -> f16x2 is exact.
+namespace {
+
+constexpr int kScF8Warps = 8;
+
+template <int D>
+__global__ void __launch_bounds__(kScF8Warps * 32)
+k_scores_fp8_decode(const Params p, const __nv_bfloat16 *__restrict__ Q, const uint8_t *__restrict__ K,
+                    const float *__restrict__ ksc, const float *__restrict__ LSE, float *__restrict__ out, int64_t out_stride)
+{
+    extern __shared__ __align__(16) unsigned char s_raw[];
+    const int GP = (p.G + 7) & ~7, NT = GP / 8;                 // heads padded to whole n-tiles of 8
+    uint2 *s_q = reinterpret_cast<uint2 *>(s_raw);              // [NT][D / 16 k-steps][32 lanes]: the B fragments
+    float *s_lse = reinterpret_cast<float *>(s_raw + (size_t)NT * (D / 16) * 32 * 8);   // [GP], natural log; +inf past the group
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int bg = blockIdx.y, gkv = bg % p.Hkv, b = bg / p.Hkv;
+    const int g = lane >> 2, t = lane & 3;
+    const int n_keys = max(0, min(pos_of(p, b, 0) - p.w + 1, kvlen_of(p, b)));
+    // query fragments: n-tile nt, k-step ks = 4 c + i (c: 64-dim slice, i: word of the 16-byte run), lane (g, t):
+    // b0 = dims (64 c + 16 t + 4 i, + 1), b1 = (+ 2, + 3) of head 8 nt + g
+    for (int e = tid; e < NT * (D / 16) * 32; e += blockDim.x) {
+        const int ln = e & 31, ks = (e >> 5) % (D / 16), nt = e / (32 * (D / 16));
+        const int hg = ln >> 2, ht = ln & 3, c = ks >> 2, i = ks & 3;
+        const int head = 8 * nt + hg;
+        uint2 frag = make_uint2(0u, 0u);
+        if (head < p.G) {
+            const __nv_bfloat16 *q = Q + b * p.qs_b + (gkv * p.G + head) * p.qs_h + 64 * c + 16 * ht + 4 * i;
+            const uint2 rawq = __ldg(reinterpret_cast<const uint2 *>(q));
+            const float2 lo = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&rawq.x));
+            const float2 hi = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&rawq.y));
+            frag = make_uint2(pack_f16(lo.x, lo.y), pack_f16(hi.x, hi.y));
+        }
+        s_q[e] = frag;
+    }
+    for (int h = tid; h < GP; h += blockDim.x) s_lse[h] = h < p.G ? LSE[((int64_t)b * p.Hq + gkv * p.G + h) * p.Lq] : INFINITY;
+    __syncthreads();
+    float *orow = out + (int64_t)bg * out_stride;
+    const uint8_t *kbase = K + b * p.ks_b + gkv * p.ks_h;
+    const int64_t rs = p.ks_t;                                   // bytes between consecutive tokens
+    const float *ksb = ksc + ((int64_t)b * p.Lk) * p.Hkv + gkv;
+    for (int j0 = (blockIdx.x * kScF8Warps + warp) * 16; j0 < n_keys; j0 += gridDim.x * kScF8Warps * 16) {
+        const int ja = j0 + g, jb = j0 + g + 8;                  // this thread's two keys
+        const bool va = ja < n_keys, vb = jb < n_keys;
+        uint4 ca[D / 64], cb[D / 64];
+#pragma unroll
+        for (int c = 0; c < D / 64; ++c) {
+            ca[c] = va ? __ldg(reinterpret_cast<const uint4 *>(kbase + (int64_t)ja * rs + 64 * c + 16 * t)) : make_uint4(0u, 0u, 0u, 0u);
+            cb[c] = vb ? __ldg(reinterpret_cast<const uint4 *>(kbase + (int64_t)jb * rs + 64 * c + 16 * t)) : make_uint4(0u, 0u, 0u, 0u);
+        }
+        const float fa = va ? __ldg(ksb + (int64_t)ja * p.Hkv) * p.scale : 0.f;
+        const float fb = vb ? __ldg(ksb + (int64_t)jb * p.Hkv) * p.scale : 0.f;
+        float best_a = -INFINITY, best_b = -INFINITY;
+        for (int nt = 0; nt < NT; ++nt) {
+            float acc[4] = {0.f, 0.f, 0.f, 0.f};
+            const uint2 *qf = s_q + (size_t)nt * (D / 16) * 32 + lane;
+#pragma unroll
+            for (int c = 0; c < D / 64; ++c) {
+                const uint32_t wa[4] = {ca[c].x, ca[c].y, ca[c].z, ca[c].w}, wb[4] = {cb[c].x, cb[c].y, cb[c].z, cb[c].w};
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const uint2 bq = qf[(4 * c + i) * 32];
+                    mma_f16(acc, cvt_e4m3x2(wa[i]), cvt_e4m3x2(wb[i]), cvt_e4m3x2(wa[i] >> 16), cvt_e4m3x2(wb[i] >> 16), bq.x, bq.y);
+                }
+            }
+            // acc[0], acc[1]: key ja, heads 8 nt + 2 t, + 1; acc[2], acc[3]: key jb
+            const float l0 = s_lse[8 * nt + 2 * t], l1 = s_lse[8 * nt + 2 * t + 1];
+            best_a = fmaxf(best_a, fmaxf(acc[0] * fa - l0, acc[1] * fa - l1));
+            best_b = fmaxf(best_b, fmaxf(acc[2] * fb - l0, acc[3] * fb - l1));
+        }
+        best_a = fmaxf(best_a, __shfl_xor_sync(0xffffffffu, best_a, 1));
+        best_a = fmaxf(best_a, __shfl_xor_sync(0xffffffffu, best_a, 2));
+        best_b = fmaxf(best_b, __shfl_xor_sync(0xffffffffu, best_b, 1));
+        best_b = fmaxf(best_b, __shfl_xor_sync(0xffffffffu, best_b, 2));
+        if (t == 0) {
+            if (va) orow[ja] = best_a;
+            if (vb) orow[jb] = best_b;
+        }
+    }
+}
+
+}  // namespace
+
+// rows = (b, g), row stride out_stride floats; keys beyond a row's candidates are not written
+cudaError_t launch_scores_fp8_decode(const Params &p, const void *Q, const void *K8, const float *ksc, const float *LSE,
+                                     float *out, int64_t out_stride, cudaStream_t st)
+{
+    const int bg = p.B * p.Hkv;
+    if (p.Lq != 1 || bg <= 0 || bg > 65535 || p.G > 128 || (p.D != 128 && p.D != 256)) return cudaErrorNotSupported;
+    const int GP = (p.G + 7) & ~7;
+    const size_t smem = (size_t)(GP / 8) * (p.D / 16) * 32 * 8 + (size_t)GP * 4;
+    int gx = (p.Lk + kScF8Warps * 16 - 1) / (kScF8Warps * 16);
+    const int cap = (148 * 8 + bg - 1) / bg;      // about eight CTAs per SM over the whole grid
+    if (gx > cap) gx = cap < 1 ? 1 : cap;
+    cudaError_t e = cudaSuccess;
+    if (p.D == 128) {
+        if (smem > 48 * 1024) e = cudaFuncSetAttribute(k_scores_fp8_decode<128>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        k_scores_fp8_decode<128><<<dim3((unsigned)gx, (unsigned)bg), kScF8Warps * 32, smem, st>>>(
+            p, (const __nv_bfloat16 *)Q, (const uint8_t *)K8, ksc, LSE, out, out_stride);
+    } else {
+        if (smem > 48 * 1024) e = cudaFuncSetAttribute(k_scores_fp8_decode<256>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        k_scores_fp8_decode<256><<<dim3((unsigned)gx, (unsigned)bg), kScF8Warps * 32, smem, st>>>(
+            p, (const __nv_bfloat16 *)Q, (const uint8_t *)K8, ksc, LSE, out, out_stride);
+    }
+    count_launch();
+    return cudaGetLastError();
+}
+
 bool sparse_fp8_supported(const Params &p, hs2_dtype dt)
 {
     auto m8 = [](int64_t x) { return x % 8 == 0; };

@@ -520,12 +520,17 @@ def test_fp8_kv_cache_on_large_head_groups_and_head_dim_256():
 
 def test_fp8_kv_cache_full_layer_decode_step():
     """The full-attention layer's decode step on the e4m3 cache: O, LSE and the selected indices against the oracle
-    run on the dequantised cache (groups of 8, 4 and 1, ragged lengths, a strided cache, several key tiles per warp)."""
+    run on the dequantised cache (groups of 8, 4 and 1, ragged lengths, a strided cache, several key tiles per warp;
+    then the paper's own shape - 64 heads on one KV head, head_dim 256 - and other large groups, which take the
+    tensor-core gather kernel for the attention and a second pass over the K codes for the scores)."""
     from gen.workloads import quantize_kv_e4m3
     cases = [
         dict(kv_len=3000, k_sel=200, window=32, batch=3),
         dict(kv_len=700, k_sel=64, window=16, n_q_heads=8, n_kv_heads=2, batch=2),
         dict(kv_len=450, k_sel=100, window=0, n_q_heads=4, n_kv_heads=4, batch=1),
+        dict(kv_len=2100, k_sel=256, window=32, n_q_heads=64, n_kv_heads=1, head_dim=256, batch=3),
+        dict(kv_len=900, k_sel=100, window=16, n_q_heads=24, n_kv_heads=2, head_dim=128, batch=2),      # G = 12: padded n-tile
+        dict(kv_len=640, k_sel=64, window=0, n_q_heads=128, n_kv_heads=1, head_dim=128, batch=1),
     ]
     for ci, over in enumerate(cases):
         wl = scaled("cfg5", q_len=1, n_needles=6, **over)
