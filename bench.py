@@ -605,7 +605,9 @@ def bench_kv_project(device, peaks, reps=7):
     t16 = med(lambda: hs2.hs2_kv_project(h, w, out=out))
     t8 = med(lambda: hs2.hs2_kv_project(h, w, out=o8, fp8=True, scales=sc))
     peak = peaks.get("bf16_tflops", peaks["bf16_tflops_sustained"])
+    tlib = med(lambda: torch.matmul(h, w.t(), out=out))     # the vendor library's GEMM on the same operands, for context only
     return {"workload": "T=32768 tokens, d_model 2048, 2048 output columns, bf16 in, fp32 accumulate",
+            "library_gemm_us": round(tlib * 1e3, 1), "library_gemm_tflops": round(fl / tlib / 1e9, 1),
             "bf16_out_us": round(t16 * 1e3, 1), "bf16_out_tflops": round(fl / t16 / 1e9, 1),
             "e4m3_out_us": round(t8 * 1e3, 1), "e4m3_out_tflops": round(fl / t8 / 1e9, 1),
             "peak_tflops_burst": peak, "frac_bf16_out": round(fl / t16 / 1e9 / peak, 4),

@@ -651,6 +651,15 @@ def test_kv_projection_bf16_and_fp8_outputs():
     assert_output_close(o8.reshape(-1, 8 * Hkv, D), Oo, torch.bfloat16, "sparse O on the projected FP8 cache")
     with pytest.raises(hs2.HS2Error):                       # n_out must be a multiple of 256
         hs2.hs2_kv_project(h, w[:128])
+    # more shapes of the CTA-pair kernel: a single tile with one row, ragged token counts across several 256-row tiles,
+    # one and many k-blocks, more tiles than CTA pairs
+    for T2, dm2, N2 in [(1, 64, 256), (257, 64, 256), (777, 128, 768), (1300, 2048, 512), (40000, 64, 512)]:
+        h2 = (torch.randn(T2, dm2, device="cuda", generator=g)).to(torch.bfloat16)
+        w2 = (torch.randn(N2, dm2, device="cuda", generator=g) / dm2 ** 0.5).to(torch.bfloat16)
+        got2 = hs2.hs2_kv_project(h2, w2).float()
+        torch.cuda.synchronize()
+        want2 = h2.double() @ w2.double().T                 # (the oracle's product, on the device for the large case)
+        assert bool(((got2.double() - want2).abs() <= want2.abs() * 2.0 ** -8 + 1e-5).all()), (T2, dm2, N2)
     assert hs2.hs2_device_error_flags() == 0
 
 
