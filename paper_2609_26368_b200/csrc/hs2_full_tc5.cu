@@ -21,6 +21,8 @@
 // TMEM before it returns.
 #include <cuda.h>
 
+#include <type_traits>
+
 #include "hs2_common.cuh"
 #include "hs2_tc5.cuh"
 
@@ -370,6 +372,9 @@ k_full_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
 // subtract LSE, take the group maximum and write 32 consecutive keys of a strip row per warp instruction.
 // The epilogue is a chain of TMEM loads and short dependent arithmetic: eight warps per CTA hide its latency
 // where four left the tensor pipe waiting for a free accumulator.
+#ifndef HS2_SC_KSTAGES
+#define HS2_SC_KSTAGES 2   // key tiles in flight in a 256-column CTA (2 to 5)
+#endif
 #ifndef HS2_SC_WIDE
 #define HS2_SC_WIDE 1   // 256-column CTAs of the score sweep for head_dim 128 and groups of 8 or 16 (0: 128 columns everywhere)
 #endif
@@ -391,8 +396,9 @@ struct ScCfg {
     static constexpr uint32_t kSlice = 128 * 128;                 // one slice of a key tile: 128 rows of 128 bytes
     static constexpr uint32_t kSliceQ = NC * 128;                 // one slice of the (query, head) rows
     static constexpr uint32_t kOffQ = 0;                          // (query, head) rows
-    static constexpr uint32_t kOffK = NQ * kSliceQ;               // 2 stages of key rows
-    static constexpr uint32_t kOffAug = kOffK + 2 * NQ * kSlice;  // one extra K step: [128][16] and [NC][16] bf16, 32-byte swizzle
+    static constexpr int KS = NC == 256 ? HS2_SC_KSTAGES : 2;     // depth of the ring of key tiles
+    static constexpr uint32_t kOffK = NQ * kSliceQ;               // KS stages of key rows
+    static constexpr uint32_t kOffAug = kOffK + KS * NQ * kSlice; // one extra K step: [128][16] and [NC][16] bf16, 32-byte swizzle
     static constexpr uint32_t kOffNl = kOffAug + 4096 + NC * 32;  // float[NC]: -LSE/scale per column
     static constexpr uint32_t kOffNq = kOffNl + NC * 4;           // int[NC]: keys needed per query
     static constexpr uint32_t kOffRow = kOffNq + NC * 4;          // int64[NC]: strip row of each query
@@ -403,7 +409,8 @@ struct ScCfg {
     static constexpr int kMinBlocks = (D <= 128 && NC == 128) ? 2 : 1;
     static_assert(kSmemBytes <= 227 * 1024, "fits the shared memory of one SM");
 };
-enum ScBar { SQ_FULL = 0, SK_FULL0, SK_FULL1, SK_EMPTY0, SK_EMPTY1, ACC_FULL0, ACC_FULL1, ACC_FREE0, ACC_FREE1, SC_N_BARS };
+// the key ring has up to five stages (SK_FULL0 + s, SK_EMPTY0 + s); the accumulator is double-buffered
+enum ScBar { SQ_FULL = 0, ACC_FULL0, ACC_FULL1, ACC_FREE0, ACC_FREE1, SK_FULL0 = 5, SK_EMPTY0 = 10, SC_N_BARS = 15 };
 
 // What the sweep does with a score:
 //   SC_STRIP   write it to the strip row at its key position (keys split into chunks over blockIdx.x)
@@ -438,7 +445,7 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
 {
     using S = ScCfg<D, NC>;
     constexpr int kScTmaWarp = S::kTmaWarp, kScMmaWarp = S::kMmaWarp;
-    constexpr int NQ = S::NQ;
+    constexpr int NQ = S::NQ, KS = S::KS;
     constexpr uint32_t kScOffQ = S::kOffQ, kScOffK = S::kOffK, kScOffNl = S::kOffNl, kScOffNq = S::kOffNq,
                        kScOffRow = S::kOffRow, kScOffTau = S::kOffTau, kScOffCnt = S::kOffCnt, kScOffBar = S::kOffBar,
                        kStage = NQ * S::kSlice, kStageQ = NQ * S::kSliceQ;
@@ -538,8 +545,7 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
     if (tid == 0) {
         *abort_flag = 0;
         mbar_init(bar(SQ_FULL), 1);
-        mbar_init(bar(SK_FULL0), 1); mbar_init(bar(SK_FULL1), 1);
-        mbar_init(bar(SK_EMPTY0), 1); mbar_init(bar(SK_EMPTY1), 1);
+        for (int s = 0; s < KS; ++s) { mbar_init(bar(SK_FULL0 + s), 1); mbar_init(bar(SK_EMPTY0 + s), 1); }
         mbar_init(bar(ACC_FULL0), 1); mbar_init(bar(ACC_FULL1), 1);
         mbar_init(bar(ACC_FREE0), kEpiThreads); mbar_init(bar(ACC_FREE1), kEpiThreads);
         asm volatile("fence.mbarrier_init.release.cluster;\n" ::: "memory");
@@ -560,8 +566,8 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             for (int sl = 0; sl < NQ; ++sl) tma_load_4d(sbase + kScOffQ + sl * S::kSliceQ, &tmQ, bar(SQ_FULL), 64 * sl, gkv * p.G, iq0, b);
             int issued = 0;
             for (int t = 0; t < ntile; ++t) {
-                const int st = t & 1;
-                if (!mbar_wait(bar(SK_EMPTY0 + st), ((t >> 1) & 1) ^ 1, abort_flag)) break;
+                const int st = t % KS;
+                if (!mbar_wait(bar(SK_EMPTY0 + st), ((t / KS) & 1) ^ 1, abort_flag)) break;
                 issued = t + 1;
                 mbar_expect_tx(bar(SK_FULL0 + st), kStage);
                 const uint32_t kdst = sbase + kScOffK + st * kStage;
@@ -570,8 +576,8 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 for (int sl = 0; sl < NQ; ++sl) tma_load_4d(kdst + sl * S::kSlice, &tmK, bar(SK_FULL0 + st), 64 * sl, gkv, krow, b);
             }
             if (*abort_flag) {
-                for (int t = max(0, issued - 2); t < issued; ++t)
-                    for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait(bar(SK_FULL0 + (t & 1)), (t >> 1) & 1); ++it) {}
+                for (int t = max(0, issued - KS); t < issued; ++t)
+                    for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait(bar(SK_FULL0 + t % KS), (t / KS) & 1); ++it) {}
                 for (uint32_t it = 0; it < kSpinLimit && !mbar_try_wait(bar(SQ_FULL), 0); ++it) {}
             }
         }
@@ -580,19 +586,19 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             constexpr uint32_t id = idesc(128, NC, 0);
             bool ok = mbar_wait(bar(SQ_FULL), 0, abort_flag);
             for (int t = 0; ok && t < ntile; ++t) {
-                const int st = t & 1, ph = (t >> 1) & 1;
-                if (!mbar_wait(bar(SK_FULL0 + st), ph, abort_flag)) break;
-                if (!mbar_wait(bar(ACC_FREE0 + st), ph ^ 1, abort_flag)) break;
+                const int st = t % KS, ab = t & 1;
+                if (!mbar_wait(bar(SK_FULL0 + st), (t / KS) & 1, abort_flag)) break;
+                if (!mbar_wait(bar(ACC_FREE0 + ab), ((t >> 1) & 1) ^ 1, abort_flag)) break;
                 tc_fence_after();
                 const uint32_t ka = sbase + kScOffK + st * kStage, qa = sbase + kScOffQ;
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks) {
                     const uint32_t off = (ks >> 2) * S::kSlice + (ks & 3) * 32, offq = (ks >> 2) * S::kSliceQ + (ks & 3) * 32;
-                    umma(tmem + st * NC, smem_desc(ka + off, 16, 1024), smem_desc(qa + offq, 16, 1024), id, ks > 0);
+                    umma(tmem + ab * NC, smem_desc(ka + off, 16, 1024), smem_desc(qa + offq, 16, 1024), id, ks > 0);
                 }
-                umma(tmem + st * NC, smem_desc_sw32(sbase + S::kOffAug, 256), smem_desc_sw32(sbase + S::kOffAug + 4096, 256), id, 1);   // - LSE / scale
+                umma(tmem + ab * NC, smem_desc_sw32(sbase + S::kOffAug, 256), smem_desc_sw32(sbase + S::kOffAug + 4096, 256), id, 1);   // - LSE / scale
                 umma_commit(bar(SK_EMPTY0 + st));
-                umma_commit(bar(ACC_FULL0 + st));
+                umma_commit(bar(ACC_FULL0 + ab));
             }
         }
     } else if (warp < 4 * EW) {
@@ -605,13 +611,25 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
         constexpr bool kHoist = TQW <= 8;
         int nq_r[kHoist ? TQW : 1];
         float *orow_r[kHoist && MODE != SC_FILTER ? TQW : 1];
-        float tau_r[kHoist && MODE == SC_FILTER ? TQW : 1];   // thresholds as floats: one compare per score
+        float tau_r[kHoist && MODE == SC_FILTER ? TQW : 1];   // thresholds in the accumulator's units: one compare per score
         int rb_r[kHoist && MODE == SC_FILTER ? TQW : 1];      // first slot of this warp's sub-list of the query's candidates (the lists of a block hold < 2^28 entries)
         int cnt_r[MODE == SC_FILTER ? TQW : 1];               // entries this warp has appended per query (warp-uniform)
         const int capq = MODE == SC_FILTER ? fb.cap >> 2 : 0;
+        // The filter compares the accumulator (score / scale) with threshold / scale, lowered by a few units in the
+        // last place: every score that reaches the threshold after the multiplication by scale passes (the list may
+        // hold a few more, which is harmless: the select works on the stored scores), and the multiplication is
+        // paid by the few scores that pass, not by all.
+        auto raw_tau = [&](uint32_t tk) {
+            const float t = key_to_float(tk) / p.scale;   // -inf stays -inf (all pass), NaN stays NaN (none)
+            return t - fabsf(t) * 4.8e-7f - 1e-30f;
+        };
+        int nq_min = 0x7fffffff;   // tiles that end below it need no causal test in this warp
         if (MODE == SC_FILTER) {
 #pragma unroll
-            for (int q = 0; q < TQW; ++q) cnt_r[q] = 0;
+            for (int q = 0; q < TQW; ++q) {
+                cnt_r[q] = 0;
+                nq_min = min(nq_min, s_nq[q_first + q]);
+            }
         }
         if (kHoist) {
 #pragma unroll
@@ -619,36 +637,30 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                 nq_r[q] = s_nq[q_first + q];
                 if (MODE != SC_FILTER) orow_r[q] = out + s_row[q_first + q] * out_stride;   // never used when nq is 0
                 if (MODE == SC_FILTER) {
-                    tau_r[q] = key_to_float(s_tau[q_first + q]);
+                    tau_r[q] = raw_tau(s_tau[q_first + q]);
                     rb_r[q] = (int)(s_row[q_first + q] * fb.cap) + quarter * capq;
                 }
             }
         }
         bool alive = true;
-        for (int t = 0; t < ntile; ++t) {
+        // one key tile: CHECK = false when every key of the tile is visible to every query of this warp
+        auto do_tile = [&](int t, auto check_tag) {
+            constexpr bool CHECK = decltype(check_tag)::value;
             const int ab = t & 1;
-            if (alive && !__all_sync(0xffffffffu, mbar_wait(bar(ACC_FULL0 + ab), (t >> 1) & 1, abort_flag))) alive = false;
-            if (MODE != SC_FILTER && !alive) break;
-            tc_fence_after();
             const int key = (kt0 + t) * kstep * 128 + row;
             const int col = MODE == SC_SAMPLE ? (kt0 + t) * 128 + row : key;
-            float aval[MODE == SC_FILTER ? TQW : 1];
-            unsigned passbits = 0;     // bit q: the score of query q_first + q passes the filter
+            float aval[MODE == SC_FILTER ? TQW : 1];      // accumulator maxima (score / scale)
+            unsigned mq[MODE == SC_FILTER ? TQW : 1];     // per query: the lanes whose score passes the filter
             float carry = -INFINITY;   // running group maximum when a group spans several chunks
 #pragma unroll
             for (int c = 0; c < CPW; ++c) {
                 const int cc = half * CPW + c;   // 32-column chunk of the accumulator
                 float v[32];
-                if (alive) {
-                    tmem_ld32(lane_base + ab * NC + cc * 32, v);
-                    tmem_wait_ld();
-                    if (c == CPW - 1) {   // the last chunk is in registers: the accumulator goes back to the tensor core
-                        tc_fence_before();   // before the arithmetic on it, not after
-                        mbar_arrive(bar(ACC_FREE0 + ab));
-                    }
-                } else {
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) v[e] = 0.f;
+                tmem_ld32(lane_base + ab * NC + cc * 32, v);
+                tmem_wait_ld();
+                if (c == CPW - 1) {   // the last chunk is in registers: the accumulator goes back to the tensor core
+                    tc_fence_before();   // before the arithmetic on it, not after
+                    mbar_arrive(bar(ACC_FREE0 + ab));
                 }
 #pragma unroll
                 for (int q = 0; q < QPC; ++q) {
@@ -665,15 +677,15 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                     }
                     const int ql = CPQ > 1 ? c / CPQ : c * QPC + q;   // query inside this warp's set
                     const int tq = q_first + ql;
-                    const float av = a * p.scale;
-                    const int nq = kHoist ? nq_r[kHoist ? ql : 0] : s_nq[tq];
                     if (MODE == SC_FILTER) {
-                        aval[ql] = av;
+                        aval[ql] = a;
                         // (float order and key order agree: -0 and +0 are one key, NaN scores are a caller error)
-                        const float tau = kHoist ? tau_r[kHoist ? ql : 0] : key_to_float(s_tau[tq]);
-                        const bool pass = alive && key < nq && av >= tau;
-                        passbits |= (pass ? 1u : 0u) << ql;
-                    } else if (key < nq) {
+                        const float tau = kHoist ? tau_r[kHoist ? ql : 0] : raw_tau(s_tau[tq]);
+                        bool pass = a >= tau;
+                        if (CHECK) pass = pass && key < (kHoist ? nq_r[kHoist ? ql : 0] : s_nq[tq]);
+                        mq[ql] = __ballot_sync(0xffffffffu, pass);
+                    } else if (key < (kHoist ? nq_r[kHoist ? ql : 0] : s_nq[tq])) {
+                        const float av = a * p.scale;
                         if (kHoist) orow_r[kHoist ? ql : 0][col] = av;
                         else out[s_row[tq] * out_stride + col] = av;
                     }
@@ -681,26 +693,29 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             }
             if (MODE == SC_FILTER) {
                 // Append in no particular order.  This warp is the only writer of its sub-list of every query it owns,
-                // so the fill counts live in registers (the same in every lane): per query one ballot, a rank inside
-                // it, two stores.  The queries are independent of one another - no atomic, no shared memory, no
-                // dependent chain from one query to the next (an atomic per (query, warp, tile) on a shared counter
-                // plus a shuffle of its result made the eight appends one long latency chain).
-                if (__any_sync(0xffffffffu, passbits != 0u)) {
+                // so the fill counts live in registers (the same in every lane): the ballot taken at the compare gives
+                // every passing lane its rank, then two stores.  The queries are independent of one another - no
+                // atomic, no shared memory, no dependent chain from one query to the next (an atomic per (query, warp,
+                // tile) on a shared counter plus a shuffle of its result made the appends one long latency chain).
 #pragma unroll
-                    for (int q = 0; q < TQW; ++q) {
-                        const bool mine = (passbits >> q) & 1u;
-                        const unsigned m = __ballot_sync(0xffffffffu, mine);
-                        const int pos = cnt_r[q] + __popc(m & lt_mask);
-                        if (mine && pos < capq) {
-                            const int64_t o = kHoist ? (int64_t)(rb_r[kHoist ? q : 0] + pos)
-                                                     : s_row[q_first + q] * fb.cap + quarter * capq + pos;
-                            fb.cand_a[o] = aval[q];
-                            fb.cand_j[o] = key;
-                        }
-                        cnt_r[q] += __popc(m);
+                for (int q = 0; q < TQW; ++q) {
+                    const unsigned m = mq[q];
+                    const int pos = cnt_r[q] + __popc(m & lt_mask);
+                    if (((m >> lane) & 1u) && pos < capq) {
+                        const int64_t o = kHoist ? (int64_t)(rb_r[kHoist ? q : 0] + pos)
+                                                 : s_row[q_first + q] * fb.cap + quarter * capq + pos;
+                        fb.cand_a[o] = aval[q] * p.scale;
+                        fb.cand_j[o] = key;
                     }
+                    cnt_r[q] += __popc(m);
                 }
             }
+        };
+        for (int t = 0; t < ntile; ++t) {
+            if (!__all_sync(0xffffffffu, mbar_wait(bar(ACC_FULL0 + (t & 1)), (t >> 1) & 1, abort_flag))) { alive = false; break; }
+            tc_fence_after();
+            if (MODE == SC_FILTER && (kt0 + t + 1) * kstep * 128 <= nq_min) do_tile(t, std::false_type{});
+            else do_tile(t, std::true_type{});
         }
         if (MODE == SC_FILTER) {
             const bool fine = alive && !*abort_flag;   // otherwise the sweep gave up: -1 sends the row to the exact redo
