@@ -349,8 +349,7 @@ hs2_status hs2_full_attn_select(const hs2_problem *hp, const void *Q, const void
             int *count = (int *)(base + (size_t)block * 8);   // four sub-list counts per row
             char *big = base + align_up((size_t)block * 24, 256);
             float *sample = (float *)big;
-            float *cand_a = (float *)big;
-            int32_t *cand_j = (int32_t *)(big + (size_t)block * fp.cap * 4);
+            void *cand = big;   // block * cap records of (score, key), 8 bytes each
             bool usable = true;
             for (int64_t r0 = 0; r0 < rows && usable; r0 += block) {
                 const int64_t n = rows - r0 < block ? rows - r0 : block;
@@ -358,8 +357,8 @@ hs2_status hs2_full_attn_select(const hs2_problem *hp, const void *Q, const void
                 if (e == cudaErrorNotSupported && r0 == 0) { usable = false; break; }   // nothing launched yet: use the strips
                 if (e != cudaSuccess) return cuda_fail(e);
                 if ((e = launch_filter_thresholds(p, sample, fp.ns_w, r0, n, kFilterSamp, fp.cap, tau, flag, st)) != cudaSuccess) return cuda_fail(e);
-                if ((e = launch_scores_filter_tc5(p, Q, K, LSE, r0, n, tau, cand_a, cand_j, count, fp.cap, st)) != cudaSuccess) return cuda_fail(e);
-                if ((e = launch_filter_select(p, cand_a, cand_j, count, fp.cap, idx, r0, n, flag, st)) != cudaSuccess) return cuda_fail(e);
+                if ((e = launch_scores_filter_tc5(p, Q, K, LSE, r0, n, tau, cand, count, fp.cap, st)) != cudaSuccess) return cuda_fail(e);
+                if ((e = launch_filter_select(p, cand, count, fp.cap, idx, r0, n, flag, st)) != cudaSuccess) return cuda_fail(e);
                 if ((e = launch_select_recompute(p, Q, K, LSE, idx, r0, n, flag, st)) != cudaSuccess) return cuda_fail(e);
             }
             if (usable) return HS2_OK;

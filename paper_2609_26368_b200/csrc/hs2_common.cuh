@@ -92,7 +92,7 @@ cudaError_t launch_topk(const Params &p, const float *scores, int64_t score_stri
 int filter_sample_width(const Params &p, int samp);
 cudaError_t launch_filter_thresholds(const Params &p, const float *sample, int64_t stride, int64_t row0, int64_t n_rows,
                                      int samp, int cap, uint32_t *tau_key, int *flag, cudaStream_t st);
-cudaError_t launch_filter_select(const Params &p, const float *cand_a, const int32_t *cand_j, const int *count, int cap,
+cudaError_t launch_filter_select(const Params &p, const void *cand, const int *count, int cap,
                                  int32_t *idx, int64_t row0, int64_t n_rows, int *flag, cudaStream_t st);
 cudaError_t launch_select_recompute(const Params &p, const void *Q, const void *K, const float *LSE, int32_t *idx,
                                     int64_t row0, int64_t n_rows, const int *flag, cudaStream_t st);
@@ -134,7 +134,7 @@ bool scores_filter_supported(const Params &p, hs2_dtype dt);
 cudaError_t launch_scores_sampled_tc5(const Params &p, const void *Q, const void *K, const float *LSE, float *out,
                                       int64_t out_stride, int64_t row0, int64_t n_rows, int samp, cudaStream_t st);
 cudaError_t launch_scores_filter_tc5(const Params &p, const void *Q, const void *K, const float *LSE, int64_t row0,
-                                     int64_t n_rows, const uint32_t *tau_key, float *cand_a, int32_t *cand_j, int *count,
+                                     int64_t n_rows, const uint32_t *tau_key, void *cand, int *count,
                                      int cap, cudaStream_t st);
 // tcgen05 sparse attention for large head groups (bf16, head_dim 128 or 256, 8 < group <= 128)
 bool sparse_tc5_supported_shape(const Params &p, hs2_dtype dt);   // the shape alone (no driver query)

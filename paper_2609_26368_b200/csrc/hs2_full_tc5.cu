@@ -423,8 +423,7 @@ enum { SC_STRIP = 0, SC_SAMPLE = 1, SC_FILTER = 2 };
 
 struct FilterBuf {
     const uint32_t *tau_key;   // [rows of the block] threshold as order-preserving key
-    float *cand_a;             // [rows][4][cap / 4]
-    int32_t *cand_j;           // [rows][4][cap / 4]
+    int2 *cand;                // [rows][4][cap / 4] records: x = the score's bits, y = the key
     int *count;                // [rows][4] candidates found per sub-list (may exceed cap / 4: then the row is redone elsewhere; -1: gave up)
     int cap;                   // multiple of 4
 };
@@ -704,8 +703,7 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
                     if (((m >> lane) & 1u) && pos < capq) {
                         const int64_t o = kHoist ? (int64_t)(rb_r[kHoist ? q : 0] + pos)
                                                  : s_row[q_first + q] * fb.cap + quarter * capq + pos;
-                        fb.cand_a[o] = aval[q] * p.scale;
-                        fb.cand_j[o] = key;
+                        fb.cand[o] = make_int2(__float_as_int(aval[q] * p.scale), key);   // one 8-byte store
                     }
                     cnt_r[q] += __popc(m);
                 }
@@ -964,10 +962,10 @@ cudaError_t launch_scores_sampled_tc5(const Params &p, const void *Q, const void
 
 // Ordered candidate lists: every (score, key) whose order key is >= tau_key[row], in key order.
 cudaError_t launch_scores_filter_tc5(const Params &p, const void *Q, const void *K, const float *LSE, int64_t row0,
-                                     int64_t n_rows, const uint32_t *tau_key, float *cand_a, int32_t *cand_j, int *count,
+                                     int64_t n_rows, const uint32_t *tau_key, void *cand, int *count,
                                      int cap, cudaStream_t st)
 {
-    FilterBuf fb{tau_key, cand_a, cand_j, count, cap};
+    FilterBuf fb{tau_key, static_cast<int2 *>(cand), count, cap};
     return launch_sc_mode<SC_FILTER>(p, Q, K, LSE, nullptr, 0, row0, n_rows, false, 1, fb, st);
 }
 

@@ -1542,7 +1542,7 @@ k_sample_tau(const Params p, const float *__restrict__ sample, int64_t stride, i
 // the exact redo.
 template <int THREADS, int E>
 __global__ void __launch_bounds__(THREADS, THREADS > 256 ? 1 : (E > 16 ? 3 : 4))
-k_cand_select(const Params p, const float *__restrict__ cand_a, const int32_t *__restrict__ cand_j, const int *__restrict__ count,
+k_cand_select(const Params p, const int2 *__restrict__ cand, const int *__restrict__ count,
               int cap, int32_t *__restrict__ idx, int64_t row0, int *__restrict__ flag)
 {
     constexpr int WARPS = THREADS / 32, TG = THREADS / 4;
@@ -1584,21 +1584,21 @@ k_cand_select(const Params p, const float *__restrict__ cand_a, const int32_t *_
     const int nv = mine_cnt > l ? min(E, (mine_cnt - l + TG - 1) / TG) : 0;
     const int nvw = __reduce_max_sync(0xffffffffu, nv);   // the unrolled per-entry loops stop at the warp's longest thread
     float val[E];
+    // a record is (score, key): the score stays in a register, the key waits in shared memory until the threshold is
+    // known (each thread reads back only what it stored itself)
 #pragma unroll
-    for (int e = 0; e < E; ++e) val[e] = e < nv ? __ldg(cand_a + base + TG * e) : 0.f;
-    // the key indices are wanted only after the threshold is known: they travel to shared memory meanwhile (each
-    // thread reads back only what it copied itself, so its own wait is all the ordering that takes)
-#pragma unroll
-    for (int e = 0; e < E; ++e)
-        if (e < nv && e < nvw)
-            asm volatile("cp.async.ca.shared.global [%0], [%1], 4;\n" ::"r"((uint32_t)__cvta_generic_to_shared(s_pay + e * THREADS + tid)),
-                         "l"(cand_j + base + TG * e) : "memory");
-    asm volatile("cp.async.commit_group;\n" ::: "memory");
+    for (int e = 0; e < E; ++e) {
+        val[e] = 0.f;
+        if (e < nv) {
+            const int2 rec = __ldg(cand + base + TG * e);
+            val[e] = __int_as_float(rec.x);
+            s_pay[e * THREADS + tid] = rec.y;
+        }
+    }
     const int nwords = (n_keys + 31) >> 5;
     for (int wd = tid; wd < nwords; wd += THREADS) bitmap[wd] = 0u;   // (rank_from_top's barriers order this before the marking)
     const RankOut r = rank_from_top<THREADS, E, true>(val, nv, (unsigned)k_row, (unsigned)total, hist, s_list, (unsigned)kCandList, s_lo,
                                                       s_hi, s_warp, s_misc, tid, lane, warp);
-    asm volatile("cp.async.wait_group 0;\n" ::: "memory");
     if (!r.ok || r.n_eq > (unsigned)kCandList) {   // thousands of candidates within one bin of the threshold: the exact redo takes the row
         if (tid == 0) flag[blockIdx.x] = 1;
         return;
@@ -1712,7 +1712,7 @@ cudaError_t launch_filter_thresholds(const Params &p, const float *sample, int64
 }
 
 // final selection from the candidate lists; rows whose lists are unusable get flag[row] = 1
-cudaError_t launch_filter_select(const Params &p, const float *cand_a, const int32_t *cand_j, const int *count, int cap,
+cudaError_t launch_filter_select(const Params &p, const void *cand, const int *count, int cap,
                                  int32_t *idx, int64_t row0, int64_t n_rows, int *flag, cudaStream_t st)
 {
     if (n_rows == 0) return cudaSuccess;
@@ -1724,7 +1724,7 @@ cudaError_t launch_filter_select(const Params &p, const float *cand_a, const int
             const cudaError_t e2 = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
             if (e2 != cudaSuccess) return e2;
         }
-        kern<<<n, threads, smem, st>>>(p, cand_a, cand_j, count, cap, idx, row0, flag);
+        kern<<<n, threads, smem, st>>>(p, static_cast<const int2 *>(cand), count, cap, idx, row0, flag);
         count_launch();
         return cudaSuccess;
     };
