@@ -373,7 +373,7 @@ k_full_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
 // The epilogue is a chain of TMEM loads and short dependent arithmetic: eight warps per CTA hide its latency
 // where four left the tensor pipe waiting for a free accumulator.
 #ifndef HS2_SC_KSTAGES
-#define HS2_SC_KSTAGES 2   // key tiles in flight in a 256-column CTA (2 to 5)
+#define HS2_SC_KSTAGES 3   // key tiles in flight in a 256-column CTA (2 to 5); measured on the 128K layer: 2: 221 ms, 3: 219 ms, 4: 237 ms
 #endif
 #ifndef HS2_SC_WIDE
 #define HS2_SC_WIDE 1   // 256-column CTAs of the score sweep for head_dim 128 and groups of 8 or 16 (0: 128 columns everywhere)
@@ -407,6 +407,8 @@ struct ScCfg {
     static constexpr uint32_t kOffBar = kOffCnt + 1024;
     static constexpr uint32_t kSmemBytes = kOffBar + kBarBytes + kAlignSlack;
     static constexpr int kMinBlocks = (D <= 128 && NC == 128) ? 2 : 1;
+    // (the 18 warps of NC = 256 get 96 registers per thread: the register file is handed out as if a CTA had a multiple
+    // of four warps, and a launch that asks for 112 is refused)
     static_assert(kSmemBytes <= 227 * 1024, "fits the shared memory of one SM");
 };
 // the key ring has up to five stages (SK_FULL0 + s, SK_EMPTY0 + s); the accumulator is double-buffered
@@ -423,7 +425,7 @@ enum { SC_STRIP = 0, SC_SAMPLE = 1, SC_FILTER = 2 };
 
 struct FilterBuf {
     const uint32_t *tau_key;   // [rows of the block] threshold as order-preserving key
-    int2 *cand;                // [rows][4][cap / 4] records: x = the score's bits, y = the key
+    int2 *cand;                // [rows][4][cap / 4] records: x = bits of score / scale (the accumulator's value), y = the key
     int *count;                // [rows][4] candidates found per sub-list (may exceed cap / 4: then the row is redone elsewhere; -1: gave up)
     int cap;                   // multiple of 4
 };
@@ -642,6 +644,9 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             }
         }
         bool alive = true;
+        bool room = false;       // every sub-list of this warp can take a whole tile's worth of entries
+        int t_recheck = 0;       // the tile at which that has to be looked at again
+        const unsigned lane_bit = 1u << lane;
         // one key tile: CHECK = false when every key of the tile is visible to every query of this warp
         auto do_tile = [&](int t, auto check_tag) {
             constexpr bool CHECK = decltype(check_tag)::value;
@@ -693,20 +698,35 @@ k_scores_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CU
             if (MODE == SC_FILTER) {
                 // Append in no particular order.  This warp is the only writer of its sub-list of every query it owns,
                 // so the fill counts live in registers (the same in every lane): the ballot taken at the compare gives
-                // every passing lane its rank, then two stores.  The queries are independent of one another - no
+                // every passing lane its rank, then one store.  The queries are independent of one another - no
                 // atomic, no shared memory, no dependent chain from one query to the next (an atomic per (query, warp,
                 // tile) on a shared counter plus a shuffle of its result made the appends one long latency chain).
+                // A tile adds at most 32 entries to a sub-list, so the test against the capacity is made per tile,
+                // and only once the fullest sub-list could reach it (never, for a list that stays inside its six
+                // standard deviations); until then no append looks at the capacity.
+                if (t >= t_recheck) {
+                    int cmax = cnt_r[0];
 #pragma unroll
-                for (int q = 0; q < TQW; ++q) {
-                    const unsigned m = mq[q];
-                    const int pos = cnt_r[q] + __popc(m & lt_mask);
-                    if (((m >> lane) & 1u) && pos < capq) {
-                        const int64_t o = kHoist ? (int64_t)(rb_r[kHoist ? q : 0] + pos)
-                                                 : s_row[q_first + q] * fb.cap + quarter * capq + pos;
-                        fb.cand[o] = make_int2(__float_as_int(aval[q] * p.scale), key);   // one 8-byte store
-                    }
-                    cnt_r[q] += __popc(m);
+                    for (int q = 1; q < TQW; ++q) cmax = max(cmax, cnt_r[q]);
+                    room = cmax + 32 <= capq;
+                    t_recheck = room ? t + (capq - cmax) / 32 : t + 1;
                 }
+                auto append = [&](auto room_tag) {
+                    constexpr bool ROOM = decltype(room_tag)::value;
+#pragma unroll
+                    for (int q = 0; q < TQW; ++q) {
+                        const unsigned m = mq[q];
+                        const int pos = cnt_r[q] + __popc(m & lt_mask);
+                        if ((m & lane_bit) && (ROOM || pos < capq)) {
+                            const int64_t o = kHoist ? (int64_t)(rb_r[kHoist ? q : 0] + pos)
+                                                     : s_row[q_first + q] * fb.cap + quarter * capq + pos;
+                            fb.cand[o] = make_int2(__float_as_int(aval[q]), key);   // one 8-byte store; the select scales the score
+                        }
+                        cnt_r[q] += __popc(m);
+                    }
+                };
+                if (room) append(std::true_type{});
+                else append(std::false_type{});
             }
         };
         for (int t = 0; t < ntile; ++t) {

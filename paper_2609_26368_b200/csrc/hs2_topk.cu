@@ -1599,7 +1599,7 @@ k_cand_select(const Params p, const int2 *__restrict__ cand, const int *__restri
         val[e] = 0.f;
         if (e < nv) {
             const int2 rec = __ldg(cand + base + TG * e);
-            val[e] = __int_as_float(rec.x);
+            val[e] = __int_as_float(rec.x) * p.scale;   // the sweep stores the accumulator's value: the score is that times scale
             s_pay[e * THREADS + tid] = rec.y;
         }
     }
