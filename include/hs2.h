@@ -291,7 +291,7 @@ int hs2_device_error_flags(unsigned *flags);
  * Returns the previous setting.  Process-wide. */
 int hs2_set_tcgen05_enabled(int enabled);
 
-/* Tuning knob of hs2_full_attn_select: from which kv_len on (default 24576) the selection thresholds a sample of
+/* Tuning knob of hs2_full_attn_select: from which kv_len on (default 18432) the selection thresholds a sample of
  * the scores and works on filtered candidate lists instead of complete score strips.  Both ways select from the same
  * tensor-core scores and give the same indices, with one exception: a row whose filtered list came out unusable
  * is redone from scores recomputed with fp32 FMAs, which can order two keys differently when their scores agree

@@ -102,9 +102,9 @@ DecodeFusedPlan decode_fused_plan(const Params &pd, size_t sweep_ws)
 // ---- filtered selection (sampled threshold -> ordered candidate lists -> select) ----
 constexpr int kFilterSamp = 16;             // every 16th key tile is scored for the threshold (every 8th: 6 ms more at 128K)
 // The filtered path wins when rows are long (measured, full layer with selection, filtered vs strips: 2 x 32768 keys
-// 35.0 vs 38.0 ms, 2 x 24576 keys 20.9 vs 21.5 ms, 2 x 16384 keys 10.3 vs 8.9 ms, 8192 keys 1.57 vs 1.12 ms): shorter
+// 30.8 vs 38.0 ms, 2 x 20480 keys 13.4 vs 14.6 ms, 2 x 16384 keys 9.1 vs 8.7 ms, 8192 keys 1.32 vs 1.10 ms): shorter
 // contexts keep the strips.
-std::atomic<int> g_filter_min_keys{24576};
+std::atomic<int> g_filter_min_keys{18432};
 std::atomic<int> g_disable_tc5{0};          // testing knob: run the mma.sync kernels instead of the tcgen05 ones
 constexpr size_t kFilterBigCap = (size_t)1 << 30;
 
