@@ -1159,6 +1159,8 @@ cudaError_t launch_topk(const Params &p, const float *scores, int64_t score_stri
 // slow, but it needs no storage, no host round trip, and handles any number of rows.
 namespace {
 
+constexpr int kRedoChunk = 64;
+
 __global__ void __launch_bounds__(256)
 k_select_recompute(const Params p, const __nv_bfloat16 *__restrict__ Q, const __nv_bfloat16 *__restrict__ K,
                    const float *__restrict__ LSE, int32_t *__restrict__ idx, int64_t row0, int64_t n_rows,
@@ -1170,92 +1172,102 @@ k_select_recompute(const Params p, const __nv_bfloat16 *__restrict__ Q, const __
     __shared__ unsigned s_warp[WARPS];
     __shared__ unsigned s_prefix, s_need, s_run_gt, s_run_eq;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    // a fixed grid walks the rows of the block: a launch that finds no flagged row (the usual case) costs a few
-    // microseconds whatever the number of rows
-    for (int64_t lr = blockIdx.x; lr < n_rows; lr += gridDim.x) {
-        if (!flag[lr]) continue;   // (the same for every thread of the CTA)
-        const int64_t row = row0 + lr;
-        const int i = (int)(row % p.Lq);
-        const int g = (int)((row / p.Lq) % p.Hkv);
-        const int b = (int)(row / ((int64_t)p.Lq * p.Hkv));
-        const int kvl = kvlen_of(p, b);
-        const int pos = pos_of(p, b, i);
-        const int nc = max(0, min(pos - p.w + 1, kvl));
-        const int take = min(p.k, nc);
-        int32_t *out = idx + row * p.k;
-        float *slse = sq + p.G * D;
-        for (int e = tid; e < p.G * D; e += THREADS)
-            sq[e] = __bfloat162float(Q[b * p.qs_b + (int64_t)i * p.qs_t + (g * p.G + e / D) * p.qs_h + e % D]);
-        for (int e = tid; e < p.G; e += THREADS) slse[e] = LSE[((int64_t)b * p.Hq + g * p.G + e) * p.Lq + i];
+    // The rows of the block are walked in chunks of kRedoChunk rows: one coalesced load and one barrier tell a CTA
+    // whether any row of its chunk is flagged, so a launch that finds none (the usual case) costs a few microseconds
+    // whatever the number of rows; the flagged rows of one chunk are redone one after the other.
+    __shared__ int s_flagged[kRedoChunk];
+    for (int64_t chunk = (int64_t)blockIdx.x * kRedoChunk; chunk < n_rows; chunk += (int64_t)gridDim.x * kRedoChunk) {
+        const int mine = tid < kRedoChunk && chunk + tid < n_rows ? flag[chunk + tid] : 0;
+        if (!__syncthreads_or(mine)) continue;
+        if (tid < kRedoChunk) s_flagged[tid] = mine;
         __syncthreads();
-        const __nv_bfloat16 *kb = K + b * p.ks_b + g * p.ks_h;
-        auto key_of = [&](int j) -> uint32_t {   // order key of a[j] = max_h (scale <q_h, k_j> - LSE_h)
-            const uint4 *kr = reinterpret_cast<const uint4 *>(kb + (int64_t)j * p.ks_t);
-            float kf[D];
-    #pragma unroll
-            for (int c = 0; c < D / 8; ++c) {
-                const uint4 v = __ldg(kr + c);
-                const uint32_t w[4] = {v.x, v.y, v.z, v.w};
-    #pragma unroll
-                for (int t = 0; t < 4; ++t) { kf[8 * c + 2 * t] = __uint_as_float(w[t] << 16); kf[8 * c + 2 * t + 1] = __uint_as_float(w[t] & 0xffff0000u); }
+        for (int r = 0; r < kRedoChunk && chunk + r < n_rows; ++r) {
+            if (!s_flagged[r]) continue;   // (the same for every thread of the CTA)
+            const int64_t lr = chunk + r;
+            const int64_t row = row0 + lr;
+            const int i = (int)(row % p.Lq);
+            const int g = (int)((row / p.Lq) % p.Hkv);
+            const int b = (int)(row / ((int64_t)p.Lq * p.Hkv));
+            const int kvl = kvlen_of(p, b);
+            const int pos = pos_of(p, b, i);
+            const int nc = max(0, min(pos - p.w + 1, kvl));
+            const int take = min(p.k, nc);
+            int32_t *out = idx + row * p.k;
+            float *slse = sq + p.G * D;
+            for (int e = tid; e < p.G * D; e += THREADS)
+                sq[e] = __bfloat162float(Q[b * p.qs_b + (int64_t)i * p.qs_t + (g * p.G + e / D) * p.qs_h + e % D]);
+            for (int e = tid; e < p.G; e += THREADS) slse[e] = LSE[((int64_t)b * p.Hq + g * p.G + e) * p.Lq + i];
+            __syncthreads();
+            const __nv_bfloat16 *kb = K + b * p.ks_b + g * p.ks_h;
+            auto key_of = [&](int j) -> uint32_t {   // order key of a[j] = max_h (scale <q_h, k_j> - LSE_h)
+                const uint4 *kr = reinterpret_cast<const uint4 *>(kb + (int64_t)j * p.ks_t);
+                float kf[D];
+        #pragma unroll
+                for (int c = 0; c < D / 8; ++c) {
+                    const uint4 v = __ldg(kr + c);
+                    const uint32_t w[4] = {v.x, v.y, v.z, v.w};
+        #pragma unroll
+                    for (int t = 0; t < 4; ++t) { kf[8 * c + 2 * t] = __uint_as_float(w[t] << 16); kf[8 * c + 2 * t + 1] = __uint_as_float(w[t] & 0xffff0000u); }
+                }
+                float best = -INFINITY;
+                for (int h = 0; h < p.G; ++h) {
+                    float acc = 0.f;
+        #pragma unroll
+                    for (int d = 0; d < D; ++d) acc = fmaf(kf[d], sq[h * D + d], acc);
+                    best = fmaxf(best, fmaf(acc, p.scale, -slse[h]));
+                }
+                return order_key(best);
+            };
+            unsigned prefix = 0, need = (unsigned)take;
+            for (int round = 0; round < 4; ++round) {
+                const int shift = 24 - 8 * round;
+                hist[tid] = 0;
+                __syncthreads();
+                for (int base = 0; base < nc; base += THREADS) {
+                    const int j = base + tid;
+                    const uint32_t kk = j < nc ? key_of(j) : 0u;
+                    const bool live = j < nc && (round == 0 || (kk >> (shift + 8)) == prefix);
+                    const unsigned digit = live ? ((kk >> shift) & 255u) : 256u;
+                    const unsigned peers = __match_any_sync(0xffffffffu, digit);
+                    if (live && lane == __ffs(peers) - 1) atomicAdd(&hist[digit], __popc(peers));
+                }
+                __syncthreads();
+                if (warp == 0) pick_digit(hist, prefix, need, lane, &s_prefix, &s_need);
+                __syncthreads();
+                prefix = s_prefix;
+                need = s_need;
             }
-            float best = -INFINITY;
-            for (int h = 0; h < p.G; ++h) {
-                float acc = 0.f;
-    #pragma unroll
-                for (int d = 0; d < D; ++d) acc = fmaf(kf[d], sq[h * D + d], acc);
-                best = fmaxf(best, fmaf(acc, p.scale, -slse[h]));
-            }
-            return order_key(best);
-        };
-        unsigned prefix = 0, need = (unsigned)take;
-        for (int round = 0; round < 4; ++round) {
-            const int shift = 24 - 8 * round;
-            hist[tid] = 0;
+            const uint32_t tau = prefix;
+            const unsigned need_eq = need;
+            if (tid == 0) { s_run_gt = 0; s_run_eq = 0; }
             __syncthreads();
             for (int base = 0; base < nc; base += THREADS) {
                 const int j = base + tid;
                 const uint32_t kk = j < nc ? key_of(j) : 0u;
-                const bool live = j < nc && (round == 0 || (kk >> (shift + 8)) == prefix);
-                const unsigned digit = live ? ((kk >> shift) & 255u) : 256u;
-                const unsigned peers = __match_any_sync(0xffffffffu, digit);
-                if (live && lane == __ffs(peers) - 1) atomicAdd(&hist[digit], __popc(peers));
+                const unsigned gt = j < nc && kk > tau, eq = j < nc && kk == tau;
+                const unsigned bg = __ballot_sync(0xffffffffu, gt), be = __ballot_sync(0xffffffffu, eq);
+                if (lane == 0) s_warp[warp] = (__popc(bg) << 16) | __popc(be);
+                __syncthreads();
+                unsigned gt_before = s_run_gt, eq_before = s_run_eq, tot_gt = 0, tot_eq = 0;
+        #pragma unroll
+                for (int w2 = 0; w2 < WARPS; ++w2) {
+                    const unsigned c = s_warp[w2];
+                    if (w2 < warp) { gt_before += c >> 16; eq_before += c & 0xffffu; }
+                    tot_gt += c >> 16; tot_eq += c & 0xffffu;
+                }
+                const unsigned lt = (1u << lane) - 1u;
+                gt_before += __popc(bg & lt);
+                eq_before += __popc(be & lt);
+                if (gt) out[gt_before + min(eq_before, need_eq)] = j;
+                else if (eq && eq_before < need_eq) out[gt_before + eq_before] = j;
+                __syncthreads();
+                if (tid == 0) { s_run_gt += tot_gt; s_run_eq += tot_eq; }
+                __syncthreads();
             }
-            __syncthreads();
-            if (warp == 0) pick_digit(hist, prefix, need, lane, &s_prefix, &s_need);
-            __syncthreads();
-            prefix = s_prefix;
-            need = s_need;
+            for (int t = take + tid; t < p.k; t += THREADS) out[t] = -1;
+                __syncthreads();   // the next row reuses the shared arrays
         }
-        const uint32_t tau = prefix;
-        const unsigned need_eq = need;
-        if (tid == 0) { s_run_gt = 0; s_run_eq = 0; }
-        __syncthreads();
-        for (int base = 0; base < nc; base += THREADS) {
-            const int j = base + tid;
-            const uint32_t kk = j < nc ? key_of(j) : 0u;
-            const unsigned gt = j < nc && kk > tau, eq = j < nc && kk == tau;
-            const unsigned bg = __ballot_sync(0xffffffffu, gt), be = __ballot_sync(0xffffffffu, eq);
-            if (lane == 0) s_warp[warp] = (__popc(bg) << 16) | __popc(be);
-            __syncthreads();
-            unsigned gt_before = s_run_gt, eq_before = s_run_eq, tot_gt = 0, tot_eq = 0;
-    #pragma unroll
-            for (int w2 = 0; w2 < WARPS; ++w2) {
-                const unsigned c = s_warp[w2];
-                if (w2 < warp) { gt_before += c >> 16; eq_before += c & 0xffffu; }
-                tot_gt += c >> 16; tot_eq += c & 0xffffu;
-            }
-            const unsigned lt = (1u << lane) - 1u;
-            gt_before += __popc(bg & lt);
-            eq_before += __popc(be & lt);
-            if (gt) out[gt_before + min(eq_before, need_eq)] = j;
-            else if (eq && eq_before < need_eq) out[gt_before + eq_before] = j;
-            __syncthreads();
-            if (tid == 0) { s_run_gt += tot_gt; s_run_eq += tot_eq; }
-            __syncthreads();
-        }
-        for (int t = take + tid; t < p.k; t += THREADS) out[t] = -1;
-        __syncthreads();   // the next row reuses the shared arrays
+        __syncthreads();   // s_flagged is rewritten for the next chunk
     }
 }
 
@@ -1754,7 +1766,7 @@ cudaError_t launch_select_recompute(const Params &p, const void *Q, const void *
     cudaError_t e = cudaGetDevice(&dev);
     if (e == cudaSuccess) e = cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
     if (e != cudaSuccess) return e;
-    const unsigned grid = (unsigned)std::min<int64_t>(n_rows, (int64_t)4 * sms);
+    const unsigned grid = (unsigned)std::min<int64_t>((n_rows + kRedoChunk - 1) / kRedoChunk, (int64_t)8 * sms);
     k_select_recompute<<<grid, 256, smem, st>>>(p, (const __nv_bfloat16 *)Q, (const __nv_bfloat16 *)K, LSE, idx, row0, n_rows,
                                                 flag);
     count_launch();
