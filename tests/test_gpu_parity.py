@@ -6,7 +6,7 @@ import torch
 import oracle
 import paper_2609_26368_b200 as hs2
 from gen import CONFIGS, make_inputs, scaled
-from parity import BlockRun, TOL, assert_output_close, check_idx_against_oracle, rows_all, to_host
+from parity import BlockRun, TOL, assert_output_close, check_idx_against_oracle, gather_rows, rows_all, to_host
 
 pytestmark = pytest.mark.gpu
 
@@ -205,6 +205,33 @@ def _filtered_equals_full_rows():
         b = BlockRun(inp).run_full(want_scores=False)
         assert torch.equal(a.idx, b.idx)
         assert hs2.hs2_device_error_flags() == 0
+
+
+def test_filtered_selection_with_ragged_lengths_offsets_and_an_explicit_scale():
+    """The filtered path under per-sequence causal offsets, cache lengths that cut the key range, and a softmax scale
+    that is not 1/sqrt(D) (the sweep compares in the accumulator's units, i.e. divides the threshold by it): same
+    indices as the selection from complete score rows, which the oracle checks."""
+    old = hs2.hs2_set_filter_min_keys(1)
+    try:
+        wl = scaled("cfg2", batch=3, q_len=600, kv_len=3000, k_sel=128, window=16, n_needles=8)
+        inp = make_inputs(wl)
+        q_start, kv_lens = [2400, 700, 0], [3000, 1500, 640]
+        qs_t = torch.tensor(q_start, dtype=torch.int32, device="cuda")
+        kl_t = torch.tensor(kv_lens, dtype=torch.int32, device="cuda")
+        q, k, v = inp.q_full.cuda(), inp.k.cuda(), inp.v.cuda()
+        for scale in (0.11, 0.023):
+            prob = hs2.Problem.from_tensors(q, k, wl.k_sel, wl.window, softmax_scale=scale, q_start=qs_t, kv_lens=kl_t)
+            Oa, LSEa, idx_a, sc = hs2.hs2_full_attn_select(prob, q, k, v, want_scores=True)    # complete rows
+            Ob, LSEb, idx_b, _ = hs2.hs2_full_attn_select(prob, q, k, v, want_scores=False)    # filtered
+            torch.cuda.synchronize()
+            assert torch.equal(idx_a, idx_b)
+            assert hs2.hs2_device_error_flags() == 0
+            rows = [(b, i) for b in range(wl.batch) for i in (0, 1, 17, 300, 598, 599)]
+            _, _, idxo, sco = oracle.full_attn_select(inp.q_full, inp.k, inp.v, wl.k_sel, wl.window, scale=scale,
+                                                      q_start=q_start, kv_lens=kv_lens, want_scores=True, rows=rows)
+            check_idx_against_oracle(gather_rows(idx_b, rows, "bgik").cpu().numpy(), idxo, sco)
+    finally:
+        hs2.hs2_set_filter_min_keys(old)
 
 
 def test_filtered_selection_breaks_ties_at_the_threshold_by_key_index():
