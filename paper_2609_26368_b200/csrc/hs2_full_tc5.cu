@@ -367,11 +367,13 @@ k_full_tc5(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUte
 // One CTA = TQ = NC/G consecutive queries of one (sequence, KV head) x one chunk of keys.  The MMA
 // computes S^T = K Q^T: 128 keys on M (TMEM lane = key), the TQ x G (query, head) pairs on N = NC columns,
 // so the G heads of a query are adjacent TMEM columns of one lane and their maximum is thread local.
-// Warp 8 feeds K tiles by TMA (2-stage ring), warp 9 issues the MMAs into two accumulator buffers,
-// warps 0-7 (thread = key; warps w and w+4 share the 32 TMEM lanes of quarter w and take 64 columns each)
-// subtract LSE, take the group maximum and write 32 consecutive keys of a strip row per warp instruction.
-// The epilogue is a chain of TMEM loads and short dependent arithmetic: eight warps per CTA hide its latency
-// where four left the tensor pipe waiting for a free accumulator.
+// The subtraction of LSE is one more K step of the same MMA (a key operand of ones against -LSE / scale split into
+// three bf16 terms), so the accumulator holds (score / scale) of every (key, query, head).  One warp feeds K tiles by
+// TMA (a ring of 2 or 3 stages), one thread issues the MMAs into two accumulator buffers, NC / 16 epilogue warps
+// (thread = key; the warps that share the 32 TMEM lanes of a quarter take 64 columns each) take the group maximum and,
+// by mode, write 32 consecutive keys of a strip row per warp instruction or append the scores that pass the query's
+// threshold to its candidate list.  The epilogue is a chain of TMEM loads and short dependent arithmetic: eight warps
+// per 128 columns hide its latency where four left the tensor pipe waiting for a free accumulator.
 #ifndef HS2_SC_KSTAGES
 #define HS2_SC_KSTAGES 3   // key tiles in flight in a 256-column CTA (2 to 5); measured on the 128K layer: 2: 221 ms, 3: 219 ms, 4: 237 ms
 #endif
