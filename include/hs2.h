@@ -86,6 +86,10 @@ typedef struct {
                                         individual tokens (the paper's method); B > 1 = aligned blocks of B tokens,
                                         the block-level variant the paper ablates against (Section 5, Ablation 1:
                                         block size 64, 1024 tokens = 16 blocks); k_sel must then be a multiple of B */
+    int64_t kv_scale_stride[3];      /* FP8 cache entry points only: floats between the scales of consecutive
+                                        (batch, token, KV head) entries, shared by the K and the V scales; all 0 =>
+                                        packed [batch, kv_len, n_kv_heads].  With kv_stride this lets a cache keep the K
+                                        codes, the V codes and both scales of a (token, KV head) in one record */
 } hs2_problem;
 
 /* Bytes of scratch `op` needs for this problem (a host-side computation; 0 is a valid answer).
@@ -173,7 +177,11 @@ hs2_status hs2_sparse_attn_decode_gated(const hs2_problem *p, const void *Q, con
  *   K8, V8   in  e4m3 codes (1 byte: sign, 4 exponent bits with bias 7, 3 mantissa bits; no infinities, the two
  *                NaN codes are a caller error) [batch, kv_len, n_kv_heads, head_dim]; p->kv_stride counts codes
  *                (= bytes), multiples of 16, or 0 for packed.
- *   k_scale, v_scale  in  float [batch, kv_len, n_kv_heads], packed: the cache value is code * scale.
+ *   k_scale, v_scale  in  float [batch, kv_len, n_kv_heads]: the cache value is code * scale.  Packed, or with the
+ *                strides p->kv_scale_stride gives (floats; shared by the two arrays).  Codes and scales may live in one
+ *                buffer of records, e.g. 288 bytes [K codes | V codes | K scale | V scale | spare] per (token, KV head)
+ *                at head_dim 128: the documented layout for decode-heavy use, since an attended token then costs one
+ *                DRAM page instead of four (see hs2_kv_project_fp8_records, which writes it).
  *   Q, O, LSE, idx, sink as for the bf16 calls; p->dtype describes Q and O and must be HS2_BF16.
  * Covers head_dim 128 and 256 with up to 128 query heads per KV head (the paper's own shape, 64 heads on one KV
  * head at head_dim 256, included) and 16-byte aligned tensors; anything else returns HS2_ERR_UNSUPPORTED.  At
@@ -254,6 +262,26 @@ hs2_status hs2_sparse_attn_decode_static(const hs2_problem *p, const void *Q, co
  */
 hs2_status hs2_kv_project(int64_t n_tokens, int32_t d_model, int32_t n_out, const void *H, int64_t ldh, const void *W,
                           int64_t ldw, void *C, int64_t ldc, float *scales, void *cuda_stream);
+
+/*
+ * The e4m3 form of hs2_kv_project writing into a cache of records, so that the K codes, the V codes and both scales
+ * of a (token, KV head) can sit side by side (one DRAM page per attended token and head instead of four; on the 64K
+ * decode step of the benchmark the sparse layer then takes 39.7 us instead of 43.7).  A column group g is the 128
+ * consecutive output columns 128 g .. 128 g + 127 (one head of dim 128):
+ *   codes of token t, group g   at byte  t * ldc + g * ld_group  of C   (128 bytes)
+ *   their scale                 at       scales[t * scale_ld_token + g * scale_ld_group]
+ * Example, records of 288 bytes [K 128 | V 128 | K scale | V scale | 24 spare] per (token, KV head) - a whole number
+ * of 32-byte sectors, which measured 39.7 us against 40.7 us for records of 272 bytes - with n_kv_heads heads: the K
+ * projection is called with C = cache, ldc = 288 n_kv_heads, ld_group = 288, scales = (float *)(cache + 256),
+ * scale_ld_token = 72 n_kv_heads, scale_ld_group = 72; the V projection with C = cache + 128 and
+ * scales = (float *)(cache + 260).  The attention calls read such a cache through kv_stride = {tokens * 288 n_kv_heads,
+ * 288 n_kv_heads, 288} and kv_scale_stride = {tokens * 72 n_kv_heads, 72 n_kv_heads, 72}.
+ * ld_group >= 128; ldc and ld_group multiples of 16 bytes; ldc >= (n_out / 128 - 1) * ld_group + 128; the other
+ * conditions and the arithmetic are those of hs2_kv_project.
+ */
+hs2_status hs2_kv_project_fp8_records(int64_t n_tokens, int32_t d_model, int32_t n_out, const void *H, int64_t ldh,
+                                      const void *W, int64_t ldw, void *C, int64_t ldc, int64_t ld_group, float *scales,
+                                      int64_t scale_ld_token, int64_t scale_ld_group, void *cuda_stream);
 
 /*
  * Measurement aid for hs2_sparse_attn_prefill (the gather of Section 3.3; no counterpart in the paper): performs

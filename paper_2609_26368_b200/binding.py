@@ -26,6 +26,7 @@ HS2_OP_FULL_ATTN_SELECT_FP8KV = 4
 EXPORTS = ["hs2_workspace_bytes", "hs2_full_attn_select", "hs2_topk_select", "hs2_sparse_attn_prefill",
            "hs2_sparse_attn_decode", "hs2_sparse_attn_prefill_gated", "hs2_sparse_attn_decode_gated",
            "hs2_sparse_attn_prefill_fp8kv", "hs2_sparse_attn_decode_fp8kv", "hs2_full_attn_select_fp8kv", "hs2_kv_project",
+           "hs2_kv_project_fp8_records",
            "hs2_sparse_attn_decode_static", "hs2_probe_gather", "hs2_status_string", "hs2_last_cuda_error",
            "hs2_launch_count", "hs2_device_error_flags", "hs2_set_filter_min_keys", "hs2_set_tcgen05_enabled"]
 
@@ -42,7 +43,7 @@ class _CProblem(C.Structure):
                 ("k_sel", C.c_int32), ("window", C.c_int32), ("softmax_scale", C.c_float),
                 ("dtype", C.c_int), ("q_start", C.c_void_p), ("kv_lens", C.c_void_p),
                 ("q_stride", C.c_int64 * 3), ("kv_stride", C.c_int64 * 3), ("o_stride", C.c_int64 * 3),
-                ("select_block", C.c_int32)]
+                ("select_block", C.c_int32), ("kv_scale_stride", C.c_int64 * 3)]
 
 
 _lib = None
@@ -76,6 +77,9 @@ def load_library():
         lib.hs2_sparse_attn_decode_gated.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
         lib.hs2_kv_project.argtypes = [C.c_int64, C.c_int32, C.c_int32, vp, C.c_int64, vp, C.c_int64, vp, C.c_int64, vp, vp]
         lib.hs2_kv_project.restype = C.c_int
+        lib.hs2_kv_project_fp8_records.argtypes = [C.c_int64, C.c_int32, C.c_int32, vp, C.c_int64, vp, C.c_int64, vp, C.c_int64,
+                                                   C.c_int64, vp, C.c_int64, C.c_int64, vp]
+        lib.hs2_kv_project_fp8_records.restype = C.c_int
         lib.hs2_sparse_attn_prefill_fp8kv.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         lib.hs2_sparse_attn_decode_fp8kv.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, vp]
         lib.hs2_full_attn_select_fp8kv.argtypes = [pp, vp, vp, vp, vp, vp, vp, vp, vp, vp, sz, vp]
@@ -276,8 +280,9 @@ def _sparse_fp8(fn_name, prob, q, k8, v8, k_scale, v_scale, idx, sink, out, lse,
         assert tuple(t.shape) == (prob.batch, prob.kv_len, prob.n_kv_heads, prob.head_dim)
     assert k8.stride() == v8.stride()
     for t in (k_scale, v_scale):
-        assert t.is_cuda and t.dtype == torch.float32 and t.is_contiguous()
+        assert t.is_cuda and t.dtype == torch.float32
         assert tuple(t.shape) == (prob.batch, prob.kv_len, prob.n_kv_heads)
+    assert k_scale.stride() == v_scale.stride()   # may be views into records that also hold the codes
     if idx is not None:
         assert idx.dtype == torch.int32 and idx.is_contiguous() and idx.is_cuda
         assert tuple(idx.shape) == (prob.batch, prob.n_kv_heads, prob.q_len, prob.k_sel)
@@ -287,6 +292,7 @@ def _sparse_fp8(fn_name, prob, q, k8, v8, k_scale, v_scale, idx, sink, out, lse,
     if lse is None and want_lse:
         lse = torch.empty(prob.batch, prob.n_q_heads, prob.q_len, dtype=torch.float32, device=q.device)
     c = prob.c_struct(q, k8, out)
+    c.kv_scale_stride = (C.c_int64 * 3)(*k_scale.stride())
     st = getattr(load_library(), fn_name)(C.byref(c), _dp(q), _dp(k8), _dp(v8), _dp(k_scale), _dp(v_scale), _dp(idx),
                                           _dp(sink), _dp(out), _dp(lse), _stream(stream))
     _check(st, fn_name)
@@ -302,8 +308,9 @@ def hs2_full_attn_select_fp8kv(prob: Problem, q, k8, v8, k_scale, v_scale, *, ou
         assert tuple(t.shape) == (prob.batch, prob.kv_len, prob.n_kv_heads, prob.head_dim)
     assert k8.stride() == v8.stride()
     for t in (k_scale, v_scale):
-        assert t.is_cuda and t.dtype == torch.float32 and t.is_contiguous()
+        assert t.is_cuda and t.dtype == torch.float32
         assert tuple(t.shape) == (prob.batch, prob.kv_len, prob.n_kv_heads)
+    assert k_scale.stride() == v_scale.stride()   # may be views into records that also hold the codes
     dev = q.device
     out = torch.empty_like(q) if out is None else out
     lse = torch.empty(prob.batch, prob.n_q_heads, prob.q_len, dtype=torch.float32, device=dev) if lse is None else lse
@@ -312,6 +319,7 @@ def hs2_full_attn_select_fp8kv(prob: Problem, q, k8, v8, k_scale, v_scale, *, ou
     if idx is not None:
         ws = _workspace(prob, HS2_OP_FULL_ATTN_SELECT_FP8KV, dev, ws)
     c = prob.c_struct(q, k8, out)
+    c.kv_scale_stride = (C.c_int64 * 3)(*k_scale.stride())
     st = load_library().hs2_full_attn_select_fp8kv(C.byref(c), _dp(q), _dp(k8), _dp(v8), _dp(k_scale), _dp(v_scale), _dp(out),
                                                    _dp(lse), _dp(idx), _dp(ws), 0 if ws is None else ws.numel(), _stream(stream))
     _check(st, "hs2_full_attn_select_fp8kv")
@@ -350,6 +358,23 @@ def hs2_kv_project(h, w, *, out=None, fp8=False, scales=None, stream=None):
                                        _dp(scales) if fp8 else None, _stream(stream))
     _check(st, "hs2_kv_project")
     return (out, scales) if fp8 else out
+
+
+def hs2_kv_project_fp8_records(h, w, codes, scales, *, stream=None):
+    """Cache producer writing e4m3 codes and scales into records: ``codes`` is a uint8 view ``[T, G, 128]`` (G column
+    groups = heads of dim 128, any 16-byte-multiple strides between tokens and groups, the 128 codes contiguous),
+    ``scales`` a float32 view ``[T, G]``; both may point into the same buffer.  Returns ``(codes, scales)``."""
+    assert h.is_cuda and w.is_cuda and h.dtype == torch.bfloat16 and w.dtype == torch.bfloat16
+    assert h.dim() == 2 and w.dim() == 2 and h.shape[1] == w.shape[1] and h.stride(1) == 1 and w.stride(1) == 1
+    T, dm = h.shape
+    N = w.shape[0]
+    assert codes.dtype == torch.uint8 and tuple(codes.shape) == (T, N // 128, 128) and codes.stride(2) == 1
+    assert scales.dtype == torch.float32 and tuple(scales.shape) == (T, N // 128)
+    st = load_library().hs2_kv_project_fp8_records(T, dm, N, _dp(h), h.stride(0), _dp(w), w.stride(0), _dp(codes),
+                                                   codes.stride(0), codes.stride(1), _dp(scales), scales.stride(0),
+                                                   scales.stride(1), _stream(stream))
+    _check(st, "hs2_kv_project_fp8_records")
+    return codes, scales
 
 
 def hs2_probe_gather(prob: Problem, k, v, idx, *, mode=0, sink_word=None, stream=None):

@@ -57,6 +57,12 @@ hs2_status resolve(const hs2_problem *hp, bool need_tensors, Params *out)
         if (!strides(hp->q_stride, p.Lq, p.Hq, p.D, p.qs_b, p.qs_t, p.qs_h)) return HS2_ERR_INVALID_ARG;
         if (!strides(hp->kv_stride, p.Lk, p.Hkv, p.D, p.ks_b, p.ks_t, p.ks_h)) return HS2_ERR_INVALID_ARG;
         if (!strides(hp->o_stride, p.Lq, p.Hq, p.D, p.os_b, p.os_t, p.os_h)) return HS2_ERR_INVALID_ARG;
+        {   // scales of an FP8 cache: one float per (batch, token, KV head)
+            const int64_t *s = hp->kv_scale_stride;
+            if (s[0] == 0 && s[1] == 0 && s[2] == 0) { p.ss_h = 1; p.ss_t = p.Hkv; p.ss_b = (int64_t)p.Lk * p.Hkv; }
+            else if (s[0] >= 0 && s[1] >= 0 && s[2] >= 1) { p.ss_b = s[0]; p.ss_t = s[1]; p.ss_h = s[2]; }
+            else return HS2_ERR_INVALID_ARG;
+        }
     } else {
         p.G = 1;
     }
@@ -593,6 +599,28 @@ hs2_status hs2_kv_project(int64_t n_tokens, int32_t d_model, int32_t n_out, cons
     hs2_status s = check_device();
     if (s != HS2_OK) return s;
     const cudaError_t e = launch_kv_project(n_tokens, n_out, d_model, H, ldh, W, ldw, C, ldc, scales, (cudaStream_t)cuda_stream);
+    if (e == cudaErrorNotSupported) {
+        (void)cudaGetLastError();
+        return HS2_ERR_UNSUPPORTED;
+    }
+    return e == cudaSuccess ? HS2_OK : cuda_fail(e);
+}
+
+hs2_status hs2_kv_project_fp8_records(int64_t n_tokens, int32_t d_model, int32_t n_out, const void *H, int64_t ldh,
+                                      const void *W, int64_t ldw, void *C, int64_t ldc, int64_t ld_group, float *scales,
+                                      int64_t scale_ld_token, int64_t scale_ld_group, void *cuda_stream)
+{
+    if (n_tokens < 0 || d_model <= 0 || n_out <= 0 || !H || !W || !C || !scales) return HS2_ERR_INVALID_ARG;
+    if (ld_group < 128 || scale_ld_token < 0 || scale_ld_group < 0) return HS2_ERR_INVALID_ARG;
+    if (n_tokens == 0) return HS2_OK;
+    // (the row stride only has to hold what a token's groups span, not n_out packed bytes)
+    if (!kv_project_supported(n_tokens, n_out, d_model, ldh, ldw, (int64_t)n_out, true) || ldc % 16 != 0 || ld_group % 16 != 0 ||
+        ldc < (n_out / 128 - 1) * ld_group + 128 || !aligned16(H, W, C, C) || (reinterpret_cast<uintptr_t>(scales) & 3u))
+        return HS2_ERR_UNSUPPORTED;
+    hs2_status s = check_device();
+    if (s != HS2_OK) return s;
+    const cudaError_t e = launch_kv_project_records(n_tokens, n_out, d_model, H, ldh, W, ldw, C, ldc, ld_group, scales,
+                                                    scale_ld_token, scale_ld_group, (cudaStream_t)cuda_stream);
     if (e == cudaErrorNotSupported) {
         (void)cudaGetLastError();
         return HS2_ERR_UNSUPPORTED;

@@ -21,6 +21,7 @@ struct Params {
     int64_t qs_b, qs_t, qs_h;   // element strides
     int64_t ks_b, ks_t, ks_h;
     int64_t os_b, os_t, os_h;
+    int64_t ss_b, ss_t, ss_h;   // FP8 cache: strides of the scale arrays, in floats
     int share;          // > 1: consecutive groups of `share` KV-head slots are one real KV head seen through sub-groups
                         // of its query heads (K, V and idx are indexed by slot / share); 0 or 1: plain
     int blk;            // selection granularity: 1 = tokens, B > 1 = aligned blocks of B tokens
@@ -163,6 +164,10 @@ cudaError_t launch_scores_fp8_decode(const Params &p, const void *Q, const void 
 bool kv_project_supported(int64_t T, int N, int dm, int64_t ldh, int64_t ldw, int64_t ldc, bool fp8);
 cudaError_t launch_kv_project(int64_t T, int N, int dm, const void *H, int64_t ldh, const void *W, int64_t ldw, void *C,
                               int64_t ldc, float *scales, cudaStream_t st);
+// the e4m3 output with a stride between the 128-column groups and strided scales (records that hold codes and scales)
+cudaError_t launch_kv_project_records(int64_t T, int N, int dm, const void *H, int64_t ldh, const void *W, int64_t ldw,
+                                      void *C, int64_t ldc, int64_t ld_group, float *scales, int64_t s_tok, int64_t s_grp,
+                                      cudaStream_t st);
 cudaError_t read_kvproj_error(unsigned *out);
 // the row fetches of the sparse prefill and nothing else (measurement aid); mode 0: L2 loads, 1: through L1
 cudaError_t launch_probe_gather(const Params &p, const void *K, const void *V, const int32_t *idx, int mode,

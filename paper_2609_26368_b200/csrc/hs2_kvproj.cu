@@ -56,11 +56,19 @@ __device__ __forceinline__ uint32_t cvt_f32x2_e4m3(float lo, float hi)
     return d;
 }
 
+// Where the e4m3 output goes: the codes of token t, column group g (columns 128 g .. 128 g + 127) start at byte
+// t * ldc + g * ld_group of C, their scale is scales[t * s_tok + g * s_grp].  (Packed: ld_group = 128, s_tok = N / 128,
+// s_grp = 1; a cache of records holds a group's codes and its scale side by side.)
+struct ScaleOut {
+    float *scales;
+    int64_t ld_group, s_tok, s_grp;
+};
+
 // Epilogue of one 128 x 256 accumulator for the thread that owns output row `tok`: bf16, or e4m3 codes with one scale
 // per 128 columns.  `release` is called once, as soon as the last accumulator column is in registers.
 template <bool FP8, class Release>
 __device__ __forceinline__ void epilogue_rows(uint32_t acc, int64_t tok, int64_t T, int n0, int N, void *C, int64_t ldc,
-                                      float *scales, Release release)
+                                      const ScaleOut so, Release release)
 {
     if (!FP8) {
         __nv_bfloat16 *crow = static_cast<__nv_bfloat16 *>(C) + tok * ldc + n0;
@@ -86,9 +94,10 @@ __device__ __forceinline__ void epilogue_rows(uint32_t acc, int64_t tok, int64_t
             }
         }
     } else {
-        uint8_t *crow = static_cast<uint8_t *>(C) + tok * ldc + n0;
 #pragma unroll 1
         for (int grp = 0; grp < BN / kQuantGroup; ++grp) {
+            const int gi = n0 / kQuantGroup + grp;   // column group of the output
+            uint8_t *crow = static_cast<uint8_t *>(C) + tok * ldc + gi * so.ld_group;
             // pass 1: the group's largest magnitude; pass 2: re-read the accumulator and encode
             float amax = 0.f;
 #pragma unroll 1
@@ -101,7 +110,7 @@ __device__ __forceinline__ void epilogue_rows(uint32_t acc, int64_t tok, int64_t
             }
             const float scale = amax > 0.f ? amax / 448.f : 1.f;
             const float inv = 1.f / scale;
-            if (tok < T) scales[tok * (N / kQuantGroup) + (n0 + grp * kQuantGroup) / kQuantGroup] = scale;
+            if (tok < T) so.scales[tok * so.s_tok + gi * so.s_grp] = scale;
 #pragma unroll 1
             for (int c = 0; c < kQuantGroup / 32; ++c) {
                 float v[32];
@@ -120,7 +129,7 @@ __device__ __forceinline__ void epilogue_rows(uint32_t acc, int64_t tok, int64_t
                             const float *x = v + 16 * q4 + 4 * u;
                             w4[u] = cvt_f32x2_e4m3(x[0] * inv, x[1] * inv) | (cvt_f32x2_e4m3(x[2] * inv, x[3] * inv) << 16);
                         }
-                        *reinterpret_cast<uint4 *>(crow + grp * kQuantGroup + c * 32 + q4 * 16) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
+                        *reinterpret_cast<uint4 *>(crow + c * 32 + q4 * 16) = make_uint4(w4[0], w4[1], w4[2], w4[3]);
                     }
                 }
             }
@@ -131,7 +140,7 @@ __device__ __forceinline__ void epilogue_rows(uint32_t acc, int64_t tok, int64_t
 template <bool FP8>
 __global__ void __launch_bounds__(kThreads, 1)
 k_kv_project(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtensorMap tmW, int64_t T, int N, int dm,
-             void *__restrict__ C, int64_t ldc, float *__restrict__ scales)
+             void *__restrict__ C, int64_t ldc, const ScaleOut so)
 {
     extern __shared__ char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -226,7 +235,7 @@ k_kv_project(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CU
             ok = __all_sync(0xffffffffu, mbar_wait(bar(ACC_FULL0 + ab), (i >> 1) & 1, abort_flag));
             if (!ok) break;
             tc_fence_after();
-            epilogue_rows<FP8>(acc, tok, T, n0, N, C, ldc, scales, [&] { mbar_arrive(bar(ACC_EMPTY0 + ab)); });
+            epilogue_rows<FP8>(acc, tok, T, n0, N, C, ldc, so, [&] { mbar_arrive(bar(ACC_EMPTY0 + ab)); });
         }
     }
     // ------------------------------------------------ teardown
@@ -298,7 +307,7 @@ __device__ __forceinline__ void umma2_commit_both(uint32_t bar)
 template <bool FP8>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 k_kv_project_pair(const __grid_constant__ CUtensorMap tmH, const __grid_constant__ CUtensorMap tmW, int64_t T, int N, int dm,
-                  void *__restrict__ C, int64_t ldc, float *__restrict__ scales)
+                  void *__restrict__ C, int64_t ldc, const ScaleOut so)
 {
     extern __shared__ char smem_raw[];
     const uint32_t raw = smem_u32(smem_raw);
@@ -398,7 +407,7 @@ k_kv_project_pair(const __grid_constant__ CUtensorMap tmH, const __grid_constant
             ok = __all_sync(0xffffffffu, mbar_wait(bar(P_ACC_FULL0 + ab), (i >> 1) & 1, abort_flag));
             if (!ok) break;
             tc_fence_after();
-            epilogue_rows<FP8>(acc, tok, T, n0, N, C, ldc, scales, [&] {
+            epilogue_rows<FP8>(acc, tok, T, n0, N, C, ldc, so, [&] {
                 if (rank == 0) {
                     mbar_arrive(bar(P_ACC_EMPTY0 + ab));
                 } else {
@@ -423,7 +432,7 @@ k_kv_project_pair(const __grid_constant__ CUtensorMap tmH, const __grid_constant
 
 template <bool FP8>
 cudaError_t launch(int64_t T, int N, int dm, const void *H, int64_t ldh, const void *W, int64_t ldw, void *C, int64_t ldc,
-                   float *scales, cudaStream_t st)
+                   const ScaleOut so, cudaStream_t st)
 {
     CUtensorMap tmH, tmW;
     // [1, rows, 1, d_model] views: token stride ld, a single "head"
@@ -454,7 +463,7 @@ cudaError_t launch(int64_t T, int N, int dm, const void *H, int64_t ldh, const v
             const int64_t n_tiles2 = ((T + 255) / 256) * (N / 256);
             const int64_t pairs = n_tiles2 < n_sm[dev] / 2 ? n_tiles2 : n_sm[dev] / 2;
             if (pairs >= 1) {
-                k_kv_project_pair<FP8><<<(unsigned)(2 * pairs), kThreads, kPSmemBytes, st>>>(tmH, tmW2, T, N, dm, C, ldc, scales);
+                k_kv_project_pair<FP8><<<(unsigned)(2 * pairs), kThreads, kPSmemBytes, st>>>(tmH, tmW2, T, N, dm, C, ldc, so);
                 count_launch();
                 return cudaGetLastError();
             }
@@ -463,7 +472,7 @@ cudaError_t launch(int64_t T, int N, int dm, const void *H, int64_t ldh, const v
 #endif
     const int64_t n_tiles = ((T + BM - 1) / BM) * (N / BN);
     const unsigned grid = (unsigned)(n_tiles < n_sm[dev] ? n_tiles : n_sm[dev]);
-    k_kv_project<FP8><<<grid, kThreads, kSmemBytes, st>>>(tmH, tmW, T, N, dm, C, ldc, scales);
+    k_kv_project<FP8><<<grid, kThreads, kSmemBytes, st>>>(tmH, tmW, T, N, dm, C, ldc, so);
     count_launch();
     return cudaGetLastError();
 }
@@ -480,8 +489,17 @@ cudaError_t launch_kv_project(int64_t T, int N, int dm, const void *H, int64_t l
                               int64_t ldc, float *scales, cudaStream_t st)
 {
     if (!tma_available()) return cudaErrorNotSupported;
-    return scales ? launch<true>(T, N, dm, H, ldh, W, ldw, C, ldc, scales, st)
-                  : launch<false>(T, N, dm, H, ldh, W, ldw, C, ldc, nullptr, st);
+    const ScaleOut so{scales, kQuantGroup, N / kQuantGroup, 1};
+    return scales ? launch<true>(T, N, dm, H, ldh, W, ldw, C, ldc, so, st)
+                  : launch<false>(T, N, dm, H, ldh, W, ldw, C, ldc, so, st);
+}
+
+cudaError_t launch_kv_project_records(int64_t T, int N, int dm, const void *H, int64_t ldh, const void *W, int64_t ldw,
+                                      void *C, int64_t ldc, int64_t ld_group, float *scales, int64_t s_tok, int64_t s_grp,
+                                      cudaStream_t st)
+{
+    if (!tma_available()) return cudaErrorNotSupported;
+    return launch<true>(T, N, dm, H, ldh, W, ldw, C, ldc, ScaleOut{scales, ld_group, s_tok, s_grp}, st);
 }
 
 cudaError_t read_kvproj_error(unsigned *out) { return cudaMemcpyFromSymbol(out, g_kvproj_error, sizeof(unsigned)); }

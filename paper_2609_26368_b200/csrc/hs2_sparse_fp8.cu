@@ -131,7 +131,7 @@ struct Item {
     const char *Kb, *Vb;          // first row of this (sequence, KV head)
     const float *ksc, *vsc;       // its scales: element j * Hkv
     int64_t row_stride;           // bytes between consecutive tokens
-    int sc_stride;                // floats between consecutive tokens' scales
+    int64_t sc_stride;            // floats between consecutive tokens' scales
     const int32_t *irow;
     int pos, kvl;
     float *raw;                   // decode-shaped full layer: dequantised q.k of every (head, key) goes here, or null
@@ -148,10 +148,10 @@ __device__ __forceinline__ Item make_item(const Params &p, const uint8_t *K, con
     const int64_t base = b * p.ks_b + g_real * p.ks_h;
     it.Kb = reinterpret_cast<const char *>(K + base);
     it.Vb = reinterpret_cast<const char *>(V + base);
-    it.ksc = ksc + (int64_t)b * p.Lk * hkv_real + g_real;
-    it.vsc = vsc + (int64_t)b * p.Lk * hkv_real + g_real;
+    it.ksc = ksc + b * p.ss_b + g_real * p.ss_h;
+    it.vsc = vsc + b * p.ss_b + g_real * p.ss_h;
     it.row_stride = p.ks_t;
-    it.sc_stride = hkv_real;
+    it.sc_stride = p.ss_t;
     it.irow = idx ? idx + (((int64_t)b * hkv_real + g_real) * p.Lq + i) * p.k : nullptr;
     it.pos = pos_of(p, b, i);
     it.kvl = kvlen_of(p, b);
@@ -615,7 +615,7 @@ k_scores_fp8_decode(const Params p, const __nv_bfloat16 *__restrict__ Q, const u
     float *orow = out + (int64_t)bg * out_stride;
     const uint8_t *kbase = K + b * p.ks_b + gkv * p.ks_h;
     const int64_t rs = p.ks_t;                                   // bytes between consecutive tokens
-    const float *ksb = ksc + ((int64_t)b * p.Lk) * p.Hkv + gkv;
+    const float *ksb = ksc + b * p.ss_b + gkv * p.ss_h;
     for (int j0 = (blockIdx.x * kScF8Warps + warp) * 16; j0 < n_keys; j0 += gridDim.x * kScF8Warps * 16) {
         const int ja = j0 + g, jb = j0 + g + 8;                  // this thread's two keys
         const bool va = ja < n_keys, vb = jb < n_keys;
@@ -625,8 +625,8 @@ k_scores_fp8_decode(const Params p, const __nv_bfloat16 *__restrict__ Q, const u
             ca[c] = va ? __ldg(reinterpret_cast<const uint4 *>(kbase + (int64_t)ja * rs + 64 * c + 16 * t)) : make_uint4(0u, 0u, 0u, 0u);
             cb[c] = vb ? __ldg(reinterpret_cast<const uint4 *>(kbase + (int64_t)jb * rs + 64 * c + 16 * t)) : make_uint4(0u, 0u, 0u, 0u);
         }
-        const float fa = va ? __ldg(ksb + (int64_t)ja * p.Hkv) * p.scale : 0.f;
-        const float fb = vb ? __ldg(ksb + (int64_t)jb * p.Hkv) * p.scale : 0.f;
+        const float fa = va ? __ldg(ksb + (int64_t)ja * p.ss_t) * p.scale : 0.f;
+        const float fb = vb ? __ldg(ksb + (int64_t)jb * p.ss_t) * p.scale : 0.f;
         float best_a = -INFINITY, best_b = -INFINITY;
         for (int nt = 0; nt < NT; ++nt) {
             float acc[4] = {0.f, 0.f, 0.f, 0.f};

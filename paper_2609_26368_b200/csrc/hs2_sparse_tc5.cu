@@ -296,7 +296,7 @@ k_sparse_tc5(const __grid_constant__ CUtensorMap tmQ, const Params p, const void
             if (F8) {
                 const int j0 = slot_fix(p, jn, q.pos, q.kvl, my_slot);
                 if (j0 >= 0) {
-                    const int64_t so = ((int64_t)q.b * p.Lk + j0) * p.Hkv + q.gkv;
+                    const int64_t so = q.b * p.ss_b + (int64_t)j0 * p.ss_t + q.gkv * p.ss_h;
                     ks_cur = __ldg(ksc + so);
                     vs_cur = __ldg(vsc + so);
                 }
@@ -316,7 +316,7 @@ k_sparse_tc5(const __grid_constant__ CUtensorMap tmQ, const Params p, const void
                     if (t + 1 < nblk) {
                         const int j1 = slot_fix(p, jn, q.pos, q.kvl, my_slot + (t + 1) * BN);
                         if (j1 >= 0) {
-                            const int64_t so = ((int64_t)q.b * p.Lk + j1) * p.Hkv + q.gkv;
+                            const int64_t so = q.b * p.ss_b + (int64_t)j1 * p.ss_t + q.gkv * p.ss_h;
                             ks_cur = __ldg(ksc + so);
                             vs_cur = __ldg(vsc + so);
                         }

@@ -498,6 +498,61 @@ def test_fp8_kv_cache_sparse_prefill_and_decode():
         hs2.hs2_sparse_attn_prefill_fp8kv(prob, inp.q_full, k8, k8, ksc, ksc, idx)
 
 
+def _fp8_records(k8, v8, ksc, vsc):
+    """One record per (token, KV head): [K codes | V codes | K scale | V scale | pad to 32 bytes]; returns views."""
+    B, Lk, Hkv, D = k8.shape
+    rec_bytes = (2 * D + 8 + 31) // 32 * 32
+    rec = torch.zeros(B, Lk, Hkv, rec_bytes, dtype=torch.uint8, device=k8.device)
+    rec[..., :D].copy_(k8)
+    rec[..., D:2 * D].copy_(v8)
+    recf = rec.view(torch.float32)                       # [B, Lk, Hkv, rec_bytes / 4]
+    recf[..., 2 * D // 4].copy_(ksc)
+    recf[..., 2 * D // 4 + 1].copy_(vsc)
+    return rec[..., :D], rec[..., D:2 * D], recf[..., 2 * D // 4], recf[..., 2 * D // 4 + 1]
+
+
+def test_fp8_cache_as_one_record_per_token_and_head():
+    """K codes, V codes and both scales of a (token, KV head) in one record (kv_stride and kv_scale_stride describe it):
+    every FP8 entry point gives bit for bit what it gives on four separate packed arrays, which the tests above hold
+    against the oracle."""
+    from gen.workloads import quantize_kv_e4m3
+    cases = [
+        dict(q_len=130, kv_len=700, k_sel=96, window=24, batch=2),                                        # mma.sync kernels, group of 8
+        dict(q_len=100, kv_len=520, k_sel=64, window=16, n_q_heads=64, n_kv_heads=4),                     # group of 16: two sub-groups
+        dict(q_len=96, kv_len=448, k_sel=80, window=32, n_q_heads=64, n_kv_heads=1, head_dim=256),       # tcgen05 gather kernel
+        dict(q_len=80, kv_len=400, k_sel=50, window=10, n_q_heads=48, n_kv_heads=2, head_dim=128, batch=2),
+    ]
+    for over in cases:
+        wl = scaled("cfg2", n_needles=4, **over)
+        inp = make_inputs(wl)
+        run = BlockRun(inp).run_full()
+        k8, ksc = quantize_kv_e4m3(run.k)
+        v8, vsc = quantize_kv_e4m3(run.v)
+        rk, rv, rks, rvs = _fp8_records(k8, v8, ksc, vsc)
+        assert not rks.is_contiguous() and rk.stride() == rv.stride()
+        q = run.qs[0]
+        prob = hs2.Problem.from_tensors(q, k8, wl.k_sel, wl.window)
+        a, la = hs2.hs2_sparse_attn_prefill_fp8kv(prob, q, k8, v8, ksc, vsc, run.idx, want_lse=True)
+        b, lb = hs2.hs2_sparse_attn_prefill_fp8kv(prob, q, rk, rv, rks, rvs, run.idx, want_lse=True)
+        torch.cuda.synchronize()
+        assert torch.equal(a, b) and torch.equal(la, lb)
+        q1 = q[:, -1:].contiguous()
+        idx1 = run.idx[:, :, -1:].contiguous()
+        prob1 = hs2.Problem.from_tensors(q1, k8, wl.k_sel, wl.window)
+        a, la = hs2.hs2_sparse_attn_decode_fp8kv(prob1, q1, k8, v8, ksc, vsc, idx1, want_lse=True)
+        b, lb = hs2.hs2_sparse_attn_decode_fp8kv(prob1, q1, rk, rv, rks, rvs, idx1, want_lse=True)
+        torch.cuda.synchronize()
+        assert_output_close(b[:, 0].float(), a[:, 0].double().cpu().numpy(), wl.torch_dtype, "record layout, decode O")
+        assert float((la - lb).abs().max()) <= 1e-5      # (the splits of a decode step may merge in another order)
+        qf = run.q[:, -1:].contiguous()
+        Oa, La, ia = hs2.hs2_full_attn_select_fp8kv(prob1, qf, k8, v8, ksc, vsc)
+        Ob, Lb, ib = hs2.hs2_full_attn_select_fp8kv(prob1, qf, rk, rv, rks, rvs)
+        torch.cuda.synchronize()
+        assert torch.equal(ia, ib)
+        assert_output_close(Ob[:, 0].float(), Oa[:, 0].double().cpu().numpy(), wl.torch_dtype, "record layout, full-layer decode O")
+        assert hs2.hs2_device_error_flags() == 0
+
+
 def test_fp8_kv_cache_on_large_head_groups_and_head_dim_256():
     """The e4m3 cache at the paper's own attention shape (Table 1: 64 query heads on one KV head, head_dim 256; the cost
     analysis of Section 4 assumes FP8 storage) and on other shapes of the tensor-core gather kernel, which dequantises
@@ -676,6 +731,23 @@ def test_kv_projection_bf16_and_fp8_outputs():
     vd = oracle.dequant_e4m3(v8.contiguous(), vsc)
     Oo, _, _ = oracle.sparse_attn(q.float().cpu().numpy(), kd, vd, idx.permute(0, 2, 1, 3).reshape(Lq, Hkv, k_sel).cpu().numpy(), win)
     assert_output_close(o8.reshape(-1, 8 * Hkv, D), Oo, torch.bfloat16, "sparse O on the projected FP8 cache")
+    # the same projections written straight into a cache of records [K codes | V codes | K scale | V scale | spare] per
+    # (token, KV head): same codes, same scales, and the sparse kernel reads the records through strides
+    rec = torch.zeros(1, T, Hkv, 272, dtype=torch.uint8, device="cuda")
+    recf = rec.view(torch.float32)
+    wk, wv = w[:Hkv * D], w[Hkv * D:]
+    hs2.hs2_kv_project_fp8_records(h, wk, rec[0, :, :, :D], recf[0, :, :, 64])
+    hs2.hs2_kv_project_fp8_records(h, wv, rec[0, :, :, D:2 * D], recf[0, :, :, 65])
+    torch.cuda.synchronize()
+    assert torch.equal(rec[..., :D], k8) and torch.equal(rec[..., D:2 * D], v8)
+    assert torch.equal(recf[..., 64], ksc) and torch.equal(recf[..., 65], vsc)
+    assert torch.count_nonzero(rec[..., 264:]) == 0
+    o8r, _ = hs2.hs2_sparse_attn_prefill_fp8kv(prob, q, rec[..., :D], rec[..., D:2 * D], recf[..., 64], recf[..., 65], idx)
+    torch.cuda.synchronize()
+    assert torch.equal(o8r, o8)
+    with pytest.raises(hs2.HS2Error):                       # a group stride below the 128 bytes of a group
+        bad = torch.zeros(T, Hkv, 128, dtype=torch.uint8, device="cuda")
+        hs2.hs2_kv_project_fp8_records(h, wk, bad.as_strided((T, Hkv, 128), (Hkv * 128, 64, 1)), recf[0, :, :, 64])
     with pytest.raises(hs2.HS2Error):                       # n_out must be a multiple of 256
         hs2.hs2_kv_project(h, w[:128])
     # more shapes of the CTA-pair kernel: a single tile with one row, ragged token counts across several 256-row tiles,
