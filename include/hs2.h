@@ -180,8 +180,9 @@ hs2_status hs2_sparse_attn_decode_gated(const hs2_problem *p, const void *Q, con
  *   k_scale, v_scale  in  float [batch, kv_len, n_kv_heads]: the cache value is code * scale.  Packed, or with the
  *                strides p->kv_scale_stride gives (floats; shared by the two arrays).  Codes and scales may live in one
  *                buffer of records, e.g. 288 bytes [K codes | V codes | K scale | V scale | spare] per (token, KV head)
- *                at head_dim 128: the documented layout for decode-heavy use, since an attended token then costs one
- *                DRAM page instead of four (see hs2_kv_project_fp8_records, which writes it).
+ *                at head_dim 128 (hs2_kv_project_fp8_records writes that): an attended token then costs a sparse
+ *                layer one DRAM page instead of four (9 % off its decode step at 64K), while the full layer's sweep
+ *                over the whole cache reads the spare bytes too (7 % more).
  *   Q, O, LSE, idx, sink as for the bf16 calls; p->dtype describes Q and O and must be HS2_BF16.
  * Covers head_dim 128 and 256 with up to 128 query heads per KV head (the paper's own shape, 64 heads on one KV
  * head at head_dim 256, included) and 16-byte aligned tensors; anything else returns HS2_ERR_UNSUPPORTED.  At
@@ -266,7 +267,7 @@ hs2_status hs2_kv_project(int64_t n_tokens, int32_t d_model, int32_t n_out, cons
 /*
  * The e4m3 form of hs2_kv_project writing into a cache of records, so that the K codes, the V codes and both scales
  * of a (token, KV head) can sit side by side (one DRAM page per attended token and head instead of four; on the 64K
- * decode step of the benchmark the sparse layer then takes 39.7 us instead of 43.7).  A column group g is the 128
+ * decode step of the benchmark a sparse layer then takes 39.7 us instead of 43.7, the full layer 1.18 ms instead of 1.10).  A column group g is the 128
  * consecutive output columns 128 g .. 128 g + 127 (one head of dim 128):
  *   codes of token t, group g   at byte  t * ldc + g * ld_group  of C   (128 bytes)
  *   their scale                 at       scales[t * scale_ld_token + g * scale_ld_group]
