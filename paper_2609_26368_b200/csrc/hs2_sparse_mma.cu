@@ -897,20 +897,37 @@ cudaError_t launch_sparse_mma_decode(const Params &p, const void *Q, const void 
 }
 
 // ---------------------------------------------------------------- selection scores from the kept raw products
-// a[j] = max over the heads h of the group of (scale * raw[h][j] - LSE_h)   (Section 3.4), one thread per key
+// a[j] = max over the heads h of the group of (scale * raw[h][j] - LSE_h)   (Section 3.4); a thread takes four
+// consecutive keys (one 16-byte load per head, several heads in flight) when the rows allow it, one key otherwise
+template <bool VEC>
 __global__ void __launch_bounds__(256)
 k_scores_from_raw(const Params p, const float *__restrict__ raw, const float *__restrict__ LSE, float *__restrict__ out,
                   int64_t out_stride)
 {
     const int bg = blockIdx.y;
     const int gkv = bg % p.Hkv, b = bg / p.Hkv;
-    const int j = blockIdx.x * 256 + threadIdx.x;
-    if (j >= p.Lk) return;
-    const float *r = raw + (int64_t)bg * p.G * p.Lk + j;
-    float a = -INFINITY;
-    for (int h = 0; h < p.G; ++h)
-        a = fmaxf(a, fmaf(p.scale, r[(int64_t)h * p.Lk], -LSE[(int64_t)b * p.Hq + gkv * p.G + h]));   // Lq == 1
-    out[(int64_t)bg * out_stride + j] = a;
+    const float *lse = LSE + (int64_t)b * p.Hq + gkv * p.G;   // Lq == 1
+    if (VEC) {
+        const int j = (blockIdx.x * 256 + threadIdx.x) * 4;
+        if (j >= p.Lk) return;
+        const float *r = raw + (int64_t)bg * p.G * p.Lk + j;
+        float4 a = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
+#pragma unroll 4
+        for (int h = 0; h < p.G; ++h) {
+            const float4 v = __ldcs(reinterpret_cast<const float4 *>(r + (int64_t)h * p.Lk));
+            const float nl = -lse[h];
+            a.x = fmaxf(a.x, fmaf(p.scale, v.x, nl)); a.y = fmaxf(a.y, fmaf(p.scale, v.y, nl));
+            a.z = fmaxf(a.z, fmaf(p.scale, v.z, nl)); a.w = fmaxf(a.w, fmaf(p.scale, v.w, nl));
+        }
+        *reinterpret_cast<float4 *>(out + (int64_t)bg * out_stride + j) = a;
+    } else {
+        const int j = blockIdx.x * 256 + threadIdx.x;
+        if (j >= p.Lk) return;
+        const float *r = raw + (int64_t)bg * p.G * p.Lk + j;
+        float a = -INFINITY;
+        for (int h = 0; h < p.G; ++h) a = fmaxf(a, fmaf(p.scale, r[(int64_t)h * p.Lk], -lse[h]));
+        out[(int64_t)bg * out_stride + j] = a;
+    }
 }
 
 cudaError_t launch_scores_from_raw(const Params &p, const float *raw, const float *LSE, float *out, int64_t out_stride,
@@ -918,8 +935,15 @@ cudaError_t launch_scores_from_raw(const Params &p, const float *raw, const floa
 {
     const int bg = p.B * p.Hkv;
     if (bg <= 0 || bg > 65535 || p.Lq != 1) return cudaErrorNotSupported;
-    dim3 grid((unsigned)((p.Lk + 255) / 256), (unsigned)bg);
-    k_scores_from_raw<<<grid, 256, 0, st>>>(p, raw, LSE, out, out_stride);
+    const bool vec = p.Lk % 4 == 0 && out_stride % 4 == 0 && (reinterpret_cast<uintptr_t>(raw) & 15u) == 0 &&
+                     (reinterpret_cast<uintptr_t>(out) & 15u) == 0;
+    if (vec) {
+        dim3 grid((unsigned)((p.Lk / 4 + 255) / 256), (unsigned)bg);
+        k_scores_from_raw<true><<<grid, 256, 0, st>>>(p, raw, LSE, out, out_stride);
+    } else {
+        dim3 grid((unsigned)((p.Lk + 255) / 256), (unsigned)bg);
+        k_scores_from_raw<false><<<grid, 256, 0, st>>>(p, raw, LSE, out, out_stride);
+    }
     count_launch();
     return cudaGetLastError();
 }
