@@ -267,7 +267,7 @@ hs2_status hs2_kv_project(int64_t n_tokens, int32_t d_model, int32_t n_out, cons
 /*
  * The e4m3 form of hs2_kv_project writing into a cache of records, so that the K codes, the V codes and both scales
  * of a (token, KV head) can sit side by side (one DRAM page per attended token and head instead of four; on the 64K
- * decode step of the benchmark a sparse layer then takes 39.7 us instead of 43.7, the full layer 1.18 ms instead of 1.10).  A column group g is the 128
+ * decode step of the benchmark a sparse layer then takes 39.7 us instead of 43.7, the full layer 1.13 ms instead of 1.04).  A column group g is the 128
  * consecutive output columns 128 g .. 128 g + 127 (one head of dim 128):
  *   codes of token t, group g   at byte  t * ldc + g * ld_group  of C   (128 bytes)
  *   their scale                 at       scales[t * scale_ld_token + g * scale_ld_group]
