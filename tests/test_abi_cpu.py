@@ -92,6 +92,25 @@ def test_unsupported_and_null_and_workspace_errors(lib):
         binding.HS2_ERR_INVALID_ARG
 
 
+def test_fp8_record_layout_argument_checks(lib):
+    one = C.c_void_p(256)
+    c = _prob(head_dim=128, dtype=torch.bfloat16).c_struct()
+    c.kv_scale_stride = (C.c_int64 * 3)(64 * 72, 72, 0)              # scales of two heads on top of each other
+    assert lib.hs2_sparse_attn_prefill_fp8kv(C.byref(c), one, one, one, one, one, one, None, one, None, None) == \
+        binding.HS2_ERR_INVALID_ARG
+    c.kv_scale_stride = (C.c_int64 * 3)(-1, 72, 72)
+    assert lib.hs2_sparse_attn_prefill_fp8kv(C.byref(c), one, one, one, one, one, one, None, one, None, None) == \
+        binding.HS2_ERR_INVALID_ARG
+    # the producer: a group stride below a group's 128 bytes, a missing scale pointer, rows that cannot hold their groups
+    assert lib.hs2_kv_project_fp8_records(256, 64, 256, one, 64, one, 64, one, 576, 64, one, 144, 72, None) == \
+        binding.HS2_ERR_INVALID_ARG
+    assert lib.hs2_kv_project_fp8_records(256, 64, 256, one, 64, one, 64, one, 576, 288, None, 144, 72, None) == \
+        binding.HS2_ERR_INVALID_ARG
+    assert lib.hs2_kv_project_fp8_records(256, 64, 256, one, 64, one, 64, one, 288, 288, one, 144, 72, None) == \
+        binding.HS2_ERR_UNSUPPORTED
+    assert lib.hs2_kv_project_fp8_records(0, 64, 256, one, 64, one, 64, one, 576, 288, one, 144, 72, None) == binding.HS2_OK
+
+
 def test_gather_probe_argument_checks(lib):
     one = C.c_void_p(256)
     bf = _prob(head_dim=128, dtype=torch.bfloat16).c_struct()
