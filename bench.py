@@ -795,6 +795,54 @@ def side_block(name, device, rank, peaks, world, steps=5):
     return out
 
 
+def bench_variants(device, peaks):
+    """The sparse layer on an e4m3 cache and the block-level selection of the paper's first ablation (Section 5), both at
+    cfg2's shape: measured numbers for the two variants that the block step itself does not run."""
+    import paper_2609_26368_b200 as hs2
+    from paper_2609_26368_b200 import binding
+    from gen.workloads import quantize_kv_e4m3
+    wl = CONFIGS["cfg2"]
+    inp = make_inputs(wl, device)
+    q, k, v = inp.q_full, inp.k, inp.v
+    prob = hs2.Problem.from_tensors(q, k, wl.k_sel, wl.window)
+    ws = torch.empty(max(256, hs2.hs2_workspace_bytes(prob, binding.HS2_OP_FULL_ATTN_SELECT)), dtype=torch.uint8, device=device)
+    _, _, idx, _ = hs2.hs2_full_attn_select(prob, q, k, v, ws=ws)
+
+    def med(fn, n=10, warm=3):
+        for _ in range(warm):
+            fn()
+        ts = []
+        for _ in range(n):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            fn()
+            b.record()
+            torch.cuda.synchronize()
+            ts.append(a.elapsed_time(b))
+        return statistics.median(ts)
+    out = torch.empty_like(q)
+    t_tok = med(lambda: hs2.hs2_full_attn_select(prob, q, k, v, ws=ws))
+    t_bf = med(lambda: hs2.hs2_sparse_attn_prefill(prob, inp.q_sparse[0], k, v, idx, out=out))
+    k8, ksc = quantize_kv_e4m3(k)
+    v8, vsc = quantize_kv_e4m3(v)
+    t_f8 = med(lambda: hs2.hs2_sparse_attn_prefill_fp8kv(prob, inp.q_sparse[0], k8, v8, ksc, vsc, idx, out=out))
+    pb = hs2.Problem.from_tensors(q, k, wl.k_sel, wl.window, select_block=64)
+    wsb = torch.empty(max(256, hs2.hs2_workspace_bytes(pb, binding.HS2_OP_FULL_ATTN_SELECT)), dtype=torch.uint8, device=device)
+    _, _, idxb, _ = hs2.hs2_full_attn_select(pb, q, k, v, ws=wsb)
+    t_blk = med(lambda: hs2.hs2_full_attn_select(pb, q, k, v, ws=wsb))
+    t_sp_blk = med(lambda: hs2.hs2_sparse_attn_prefill(prob, inp.q_sparse[0], k, v, idxb, out=out))
+    gb = gathered_kv_bytes(wl)
+    return {"workload": workload_config(wl, 1)["workload"],
+            "fp8_kv_cache": {"sparse_prefill_ms": round(t_f8, 4), "bf16_cache_ms": round(t_bf, 4),
+                             "gathered_kv_bytes": gb / 512.0 * 264.0,
+                             "note": "the cache is L2 resident at this size: the e4m3 rows halve the copies and the shared memory per warp"},
+            "block_level_selection": {"block": 64, "full_attn_select_ms": round(t_blk, 4), "token_level_ms": round(t_tok, 4),
+                                      "sparse_prefill_on_block_indices_ms": round(t_sp_blk, 4),
+                                      "sparse_prefill_on_token_indices_ms": round(t_bf, 4),
+                                      "note": "Section 5, Ablation 1: 16 blocks of 64 tokens against 1024 tokens; the sparse kernel is the same, "
+                                              "block indices gather contiguous runs of rows"}}
+
+
 # ------------------------------------------------------------------ main
 
 def main():
@@ -806,7 +854,7 @@ def main():
     ap.add_argument("--workload", default="cfg4", choices=sorted(CONFIGS))
     ap.add_argument("--cpu-rows", type=int, default=0,
                     help="query rows of the CPU-oracle sample (0: as many as about 3.5e11 oracle flops, 10-20 s)")
-    ap.add_argument("--skip", default="", help="comma list of: block, small, decode64k, native, kvproj, e2e, cpu")
+    ap.add_argument("--skip", default="", help="comma list of: block, small, decode64k, native, kvproj, variants, e2e, cpu")
     ap.add_argument("--decode-ctx", type=int, default=65536, help="context length of the decode section (profiling: 8192)")
     ap.add_argument("--decode-batch", type=int, default=0, help="profiling captures only: batch of the decode section (default 64)")
     ap.add_argument("--profile-len", type=int, default=0,
@@ -845,6 +893,8 @@ def main():
             side["paper_native_shape"] = bench_native(device, peaks)
         if "kvproj" not in skip:
             side["kv_project"] = bench_kv_project(device, peaks)
+        if "variants" not in skip:
+            side["variants_cfg2"] = bench_variants(device, peaks)
         print(json.dumps(side))
         return
     block = Block(wl, device, rank)
@@ -908,6 +958,9 @@ def main():
     if "kvproj" not in skip and world == 1:
         torch.cuda.empty_cache()
         line["kv_project"] = bench_kv_project(device, peaks)
+    if "variants" not in skip and world == 1:
+        torch.cuda.empty_cache()
+        line["variants_cfg2"] = bench_variants(device, peaks)
     if "cpu" not in skip and world == 1:
         torch.cuda.empty_cache()
         n = args.cpu_rows if args.cpu_rows > 0 else rows_for_flops(wl, 3.5e11)
