@@ -1561,7 +1561,7 @@ k_sample_tau(const Params p, const float *__restrict__ sample, int64_t stride, i
 // Rows whose list is unusable (a sub-list overflowed or was abandoned, fewer candidates than wanted) are flagged for
 // the exact redo.
 template <int THREADS, int E>
-__global__ void __launch_bounds__(THREADS, THREADS > 256 ? 1 : (E > 16 ? 3 : 4))
+__global__ void __launch_bounds__(THREADS, THREADS > 256 ? 1 : (E > 16 ? 3 : 1024 / THREADS))
 k_cand_select(const Params p, const int2 *__restrict__ cand, const int *__restrict__ count,
               int cap, int32_t *__restrict__ idx, int64_t row0, int *__restrict__ flag)
 {
@@ -1750,7 +1750,8 @@ cudaError_t launch_filter_select(const Params &p, const void *cand, const int *c
     };
     // a thread group of THREADS / 4 takes one sub-list of cap / 4 slots, E slots per thread
     cudaError_t e;
-    if (cap <= 4096) e = go(k_cand_select<256, 16>, 256, 16);
+    if (cap <= 2048) e = go(k_cand_select<128, 16>, 128, 16);
+    else if (cap <= 4096) e = go(k_cand_select<256, 16>, 256, 16);
     else if (cap <= 8192) e = go(k_cand_select<256, 32>, 256, 32);
     else e = go(k_cand_select<512, 64>, 512, 64);
     if (e != cudaSuccess) return e;
