@@ -566,6 +566,32 @@ def bench_native(device, peaks, reps=5):
     del inp, q, k, v, O, LSE, idx, osp, ws, k8, v8, ksc, vsc
     torch.cuda.empty_cache()
 
+    # the same shape at a context of 32K: the full layer (attention + a score sweep of half its flops + top-k) dwarfs the
+    # sparse layers, which is the cost structure the hybrid block is built on (Section 3.4)
+    from dataclasses import replace
+    wl = replace(NATIVE["native8k"], q_len=32768, kv_len=32768, name="native32k")
+    inp = make_inputs(wl, device)
+    q, k, v = inp.q_full, inp.k, inp.v
+    prob = hs2.Problem.from_tensors(q, k, wl.k_sel, wl.window)
+    ws = torch.empty(max(256, hs2.hs2_workspace_bytes(prob, binding.HS2_OP_FULL_ATTN_SELECT)), dtype=torch.uint8, device=device)
+    O, LSE, idx, _ = hs2.hs2_full_attn_select(prob, q, k, v, ws=ws)
+    t_full = med(lambda: hs2.hs2_full_attn_select(prob, q, k, v, out=O, lse=LSE, idx=idx, ws=ws), n=3, warm=1)
+    t_att = med(lambda: hs2.hs2_full_attn_select(prob, q, k, v, out=O, lse=LSE, want_idx=False, ws=ws), n=3, warm=1)
+    osp = torch.empty_like(q)
+    t_sp = med(lambda: hs2.hs2_sparse_attn_prefill(prob, inp.q_sparse[0], k, v, idx, out=osp), n=3, warm=1)
+    gb = gathered_kv_bytes(wl)
+    fl = full_attn_flops(wl)
+    out["prefill_32k"] = {
+        "workload": "native32k: B=1, L=32768, 64q/1kv heads, D=256, bf16, k=1024, w=128",
+        "full_attn_select_ms": round(t_full, 2), "attention_only_ms": round(t_att, 2),
+        "attention_tflops": round(fl / (t_att * 1e-3) / 1e12, 1),
+        "attention_frac_of_bf16_peak": round(fl / (t_att * 1e-3) / 1e12 / tensor_peak_for(t_att, peaks)[0], 4),
+        "attention_peak_kind": tensor_peak_for(t_att, peaks)[1],
+        "sparse_prefill_ms": round(t_sp, 2), "gathered_kv_bytes": gb,
+        "sparse_prefill_frac_of_hbm_peak": round(gb / (t_sp * 1e-3) / 1e9 / peaks["hbm_gbs"], 4)}
+    del inp, q, k, v, O, LSE, idx, osp, ws
+    torch.cuda.empty_cache()
+
     wl = NATIVE["native_decode"]
     inp = make_inputs(wl, device)
     k, v = inp.k, inp.v
