@@ -30,8 +30,9 @@ def _index_properties(run, stride=1):
     assert bool(inc.all())                                         # strictly ascending => unique
 
 
-def _run_block(name, n_rows, layers=None):
-    wl = CONFIGS[name] if name in CONFIGS else NATIVE[name]
+def _run_block(name, n_rows, layers=None, wl=None):
+    if wl is None:
+        wl = CONFIGS[name] if name in CONFIGS else NATIVE[name]
     inp = make_inputs(wl, "cuda")
     run = BlockRun(inp).run_full()
     rows = [(b, i) for b in range(wl.batch) for i in sample_rows(wl, n_rows)]
@@ -70,3 +71,11 @@ def test_native8k_full_size_sampled():
 def test_native_decode_full_size_every_sequence():
     """Decode at the paper's shape, batch 64 on a 64K-token cache: the splits of a sequence merge inside a cluster."""
     _run_block("native_decode", 1, layers=[0])
+
+
+def test_native_shape_at_a_32k_context_sampled():
+    """The paper's shape at the longer context bench.py also times: score strips of 32768 keys, rows for the cluster
+    top-k's smaller sibling, 32768 work items of the tensor-core gather kernel."""
+    import dataclasses
+    wl = dataclasses.replace(NATIVE["native8k"], q_len=32768, kv_len=32768, name="native32k")
+    _run_block("native32k", 16, layers=[0], wl=wl)
