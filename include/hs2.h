@@ -16,7 +16,8 @@
  *   ..._gated                the two SA calls with the sigmoid output gate of the sparse layers fused in.
  *   ..._fp8kv                the two SA calls on an e4m3 KV cache with per-token scales.
  *   hs2_kv_project           the producer of those caches: the K/V projection of KV Bridging (Section 3.2),
- *                            bf16 or quantised to the e4m3 cache format in its epilogue.
+ *                            bf16 or quantised to the e4m3 cache format in its epilogue
+ *                            (hs2_kv_project_fp8_records: codes and scales into one record per token and KV head).
  *
  * Conventions
  *   - Every tensor pointer is a DEVICE pointer owned by the caller; `hs2_problem` itself is a
