@@ -825,6 +825,73 @@ def test_ragged_lengths_offsets_strides_and_sink():
         assert np.abs(l[fin] - LSEs[fin]).max() <= TOL[dt]["lse"]
 
 
+def test_seeded_random_problems_against_the_oracle():
+    """Forty problems drawn from a fixed seed: head dims, group sizes, lengths, budgets, causal offsets and cache
+    lengths at random, so that shapes nobody thought of reach every kernel family (SIMT, mma.sync, tcgen05; strips and
+    the filtered selection, which is forced on every other case).  Every row of the full layer, the sparse layer and
+    the decode step is held against the oracle."""
+    import random
+    rnd = random.Random(260926368)
+    old = hs2.hs2_set_filter_min_keys(0)
+    try:
+        for case in range(40):
+            D = rnd.choice([64, 128, 128, 128, 256])
+            Hkv = rnd.choice([1, 2, 4])
+            G = rnd.choice([1, 2, 4, 8, 8, 16]) if D != 256 else rnd.choice([2, 8, 32])
+            B = rnd.choice([1, 2, 3])
+            Lq = rnd.randint(1, 160)
+            Lk = Lq + rnd.randint(0, 500)
+            k = rnd.choice([0, 1, 7, 32, 100, 128])
+            w = rnd.choice([0, 1, 5, 16, 64]) if k > 0 else rnd.choice([1, 5, 16, 64])
+            dtype = "f32" if (D == 64 or rnd.random() < 0.15) else "bf16"
+            wl = scaled("cfg2", batch=B, q_len=Lq, kv_len=Lk, n_q_heads=G * Hkv, n_kv_heads=Hkv, head_dim=D, dtype=dtype,
+                        k_sel=k, window=w, n_needles=min(4, max(1, Lk // 8)), seed=1000 + case)
+            inp = make_inputs(wl)
+            kv_lens = [rnd.randint(max(1, Lk // 3), Lk) for _ in range(B)]
+            q_start = [rnd.randint(-2, max(0, kv_lens[b] - Lq)) for b in range(B)]
+            if rnd.random() < 0.3:
+                q_start = [kv_lens[b] - Lq for b in range(B)]            # the default alignment, some of it negative
+            qs_t = torch.tensor(q_start, dtype=torch.int32, device="cuda")
+            kl_t = torch.tensor(kv_lens, dtype=torch.int32, device="cuda")
+            scale = rnd.choice([0.0, 0.0, 0.07, 0.2])
+            q, kk, v = inp.q_full.cuda(), inp.k.cuda(), inp.v.cuda()
+            hs2.hs2_set_filter_min_keys(1 if case % 2 else 1 << 30)
+            prob = hs2.Problem.from_tensors(q, kk, k, w, softmax_scale=scale, q_start=qs_t, kv_lens=kl_t)
+            what = "case %d: D=%d G=%d Hkv=%d B=%d Lq=%d Lk=%d k=%d w=%d %s q_start=%s kv_lens=%s" % (
+                case, D, G, Hkv, B, Lq, Lk, k, w, dtype, q_start, kv_lens)
+            O, LSE, idx, _ = hs2.hs2_full_attn_select(prob, q, kk, v, want_idx=k > 0)
+            torch.cuda.synchronize()
+            okw = dict(scale=scale if scale > 0 else None, q_start=q_start, kv_lens=kv_lens)
+            Oo, LSEo, idxo, sco = oracle.full_attn_select(inp.q_full, inp.k, inp.v, k, w, want_idx=k > 0, want_scores=k > 0, **okw)
+            dt = wl.torch_dtype
+            Hq = G * Hkv
+            assert_output_close(O.reshape(-1, Hq, D), Oo, dt, what + ": full O")
+            l = LSE.permute(0, 2, 1).reshape(B * Lq, Hq).cpu().numpy()
+            fin = np.isfinite(LSEo)
+            assert np.array_equal(np.isfinite(l), fin), what
+            assert not fin.any() or np.abs(l[fin] - LSEo[fin]).max() <= TOL[dt]["lse"], what
+            if k > 0:
+                idx_rows = idx.permute(0, 2, 1, 3).reshape(B * Lq, Hkv, k).cpu().numpy()
+                check_idx_against_oracle(idx_rows, idxo, sco)
+            else:
+                idx_rows = np.zeros((B * Lq, Hkv, 0), dtype=np.int32)
+            qsp = inp.q_sparse[0].cuda()
+            out, lse = hs2.hs2_sparse_attn_prefill(prob, qsp, kk, v, idx if k > 0 else None, want_lse=True)
+            torch.cuda.synchronize()
+            Os, LSEs, _ = oracle.sparse_attn(inp.q_sparse[0], inp.k, inp.v, idx_rows, w, **okw)
+            assert_output_close(out.reshape(-1, Hq, D), Os, dt, what + ": sparse O")
+            q1 = qsp[:, -1:].contiguous()
+            qs1 = torch.tensor([q_start[b] + Lq - 1 for b in range(B)], dtype=torch.int32, device="cuda")
+            prob1 = hs2.Problem.from_tensors(q1, kk, k, w, softmax_scale=scale, q_start=qs1, kv_lens=kl_t)
+            od, _ = hs2.hs2_sparse_attn_decode(prob1, q1, kk, v, idx[:, :, -1:].contiguous() if k > 0 else None)
+            torch.cuda.synchronize()
+            last = [b * Lq + Lq - 1 for b in range(B)]
+            assert_output_close(od[:, 0], Os[last], dt, what + ": decode O")
+            assert hs2.hs2_device_error_flags() == 0, what
+    finally:
+        hs2.hs2_set_filter_min_keys(old)
+
+
 def test_malformed_indices_cannot_read_out_of_bounds():
     wl = scaled("cfg2", q_len=64, kv_len=64, k_sel=32, window=8, n_needles=4)
     inp = make_inputs(wl)
