@@ -892,6 +892,57 @@ def test_seeded_random_problems_against_the_oracle():
         hs2.hs2_set_filter_min_keys(old)
 
 
+def test_seeded_random_medium_problems_on_the_tensor_core_kernels():
+    """Eight larger draws at head_dim 128 and 256 in bf16 (several query and key tiles, ragged tails, offsets, cache
+    lengths), the filtered selection forced on every other one; every seventh row against the oracle."""
+    import random
+    rnd = random.Random(26368)
+    old = hs2.hs2_set_filter_min_keys(0)
+    try:
+        for case in range(8):
+            D = rnd.choice([128, 128, 128, 256])
+            Hkv = rnd.choice([1, 2])
+            G = rnd.choice([4, 8, 16]) if D == 128 else rnd.choice([8, 64])
+            B = rnd.choice([1, 2])
+            Lq = rnd.randint(300, 900)
+            Lk = Lq + rnd.randint(0, 4000)
+            k = rnd.choice([64, 200, 512])
+            w = rnd.choice([0, 8, 100])
+            wl = scaled("cfg2", batch=B, q_len=Lq, kv_len=Lk, n_q_heads=G * Hkv, n_kv_heads=Hkv, head_dim=D, k_sel=k,
+                        window=w, n_needles=8, seed=2000 + case)
+            inp = make_inputs(wl)
+            kv_lens = [rnd.randint(Lk // 2, Lk) for _ in range(B)]
+            q_start = [rnd.randint(0, max(0, kv_lens[b] - Lq)) for b in range(B)]
+            qs_t = torch.tensor(q_start, dtype=torch.int32, device="cuda")
+            kl_t = torch.tensor(kv_lens, dtype=torch.int32, device="cuda")
+            q, kk, v = inp.q_full.cuda(), inp.k.cuda(), inp.v.cuda()
+            hs2.hs2_set_filter_min_keys(1 if case % 2 else 1 << 30)
+            prob = hs2.Problem.from_tensors(q, kk, k, w, q_start=qs_t, kv_lens=kl_t)
+            what = "case %d: D=%d G=%d Hkv=%d B=%d Lq=%d Lk=%d k=%d w=%d q_start=%s kv_lens=%s" % (
+                case, D, G, Hkv, B, Lq, Lk, k, w, q_start, kv_lens)
+            O, LSE, idx, _ = hs2.hs2_full_attn_select(prob, q, kk, v)
+            torch.cuda.synchronize()
+            rows = [(b, i) for b in range(B) for i in sorted(set(range(0, Lq, 7)) | {Lq - 1})]
+            okw = dict(q_start=q_start, kv_lens=kv_lens, rows=rows)
+            Oo, LSEo, idxo, sco = oracle.full_attn_select(inp.q_full, inp.k, inp.v, k, w, want_scores=True, **okw)
+            dt = wl.torch_dtype
+            assert_output_close(gather_rows(O, rows, "bihd"), Oo, dt, what + ": full O")
+            l = gather_rows(LSE, rows, "bhi").cpu().numpy()
+            fin = np.isfinite(LSEo)
+            assert np.array_equal(np.isfinite(l), fin), what
+            assert np.abs(l[fin] - LSEo[fin]).max() <= TOL[dt]["lse"], what
+            idx_rows = gather_rows(idx, rows, "bgik").cpu().numpy()
+            check_idx_against_oracle(idx_rows, idxo, sco)
+            qsp = inp.q_sparse[0].cuda()
+            out, _ = hs2.hs2_sparse_attn_prefill(prob, qsp, kk, v, idx)
+            torch.cuda.synchronize()
+            Os, _, _ = oracle.sparse_attn(inp.q_sparse[0], inp.k, inp.v, idx_rows, w, **okw)
+            assert_output_close(gather_rows(out, rows, "bihd"), Os, dt, what + ": sparse O")
+            assert hs2.hs2_device_error_flags() == 0, what
+    finally:
+        hs2.hs2_set_filter_min_keys(old)
+
+
 def test_malformed_indices_cannot_read_out_of_bounds():
     wl = scaled("cfg2", q_len=64, kv_len=64, k_sel=32, window=8, n_needles=4)
     inp = make_inputs(wl)
