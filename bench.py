@@ -858,7 +858,21 @@ def bench_variants(device, peaks):
     t_blk = med(lambda: hs2.hs2_full_attn_select(pb, q, k, v, ws=wsb))
     t_sp_blk = med(lambda: hs2.hs2_sparse_attn_prefill(prob, inp.q_sparse[0], k, v, idxb, out=out))
     gb = gathered_kv_bytes(wl)
+    # hs2_topk_select on a materialised score tensor [B, Hkv, Lq, Lk] fp32 (the debug scores of the full layer): the
+    # kernel reads each row's candidates (keys 0 .. pos - w) once
+    del k8, v8, ksc, vsc
+    _, _, _, sc = hs2.hs2_full_attn_select(prob, q, k, v, want_scores=True)
+    idx2 = torch.empty_like(idx)
+    t_topk = med(lambda: hs2.hs2_topk_select(prob, sc, idx=idx2))
+    cand_bytes = 4.0 * wl.batch * wl.n_kv_heads * sum(max(0, i - wl.window + 1) for i in range(wl.kv_len - wl.q_len, wl.kv_len))
+    same = bool(torch.equal(idx2, idx))
+    del sc
     return {"workload": workload_config(wl, 1)["workload"],
+            "topk_select": {"ms": round(t_topk, 4), "candidate_bytes": cand_bytes,
+                            "achieved_gbs": round(cand_bytes / (t_topk * 1e-3) / 1e9, 1),
+                            "frac_of_hbm_peak": round(cand_bytes / (t_topk * 1e-3) / 1e9 / peaks["hbm_gbs"], 4),
+                            "same_indices_as_full_layer": same,
+                            "note": "fp32 scores read once; instruction-bound (about 50 instructions per candidate), not bandwidth-bound"},
             "fp8_kv_cache": {"sparse_prefill_ms": round(t_f8, 4), "bf16_cache_ms": round(t_bf, 4),
                              "gathered_kv_bytes": gb / 512.0 * 264.0,
                              "note": "the cache is L2 resident at this size: the e4m3 rows halve the copies and the shared memory per warp"},
