@@ -226,6 +226,7 @@ class Block:
         """Duration of the bare row gather of one sparse layer (hs2_probe_gather: the same rows in the same order,
         nothing else), best of the two load modes, median of `reps` after one warm-up each.  Needs self.idx."""
         best = None
+        self.probe_ms_by_mode = {}
         word = torch.zeros(1, dtype=torch.int32, device=self.dev)
         for mode in (0, 1):
             self.hs2.hs2_probe_gather(self.prob, self.k, self.v, self.idx, mode=mode, sink_word=word)
@@ -238,6 +239,7 @@ class Block:
                 torch.cuda.synchronize()
                 ts.append(a.elapsed_time(b))
             t = statistics.median(ts)
+            self.probe_ms_by_mode[mode] = t
             if best is None or t < best[0]:
                 best = (t, mode)
         return best
@@ -786,13 +788,17 @@ def sparse_roofline(wl, block, sp_ms, peaks):
             "tokens_per_s": round(tokens / (sp_ms * 1e-3), 1),
             "l2_gather_ceiling": {"ms": round(probe_ms, 4), "gbs": round(gb / (probe_ms * 1e-3) / 1e9, 1),
                                   "loads": "past L1" if probe_mode == 0 else "through L1",
+                                  "ms_past_l1": round(block.probe_ms_by_mode[0], 4),
+                                  "ms_through_l1": round(block.probe_ms_by_mode[1], 4),
+                                  "frac_of_the_gather_past_l1": round(block.probe_ms_by_mode[0] / sp_ms, 4),
                                   "how": "hs2_probe_gather on the same K, V and idx: every attended row fetched in the "
                                          "attention kernel's item order, no arithmetic, full occupancy"},
             "frac_l2": round(probe_ms / sp_ms, 4),
             "binding_limit": dict(limits, frac=round(limit / sp_ms, 4), tensor_peak=which),
             "note": "achieved counts gathered K/V rows (512 B per attended token per KV head); one KV head's cache is "
                     "L2 resident in prefill, so frac (of the HBM peak) exceeds 1 and is no measure of distance to a "
-                    "limit; frac_l2 is"}
+                    "limit; frac_l2 is (against the faster of the probe's two load modes; the attention kernel itself "
+                    "copies past L1, whose capacity its shared memory takes)"}
 
 
 def full_layer_summary(wl, fa_ms, peaks):
